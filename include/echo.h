@@ -1,0 +1,214 @@
+/*
+ * echo.h — C ABI of the B200 rollout-generation library.
+ *
+ * The library implements the step that a rollout worker of the ECHO-2 paper
+ * (arXiv 2602.02192) spends its time in: for each prompt x, sample G responses
+ * y ~ pi_v(. | x) from the installed policy snapshot v, record the sampler's
+ * per-token log-probabilities, and tag every trajectory with v (Section 4.2
+ * "Rollout generation"; Algorithm 1, rollout plane).  A newer snapshot can be
+ * installed while generation continues on the previous one (Section 4.3: a
+ * worker switches its local version only once installation is complete), and
+ * rewards are normalised per group for GRPO (Appendix F, group-wise
+ * normalisation).
+ *
+ * Conventions
+ *   - Every call returns an int: ECHO_OK (0) or a negative ECHO_ERR_* code.
+ *     Nothing throws, aborts or exits.  A failed call leaves the context usable.
+ *   - "dev" pointers are CUDA device pointers on the context's device; "host"
+ *     pointers are ordinary host memory unless stated otherwise.
+ *   - All matrices are row-major.  Weight matrices are bf16, shape [out, in].
+ *   - The caller owns every buffer it passes, including the arena and the CUDA
+ *     stream.  The library never calls cudaMalloc/cudaFree after echo_create
+ *     (echo_create itself allocates only streams and events, no device memory).
+ *   - Work is enqueued on the stream given to echo_create.  Device outputs are
+ *     valid once that stream (or echo_sync) has been synchronised.
+ *   - One context serves one GPU and is not thread-safe; use one context per
+ *     thread or serialise calls.
+ */
+#ifndef ECHO_B200_H
+#define ECHO_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- error codes -------------------------------------------------------- */
+#define ECHO_OK                 0
+#define ECHO_ERR_INVALID       -1   /* null pointer, size out of the configured range, T <= 0, ... */
+#define ECHO_ERR_ARENA         -2   /* arena too small or misaligned                                */
+#define ECHO_ERR_NO_POLICY     -3   /* rollout requested before any echo_load_policy                */
+#define ECHO_ERR_VERSION       -4   /* version not strictly greater than every earlier one          */
+#define ECHO_ERR_BUSY          -5   /* an install is still pending: a third live version would
+                                       exceed what the weight buffers can hold                      */
+#define ECHO_ERR_CUDA          -6   /* a CUDA call failed; text in echo_last_error                  */
+#define ECHO_ERR_DEVICE_CHECK  -7   /* a kernel's own range check tripped (status word set)         */
+#define ECHO_ERR_TIMEOUT       -8   /* a bounded device-side wait ran out                           */
+#define ECHO_ERR_UNSUPPORTED   -9   /* shape the kernels do not cover (e.g. head_dim not 64/128)    */
+
+typedef struct echo_ctx echo_ctx;   /* opaque */
+
+/* Decoder shape and capacity limits, fixed at echo_create. */
+typedef struct echo_config {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
+  float   rms_eps;            /* e.g. 1e-6 */
+  float   rope_theta;         /* e.g. 1e4  */
+  int32_t kv_page_size;       /* tokens per KV page; 16 */
+  int32_t max_prompts;        /* largest P of one echo_rollout call */
+  int32_t max_G;              /* largest group size G               */
+  int32_t max_prompt_len;     /* row width of the prompts array     */
+  int32_t max_new_tokens;     /* largest T                          */
+  int32_t n_weight_buffers;   /* 2: a new snapshot installs while the old one serves
+                                 (staleness bound 1); 1: installs block generation  */
+  int32_t eos_id;             /* must be -1: every sequence produces exactly T tokens */
+} echo_config;
+
+/* One snapshot: a pointer per tensor, bf16, row-major [out, in]; each pointer
+ * is device memory or page-locked host memory.  Per-layer entries are arrays of
+ * n_layers pointers (the arrays themselves live in host memory).
+ *   embed [vocab, d]  lm_head [vocab, d]  final_norm [d]
+ *   wq [Hq*hd, d]  wk [Hkv*hd, d]  wv [Hkv*hd, d]  wo [d, Hq*hd]
+ *   w_gate [F, d]  w_up [F, d]  w_down [d, F]  attn_norm [d]  mlp_norm [d] */
+typedef struct echo_weights {
+  const void *embed, *lm_head, *final_norm;
+  const void *const *wq, *const *wk, *const *wv, *const *wo;
+  const void *const *w_gate, *const *w_up, *const *w_down;
+  const void *const *attn_norm, *const *mlp_norm;
+} echo_weights;
+
+/* Counters of the most recent echo_rollout on this context. */
+typedef struct echo_stats {
+  int64_t version_served;     /* tag of the last rollout                        */
+  int64_t tokens_generated;   /* P*G*T of the last rollout                      */
+  int64_t kernels_launched;   /* this library's kernel launches in that rollout
+                                 (graph replays count the kernels they contain) */
+  int64_t decode_steps;       /* T-1                                            */
+  int64_t n_pages;            /* KV pages the plan used                         */
+  float   install_ms;         /* duration of the last completed install (device) */
+  float   reserved;
+} echo_stats;
+
+/* Bytes of device memory echo_create needs for this configuration (weight
+ * buffers, KV page pool, activations, logits, tables).  0 if cfg is invalid. */
+size_t echo_arena_bytes(const echo_config *cfg);
+
+/* Create a context on CUDA device `device`.  `arena` is device memory of at
+ * least echo_arena_bytes(cfg) bytes, 256-byte aligned, owned by the caller and
+ * kept alive until echo_destroy.  `cuda_stream` is a cudaStream_t (may be 0 for
+ * the legacy default stream, which cannot be graph-captured: decode steps are
+ * then launched kernel by kernel). */
+int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_bytes,
+                void *cuda_stream, echo_ctx **out);
+int echo_destroy(echo_ctx *ctx);
+
+/* Install snapshot `version` (Section 4.2 "Policy publication"; Section 4.3;
+ * Algorithm 1: the worker updates its local version once a newer snapshot is
+ * fully installed).  The copy into the inactive weight buffer is enqueued on the
+ * library's own copy stream, ordered after every rollout that still reads that
+ * buffer, and the call returns at once; generation on the previous version
+ * continues meanwhile.  The source tensors must stay alive and unchanged until
+ * the install has completed (echo_wait_policy, echo_sync, or a later rollout
+ * tagged with this version).  Versions must strictly increase (else
+ * ECHO_ERR_VERSION).  With an install pending a further offer is refused with
+ * ECHO_ERR_BUSY.  With n_weight_buffers == 1 the install overwrites the only
+ * buffer: it is ordered after all enqueued rollouts and the next rollout waits
+ * for it. */
+int echo_load_policy(echo_ctx *ctx, const echo_weights *w, int64_t version);
+
+/* Block the host until a pending install, if any, has completed. */
+int echo_wait_policy(echo_ctx *ctx);
+
+/* Generate G completions of T = max_new_tokens tokens for each of P prompts
+ * (Section 4.2 "Rollout generation": y ~ pi_v(. | x); the rollout multiplicity
+ * and temperature of Section 5.1).
+ *   prompts      dev  int32 [P][cfg.max_prompt_len]   (row p uses its first prompt_lens[p] ids)
+ *   prompt_lens  host int32 [P], each in [1, max_prompt_len]
+ *   temperature  > 0
+ *   seed         keys the Philox4x32-10 streams: key = (seed lo, seed hi),
+ *                counter = (v >> 2, j, s, 0), word v & 3 for vocab id v, new-token
+ *                index j, sequence id s = p*G + g
+ *   out_tokens   dev  int32 [P][G][T]
+ *   out_logprobs dev  fp32  [P][G][T]: log-probability of each token under the
+ *                temperature-scaled distribution it was drawn from (the sampler
+ *                policy of Appendix F's truncated importance ratio)
+ *   out_versions host int64 [P][G]: the snapshot version every token of that
+ *                trajectory was generated under; filled before the call returns.
+ * The version served is the newest whose install had completed when the call
+ * began; an install still running does not affect this rollout.  The prompt is
+ * prefilled once per prompt into KV pages shared by its G samples.  The call
+ * returns after enqueueing; outputs are stream-ordered. */
+int echo_rollout(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens,
+                 int32_t P, int32_t G, int32_t max_new_tokens, float temperature,
+                 uint64_t seed, int32_t *out_tokens, float *out_logprobs,
+                 int64_t *out_versions);
+
+/* Teacher-forced variant: step j feeds forced_tokens[p][g][j] (dev int32
+ * [P][G][T]) instead of the sampled token.  out_tokens[p][g][j] is the token
+ * that would have been sampled at step j, out_logprobs[p][g][j] the
+ * log-probability of the forced token.  Same noise streams as echo_rollout. */
+int echo_rollout_forced(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens,
+                        int32_t P, int32_t G, int32_t max_new_tokens, float temperature,
+                        uint64_t seed, const int32_t *forced_tokens, int32_t *out_tokens,
+                        float *out_logprobs, int64_t *out_versions);
+
+/* echo_rollout with every buffer in HOST memory (prompts, outputs): copies the
+ * prompts in, runs the rollout, copies tokens and log-probabilities out and
+ * synchronises.  Page-locked buffers make the copies asynchronous. */
+int echo_rollout_host(echo_ctx *ctx, const int32_t *prompts_host, const int32_t *prompt_lens,
+                      int32_t P, int32_t G, int32_t max_new_tokens, float temperature,
+                      uint64_t seed, int32_t *out_tokens_host, float *out_logprobs_host,
+                      int64_t *out_versions);
+
+/* GRPO group-wise normalisation (Appendix F): for each of P groups of G rewards,
+ * A = (R - mean) / (std + eps), std with the (G-1) divisor as in the listing
+ * printed under that equation, eps added to the std.  rewards / out_adv: dev
+ * fp32 [P][G] (may alias).  G < 2 is ECHO_ERR_INVALID.  Runs on `cuda_stream`
+ * (a cudaStream_t, may be 0); needs no context. */
+int echo_group_advantage(const float *rewards, int32_t P, int32_t G, float eps,
+                         float *out_adv, void *cuda_stream);
+
+/* Block until everything this context enqueued (rollouts and installs) is done;
+ * reports ECHO_ERR_DEVICE_CHECK / ECHO_ERR_TIMEOUT if a kernel flagged one. */
+int echo_sync(echo_ctx *ctx);
+
+int echo_get_stats(echo_ctx *ctx, echo_stats *out);
+
+/* Copy the page table of the most recent rollout to host memory:
+ * int32 [P*G][width]; entries past a sequence's last page are -1.  `width` and
+ * the number of rows are returned through the pointers; `out` may be NULL to
+ * query them.  n is the capacity of `out` in int32 elements. */
+int echo_debug_page_table(echo_ctx *ctx, int32_t *out, size_t n, int32_t *rows, int32_t *width);
+
+/* ---- stand-alone kernel entry points (used by the parity tests) ---------- */
+
+/* Philox words and uniforms exactly as the sampler draws them: for vocab ids
+ * v in [v0, v0+n), out_words[i] (dev uint32) and out_uniform[i] (dev fp32,
+ * w = (float(word) + 0.5f) * 2^-32) for sequence s, new-token index j. */
+int echo_debug_noise(uint64_t seed, uint32_t s, uint32_t j, uint32_t v0, uint32_t n,
+                     uint32_t *out_words, float *out_uniform, void *cuda_stream);
+
+/* Sampler alone: for r in [0, R): sequence id seq_ids[r] (dev int32, or NULL for
+ * seq id r) draws new-token index j from logits row (r / rows_per_logit_row) of
+ * dev fp32 logits [.][V]; writes out_tokens[r] (dev int32) and out_logprobs[r]
+ * (dev fp32, log-prob of forced[r] if forced != NULL else of the drawn token). */
+int echo_sample(const float *logits, int32_t R, int32_t V, int32_t rows_per_logit_row,
+                const int32_t *seq_ids, uint32_t j, float temperature, uint64_t seed,
+                const int32_t *forced, int32_t *out_tokens, float *out_logprobs,
+                void *cuda_stream);
+
+/* Dense projection alone: Y[M][N] (dev fp32) = X[M][K] (dev bf16) * W[N][K]^T
+ * (dev bf16) with fp32 accumulation on the tcgen05 tensor cores.  K must be a
+ * multiple of 64 and N a multiple of 128; M in [1, 4096].  All pointers 256-byte
+ * aligned.  `impl`: 0 = tensor-core kernel, 1 = plain SIMT reference kernel. */
+int echo_gemm_bf16(const void *X, const void *W, float *Y, int32_t M, int32_t N, int32_t K,
+                   int32_t impl, void *cuda_stream);
+
+const char *echo_strerror(int code);
+const char *echo_last_error(echo_ctx *ctx);   /* text of the last ECHO_ERR_CUDA on this context */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ECHO_B200_H */

@@ -1,0 +1,289 @@
+"""ctypes binding of libecho_b200.so: argument marshalling only.
+
+Every step of the rollout path runs in the library's CUDA kernels; torch is used here
+for device memory and streams.  There is no CPU fallback: if the library is missing the
+import of this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libecho_b200.so")
+
+ECHO_OK = 0
+ERRORS = {
+    -1: "ECHO_ERR_INVALID", -2: "ECHO_ERR_ARENA", -3: "ECHO_ERR_NO_POLICY", -4: "ECHO_ERR_VERSION",
+    -5: "ECHO_ERR_BUSY", -6: "ECHO_ERR_CUDA", -7: "ECHO_ERR_DEVICE_CHECK", -8: "ECHO_ERR_TIMEOUT",
+    -9: "ECHO_ERR_UNSUPPORTED",
+}
+
+
+class EchoError(RuntimeError):
+    def __init__(self, code: int, detail: str = ""):
+        self.code = code
+        super().__init__(f"{ERRORS.get(code, code)} {detail}".strip())
+
+
+class EchoConfig(C.Structure):
+    _fields_ = [
+        ("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("vocab", C.c_int32),
+        ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("kv_page_size", C.c_int32),
+        ("max_prompts", C.c_int32), ("max_G", C.c_int32), ("max_prompt_len", C.c_int32),
+        ("max_new_tokens", C.c_int32), ("n_weight_buffers", C.c_int32), ("eos_id", C.c_int32),
+    ]
+
+
+class EchoWeights(C.Structure):
+    _fields_ = [
+        ("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
+        ("wq", C.POINTER(C.c_void_p)), ("wk", C.POINTER(C.c_void_p)), ("wv", C.POINTER(C.c_void_p)),
+        ("wo", C.POINTER(C.c_void_p)), ("w_gate", C.POINTER(C.c_void_p)), ("w_up", C.POINTER(C.c_void_p)),
+        ("w_down", C.POINTER(C.c_void_p)), ("attn_norm", C.POINTER(C.c_void_p)),
+        ("mlp_norm", C.POINTER(C.c_void_p)),
+    ]
+
+
+class EchoStats(C.Structure):
+    _fields_ = [
+        ("version_served", C.c_int64), ("tokens_generated", C.c_int64), ("kernels_launched", C.c_int64),
+        ("decode_steps", C.c_int64), ("n_pages", C.c_int64), ("install_ms", C.c_float), ("reserved", C.c_float),
+    ]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_02192_b200.build` "
+                          "(there is no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, u32, u64, i64, f32 = C.c_void_p, C.c_int32, C.c_uint32, C.c_uint64, C.c_int64, C.c_float
+    lib.echo_arena_bytes.restype = C.c_size_t
+    lib.echo_arena_bytes.argtypes = [C.POINTER(EchoConfig)]
+    lib.echo_create.argtypes = [C.POINTER(EchoConfig), C.c_int, vp, C.c_size_t, vp, C.POINTER(vp)]
+    lib.echo_destroy.argtypes = [vp]
+    lib.echo_load_policy.argtypes = [vp, C.POINTER(EchoWeights), i64]
+    lib.echo_wait_policy.argtypes = [vp]
+    lib.echo_rollout.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp]
+    lib.echo_rollout_forced.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp, vp]
+    lib.echo_rollout_host.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp]
+    lib.echo_group_advantage.argtypes = [vp, i32, i32, f32, vp, vp]
+    lib.echo_sync.argtypes = [vp]
+    lib.echo_get_stats.argtypes = [vp, C.POINTER(EchoStats)]
+    lib.echo_debug_page_table.argtypes = [vp, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32)]
+    lib.echo_debug_noise.argtypes = [u64, u32, u32, u32, u32, vp, vp, vp]
+    lib.echo_sample.argtypes = [vp, i32, i32, i32, vp, u32, f32, u64, vp, vp, vp, vp]
+    lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.echo_strerror.restype = C.c_char_p
+    lib.echo_strerror.argtypes = [C.c_int]
+    lib.echo_last_error.restype = C.c_char_p
+    lib.echo_last_error.argtypes = [vp]
+    for name in ("echo_create", "echo_destroy", "echo_load_policy", "echo_wait_policy", "echo_rollout",
+                 "echo_rollout_forced", "echo_rollout_host", "echo_group_advantage", "echo_sync",
+                 "echo_get_stats", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16"):
+        getattr(lib, name).restype = C.c_int
+    return lib
+
+
+lib = _load()
+
+EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy", "echo_wait_policy",
+            "echo_rollout", "echo_rollout_forced", "echo_rollout_host", "echo_group_advantage", "echo_sync",
+            "echo_get_stats", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
+            "echo_strerror", "echo_last_error"]
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _check(rc: int, ctx=None):
+    if rc != ECHO_OK:
+        detail = ""
+        if ctx is not None and rc == -6:
+            detail = lib.echo_last_error(ctx).decode()
+        raise EchoError(rc, detail)
+
+
+def make_config(shape, max_prompts: int, max_G: int, max_prompt_len: int, max_new_tokens: int,
+                n_weight_buffers: int = 2, page_size: int = 16) -> EchoConfig:
+    """shape: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab,
+    rms_eps, rope_theta attributes."""
+    return EchoConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                      shape.d_ff, shape.vocab, shape.rms_eps, shape.rope_theta, page_size,
+                      max_prompts, max_G, max_prompt_len, max_new_tokens, n_weight_buffers, -1)
+
+
+def echo_arena_bytes(cfg: EchoConfig) -> int:
+    return int(lib.echo_arena_bytes(C.byref(cfg)))
+
+
+class Engine:
+    """One context on one GPU.  Owns the arena tensor and a dedicated CUDA stream."""
+
+    def __init__(self, cfg: EchoConfig, device: int = 0, stream: Optional[torch.cuda.Stream] = None):
+        self.cfg = cfg
+        self.device = torch.device("cuda", device)
+        nbytes = echo_arena_bytes(cfg)
+        if nbytes == 0:
+            raise EchoError(-1, "configuration rejected")
+        self.arena = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        self.stream = stream if stream is not None else torch.cuda.Stream(device=self.device)
+        self._ctx = C.c_void_p()
+        self._keep = []          # weight tensors of installs that may still be running
+        _check(lib.echo_create(C.byref(cfg), device, self.arena.data_ptr(), nbytes,
+                               int(self.stream.cuda_stream), C.byref(self._ctx)))
+
+    def close(self):
+        if self._ctx:
+            lib.echo_destroy(self._ctx)
+            self._ctx = C.c_void_p()
+            self._keep = []
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- policy ------------------------------------------------------------
+    def echo_load_policy(self, weights: dict, version: int):
+        """weights: name -> bf16 tensor (globals) or list of bf16 tensors (per layer); device or
+        pinned host memory."""
+        L = self.cfg.n_layers
+
+        def arr(name):
+            ts = weights[name]
+            assert len(ts) == L
+            for t in ts:
+                assert t.dtype == torch.bfloat16 and t.is_contiguous()
+            return (C.c_void_p * L)(*[t.data_ptr() for t in ts])
+
+        for n in ("embed", "lm_head", "final_norm"):
+            assert weights[n].dtype == torch.bfloat16 and weights[n].is_contiguous()
+        arrays = {n: arr(n) for n in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "attn_norm", "mlp_norm")}
+        w = EchoWeights(weights["embed"].data_ptr(), weights["lm_head"].data_ptr(),
+                        weights["final_norm"].data_ptr(),
+                        *[C.cast(arrays[n], C.POINTER(C.c_void_p)) for n in
+                          ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "attn_norm", "mlp_norm")])
+        # source tensors written on torch's current stream must be complete before the copy reads them
+        torch.cuda.current_stream(self.device).synchronize()
+        _check(lib.echo_load_policy(self._ctx, C.byref(w), int(version)), self._ctx)
+        self._keep.append(weights)
+        self._keep = self._keep[-2:]
+
+    def echo_wait_policy(self):
+        _check(lib.echo_wait_policy(self._ctx), self._ctx)
+
+    # -- rollouts ------------------------------------------------------------
+    def echo_rollout(self, prompts: torch.Tensor, prompt_lens: Sequence[int], G: int, max_new_tokens: int,
+                     temperature: float, seed: int, forced: Optional[torch.Tensor] = None,
+                     out_tokens: Optional[torch.Tensor] = None, out_logprobs: Optional[torch.Tensor] = None):
+        """prompts: int32 cuda tensor [P][cfg.max_prompt_len].  Returns (tokens int32 [P][G][T],
+        logprobs fp32 [P][G][T] — both on the device, stream-ordered on self.stream — and versions
+        int64 numpy [P][G])."""
+        P = prompts.shape[0]
+        assert prompts.dtype == torch.int32 and prompts.is_cuda and prompts.is_contiguous()
+        assert prompts.shape[1] == self.cfg.max_prompt_len
+        lens = np.ascontiguousarray(np.asarray(prompt_lens, dtype=np.int32))
+        assert lens.shape == (P,)
+        T = max_new_tokens
+        if out_tokens is None:
+            out_tokens = torch.empty((P, G, T), dtype=torch.int32, device=self.device)
+        if out_logprobs is None:
+            out_logprobs = torch.empty((P, G, T), dtype=torch.float32, device=self.device)
+        versions = np.zeros((P, G), dtype=np.int64)
+        # inputs produced on torch's current stream must be visible to the engine's stream
+        self.stream.wait_stream(torch.cuda.current_stream(self.device))
+        if forced is None:
+            rc = lib.echo_rollout(self._ctx, prompts.data_ptr(), lens.ctypes.data, P, G, T, float(temperature),
+                                  int(seed), out_tokens.data_ptr(), out_logprobs.data_ptr(), versions.ctypes.data)
+        else:
+            assert forced.dtype == torch.int32 and forced.is_cuda and forced.is_contiguous()
+            assert tuple(forced.shape) == (P, G, T)
+            rc = lib.echo_rollout_forced(self._ctx, prompts.data_ptr(), lens.ctypes.data, P, G, T,
+                                         float(temperature), int(seed), forced.data_ptr(),
+                                         out_tokens.data_ptr(), out_logprobs.data_ptr(), versions.ctypes.data)
+        _check(rc, self._ctx)
+        return out_tokens, out_logprobs, versions
+
+    def echo_rollout_host(self, prompts: torch.Tensor, prompt_lens: Sequence[int], G: int, max_new_tokens: int,
+                          temperature: float, seed: int, out_tokens: torch.Tensor, out_logprobs: torch.Tensor):
+        """All buffers are host tensors (ideally pinned); returns versions.  Synchronous."""
+        P = prompts.shape[0]
+        assert not prompts.is_cuda and prompts.dtype == torch.int32 and prompts.is_contiguous()
+        assert prompts.shape[1] == self.cfg.max_prompt_len
+        assert not out_tokens.is_cuda and not out_logprobs.is_cuda
+        lens = np.ascontiguousarray(np.asarray(prompt_lens, dtype=np.int32))
+        versions = np.zeros((P, G), dtype=np.int64)
+        _check(lib.echo_rollout_host(self._ctx, prompts.data_ptr(), lens.ctypes.data, P, G, max_new_tokens,
+                                     float(temperature), int(seed), out_tokens.data_ptr(),
+                                     out_logprobs.data_ptr(), versions.ctypes.data), self._ctx)
+        return versions
+
+    def echo_sync(self):
+        _check(lib.echo_sync(self._ctx), self._ctx)
+
+    def echo_get_stats(self) -> dict:
+        st = EchoStats()
+        _check(lib.echo_get_stats(self._ctx, C.byref(st)))
+        return {k: getattr(st, k) for k, _ in EchoStats._fields_ if k != "reserved"}
+
+    def echo_debug_page_table(self) -> np.ndarray:
+        rows, width = C.c_int32(), C.c_int32()
+        _check(lib.echo_debug_page_table(self._ctx, None, 0, C.byref(rows), C.byref(width)))
+        out = np.zeros((rows.value, width.value), dtype=np.int32)
+        if out.size:
+            _check(lib.echo_debug_page_table(self._ctx, out.ctypes.data, out.size, C.byref(rows), C.byref(width)))
+        return out
+
+
+# -- context-free entry points --------------------------------------------------
+def echo_group_advantage(rewards: torch.Tensor, eps: float = 1e-6, out: Optional[torch.Tensor] = None,
+                         stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    assert rewards.is_cuda and rewards.dtype == torch.float32 and rewards.is_contiguous() and rewards.dim() == 2
+    P, G = rewards.shape
+    if out is None:
+        out = torch.empty_like(rewards)
+    with torch.cuda.device(rewards.device):
+        _check(lib.echo_group_advantage(rewards.data_ptr(), P, G, float(eps), out.data_ptr(), _stream_ptr(stream)))
+    return out
+
+
+def echo_debug_noise(seed: int, s: int, j: int, v0: int, n: int, device="cuda"):
+    words = torch.empty(n, dtype=torch.int32, device=device)
+    uni = torch.empty(n, dtype=torch.float32, device=device)
+    with torch.cuda.device(words.device):
+        _check(lib.echo_debug_noise(int(seed), s, j, v0, n, words.data_ptr(), uni.data_ptr(), _stream_ptr(None)))
+    return words, uni
+
+
+def echo_sample(logits: torch.Tensor, rows: int, rows_per_logit_row: int, j: int, temperature: float, seed: int,
+                seq_ids: Optional[torch.Tensor] = None, forced: Optional[torch.Tensor] = None):
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous() and logits.dim() == 2
+    V = logits.shape[1]
+    tok = torch.empty(rows, dtype=torch.int32, device=logits.device)
+    lp = torch.empty(rows, dtype=torch.float32, device=logits.device)
+    with torch.cuda.device(logits.device):
+        _check(lib.echo_sample(logits.data_ptr(), rows, V, rows_per_logit_row,
+                               seq_ids.data_ptr() if seq_ids is not None else None, j, float(temperature),
+                               int(seed), forced.data_ptr() if forced is not None else None,
+                               tok.data_ptr(), lp.data_ptr(), _stream_ptr(None)))
+    return tok, lp
+
+
+def echo_gemm_bf16(X: torch.Tensor, W: torch.Tensor, impl: int = 0) -> torch.Tensor:
+    assert X.is_cuda and W.is_cuda and X.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
+    assert X.is_contiguous() and W.is_contiguous() and X.shape[1] == W.shape[1]
+    M, K = X.shape
+    N = W.shape[0]
+    Y = torch.empty((M, N), dtype=torch.float32, device=X.device)
+    with torch.cuda.device(X.device):
+        _check(lib.echo_gemm_bf16(X.data_ptr(), W.data_ptr(), Y.data_ptr(), M, N, K, impl, _stream_ptr(None)))
+    return Y

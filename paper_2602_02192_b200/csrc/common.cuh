@@ -1,0 +1,94 @@
+// Shared declarations of the rollout library's translation units (sm_100a only).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/echo.h"
+
+namespace echo {
+
+// Status word written by kernels that detect a problem themselves (never trap).
+enum : int {
+  STATUS_OK = 0,
+  STATUS_BAD_PAGE = 1,        // page id / position outside the pool
+  STATUS_BAD_TOKEN = 2,       // token id outside [0, vocab)
+  STATUS_WAIT_TIMEOUT = 3,    // a bounded mbarrier wait ran out
+};
+
+constexpr int kGemmTileN = 128;      // output features per CTA (UMMA M)
+constexpr int kGemmTileK = 64;       // bf16 elements per pipeline stage (one 128-byte swizzle row)
+constexpr int kMaxBatchTile = 256;   // rows of activations per MMA (UMMA N)
+
+// ---- dense projections (gemm.cu) ------------------------------------------
+// Y[m][n] (+)= sum_k X[m][k] * W[n][k], bf16 inputs, fp32 accumulation.
+// tmW: tensor map over W [N][K] with box {64, 128}; tmX over X [M][K] with box {64, bnb}.
+enum GemmEpilogue : int {
+  EPI_STORE = 0,      // Y = acc
+  EPI_ACCUM = 1,      // Y += acc              (residual add)
+  EPI_SWIGLU = 2,     // two W row blocks (gate at n, up at n + N): Yb = bf16(silu(g) * u)
+};
+
+struct GemmArgs {
+  const CUtensorMap *tmW;
+  const CUtensorMap *tmX;
+  void *Y;            // fp32 [M][ldY], or bf16 for EPI_SWIGLU
+  int ldY;
+  int M, N, K;        // N counts output features per accumulator (F for SWIGLU)
+  int bnb;            // activation rows per CTA: 32, 64, 128 or 256
+  int epilogue;
+  int *status;
+};
+cudaError_t gemm_tc_launch(const GemmArgs &a, cudaStream_t stream);
+cudaError_t gemm_tc_configure();     // sets the dynamic shared memory attribute once per device
+cudaError_t gemm_simt_launch(const __nv_bfloat16 *X, const __nv_bfloat16 *W, float *Y, int ldY,
+                             int M, int N, int K, int accumulate, cudaStream_t stream);
+// Tensor map over a row-major bf16 matrix [rows][cols] (leading dimension ld elements),
+// 128-byte swizzle, box {64, box_rows}.
+int make_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
+                    uint32_t box_rows);
+
+// ---- element-wise / row-wise kernels (elementwise.cu) ------------------------
+struct RowMeta {
+  const int32_t *row_pt;     // page-table row of each activation row
+  const int32_t *row_pos;    // absolute position of each activation row
+};
+
+cudaError_t embed_launch(const __nv_bfloat16 *embed, const int32_t *tok_src, const int32_t *tok_idx,
+                         float *x, int R, int d, int vocab, int *status, cudaStream_t s);
+cudaError_t rmsnorm_launch(const float *x, const __nv_bfloat16 *gain, __nv_bfloat16 *h, int R, int d,
+                           float eps, cudaStream_t s);
+cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double theta, cudaStream_t s);
+// qkv fp32 [R][(Hq+2Hkv)*hd] -> q bf16 [R][Hq*hd], K/V into the paged cache of one layer
+cudaError_t rope_append_launch(const float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer,
+                               const float2 *rope_table, RowMeta meta, const int32_t *page_table,
+                               int pt_width, int R, int Hq, int Hkv, int hd, int page_size,
+                               int n_pages, int max_pos, int *status, cudaStream_t s);
+cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s);
+cudaError_t gather_rows_launch(const float *x, const int32_t *src_rows, float *dst, int n, int d,
+                               cudaStream_t s);
+cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page, const int32_t *dst_page,
+                                      int n_copies, int n_layers, size_t layer_stride_elems,
+                                      int page_elems, cudaStream_t s);
+// decode-step preparation: advances the step counter, sets the rows' token and position
+cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
+                               int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s);
+cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row,
+                           const int32_t *seq_ids, const int32_t *d_step, uint32_t j_host,
+                           float temperature, uint64_t seed, const int32_t *forced, int forced_stride,
+                           int32_t *out_tok, float *out_lp, int out_stride, cudaStream_t s);
+cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n,
+                               uint32_t *words, float *uniform, cudaStream_t s);
+cudaError_t advantage_launch(const float *r, int P, int G, float eps, float *out, cudaStream_t s);
+cudaError_t set_int_launch(int32_t *p, int32_t v, cudaStream_t s);
+
+// ---- attention (attention.cu) ------------------------------------------------
+// One query row per activation row, keys 0..pos of its page-table row (causal by construction).
+cudaError_t attention_rows_launch(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer,
+                                  __nv_bfloat16 *out, RowMeta meta, const int32_t *page_table,
+                                  int pt_width, int R, int Hq, int Hkv, int hd, int page_size,
+                                  int n_pages, int *status, cudaStream_t s);
+
+}  // namespace echo

@@ -1,0 +1,385 @@
+// Row-wise kernels of the rollout path: embedding gather, RMSNorm, RoPE + paged-KV
+// append, SwiGLU, the Philox / Gumbel-max sampler with its log-probability, GRPO's
+// group advantage, and the small bookkeeping kernels a decode step needs.
+
+#include "common.cuh"
+
+namespace echo {
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11), restated from its published definition.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+    k.x += 0x9E3779B9u;
+    k.y += 0xBB67AE85u;
+  }
+  return c;
+}
+// w = (float(word) + 0.5f) * 2^-32 in IEEE fp32, each operation rounded on its own.
+__device__ __forceinline__ float uniform_from_word(uint32_t x) {
+  return __fmul_rn(__fadd_rn(__uint2float_rn(x), 0.5f), 2.3283064365386963e-10f);
+}
+// g = -log(-log1p(-w)); w == 1 gives -inf.
+__device__ __forceinline__ float gumbel_from_uniform(float w) { return -logf(-log1pf(-w)); }
+
+// ---------------------------------------------------------------------------
+__global__ void embed_kernel(const __nv_bfloat16 *embed, const int32_t *tok_src, const int32_t *tok_idx, float *x,
+                             int R, int d, int vocab, int *status) {
+  const int r = blockIdx.x;
+  if (r >= R) return;
+  int tok = tok_src[tok_idx ? tok_idx[r] : r];
+  if (tok < 0 || tok >= vocab) {
+    if (threadIdx.x == 0) atomicExch(status, STATUS_BAD_TOKEN);
+    tok = 0;
+  }
+  const __nv_bfloat162 *src = reinterpret_cast<const __nv_bfloat162 *>(embed + static_cast<size_t>(tok) * d);
+  float2 *dst = reinterpret_cast<float2 *>(x + static_cast<size_t>(r) * d);
+  for (int i = threadIdx.x; i < d / 2; i += blockDim.x) dst[i] = __bfloat1622float2(src[i]);
+}
+
+__device__ __forceinline__ float block_sum(float v, float *scratch) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int i = 0; i < nw; ++i) t += scratch[i];      // same order in every thread: deterministic
+  __syncthreads();
+  return t;
+}
+
+// h = bf16( x * rsqrt(mean(x^2) + eps) * gain )
+__global__ void rmsnorm_kernel(const float *x, const __nv_bfloat16 *gain, __nv_bfloat16 *h, int R, int d, float eps) {
+  __shared__ float scratch[32];
+  const int r = blockIdx.x;
+  const float *xr = x + static_cast<size_t>(r) * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = xr[i];
+    ss = fmaf(v, v, ss);
+  }
+  ss = block_sum(ss, scratch);
+  const float scale = rsqrtf(ss / static_cast<float>(d) + eps);
+  __nv_bfloat16 *hr = h + static_cast<size_t>(r) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x)
+    hr[i] = __float2bfloat16(xr[i] * scale * __bfloat162float(gain[i]));
+}
+
+// table[pos][i] = (cos, sin)(pos * theta^(-2i/hd)), angles in fp64
+__global__ void rope_table_kernel(float2 *table, int max_pos, int half, double theta, int hd) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= max_pos * half) return;
+  const int pos = idx / half, i = idx % half;
+  const double ang = static_cast<double>(pos) * pow(theta, -2.0 * i / hd);
+  table[idx] = make_float2(static_cast<float>(cos(ang)), static_cast<float>(sin(ang)));
+}
+
+// One block per activation row.  Rotates q and k heads (pairs (i, i + hd/2)), writes q as
+// bf16 and k, v as bf16 into the row's page slot.
+__global__ void rope_append_kernel(const float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer,
+                                   const float2 *rope_table, const int32_t *row_pt, const int32_t *row_pos,
+                                   const int32_t *page_table, int pt_width, int R, int Hq, int Hkv, int hd,
+                                   int page_size, int n_pages, int max_pos, int *status) {
+  const int r = blockIdx.x;
+  const int pos = row_pos[r];
+  const int half = hd / 2;
+  const int ld = (Hq + 2 * Hkv) * hd;
+  const float *src = qkv + static_cast<size_t>(r) * ld;
+  if (pos < 0 || pos >= max_pos) {
+    if (threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
+    return;
+  }
+  const int page = page_table[static_cast<size_t>(row_pt[r]) * pt_width + pos / page_size];
+  const int off = pos % page_size;
+  if (page < 0 || page >= n_pages) {
+    if (threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
+    return;
+  }
+  const float2 *cs = rope_table + static_cast<size_t>(pos) * half;
+  // q heads
+  for (int idx = threadIdx.x; idx < Hq * half; idx += blockDim.x) {
+    const int head = idx / half, i = idx % half;
+    const float a = src[head * hd + i], b = src[head * hd + i + half];
+    const float2 t = cs[i];
+    __nv_bfloat16 *dst = q + static_cast<size_t>(r) * Hq * hd + head * hd;
+    dst[i] = __float2bfloat16(a * t.x - b * t.y);
+    dst[i + half] = __float2bfloat16(b * t.x + a * t.y);
+  }
+  // k heads (rotated) and v heads (plain) into the page slot
+  const size_t page_elems = static_cast<size_t>(page_size) * hd;
+  for (int idx = threadIdx.x; idx < Hkv * half; idx += blockDim.x) {
+    const int head = idx / half, i = idx % half;
+    const float *ks = src + (Hq + head) * hd;
+    const float *vs = src + (Hq + Hkv + head) * hd;
+    const float2 t = cs[i];
+    __nv_bfloat16 *kd = kv_layer + ((static_cast<size_t>(page) * Hkv + head) * 2 + 0) * page_elems + off * hd;
+    __nv_bfloat16 *vd = kd + page_elems;
+    const float a = ks[i], b = ks[i + half];
+    kd[i] = __float2bfloat16(a * t.x - b * t.y);
+    kd[i + half] = __float2bfloat16(b * t.x + a * t.y);
+    vd[i] = __float2bfloat16(vs[i]);
+    vd[i + half] = __float2bfloat16(vs[i + half]);
+  }
+}
+
+__global__ void swiglu_kernel(const float *gu, __nv_bfloat16 *act, int R, int F) {
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(R) * F) return;
+  const size_t r = idx / F, f = idx % F;
+  const float g = gu[r * 2 * F + f], u = gu[r * 2 * F + F + f];
+  act[idx] = __float2bfloat16(g / (1.0f + __expf(-g)) * u);
+}
+
+__global__ void gather_rows_kernel(const float *x, const int32_t *src_rows, float *dst, int n, int d) {
+  const int i = blockIdx.x;
+  const int r = src_rows[i];
+  if (r < 0) return;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) dst[static_cast<size_t>(i) * d + c] = x[static_cast<size_t>(r) * d + c];
+}
+
+// Copies whole KV pages (all kv heads, K and V) in every layer: grid (n_copies, n_layers).
+__global__ void copy_pages_kernel(__nv_bfloat16 *kv, const int32_t *src_page, const int32_t *dst_page,
+                                  size_t layer_stride_elems, int page_elems) {
+  const int c = blockIdx.x, l = blockIdx.y;
+  const uint4 *src = reinterpret_cast<const uint4 *>(kv + l * layer_stride_elems + static_cast<size_t>(src_page[c]) * page_elems);
+  uint4 *dst = reinterpret_cast<uint4 *>(kv + l * layer_stride_elems + static_cast<size_t>(dst_page[c]) * page_elems);
+  for (int i = threadIdx.x; i < page_elems / 8; i += blockDim.x) dst[i] = src[i];
+}
+
+// Start of decode step j = *d_step + 1: row b feeds the token produced at step j-1 at
+// position len0[b] + j - 1.  One block; the counter is bumped after every thread has read it.
+__global__ void decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
+                                   int32_t *row_tok, int32_t *row_pos, int B) {
+  const int j = *d_step + 1;
+  __syncthreads();
+  for (int b = threadIdx.x; b < B; b += blockDim.x) {
+    row_tok[b] = tok_hist[static_cast<size_t>(b) * T + (j - 1)];
+    row_pos[b] = seq_len0[b] + j - 1;
+  }
+  if (threadIdx.x == 0) *d_step = j;
+}
+
+__global__ void set_int_kernel(int32_t *p, int32_t v) { *p = v; }
+
+// ---------------------------------------------------------------------------
+// Sampler: one block per sequence row.  Single pass over the logits row keeps, per
+// thread, the running (max, sum of exp) of s = z / T and the best perturbed score
+// s + g with its id (ties -> lowest id); warp shuffles and one shared-memory stage
+// combine them.
+// ---------------------------------------------------------------------------
+struct Best {
+  float score;
+  int id;
+};
+__device__ __forceinline__ void best_update(Best &b, float sc, int id) {
+  if (sc > b.score || (sc == b.score && id < b.id)) {
+    b.score = sc;
+    b.id = id;
+  }
+}
+__device__ __forceinline__ void lse_update(float &m, float &l, float s) {
+  if (s > m) {
+    l = l * __expf(m - s) + 1.0f;
+    m = s;
+  } else {
+    l += __expf(s - m);
+  }
+}
+__device__ __forceinline__ void lse_merge(float &m, float &l, float m2, float l2) {
+  if (m2 == -INFINITY) return;
+  if (m == -INFINITY) {
+    m = m2;
+    l = l2;
+    return;
+  }
+  const float mm = fmaxf(m, m2);
+  l = l * __expf(m - mm) + l2 * __expf(m2 - mm);
+  m = mm;
+}
+
+constexpr int kSamplerThreads = 1024;
+
+__global__ void __launch_bounds__(kSamplerThreads)
+sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t *seq_ids, const int32_t *d_step,
+               uint32_t j_host, float inv_temperature, uint32_t key0, uint32_t key1, const int32_t *forced,
+               int forced_stride, int32_t *out_tok, float *out_lp, int out_stride) {
+  __shared__ float sm_m[32], sm_l[32], sm_score[32];
+  __shared__ int sm_id[32];
+  const int r = blockIdx.x;
+  const uint32_t j = d_step ? static_cast<uint32_t>(*d_step) : j_host;
+  const uint32_t s_id = seq_ids ? static_cast<uint32_t>(seq_ids[r]) : static_cast<uint32_t>(r);
+  const float *z = logits + static_cast<size_t>(r / rows_per_logit_row) * V;
+  const uint2 key = make_uint2(key0, key1);
+
+  float m = -INFINITY, l = 0.f;
+  Best best = {-INFINITY, 0x7fffffff};
+  const int nblk = (V + 3) >> 2;
+  const bool vec_ok = (V & 3) == 0;
+  for (int blk = threadIdx.x; blk < nblk; blk += blockDim.x) {
+    const uint4 w = philox4x32_10(make_uint4(static_cast<uint32_t>(blk), j, s_id, 0u), key);
+    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+    float zz[4];
+    const int v0 = blk << 2;
+    if (vec_ok) {
+      const float4 t = *reinterpret_cast<const float4 *>(z + v0);
+      zz[0] = t.x; zz[1] = t.y; zz[2] = t.z; zz[3] = t.w;
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) zz[i] = (v0 + i < V) ? z[v0 + i] : -INFINITY;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (v0 + i < V) {
+        const float s = zz[i] * inv_temperature;
+        lse_update(m, l, s);
+        best_update(best, s + gumbel_from_uniform(uniform_from_word(words[i])), v0 + i);
+      }
+    }
+  }
+  // warp reduction
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, o), l2 = __shfl_xor_sync(0xffffffffu, l, o);
+    lse_merge(m, l, m2, l2);
+    const float sc = __shfl_xor_sync(0xffffffffu, best.score, o);
+    const int id = __shfl_xor_sync(0xffffffffu, best.id, o);
+    best_update(best, sc, id);
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) {
+    sm_m[warp] = m; sm_l[warp] = l; sm_score[warp] = best.score; sm_id[warp] = best.id;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int nw = blockDim.x >> 5;
+    float mm = -INFINITY, ll = 0.f;
+    Best bb = {-INFINITY, 0x7fffffff};
+    for (int i = 0; i < nw; ++i) {
+      lse_merge(mm, ll, sm_m[i], sm_l[i]);
+      best_update(bb, sm_score[i], sm_id[i]);
+    }
+    const int tok = bb.id < V ? bb.id : 0;
+    const size_t o = static_cast<size_t>(r) * out_stride + j;
+    out_tok[o] = tok;
+    const int scored = forced ? forced[static_cast<size_t>(r) * forced_stride + j] : tok;
+    const int sc_id = (scored >= 0 && scored < V) ? scored : 0;
+    out_lp[o] = z[sc_id] * inv_temperature - (mm + logf(ll));
+  }
+}
+
+__global__ void noise_debug_kernel(uint32_t key0, uint32_t key1, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n,
+                                   uint32_t *words, float *uniform) {
+  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint32_t v = v0 + i;
+  const uint4 w = philox4x32_10(make_uint4(v >> 2, j, s_id, 0u), make_uint2(key0, key1));
+  const uint32_t arr[4] = {w.x, w.y, w.z, w.w};
+  const uint32_t x = arr[v & 3];
+  words[i] = x;
+  uniform[i] = uniform_from_word(x);
+}
+
+// A = (R - mean) / (std + eps), std with divisor (G - 1).  One warp per group.
+__global__ void advantage_kernel(const float *r, int P, int G, float eps, float *out) {
+  const int p = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (p >= P) return;
+  const float *rp = r + static_cast<size_t>(p) * G;
+  float s = 0.f;
+  for (int g = lane; g < G; g += 32) s += rp[g];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  const float mean = s / static_cast<float>(G);
+  float ss = 0.f;
+  for (int g = lane; g < G; g += 32) {
+    const float dlt = rp[g] - mean;
+    ss = fmaf(dlt, dlt, ss);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float denom = sqrtf(ss / static_cast<float>(G - 1)) + eps;
+  for (int g = lane; g < G; g += 32) out[static_cast<size_t>(p) * G + g] = (rp[g] - mean) / denom;
+}
+
+}  // namespace
+
+cudaError_t embed_launch(const __nv_bfloat16 *embed, const int32_t *tok_src, const int32_t *tok_idx, float *x, int R,
+                         int d, int vocab, int *status, cudaStream_t s) {
+  embed_kernel<<<R, 256, 0, s>>>(embed, tok_src, tok_idx, x, R, d, vocab, status);
+  return cudaGetLastError();
+}
+cudaError_t rmsnorm_launch(const float *x, const __nv_bfloat16 *gain, __nv_bfloat16 *h, int R, int d, float eps,
+                           cudaStream_t s) {
+  rmsnorm_kernel<<<R, 256, 0, s>>>(x, gain, h, R, d, eps);
+  return cudaGetLastError();
+}
+cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double theta, cudaStream_t s) {
+  const int half = head_dim / 2, n = max_pos * half;
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(table, max_pos, half, theta, head_dim);
+  return cudaGetLastError();
+}
+cudaError_t rope_append_launch(const float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer, const float2 *rope_table,
+                               RowMeta meta, const int32_t *page_table, int pt_width, int R, int Hq, int Hkv, int hd,
+                               int page_size, int n_pages, int max_pos, int *status, cudaStream_t s) {
+  rope_append_kernel<<<R, 256, 0, s>>>(qkv, q, kv_layer, rope_table, meta.row_pt, meta.row_pos, page_table, pt_width,
+                                       R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
+  return cudaGetLastError();
+}
+cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s) {
+  const size_t n = static_cast<size_t>(R) * F;
+  swiglu_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(gu, act, R, F);
+  return cudaGetLastError();
+}
+cudaError_t gather_rows_launch(const float *x, const int32_t *src_rows, float *dst, int n, int d, cudaStream_t s) {
+  gather_rows_kernel<<<n, 256, 0, s>>>(x, src_rows, dst, n, d);
+  return cudaGetLastError();
+}
+cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page, const int32_t *dst_page,
+                                      int n_copies, int n_layers, size_t layer_stride_elems, int page_elems,
+                                      cudaStream_t s) {
+  if (n_copies == 0) return cudaSuccess;
+  copy_pages_kernel<<<dim3(n_copies, n_layers), 256, 0, s>>>(kv, src_page, dst_page, layer_stride_elems, page_elems);
+  return cudaGetLastError();
+}
+cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
+                               int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s) {
+  decode_prep_kernel<<<1, 512, 0, s>>>(d_step, tok_hist, T, seq_len0, row_tok, row_pos, B);
+  return cudaGetLastError();
+}
+cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row, const int32_t *seq_ids,
+                           const int32_t *d_step, uint32_t j_host, float temperature, uint64_t seed,
+                           const int32_t *forced, int forced_stride, int32_t *out_tok, float *out_lp, int out_stride,
+                           cudaStream_t s) {
+  sampler_kernel<<<R, kSamplerThreads, 0, s>>>(logits, V, rows_per_logit_row, seq_ids, d_step, j_host,
+                                               1.0f / temperature, static_cast<uint32_t>(seed & 0xffffffffu),
+                                               static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok,
+                                               out_lp, out_stride);
+  return cudaGetLastError();
+}
+cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n, uint32_t *words,
+                               float *uniform, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  noise_debug_kernel<<<(n + 255) / 256, 256, 0, s>>>(static_cast<uint32_t>(seed & 0xffffffffu),
+                                                     static_cast<uint32_t>(seed >> 32), s_id, j, v0, n, words,
+                                                     uniform);
+  return cudaGetLastError();
+}
+cudaError_t advantage_launch(const float *r, int P, int G, float eps, float *out, cudaStream_t s) {
+  if (P == 0) return cudaSuccess;
+  advantage_kernel<<<(P + 7) / 8, 256, 0, s>>>(r, P, G, eps, out);
+  return cudaGetLastError();
+}
+cudaError_t set_int_launch(int32_t *p, int32_t v, cudaStream_t s) {
+  set_int_kernel<<<1, 1, 0, s>>>(p, v);
+  return cudaGetLastError();
+}
+
+}  // namespace echo

@@ -1,0 +1,882 @@
+// Host runtime and C ABI of the rollout library: arena carve-up, double weight buffer
+// with the version state machine, page-table plan, prefill + decode orchestration
+// (decode step captured once as a CUDA graph and replayed), stand-alone test entry points.
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace echo;
+
+namespace {
+
+constexpr size_t kAlign = 1024;
+constexpr int kChunkRows = 256;       // prompt tokens per prefill forward
+
+size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
+int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+struct Dims {
+  int L, d, Hq, Hkv, hd, F, V, Z;
+  int n_qkv() const { return (Hq + 2 * Hkv) * hd; }
+  size_t layer_weight_elems() const {
+    return static_cast<size_t>(n_qkv()) * d + static_cast<size_t>(d) * Hq * hd + 3ull * F * d + 2ull * d;
+  }
+  size_t weight_elems() const { return L * layer_weight_elems() + 2ull * V * d + d; }
+};
+
+struct Limits {
+  int P, G, Lp, T, B, R;            // R = rows of the activation buffers
+  int n_pre, n_dec, n_pages, pt_width, max_pos;
+};
+
+bool config_ok(const echo_config *c) {
+  if (!c) return false;
+  if (c->n_layers < 1 || c->d_model < 8 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->d_ff < 8 || c->vocab < 2)
+    return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->n_q_heads % c->n_kv_heads) return false;
+  const int rep = c->n_q_heads / c->n_kv_heads;
+  if (rep != 1 && rep != 2 && rep != 4 && rep != 8) return false;
+  if (c->head_dim == 64 && rep == 8) return false;
+  if (c->d_model % 8 || c->d_ff % 8) return false;
+  if (c->kv_page_size < 1 || c->kv_page_size > 256 || (c->kv_page_size * c->head_dim) % 8) return false;
+  if (c->max_prompts < 1 || c->max_G < 1 || c->max_prompt_len < 1 || c->max_new_tokens < 1) return false;
+  if (c->n_weight_buffers != 1 && c->n_weight_buffers != 2) return false;
+  if (c->eos_id != -1) return false;
+  if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return false;
+  if (static_cast<long long>(c->max_prompts) * c->max_G > (1 << 20)) return false;
+  return true;
+}
+
+Dims dims_of(const echo_config &c) {
+  return Dims{c.n_layers, c.d_model, c.n_q_heads, c.n_kv_heads, c.head_dim, c.d_ff, c.vocab, c.kv_page_size};
+}
+
+Limits limits_of(const echo_config &c) {
+  Limits m;
+  m.P = c.max_prompts; m.G = c.max_G; m.Lp = c.max_prompt_len; m.T = c.max_new_tokens;
+  m.B = m.P * m.G;
+  m.R = std::max(m.B, kChunkRows);
+  const int Z = c.kv_page_size;
+  m.n_pre = ceil_div(m.Lp, Z);
+  int nd = 0;
+  for (int b = 0; b < Z && b <= m.Lp; ++b) nd = std::max(nd, ceil_div(b + m.T - 1, Z));
+  m.n_dec = nd;
+  m.n_pages = m.P * m.n_pre + m.B * m.n_dec;
+  m.pt_width = std::max(ceil_div(m.Lp + m.T - 1, Z), m.n_pre);
+  m.max_pos = m.Lp + m.T;
+  return m;
+}
+
+// Arena layout: offsets in bytes.
+struct Layout {
+  size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
+  size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
+      seq_len0, copy_src, copy_dst, d_step, status, stage_prompts, stage_tok, stage_lp, total;
+  size_t weight_bytes, kv_layer_elems, n_tables_ints;
+  int n_chunks_max;
+};
+
+Layout layout_of(const echo_config &c) {
+  const Dims D = dims_of(c);
+  const Limits M = limits_of(c);
+  Layout lo;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  lo.weight_bytes = align_up(D.weight_elems() * 2 + (static_cast<size_t>(D.L) * 9 + 3) * kAlign);
+  for (int b = 0; b < 2; ++b) lo.weights[b] = b < c.n_weight_buffers ? take(lo.weight_bytes) : 0;
+  lo.kv_layer_elems = static_cast<size_t>(M.n_pages) * D.Hkv * 2 * D.Z * D.hd;
+  lo.kv = take(lo.kv_layer_elems * D.L * 2);
+  lo.rope = take(static_cast<size_t>(M.max_pos) * (D.hd / 2) * sizeof(float2));
+  lo.x = take(static_cast<size_t>(M.R) * D.d * 4);
+  lo.h = take(static_cast<size_t>(M.R) * D.d * 2);
+  lo.qkv = take(static_cast<size_t>(M.R) * D.n_qkv() * 4);
+  lo.q = take(static_cast<size_t>(M.R) * D.Hq * D.hd * 2);
+  lo.attn = take(static_cast<size_t>(M.R) * D.Hq * D.hd * 2);
+  lo.act = take(static_cast<size_t>(M.R) * D.F * 2);
+  lo.gu = take(static_cast<size_t>(M.R) * 2 * D.F * 4);
+  lo.xlast = take(static_cast<size_t>(M.R) * D.d * 4);
+  lo.hlast = take(static_cast<size_t>(M.R) * D.d * 2);
+  lo.logits = take(static_cast<size_t>(M.R) * D.V * 4);
+  const size_t n_pre_tok = static_cast<size_t>(M.P) * M.Lp;
+  lo.n_chunks_max = static_cast<int>((n_pre_tok + kChunkRows - 1) / kChunkRows);
+  lo.page_table = take(static_cast<size_t>(M.B + M.P) * M.pt_width * 4);
+  lo.pre_row_pt = take(n_pre_tok * 4);
+  lo.pre_row_pos = take(n_pre_tok * 4);
+  lo.pre_tok_idx = take(n_pre_tok * 4);
+  lo.gather_map = take(static_cast<size_t>(lo.n_chunks_max) * M.P * 4);
+  lo.dec_row_tok = take(static_cast<size_t>(M.B) * 4);
+  lo.dec_row_pos = take(static_cast<size_t>(M.B) * 4);
+  lo.dec_row_pt = take(static_cast<size_t>(M.B) * 4);
+  lo.seq_len0 = take(static_cast<size_t>(M.B) * 4);
+  lo.copy_src = take(static_cast<size_t>(M.B) * 4);
+  lo.copy_dst = take(static_cast<size_t>(M.B) * 4);
+  lo.d_step = take(4);
+  lo.status = take(4);
+  lo.stage_prompts = take(static_cast<size_t>(M.P) * M.Lp * 4);
+  lo.stage_tok = take(static_cast<size_t>(M.B) * M.T * 4);
+  lo.stage_lp = take(static_cast<size_t>(M.B) * M.T * 4);
+  lo.total = off;
+  return lo;
+}
+
+struct WeightBuf {
+  uint8_t *base = nullptr;
+  __nv_bfloat16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
+  std::vector<__nv_bfloat16 *> wqkv, wo, wgu, wdown, attn_norm, mlp_norm;
+  std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
+  CUtensorMap tm_lm;
+  int64_t version = -1;
+  bool has_data = false;       // an install was enqueued into this buffer
+  cudaEvent_t installed = nullptr, inst_begin = nullptr, last_use = nullptr;
+  bool used = false;           // last_use has been recorded at least once
+};
+
+}  // namespace
+
+struct echo_ctx {
+  echo_config cfg;
+  Dims D;
+  Limits M;
+  Layout lo;
+  int device = 0;
+  uint8_t *arena = nullptr;
+  cudaStream_t stream = nullptr, copy_stream = nullptr;
+  WeightBuf wb[2];
+  int active = -1, pending = -1, last_install = -1;
+  int64_t newest_version = 0;
+  bool any_version = false;
+  cudaEvent_t plan_done = nullptr, all_done = nullptr;
+  bool plan_in_flight = false;
+  // pinned staging for the plan tables
+  int32_t *h_tables = nullptr;
+  size_t h_tables_ints = 0;
+  // last plan (host copy) for echo_debug_page_table
+  std::vector<int32_t> last_table;
+  int last_rows = 0, last_width = 0;
+  echo_stats stats{};
+  int64_t launches = 0;
+  bool use_simt = false, use_graph = true;
+  std::string last_error;
+
+  template <typename T>
+  T *ptr(size_t off) const { return reinterpret_cast<T *>(arena + off); }
+};
+
+namespace {
+
+int fail_cuda(echo_ctx *ctx, cudaError_t e, const char *what) {
+  if (ctx) {
+    char buf[256];
+    snprintf(buf, sizeof buf, "%s: %s", what, cudaGetErrorString(e));
+    ctx->last_error = buf;
+  }
+  return ECHO_ERR_CUDA;
+}
+
+#define CK(expr)                                            \
+  do {                                                      \
+    cudaError_t e__ = (expr);                               \
+    if (e__ != cudaSuccess) return fail_cuda(ctx, e__, #expr); \
+  } while (0)
+#define LAUNCH(expr)                                        \
+  do {                                                      \
+    cudaError_t e__ = (expr);                               \
+    if (e__ != cudaSuccess) return fail_cuda(ctx, e__, #expr); \
+    ctx->launches++;                                        \
+  } while (0)
+
+struct DeviceGuard {
+  int prev = -1;
+  explicit DeviceGuard(int dev) {
+    cudaGetDevice(&prev);
+    if (prev != dev) cudaSetDevice(dev);
+    else prev = -1;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+int pick_bnb(int rows) {
+  if (rows <= 32) return 32;
+  if (rows <= 64) return 64;
+  if (rows <= 128) return 128;
+  return 256;
+}
+
+// Y = X * W^T through the tensor-core kernel (or the SIMT reference when selected).
+int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, const __nv_bfloat16 *X, void *Y, int ldY,
+             int M, int N, int K, int epilogue) {
+  if (ctx->use_simt) {
+    if (epilogue == EPI_SWIGLU) {
+      float *gu = ctx->ptr<float>(ctx->lo.gu);
+      LAUNCH(gemm_simt_launch(X, W, gu, 2 * N, M, 2 * N, K, 0, ctx->stream));
+      LAUNCH(swiglu_launch(gu, reinterpret_cast<__nv_bfloat16 *>(Y), M, N, ctx->stream));
+      return ECHO_OK;
+    }
+    LAUNCH(gemm_simt_launch(X, W, reinterpret_cast<float *>(Y), ldY, M, N, K, epilogue == EPI_ACCUM, ctx->stream));
+    return ECHO_OK;
+  }
+  CUtensorMap tmX;
+  const int bnb = pick_bnb(M);
+  if (make_tensor_map(&tmX, X, M, K, K, bnb) != 0) {
+    ctx->last_error = "tensor map encode failed (activation)";
+    return ECHO_ERR_CUDA;
+  }
+  GemmArgs a{tmW, &tmX, Y, ldY, M, N, K, bnb, epilogue, ctx->ptr<int>(ctx->lo.status)};
+  LAUNCH(gemm_tc_launch(a, ctx->stream));
+  return ECHO_OK;
+}
+
+#define TRY(expr)                 \
+  do {                            \
+    int rc__ = (expr);            \
+    if (rc__ != ECHO_OK) return rc__; \
+  } while (0)
+
+// All layers for R activation rows already embedded in x.
+int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta) {
+  const Dims &D = ctx->D;
+  const Layout &lo = ctx->lo;
+  float *x = ctx->ptr<float>(lo.x);
+  __nv_bfloat16 *h = ctx->ptr<__nv_bfloat16>(lo.h);
+  float *qkv = ctx->ptr<float>(lo.qkv);
+  __nv_bfloat16 *q = ctx->ptr<__nv_bfloat16>(lo.q);
+  __nv_bfloat16 *attn = ctx->ptr<__nv_bfloat16>(lo.attn);
+  __nv_bfloat16 *act = ctx->ptr<__nv_bfloat16>(lo.act);
+  const int32_t *pt = ctx->ptr<int32_t>(lo.page_table);
+  int *status = ctx->ptr<int>(lo.status);
+  const float2 *rope = ctx->ptr<float2>(lo.rope);
+  for (int l = 0; l < D.L; ++l) {
+    __nv_bfloat16 *kv_layer = ctx->ptr<__nv_bfloat16>(lo.kv) + static_cast<size_t>(l) * lo.kv_layer_elems;
+    LAUNCH(rmsnorm_launch(x, w.attn_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream));
+    TRY(run_gemm(ctx, &w.tm_qkv[l], w.wqkv[l], h, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE));
+    LAUNCH(rope_append_launch(qkv, q, kv_layer, rope, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
+                              ctx->M.n_pages, ctx->M.max_pos, status, ctx->stream));
+    LAUNCH(attention_rows_launch(q, kv_layer, attn, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
+                                 ctx->M.n_pages, status, ctx->stream));
+    TRY(run_gemm(ctx, &w.tm_o[l], w.wo[l], attn, x, D.d, R, D.d, D.Hq * D.hd, EPI_ACCUM));
+    LAUNCH(rmsnorm_launch(x, w.mlp_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream));
+    TRY(run_gemm(ctx, &w.tm_gu[l], w.wgu[l], h, act, D.F, R, D.F, D.d, EPI_SWIGLU));
+    TRY(run_gemm(ctx, &w.tm_down[l], w.wdown[l], act, x, D.d, R, D.d, D.F, EPI_ACCUM));
+  }
+  return ECHO_OK;
+}
+
+// final norm + lm_head on `rows` rows of xsrc -> logits
+int lm_head(echo_ctx *ctx, const WeightBuf &w, const float *xsrc, int rows) {
+  const Dims &D = ctx->D;
+  __nv_bfloat16 *hl = ctx->ptr<__nv_bfloat16>(ctx->lo.hlast);
+  LAUNCH(rmsnorm_launch(xsrc, w.final_norm, hl, rows, D.d, ctx->cfg.rms_eps, ctx->stream));
+  return run_gemm(ctx, &w.tm_lm, w.lm_head, hl, ctx->ptr<float>(ctx->lo.logits), D.V, rows, D.V, D.d, EPI_STORE);
+}
+
+void carve_weights(echo_ctx *ctx, WeightBuf &w, uint8_t *base) {
+  const Dims &D = ctx->D;
+  w.base = base;
+  size_t off = 0;
+  auto take = [&](size_t elems) {
+    __nv_bfloat16 *p = reinterpret_cast<__nv_bfloat16 *>(base + off);
+    off = align_up(off + elems * 2);
+    return p;
+  };
+  w.embed = take(static_cast<size_t>(D.V) * D.d);
+  w.lm_head = take(static_cast<size_t>(D.V) * D.d);
+  w.final_norm = take(D.d);
+  w.wqkv.resize(D.L); w.wo.resize(D.L); w.wgu.resize(D.L); w.wdown.resize(D.L);
+  w.attn_norm.resize(D.L); w.mlp_norm.resize(D.L);
+  w.tm_qkv.resize(D.L); w.tm_o.resize(D.L); w.tm_gu.resize(D.L); w.tm_down.resize(D.L);
+  for (int l = 0; l < D.L; ++l) {
+    w.wqkv[l] = take(static_cast<size_t>(D.n_qkv()) * D.d);
+    w.wo[l] = take(static_cast<size_t>(D.d) * D.Hq * D.hd);
+    w.wgu[l] = take(2ull * D.F * D.d);
+    w.wdown[l] = take(static_cast<size_t>(D.d) * D.F);
+    w.attn_norm[l] = take(D.d);
+    w.mlp_norm[l] = take(D.d);
+  }
+}
+
+int make_weight_maps(echo_ctx *ctx, WeightBuf &w) {
+  const Dims &D = ctx->D;
+  int rc = 0;
+  rc |= make_tensor_map(&w.tm_lm, w.lm_head, D.V, D.d, D.d, kGemmTileN);
+  for (int l = 0; l < D.L; ++l) {
+    rc |= make_tensor_map(&w.tm_qkv[l], w.wqkv[l], D.n_qkv(), D.d, D.d, kGemmTileN);
+    rc |= make_tensor_map(&w.tm_o[l], w.wo[l], D.d, D.Hq * D.hd, D.Hq * D.hd, kGemmTileN);
+    rc |= make_tensor_map(&w.tm_gu[l], w.wgu[l], 2ull * D.F, D.d, D.d, kGemmTileN);
+    rc |= make_tensor_map(&w.tm_down[l], w.wdown[l], D.d, D.F, D.F, kGemmTileN);
+  }
+  if (rc) {
+    ctx->last_error = "tensor map encode failed (weights)";
+    return ECHO_ERR_CUDA;
+  }
+  return ECHO_OK;
+}
+
+// Flip to a newer snapshot if one is ready; returns the buffer to serve, or nullptr.
+WeightBuf *begin_rollout_version(echo_ctx *ctx, int *rc) {
+  *rc = ECHO_OK;
+  if (ctx->pending >= 0) {
+    WeightBuf &p = ctx->wb[ctx->pending];
+    bool take = ctx->active < 0;
+    if (!take) take = cudaEventQuery(p.installed) == cudaSuccess;
+    if (take) {
+      // order the compute stream after the install (a no-op when it has completed)
+      cudaError_t e = cudaStreamWaitEvent(ctx->stream, p.installed, 0);
+      if (e != cudaSuccess) {
+        *rc = fail_cuda(ctx, e, "cudaStreamWaitEvent(installed)");
+        return nullptr;
+      }
+      ctx->active = ctx->pending;
+      ctx->pending = -1;
+    }
+  }
+  if (ctx->active < 0) {
+    *rc = ECHO_ERR_NO_POLICY;
+    return nullptr;
+  }
+  return &ctx->wb[ctx->active];
+}
+
+struct Plan {
+  int P, G, T, B, n_tok, n_chunks, n_copies, n_pages, width;
+};
+
+// Page tables and row lists, written into the pinned staging block in the order of the
+// device-side table regions.  Sequence id s = p*G + g.  Prefix pages of prompt p:
+// pre_base[p] + [0, ceil(Lp/Z)); decode pages of s: dec_base[s] + [0, n_dec_p).
+int build_plan(echo_ctx *ctx, const int32_t *lens, int P, int G, int T, Plan *plan) {
+  const int Z = ctx->D.Z;
+  const Limits &M = ctx->M;
+  const int B = P * G, W = M.pt_width;
+  int32_t *h = ctx->h_tables;
+  int32_t *h_pt = h;
+  int32_t *h_row_pt = h_pt + static_cast<size_t>(M.B + M.P) * W;
+  int32_t *h_row_pos = h_row_pt + static_cast<size_t>(M.P) * M.Lp;
+  int32_t *h_tok_idx = h_row_pos + static_cast<size_t>(M.P) * M.Lp;
+  int32_t *h_gather = h_tok_idx + static_cast<size_t>(M.P) * M.Lp;
+  int32_t *h_dec_pt = h_gather + static_cast<size_t>(ctx->lo.n_chunks_max) * M.P;
+  int32_t *h_len0 = h_dec_pt + M.B;
+  int32_t *h_csrc = h_len0 + M.B;
+  int32_t *h_cdst = h_csrc + M.B;
+
+  std::fill(h_pt, h_pt + static_cast<size_t>(M.B + M.P) * W, -1);
+  int next_page = 0;
+  std::vector<int> pre_base(P);
+  for (int p = 0; p < P; ++p) {
+    pre_base[p] = next_page;
+    next_page += ceil_div(lens[p], Z);
+  }
+  int n_copies = 0;
+  for (int p = 0; p < P; ++p) {
+    const int full = lens[p] / Z, n_pre = ceil_div(lens[p], Z);
+    const int n_dec = ceil_div(lens[p] + T - 1, Z) - full;
+    // prefill row of prompt p sits after the B sequence rows
+    int32_t *pre_row = h_pt + static_cast<size_t>(B + p) * W;
+    for (int qi = 0; qi < n_pre; ++qi) pre_row[qi] = pre_base[p] + qi;
+    for (int g = 0; g < G; ++g) {
+      const int s = p * G + g;
+      int32_t *row = h_pt + static_cast<size_t>(s) * W;
+      for (int qi = 0; qi < full; ++qi) row[qi] = pre_base[p] + qi;
+      for (int qi = 0; qi < n_dec; ++qi) row[full + qi] = next_page + qi;
+      if (n_pre > full && n_dec > 0) {          // partial last prompt page: private copy per sample
+        h_csrc[n_copies] = pre_base[p] + full;
+        h_cdst[n_copies] = next_page;
+        ++n_copies;
+      }
+      next_page += n_dec;
+      h_dec_pt[s] = s;
+      h_len0[s] = lens[p];
+    }
+  }
+  if (next_page > M.n_pages) return ECHO_ERR_INVALID;
+  int n_tok = 0;
+  for (int p = 0; p < P; ++p) n_tok += lens[p];
+  const int n_chunks = ceil_div(n_tok, kChunkRows);
+  std::fill(h_gather, h_gather + static_cast<size_t>(n_chunks) * P, -1);
+  int i = 0;
+  for (int p = 0; p < P; ++p) {
+    for (int t = 0; t < lens[p]; ++t, ++i) {
+      h_row_pt[i] = B + p;
+      h_row_pos[i] = t;
+      h_tok_idx[i] = p * M.Lp + t;
+    }
+    const int last = i - 1;
+    h_gather[static_cast<size_t>(last / kChunkRows) * P + p] = last % kChunkRows;
+  }
+  *plan = Plan{P, G, T, B, n_tok, n_chunks, n_copies, next_page, W};
+  ctx->last_table.assign(h_pt, h_pt + static_cast<size_t>(B) * W);
+  ctx->last_rows = B;
+  ctx->last_width = W;
+  return ECHO_OK;
+}
+
+int upload_plan(echo_ctx *ctx, const Plan &pl) {
+  const Limits &M = ctx->M;
+  const Layout &lo = ctx->lo;
+  const int W = M.pt_width;
+  int32_t *h = ctx->h_tables;
+  size_t o = 0;
+  auto up = [&](size_t dev_off, size_t cap_ints, size_t n_ints) -> cudaError_t {
+    cudaError_t e = cudaSuccess;
+    if (n_ints) e = cudaMemcpyAsync(ctx->arena + dev_off, h + o, n_ints * 4, cudaMemcpyHostToDevice, ctx->stream);
+    o += cap_ints;
+    return e;
+  };
+  const size_t npt = static_cast<size_t>(M.P) * M.Lp;
+  // the prefill rows of the table sit at row index B of *this* call, so upload B+P rows contiguously
+  CK(up(lo.page_table, static_cast<size_t>(M.B + M.P) * W, static_cast<size_t>(pl.B + pl.P) * W));
+  CK(up(lo.pre_row_pt, npt, pl.n_tok));
+  CK(up(lo.pre_row_pos, npt, pl.n_tok));
+  CK(up(lo.pre_tok_idx, npt, pl.n_tok));
+  CK(up(lo.gather_map, static_cast<size_t>(lo.n_chunks_max) * M.P, static_cast<size_t>(pl.n_chunks) * pl.P));
+  CK(up(lo.dec_row_pt, M.B, pl.B));
+  CK(up(lo.seq_len0, M.B, pl.B));
+  CK(up(lo.copy_src, M.B, pl.n_copies));
+  CK(up(lo.copy_dst, M.B, pl.n_copies));
+  CK(cudaEventRecord(ctx->plan_done, ctx->stream));
+  ctx->plan_in_flight = true;
+  return ECHO_OK;
+}
+
+// One decode step: token j-1 in, token j out.  Every kernel reads the step index from
+// device memory, so the same launches (or the same captured graph) serve every step.
+int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t *tok_hist, float temperature,
+                uint64_t seed, const int32_t *forced, int32_t *out_tokens, float *out_logprobs) {
+  const Layout &lo = ctx->lo;
+  int32_t *d_step = ctx->ptr<int32_t>(lo.d_step);
+  int32_t *row_tok = ctx->ptr<int32_t>(lo.dec_row_tok);
+  int32_t *row_pos = ctx->ptr<int32_t>(lo.dec_row_pos);
+  LAUNCH(decode_prep_launch(d_step, tok_hist, pl.T, ctx->ptr<int32_t>(lo.seq_len0), row_tok, row_pos, pl.B,
+                            ctx->stream));
+  LAUNCH(embed_launch(w.embed, row_tok, nullptr, ctx->ptr<float>(lo.x), pl.B, ctx->D.d, ctx->D.V,
+                      ctx->ptr<int>(lo.status), ctx->stream));
+  RowMeta meta{ctx->ptr<int32_t>(lo.dec_row_pt), row_pos};
+  TRY(forward_layers(ctx, w, pl.B, meta));
+  TRY(lm_head(ctx, w, ctx->ptr<float>(lo.x), pl.B));
+  LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, ctx->D.V, 1, nullptr, d_step, 0, temperature, seed, forced,
+                        pl.T, out_tokens, out_logprobs, pl.T, ctx->stream));
+  return ECHO_OK;
+}
+
+int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int P, int G, int T,
+                 float temperature, uint64_t seed, const int32_t *forced, int32_t *out_tokens, float *out_logprobs,
+                 int64_t *out_versions) {
+  if (!ctx || !prompts || !prompt_lens || !out_tokens || !out_logprobs || !out_versions) return ECHO_ERR_INVALID;
+  const Limits &M = ctx->M;
+  if (P < 1 || P > M.P || G < 1 || G > M.G || T < 1 || T > M.T) return ECHO_ERR_INVALID;
+  if (!(temperature > 0.f) || !std::isfinite(temperature)) return ECHO_ERR_INVALID;
+  for (int p = 0; p < P; ++p)
+    if (prompt_lens[p] < 1 || prompt_lens[p] > M.Lp) return ECHO_ERR_INVALID;
+  DeviceGuard guard(ctx->device);
+
+  int rc;
+  WeightBuf *wp = begin_rollout_version(ctx, &rc);
+  if (!wp) return rc;
+  const WeightBuf &w = *wp;
+  for (int i = 0; i < P * G; ++i) out_versions[i] = w.version;
+
+  if (ctx->plan_in_flight) {       // the staging block is still being read by an earlier upload
+    CK(cudaEventSynchronize(ctx->plan_done));
+    ctx->plan_in_flight = false;
+  }
+  Plan pl;
+  TRY(build_plan(ctx, prompt_lens, P, G, T, &pl));
+  TRY(upload_plan(ctx, pl));
+
+  const Layout &lo = ctx->lo;
+  const Dims &D = ctx->D;
+  const int64_t launches0 = ctx->launches;
+  float *x = ctx->ptr<float>(lo.x);
+  int *status = ctx->ptr<int>(lo.status);
+
+  // ---- prefill: once per prompt, in chunks of kChunkRows tokens -------------
+  for (int c = 0; c < pl.n_chunks; ++c) {
+    const int r0 = c * kChunkRows, R = std::min(kChunkRows, pl.n_tok - r0);
+    LAUNCH(embed_launch(w.embed, prompts, ctx->ptr<int32_t>(lo.pre_tok_idx) + r0, x, R, D.d, D.V, status,
+                        ctx->stream));
+    RowMeta meta{ctx->ptr<int32_t>(lo.pre_row_pt) + r0, ctx->ptr<int32_t>(lo.pre_row_pos) + r0};
+    TRY(forward_layers(ctx, w, R, meta));
+    LAUNCH(gather_rows_launch(x, ctx->ptr<int32_t>(lo.gather_map) + static_cast<size_t>(c) * P,
+                              ctx->ptr<float>(lo.xlast), P, D.d, ctx->stream));
+  }
+  if (pl.n_copies) {
+    LAUNCH(copy_partial_pages_launch(ctx->ptr<__nv_bfloat16>(lo.kv), ctx->ptr<int32_t>(lo.copy_src),
+                                     ctx->ptr<int32_t>(lo.copy_dst), pl.n_copies, D.L, lo.kv_layer_elems,
+                                     D.Hkv * 2 * D.Z * D.hd, ctx->stream));
+  }
+  // ---- first token of every sample from the prompt's last logits row --------
+  TRY(lm_head(ctx, w, ctx->ptr<float>(lo.xlast), P));
+  LAUNCH(set_int_launch(ctx->ptr<int32_t>(lo.d_step), 0, ctx->stream));
+  LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, D.V, G, nullptr, nullptr, 0, temperature, seed, forced, T,
+                        out_tokens, out_logprobs, T, ctx->stream));
+
+  // ---- decode steps 1..T-1 ----------------------------------------------------
+  const int32_t *tok_hist = forced ? forced : out_tokens;
+  const int n_steps = T - 1;
+  bool graphed = false;
+  if (n_steps > 1 && ctx->use_graph && ctx->stream != nullptr) {
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    const int64_t before = ctx->launches;
+    if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+      int src = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs);
+      cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
+      const int64_t per_step = ctx->launches - before;
+      ctx->launches = before;
+      if (src != ECHO_OK) {
+        if (graph) cudaGraphDestroy(graph);
+        return src;
+      }
+      if (e == cudaSuccess && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+        for (int j = 1; j <= n_steps; ++j) {
+          cudaError_t le = cudaGraphLaunch(exec, ctx->stream);
+          if (le != cudaSuccess) {
+            cudaGraphExecDestroy(exec);
+            cudaGraphDestroy(graph);
+            return fail_cuda(ctx, le, "cudaGraphLaunch");
+          }
+        }
+        ctx->launches += per_step * n_steps;
+        graphed = true;
+        cudaGraphExecDestroy(exec);      // executions already enqueued keep their resources
+      } else {
+        cudaGetLastError();
+      }
+      if (graph) cudaGraphDestroy(graph);
+    } else {
+      cudaGetLastError();
+    }
+  }
+  if (!graphed) {
+    for (int j = 1; j <= n_steps; ++j)
+      TRY(decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs));
+  }
+  CK(cudaEventRecord(wp->last_use, ctx->stream));
+  wp->used = true;
+
+  ctx->stats.version_served = w.version;
+  ctx->stats.tokens_generated = static_cast<int64_t>(pl.B) * T;
+  ctx->stats.kernels_launched = ctx->launches - launches0;
+  ctx->stats.decode_steps = n_steps;
+  ctx->stats.n_pages = pl.n_pages;
+  return ECHO_OK;
+}
+
+}  // namespace
+
+// ============================================================================
+// C ABI
+// ============================================================================
+extern "C" {
+
+size_t echo_arena_bytes(const echo_config *cfg) {
+  if (!config_ok(cfg)) return 0;
+  return layout_of(*cfg).total;
+}
+
+int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_bytes, void *cuda_stream,
+                echo_ctx **out) {
+  if (!out) return ECHO_ERR_INVALID;
+  *out = nullptr;
+  if (!config_ok(cfg) || !arena) return ECHO_ERR_INVALID;
+  Layout lo = layout_of(*cfg);
+  if (arena_bytes < lo.total || (reinterpret_cast<uintptr_t>(arena) & 255)) return ECHO_ERR_ARENA;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return ECHO_ERR_CUDA;
+  DeviceGuard guard(device);
+  echo_ctx *ctx = new (std::nothrow) echo_ctx();
+  if (!ctx) return ECHO_ERR_INVALID;
+  ctx->cfg = *cfg;
+  ctx->D = dims_of(*cfg);
+  ctx->M = limits_of(*cfg);
+  ctx->lo = lo;
+  ctx->device = device;
+  // sub-allocations are 1 KiB-aligned relative to the base; the base's own 256-byte
+  // alignment satisfies every consumer (tensor maps need 16 bytes, vector loads 16 bytes)
+  ctx->arena = static_cast<uint8_t *>(arena);
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  const char *impl = getenv("ECHO_GEMM_IMPL");
+  ctx->use_simt = impl && !strcmp(impl, "simt");
+  const char *ng = getenv("ECHO_NO_GRAPH");
+  ctx->use_graph = !(ng && ng[0] == '1');
+
+  auto bail = [&](cudaError_t e, const char *what) {
+    fail_cuda(ctx, e, what);
+    fprintf(stderr, "echo_create: %s\n", ctx->last_error.c_str());
+    echo_destroy(ctx);
+    return ECHO_ERR_CUDA;
+  };
+  cudaError_t e;
+  if ((e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking)) != cudaSuccess)
+    return bail(e, "cudaStreamCreate");
+  for (int b = 0; b < cfg->n_weight_buffers; ++b) {
+    carve_weights(ctx, ctx->wb[b], ctx->arena + lo.weights[b]);
+    if ((e = cudaEventCreate(&ctx->wb[b].installed)) != cudaSuccess) return bail(e, "cudaEventCreate");
+    if ((e = cudaEventCreate(&ctx->wb[b].inst_begin)) != cudaSuccess) return bail(e, "cudaEventCreate");
+    if ((e = cudaEventCreateWithFlags(&ctx->wb[b].last_use, cudaEventDisableTiming)) != cudaSuccess)
+      return bail(e, "cudaEventCreate");
+    if (make_weight_maps(ctx, ctx->wb[b]) != ECHO_OK) {
+      fprintf(stderr, "echo_create: %s\n", ctx->last_error.c_str());
+      echo_destroy(ctx);
+      return ECHO_ERR_CUDA;
+    }
+  }
+  if ((e = cudaEventCreateWithFlags(&ctx->plan_done, cudaEventDisableTiming)) != cudaSuccess)
+    return bail(e, "cudaEventCreate");
+  if ((e = cudaEventCreateWithFlags(&ctx->all_done, cudaEventDisableTiming)) != cudaSuccess)
+    return bail(e, "cudaEventCreate");
+  const Limits &M = ctx->M;
+  ctx->h_tables_ints = static_cast<size_t>(M.B + M.P) * M.pt_width + 3ull * M.P * M.Lp +
+                       static_cast<size_t>(lo.n_chunks_max) * M.P + 4ull * M.B;
+  if ((e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_tables), ctx->h_tables_ints * 4, cudaHostAllocDefault)) !=
+      cudaSuccess)
+    return bail(e, "cudaHostAlloc");
+  if ((e = gemm_tc_configure()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute");
+  if ((e = cudaMemsetAsync(ctx->arena + lo.status, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
+  if ((e = cudaMemsetAsync(ctx->arena + lo.d_step, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
+  if ((e = rope_table_launch(ctx->ptr<float2>(lo.rope), M.max_pos, ctx->D.hd, static_cast<double>(cfg->rope_theta),
+                             ctx->stream)) != cudaSuccess)
+    return bail(e, "rope_table");
+  *out = ctx;
+  return ECHO_OK;
+}
+
+int echo_destroy(echo_ctx *ctx) {
+  if (!ctx) return ECHO_ERR_INVALID;
+  DeviceGuard guard(ctx->device);
+  if (ctx->stream || true) cudaStreamSynchronize(ctx->stream);
+  if (ctx->copy_stream) {
+    cudaStreamSynchronize(ctx->copy_stream);
+    cudaStreamDestroy(ctx->copy_stream);
+  }
+  for (int b = 0; b < 2; ++b) {
+    if (ctx->wb[b].installed) cudaEventDestroy(ctx->wb[b].installed);
+    if (ctx->wb[b].inst_begin) cudaEventDestroy(ctx->wb[b].inst_begin);
+    if (ctx->wb[b].last_use) cudaEventDestroy(ctx->wb[b].last_use);
+  }
+  if (ctx->plan_done) cudaEventDestroy(ctx->plan_done);
+  if (ctx->all_done) cudaEventDestroy(ctx->all_done);
+  if (ctx->h_tables) cudaFreeHost(ctx->h_tables);
+  delete ctx;
+  return ECHO_OK;
+}
+
+int echo_load_policy(echo_ctx *ctx, const echo_weights *src, int64_t version) {
+  if (!ctx || !src) return ECHO_ERR_INVALID;
+  if (!src->embed || !src->lm_head || !src->final_norm || !src->wq || !src->wk || !src->wv || !src->wo ||
+      !src->w_gate || !src->w_up || !src->w_down || !src->attn_norm || !src->mlp_norm)
+    return ECHO_ERR_INVALID;
+  const Dims &D = ctx->D;
+  for (int l = 0; l < D.L; ++l)
+    if (!src->wq[l] || !src->wk[l] || !src->wv[l] || !src->wo[l] || !src->w_gate[l] || !src->w_up[l] ||
+        !src->w_down[l] || !src->attn_norm[l] || !src->mlp_norm[l])
+      return ECHO_ERR_INVALID;
+  if (ctx->any_version && version <= ctx->newest_version) return ECHO_ERR_VERSION;
+  if (ctx->pending >= 0) return ECHO_ERR_BUSY;
+  DeviceGuard guard(ctx->device);
+
+  int target;
+  if (ctx->cfg.n_weight_buffers == 1) {
+    target = 0;
+  } else {
+    target = ctx->active < 0 ? 0 : 1 - ctx->active;
+  }
+  WeightBuf &w = ctx->wb[target];
+  cudaStream_t cs = ctx->copy_stream;
+  // the copy may not start before every rollout that reads this buffer has finished
+  if (w.used) CK(cudaStreamWaitEvent(cs, w.last_use, 0));
+  if (ctx->cfg.n_weight_buffers == 1) {
+    CK(cudaEventRecord(ctx->all_done, ctx->stream));
+    CK(cudaStreamWaitEvent(cs, ctx->all_done, 0));
+  }
+  CK(cudaEventRecord(w.inst_begin, cs));
+  auto cp = [&](void *dst, const void *s, size_t elems) {
+    return cudaMemcpyAsync(dst, s, elems * 2, cudaMemcpyDefault, cs);
+  };
+  const size_t d = D.d, qd = static_cast<size_t>(D.Hq) * D.hd, kd = static_cast<size_t>(D.Hkv) * D.hd;
+  CK(cp(w.embed, src->embed, static_cast<size_t>(D.V) * d));
+  CK(cp(w.lm_head, src->lm_head, static_cast<size_t>(D.V) * d));
+  CK(cp(w.final_norm, src->final_norm, d));
+  for (int l = 0; l < D.L; ++l) {
+    CK(cp(w.wqkv[l], src->wq[l], qd * d));
+    CK(cp(w.wqkv[l] + qd * d, src->wk[l], kd * d));
+    CK(cp(w.wqkv[l] + (qd + kd) * d, src->wv[l], kd * d));
+    CK(cp(w.wo[l], src->wo[l], d * qd));
+    CK(cp(w.wgu[l], src->w_gate[l], static_cast<size_t>(D.F) * d));
+    CK(cp(w.wgu[l] + static_cast<size_t>(D.F) * d, src->w_up[l], static_cast<size_t>(D.F) * d));
+    CK(cp(w.wdown[l], src->w_down[l], d * D.F));
+    CK(cp(w.attn_norm[l], src->attn_norm[l], d));
+    CK(cp(w.mlp_norm[l], src->mlp_norm[l], d));
+  }
+  CK(cudaEventRecord(w.installed, cs));
+  w.version = version;
+  w.has_data = true;
+  ctx->pending = target;
+  ctx->last_install = target;
+  if (ctx->cfg.n_weight_buffers == 1) ctx->active = -1;   // the old weights are being overwritten
+  ctx->newest_version = version;
+  ctx->any_version = true;
+  return ECHO_OK;
+}
+
+int echo_wait_policy(echo_ctx *ctx) {
+  if (!ctx) return ECHO_ERR_INVALID;
+  DeviceGuard guard(ctx->device);
+  if (ctx->pending >= 0) {
+    WeightBuf &w = ctx->wb[ctx->pending];
+    CK(cudaEventSynchronize(w.installed));
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, w.inst_begin, w.installed) == cudaSuccess) ctx->stats.install_ms = ms;
+  }
+  return ECHO_OK;
+}
+
+int echo_rollout(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int32_t P, int32_t G,
+                 int32_t max_new_tokens, float temperature, uint64_t seed, int32_t *out_tokens, float *out_logprobs,
+                 int64_t *out_versions) {
+  return rollout_impl(ctx, prompts, prompt_lens, P, G, max_new_tokens, temperature, seed, nullptr, out_tokens,
+                      out_logprobs, out_versions);
+}
+
+int echo_rollout_forced(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int32_t P, int32_t G,
+                        int32_t max_new_tokens, float temperature, uint64_t seed, const int32_t *forced_tokens,
+                        int32_t *out_tokens, float *out_logprobs, int64_t *out_versions) {
+  if (!forced_tokens) return ECHO_ERR_INVALID;
+  return rollout_impl(ctx, prompts, prompt_lens, P, G, max_new_tokens, temperature, seed, forced_tokens, out_tokens,
+                      out_logprobs, out_versions);
+}
+
+int echo_rollout_host(echo_ctx *ctx, const int32_t *prompts_host, const int32_t *prompt_lens, int32_t P, int32_t G,
+                      int32_t max_new_tokens, float temperature, uint64_t seed, int32_t *out_tokens_host,
+                      float *out_logprobs_host, int64_t *out_versions) {
+  if (!ctx || !prompts_host || !out_tokens_host || !out_logprobs_host) return ECHO_ERR_INVALID;
+  const Limits &M = ctx->M;
+  if (P < 1 || P > M.P || G < 1 || G > M.G || max_new_tokens < 1 || max_new_tokens > M.T) return ECHO_ERR_INVALID;
+  DeviceGuard guard(ctx->device);
+  const Layout &lo = ctx->lo;
+  int32_t *d_prompts = ctx->ptr<int32_t>(lo.stage_prompts);
+  int32_t *d_tok = ctx->ptr<int32_t>(lo.stage_tok);
+  float *d_lp = ctx->ptr<float>(lo.stage_lp);
+  CK(cudaMemcpyAsync(d_prompts, prompts_host, static_cast<size_t>(P) * M.Lp * 4, cudaMemcpyHostToDevice,
+                     ctx->stream));
+  TRY(rollout_impl(ctx, d_prompts, prompt_lens, P, G, max_new_tokens, temperature, seed, nullptr, d_tok, d_lp,
+                   out_versions));
+  const size_t n = static_cast<size_t>(P) * G * max_new_tokens;
+  CK(cudaMemcpyAsync(out_tokens_host, d_tok, n * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  CK(cudaMemcpyAsync(out_logprobs_host, d_lp, n * 4, cudaMemcpyDeviceToHost, ctx->stream));
+  return echo_sync(ctx);
+}
+
+int echo_group_advantage(const float *rewards, int32_t P, int32_t G, float eps, float *out_adv, void *cuda_stream) {
+  if (!rewards || !out_adv || P < 0 || G < 2 || !(eps >= 0.f)) return ECHO_ERR_INVALID;
+  cudaError_t e = advantage_launch(rewards, P, G, eps, out_adv, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+int echo_sync(echo_ctx *ctx) {
+  if (!ctx) return ECHO_ERR_INVALID;
+  DeviceGuard guard(ctx->device);
+  CK(cudaStreamSynchronize(ctx->stream));
+  CK(cudaStreamSynchronize(ctx->copy_stream));
+  ctx->plan_in_flight = false;
+  if (ctx->last_install >= 0) {
+    WeightBuf &w = ctx->wb[ctx->last_install];
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, w.inst_begin, w.installed) == cudaSuccess) ctx->stats.install_ms = ms;
+    else cudaGetLastError();
+  }
+  int status = 0;
+  CK(cudaMemcpy(&status, ctx->arena + ctx->lo.status, 4, cudaMemcpyDeviceToHost));
+  if (status != STATUS_OK) {
+    cudaMemset(ctx->arena + ctx->lo.status, 0, 4);
+    return status == STATUS_WAIT_TIMEOUT ? ECHO_ERR_TIMEOUT : ECHO_ERR_DEVICE_CHECK;
+  }
+  return ECHO_OK;
+}
+
+int echo_get_stats(echo_ctx *ctx, echo_stats *out) {
+  if (!ctx || !out) return ECHO_ERR_INVALID;
+  *out = ctx->stats;
+  return ECHO_OK;
+}
+
+int echo_debug_page_table(echo_ctx *ctx, int32_t *out, size_t n, int32_t *rows, int32_t *width) {
+  if (!ctx) return ECHO_ERR_INVALID;
+  if (rows) *rows = ctx->last_rows;
+  if (width) *width = ctx->last_width;
+  if (out) {
+    if (n < ctx->last_table.size()) return ECHO_ERR_INVALID;
+    std::copy(ctx->last_table.begin(), ctx->last_table.end(), out);
+  }
+  return ECHO_OK;
+}
+
+int echo_debug_noise(uint64_t seed, uint32_t s, uint32_t j, uint32_t v0, uint32_t n, uint32_t *out_words,
+                     float *out_uniform, void *cuda_stream) {
+  if (!out_words || !out_uniform) return ECHO_ERR_INVALID;
+  cudaError_t e = noise_debug_launch(seed, s, j, v0, n, out_words, out_uniform, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+int echo_sample(const float *logits, int32_t R, int32_t V, int32_t rows_per_logit_row, const int32_t *seq_ids,
+                uint32_t j, float temperature, uint64_t seed, const int32_t *forced, int32_t *out_tokens,
+                float *out_logprobs, void *cuda_stream) {
+  if (!logits || !out_tokens || !out_logprobs || R < 0 || V < 1 || rows_per_logit_row < 1) return ECHO_ERR_INVALID;
+  if (!(temperature > 0.f) || !std::isfinite(temperature)) return ECHO_ERR_INVALID;
+  if (R == 0) return ECHO_OK;
+  // stand-alone call: outputs are dense [R], so the stride is 1 and the step index is folded
+  // into the base pointers
+  cudaError_t e = sampler_launch(logits, R, V, rows_per_logit_row, seq_ids, nullptr, j, temperature, seed,
+                                 forced ? forced - j : nullptr, 1, out_tokens - j, out_logprobs - j, 1,
+                                 static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+int echo_gemm_bf16(const void *X, const void *W, float *Y, int32_t M, int32_t N, int32_t K, int32_t impl,
+                   void *cuda_stream) {
+  if (!X || !W || !Y || M < 1 || M > 4096 || N < 1 || K < 8 || (K % 8)) return ECHO_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (impl == 1) {
+    cudaError_t e = gemm_simt_launch(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(W), Y,
+                                     N, M, N, K, 0, s);
+    return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+  }
+  if (gemm_tc_configure() != cudaSuccess) return ECHO_ERR_CUDA;
+  CUtensorMap tmW, tmX;
+  const int bnb = pick_bnb(M);
+  if (make_tensor_map(&tmW, W, N, K, K, kGemmTileN) != 0) return ECHO_ERR_CUDA;
+  if (make_tensor_map(&tmX, X, M, K, K, bnb) != 0) return ECHO_ERR_CUDA;
+  GemmArgs a{&tmW, &tmX, Y, N, M, N, K, bnb, EPI_STORE, nullptr};
+  cudaError_t e = gemm_tc_launch(a, s);
+  return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+const char *echo_strerror(int code) {
+  switch (code) {
+    case ECHO_OK: return "ok";
+    case ECHO_ERR_INVALID: return "invalid argument";
+    case ECHO_ERR_ARENA: return "arena too small or misaligned";
+    case ECHO_ERR_NO_POLICY: return "no policy installed";
+    case ECHO_ERR_VERSION: return "version not strictly increasing";
+    case ECHO_ERR_BUSY: return "an install is still pending";
+    case ECHO_ERR_CUDA: return "CUDA error";
+    case ECHO_ERR_DEVICE_CHECK: return "device-side range check failed";
+    case ECHO_ERR_TIMEOUT: return "device-side wait timed out";
+    case ECHO_ERR_UNSUPPORTED: return "unsupported shape";
+    default: return "unknown error";
+  }
+}
+
+const char *echo_last_error(echo_ctx *ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+}  // extern "C"

@@ -1,0 +1,183 @@
+"""End-to-end GPU rollouts against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import decoder, pages
+from paper_2602_02192_b200 import synth
+from helpers import check_sequences, dims_of
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2602_02192_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def tiny(B):
+    wl = synth.WORKLOADS["tiny"]
+    w_t = synth.make_weights(wl.shape, wl.weight_seed)
+    w_o = decoder.Weights(synth.weights_to_bits(w_t))
+    w_d = {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in w_t.items()}
+    return wl, w_o, w_d
+
+
+def _engine(B, shape, P, G, Lp, T, nbuf=2):
+    return B.Engine(B.make_config(shape, P, G, Lp, T, nbuf))
+
+
+def test_tiny_config_full_parity(B, tiny):
+    wl, w_o, w_d = tiny
+    eng = _engine(B, wl.shape, wl.n_prompts, wl.G, wl.prompt_len, wl.new_tokens)
+    eng.echo_load_policy(w_d, 5)
+    prompts = synth.make_prompts(wl.n_prompts, wl.prompt_len, wl.shape.vocab, wl.prompt_seed)
+    lens = [wl.prompt_len] * wl.n_prompts
+    tok, lp, ver = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, wl.G, wl.new_tokens,
+                                    wl.temperature, wl.sample_seed)
+    eng.echo_sync()
+    tok, lp = tok.cpu().numpy(), lp.cpu().numpy()
+    assert np.all(ver == 5)
+    # page table: bit-exact against the oracle's plan
+    plan = pages.build(lens, wl.G, wl.new_tokens, 16)
+    got = eng.echo_debug_page_table()
+    assert got.shape[0] == wl.n_prompts * wl.G
+    assert np.array_equal(got[:, : plan.width], plan.table)
+    assert np.all(got[:, plan.width:] == -1)
+    assert eng.echo_get_stats()["n_pages"] == plan.n_pages
+    n, ex, worst = check_sequences(dims_of(wl.shape), w_o, prompts, lens, wl.G, wl.temperature, wl.sample_seed,
+                                   tok, lp, range(wl.n_prompts * wl.G))
+    assert n == wl.n_prompts * wl.G * wl.new_tokens
+    assert ex <= 0.05 * n
+    assert np.all(lp <= 0)
+    # samples of one group differ, and the run is reproducible
+    assert len({tuple(tok[0, g]) for g in range(wl.G)}) == wl.G
+    tok2, lp2, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, wl.G, wl.new_tokens,
+                                    wl.temperature, wl.sample_seed)
+    eng.echo_sync()
+    assert np.array_equal(tok2.cpu().numpy(), tok) and np.array_equal(lp2.cpu().numpy(), lp)
+    st = eng.echo_get_stats()
+    assert st["tokens_generated"] == tok.size and st["kernels_launched"] > 100
+    eng.close()
+
+
+def test_forced_rollout_scores_oracle_trajectory(B, tiny):
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 2, 3, 20, 12                    # Lp not a multiple of the page size
+    eng = _engine(B, wl.shape, P, G, 24, T)
+    eng.echo_load_policy(w_d, 0)
+    prompts, lens = synth.make_ragged_prompts([20, 13], wl.shape.vocab, 77, pad_to=24)
+    ref = decoder.rollout_cached(dims_of(wl.shape), w_o, prompts, lens, G, T, 1.0, 31)
+    forced = torch.from_numpy(ref.tokens).cuda()
+    tok, lp, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, G, T, 1.0, 31, forced=forced)
+    eng.echo_sync()
+    tok, lp = tok.cpu().numpy(), lp.cpu().numpy()
+    assert np.max(np.abs(lp - ref.logprobs)) <= 5e-2
+    diff = tok != ref.tokens
+    assert np.all(ref.margins[diff] < 1e-2) and np.all(tok[diff] == ref.runner_up[diff])
+    # page plan with ragged, non-page-aligned prompts
+    plan = pages.build(lens, G, T, 16)
+    got = eng.echo_debug_page_table()
+    assert np.array_equal(got[:, : plan.width], plan.table)
+    # free-running rollout on the same ragged prompts follows the acceptance rule too
+    tok, lp, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, G, T, 1.0, 31)
+    eng.echo_sync()
+    check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 1.0, 31, tok.cpu().numpy(), lp.cpu().numpy(),
+                    range(P * G))
+    eng.close()
+
+
+def test_edge_shapes(B, tiny):
+    wl, w_o, w_d = tiny
+    eng = _engine(B, wl.shape, 3, 5, 40, 9)
+    eng.echo_load_policy(w_d, 1)
+    for P, G, T, lens in [(1, 1, 1, [1]), (1, 2, 2, [16]), (3, 5, 9, [40, 17, 1]), (2, 1, 3, [33, 32])]:
+        prompts, lens_a = synth.make_ragged_prompts(lens, wl.shape.vocab, 5 + P, pad_to=40)
+        tok, lp, ver = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens_a, G, T, 0.8, 1234)
+        eng.echo_sync()
+        assert tok.shape == (P, G, T) and np.all(ver == 1)
+        check_sequences(dims_of(wl.shape), w_o, prompts, lens_a, G, 0.8, 1234, tok.cpu().numpy(),
+                        lp.cpu().numpy(), range(P * G))
+    # argument errors
+    prompts = torch.zeros((1, 40), dtype=torch.int32, device="cuda")
+    for kwargs in [dict(G=6), dict(T=10), dict(temp=0.0), dict(lens=[41]), dict(lens=[0])]:
+        with pytest.raises(B.EchoError) as ei:
+            eng.echo_rollout(prompts, kwargs.get("lens", [5]), kwargs.get("G", 2), kwargs.get("T", 3),
+                             kwargs.get("temp", 1.0), 0)
+        assert ei.value.code == -1
+    # an out-of-range token id is reported, not trapped on
+    bad = torch.full((1, 40), wl.shape.vocab + 3, dtype=torch.int32, device="cuda")
+    eng.echo_rollout(bad, [4], 1, 2, 1.0, 0)
+    with pytest.raises(B.EchoError) as ei:
+        eng.echo_sync()
+    assert ei.value.code == -7
+    eng.echo_sync()                                  # status is cleared; the context stays usable
+    eng.close()
+
+
+def test_versions_and_double_buffer(B, tiny):
+    wl, w_o, w_d = tiny
+    w1_t = synth.make_weights(wl.shape, 1)
+    w1_o = decoder.Weights(synth.weights_to_bits(w1_t))
+    w1_d = {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in w1_t.items()}
+    P, G, Lp, T = 2, 2, 16, 6
+    eng = _engine(B, wl.shape, P, G, Lp, T)
+    prompts = synth.make_prompts(P, Lp, wl.shape.vocab, 3)
+    dp = torch.from_numpy(prompts).cuda()
+    with pytest.raises(B.EchoError) as ei:
+        eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 0)
+    assert ei.value.code == -3                        # no policy yet
+    eng.echo_load_policy(w_d, 10)
+    with pytest.raises(B.EchoError) as ei:
+        eng.echo_load_policy(w1_d, 11)
+    assert ei.value.code == -5                        # first install not yet picked up
+    t0, l0, v0 = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
+    assert np.all(v0 == 10)
+    with pytest.raises(B.EchoError) as ei:
+        eng.echo_load_policy(w1_d, 10)
+    assert ei.value.code == -4                        # versions strictly increase
+    eng.echo_load_policy(w1_d, 11)
+    eng.echo_wait_policy()
+    t1, l1, v1 = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
+    assert np.all(v1 == 11)
+    eng.echo_sync()
+    d = dims_of(wl.shape)
+    check_sequences(d, w_o, prompts, [Lp] * P, G, 1.0, 7, t0.cpu().numpy(), l0.cpu().numpy(), range(P * G))
+    check_sequences(d, w1_o, prompts, [Lp] * P, G, 1.0, 7, t1.cpu().numpy(), l1.cpu().numpy(), range(P * G))
+    assert not np.array_equal(t0.cpu().numpy(), t1.cpu().numpy())
+    # a third snapshot goes back into the first buffer while version 11 serves
+    eng.echo_load_policy(w_d, 12)
+    eng.echo_wait_policy()
+    t2, l2, v2 = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
+    eng.echo_sync()
+    assert np.all(v2 == 12) and np.array_equal(t2.cpu().numpy(), t0.cpu().numpy())
+    eng.close()
+    # single buffer: the next rollout waits for the install and serves the new version
+    eng = _engine(B, wl.shape, P, G, Lp, T, nbuf=1)
+    eng.echo_load_policy(w_d, 0)
+    ta, _, va = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
+    eng.echo_load_policy(w1_d, 1)
+    tb, _, vb = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
+    eng.echo_sync()
+    assert np.all(va == 0) and np.all(vb == 1)
+    assert np.array_equal(ta.cpu().numpy(), t0.cpu().numpy()) and np.array_equal(tb.cpu().numpy(), t1.cpu().numpy())
+    eng.close()
+
+
+def test_host_buffer_entry_point(B, tiny):
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 2, 2, 16, 5
+    eng = _engine(B, wl.shape, P, G, Lp, T)
+    eng.echo_load_policy(w_d, 0)
+    prompts = synth.make_prompts(P, Lp, wl.shape.vocab, 8)
+    hp = torch.from_numpy(prompts).pin_memory()
+    ht = torch.empty((P, G, T), dtype=torch.int32).pin_memory()
+    hl = torch.empty((P, G, T), dtype=torch.float32).pin_memory()
+    ver = eng.echo_rollout_host(hp, [Lp] * P, G, T, 1.0, 3, ht, hl)
+    assert np.all(ver == 0)
+    tok, lp, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), [Lp] * P, G, T, 1.0, 3)
+    eng.echo_sync()
+    assert np.array_equal(ht.numpy(), tok.cpu().numpy()) and np.array_equal(hl.numpy(), lp.cpu().numpy())
+    eng.close()
