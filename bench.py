@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Rollout-generation benchmark: generated tokens/s on B200 for a named decoder shape.
+
+One "step" is one whole rollout of the workload: prefill of every prompt once, then T-1
+decode steps for all P*G sequences, sampling and log-probabilities included.  Inputs are
+seeded and synthetic (random-init bf16 weights, uniform token ids).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 8B] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  With --impl reference the CPU oracle is timed instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "rollout generated tokens/s"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = f"/tmp/echo_bench_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu_index), "-lms", "200"],
+                                         stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    smax.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# algorithmic bytes / flops of the workload (what the method must move, not what the kernels do)
+# ---------------------------------------------------------------------------------------------
+def model_counts(shape):
+    d, hd = shape.d_model, shape.head_dim
+    n_layer = d * hd * (2 * shape.n_q_heads + 2 * shape.n_kv_heads) + 3 * d * shape.d_ff
+    n_body = shape.n_layers * n_layer
+    n_lm = shape.vocab * d
+    kv_tok = 2 * shape.n_layers * shape.n_kv_heads * hd * 2          # bytes of K+V per token, all layers
+    return n_body, n_lm, kv_tok
+
+
+def step_bytes_flops(shape, P, G, Lp, i):
+    """Decode step i (1-based): weights once, each group's prefix once, each sample's own i
+    generated tokens, plus the new token's K/V write."""
+    n_body, n_lm, kv_tok = model_counts(shape)
+    B = P * G
+    byts = 2 * (n_body + n_lm) + kv_tok * (P * Lp + B * i) + kv_tok * B
+    flops = 2 * (n_body + n_lm) * B + 4 * shape.n_q_heads * shape.head_dim * shape.n_layers * B * (Lp + i)
+    return byts, flops
+
+
+def attention_bytes(shape, P, G, Lp, i):
+    """Algorithmic bytes of ONE layer's decode attention at step i: the group's prefix K/V once,
+    each sample's own generated K/V, q in and output out (bf16)."""
+    kv_tok_layer = 2 * shape.n_kv_heads * shape.head_dim * 2
+    B = P * G
+    return kv_tok_layer * (P * Lp + B * i) + 2 * B * shape.n_q_heads * shape.head_dim * 2
+
+
+def rollout_roofline_seconds(shape, P, G, Lp, T, bw_gbs, tflops):
+    n_body, n_lm, kv_tok = model_counts(shape)
+    pre_flops = 2 * n_body * P * Lp + 2 * shape.n_q_heads * shape.head_dim * shape.n_layers * P * Lp * Lp
+    pre_bytes = 2 * n_body + kv_tok * P * Lp
+    t = max(pre_bytes / (bw_gbs * 1e9), pre_flops / (tflops * 1e12))
+    for i in range(1, T):
+        b, f = step_bytes_flops(shape, P, G, Lp, i)
+        t += max(b / (bw_gbs * 1e9), f / (tflops * 1e12))
+    return t
+
+
+# ---------------------------------------------------------------------------------------------
+def run_ours(args):
+    from paper_2602_02192_b200 import binding, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    peaks = load_peaks()
+
+    wl = synth.WORKLOADS[args.workload]
+    shape, P, G, Lp, T = wl.shape, wl.n_prompts, wl.G, wl.prompt_len, wl.new_tokens
+    if args.new_tokens:
+        T = args.new_tokens
+    swap = args.workload == "8B" and not args.no_swap
+    nbuf = 1 if args.workload == "32B" else 2
+    eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, nbuf), device=local_rank)
+    weights = synth.make_weights(shape, wl.weight_seed, device=dev)
+    eng.echo_load_policy(weights, 0)
+    eng.echo_wait_policy()
+    w_next = None
+    if swap:
+        del weights
+        torch.cuda.empty_cache()
+        w_next = synth.make_weights(shape, wl.weight_seed + 1, device=dev)
+        torch.cuda.synchronize()
+
+    # every rank is an independent replica working on its own prompts (groups never split)
+    prompts = torch.from_numpy(synth.make_prompts(P, Lp, shape.vocab, wl.prompt_seed + 7919 * rank)).to(dev)
+    lens = [Lp] * P
+    out_tok = torch.empty((P, G, T), dtype=torch.int32, device=dev)
+    out_lp = torch.empty((P, G, T), dtype=torch.float32, device=dev)
+
+    def one_rollout(seed):
+        return eng.echo_rollout(prompts, lens, G, T, wl.temperature, seed, out_tokens=out_tok, out_logprobs=out_lp)
+
+    for w in range(args.warmup):
+        one_rollout(wl.sample_seed + w)
+    eng.echo_sync()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: K rollouts, device-resident inputs ---------------------------------
+    prof_every = max(1, (T - 1) // 16)
+    eng.echo_profile_config(prof_every)
+    clocks = ClockSampler(local_rank)
+    if rank == 0:
+        clocks.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    launches = 0
+    versions_seen = []
+    ev0.record(eng.stream)
+    for k in range(args.steps):
+        _, _, ver = one_rollout(wl.sample_seed + 100 + k)
+        versions_seen.append(int(ver[0, 0]))
+        launches += eng.echo_get_stats()["kernels_launched"]
+        if swap and k == 0:
+            eng.echo_load_policy(w_next, 1)       # overlaps the decode steps already enqueued
+    ev1.record(eng.stream)
+    eng.echo_sync()
+    barrier()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    clk = clocks.stop() if rank == 0 else None
+    prof_steps, prof_ms = eng.echo_profile_read()
+    eng.echo_profile_config(0)
+    install_ms = eng.echo_get_stats()["install_ms"]
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    tokens_total = world * args.steps * P * G * T
+    value = tokens_total / (elapsed_ms / 1e3)
+
+    # ---- end to end: host buffers, copies inside the timed region -------------------------
+    hp = prompts.cpu().pin_memory()
+    ht = torch.empty((P, G, T), dtype=torch.int32).pin_memory()
+    hl = torch.empty((P, G, T), dtype=torch.float32).pin_memory()
+    barrier()
+    t0 = time.perf_counter()
+    ver_e2e = eng.echo_rollout_host(hp, lens, G, T, wl.temperature, wl.sample_seed + 999, ht, hl)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = world * P * G * T / e2e_s
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (decode attention), from the sampled steps ---------
+    attn_launches = len(prof_steps) * shape.n_layers
+    roof = None
+    if attn_launches:
+        alg = sum(attention_bytes(shape, P, G, Lp, int(j)) for j in prof_steps) * shape.n_layers
+        dur_s = float(prof_ms[:, 0].sum()) / 1e3
+        achieved = alg / dur_s / 1e9
+        tot = float(prof_ms[:, 3].sum())
+        roof = {"bound": "hbm", "kernel": "decode attention (paged GQA)", "achieved": round(achieved, 1),
+                "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
+                "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None,
+                "launches_timed": attn_launches,
+                "avg_launch_us": round(dur_s / attn_launches * 1e6, 2),
+                "sampled_steps": [int(j) for j in prof_steps],
+                "share_of_step": {"attention": round(float(prof_ms[:, 0].sum()) / tot, 4),
+                                  "projections": round(float(prof_ms[:, 1].sum()) / tot, 4),
+                                  "sampler": round(float(prof_ms[:, 2].sum()) / tot, 4)},
+                "step_ms": [round(float(x), 3) for x in prof_ms[:, 3]],
+                "attn_ms": [round(float(x), 3) for x in prof_ms[:, 0]],
+                "gemm_ms": [round(float(x), 3) for x in prof_ms[:, 1]]}
+    t_meas = rollout_roofline_seconds(shape, P, G, Lp, T, peaks["hbm_gbs"], peaks["bf16_tflops_sustained"])
+    t_nom = rollout_roofline_seconds(shape, P, G, Lp, T, 8000.0, 2250.0)
+    per_rollout_s = elapsed_ms / 1e3 / args.steps
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        cpu = cpu_baseline_sample(shape, w_next if swap else weights, prompts, ht, wl)
+
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(elapsed_ms / args.steps, 2), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{wl.name}-shape decoder: L{shape.n_layers} d{shape.d_model} "
+                               f"{shape.n_q_heads}q/{shape.n_kv_heads}kv hd{shape.head_dim} F{shape.d_ff} "
+                               f"V{shape.vocab}; {P} prompts x G={G}, prompt {Lp}, {T} new tokens, T=1.0",
+                   "policy_swap": "one echo_load_policy of a re-seeded weight set during timed step 0" if swap
+                   else "none", "versions_served": versions_seen, "e2e_version": int(ver_e2e[0, 0]),
+                   "install_ms": round(install_ms, 1),
+                   "l2": "inputs larger than L2 (weights + KV >> 126 MB)", "parallelism": f"replicas x{world}"},
+        "clocks": clk,
+        "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": int(hp.numel() * 4),
+                "d2h_bytes_per_step": int(ht.numel() * 4 + hl.numel() * 4)},
+        "gpu_launches": int(launches),
+        "roofline": roof,
+        "rollout_roofline": {"frac_of_measured": round(t_meas / per_rollout_s, 4),
+                             "frac_of_nominal_8TBs_2250TF": round(t_nom / per_rollout_s, 4),
+                             "roofline_s_measured": round(t_meas, 3), "roofline_s_nominal": round(t_nom, 3)},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    eng.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ---------------------------------------------------------------------------------------------
+def _oracle_dims(shape):
+    from oracle import decoder
+    return decoder.ModelDims(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                             shape.d_ff, shape.vocab, shape.rms_eps, shape.rope_theta)
+
+
+class _StreamedWeights:
+    """Feeds the oracle one layer at a time from bf16 tensors (exact widening to fp64)."""
+
+    def __init__(self, weights, cache=False):
+        self.w = weights
+        self.cache = {} if cache else None
+        self._wide = lambda t: t.detach().to("cpu").to(torch.float64).numpy()
+        self.embed = _EmbedRows(weights["embed"], self._wide)
+        self.lm_head = self._wide(weights["lm_head"])
+        self.final_norm = self._wide(weights["final_norm"])
+
+    def layer(self, l):
+        if self.cache is not None and l in self.cache:
+            return self.cache[l]
+        lw = {k: self._wide(self.w[k][l]) for k in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down",
+                                                    "attn_norm", "mlp_norm")}
+        if self.cache is not None:
+            self.cache[l] = lw
+        return lw
+
+
+class _EmbedRows:
+    def __init__(self, t, wide):
+        self.t, self.wide = t, wide
+
+    def __getitem__(self, ids):
+        idx = torch.as_tensor(np.asarray(ids), device=self.t.device, dtype=torch.long)
+        return self.wide(self.t[idx])
+
+
+def _oracle_sample_pass(shape, sw, prompt_ids, given, temperature, seed, s):
+    from oracle import decoder
+    return decoder.score_forced(_oracle_dims(shape), sw, prompt_ids, given, temperature, seed, s,
+                                layer_provider=sw.layer)
+
+
+SAMPLE_PROMPT = 24
+SAMPLE_NEW = 8
+
+
+def cpu_baseline_sample(shape, weights, prompts, host_tokens, wl):
+    """Times the oracle, as it stands, on a bounded sample of the same workload."""
+    cores = os.cpu_count() or 1
+    prompt_ids = prompts[0, :SAMPLE_PROMPT].cpu().numpy()
+    given = host_tokens[0, 0, :SAMPLE_NEW].numpy()
+    t0 = time.perf_counter()
+    sw = _StreamedWeights(weights)
+    _oracle_sample_pass(shape, sw, prompt_ids, given, wl.temperature, wl.sample_seed, 0)
+    dt = time.perf_counter() - t0
+    return {"value": round(SAMPLE_NEW / dt, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "seconds": round(dt, 2),
+            "sample": f"1 sequence of the {wl.name}-shape workload: first {SAMPLE_PROMPT} prompt tokens + "
+                      f"{SAMPLE_NEW} generated tokens scored teacher-forced in one causal pass (fp64 numpy), "
+                      f"all {shape.n_layers} layers streamed from the bf16 weights (widening included)"}
+
+
+def run_reference(args):
+    """The CPU oracle timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2602_02192_b200 import synth
+    wl = synth.WORKLOADS[args.workload]
+    shape = wl.shape
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    weights = synth.make_weights(shape, wl.weight_seed, device=dev)
+    sw = _StreamedWeights(weights, cache=True)
+    prompts = synth.make_prompts(wl.n_prompts, wl.prompt_len, shape.vocab, wl.prompt_seed)
+    rng = np.random.default_rng(0)
+    given = rng.integers(0, shape.vocab, size=SAMPLE_NEW)
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        _oracle_sample_pass(shape, sw, prompts[0, :SAMPLE_PROMPT], given, wl.temperature, wl.sample_seed, 0)
+        dt = time.perf_counter() - t0
+        if it >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = SAMPLE_NEW * len(times) / total
+    cores = os.cpu_count() or 1
+    sample = (f"per step: 1 sequence of the {wl.name}-shape workload, first {SAMPLE_PROMPT} prompt tokens + "
+              f"{SAMPLE_NEW} tokens scored teacher-forced in one causal pass (fp64 numpy); weights widened "
+              f"to fp64 once before timing")
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total / len(times) * 1e3, 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic",
+            "config": {"workload": f"{wl.name}-shape decoder; bounded sample of {wl.n_prompts} prompts x "
+                                   f"G={wl.G}, prompt {wl.prompt_len}, {wl.new_tokens} new tokens"},
+            "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="8B", choices=["tiny", "0.6B", "4B", "8B", "32B"])
+    ap.add_argument("--new-tokens", type=int, default=0, help="override T (diagnostic runs only)")
+    ap.add_argument("--no-swap", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -175,6 +175,17 @@ int echo_sync(echo_ctx *ctx);
 
 int echo_get_stats(echo_ctx *ctx, echo_stats *out);
 
+/* Sampled per-kernel timing.  With every_n_steps = n > 0, every n-th decode step of later
+ * rollouts is launched kernel by kernel (not as a graph replay) with CUDA events around the
+ * attention launches, the dense projections, the sampler and the whole step; 0 turns it off.
+ * echo_profile_read waits for the stream and returns, for each sampled step of the most
+ * recent rollout, its index in steps[i] (host int32) and four summed durations in
+ * milliseconds in ms[4*i + c] (host fp32): c = 0 attention, 1 projections, 2 sampler,
+ * 3 whole step.  capacity is the number of steps both arrays can hold; *n_out receives the
+ * number of sampled steps (pass steps = ms = NULL to query it). */
+int echo_profile_config(echo_ctx *ctx, int32_t every_n_steps);
+int echo_profile_read(echo_ctx *ctx, int32_t *steps, float *ms, int32_t capacity, int32_t *n_out);
+
 /* Copy the page table of the most recent rollout to host memory:
  * int32 [P*G][width]; entries past a sequence's last page are -1.  `width` and
  * the number of rows are returned through the pointers; `out` may be NULL to

@@ -75,6 +75,8 @@ def _load() -> C.CDLL:
     lib.echo_group_advantage.argtypes = [vp, i32, i32, f32, vp, vp]
     lib.echo_sync.argtypes = [vp]
     lib.echo_get_stats.argtypes = [vp, C.POINTER(EchoStats)]
+    lib.echo_profile_config.argtypes = [vp, i32]
+    lib.echo_profile_read.argtypes = [vp, vp, vp, i32, C.POINTER(i32)]
     lib.echo_debug_page_table.argtypes = [vp, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32)]
     lib.echo_debug_noise.argtypes = [u64, u32, u32, u32, u32, vp, vp, vp]
     lib.echo_sample.argtypes = [vp, i32, i32, i32, vp, u32, f32, u64, vp, vp, vp, vp]
@@ -85,7 +87,8 @@ def _load() -> C.CDLL:
     lib.echo_last_error.argtypes = [vp]
     for name in ("echo_create", "echo_destroy", "echo_load_policy", "echo_wait_policy", "echo_rollout",
                  "echo_rollout_forced", "echo_rollout_host", "echo_group_advantage", "echo_sync",
-                 "echo_get_stats", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16"):
+                 "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
+                 "echo_profile_config", "echo_profile_read"):
         getattr(lib, name).restype = C.c_int
     return lib
 
@@ -94,7 +97,7 @@ lib = _load()
 
 EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy", "echo_wait_policy",
             "echo_rollout", "echo_rollout_forced", "echo_rollout_host", "echo_group_advantage", "echo_sync",
-            "echo_get_stats", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
+            "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
             "echo_strerror", "echo_last_error"]
 
 
@@ -234,6 +237,20 @@ class Engine:
         st = EchoStats()
         _check(lib.echo_get_stats(self._ctx, C.byref(st)))
         return {k: getattr(st, k) for k, _ in EchoStats._fields_ if k != "reserved"}
+
+    def echo_profile_config(self, every_n_steps: int):
+        _check(lib.echo_profile_config(self._ctx, int(every_n_steps)))
+
+    def echo_profile_read(self):
+        """(steps int32 [n], ms fp32 [n][4]) of the last rollout: attention, projections, sampler, step."""
+        n = C.c_int32()
+        _check(lib.echo_profile_read(self._ctx, None, None, 0, C.byref(n)), self._ctx)
+        steps = np.zeros(n.value, dtype=np.int32)
+        ms = np.zeros((n.value, 4), dtype=np.float32)
+        if n.value:
+            _check(lib.echo_profile_read(self._ctx, steps.ctypes.data, ms.ctypes.data, n.value, C.byref(n)),
+                   self._ctx)
+        return steps, ms
 
     def echo_debug_page_table(self) -> np.ndarray:
         rows, width = C.c_int32(), C.c_int32()

@@ -166,6 +166,14 @@ struct echo_ctx {
   int64_t launches = 0;
   bool use_simt = false, use_graph = true;
   std::string last_error;
+  // sampled per-kernel timing (echo_profile_config / echo_profile_read)
+  int prof_every = 0;
+  bool prof_now = false;
+  int prof_step = 0;
+  struct ProfRec { int step, cls; cudaEvent_t a, b; };
+  std::vector<ProfRec> prof_recs;
+  std::vector<cudaEvent_t> prof_pool;
+  size_t prof_pool_used = 0;
 
   template <typename T>
   T *ptr(size_t off) const { return reinterpret_cast<T *>(arena + off); }
@@ -181,6 +189,33 @@ int fail_cuda(echo_ctx *ctx, cudaError_t e, const char *what) {
   }
   return ECHO_ERR_CUDA;
 }
+
+cudaEvent_t prof_event(echo_ctx *ctx) {
+  if (ctx->prof_pool_used == ctx->prof_pool.size()) {
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    ctx->prof_pool.push_back(e);
+  }
+  return ctx->prof_pool[ctx->prof_pool_used++];
+}
+// Brackets the launches issued inside its scope with two events when the step is sampled.
+struct ProfScope {
+  echo_ctx *ctx;
+  cudaEvent_t a = nullptr, b = nullptr;
+  int cls;
+  ProfScope(echo_ctx *c, int cls_) : ctx(c), cls(cls_) {
+    if (!ctx->prof_now) return;
+    a = prof_event(ctx);
+    b = prof_event(ctx);
+    if (a && b) cudaEventRecord(a, ctx->stream);
+  }
+  ~ProfScope() {
+    if (!a || !b) return;
+    cudaEventRecord(b, ctx->stream);
+    ctx->prof_recs.push_back({ctx->prof_step, cls, a, b});
+  }
+};
+enum { PROF_ATTN = 0, PROF_GEMM = 1, PROF_SAMPLER = 2, PROF_STEP = 3, PROF_NCLS = 4 };
 
 #define CK(expr)                                            \
   do {                                                      \
@@ -216,6 +251,7 @@ int pick_bnb(int rows) {
 // Y = X * W^T through the tensor-core kernel (or the SIMT reference when selected).
 int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, const __nv_bfloat16 *X, void *Y, int ldY,
              int M, int N, int K, int epilogue) {
+  ProfScope prof(ctx, PROF_GEMM);
   if (ctx->use_simt) {
     if (epilogue == EPI_SWIGLU) {
       float *gu = ctx->ptr<float>(ctx->lo.gu);
@@ -262,8 +298,11 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta) {
     TRY(run_gemm(ctx, &w.tm_qkv[l], w.wqkv[l], h, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE));
     LAUNCH(rope_append_launch(qkv, q, kv_layer, rope, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
                               ctx->M.n_pages, ctx->M.max_pos, status, ctx->stream));
-    LAUNCH(attention_rows_launch(q, kv_layer, attn, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
-                                 ctx->M.n_pages, status, ctx->stream));
+    {
+      ProfScope prof(ctx, PROF_ATTN);
+      LAUNCH(attention_rows_launch(q, kv_layer, attn, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
+                                   ctx->M.n_pages, status, ctx->stream));
+    }
     TRY(run_gemm(ctx, &w.tm_o[l], w.wo[l], attn, x, D.d, R, D.d, D.Hq * D.hd, EPI_ACCUM));
     LAUNCH(rmsnorm_launch(x, w.mlp_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream));
     TRY(run_gemm(ctx, &w.tm_gu[l], w.wgu[l], h, act, D.F, R, D.F, D.d, EPI_SWIGLU));
@@ -456,6 +495,7 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
   int32_t *d_step = ctx->ptr<int32_t>(lo.d_step);
   int32_t *row_tok = ctx->ptr<int32_t>(lo.dec_row_tok);
   int32_t *row_pos = ctx->ptr<int32_t>(lo.dec_row_pos);
+  ProfScope prof_step(ctx, PROF_STEP);
   LAUNCH(decode_prep_launch(d_step, tok_hist, pl.T, ctx->ptr<int32_t>(lo.seq_len0), row_tok, row_pos, pl.B,
                             ctx->stream));
   LAUNCH(embed_launch(w.embed, row_tok, nullptr, ctx->ptr<float>(lo.x), pl.B, ctx->D.d, ctx->D.V,
@@ -463,8 +503,11 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
   RowMeta meta{ctx->ptr<int32_t>(lo.dec_row_pt), row_pos};
   TRY(forward_layers(ctx, w, pl.B, meta));
   TRY(lm_head(ctx, w, ctx->ptr<float>(lo.x), pl.B));
-  LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, ctx->D.V, 1, nullptr, d_step, 0, temperature, seed, forced,
-                        pl.T, out_tokens, out_logprobs, pl.T, ctx->stream));
+  {
+    ProfScope prof(ctx, PROF_SAMPLER);
+    LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, ctx->D.V, 1, nullptr, d_step, 0, temperature, seed,
+                          forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream));
+  }
   return ECHO_OK;
 }
 
@@ -523,44 +566,47 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   // ---- decode steps 1..T-1 ----------------------------------------------------
   const int32_t *tok_hist = forced ? forced : out_tokens;
   const int n_steps = T - 1;
-  bool graphed = false;
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  int64_t per_step = 0;
   if (n_steps > 1 && ctx->use_graph && ctx->stream != nullptr) {
-    cudaGraph_t graph = nullptr;
-    cudaGraphExec_t exec = nullptr;
     const int64_t before = ctx->launches;
     if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
       int src = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs);
       cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
-      const int64_t per_step = ctx->launches - before;
+      per_step = ctx->launches - before;
       ctx->launches = before;
       if (src != ECHO_OK) {
         if (graph) cudaGraphDestroy(graph);
         return src;
       }
-      if (e == cudaSuccess && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
-        for (int j = 1; j <= n_steps; ++j) {
-          cudaError_t le = cudaGraphLaunch(exec, ctx->stream);
-          if (le != cudaSuccess) {
-            cudaGraphExecDestroy(exec);
-            cudaGraphDestroy(graph);
-            return fail_cuda(ctx, le, "cudaGraphLaunch");
-          }
-        }
-        ctx->launches += per_step * n_steps;
-        graphed = true;
-        cudaGraphExecDestroy(exec);      // executions already enqueued keep their resources
-      } else {
+      if (e != cudaSuccess || cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) {
         cudaGetLastError();
+        exec = nullptr;
       }
-      if (graph) cudaGraphDestroy(graph);
     } else {
       cudaGetLastError();
     }
   }
-  if (!graphed) {
-    for (int j = 1; j <= n_steps; ++j)
-      TRY(decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs));
+  ctx->prof_recs.clear();
+  ctx->prof_pool_used = 0;
+  int rc_steps = ECHO_OK;
+  for (int j = 1; j <= n_steps && rc_steps == ECHO_OK; ++j) {
+    const bool sampled = ctx->prof_every > 0 && (j % ctx->prof_every == 0);
+    if (exec && !sampled) {
+      cudaError_t le = cudaGraphLaunch(exec, ctx->stream);
+      if (le != cudaSuccess) rc_steps = fail_cuda(ctx, le, "cudaGraphLaunch");
+      ctx->launches += per_step;
+    } else {
+      ctx->prof_now = sampled;
+      ctx->prof_step = j;
+      rc_steps = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs);
+      ctx->prof_now = false;
+    }
   }
+  if (exec) cudaGraphExecDestroy(exec);      // executions already enqueued keep their resources
+  if (graph) cudaGraphDestroy(graph);
+  if (rc_steps != ECHO_OK) return rc_steps;
   CK(cudaEventRecord(wp->last_use, ctx->stream));
   wp->used = true;
 
@@ -667,6 +713,7 @@ int echo_destroy(echo_ctx *ctx) {
   if (ctx->plan_done) cudaEventDestroy(ctx->plan_done);
   if (ctx->all_done) cudaEventDestroy(ctx->all_done);
   if (ctx->h_tables) cudaFreeHost(ctx->h_tables);
+  for (cudaEvent_t e : ctx->prof_pool) cudaEventDestroy(e);
   delete ctx;
   return ECHO_OK;
 }
@@ -859,6 +906,36 @@ int echo_gemm_bf16(const void *X, const void *W, float *Y, int32_t M, int32_t N,
   GemmArgs a{&tmW, &tmX, Y, N, M, N, K, bnb, EPI_STORE, nullptr};
   cudaError_t e = gemm_tc_launch(a, s);
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+int echo_profile_config(echo_ctx *ctx, int32_t every_n_steps) {
+  if (!ctx || every_n_steps < 0) return ECHO_ERR_INVALID;
+  ctx->prof_every = every_n_steps;
+  return ECHO_OK;
+}
+
+int echo_profile_read(echo_ctx *ctx, int32_t *steps, float *ms, int32_t capacity, int32_t *n_out) {
+  if (!ctx || !n_out) return ECHO_ERR_INVALID;
+  DeviceGuard guard(ctx->device);
+  CK(cudaStreamSynchronize(ctx->stream));
+  std::vector<int> order;
+  for (const auto &r : ctx->prof_recs)
+    if (order.empty() || order.back() != r.step) order.push_back(r.step);
+  *n_out = static_cast<int32_t>(order.size());
+  if (!steps || !ms) return ECHO_OK;
+  if (capacity < *n_out) return ECHO_ERR_INVALID;
+  for (size_t i = 0; i < order.size(); ++i) {
+    steps[i] = order[i];
+    for (int c = 0; c < PROF_NCLS; ++c) ms[i * PROF_NCLS + c] = 0.f;
+  }
+  size_t idx = 0;
+  for (const auto &r : ctx->prof_recs) {
+    while (order[idx] != r.step) ++idx;
+    float t = 0.f;
+    CK(cudaEventElapsedTime(&t, r.a, r.b));
+    ms[idx * PROF_NCLS + r.cls] += t;
+  }
+  return ECHO_OK;
 }
 
 const char *echo_strerror(int code) {
