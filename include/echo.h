@@ -209,12 +209,21 @@ int echo_sample(const float *logits, int32_t R, int32_t V, int32_t rows_per_logi
                 const int32_t *forced, int32_t *out_tokens, float *out_logprobs,
                 void *cuda_stream);
 
-/* Dense projection alone: Y[M][N] (dev fp32) = X[M][K] (dev bf16) * W[N][K]^T
- * (dev bf16) with fp32 accumulation on the tcgen05 tensor cores.  K must be a
- * multiple of 64 and N a multiple of 128; M in [1, 4096].  All pointers 256-byte
- * aligned.  `impl`: 0 = tensor-core kernel, 1 = plain SIMT reference kernel. */
-int echo_gemm_bf16(const void *X, const void *W, float *Y, int32_t M, int32_t N, int32_t K,
-                   int32_t impl, void *cuda_stream);
+/* Dense projection alone, on the tcgen05 tensor cores with fp32 accumulation:
+ *   epilogue 0:  Y[M][N] (dev fp32)  = X[M][K] (dev bf16) * W[N][K]^T (dev bf16)
+ *   epilogue 1:  Y[M][N] (dev fp32) += X * W^T                        (residual add)
+ *   epilogue 2:  Y[M][N] (dev bf16)  = silu(X * Wg^T) * (X * Wu^T), W = [Wg; Wu] of shape [2N][K]
+ * K must be a multiple of 8, M in [1, 4096]; all pointers 256-byte aligned.  The kernel splits
+ * tiles along K across CTAs and needs scratch memory for the partial sums: `workspace` is
+ * device memory of at least echo_gemm_workspace_bytes(M) bytes, owned by the caller, used only
+ * during the call's kernels.  `impl`: 0 = tensor-core kernel (cluster split-K for few output
+ * tiles, persistent stream-K otherwise), 2 = always the persistent stream-K kernel, 100 + s =
+ * cluster split-K by s in [1, 8], 1 = plain SIMT reference kernel (epilogues 0 and 1 only;
+ * needs no workspace). */
+size_t echo_gemm_workspace_bytes(int32_t M);
+int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, int32_t K,
+                   int32_t epilogue, int32_t impl, void *workspace, size_t workspace_bytes,
+                   void *cuda_stream);
 
 const char *echo_strerror(int code);
 const char *echo_last_error(echo_ctx *ctx);   /* text of the last ECHO_ERR_CUDA on this context */

@@ -80,7 +80,9 @@ def _load() -> C.CDLL:
     lib.echo_debug_page_table.argtypes = [vp, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32)]
     lib.echo_debug_noise.argtypes = [u64, u32, u32, u32, u32, vp, vp, vp]
     lib.echo_sample.argtypes = [vp, i32, i32, i32, vp, u32, f32, u64, vp, vp, vp, vp]
-    lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]
+    lib.echo_gemm_workspace_bytes.restype = C.c_size_t
+    lib.echo_gemm_workspace_bytes.argtypes = [i32]
     lib.echo_strerror.restype = C.c_char_p
     lib.echo_strerror.argtypes = [C.c_int]
     lib.echo_last_error.restype = C.c_char_p
@@ -98,7 +100,7 @@ lib = _load()
 EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy", "echo_wait_policy",
             "echo_rollout", "echo_rollout_forced", "echo_rollout_host", "echo_group_advantage", "echo_sync",
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
-            "echo_strerror", "echo_last_error"]
+            "echo_gemm_workspace_bytes", "echo_strerror", "echo_last_error"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -295,12 +297,20 @@ def echo_sample(logits: torch.Tensor, rows: int, rows_per_logit_row: int, j: int
     return tok, lp
 
 
-def echo_gemm_bf16(X: torch.Tensor, W: torch.Tensor, impl: int = 0) -> torch.Tensor:
+def echo_gemm_bf16(X: torch.Tensor, W: torch.Tensor, impl: int = 0, epilogue: int = 0,
+                   Y: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """epilogue 0: Y = X W^T (fp32); 1: Y += X W^T (fp32, Y given); 2: W = [Wg; Wu], Y = silu(X Wg^T) * (X Wu^T)
+    (bf16)."""
     assert X.is_cuda and W.is_cuda and X.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
     assert X.is_contiguous() and W.is_contiguous() and X.shape[1] == W.shape[1]
     M, K = X.shape
-    N = W.shape[0]
-    Y = torch.empty((M, N), dtype=torch.float32, device=X.device)
+    N = W.shape[0] // 2 if epilogue == 2 else W.shape[0]
+    if Y is None:
+        Y = torch.zeros((M, N), dtype=torch.bfloat16 if epilogue == 2 else torch.float32, device=X.device)
     with torch.cuda.device(X.device):
-        _check(lib.echo_gemm_bf16(X.data_ptr(), W.data_ptr(), Y.data_ptr(), M, N, K, impl, _stream_ptr(None)))
+        nws = int(lib.echo_gemm_workspace_bytes(M)) if impl != 1 else 256
+        ws = torch.empty(nws, dtype=torch.uint8, device=X.device)
+        _check(lib.echo_gemm_bf16(X.data_ptr(), W.data_ptr(), Y.data_ptr(), M, N, K, epilogue, impl,
+                                  ws.data_ptr(), nws, _stream_ptr(None)))
+        torch.cuda.current_stream().synchronize()      # the workspace must outlive the kernel
     return Y

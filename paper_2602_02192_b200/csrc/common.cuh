@@ -21,6 +21,7 @@ enum : int {
 constexpr int kGemmTileN = 128;      // output features per CTA (UMMA M)
 constexpr int kGemmTileK = 64;       // bf16 elements per pipeline stage (one 128-byte swizzle row)
 constexpr int kMaxBatchTile = 256;   // rows of activations per MMA (UMMA N)
+constexpr int kGemmMaxUnits = 8192;  // output tiles per launch the tile counters cover
 
 // ---- dense projections (gemm.cu) ------------------------------------------
 // Y[m][n] (+)= sum_k X[m][k] * W[n][k], bf16 inputs, fp32 accumulation.
@@ -28,7 +29,8 @@ constexpr int kMaxBatchTile = 256;   // rows of activations per MMA (UMMA N)
 enum GemmEpilogue : int {
   EPI_STORE = 0,      // Y = acc
   EPI_ACCUM = 1,      // Y += acc              (residual add)
-  EPI_SWIGLU = 2,     // two W row blocks (gate at n, up at n + N): Yb = bf16(silu(g) * u)
+  EPI_SWIGLU = 2,     // W holds gate rows [0, N) and up rows [N, 2N): Y = bf16(silu(g) * u);
+                      // its tensor map must use a 64-row box (64 gate + 64 up rows per tile)
 };
 
 struct GemmArgs {
@@ -40,7 +42,12 @@ struct GemmArgs {
   int bnb;            // activation rows per CTA: 32, 64, 128 or 256
   int epilogue;
   int *status;
+  float *workspace;   // gemm_workspace_bytes(bnb) bytes: partial accumulators of split tiles
+  int *counters;      // kGemmMaxUnits ints, zero before the first launch (the kernel re-zeroes them)
+  int max_ctas;       // 0 = one CTA per SM
+  int force_split;    // 0 = choose; k > 0 = cluster split-K by k; -1 = always the persistent stream-K kernel
 };
+size_t gemm_workspace_bytes(int bnb);
 cudaError_t gemm_tc_launch(const GemmArgs &a, cudaStream_t stream);
 cudaError_t gemm_tc_configure();     // sets the dynamic shared memory attribute once per device
 cudaError_t gemm_simt_launch(const __nv_bfloat16 *X, const __nv_bfloat16 *W, float *Y, int ldY,

@@ -5,269 +5,341 @@
 // Operand roles are swapped with respect to the usual GEMM picture: the WEIGHT tile
 // (128 output features x 64 k) is the UMMA "A" operand and fills the 128 TMEM lanes,
 // the ACTIVATION tile (bnb rows x 64 k) is the "B" operand and fills bnb TMEM columns.
-// A CTA therefore streams each weight byte from HBM exactly once for up to 256
-// activation rows, which is what a decode step (a few hundred rows against gigabytes
-// of weights) needs; the activation tile is re-read from L2.
+// Each weight byte is therefore streamed from HBM exactly once for up to 256 activation
+// rows, which is what a decode step (a few hundred rows against gigabytes of weights)
+// needs; the activation tile is re-read from L2.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
-// warps 2..5 = epilogue (each reads the TMEM lane quarter its warp id selects).
+// The kernel is persistent (one CTA per SM) and splits the work stream-K fashion: the
+// list of (output tile, k-block) pairs is cut into equal contiguous ranges, one per CTA,
+// so that every SM streams the same number of weight bytes whatever N and K are.  A CTA
+// whose range covers only part of a tile's k-blocks writes its partial accumulator to a
+// per-CTA workspace slot; the CTA that finishes a tile last (an atomic counter per tile,
+// no waiting) sums the partials in k order and applies the epilogue, so results do not
+// depend on timing.
+//
+// A CTA's output tile is two 128-lane accumulators (256 features) against one activation
+// tile, so that the activation bytes an SM pulls from L2 do not exceed the weight bytes it
+// pulls from HBM (an SM ingests roughly 64 bytes per clock in total).
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..17 =
+// epilogue (each reads the TMEM lane quarter its warp id selects; the four warps of a quarter
+// split the columns - a warp keeps only one global store in flight at a time, so the store
+// rate of the epilogue grows with the number of warps).
 // Every mbarrier wait is bounded; on expiry the kernel records STATUS_WAIT_TIMEOUT,
 // drains, frees its tensor memory and returns.
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace echo {
 
+using namespace ptx;
+
 namespace {
 
-constexpr int kThreads = 192;
-constexpr uint32_t kSpinLimit = 1u << 26;
-constexpr uint64_t kWaitLimitNs = 1000000000ull;
+constexpr int kEpiGroups = 4;         // epilogue warps per TMEM lane quarter (they split the columns)
+constexpr int kEpiWarps = 4 * kEpiGroups;
+constexpr int kEpiThreads = 128 * kEpiGroups;
+constexpr int kThreads = 64 + kEpiThreads;
+constexpr int kAcc = 2;              // accumulators (128-lane weight blocks) per output tile
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait (about one second of wall time).  Returns false if the limit ran out or
-// another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 63u) {
-      if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) break;
-    }
-  }
-  *abort_flag = 1;
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(const CUtensorMap *map, uint64_t *bar, void *dst, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
-      : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t *bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                            uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16)
-// laid out by TMA with the 128-byte swizzle: groups of 8 rows are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);        // start address / 16
-  d |= static_cast<uint64_t>(1) << 16;                         // leading byte offset (unused with swizzle)
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;                 // stride between 8-row groups / 16
-  d |= static_cast<uint64_t>(1) << 46;                         // descriptor version of this architecture
-  d |= static_cast<uint64_t>(2) << 61;                         // 128-byte swizzle
-  return d;
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = bnb.
-__host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (8u << 24);
-}
-
-template <int BNB, int NACC>
+template <int BNB>
 struct GemmSmem {
-  static constexpr int kWBytes = kGemmTileN * kGemmTileK * 2;      // 16 KiB per weight block
+  static constexpr int kWBlock = kGemmTileN * kGemmTileK * 2;      // 16 KiB per weight block
+  static constexpr int kWBytes = kAcc * kWBlock;
   static constexpr int kXBytes = BNB * kGemmTileK * 2;
-  static constexpr int kStageBytes = NACC * kWBytes + kXBytes;
-  static constexpr int kBudget = 220 * 1024;
+  static constexpr int kStageBytes = kWBytes + kXBytes;
+  static constexpr int kBudget = 200 * 1024;
   static constexpr int kStagesRaw = kBudget / kStageBytes;
   static constexpr int kStages = kStagesRaw > 8 ? 8 : kStagesRaw;
-  static constexpr int kBarBytes = 256;
+  static constexpr int kBarBytes = 1024;
   static constexpr int kTotal = kStages * kStageBytes + kBarBytes + 1024;   // + alignment slack
-  static constexpr int kTmemCols = (BNB * NACC) < 32 ? 32 : BNB * NACC;      // power of two by construction
+  static constexpr int kTmemCols = kAcc * BNB < 32 ? 32 : kAcc * BNB;
 };
 
 __device__ __forceinline__ float silu_f(float a) { return a / (1.0f + __expf(-a)); }
+// store, or add in memory without reading back (one add per element per launch: order-free)
+__device__ __forceinline__ void put(float *y, float v, int epilogue) {
+  if (epilogue == EPI_ACCUM) atomicAdd(y, v);
+  else *y = v;
+}
 
-template <int BNB, int NACC>
+// Stream-K split of `total` k-blocks over `n_cta` CTAs: CTA c owns [beg(c), beg(c+1)).
+struct Split {
+  int total, n_cta, q, r;
+  __host__ __device__ int beg(int c) const { return c * q + (c < r ? c : r); }
+  __host__ __device__ int cta_of(int g) const {
+    const int edge = r * (q + 1);
+    return g < edge ? g / (q + 1) : r + (g - edge) / q;
+  }
+};
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+
+// Loads of one k-block: kAcc weight blocks (each 128 rows, or 64 gate + 64 up rows) and the
+// activation tile.  `wait_dep` defers the activation load until the producing kernel is done.
+template <int BNB>
+__device__ __forceinline__ void load_stage(const CUtensorMap *tmW, const CUtensorMap *tmX, uint64_t *bar,
+                                           uint8_t *stage, int kb, int nt, int m0, int N, bool gu) {
+  using S = GemmSmem<BNB>;
+  mbar_expect_tx(bar, S::kStageBytes);
+#pragma unroll
+  for (int a = 0; a < kAcc; ++a) {
+    uint8_t *dst = stage + a * S::kWBlock;
+    if (gu) {
+      const int f0 = (nt * kAcc + a) * 64;
+      tma_load_2d(tmW, bar, dst, kb * kGemmTileK, f0);
+      tma_load_2d(tmW, bar, dst + S::kWBlock / 2, kb * kGemmTileK, N + f0);
+    } else {
+      tma_load_2d(tmW, bar, dst, kb * kGemmTileK, (nt * kAcc + a) * kGemmTileN);
+    }
+  }
+  tma_load_2d(tmX, bar, stage + S::kWBytes, kb * kGemmTileK, m0);
+}
+
+template <int BNB>
+__device__ __forceinline__ void mma_stage(uint32_t tmem_base, uint32_t stage_addr, bool first) {
+  using S = GemmSmem<BNB>;
+  constexpr uint32_t idesc = instr_desc_bf16(BNB);
+  const uint64_t xdesc = smem_desc_sw128(stage_addr + S::kWBytes);
+#pragma unroll
+  for (int a = 0; a < kAcc; ++a) {
+    const uint64_t wdesc = smem_desc_sw128(stage_addr + a * S::kWBlock);
+#pragma unroll
+    for (int k = 0; k < kGemmTileK / 16; ++k) {
+      // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte units
+      tc_mma_bf16(tmem_base + a * BNB, wdesc + 2 * k, xdesc + 2 * k, idesc, (!first || k > 0) ? 1u : 0u);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Persistent stream-K kernel (many output tiles: the lm_head).
+// ---------------------------------------------------------------------------------------
+template <int BNB>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-               void *Yv, int ldY, int M, int N, int K, int epilogue, int *status) {
-  using S = GemmSmem<BNB, NACC>;
+gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, void *Yv,
+                    int ldY, int M, int N, int K, int epilogue, int n_tiles, float *workspace, int *counters,
+                    int *status) {
+  using S = GemmSmem<BNB>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + S::kStages * S::kStageBytes);
   uint64_t *empty_bar = full_bar + S::kStages;
-  uint64_t *acc_bar = empty_bar + S::kStages;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_bar + 1);
+  uint64_t *acc_full = empty_bar + S::kStages;
+  uint64_t *acc_empty = acc_full + 1;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 1);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  volatile int *last_flag = abort_flag + 1;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * kGemmTileN;
-  const int m0 = blockIdx.y * BNB;
-  const int num_kb = (K + kGemmTileK - 1) / kGemmTileK;
+  const bool gu = epilogue == EPI_SWIGLU;
+  const int KB = (K + kGemmTileK - 1) / kGemmTileK;
+  const int m_tiles = (M + BNB - 1) / BNB;
+  Split sp;
+  sp.total = n_tiles * m_tiles * KB;
+  sp.n_cta = gridDim.x;
+  sp.q = sp.total / sp.n_cta;
+  sp.r = sp.total % sp.n_cta;
+  const int cta = blockIdx.x;
+  const int g_beg = sp.beg(cta), g_end = sp.beg(cta + 1);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S::kStages; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(acc_bar, 1);
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, kEpiThreads);
     *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    *last_flag = 0;
+    mbar_fence_init();
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(static_cast<uint32_t>(S::kTmemCols))
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
+  if (warp == 1) tc_alloc(tmem_slot, S::kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();          // inputs produced by the preceding kernel are complete from here on
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      int issued = 0;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % S::kStages;
-        const uint32_t ph = (kb / S::kStages) & 1;
-        if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag)) break;
-        uint8_t *stage = smem + s * S::kStageBytes;
-        mbar_expect_tx(&full_bar[s], S::kStageBytes);
-#pragma unroll
-        for (int a = 0; a < NACC; ++a)
-          tma_load_2d(&tmW, &full_bar[s], stage + a * S::kWBytes, kb * kGemmTileK, n0 + a * N);
-        tma_load_2d(&tmX, &full_bar[s], stage + NACC * S::kWBytes, kb * kGemmTileK, m0);
-        issued = kb + 1;
-      }
-      if (*abort_flag) {
-        // let copies already in flight land before the CTA's shared memory is released
-        for (int kb = issued > S::kStages ? issued - S::kStages : 0; kb < issued; ++kb) {
-          const int s = kb % S::kStages;
-          const uint32_t ph = (kb / S::kStages) & 1;
-          for (uint32_t i = 0; i < (1u << 16); ++i)
-            if (mbar_try_wait(&full_bar[s], ph)) break;
+      int it = 0;
+      bool ok = true;
+      for (int g = g_beg; g < g_end && ok;) {
+        const int unit = g / KB, kb0 = g % KB;
+        const int len = min(KB - kb0, g_end - g);
+        const int nt = unit % n_tiles, mt = unit / n_tiles;
+        for (int kb = kb0; kb < kb0 + len; ++kb, ++it) {
+          const int s = it % S::kStages;
+          ok = mbar_wait(&empty_bar[s], ((it / S::kStages) & 1) ^ 1u, abort_flag);
+          if (!ok) break;
+          load_stage<BNB>(&tmW, &tmX, &full_bar[s], smem + s * S::kStageBytes, kb, nt, mt * BNB, N, gu);
         }
+        g += len;
+      }
+      if (!ok) {
+        // let copies already in flight land before the CTA's shared memory is released
+        for (int k = it > S::kStages ? it - S::kStages : 0; k < it; ++k)
+          mbar_drain(&full_bar[k % S::kStages], (k / S::kStages) & 1);
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc_bf16(BNB);
+      int it = 0, seg = 0;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % S::kStages;
-        const uint32_t ph = (kb / S::kStages) & 1;
-        ok = mbar_wait(&full_bar[s], ph, abort_flag);
+      for (int g = g_beg; g < g_end && ok; ++seg) {
+        const int kb0 = g % KB;
+        const int len = min(KB - kb0, g_end - g);
+        ok = mbar_wait(acc_empty, (seg & 1) ^ 1u, abort_flag);     // epilogue has drained the accumulators
         if (!ok) break;
         tc_fence_after();
-        const uint32_t stage = smem_u32(smem + s * S::kStageBytes);
-        const uint64_t xdesc = smem_desc_sw128(stage + NACC * S::kWBytes);
-#pragma unroll
-        for (int a = 0; a < NACC; ++a) {
-          const uint64_t wdesc = smem_desc_sw128(stage + a * S::kWBytes);
-#pragma unroll
-          for (int k = 0; k < kGemmTileK / 16; ++k) {
-            // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte units
-            tc_mma_bf16(tmem_base + a * BNB, wdesc + 2 * k, xdesc + 2 * k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-          }
+        for (int kb = 0; kb < len; ++kb, ++it) {
+          const int s = it % S::kStages;
+          ok = mbar_wait(&full_bar[s], (it / S::kStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          mma_stage<BNB>(tmem_base, smem_u32(smem + s * S::kStageBytes), kb == 0);
+          tc_commit(&empty_bar[s]);      // frees the stage once these MMAs have read it
         }
-        tc_commit(&empty_bar[s]);      // frees the stage once these MMAs have read it
+        if (ok) tc_commit(acc_full);
+        g += len;
       }
-      if (ok) tc_commit(acc_bar);      // accumulator complete
     }
   } else {
-    // ---------------- epilogue: TMEM -> registers -> global ----------------
-    const int quarter = warp & 3;                      // TMEM lanes 32*quarter .. +31
-    const int n = n0 + quarter * 32 + lane;            // output feature of this thread
-    const bool got = mbar_wait(acc_bar, 0, abort_flag);
-    tc_fence_after();
-    if (got) {
+    // ---------------- epilogue: TMEM -> registers -> global / workspace ----------------
+    const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31
+    const int row = quarter * 32 + lane;                // accumulator lane
+    const int et = (threadIdx.x - 64) & 127;            // position within the 128-lane tile
+    const int grp = (warp - 2) >> 2;                    // which share of the columns this warp takes
+    const int first_unit = g_beg / KB;
+    const size_t acc_elems = static_cast<size_t>(kGemmTileN) * BNB;
+    const size_t slot_elems = kAcc * acc_elems;
+    int seg = 0;
+    bool ok = true;
+    for (int g = g_beg; g < g_end && ok; ++seg) {
+      const int unit = g / KB, kb0 = g % KB;
+      const int len = min(KB - kb0, g_end - g);
+      g += len;
+      const int nt = unit % n_tiles, mt = unit / n_tiles;
+      const int m0 = mt * BNB;
+      const int cols = min(BNB, M - m0);
+      ok = mbar_wait(acc_full, seg & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
       const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+      const bool whole = kb0 == 0 && len == KB;
+      if (whole && !gu) {
+        float *Y = reinterpret_cast<float *>(Yv);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BNB; c0 += 32) {
-        if (m0 + c0 >= M) break;                       // warp-uniform
-        uint32_t r[32];
-        tc_ld32(lane_addr + c0, r);
-        if (NACC == 2) {
-          uint32_t u[32];
-          tc_ld32(lane_addr + BNB + c0, u);
-          tc_wait_ld();
-          if (n < N) {
-            __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(Yv);
+        for (int a = 0; a < kAcc; ++a) {
+          const int n = (nt * kAcc + a) * kGemmTileN + row;
+#pragma unroll 1
+          for (int c0 = 32 * grp; c0 < cols; c0 += 32 * kEpiGroups) {
+            uint32_t r[32];
+            tc_ld32(lane_addr + a * BNB + c0, r);
+            tc_wait_ld();
+            if (n < N) {
+              float *y0 = Y + static_cast<size_t>(m0 + c0) * ldY + n;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const int m = m0 + c0 + c;
-              if (m < M)
-                Y[static_cast<size_t>(m) * ldY + n] =
-                    __float2bfloat16(silu_f(__uint_as_float(r[c])) * __uint_as_float(u[c]));
+              for (int c = 0; c < 32; ++c)
+                if (c0 + c < cols) put(y0 + static_cast<size_t>(c) * ldY, __uint_as_float(r[c]), epilogue);
             }
           }
-        } else {
+        }
+        tc_fence_before();
+        mbar_arrive(acc_empty);
+        continue;
+      }
+      // partial (or gate/up) accumulators -> this CTA's workspace slot, layout [acc][column][lane]
+      const int slot = whole ? 2 : (unit == first_unit ? 0 : 1);
+      float *ws = workspace + (static_cast<size_t>(cta) * 3 + slot) * slot_elems;
+#pragma unroll 1
+      for (int a = 0; a < kAcc; ++a) {
+#pragma unroll 1
+        for (int c0 = 32 * grp; c0 < cols; c0 += 32 * kEpiGroups) {
+          uint32_t r[32];
+          tc_ld32(lane_addr + a * BNB + c0, r);
           tc_wait_ld();
-          if (n < N) {
-            float *Y = reinterpret_cast<float *>(Yv);
-            if (epilogue == EPI_ACCUM) {
 #pragma unroll
-              for (int c = 0; c < 32; ++c) {
-                const int m = m0 + c0 + c;
-                if (m < M) Y[static_cast<size_t>(m) * ldY + n] += __uint_as_float(r[c]);
+          for (int c = 0; c < 32; ++c)
+            __stcg(ws + a * acc_elems + static_cast<size_t>(c0 + c) * kGemmTileN + row, __uint_as_float(r[c]));
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(acc_empty);
+      // count this segment; the CTA that completes the tile reduces it
+      const int c_first = sp.cta_of(unit * KB), c_last = sp.cta_of(unit * KB + KB - 1);
+      __threadfence();
+      epi_bar();
+      if (threadIdx.x == 64) {
+        const int old = atomicAdd(&counters[unit], 1);
+        *last_flag = (old == c_last - c_first) ? 1 : 0;
+      }
+      epi_bar();
+      const bool last = *last_flag != 0;
+      if (last) {
+        __threadfence();
+#pragma unroll 1
+        for (int a = 0; a < kAcc; ++a) {
+          if (gu) {
+            // thread -> feature f of the 64-wide block and every second column of a 32-column chunk
+            __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(Yv);
+            const int f = et & 63, half = et >> 6;
+            const int n = (nt * kAcc + a) * 64 + f;
+#pragma unroll 1
+            for (int c0 = 32 * grp; c0 < cols; c0 += 32 * kEpiGroups) {
+              float gs[16], us[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i) gs[i] = us[i] = 0.f;
+              for (int cc = c_first; cc <= c_last; ++cc) {
+                const int sl = c_first == c_last ? 2 : (sp.beg(cc) / KB == unit ? 0 : 1);
+                const float *p = workspace + (static_cast<size_t>(cc) * 3 + sl) * slot_elems + a * acc_elems +
+                                 static_cast<size_t>(c0 + half) * kGemmTileN + f;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  gs[i] += __ldcg(p + static_cast<size_t>(2 * i) * kGemmTileN);
+                  us[i] += __ldcg(p + static_cast<size_t>(2 * i) * kGemmTileN + 64);
+                }
               }
-            } else {
+              if (n < N) {
 #pragma unroll
-              for (int c = 0; c < 32; ++c) {
-                const int m = m0 + c0 + c;
-                if (m < M) Y[static_cast<size_t>(m) * ldY + n] = __uint_as_float(r[c]);
+                for (int i = 0; i < 16; ++i) {
+                  const int c = c0 + half + 2 * i;
+                  if (c < cols) Y[static_cast<size_t>(m0 + c) * ldY + n] = __float2bfloat16(silu_f(gs[i]) * us[i]);
+                }
+              }
+            }
+          } else {
+            float *Y = reinterpret_cast<float *>(Yv);
+            const int n = (nt * kAcc + a) * kGemmTileN + et;
+#pragma unroll 1
+            for (int c0 = 32 * grp; c0 < cols; c0 += 32 * kEpiGroups) {
+              float acc[32];
+#pragma unroll
+              for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+              for (int cc = c_first; cc <= c_last; ++cc) {
+                const int sl = sp.beg(cc) / KB == unit ? 0 : 1;
+                const float *p = workspace + (static_cast<size_t>(cc) * 3 + sl) * slot_elems + a * acc_elems +
+                                 static_cast<size_t>(c0) * kGemmTileN + et;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) acc[i] += __ldcg(p + static_cast<size_t>(i) * kGemmTileN);
+              }
+              if (n < N) {
+                float *y0 = Y + static_cast<size_t>(m0 + c0) * ldY + n;
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (c0 + i < cols) put(y0 + static_cast<size_t>(i) * ldY, acc[i], epilogue);
               }
             }
           }
         }
+        if (threadIdx.x == 64) counters[unit] = 0;   // ready for the next launch
       }
+      epi_bar();                                      // last_flag is reused by the next segment
     }
   }
 
@@ -275,26 +347,312 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                 "r"(static_cast<uint32_t>(S::kTmemCols))
-                 : "memory");
+    tc_dealloc(tmem_base, S::kTmemCols);
   }
   if (threadIdx.x == 0 && *abort_flag && status) atomicExch(status, STATUS_WAIT_TIMEOUT);
 }
 
-template <int BNB, int NACC>
+// ---------------------------------------------------------------------------------------
+// Split-K over a thread-block cluster (few output tiles: the per-layer projections).  The S
+// CTAs of a cluster share one output tile and each streams 1/S of its k-blocks; the partial
+// accumulators are then summed through distributed shared memory in rank order (so the
+// result does not depend on timing), each CTA reducing and writing a 1/S slice of the tile's
+// columns.  No global scratch, no atomics between CTAs, no waiting other than the hardware
+// cluster barrier.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t cta_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(cta_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_dsmem_v4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 ld_dsmem_v2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+
+template <int BNB>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+                    const __grid_constant__ CUtensorMap tmY, int M, int N, int K, int epilogue, int S_split,
+                    int *status) {
+  using S = GemmSmem<BNB>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + S::kStages * S::kStageBytes);
+  uint64_t *empty_bar = full_bar + S::kStages;
+  uint64_t *acc_full = empty_bar + S::kStages;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  float *part = reinterpret_cast<float *>(smem);      // [column][lane], reuses the pipeline stages
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const bool gu = epilogue == EPI_SWIGLU;
+  const int KB = (K + kGemmTileK - 1) / kGemmTileK;
+  const int nt = blockIdx.x / S_split;
+  const int rank = blockIdx.x % S_split;              // == rank in the cluster (cluster spans x only)
+  const int m0 = blockIdx.y * BNB;
+  const int kq = KB / S_split, kr = KB % S_split;
+  const int kb_beg = rank * kq + min(rank, kr);
+  const int kb_len = kq + (rank < kr ? 1 : 0);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S::kStages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) tc_alloc(tmem_slot, S::kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int kb = kb_beg; kb < kb_beg + kb_len; ++kb, ++it) {
+        const int s = it % S::kStages;
+        ok = mbar_wait(&empty_bar[s], ((it / S::kStages) & 1) ^ 1u, abort_flag);
+        if (!ok) break;
+        load_stage<BNB>(&tmW, &tmX, &full_bar[s], smem + s * S::kStageBytes, kb, nt, m0, N, gu);
+      }
+      if (!ok) {
+        for (int k = it > S::kStages ? it - S::kStages : 0; k < it; ++k)
+          mbar_drain(&full_bar[k % S::kStages], (k / S::kStages) & 1);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      bool ok = true;
+      for (int it = 0; it < kb_len; ++it) {
+        const int s = it % S::kStages;
+        ok = mbar_wait(&full_bar[s], (it / S::kStages) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        mma_stage<BNB>(tmem_base, smem_u32(smem + s * S::kStageBytes), it == 0);
+        tc_commit(&empty_bar[s]);
+      }
+      if (ok) tc_commit(acc_full);
+    }
+  }
+
+  // ---- epilogue.  Per accumulator: TMEM -> shared memory ([column][lane] fp32, reusing the
+  // pipeline stages, which no MMA reads any more once acc_full has fired); with a split, the
+  // cluster's partials are summed through distributed shared memory in rank order, each CTA
+  // taking a slice of columns; the finished tile leaves through TMA stores (or TMA reduce-adds
+  // for the residual epilogue), which keep the few epilogue warps off the global store path.
+  const bool plain = S_split == 1 && !gu;
+  const int cols = min(BNB, M - m0);
+  const int quarter = warp & 3;
+  const int row = quarter * 32 + lane;
+  const int grp = (warp - 2) >> 2;
+  const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+  uint8_t *out_stage = smem + static_cast<size_t>(kGemmTileN) * BNB * 4;     // behind the partial
+  const int units = (cols + 7) / 8;                                           // slices in 8-column units
+  const int c_lo = 8 * (rank * units / S_split), c_hi = 8 * ((rank + 1) * units / S_split);
+  const uint32_t part_addr = smem_u32(part);
+  bool got = false;
+  if (warp >= 2) {
+    got = mbar_wait(acc_full, 0, abort_flag);
+    tc_fence_after();
+  }
+#pragma unroll 1
+  for (int a = 0; a < kAcc; ++a) {
+    if (warp >= 2) {
+      if (a > 0) {
+        if (lane == 0) bulk_wait_read();                  // TMA has read the previous accumulator's staging
+        epi_bar();
+      }
+      if (got) {
+#pragma unroll 1
+        for (int c0 = 32 * grp; c0 < cols; c0 += 32 * kEpiGroups) {
+          uint32_t r[32];
+          tc_ld32(lane_addr + a * BNB + c0, r);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) part[(c0 + c) * kGemmTileN + row] = __uint_as_float(r[c]);
+        }
+      }
+    }
+    __syncwarp();
+    if (!plain) {
+      cluster_sync_all();                                 // all partials of this accumulator are in place
+      if (warp >= 2 && got) {
+        // one warp per column: a lane owns 4 consecutive features (2 gate + 2 up for SwiGLU), so a
+        // warp reads a whole 512-byte row of every rank's partial with one vector load per rank;
+        // four columns are in flight at a time to cover the remote shared-memory latency
+        const int ew = warp - 2;
+#pragma unroll 1
+        for (int cb = c_lo + ew; cb < c_hi; cb += 4 * kEpiWarps) {
+          if (gu) {
+            float2 gs[4], us[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) gs[j] = us[j] = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+              if (r < S_split) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int c = cb + j * kEpiWarps;
+                  if (c < c_hi) {
+                    const uint32_t base = dsmem_addr(part_addr + static_cast<uint32_t>(c * kGemmTileN + 2 * lane) * 4u, r);
+                    const float2 g = ld_dsmem_v2(base), u = ld_dsmem_v2(base + 64u * 4u);
+                    gs[j].x += g.x; gs[j].y += g.y; us[j].x += u.x; us[j].y += u.y;
+                  }
+                }
+              }
+            }
+            __nv_bfloat162 *o = reinterpret_cast<__nv_bfloat162 *>(out_stage);   // [column - c_lo][64]
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int c = cb + j * kEpiWarps;
+              if (c < c_hi)
+                o[(c - c_lo) * 32 + lane] = __floats2bfloat162_rn(silu_f(gs[j].x) * us[j].x, silu_f(gs[j].y) * us[j].y);
+            }
+          } else {
+            float4 acc[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+              if (r < S_split) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int c = cb + j * kEpiWarps;
+                  if (c < c_hi) {
+                    const float4 v = ld_dsmem_v4(
+                        dsmem_addr(part_addr + static_cast<uint32_t>(c * kGemmTileN + 4 * lane) * 4u, r));
+                    acc[j].x += v.x; acc[j].y += v.y; acc[j].z += v.z; acc[j].w += v.w;
+                  }
+                }
+              }
+            }
+            float4 *o = reinterpret_cast<float4 *>(out_stage);                      // [column - c_lo][128]
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int c = cb + j * kEpiWarps;
+              if (c < c_hi) o[(c - c_lo) * 32 + lane] = acc[j];
+            }
+          }
+        }
+      }
+    }
+    if (warp >= 2) {
+      fence_proxy_async();
+      epi_bar();
+      if (lane == 0 && got) {
+        // every epilogue warp issues a share of the 8-column boxes
+        const int x = (nt * kAcc + a) * (gu ? 64 : kGemmTileN);
+        const uint8_t *src = plain ? reinterpret_cast<const uint8_t *>(part) : out_stage;
+        const int row_bytes = gu ? 64 * 2 : kGemmTileN * 4;
+        const int lo = plain ? 0 : c_lo, hi = plain ? 8 * units : c_hi;
+        for (int c = lo + 8 * (warp - 2); c < hi; c += 8 * kEpiWarps) {
+          const uint8_t *p8 = src + static_cast<size_t>(c - lo) * row_bytes;
+          if (epilogue == EPI_ACCUM) tma_reduce_add_2d(&tmY, p8, x, m0 + c);
+          else tma_store_2d(&tmY, p8, x, m0 + c);
+        }
+        bulk_commit();
+      }
+    }
+    __syncwarp();
+    if (!plain) cluster_sync_all();                       // peers have finished reading this CTA's partial
+  }
+  if (warp >= 2 && lane == 0) bulk_wait_read();
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tc_dealloc(tmem_base, S::kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag && status) atomicExch(status, STATUS_WAIT_TIMEOUT);
+}
+
+int g_num_sms = 0;
+
+// Split factor for the cluster kernel: the smallest of 1, 2, 4 that puts a CTA on at least
+// ~40% of the SMs.  Measured on B200 at 256 activation rows: larger clusters lose more in the
+// cluster barriers and the remote shared-memory reduction than they gain in parallelism.
+int pick_split(int tiles, int KB, int sms) {
+  int s = 1;
+  while (s < 4 && tiles * s * 5 < sms * 2 && 2 * s <= KB) s *= 2;
+  return s;
+}
+
+int make_out_map(CUtensorMap *out, void *base, uint64_t rows, uint64_t cols, uint64_t ld, bool bf16);
+
+template <int BNB>
+cudaError_t launch_cluster_variant(const GemmArgs &a, int n_tiles, int m_tiles, int split, cudaStream_t stream) {
+  using S = GemmSmem<BNB>;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_tiles * split, m_tiles, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = S::kTotal;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = split;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  CUtensorMap tmY;
+  const bool gu = a.epilogue == EPI_SWIGLU;
+  if (make_out_map(&tmY, a.Y, a.M, a.N, a.ldY, gu) != 0) return cudaErrorInvalidValue;
+  return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<BNB>, *a.tmW, *a.tmX, tmY, a.M, a.N, a.K, a.epilogue, split,
+                            a.status);
+}
+
+template <int BNB>
 cudaError_t launch_variant(const GemmArgs &a, cudaStream_t stream) {
-  using S = GemmSmem<BNB, NACC>;
-  dim3 grid((a.N + kGemmTileN - 1) / kGemmTileN, (a.M + BNB - 1) / BNB, 1);
-  gemm_tc_kernel<BNB, NACC><<<grid, kThreads, S::kTotal, stream>>>(*a.tmW, *a.tmX, a.Y, a.ldY, a.M, a.N, a.K,
-                                                                  a.epilogue, a.status);
+  using S = GemmSmem<BNB>;
+  const bool gu = a.epilogue == EPI_SWIGLU;
+  const int per_tile = kAcc * (gu ? 64 : kGemmTileN);
+  const int n_tiles = (a.N + per_tile - 1) / per_tile;
+  const int m_tiles = (a.M + BNB - 1) / BNB;
+  const int KB = (a.K + kGemmTileK - 1) / kGemmTileK;
+  const long total = static_cast<long>(n_tiles) * m_tiles * KB;
+  if (n_tiles * m_tiles > kGemmMaxUnits || total > (1l << 30)) return cudaErrorInvalidValue;
+  int grid = g_num_sms > 0 ? g_num_sms : 148;
+  const bool out_ok = (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0 && (a.ldY * (gu ? 2 : 4)) % 16 == 0;
+  if (out_ok && a.force_split >= 0 && (a.force_split > 0 || n_tiles * m_tiles < 2 * grid)) {
+    const int split = a.force_split > 0 ? (a.force_split < KB ? a.force_split : KB)
+                                        : pick_split(n_tiles * m_tiles, KB, grid);
+    return launch_cluster_variant<BNB>(a, n_tiles, m_tiles, split, stream);
+  }
+  if (a.max_ctas > 0 && grid > a.max_ctas) grid = a.max_ctas;
+  if (grid > total) grid = static_cast<int>(total);
+  gemm_streamk_kernel<BNB><<<grid, kThreads, S::kTotal, stream>>>(*a.tmW, *a.tmX, a.Y, a.ldY, a.M, a.N, a.K,
+                                                                 a.epilogue, n_tiles, a.workspace, a.counters,
+                                                                 a.status);
   return cudaGetLastError();
 }
 
-template <int BNB, int NACC>
+template <int BNB>
 cudaError_t configure_variant() {
-  return cudaFuncSetAttribute(gemm_tc_kernel<BNB, NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              GemmSmem<BNB, NACC>::kTotal);
+  cudaError_t e = cudaFuncSetAttribute(gemm_cluster_kernel<BNB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       GemmSmem<BNB>::kTotal);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(gemm_streamk_kernel<BNB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              GemmSmem<BNB>::kTotal);
 }
 
 // ---- plain SIMT reference kernel (debugging aid; never on the default path) ----
@@ -336,6 +694,21 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// Output tile map: row-major [rows][cols] fp32 (box 128 x 8) or bf16 (box 64 x 8), no swizzle.
+int make_out_map(CUtensorMap *out, void *base, uint64_t rows, uint64_t cols, uint64_t ld, bool bf16) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return -1;
+  const uint64_t es = bf16 ? 2 : 4;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld * es};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(bf16 ? 64 : kGemmTileN), 8};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -3;
+}
+
 }  // namespace
 
 int make_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
@@ -353,26 +726,29 @@ int make_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t 
   return r == CUDA_SUCCESS ? 0 : -3;
 }
 
+size_t gemm_workspace_bytes(int bnb) {
+  const int ctas = g_num_sms > 0 ? g_num_sms : 148;
+  return static_cast<size_t>(ctas) * 3 * kAcc * kGemmTileN * bnb * sizeof(float);
+}
+
 cudaError_t gemm_tc_configure() {
   cudaError_t e;
-  if ((e = configure_variant<32, 1>()) != cudaSuccess) return e;
-  if ((e = configure_variant<64, 1>()) != cudaSuccess) return e;
-  if ((e = configure_variant<128, 1>()) != cudaSuccess) return e;
-  if ((e = configure_variant<256, 1>()) != cudaSuccess) return e;
-  if ((e = configure_variant<32, 2>()) != cudaSuccess) return e;
-  if ((e = configure_variant<64, 2>()) != cudaSuccess) return e;
-  if ((e = configure_variant<128, 2>()) != cudaSuccess) return e;
-  if ((e = configure_variant<256, 2>()) != cudaSuccess) return e;
+  int dev = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if ((e = configure_variant<32>()) != cudaSuccess) return e;
+  if ((e = configure_variant<64>()) != cudaSuccess) return e;
+  if ((e = configure_variant<128>()) != cudaSuccess) return e;
+  if ((e = configure_variant<256>()) != cudaSuccess) return e;
   return cudaSuccess;
 }
 
 cudaError_t gemm_tc_launch(const GemmArgs &a, cudaStream_t stream) {
-  const bool two = a.epilogue == EPI_SWIGLU;
   switch (a.bnb) {
-    case 32: return two ? launch_variant<32, 2>(a, stream) : launch_variant<32, 1>(a, stream);
-    case 64: return two ? launch_variant<64, 2>(a, stream) : launch_variant<64, 1>(a, stream);
-    case 128: return two ? launch_variant<128, 2>(a, stream) : launch_variant<128, 1>(a, stream);
-    case 256: return two ? launch_variant<256, 2>(a, stream) : launch_variant<256, 1>(a, stream);
+    case 32: return launch_variant<32>(a, stream);
+    case 64: return launch_variant<64>(a, stream);
+    case 128: return launch_variant<128>(a, stream);
+    case 256: return launch_variant<256>(a, stream);
     default: return cudaErrorInvalidValue;
   }
 }

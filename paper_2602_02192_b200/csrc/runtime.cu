@@ -19,6 +19,7 @@ namespace {
 
 constexpr size_t kAlign = 1024;
 constexpr int kChunkRows = 256;       // prompt tokens per prefill forward
+constexpr int kMaxCtas = 160;         // persistent GEMM grid never exceeds this (148 SMs on B200)
 
 size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -80,7 +81,7 @@ Limits limits_of(const echo_config &c) {
 struct Layout {
   size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
   size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
-      seq_len0, copy_src, copy_dst, d_step, status, stage_prompts, stage_tok, stage_lp, total;
+      seq_len0, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
   size_t weight_bytes, kv_layer_elems, n_tables_ints;
   int n_chunks_max;
 };
@@ -121,6 +122,8 @@ Layout layout_of(const echo_config &c) {
   lo.copy_dst = take(static_cast<size_t>(M.B) * 4);
   lo.d_step = take(4);
   lo.status = take(4);
+  lo.gemm_ws = take(static_cast<size_t>(kMaxCtas) * 3 * 2 * kGemmTileN * kMaxBatchTile * sizeof(float));
+  lo.gemm_counters = take(static_cast<size_t>(kGemmMaxUnits) * 4);
   lo.stage_prompts = take(static_cast<size_t>(M.P) * M.Lp * 4);
   lo.stage_tok = take(static_cast<size_t>(M.B) * M.T * 4);
   lo.stage_lp = take(static_cast<size_t>(M.B) * M.T * 4);
@@ -268,7 +271,8 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
     ctx->last_error = "tensor map encode failed (activation)";
     return ECHO_ERR_CUDA;
   }
-  GemmArgs a{tmW, &tmX, Y, ldY, M, N, K, bnb, epilogue, ctx->ptr<int>(ctx->lo.status)};
+  GemmArgs a{tmW, &tmX, Y, ldY, M, N, K, bnb, epilogue, ctx->ptr<int>(ctx->lo.status),
+             ctx->ptr<float>(ctx->lo.gemm_ws), ctx->ptr<int>(ctx->lo.gemm_counters), kMaxCtas, 0};
   LAUNCH(gemm_tc_launch(a, ctx->stream));
   return ECHO_OK;
 }
@@ -351,7 +355,7 @@ int make_weight_maps(echo_ctx *ctx, WeightBuf &w) {
   for (int l = 0; l < D.L; ++l) {
     rc |= make_tensor_map(&w.tm_qkv[l], w.wqkv[l], D.n_qkv(), D.d, D.d, kGemmTileN);
     rc |= make_tensor_map(&w.tm_o[l], w.wo[l], D.d, D.Hq * D.hd, D.Hq * D.hd, kGemmTileN);
-    rc |= make_tensor_map(&w.tm_gu[l], w.wgu[l], 2ull * D.F, D.d, D.d, kGemmTileN);
+    rc |= make_tensor_map(&w.tm_gu[l], w.wgu[l], 2ull * D.F, D.d, D.d, 64);
     rc |= make_tensor_map(&w.tm_down[l], w.wdown[l], D.d, D.F, D.F, kGemmTileN);
   }
   if (rc) {
@@ -690,6 +694,9 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
   if ((e = gemm_tc_configure()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute");
   if ((e = cudaMemsetAsync(ctx->arena + lo.status, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
   if ((e = cudaMemsetAsync(ctx->arena + lo.d_step, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
+  if ((e = cudaMemsetAsync(ctx->arena + lo.gemm_counters, 0, static_cast<size_t>(kGemmMaxUnits) * 4, ctx->stream)) !=
+      cudaSuccess)
+    return bail(e, "cudaMemset");
   if ((e = rope_table_launch(ctx->ptr<float2>(lo.rope), M.max_pos, ctx->D.hd, static_cast<double>(cfg->rope_theta),
                              ctx->stream)) != cudaSuccess)
     return bail(e, "rope_table");
@@ -846,6 +853,7 @@ int echo_sync(echo_ctx *ctx) {
   CK(cudaMemcpy(&status, ctx->arena + ctx->lo.status, 4, cudaMemcpyDeviceToHost));
   if (status != STATUS_OK) {
     cudaMemset(ctx->arena + ctx->lo.status, 0, 4);
+    cudaMemset(ctx->arena + ctx->lo.gemm_counters, 0, static_cast<size_t>(kGemmMaxUnits) * 4);
     return status == STATUS_WAIT_TIMEOUT ? ECHO_ERR_TIMEOUT : ECHO_ERR_DEVICE_CHECK;
   }
   return ECHO_OK;
@@ -889,21 +897,37 @@ int echo_sample(const float *logits, int32_t R, int32_t V, int32_t rows_per_logi
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }
 
-int echo_gemm_bf16(const void *X, const void *W, float *Y, int32_t M, int32_t N, int32_t K, int32_t impl,
-                   void *cuda_stream) {
+size_t echo_gemm_workspace_bytes(int32_t M) {
+  if (M < 1) return 0;
+  if (gemm_tc_configure() != cudaSuccess) return 0;
+  return align_up(gemm_workspace_bytes(pick_bnb(M))) + static_cast<size_t>(kGemmMaxUnits) * 4;
+}
+
+int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, int32_t K, int32_t epilogue,
+                   int32_t impl, void *workspace, size_t workspace_bytes, void *cuda_stream) {
   if (!X || !W || !Y || M < 1 || M > 4096 || N < 1 || K < 8 || (K % 8)) return ECHO_ERR_INVALID;
+  if (epilogue != EPI_STORE && epilogue != EPI_ACCUM && epilogue != EPI_SWIGLU) return ECHO_ERR_INVALID;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (impl == 1) {
-    cudaError_t e = gemm_simt_launch(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(W), Y,
-                                     N, M, N, K, 0, s);
+    if (epilogue == EPI_SWIGLU) return ECHO_ERR_INVALID;
+    cudaError_t e = gemm_simt_launch(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(W),
+                                     static_cast<float *>(Y), N, M, N, K, epilogue == EPI_ACCUM, s);
     return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
   }
   if (gemm_tc_configure() != cudaSuccess) return ECHO_ERR_CUDA;
-  CUtensorMap tmW, tmX;
   const int bnb = pick_bnb(M);
-  if (make_tensor_map(&tmW, W, N, K, K, kGemmTileN) != 0) return ECHO_ERR_CUDA;
+  const size_t ws_bytes = align_up(gemm_workspace_bytes(bnb));
+  if (!workspace || workspace_bytes < ws_bytes + static_cast<size_t>(kGemmMaxUnits) * 4 ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return ECHO_ERR_ARENA;
+  int *counters = reinterpret_cast<int *>(static_cast<uint8_t *>(workspace) + ws_bytes);
+  if (cudaMemsetAsync(counters, 0, static_cast<size_t>(kGemmMaxUnits) * 4, s) != cudaSuccess) return ECHO_ERR_CUDA;
+  CUtensorMap tmW, tmX;
+  const bool gu = epilogue == EPI_SWIGLU;
+  if (make_tensor_map(&tmW, W, gu ? 2ull * N : N, K, K, gu ? 64 : kGemmTileN) != 0) return ECHO_ERR_CUDA;
   if (make_tensor_map(&tmX, X, M, K, K, bnb) != 0) return ECHO_ERR_CUDA;
-  GemmArgs a{&tmW, &tmX, Y, N, M, N, K, bnb, EPI_STORE, nullptr};
+  const int split = impl >= 100 ? impl - 100 : (impl == 2 ? -1 : 0);
+  GemmArgs a{&tmW, &tmX, Y, N, M, N, K, bnb, epilogue, nullptr, static_cast<float *>(workspace), counters, 0, split};
   cudaError_t e = gemm_tc_launch(a, s);
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }

@@ -73,19 +73,46 @@ def test_sampler_seq_ids_and_tie_rule(B):
 
 
 @pytest.mark.parametrize("M,N,K", [(256, 384, 256), (16, 256, 256), (1, 128, 64), (100, 688, 256),
-                                   (37, 256, 688), (300, 1024, 512), (256, 4096, 4096), (512, 640, 1024)])
+                                   (37, 256, 688), (300, 1024, 512), (256, 4096, 4096), (512, 640, 1024),
+                                   (256, 4096, 12288), (130, 151936, 256)])
 def test_gemm_tensor_core_matches_fp64(B, M, N, K):
     rng = np.random.default_rng(M * 1000003 + N * 101 + K)
     X = torch.from_numpy(rng.normal(size=(M, K)).astype(np.float32)).to(torch.bfloat16)
     W = torch.from_numpy((rng.normal(size=(N, K)) * 0.05).astype(np.float32)).to(torch.bfloat16)
     want = widen_bf16(synth.bf16_bits(X)) @ widen_bf16(synth.bf16_bits(W)).T
-    for impl in (1, 0):
+    # fp32 accumulation of K products of magnitude ~0.05: error ~ K * 2^-24 * |terms|
+    tol = 2e-6 * K * 0.05 * 4 + 1e-6
+    # 1 = SIMT reference, 0 = automatic choice, 2 = persistent stream-K, 100+s = cluster split-K by s
+    impls = (1, 0, 2, 101, 103, 108) if N * K <= 4096 * 4096 else (0, 2)
+    for impl in impls:
         Y = B.echo_gemm_bf16(X.cuda(), W.cuda(), impl=impl)
-        torch.cuda.synchronize()
         got = Y.cpu().numpy().astype(np.float64)
-        # fp32 accumulation of K products of magnitude ~0.05: error ~ K * 2^-24 * |terms|
-        tol = 2e-6 * K * 0.05 * 4 + 1e-6
         assert np.max(np.abs(got - want)) < tol, (impl, np.max(np.abs(got - want)))
+    # residual-add epilogue, twice in a row (the tile counters must return to zero)
+    Y0 = torch.from_numpy(rng.normal(size=(M, N)).astype(np.float32)).cuda()
+    Y = Y0.clone()
+    B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=1, Y=Y, impl=2)
+    B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=1, Y=Y, impl=0)
+    got = Y.cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(got - (Y0.cpu().numpy() + 2 * want))) < 2 * tol + 1e-5
+
+
+@pytest.mark.parametrize("M,F,K", [(256, 688, 256), (16, 64, 64), (77, 1000, 512), (256, 12288, 4096),
+                                   (512, 3072, 1024)])
+def test_gemm_swiglu_epilogue(B, M, F, K):
+    rng = np.random.default_rng(M + F + K)
+    X = torch.from_numpy(rng.normal(size=(M, K)).astype(np.float32)).to(torch.bfloat16)
+    W = torch.from_numpy((rng.normal(size=(2 * F, K)) * 0.05).astype(np.float32)).to(torch.bfloat16)
+    xf, wf = widen_bf16(synth.bf16_bits(X)), widen_bf16(synth.bf16_bits(W))
+    g, u = xf @ wf[:F].T, xf @ wf[F:].T
+    want = g / (1 + np.exp(-g)) * u
+    for impl in (0, 2, 101, 104):
+        Y = B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=2, impl=impl)
+        got = Y.float().cpu().numpy().astype(np.float64)
+        # the output is rounded to bf16 (relative 2^-9) on top of the fp32 accumulation error
+        assert np.all(np.abs(got - want) <= 2.0 ** -8 * np.abs(want) + 1e-4 * K / 256), impl
+        Y2 = B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=2, impl=impl)
+        assert torch.equal(Y, Y2)                          # deterministic reduction order
 
 
 def test_group_advantage_matches_oracle(B):
