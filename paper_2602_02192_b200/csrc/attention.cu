@@ -10,13 +10,13 @@
 // one kv head is one contiguous K burst followed by one contiguous V burst.
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace echo {
 
 namespace {
 
 constexpr int kAttnWarps = 4;
-constexpr int kMaxRep = 8;        // query heads per kv head
 
 template <int HD, int REP>
 __global__ void __launch_bounds__(kAttnWarps * 32)
@@ -179,6 +179,355 @@ cudaError_t attention_rows_launch(const __nv_bfloat16 *q, const __nv_bfloat16 *k
   ECHO_ATTN_CASE(64, 1) ECHO_ATTN_CASE(64, 2) ECHO_ATTN_CASE(64, 4)
   ECHO_ATTN_CASE(128, 1) ECHO_ATTN_CASE(128, 2) ECHO_ATTN_CASE(128, 4) ECHO_ATTN_CASE(128, 8)
 #undef ECHO_ATTN_CASE
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace echo
+
+// =============================================================================================
+// Decode attention for GRPO rollouts: the G samples of a group share the prompt's KV pages, so
+// the prefix is attended ONCE per (group, kv head) for all G * (Hq/Hkv) query rows that use it,
+// and only each sample's own generated tokens are read per sample.
+//
+//   prefix kernel   one CTA per (prompt, kv head, 16-row tile of the group's query rows); keys =
+//                   the prompt's full pages; writes un-normalised partial outputs with their
+//                   running max and sum to scratch.
+//   suffix kernel   one CTA per (sequence, kv head); keys = the sequence's private pages (copy of
+//                   the prompt's partial last page + generated tokens); merges with the prefix
+//                   partial and writes the final bf16 output.
+//
+// Both run the same tile loop: the four warps of a CTA take pages round-robin; each warp streams
+// its pages (one 16-token page of one kv head = K burst + V burst) through its own TMA pipeline
+// into 128-byte-swizzled shared memory and does S = Q K^T and O += P V with warp-level bf16 MMAs
+// (the query rows are padded to the 16-row MMA tile; the kernel is bound by the KV byte stream,
+// not by the tensor pipe).  Softmax runs in the exp2 domain in fp32.
+// =============================================================================================
+namespace echo {
+namespace {
+
+using namespace ptx;
+
+constexpr int kDecWarps = 4;
+constexpr int kDecStages = 3;
+constexpr int kPageTokens = 16;
+
+template <int HD>
+struct DecSmem {
+  static constexpr int kStageBytes = 2 * kPageTokens * HD * 2;                 // K + V of one page, one head
+  static constexpr int kPipeBytes = kDecWarps * kDecStages * kStageBytes;
+  static constexpr int kMergeBytes = kDecWarps * 16 * (HD + 2) * 4;
+  static constexpr int kBody = kPipeBytes > kMergeBytes ? kPipeBytes : kMergeBytes;
+  static constexpr int kTotal = kBody + 256 + 1024;                            // barriers + alignment slack
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+template <int HD, bool PREFIX>
+__global__ void __launch_bounds__(kDecWarps * 32)
+attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16 *__restrict__ q,
+                   __nv_bfloat16 *__restrict__ out, float *__restrict__ pre_o, float2 *__restrict__ pre_ml,
+                   const int32_t *__restrict__ page_table, int pt_width, const int32_t *__restrict__ row_pos,
+                   const int32_t *__restrict__ full_pages, int layer_row0, int Hq, int Hkv, int G, int n_pages,
+                   float scale_log2, int *status) {
+  using S = DecSmem<HD>;
+  constexpr int KSTEPS = HD / 16;           // MMA k-steps over the head dimension
+  constexpr int HALVES = HD / 64;           // 64-element (128-byte) column blocks per row
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + S::kBody);              // [warp][stage]
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + kDecWarps * kDecStages);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int REP = Hq / Hkv;
+  const int quad = lane >> 2, qi = lane & 3;
+
+  // ---- which query rows and which keys this CTA handles ------------------------------------
+  int h, seq0, first_page, n_keys, mt = 0;
+  if (PREFIX) {
+    const int MT = (G * REP + 15) / 16;
+    mt = blockIdx.x % MT;
+    const int ph = blockIdx.x / MT;
+    h = ph % Hkv;
+    seq0 = (ph / Hkv) * G;                   // first sequence of the group
+    first_page = 0;
+    n_keys = full_pages[seq0] * kPageTokens;
+  } else {
+    h = blockIdx.x % Hkv;
+    seq0 = blockIdx.x / Hkv;
+    first_page = full_pages[seq0];
+    n_keys = row_pos[seq0] + 1 - first_page * kPageTokens;
+  }
+  const int n_tiles = (n_keys + kPageTokens - 1) / kPageTokens;
+  const int32_t *pt = page_table + static_cast<size_t>(seq0) * pt_width + first_page;
+
+  // row r (0..15) of the MMA tile -> (batch row, q head); -1 when the row is padding
+  auto row_seq = [&](int r) -> int {
+    if (PREFIX) {
+      const int gr = mt * 16 + r;
+      return gr < G * REP ? seq0 + gr / REP : -1;
+    }
+    return r < REP ? seq0 : -1;
+  };
+  auto row_head = [&](int r) -> int { return h * REP + (PREFIX ? (mt * 16 + r) % REP : r); };
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kDecWarps * kDecStages; ++i) mbar_init(&bars[i], 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  // ---- Q fragments (A operand), kept in registers for the whole loop ---------------------------
+  uint32_t qf[KSTEPS][4];
+  {
+    const int s_lo = row_seq(quad), s_hi = row_seq(quad + 8);
+    const uint32_t *q_lo = s_lo >= 0 ? reinterpret_cast<const uint32_t *>(
+                                           q + (static_cast<size_t>(s_lo) * Hq + row_head(quad)) * HD)
+                                     : nullptr;
+    const uint32_t *q_hi = s_hi >= 0 ? reinterpret_cast<const uint32_t *>(
+                                           q + (static_cast<size_t>(s_hi) * Hq + row_head(quad + 8)) * HD)
+                                     : nullptr;
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+      qf[kk][0] = q_lo ? q_lo[kk * 8 + qi] : 0u;
+      qf[kk][1] = q_hi ? q_hi[kk * 8 + qi] : 0u;
+      qf[kk][2] = q_lo ? q_lo[kk * 8 + 4 + qi] : 0u;
+      qf[kk][3] = q_hi ? q_hi[kk * 8 + 4 + qi] : 0u;
+    }
+  }
+
+  float o_acc[HD / 8][4];
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+
+  uint8_t *my_stages = smem + warp * kDecStages * S::kStageBytes;
+  uint64_t *my_bars = bars + warp * kDecStages;
+  const int n_my = n_tiles > warp ? (n_tiles - warp + kDecWarps - 1) / kDecWarps : 0;
+
+  int pg_cache = 0, pg_base = -1;            // page ids of 32 of this warp's tiles, one per lane
+  auto page_of = [&](int k) -> int {         // warp-uniform k
+    if (k < pg_base || k >= pg_base + 32 || pg_base < 0) {
+      pg_base = k;
+      const int kk = k + lane;
+      pg_cache = kk < n_my ? pt[warp + kDecWarps * kk] : 0;
+    }
+    return __shfl_sync(0xffffffffu, pg_cache, k - pg_base);
+  };
+  auto issue = [&](int k) {
+    const int page = page_of(k);
+    if (lane == 0) {
+      uint64_t *bar = &my_bars[k % kDecStages];
+      uint8_t *dst = my_stages + (k % kDecStages) * S::kStageBytes;
+      if (page < 0 || page >= n_pages) {
+        atomicExch(status, STATUS_BAD_PAGE);
+        mbar_arrive(bar);                    // nothing to load: complete the phase by hand
+      } else {
+        const int row = layer_row0 + (page * Hkv + h) * 2 * kPageTokens;
+        mbar_expect_tx(bar, S::kStageBytes);
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf) tma_load_2d(&tmKV, bar, dst + hf * (S::kStageBytes / HALVES), hf * 64, row);
+      }
+    }
+  };
+
+  const int n_pro = n_my < kDecStages ? n_my : kDecStages;
+  for (int k = 0; k < n_pro; ++k) issue(k);
+
+  bool ok = true;
+  for (int k = 0; k < n_my; ++k) {
+    ok = mbar_wait(&my_bars[k % kDecStages], (k / kDecStages) & 1, abort_flag);
+    if (!ok) break;
+    const uint32_t st = smem_u32(my_stages + (k % kDecStages) * S::kStageBytes);
+    const int key0 = (warp + kDecWarps * k) * kPageTokens;
+
+    // ---- S = Q K^T : 16 rows x 16 keys -------------------------------------------------------
+    float sc[2][4];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f;
+    {
+      const int id = lane >> 3, rr = lane & 7;
+      const int key = (id >> 1) * 8 + rr;
+#pragma unroll
+      for (int kk = 0; kk < KSTEPS; ++kk) {
+        const int c = 2 * (kk & 3) + (id & 1);
+        const uint32_t addr = st + (kk >> 2) * (S::kStageBytes / HALVES) + key * 128 + ((c ^ (key & 7)) << 4);
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4(addr, b0, b1, b2, b3);
+        mma_bf16_16816(sc[0], qf[kk], b0, b1);
+        mma_bf16_16816(sc[1], qf[kk], b2, b3);
+      }
+    }
+    // ---- online softmax (exp2 domain) ---------------------------------------------------------
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int key = key0 + 8 * nt + 2 * qi + (e & 1);
+        const float v = key < n_keys ? sc[nt][e] * scale_log2 : -INFINITY;
+        sc[nt][e] = v;
+        mx[e >> 1] = fmaxf(mx[e >> 1], v);
+      }
+    }
+    uint32_t pa[4];
+    {
+      float corr[2], msafe[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+        const float m_new = fmaxf(m_run[r], mx[r]);
+        msafe[r] = m_new == -INFINITY ? 0.f : m_new;
+        corr[r] = exp2f(m_run[r] - msafe[r]);           // 0 when nothing was accumulated yet
+        m_run[r] = m_new;
+      }
+      float p[2][4], ps[2] = {0.f, 0.f};
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          p[nt][e] = exp2f(sc[nt][e] - msafe[e >> 1]);
+          ps[e >> 1] += p[nt][e];
+        }
+      l_run[0] = l_run[0] * corr[0] + ps[0];
+      l_run[1] = l_run[1] * corr[1] + ps[1];
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i) {
+        o_acc[i][0] *= corr[0]; o_acc[i][1] *= corr[0];
+        o_acc[i][2] *= corr[1]; o_acc[i][3] *= corr[1];
+      }
+      pa[0] = pack_bf16(p[0][0], p[0][1]);
+      pa[1] = pack_bf16(p[0][2], p[0][3]);
+      pa[2] = pack_bf16(p[1][0], p[1][1]);
+      pa[3] = pack_bf16(p[1][2], p[1][3]);
+    }
+    // ---- O += P V ---------------------------------------------------------------------------
+    {
+      const int id = lane >> 3, rr = lane & 7;
+      const int key = (id & 1) * 8 + rr;
+#pragma unroll
+      for (int dt = 0; dt < KSTEPS; ++dt) {
+        const int c = 2 * (dt & 3) + (id >> 1);
+        const uint32_t addr = st + (dt >> 2) * (S::kStageBytes / HALVES) + kPageTokens * 128 + key * 128 +
+                              ((c ^ (key & 7)) << 4);
+        uint32_t v0, v1, v2, v3;
+        ldmatrix_x4_trans(addr, v0, v1, v2, v3);
+        mma_bf16_16816(o_acc[2 * dt], pa, v0, v1);
+        mma_bf16_16816(o_acc[2 * dt + 1], pa, v2, v3);
+      }
+    }
+    __syncwarp();
+    if (k + kDecStages < n_my) issue(k + kDecStages);
+  }
+  if (!ok) {
+    // give copies already in flight a chance to land before shared memory is reused or released
+    for (int k = 0; k < n_my; ++k) mbar_drain(&my_bars[k % kDecStages], (k / kDecStages) & 1);
+  }
+  // row sums: combine the four lanes that share a row
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+  }
+
+  // ---- combine the four warps through shared memory (the pipeline buffers are free now) -------
+  __syncthreads();
+  float *m_s = reinterpret_cast<float *>(smem);                      // [warp][16]
+  float *l_s = m_s + kDecWarps * 16;
+  float *o_s = l_s + kDecWarps * 16;                                 // [warp][16][HD]
+  if (qi == 0) {
+    m_s[warp * 16 + quad] = m_run[0];
+    m_s[warp * 16 + quad + 8] = m_run[1];
+    l_s[warp * 16 + quad] = l_run[0];
+    l_s[warp * 16 + quad + 8] = l_run[1];
+  }
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) {
+    float *o_lo = o_s + (warp * 16 + quad) * HD + 8 * i + 2 * qi;
+    float *o_hi = o_s + (warp * 16 + quad + 8) * HD + 8 * i + 2 * qi;
+    o_lo[0] = o_acc[i][0]; o_lo[1] = o_acc[i][1];
+    o_hi[0] = o_acc[i][2]; o_hi[1] = o_acc[i][3];
+  }
+  __syncthreads();
+  const int n_rows = PREFIX ? 16 : REP;
+  for (int idx = threadIdx.x; idx < n_rows * HD; idx += blockDim.x) {
+    const int r = idx / HD, d = idx % HD;
+    const int s = row_seq(r);
+    if (s < 0) continue;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, m_s[w * 16 + r]);
+    float L = 0.f, O = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) {
+      const float mw = m_s[w * 16 + r];
+      if (mw != -INFINITY) {
+        const float c = exp2f(mw - M);
+        L += l_s[w * 16 + r] * c;
+        O += o_s[(w * 16 + r) * HD + d] * c;
+      }
+    }
+    const size_t oi = (static_cast<size_t>(s) * Hq + row_head(r)) * HD + d;
+    if (PREFIX) {
+      pre_o[oi] = O;
+      if (d == 0) pre_ml[static_cast<size_t>(s) * Hq + row_head(r)] = make_float2(M, L);
+    } else {
+      const float2 ml = pre_ml[static_cast<size_t>(s) * Hq + row_head(r)];
+      float Mt = fmaxf(M, ml.x);
+      if (Mt == -INFINITY) Mt = 0.f;
+      const float c_suf = M == -INFINITY ? 0.f : exp2f(M - Mt);
+      const float c_pre = ml.x == -INFINITY ? 0.f : exp2f(ml.x - Mt);
+      const float Lt = L * c_suf + ml.y * c_pre;
+      const float Ot = O * c_suf + (c_pre != 0.f ? pre_o[oi] * c_pre : 0.f);
+      out[oi] = __float2bfloat16(Ot / Lt);
+    }
+  }
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(status, STATUS_WAIT_TIMEOUT);
+}
+
+template <int HD>
+cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
+  using S = DecSmem<HD>;
+  const int REP = a.Hq / a.Hkv;
+  const int MT = (a.G * REP + 15) / 16;
+  const float scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(HD));
+  attn_decode_kernel<HD, true><<<a.P * a.Hkv * MT, kDecWarps * 32, S::kTotal, s>>>(
+      *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages, a.layer_row0, a.Hq,
+      a.Hkv, a.G, a.n_pages, scale_log2, a.status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  attn_decode_kernel<HD, false><<<a.P * a.G * a.Hkv, kDecWarps * 32, S::kTotal, s>>>(
+      *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages, a.layer_row0, a.Hq,
+      a.Hkv, a.G, a.n_pages, scale_log2, a.status);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t attention_decode_configure() {
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(attn_decode_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                DecSmem<128>::kTotal)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(attn_decode_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                DecSmem<128>::kTotal)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(attn_decode_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                DecSmem<64>::kTotal)) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_decode_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              DecSmem<64>::kTotal);
+}
+
+bool attention_decode_supported(int hd, int page_size, int Hq, int Hkv) {
+  const int rep = Hq / Hkv;
+  return (hd == 64 || hd == 128) && page_size == kPageTokens && rep >= 1 && rep <= 16;
+}
+
+cudaError_t attention_decode_launch(const DecodeAttnArgs &a, cudaStream_t s) {
+  if (a.hd == 128) return launch_decode<128>(a, s);
+  if (a.hd == 64) return launch_decode<64>(a, s);
   return cudaErrorInvalidValue;
 }
 

@@ -98,4 +98,25 @@ cudaError_t attention_rows_launch(const __nv_bfloat16 *q, const __nv_bfloat16 *k
                                   int pt_width, int R, int Hq, int Hkv, int hd, int page_size,
                                   int n_pages, int *status, cudaStream_t s);
 
+
+// Decode-step attention with the group's prompt prefix read once for all G samples.
+// Scratch: pre_o fp32 [B][Hq][hd] and pre_ml float2 [B][Hq] (prefix partials between the two kernels).
+struct DecodeAttnArgs {
+  const CUtensorMap *tmKV;        // whole KV pool as [rows][hd] bf16, box {64, 2 * page}, 128-byte swizzle
+  const __nv_bfloat16 *q;         // [B][Hq][hd]
+  __nv_bfloat16 *out;             // [B][Hq][hd]
+  float *pre_o;
+  float2 *pre_ml;
+  const int32_t *page_table;      // row s = sequence s
+  int pt_width;
+  const int32_t *row_pos;         // position of the token each sequence feeds in this step
+  const int32_t *full_pages;      // full prompt pages (shared by the group) per sequence
+  int layer_row0;                 // first row of this layer in the pool's row space
+  int P, G, Hq, Hkv, hd, n_pages;
+  int *status;
+};
+cudaError_t attention_decode_configure();
+bool attention_decode_supported(int hd, int page_size, int Hq, int Hkv);
+cudaError_t attention_decode_launch(const DecodeAttnArgs &a, cudaStream_t s);
+
 }  // namespace echo

@@ -81,7 +81,7 @@ Limits limits_of(const echo_config &c) {
 struct Layout {
   size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
   size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
-      seq_len0, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
+      seq_len0, full_pages, pre_o, pre_ml, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
   size_t weight_bytes, kv_layer_elems, n_tables_ints;
   int n_chunks_max;
 };
@@ -118,6 +118,9 @@ Layout layout_of(const echo_config &c) {
   lo.dec_row_pos = take(static_cast<size_t>(M.B) * 4);
   lo.dec_row_pt = take(static_cast<size_t>(M.B) * 4);
   lo.seq_len0 = take(static_cast<size_t>(M.B) * 4);
+  lo.full_pages = take(static_cast<size_t>(M.B) * 4);
+  lo.pre_o = take(static_cast<size_t>(M.B) * D.Hq * D.hd * 4);
+  lo.pre_ml = take(static_cast<size_t>(M.B) * D.Hq * 8);
   lo.copy_src = take(static_cast<size_t>(M.B) * 4);
   lo.copy_dst = take(static_cast<size_t>(M.B) * 4);
   lo.d_step = take(4);
@@ -167,7 +170,8 @@ struct echo_ctx {
   int last_rows = 0, last_width = 0;
   echo_stats stats{};
   int64_t launches = 0;
-  bool use_simt = false, use_graph = true;
+  bool use_simt = false, use_graph = true, fast_decode = false;
+  CUtensorMap tm_kv;
   std::string last_error;
   // sampled per-kernel timing (echo_profile_config / echo_profile_read)
   int prof_every = 0;
@@ -284,7 +288,7 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
   } while (0)
 
 // All layers for R activation rows already embedded in x.
-int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta) {
+int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int decode_P = 0, int decode_G = 0) {
   const Dims &D = ctx->D;
   const Layout &lo = ctx->lo;
   float *x = ctx->ptr<float>(lo.x);
@@ -302,7 +306,15 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta) {
     TRY(run_gemm(ctx, &w.tm_qkv[l], w.wqkv[l], h, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE));
     LAUNCH(rope_append_launch(qkv, q, kv_layer, rope, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
                               ctx->M.n_pages, ctx->M.max_pos, status, ctx->stream));
-    {
+    if (decode_P > 0 && ctx->fast_decode) {
+      ProfScope prof(ctx, PROF_ATTN);
+      DecodeAttnArgs da{&ctx->tm_kv, q, attn, ctx->ptr<float>(lo.pre_o), ctx->ptr<float2>(lo.pre_ml), pt,
+                        ctx->M.pt_width, meta.row_pos, ctx->ptr<int32_t>(lo.full_pages),
+                        static_cast<int>(static_cast<size_t>(l) * (lo.kv_layer_elems / D.hd)), decode_P, decode_G,
+                        D.Hq, D.Hkv, D.hd, ctx->M.n_pages, status};
+      LAUNCH(attention_decode_launch(da, ctx->stream));
+      ctx->launches++;                      // two kernels per call
+    } else {
       ProfScope prof(ctx, PROF_ATTN);
       LAUNCH(attention_rows_launch(q, kv_layer, attn, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
                                    ctx->M.n_pages, status, ctx->stream));
@@ -409,7 +421,8 @@ int build_plan(echo_ctx *ctx, const int32_t *lens, int P, int G, int T, Plan *pl
   int32_t *h_gather = h_tok_idx + static_cast<size_t>(M.P) * M.Lp;
   int32_t *h_dec_pt = h_gather + static_cast<size_t>(ctx->lo.n_chunks_max) * M.P;
   int32_t *h_len0 = h_dec_pt + M.B;
-  int32_t *h_csrc = h_len0 + M.B;
+  int32_t *h_full = h_len0 + M.B;
+  int32_t *h_csrc = h_full + M.B;
   int32_t *h_cdst = h_csrc + M.B;
 
   std::fill(h_pt, h_pt + static_cast<size_t>(M.B + M.P) * W, -1);
@@ -439,6 +452,7 @@ int build_plan(echo_ctx *ctx, const int32_t *lens, int P, int G, int T, Plan *pl
       next_page += n_dec;
       h_dec_pt[s] = s;
       h_len0[s] = lens[p];
+      h_full[s] = full;
     }
   }
   if (next_page > M.n_pages) return ECHO_ERR_INVALID;
@@ -484,6 +498,7 @@ int upload_plan(echo_ctx *ctx, const Plan &pl) {
   CK(up(lo.gather_map, static_cast<size_t>(lo.n_chunks_max) * M.P, static_cast<size_t>(pl.n_chunks) * pl.P));
   CK(up(lo.dec_row_pt, M.B, pl.B));
   CK(up(lo.seq_len0, M.B, pl.B));
+  CK(up(lo.full_pages, M.B, pl.B));
   CK(up(lo.copy_src, M.B, pl.n_copies));
   CK(up(lo.copy_dst, M.B, pl.n_copies));
   CK(cudaEventRecord(ctx->plan_done, ctx->stream));
@@ -505,7 +520,7 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
   LAUNCH(embed_launch(w.embed, row_tok, nullptr, ctx->ptr<float>(lo.x), pl.B, ctx->D.d, ctx->D.V,
                       ctx->ptr<int>(lo.status), ctx->stream));
   RowMeta meta{ctx->ptr<int32_t>(lo.dec_row_pt), row_pos};
-  TRY(forward_layers(ctx, w, pl.B, meta));
+  TRY(forward_layers(ctx, w, pl.B, meta, pl.P, pl.G));
   TRY(lm_head(ctx, w, ctx->ptr<float>(lo.x), pl.B));
   {
     ProfScope prof(ctx, PROF_SAMPLER);
@@ -687,11 +702,30 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
     return bail(e, "cudaEventCreate");
   const Limits &M = ctx->M;
   ctx->h_tables_ints = static_cast<size_t>(M.B + M.P) * M.pt_width + 3ull * M.P * M.Lp +
-                       static_cast<size_t>(lo.n_chunks_max) * M.P + 4ull * M.B;
+                       static_cast<size_t>(lo.n_chunks_max) * M.P + 5ull * M.B;
   if ((e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_tables), ctx->h_tables_ints * 4, cudaHostAllocDefault)) !=
       cudaSuccess)
     return bail(e, "cudaHostAlloc");
   if ((e = gemm_tc_configure()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute");
+  // padding keys of a partly filled page take part in the P*V products with weight zero: the pool
+  // must never hold NaN/Inf bit patterns
+  if ((e = cudaMemsetAsync(ctx->arena + lo.kv, 0, lo.kv_layer_elems * ctx->D.L * 2, ctx->stream)) != cudaSuccess)
+    return bail(e, "cudaMemset(kv)");
+  {
+    const char *na = getenv("ECHO_ATTN_IMPL");
+    const size_t kv_rows = lo.kv_layer_elems / ctx->D.hd * ctx->D.L;
+    if (!(na && !strcmp(na, "rows")) && kv_rows < (1ull << 31) &&
+        attention_decode_supported(ctx->D.hd, ctx->D.Z, ctx->D.Hq, ctx->D.Hkv)) {
+      if ((e = attention_decode_configure()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute(attn)");
+      if (make_tensor_map(&ctx->tm_kv, ctx->arena + lo.kv, kv_rows, ctx->D.hd, ctx->D.hd, 2 * ctx->D.Z) != 0) {
+        ctx->last_error = "tensor map encode failed (kv)";
+        fprintf(stderr, "echo_create: %s\n", ctx->last_error.c_str());
+        echo_destroy(ctx);
+        return ECHO_ERR_CUDA;
+      }
+      ctx->fast_decode = true;
+    }
+  }
   if ((e = cudaMemsetAsync(ctx->arena + lo.status, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
   if ((e = cudaMemsetAsync(ctx->arena + lo.d_step, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
   if ((e = cudaMemsetAsync(ctx->arena + lo.gemm_counters, 0, static_cast<size_t>(kGemmMaxUnits) * 4, ctx->stream)) !=
