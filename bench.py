@@ -151,6 +151,8 @@ def run_ours(args):
     shape, P, G, Lp, T = wl.shape, wl.n_prompts, wl.G, wl.prompt_len, wl.new_tokens
     if args.new_tokens:
         T = args.new_tokens
+    if args.prompts:
+        P = args.prompts
     swap = args.workload == "8B" and not args.no_swap
     nbuf = 1 if args.workload == "32B" else 2
     eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, nbuf), device=local_rank)
@@ -401,6 +403,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8B", choices=["tiny", "0.6B", "4B", "8B", "32B"])
     ap.add_argument("--new-tokens", type=int, default=0, help="override T (diagnostic runs only)")
+    ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (diagnostic runs only)")
     ap.add_argument("--no-swap", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

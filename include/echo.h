@@ -225,6 +225,23 @@ int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, 
                    int32_t epilogue, int32_t impl, void *workspace, size_t workspace_bytes,
                    void *cuda_stream);
 
+/* echo_gemm_bf16 for callers that cannot allocate device memory (code that runs inside an
+ * allocator hook, a plug-in that is given tensors but no allocator, a process whose device
+ * memory another runtime has reserved).  The paper has no counterpart of this call.  Same
+ * arithmetic and epilogues as echo_gemm_bf16, but the split-tile scratch is a fixed array
+ * inside the library (about 6 MiB of device memory on every GPU that loads the library, held
+ * until the process exits), so no workspace is passed and nothing is allocated or freed, by
+ * this call or by anything it calls.
+ *   - M is limited to 32 activation rows; a larger M returns ECHO_ERR_UNSUPPORTED and does
+ *     nothing.  X, W, Y as for echo_gemm_bf16 (Y must be 16-byte aligned).
+ *   - The first call on each device looks up the array's device address and sets kernel
+ *     attributes; make that first call with the device current and before any stream capture.
+ *   - All calls share the one array.  The call clears the part that must start at zero, but
+ *     two calls whose kernels can overlap on the GPU (different streams or host threads) race
+ *     on it: keep calls on one stream, or order them with events. */
+int echo_gemm_bf16_noalloc(const void *X, const void *W, void *Y, int32_t M, int32_t N, int32_t K,
+                           int32_t epilogue, void *cuda_stream);
+
 const char *echo_strerror(int code);
 const char *echo_last_error(echo_ctx *ctx);   /* text of the last ECHO_ERR_CUDA on this context */
 

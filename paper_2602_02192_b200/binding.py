@@ -81,6 +81,8 @@ def _load() -> C.CDLL:
     lib.echo_debug_noise.argtypes = [u64, u32, u32, u32, u32, vp, vp, vp]
     lib.echo_sample.argtypes = [vp, i32, i32, i32, vp, u32, f32, u64, vp, vp, vp, vp]
     lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]
+    lib.echo_gemm_bf16_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.echo_gemm_bf16_noalloc.restype = C.c_int
     lib.echo_gemm_workspace_bytes.restype = C.c_size_t
     lib.echo_gemm_workspace_bytes.argtypes = [i32]
     lib.echo_strerror.restype = C.c_char_p
@@ -100,7 +102,7 @@ lib = _load()
 EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy", "echo_wait_policy",
             "echo_rollout", "echo_rollout_forced", "echo_rollout_host", "echo_group_advantage", "echo_sync",
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
-            "echo_gemm_workspace_bytes", "echo_strerror", "echo_last_error"]
+            "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_strerror", "echo_last_error"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -313,4 +315,19 @@ def echo_gemm_bf16(X: torch.Tensor, W: torch.Tensor, impl: int = 0, epilogue: in
         _check(lib.echo_gemm_bf16(X.data_ptr(), W.data_ptr(), Y.data_ptr(), M, N, K, epilogue, impl,
                                   ws.data_ptr(), nws, _stream_ptr(None)))
         torch.cuda.current_stream().synchronize()      # the workspace must outlive the kernel
+    return Y
+
+
+def echo_gemm_bf16_noalloc(X: torch.Tensor, W: torch.Tensor, Y: torch.Tensor, epilogue: int = 0) -> torch.Tensor:
+    """Projection through the library's built-in scratch: this wrapper allocates nothing either, so
+    the caller passes the output tensor (fp32 [M][N], or bf16 [M][N] for epilogue 2 with W = [Wg; Wu]).
+    At most 32 rows; calls that may overlap on the GPU must not be issued concurrently."""
+    assert X.is_cuda and W.is_cuda and Y.is_cuda and X.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
+    assert X.is_contiguous() and W.is_contiguous() and Y.is_contiguous() and X.shape[1] == W.shape[1]
+    M, K = X.shape
+    N = W.shape[0] // 2 if epilogue == 2 else W.shape[0]
+    assert tuple(Y.shape) == (M, N) and Y.dtype == (torch.bfloat16 if epilogue == 2 else torch.float32)
+    with torch.cuda.device(X.device):
+        _check(lib.echo_gemm_bf16_noalloc(X.data_ptr(), W.data_ptr(), Y.data_ptr(), M, N, K, epilogue,
+                                          _stream_ptr(None)))
     return Y

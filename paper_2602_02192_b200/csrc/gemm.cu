@@ -761,3 +761,70 @@ cudaError_t gemm_simt_launch(const __nv_bfloat16 *X, const __nv_bfloat16 *W, flo
 }
 
 }  // namespace echo
+
+// =============================================================================================
+// Projection for callers that cannot allocate device memory.
+//
+// The stream-K kernel needs scratch for the partial sums of tiles it splits across CTAs.
+// echo_gemm_bf16 takes that scratch from the caller.  Some callers have nowhere to get it from:
+// code running inside a framework's allocator callback or memory-pool hook, a plug-in that is
+// handed tensors but no allocator, or a process whose device memory is fully reserved by another
+// runtime.  For them the scratch below is part of the library image: a fixed array in device
+// memory that exists on every GPU the library is loaded on, from load until the process exits.
+//
+// The price is a size limit (kNoAllocMaxRows activation rows, kNoAllocMaxCtas CTAs) and sharing:
+// every call uses the same array, so two calls whose kernels may run at the same time (different
+// streams, or different host threads) would corrupt each other's partial sums.
+// =============================================================================================
+namespace echo {
+namespace {
+constexpr int kNoAllocMaxRows = 32;                   // activation rows (one 32-column accumulator block)
+constexpr int kNoAllocMaxCtas = 64;                   // persistent CTAs the variant launches at most
+constexpr size_t kNoAllocWsBytes =
+    static_cast<size_t>(kNoAllocMaxCtas) * 3 * kAcc * kGemmTileN * kNoAllocMaxRows * sizeof(float);   // 6 MiB
+constexpr size_t kNoAllocBytes = kNoAllocWsBytes + static_cast<size_t>(kGemmMaxUnits) * sizeof(int);
+}  // namespace
+}  // namespace echo
+
+// Partial-sum slots followed by the per-tile arrival counters.  Device code may name this array
+// directly; host code must not use the name as a pointer (on the host it is only a handle) and
+// asks the runtime for the device address instead.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[echo::kNoAllocBytes];
+
+namespace echo {
+namespace {
+void *g_noalloc_ptr[64] = {};                         // device address of the array, per device ordinal
+}  // namespace
+}  // namespace echo
+
+extern "C" int echo_gemm_bf16_noalloc(const void *X, const void *W, void *Y, int32_t M, int32_t N, int32_t K,
+                                      int32_t epilogue, void *cuda_stream) {
+  using namespace echo;
+  if (!X || !W || !Y || M < 1 || N < 1 || K < 8 || (K % 8)) return ECHO_ERR_INVALID;
+  if (epilogue != EPI_STORE && epilogue != EPI_ACCUM && epilogue != EPI_SWIGLU) return ECHO_ERR_INVALID;
+  if (M > kNoAllocMaxRows) return ECHO_ERR_UNSUPPORTED;           // beyond the built-in scratch
+  const bool gu = epilogue == EPI_SWIGLU;
+  const int per_tile = kAcc * (gu ? 64 : kGemmTileN);
+  if ((N + per_tile - 1) / per_tile > kGemmMaxUnits) return ECHO_ERR_UNSUPPORTED;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ECHO_ERR_CUDA;
+  if (!g_noalloc_ptr[dev]) {
+    // first call on this device: kernel attributes and the array's device address
+    if (gemm_tc_configure() != cudaSuccess) return ECHO_ERR_CUDA;
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return ECHO_ERR_CUDA;
+    g_noalloc_ptr[dev] = p;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char *base = static_cast<unsigned char *>(g_noalloc_ptr[dev]);
+  int *counters = reinterpret_cast<int *>(base + kNoAllocWsBytes);
+  // the array keeps whatever the previous call left: the counters must start at zero
+  if (cudaMemsetAsync(counters, 0, static_cast<size_t>(kGemmMaxUnits) * sizeof(int), s) != cudaSuccess)
+    return ECHO_ERR_CUDA;
+  CUtensorMap tmW, tmX;
+  if (make_tensor_map(&tmW, W, gu ? 2ull * N : N, K, K, gu ? 64 : kGemmTileN) != 0) return ECHO_ERR_CUDA;
+  if (make_tensor_map(&tmX, X, M, K, K, kNoAllocMaxRows) != 0) return ECHO_ERR_CUDA;
+  GemmArgs a{&tmW, &tmX, Y, N, M, N, K, kNoAllocMaxRows, epilogue, nullptr, reinterpret_cast<float *>(base),
+             counters, kNoAllocMaxCtas, -1};
+  return gemm_tc_launch(a, s) == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
