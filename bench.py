@@ -153,6 +153,8 @@ def run_ours(args):
         T = args.new_tokens
     if args.prompts:
         P = args.prompts
+    if args.prompt_len:
+        Lp = args.prompt_len
     swap = args.workload == "8B" and not args.no_swap
     nbuf = 1 if args.workload == "32B" else 2
     eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, nbuf), device=local_rank)
@@ -404,6 +406,7 @@ def main():
     ap.add_argument("--workload", default="8B", choices=["tiny", "0.6B", "4B", "8B", "32B"])
     ap.add_argument("--new-tokens", type=int, default=0, help="override T (diagnostic runs only)")
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (diagnostic runs only)")
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (diagnostic runs only)")
     ap.add_argument("--no-swap", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -209,6 +209,25 @@ int echo_sample(const float *logits, int32_t R, int32_t V, int32_t rows_per_logi
                 const int32_t *forced, int32_t *out_tokens, float *out_logprobs,
                 void *cuda_stream);
 
+/* Decode-step attention alone (paged GQA with the group's prompt pages read once for all G
+ * samples).  B = P*G sequences, sequence s = p*G + g.
+ *   q           dev bf16 [B][Hq][hd]            (already rotated)
+ *   kv_pool     dev bf16 [n_pages][Hkv][2][16][hd]: per page and kv head, 16 K rows then 16 V rows
+ *   page_table  dev int32 [B][pt_width]: physical page of each logical page of a sequence
+ *   row_pos     dev int32 [B]: position of the newest token of each sequence (keys 0..row_pos)
+ *   full_pages  dev int32 [B]: leading pages shared by the whole group (same value for its G
+ *               sequences; the shared pages are taken from the group's first sequence)
+ *   scratch     dev, echo_decode_attention_scratch_bytes(B, Hq, hd) bytes, 256-byte aligned:
+ *               the prefix partial results handed from the first kernel to the second
+ *   out         dev bf16 [B][Hq][hd]
+ * hd must be 64 or 128, pages hold 16 tokens.  Synchronises the stream and returns
+ * ECHO_ERR_DEVICE_CHECK if a page id was out of range. */
+size_t echo_decode_attention_scratch_bytes(int32_t B, int32_t Hq, int32_t hd);
+int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, const int32_t *page_table,
+                          int32_t pt_width, const int32_t *row_pos, const int32_t *full_pages, int32_t P,
+                          int32_t G, int32_t Hq, int32_t Hkv, int32_t hd, void *scratch, size_t scratch_bytes,
+                          void *out, void *cuda_stream);
+
 /* Dense projection alone, on the tcgen05 tensor cores with fp32 accumulation:
  *   epilogue 0:  Y[M][N] (dev fp32)  = X[M][K] (dev bf16) * W[N][K]^T (dev bf16)
  *   epilogue 1:  Y[M][N] (dev fp32) += X * W^T                        (residual add)

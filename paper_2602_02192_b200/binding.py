@@ -81,6 +81,10 @@ def _load() -> C.CDLL:
     lib.echo_debug_noise.argtypes = [u64, u32, u32, u32, u32, vp, vp, vp]
     lib.echo_sample.argtypes = [vp, i32, i32, i32, vp, u32, f32, u64, vp, vp, vp, vp]
     lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]
+    lib.echo_decode_attention.argtypes = [vp, vp, i32, vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, vp]
+    lib.echo_decode_attention.restype = C.c_int
+    lib.echo_decode_attention_scratch_bytes.argtypes = [i32, i32, i32]
+    lib.echo_decode_attention_scratch_bytes.restype = C.c_size_t
     lib.echo_gemm_bf16_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
     lib.echo_gemm_bf16_noalloc.restype = C.c_int
     lib.echo_gemm_workspace_bytes.restype = C.c_size_t
@@ -102,7 +106,8 @@ lib = _load()
 EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy", "echo_wait_policy",
             "echo_rollout", "echo_rollout_forced", "echo_rollout_host", "echo_group_advantage", "echo_sync",
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
-            "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_strerror", "echo_last_error"]
+            "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_decode_attention",
+            "echo_decode_attention_scratch_bytes", "echo_strerror", "echo_last_error"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -331,3 +336,20 @@ def echo_gemm_bf16_noalloc(X: torch.Tensor, W: torch.Tensor, Y: torch.Tensor, ep
         _check(lib.echo_gemm_bf16_noalloc(X.data_ptr(), W.data_ptr(), Y.data_ptr(), M, N, K, epilogue,
                                           _stream_ptr(None)))
     return Y
+
+
+def echo_decode_attention(q: torch.Tensor, kv_pool: torch.Tensor, page_table: torch.Tensor, row_pos: torch.Tensor,
+                          full_pages: torch.Tensor, P: int, G: int) -> torch.Tensor:
+    """q bf16 [B][Hq][hd]; kv_pool bf16 [n_pages][Hkv][2][16][hd]; int32 device tensors for the tables."""
+    B, Hq, hd = q.shape
+    n_pages, Hkv = kv_pool.shape[0], kv_pool.shape[1]
+    assert B == P * G and q.is_contiguous() and kv_pool.is_contiguous() and page_table.is_contiguous()
+    assert page_table.dtype == torch.int32 and row_pos.dtype == torch.int32 and full_pages.dtype == torch.int32
+    out = torch.empty_like(q)
+    with torch.cuda.device(q.device):
+        n = int(lib.echo_decode_attention_scratch_bytes(B, Hq, hd))
+        scratch = torch.empty(n, dtype=torch.uint8, device=q.device)
+        _check(lib.echo_decode_attention(q.data_ptr(), kv_pool.data_ptr(), n_pages, page_table.data_ptr(),
+                                         page_table.shape[1], row_pos.data_ptr(), full_pages.data_ptr(), P, G, Hq,
+                                         Hkv, hd, scratch.data_ptr(), n, out.data_ptr(), _stream_ptr(None)))
+    return out

@@ -931,6 +931,42 @@ int echo_sample(const float *logits, int32_t R, int32_t V, int32_t rows_per_logi
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }
 
+size_t echo_decode_attention_scratch_bytes(int32_t B, int32_t Hq, int32_t hd) {
+  if (B < 1 || Hq < 1 || hd < 1) return 0;
+  return align_up(static_cast<size_t>(B) * Hq * hd * 4) + align_up(static_cast<size_t>(B) * Hq * 8) + kAlign;
+}
+
+int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, const int32_t *page_table,
+                          int32_t pt_width, const int32_t *row_pos, const int32_t *full_pages, int32_t P, int32_t G,
+                          int32_t Hq, int32_t Hkv, int32_t hd, void *scratch, size_t scratch_bytes, void *out,
+                          void *cuda_stream) {
+  if (!q || !kv_pool || !page_table || !row_pos || !full_pages || !scratch || !out) return ECHO_ERR_INVALID;
+  if (P < 1 || G < 1 || n_pages < 1 || pt_width < 1 || Hkv < 1 || Hq % Hkv) return ECHO_ERR_INVALID;
+  if (!attention_decode_supported(hd, 16, Hq, Hkv)) return ECHO_ERR_UNSUPPORTED;
+  const int B = P * G;
+  if (scratch_bytes < echo_decode_attention_scratch_bytes(B, Hq, hd) || (reinterpret_cast<uintptr_t>(scratch) & 255))
+    return ECHO_ERR_ARENA;
+  const size_t rows = static_cast<size_t>(n_pages) * Hkv * 2 * 16;
+  if (rows >= (1ull << 31)) return ECHO_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (attention_decode_configure() != cudaSuccess) return ECHO_ERR_CUDA;
+  CUtensorMap tm;
+  if (make_tensor_map(&tm, kv_pool, rows, hd, hd, 32) != 0) return ECHO_ERR_CUDA;
+  uint8_t *sc = static_cast<uint8_t *>(scratch);
+  float *pre_o = reinterpret_cast<float *>(sc);
+  float2 *pre_ml = reinterpret_cast<float2 *>(sc + align_up(static_cast<size_t>(B) * Hq * hd * 4));
+  int *status = reinterpret_cast<int *>(reinterpret_cast<uint8_t *>(pre_ml) + align_up(static_cast<size_t>(B) * Hq * 8));
+  if (cudaMemsetAsync(status, 0, 4, s) != cudaSuccess) return ECHO_ERR_CUDA;
+  DecodeAttnArgs da{&tm, static_cast<const __nv_bfloat16 *>(q), static_cast<__nv_bfloat16 *>(out), pre_o, pre_ml,
+                    page_table, pt_width, row_pos, full_pages, 0, P, G, Hq, Hkv, hd, n_pages, status};
+  if (attention_decode_launch(da, s) != cudaSuccess) return ECHO_ERR_CUDA;
+  int st = 0;
+  if (cudaMemcpyAsync(&st, status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ECHO_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return ECHO_ERR_CUDA;
+  if (st == STATUS_WAIT_TIMEOUT) return ECHO_ERR_TIMEOUT;
+  return st == STATUS_OK ? ECHO_OK : ECHO_ERR_DEVICE_CHECK;
+}
+
 size_t echo_gemm_workspace_bytes(int32_t M) {
   if (M < 1) return 0;
   if (gemm_tc_configure() != cudaSuccess) return 0;

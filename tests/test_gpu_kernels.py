@@ -115,6 +115,37 @@ def test_gemm_swiglu_epilogue(B, M, F, K):
         assert torch.equal(Y, Y2)                          # deterministic reduction order
 
 
+@pytest.mark.parametrize("P,G,Hq,Hkv,hd,Lp,steps", [(4, 8, 32, 8, 128, 512, 1200), (3, 4, 4, 2, 64, 40, 37),
+                                                     (2, 2, 16, 2, 128, 7, 1), (2, 8, 8, 8, 128, 64, 300)])
+def test_decode_attention_matches_oracle(B, P, G, Hq, Hkv, hd, Lp, steps):
+    """Shared-prefix decode attention against the oracle's single-query attention (fp64) on the same
+    bf16-rounded q, K, V, gathered through the oracle's page plan."""
+    from oracle import decoder as o_dec
+    from oracle import pages as o_pages
+    rng = np.random.default_rng(P * 131 + Lp)
+    plan = o_pages.build([Lp] * P, G, steps + 1, 16)
+    n_pages, Bq = plan.n_pages, P * G
+    pool = torch.from_numpy(rng.normal(size=(n_pages, Hkv, 2, 16, hd)).astype(np.float32)).to(torch.bfloat16)
+    q = torch.from_numpy(rng.normal(size=(Bq, Hq, hd)).astype(np.float32)).to(torch.bfloat16)
+    pos = np.full(Bq, Lp + steps - 1, dtype=np.int32)
+    pos[::3] -= min(steps - 1, 5)                       # sequences need not be at the same position
+    full = np.repeat(plan.full_prefix_pages, G).astype(np.int32)
+    out = B.echo_decode_attention(q.cuda(), pool.cuda(), torch.from_numpy(plan.table).cuda(),
+                                  torch.from_numpy(pos).cuda(), torch.from_numpy(full).cuda(), P, G)
+    out = out.float().cpu().numpy().astype(np.float64)
+    poolf = widen_bf16(synth.bf16_bits(pool))
+    qf = widen_bf16(synth.bf16_bits(q))
+    for s in sorted(set([0, 1, Bq // 2, Bq - 1])):
+        n = int(pos[s]) + 1
+        pg = plan.table[s, np.arange(n) // 16]
+        K = poolf[pg, :, 0, np.arange(n) % 16, :]         # [n, Hkv, hd]
+        V = poolf[pg, :, 1, np.arange(n) % 16, :]
+        want = o_dec.attend_one(qf[s], K, V, Hq, Hkv)
+        err = np.abs(out[s] - want)
+        # probabilities and the output are rounded to bf16 (2^-9 relative each)
+        assert np.all(err <= 1.5e-2 * np.abs(want) + 4e-3), (s, err.max())
+
+
 def test_group_advantage_matches_oracle(B):
     for P, G, seed in [(4, 4, 0), (32, 8, 1), (1, 2, 2), (7, 33, 3), (100, 16, 4)]:
         r = synth.make_rewards(P, G, seed)
