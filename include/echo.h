@@ -237,8 +237,10 @@ int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, c
  * device memory of at least echo_gemm_workspace_bytes(M) bytes, owned by the caller, used only
  * during the call's kernels.  `impl`: 0 = tensor-core kernel (cluster split-K for few output
  * tiles, persistent stream-K otherwise), 2 = always the persistent stream-K kernel, 100 + s =
- * cluster split-K by s in [1, 8], 1 = plain SIMT reference kernel (epilogues 0 and 1 only;
- * needs no workspace). */
+ * cluster split-K by s in [1, 8] (partials summed in a fixed order), 200 + s = s independent
+ * k-slices per tile that add their partial sums into Y in memory (s = 0: as many as fill the GPU;
+ * faster, but the order of the fp32 additions varies from run to run; epilogues 0 and 1),
+ * 1 = plain SIMT reference kernel (epilogues 0 and 1 only; needs no workspace). */
 size_t echo_gemm_workspace_bytes(int32_t M);
 int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, int32_t K,
                    int32_t epilogue, int32_t impl, void *workspace, size_t workspace_bytes,

@@ -45,7 +45,9 @@ struct GemmArgs {
   float *workspace;   // gemm_workspace_bytes(bnb) bytes: partial accumulators of split tiles
   int *counters;      // kGemmMaxUnits ints, zero before the first launch (the kernel re-zeroes them)
   int max_ctas;       // 0 = one CTA per SM
-  int force_split;    // 0 = choose; k > 0 = cluster split-K by k; -1 = always the persistent stream-K kernel
+  int force_split;    // 0 = choose; k > 0 = split-K by k; -1 = always the persistent stream-K kernel
+  int independent_splits;   // 1: k-slices add into Y in memory (Y must hold zeros for EPI_STORE; the order of
+                            // the additions is not fixed); 0: slices are reduced in rank order inside a cluster
 };
 size_t gemm_workspace_bytes(int bnb);
 cudaError_t gemm_tc_launch(const GemmArgs &a, cudaStream_t stream);

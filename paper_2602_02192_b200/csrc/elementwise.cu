@@ -56,11 +56,47 @@ __device__ __forceinline__ float block_sum(float v, float *scratch) {
   return t;
 }
 
-// h = bf16( x * rsqrt(mean(x^2) + eps) * gain )
-__global__ void rmsnorm_kernel(const float *x, const __nv_bfloat16 *gain, __nv_bfloat16 *h, int R, int d, float eps) {
+// h = bf16( x * rsqrt(mean(x^2) + eps) * gain ).  One block per row; the row is read once
+// (float4 per thread, kept in registers) when d <= 4 * 4 * blockDim.
+constexpr int kNormThreads = 256;
+constexpr int kNormVecs = 8;          // float4 per thread held in registers (d <= 8192)
+__global__ void __launch_bounds__(kNormThreads)
+rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ gain, __nv_bfloat16 *__restrict__ h,
+               int R, int d, float eps) {
   __shared__ float scratch[32];
   const int r = blockIdx.x;
   const float *xr = x + static_cast<size_t>(r) * d;
+  __nv_bfloat16 *hr = h + static_cast<size_t>(r) * d;
+  const bool fast = (d % 4 == 0) && d <= 4 * kNormVecs * kNormThreads;
+  if (fast) {
+    const int nv = d / 4;
+    float4 v[kNormVecs];
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < kNormVecs; ++i) {
+      const int idx = threadIdx.x + i * kNormThreads;
+      v[i] = idx < nv ? reinterpret_cast<const float4 *>(xr)[idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+      ss = fmaf(v[i].x, v[i].x, fmaf(v[i].y, v[i].y, fmaf(v[i].z, v[i].z, fmaf(v[i].w, v[i].w, ss))));
+    }
+    ss = block_sum(ss, scratch);
+    const float scale = rsqrtf(ss / static_cast<float>(d) + eps);
+#pragma unroll
+    for (int i = 0; i < kNormVecs; ++i) {
+      const int idx = threadIdx.x + i * kNormThreads;
+      if (idx < nv) {
+        const uint2 graw = reinterpret_cast<const uint2 *>(gain)[idx];
+        const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw.x));
+        const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw.y));
+        __nv_bfloat162 o0 = __floats2bfloat162_rn(v[i].x * scale * g0.x, v[i].y * scale * g0.y);
+        __nv_bfloat162 o1 = __floats2bfloat162_rn(v[i].z * scale * g1.x, v[i].w * scale * g1.y);
+        uint2 o;
+        o.x = *reinterpret_cast<uint32_t *>(&o0);
+        o.y = *reinterpret_cast<uint32_t *>(&o1);
+        reinterpret_cast<uint2 *>(hr)[idx] = o;
+      }
+    }
+    return;
+  }
   float ss = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     const float v = xr[i];
@@ -68,7 +104,6 @@ __global__ void rmsnorm_kernel(const float *x, const __nv_bfloat16 *gain, __nv_b
   }
   ss = block_sum(ss, scratch);
   const float scale = rsqrtf(ss / static_cast<float>(d) + eps);
-  __nv_bfloat16 *hr = h + static_cast<size_t>(r) * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x)
     hr[i] = __float2bfloat16(xr[i] * scale * __bfloat162float(gain[i]));
 }
@@ -318,7 +353,7 @@ cudaError_t embed_launch(const __nv_bfloat16 *embed, const int32_t *tok_src, con
 }
 cudaError_t rmsnorm_launch(const float *x, const __nv_bfloat16 *gain, __nv_bfloat16 *h, int R, int d, float eps,
                            cudaStream_t s) {
-  rmsnorm_kernel<<<R, 256, 0, s>>>(x, gain, h, R, d, eps);
+  rmsnorm_kernel<<<R, kNormThreads, 0, s>>>(x, gain, h, R, d, eps);
   return cudaGetLastError();
 }
 cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double theta, cudaStream_t s) {

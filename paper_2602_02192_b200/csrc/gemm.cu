@@ -77,7 +77,7 @@ struct Split {
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
 // Loads of one k-block: kAcc weight blocks (each 128 rows, or 64 gate + 64 up rows) and the
-// activation tile.  `wait_dep` defers the activation load until the producing kernel is done.
+// activation tile.
 template <int BNB>
 __device__ __forceinline__ void load_stage(const CUtensorMap *tmW, const CUtensorMap *tmX, uint64_t *bar,
                                            uint8_t *stage, int kb, int nt, int m0, int N, bool gu) {
@@ -386,7 +386,7 @@ template <int BNB>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                     const __grid_constant__ CUtensorMap tmY, int M, int N, int K, int epilogue, int S_split,
-                    int *status) {
+                    int independent, int *status) {
   using S = GemmSmem<BNB>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -459,7 +459,10 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   // cluster's partials are summed through distributed shared memory in rank order, each CTA
   // taking a slice of columns; the finished tile leaves through TMA stores (or TMA reduce-adds
   // for the residual epilogue), which keep the few epilogue warps off the global store path.
-  const bool plain = S_split == 1 && !gu;
+  // `independent`: the S_split CTAs of a tile are not a cluster; each adds its partial tile to the
+  // output in memory (TMA reduce-add), so the summation order across them is not fixed
+  const bool plain = (S_split == 1 || independent) && !gu;
+  const bool add_out = epilogue == EPI_ACCUM || (independent && S_split > 1);
   const int cols = min(BNB, M - m0);
   const int quarter = warp & 3;
   const int row = quarter * 32 + lane;
@@ -477,24 +480,34 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll 1
   for (int a = 0; a < kAcc; ++a) {
     if (warp >= 2) {
-      if (a > 0) {
-        if (lane == 0) bulk_wait_read();                  // TMA has read the previous accumulator's staging
+      if (a > 0 && plain) {
+        if (lane == 0) bulk_wait_read();                  // TMA has read the previous accumulator out of `part`
         epi_bar();
       }
       if (got) {
-#pragma unroll 1
-        for (int c0 = 32 * grp; c0 < cols; c0 += 32 * kEpiGroups) {
-          uint32_t r[32];
-          tc_ld32(lane_addr + a * BNB + c0, r);
-          tc_wait_ld();
+        // two 32-column blocks per warp, both TMEM loads in flight before the first store
+        const int c0 = 32 * grp, c1 = c0 + 32 * kEpiGroups;
+        uint32_t r0[32], r1[32];
+        if (c0 < cols) tc_ld32(lane_addr + a * BNB + c0, r0);
+        if (c1 < cols) tc_ld32(lane_addr + a * BNB + c1, r1);
+        tc_wait_ld();
+        if (c0 < cols) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) part[(c0 + c) * kGemmTileN + row] = __uint_as_float(r[c]);
+          for (int c = 0; c < 32; ++c) part[(c0 + c) * kGemmTileN + row] = __uint_as_float(r0[c]);
+        }
+        if (c1 < cols) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) part[(c1 + c) * kGemmTileN + row] = __uint_as_float(r1[c]);
         }
       }
     }
     __syncwarp();
     if (!plain) {
       cluster_sync_all();                                 // all partials of this accumulator are in place
+      if (warp >= 2 && a > 0) {
+        if (lane == 0) bulk_wait_read();                  // TMA has read the previous result out of out_stage
+        epi_bar();
+      }
       if (warp >= 2 && got) {
         // one warp per column: a lane owns 4 consecutive features (2 gate + 2 up for SwiGLU), so a
         // warp reads a whole 512-byte row of every rank's partial with one vector load per rank;
@@ -555,6 +568,8 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
       }
     }
+    __syncwarp();
+    if (!plain) cluster_sync_all();                       // peers have finished reading this CTA's partial
     if (warp >= 2) {
       fence_proxy_async();
       epi_bar();
@@ -566,14 +581,12 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int lo = plain ? 0 : c_lo, hi = plain ? 8 * units : c_hi;
         for (int c = lo + 8 * (warp - 2); c < hi; c += 8 * kEpiWarps) {
           const uint8_t *p8 = src + static_cast<size_t>(c - lo) * row_bytes;
-          if (epilogue == EPI_ACCUM) tma_reduce_add_2d(&tmY, p8, x, m0 + c);
+          if (add_out) tma_reduce_add_2d(&tmY, p8, x, m0 + c);
           else tma_store_2d(&tmY, p8, x, m0 + c);
         }
         bulk_commit();
       }
     }
-    __syncwarp();
-    if (!plain) cluster_sync_all();                       // peers have finished reading this CTA's partial
   }
   if (warp >= 2 && lane == 0) bulk_wait_read();
 
@@ -600,7 +613,8 @@ int pick_split(int tiles, int KB, int sms) {
 int make_out_map(CUtensorMap *out, void *base, uint64_t rows, uint64_t cols, uint64_t ld, bool bf16);
 
 template <int BNB>
-cudaError_t launch_cluster_variant(const GemmArgs &a, int n_tiles, int m_tiles, int split, cudaStream_t stream) {
+cudaError_t launch_cluster_variant(const GemmArgs &a, int n_tiles, int m_tiles, int split, bool independent,
+                                   cudaStream_t stream) {
   using S = GemmSmem<BNB>;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_tiles * split, m_tiles, 1);
@@ -609,7 +623,7 @@ cudaError_t launch_cluster_variant(const GemmArgs &a, int n_tiles, int m_tiles, 
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = split;
+  attr[0].val.clusterDim.x = independent ? 1 : split;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
@@ -618,7 +632,7 @@ cudaError_t launch_cluster_variant(const GemmArgs &a, int n_tiles, int m_tiles, 
   const bool gu = a.epilogue == EPI_SWIGLU;
   if (make_out_map(&tmY, a.Y, a.M, a.N, a.ldY, gu) != 0) return cudaErrorInvalidValue;
   return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<BNB>, *a.tmW, *a.tmX, tmY, a.M, a.N, a.K, a.epilogue, split,
-                            a.status);
+                            independent ? 1 : 0, a.status);
 }
 
 template <int BNB>
@@ -634,9 +648,17 @@ cudaError_t launch_variant(const GemmArgs &a, cudaStream_t stream) {
   int grid = g_num_sms > 0 ? g_num_sms : 148;
   const bool out_ok = (reinterpret_cast<uintptr_t>(a.Y) & 15) == 0 && (a.ldY * (gu ? 2 : 4)) % 16 == 0;
   if (out_ok && a.force_split >= 0 && (a.force_split > 0 || n_tiles * m_tiles < 2 * grid)) {
+    if (a.independent_splits && !gu) {
+      // as many k-slices as it takes to put a CTA on every SM (at least 4 k-blocks each)
+      int split = a.force_split > 0 ? a.force_split : grid / (n_tiles * m_tiles);
+      if (split > KB / 4) split = KB / 4;
+      if (split > 16) split = 16;
+      if (split < 1) split = 1;
+      return launch_cluster_variant<BNB>(a, n_tiles, m_tiles, split, split > 1, stream);
+    }
     const int split = a.force_split > 0 ? (a.force_split < KB ? a.force_split : KB)
                                         : pick_split(n_tiles * m_tiles, KB, grid);
-    return launch_cluster_variant<BNB>(a, n_tiles, m_tiles, split, stream);
+    return launch_cluster_variant<BNB>(a, n_tiles, m_tiles, split > 8 ? 8 : split, false, stream);
   }
   if (a.max_ctas > 0 && grid > a.max_ctas) grid = a.max_ctas;
   if (grid > total) grid = static_cast<int>(total);
@@ -825,6 +847,6 @@ extern "C" int echo_gemm_bf16_noalloc(const void *X, const void *W, void *Y, int
   if (make_tensor_map(&tmW, W, gu ? 2ull * N : N, K, K, gu ? 64 : kGemmTileN) != 0) return ECHO_ERR_CUDA;
   if (make_tensor_map(&tmX, X, M, K, K, kNoAllocMaxRows) != 0) return ECHO_ERR_CUDA;
   GemmArgs a{&tmW, &tmX, Y, N, M, N, K, kNoAllocMaxRows, epilogue, nullptr, reinterpret_cast<float *>(base),
-             counters, kNoAllocMaxCtas, -1};
+             counters, kNoAllocMaxCtas, -1, 0};
   return gemm_tc_launch(a, s) == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }

@@ -83,7 +83,8 @@ def test_gemm_tensor_core_matches_fp64(B, M, N, K):
     # fp32 accumulation of K products of magnitude ~0.05: error ~ K * 2^-24 * |terms|
     tol = 2e-6 * K * 0.05 * 4 + 1e-6
     # 1 = SIMT reference, 0 = automatic choice, 2 = persistent stream-K, 100+s = cluster split-K by s
-    impls = (1, 0, 2, 101, 103, 108) if N * K <= 4096 * 4096 else (0, 2)
+    # 200+s = independent k-slices added into the output in memory (s = 0: automatic)
+    impls = (1, 0, 2, 101, 103, 108, 200, 206) if N * K <= 4096 * 4096 else (0, 2, 200)
     for impl in impls:
         Y = B.echo_gemm_bf16(X.cuda(), W.cuda(), impl=impl)
         got = Y.cpu().numpy().astype(np.float64)
@@ -92,7 +93,7 @@ def test_gemm_tensor_core_matches_fp64(B, M, N, K):
     Y0 = torch.from_numpy(rng.normal(size=(M, N)).astype(np.float32)).cuda()
     Y = Y0.clone()
     B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=1, Y=Y, impl=2)
-    B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=1, Y=Y, impl=0)
+    B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=1, Y=Y, impl=200)
     got = Y.cpu().numpy().astype(np.float64)
     assert np.max(np.abs(got - (Y0.cpu().numpy() + 2 * want))) < 2 * tol + 1e-5
 

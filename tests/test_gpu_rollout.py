@@ -5,7 +5,7 @@ import torch
 
 from oracle import decoder, pages
 from paper_2602_02192_b200 import synth
-from helpers import check_sequences, dims_of
+from helpers import assert_same_rollout, check_sequences, dims_of
 
 pytestmark = pytest.mark.gpu
 
@@ -57,7 +57,7 @@ def test_tiny_config_full_parity(B, tiny):
     tok2, lp2, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, wl.G, wl.new_tokens,
                                     wl.temperature, wl.sample_seed)
     eng.echo_sync()
-    assert np.array_equal(tok2.cpu().numpy(), tok) and np.array_equal(lp2.cpu().numpy(), lp)
+    assert_same_rollout(tok2.cpu().numpy(), lp2.cpu().numpy(), tok, lp)
     st = eng.echo_get_stats()
     assert st["tokens_generated"] == tok.size and st["kernels_launched"] > 100
     eng.close()
@@ -152,17 +152,19 @@ def test_versions_and_double_buffer(B, tiny):
     eng.echo_wait_policy()
     t2, l2, v2 = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
     eng.echo_sync()
-    assert np.all(v2 == 12) and np.array_equal(t2.cpu().numpy(), t0.cpu().numpy())
+    assert np.all(v2 == 12)
+    assert_same_rollout(t2.cpu().numpy(), l2.cpu().numpy(), t0.cpu().numpy(), l0.cpu().numpy())
     eng.close()
     # single buffer: the next rollout waits for the install and serves the new version
     eng = _engine(B, wl.shape, P, G, Lp, T, nbuf=1)
     eng.echo_load_policy(w_d, 0)
-    ta, _, va = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
+    ta, la, va = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
     eng.echo_load_policy(w1_d, 1)
-    tb, _, vb = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
+    tb, lb, vb = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 7)
     eng.echo_sync()
     assert np.all(va == 0) and np.all(vb == 1)
-    assert np.array_equal(ta.cpu().numpy(), t0.cpu().numpy()) and np.array_equal(tb.cpu().numpy(), t1.cpu().numpy())
+    assert_same_rollout(ta.cpu().numpy(), la.cpu().numpy(), t0.cpu().numpy(), l0.cpu().numpy())
+    assert_same_rollout(tb.cpu().numpy(), lb.cpu().numpy(), t1.cpu().numpy(), l1.cpu().numpy())
     eng.close()
 
 
@@ -179,5 +181,5 @@ def test_host_buffer_entry_point(B, tiny):
     assert np.all(ver == 0)
     tok, lp, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), [Lp] * P, G, T, 1.0, 3)
     eng.echo_sync()
-    assert np.array_equal(ht.numpy(), tok.cpu().numpy()) and np.array_equal(hl.numpy(), lp.cpu().numpy())
+    assert_same_rollout(ht.numpy(), hl.numpy(), tok.cpu().numpy(), lp.cpu().numpy())
     eng.close()
