@@ -280,25 +280,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
   }
   __syncthreads();
 
-  // ---- Q fragments (A operand), kept in registers for the whole loop ---------------------------
-  uint32_t qf[KSTEPS][4];
-  {
-    const int s_lo = row_seq(quad), s_hi = row_seq(quad + 8);
-    const uint32_t *q_lo = s_lo >= 0 ? reinterpret_cast<const uint32_t *>(
-                                           q + (static_cast<size_t>(s_lo) * Hq + row_head(quad)) * HD)
-                                     : nullptr;
-    const uint32_t *q_hi = s_hi >= 0 ? reinterpret_cast<const uint32_t *>(
-                                           q + (static_cast<size_t>(s_hi) * Hq + row_head(quad + 8)) * HD)
-                                     : nullptr;
-#pragma unroll
-    for (int kk = 0; kk < KSTEPS; ++kk) {
-      qf[kk][0] = q_lo ? q_lo[kk * 8 + qi] : 0u;
-      qf[kk][1] = q_hi ? q_hi[kk * 8 + qi] : 0u;
-      qf[kk][2] = q_lo ? q_lo[kk * 8 + 4 + qi] : 0u;
-      qf[kk][3] = q_hi ? q_hi[kk * 8 + 4 + qi] : 0u;
-    }
-  }
-
   float o_acc[HD / 8][4];
 #pragma unroll
   for (int i = 0; i < HD / 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
@@ -336,6 +317,47 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
 
   const int n_pro = n_my < kDecStages ? n_my : kDecStages;
   for (int k = 0; k < n_pro; ++k) issue(k);
+
+  // (the first pages are on their way; everything below overlaps their latency)
+  // prefix partials this thread will merge at the end (suffix kernel): fetched now, used last
+  constexpr int kPre = 4;
+  float pre_val[kPre];
+  float2 pre_stat[kPre];
+  const bool pre_ok = !PREFIX && REP * HD <= kPre * kDecWarps * 32;
+  if (pre_ok) {
+#pragma unroll
+    for (int i = 0; i < kPre; ++i) {
+      const int idx = threadIdx.x + i * kDecWarps * 32;
+      pre_val[i] = 0.f;
+      pre_stat[i] = make_float2(-INFINITY, 0.f);
+      if (idx < REP * HD) {
+        const int r = idx / HD, d = idx % HD;
+        const size_t rh = static_cast<size_t>(seq0) * Hq + h * REP + r;
+        pre_stat[i] = pre_ml[rh];
+        pre_val[i] = pre_o[rh * HD + d];
+      }
+    }
+  }
+
+  // ---- Q fragments (A operand), kept in registers for the whole loop ---------------------------
+  uint32_t qf[KSTEPS][4];
+  {
+    const int s_lo = row_seq(quad), s_hi = row_seq(quad + 8);
+    const uint32_t *q_lo = s_lo >= 0 ? reinterpret_cast<const uint32_t *>(
+                                           q + (static_cast<size_t>(s_lo) * Hq + row_head(quad)) * HD)
+                                     : nullptr;
+    const uint32_t *q_hi = s_hi >= 0 ? reinterpret_cast<const uint32_t *>(
+                                           q + (static_cast<size_t>(s_hi) * Hq + row_head(quad + 8)) * HD)
+                                     : nullptr;
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+      qf[kk][0] = q_lo ? q_lo[kk * 8 + qi] : 0u;
+      qf[kk][1] = q_hi ? q_hi[kk * 8 + qi] : 0u;
+      qf[kk][2] = q_lo ? q_lo[kk * 8 + 4 + qi] : 0u;
+      qf[kk][3] = q_hi ? q_hi[kk * 8 + 4 + qi] : 0u;
+    }
+  }
+
 
   bool ok = true;
   for (int k = 0; k < n_my; ++k) {
@@ -476,13 +498,28 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
       pre_o[oi] = O;
       if (d == 0) pre_ml[static_cast<size_t>(s) * Hq + row_head(r)] = make_float2(M, L);
     } else {
-      const float2 ml = pre_ml[static_cast<size_t>(s) * Hq + row_head(r)];
+      const int it = idx / (kDecWarps * 32);
+      float2 ml;
+      float po;
+      if (pre_ok) {
+        ml = pre_stat[0];
+        po = pre_val[0];
+#pragma unroll
+        for (int i = 1; i < kPre; ++i)
+          if (it == i) {
+            ml = pre_stat[i];
+            po = pre_val[i];
+          }
+      } else {
+        ml = pre_ml[static_cast<size_t>(s) * Hq + row_head(r)];
+        po = pre_o[oi];
+      }
       float Mt = fmaxf(M, ml.x);
       if (Mt == -INFINITY) Mt = 0.f;
       const float c_suf = M == -INFINITY ? 0.f : exp2f(M - Mt);
       const float c_pre = ml.x == -INFINITY ? 0.f : exp2f(ml.x - Mt);
       const float Lt = L * c_suf + ml.y * c_pre;
-      const float Ot = O * c_suf + (c_pre != 0.f ? pre_o[oi] * c_pre : 0.f);
+      const float Ot = O * c_suf + (c_pre != 0.f ? po * c_pre : 0.f);
       out[oi] = __float2bfloat16(Ot / Lt);
     }
   }

@@ -119,9 +119,10 @@ __global__ void rope_table_kernel(float2 *table, int max_pos, int half, double t
 
 // One block per activation row.  Rotates q and k heads (pairs (i, i + hd/2)), writes q as
 // bf16 and k, v as bf16 into the row's page slot.
-__global__ void rope_append_kernel(const float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer,
-                                   const float2 *rope_table, const int32_t *row_pt, const int32_t *row_pos,
-                                   const int32_t *page_table, int pt_width, int R, int Hq, int Hkv, int hd,
+__global__ void rope_append_kernel(const float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q,
+                                   __nv_bfloat16 *__restrict__ kv_layer, const float2 *__restrict__ rope_table,
+                                   const int32_t *__restrict__ row_pt, const int32_t *__restrict__ row_pos,
+                                   const int32_t *__restrict__ page_table, int pt_width, int R, int Hq, int Hkv, int hd,
                                    int page_size, int n_pages, int max_pos, int *status) {
   const int r = blockIdx.x;
   const int pos = row_pos[r];
@@ -140,6 +141,7 @@ __global__ void rope_append_kernel(const float *qkv, __nv_bfloat16 *q, __nv_bflo
   }
   const float2 *cs = rope_table + static_cast<size_t>(pos) * half;
   // q heads
+#pragma unroll 4
   for (int idx = threadIdx.x; idx < Hq * half; idx += blockDim.x) {
     const int head = idx / half, i = idx % half;
     const float a = src[head * hd + i], b = src[head * hd + i + half];
@@ -150,6 +152,7 @@ __global__ void rope_append_kernel(const float *qkv, __nv_bfloat16 *q, __nv_bflo
   }
   // k heads (rotated) and v heads (plain) into the page slot
   const size_t page_elems = static_cast<size_t>(page_size) * hd;
+#pragma unroll 2
   for (int idx = threadIdx.x; idx < Hkv * half; idx += blockDim.x) {
     const int head = idx / half, i = idx % half;
     const float *ks = src + (Hq + head) * hd;
