@@ -273,6 +273,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
   };
   auto row_head = [&](int r) -> int { return h * REP + (PREFIX ? (mt * 16 + r) % REP : r); };
 
+  if (!PREFIX) griddep_launch();             // the output projection may start prefetching its weights
   if (threadIdx.x == 0) {
     for (int i = 0; i < kDecWarps * kDecStages; ++i) mbar_init(&bars[i], 1);
     *abort_flag = 0;

@@ -46,6 +46,7 @@ struct GemmArgs {
   int *counters;      // kGemmMaxUnits ints, zero before the first launch (the kernel re-zeroes them)
   int max_ctas;       // 0 = one CTA per SM
   int force_split;    // 0 = choose; k > 0 = split-K by k; -1 = always the persistent stream-K kernel
+  int allow_early_start;    // 1: launch with programmatic stream serialization (see gemm.cu)
   int independent_splits;   // 1: k-slices add into Y in memory (Y must hold zeros for EPI_STORE; the order of
                             // the additions is not fixed); 0: slices are reduced in rank order inside a cluster
 };

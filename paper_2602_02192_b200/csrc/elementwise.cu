@@ -64,6 +64,8 @@ __global__ void __launch_bounds__(kNormThreads)
 rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ gain, __nv_bfloat16 *__restrict__ h,
                int R, int d, float eps) {
   __shared__ float scratch[32];
+  // lets a projection launched with programmatic serialization begin its weight prefetch now
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int r = blockIdx.x;
   const float *xr = x + static_cast<size_t>(r) * d;
   __nv_bfloat16 *hr = h + static_cast<size_t>(r) * d;

@@ -79,10 +79,10 @@ __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"
 // Loads of one k-block: kAcc weight blocks (each 128 rows, or 64 gate + 64 up rows) and the
 // activation tile.
 template <int BNB>
-__device__ __forceinline__ void load_stage(const CUtensorMap *tmW, const CUtensorMap *tmX, uint64_t *bar,
-                                           uint8_t *stage, int kb, int nt, int m0, int N, bool gu) {
+__device__ __forceinline__ void load_stage_w(const CUtensorMap *tmW, uint64_t *bar, uint8_t *stage, int kb, int nt,
+                                             int N, bool gu) {
   using S = GemmSmem<BNB>;
-  mbar_expect_tx(bar, S::kStageBytes);
+  mbar_expect_tx(bar, S::kStageBytes);                 // covers the activation tile loaded afterwards as well
 #pragma unroll
   for (int a = 0; a < kAcc; ++a) {
     uint8_t *dst = stage + a * S::kWBlock;
@@ -94,7 +94,16 @@ __device__ __forceinline__ void load_stage(const CUtensorMap *tmW, const CUtenso
       tma_load_2d(tmW, bar, dst, kb * kGemmTileK, (nt * kAcc + a) * kGemmTileN);
     }
   }
-  tma_load_2d(tmX, bar, stage + S::kWBytes, kb * kGemmTileK, m0);
+}
+template <int BNB>
+__device__ __forceinline__ void load_stage_x(const CUtensorMap *tmX, uint64_t *bar, uint8_t *stage, int kb, int m0) {
+  tma_load_2d(tmX, bar, stage + GemmSmem<BNB>::kWBytes, kb * kGemmTileK, m0);
+}
+template <int BNB>
+__device__ __forceinline__ void load_stage(const CUtensorMap *tmW, const CUtensorMap *tmX, uint64_t *bar,
+                                           uint8_t *stage, int kb, int nt, int m0, int N, bool gu) {
+  load_stage_w<BNB>(tmW, bar, stage, kb, nt, N, gu);
+  load_stage_x<BNB>(tmX, bar, stage, kb, m0);
 }
 
 template <int BNB>
@@ -422,13 +431,21 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  griddep_wait();
+  griddep_launch();        // the next kernel may start its own prologue and weight prefetch
 
   if (warp == 0) {
     if (lane == 0) {
-      int it = 0;
+      // Weights do not depend on the preceding kernel: fill the pipeline with weight tiles first,
+      // then wait for that kernel to finish before touching the activations it wrote.
+      const int n_pre = kb_len < S::kStages ? kb_len : S::kStages;
+      for (int it = 0; it < n_pre; ++it)
+        load_stage_w<BNB>(&tmW, &full_bar[it], smem + it * S::kStageBytes, kb_beg + it, nt, N, gu);
+      griddep_wait();
+      for (int it = 0; it < n_pre; ++it)
+        load_stage_x<BNB>(&tmX, &full_bar[it], smem + it * S::kStageBytes, kb_beg + it, m0);
+      int it = n_pre;
       bool ok = true;
-      for (int kb = kb_beg; kb < kb_beg + kb_len; ++kb, ++it) {
+      for (int kb = kb_beg + n_pre; kb < kb_beg + kb_len; ++kb, ++it) {
         const int s = it % S::kStages;
         ok = mbar_wait(&empty_bar[s], ((it / S::kStages) & 1) ^ 1u, abort_flag);
         if (!ok) break;
@@ -621,13 +638,17 @@ cudaError_t launch_cluster_variant(const GemmArgs &a, int n_tiles, int m_tiles, 
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = S::kTotal;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = independent ? 1 : split;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // programmatic dependent launch: this kernel may begin (prologue, weight prefetch) while the
+  // preceding kernel drains; it waits for that kernel's results before loading activations
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = a.allow_early_start ? 2 : 1;
   CUtensorMap tmY;
   const bool gu = a.epilogue == EPI_SWIGLU;
   if (make_out_map(&tmY, a.Y, a.M, a.N, a.ldY, gu) != 0) return cudaErrorInvalidValue;
@@ -847,6 +868,6 @@ extern "C" int echo_gemm_bf16_noalloc(const void *X, const void *W, void *Y, int
   if (make_tensor_map(&tmW, W, gu ? 2ull * N : N, K, K, gu ? 64 : kGemmTileN) != 0) return ECHO_ERR_CUDA;
   if (make_tensor_map(&tmX, X, M, K, K, kNoAllocMaxRows) != 0) return ECHO_ERR_CUDA;
   GemmArgs a{&tmW, &tmX, Y, N, M, N, K, kNoAllocMaxRows, epilogue, nullptr, reinterpret_cast<float *>(base),
-             counters, kNoAllocMaxCtas, -1, 0};
+             counters, kNoAllocMaxCtas, -1, 0, 0};
   return gemm_tc_launch(a, s) == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }

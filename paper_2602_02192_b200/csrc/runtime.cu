@@ -170,7 +170,7 @@ struct echo_ctx {
   int last_rows = 0, last_width = 0;
   echo_stats stats{};
   int64_t launches = 0;
-  bool use_simt = false, use_graph = true, fast_decode = false, deterministic = false;
+  bool use_simt = false, use_graph = true, fast_decode = false, deterministic = false, use_pdl = true;
   CUtensorMap tm_kv;
   std::string last_error;
   // sampled per-kernel timing (echo_profile_config / echo_profile_read)
@@ -276,10 +276,14 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
     return ECHO_ERR_CUDA;
   }
   GemmArgs a{tmW, &tmX, Y, ldY, M, N, K, bnb, epilogue, ctx->ptr<int>(ctx->lo.status),
-             ctx->ptr<float>(ctx->lo.gemm_ws), ctx->ptr<int>(ctx->lo.gemm_counters), kMaxCtas, 0,
+             ctx->ptr<float>(ctx->lo.gemm_ws), ctx->ptr<int>(ctx->lo.gemm_counters), kMaxCtas, 0, ctx->use_pdl ? 1 : 0,
              ctx->deterministic ? 0 : 1};
-  if (a.independent_splits && epilogue == EPI_STORE && N < 8 * 4096)
+  if (a.independent_splits && epilogue == EPI_STORE && N < 8 * 4096) {
+    // the k-slices add into Y: it must start at zero.  The memset is the GEMM's predecessor on the
+    // stream, so this launch does not use the early start.
     CK(cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * ldY * sizeof(float), ctx->stream));
+    a.allow_early_start = 0;
+  }
   LAUNCH(gemm_tc_launch(a, ctx->stream));
   return ECHO_OK;
 }
@@ -679,6 +683,8 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
   ctx->use_graph = !(ng && ng[0] == '1');
   const char *det = getenv("ECHO_DETERMINISTIC");
   ctx->deterministic = det && det[0] == '1';
+  const char *pdl = getenv("ECHO_NO_PDL");
+  ctx->use_pdl = !(pdl && pdl[0] == '1');
 
   auto bail = [&](cudaError_t e, const char *what) {
     fail_cuda(ctx, e, what);
@@ -1007,7 +1013,7 @@ int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, 
   if (indep && epilogue == EPI_STORE &&
       cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * N * sizeof(float), s) != cudaSuccess)
     return ECHO_ERR_CUDA;
-  GemmArgs a{&tmW, &tmX, Y, N, M, N, K, bnb, epilogue, nullptr, static_cast<float *>(workspace), counters, 0, split,
+  GemmArgs a{&tmW, &tmX, Y, N, M, N, K, bnb, epilogue, nullptr, static_cast<float *>(workspace), counters, 0, split, 0,
              indep ? 1 : 0};
   cudaError_t e = gemm_tc_launch(a, s);
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
