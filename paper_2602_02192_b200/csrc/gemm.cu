@@ -9,13 +9,20 @@
 // rows, which is what a decode step (a few hundred rows against gigabytes of weights)
 // needs; the activation tile is re-read from L2.
 //
-// The kernel is persistent (one CTA per SM) and splits the work stream-K fashion: the
-// list of (output tile, k-block) pairs is cut into equal contiguous ranges, one per CTA,
-// so that every SM streams the same number of weight bytes whatever N and K are.  A CTA
-// whose range covers only part of a tile's k-blocks writes its partial accumulator to a
-// per-CTA workspace slot; the CTA that finishes a tile last (an atomic counter per tile,
-// no waiting) sums the partials in k order and applies the epilogue, so results do not
-// depend on timing.
+// Two kernels share the main loop.  A decode step's projections are 5-30 us of weight
+// streaming each, with 16-96 output tiles for 148 SMs, so both split tiles along K:
+//   gemm_cluster_kernel   one CTA per (tile, k-slice).  By default the slices of a tile add their
+//                         partial tiles into the output in memory (TMA reduce-add; the order of
+//                         the fp32 additions is not fixed); alternatively the slices form a
+//                         thread-block cluster and are summed in rank order through distributed
+//                         shared memory (bit-reproducible, slower).  Launched with programmatic
+//                         stream serialization: weight tiles are prefetched before the kernel
+//                         waits for its predecessor, activations after.
+//   gemm_streamk_kernel   persistent, one CTA per SM, for many-tile problems (the lm_head): the
+//                         list of (tile, k-block) pairs is cut into equal contiguous ranges; a CTA
+//                         that covers only part of a tile writes its partial to a workspace slot,
+//                         and the CTA that finishes a tile last (an atomic counter per tile, no
+//                         waiting) sums the partials in k order and applies the epilogue.
 //
 // A CTA's output tile is two 128-lane accumulators (256 features) against one activation
 // tile, so that the activation bytes an SM pulls from L2 do not exceed the weight bytes it
