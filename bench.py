@@ -134,6 +134,28 @@ def rollout_roofline_seconds(shape, P, G, Lp, T, bw_gbs, tflops):
 
 
 # ---------------------------------------------------------------------------------------------
+# multi-GPU: independent replicas (no data-path collective); helpers shared with the CPU tests
+# ---------------------------------------------------------------------------------------------
+def rank_prompt_seed(base_seed: int, rank: int) -> int:
+    """Every rank works on its own prompts (groups are never split across ranks)."""
+    return base_seed + 7919 * rank
+
+
+def max_over_ranks(value: float, device, world: int) -> float:
+    """The job's time is the slowest rank's time."""
+    if world == 1:
+        return float(value)
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_second(tokens_per_rank_step: int, world: int, steps: int, elapsed_ms: float) -> float:
+    return world * steps * tokens_per_rank_step / (elapsed_ms / 1e3)
+
+
+# ---------------------------------------------------------------------------------------------
 def run_ours(args):
     from paper_2602_02192_b200 import binding, synth
 
@@ -158,7 +180,11 @@ def run_ours(args):
     swap = args.workload == "8B" and not args.no_swap
     nbuf = 1 if args.workload == "32B" else 2
     eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, nbuf), device=local_rank)
-    weights = synth.make_weights(shape, wl.weight_seed, device=dev)
+    if args.workload == "32B":
+        # 65 GB of weights: the snapshot stays in page-locked host memory so that the device holds it once
+        weights = synth.make_weights_pinned(shape, wl.weight_seed, gen_device=dev)
+    else:
+        weights = synth.make_weights(shape, wl.weight_seed, device=dev)
     eng.echo_load_policy(weights, 0)
     eng.echo_wait_policy()
     w_next = None
@@ -169,7 +195,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     # every rank is an independent replica working on its own prompts (groups never split)
-    prompts = torch.from_numpy(synth.make_prompts(P, Lp, shape.vocab, wl.prompt_seed + 7919 * rank)).to(dev)
+    prompts = torch.from_numpy(synth.make_prompts(P, Lp, shape.vocab, rank_prompt_seed(wl.prompt_seed, rank))).to(dev)
     lens = [Lp] * P
     out_tok = torch.empty((P, G, T), dtype=torch.int32, device=dev)
     out_lp = torch.empty((P, G, T), dtype=torch.float32, device=dev)
@@ -211,12 +237,8 @@ def run_ours(args):
     prof_steps, prof_ms = eng.echo_profile_read()
     eng.echo_profile_config(0)
     install_ms = eng.echo_get_stats()["install_ms"]
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
-    tokens_total = world * args.steps * P * G * T
-    value = tokens_total / (elapsed_ms / 1e3)
+    elapsed_ms = max_over_ranks(elapsed_ms, dev, world)
+    value = job_tokens_per_second(P * G * T, world, args.steps, elapsed_ms)
 
     # ---- end to end: host buffers, copies inside the timed region -------------------------
     hp = prompts.cpu().pin_memory()
@@ -227,11 +249,8 @@ def run_ours(args):
     ver_e2e = eng.echo_rollout_host(hp, lens, G, T, wl.temperature, wl.sample_seed + 999, ht, hl)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = world * P * G * T / e2e_s
+    e2e_s = max_over_ranks(e2e_s, dev, world)
+    e2e_value = job_tokens_per_second(P * G * T, world, 1, e2e_s * 1e3)
 
     if rank != 0:
         if world > 1:

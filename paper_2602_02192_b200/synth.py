@@ -126,6 +126,21 @@ def make_weights(shape: DecoderShape, weight_seed: int = 0, device: str = "cpu",
     return w
 
 
+def make_weights_pinned(shape: DecoderShape, weight_seed: int = 0, gen_device: str = "cuda",
+                        std: float = 0.02) -> dict:
+    """Same tensors as make_weights(device=gen_device), generated one at a time on gen_device and
+    kept in page-locked host memory: for shapes whose snapshot must not take device memory twice."""
+    def one(name, layer):
+        t = make_tensor(shape, name, layer, weight_seed, gen_device, std)
+        host = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+        host.copy_(t)
+        return host
+    w = {n: one(n, -1) for n in GLOBAL_TENSORS}
+    for n in LAYER_TENSORS:
+        w[n] = [one(n, l) for l in range(shape.n_layers)]
+    return w
+
+
 def bf16_bits(t: torch.Tensor) -> np.ndarray:
     """bf16 tensor → numpy uint16 array of its bit patterns (on the host)."""
     return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)

@@ -1,0 +1,61 @@
+"""The N > 1 path of the benchmark is N independent replicas: each rank takes its own prompts, no
+data-path collective, and the job's time is the slowest rank's.  Covered here with two gloo ranks
+on the CPU (no GPU needed)."""
+import os
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    import bench
+    from oracle import advantage
+    from paper_2602_02192_b200 import synth
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    prompts = synth.make_prompts(4, 8, 4096, bench.rank_prompt_seed(1001, rank))
+    gathered = [torch.zeros(4, 8, dtype=torch.int32) for _ in range(world)]
+    dist.all_gather(gathered, torch.from_numpy(prompts))
+    distinct = all(not torch.equal(gathered[i], gathered[j]) for i in range(world) for j in range(i + 1, world))
+    # each rank is slower or faster; the job's time is the maximum
+    elapsed = bench.max_over_ranks(100.0 * (rank + 1), "cpu", world)
+    value = bench.job_tokens_per_second(4 * 4 * 32, world, 3, elapsed)
+    # groups never cross ranks, so group-normalised rewards need nothing from another rank
+    rewards = synth.make_rewards(4, 4, 7 + rank)
+    adv_local = advantage.group_advantage(rewards)
+    all_rewards = [torch.zeros(4, 4, dtype=torch.float32) for _ in range(world)]
+    dist.all_gather(all_rewards, torch.from_numpy(rewards))
+    adv_global = advantage.group_advantage(torch.cat(all_rewards).numpy())
+    same_adv = np.allclose(adv_global[4 * rank: 4 * rank + 4], adv_local)
+    dist.barrier()
+    out[rank] = (distinct, elapsed, value, same_adv)
+    dist.destroy_process_group()
+
+
+def test_two_replica_ranks_on_gloo():
+    world = 2
+    port = 29500 + os.getpid() % 2000
+    mgr = mp.get_context("spawn").Manager()
+    out = mgr.dict()
+    mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
+    assert len(out) == world
+    for rank in range(world):
+        distinct, elapsed, value, same_adv = out[rank]
+        assert distinct and same_adv
+        assert elapsed == 200.0                                   # max over ranks
+        assert abs(value - 2 * 3 * 512 / 0.2) < 1e-6              # whole-job tokens / slowest rank's time
+
+
+def test_reference_arm_is_rank_zero_only(monkeypatch, capsys):
+    sys.path.insert(0, ROOT)
+    import bench
+    monkeypatch.setenv("RANK", "1")
+    bench.run_reference(type("A", (), {"workload": "tiny", "warmup": 1, "steps": 1, "gpus": 2})())
+    assert capsys.readouterr().out == ""
