@@ -71,8 +71,9 @@ cudaError_t embed_launch(const __nv_bfloat16 *embed, const int32_t *tok_src, con
 cudaError_t rmsnorm_launch(const float *x, const __nv_bfloat16 *gain, __nv_bfloat16 *h, int R, int d,
                            float eps, cudaStream_t s);
 cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double theta, cudaStream_t s);
-// qkv fp32 [R][(Hq+2Hkv)*hd] -> q bf16 [R][Hq*hd], K/V into the paged cache of one layer
-cudaError_t rope_append_launch(const float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer,
+// qkv fp32 [R][(Hq+2Hkv)*hd] -> q bf16 [R][Hq*hd], K/V into the paged cache of one layer; the rows
+// of qkv it consumes are left holding zeros
+cudaError_t rope_append_launch(float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer,
                                const float2 *rope_table, RowMeta meta, const int32_t *page_table,
                                int pt_width, int R, int Hq, int Hkv, int hd, int page_size,
                                int n_pages, int max_pos, int *status, cudaStream_t s);

@@ -121,7 +121,7 @@ __global__ void rope_table_kernel(float2 *table, int max_pos, int half, double t
 
 // One block per activation row.  Rotates q and k heads (pairs (i, i + hd/2)), writes q as
 // bf16 and k, v as bf16 into the row's page slot.
-__global__ void rope_append_kernel(const float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q,
+__global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q,
                                    __nv_bfloat16 *__restrict__ kv_layer, const float2 *__restrict__ rope_table,
                                    const int32_t *__restrict__ row_pt, const int32_t *__restrict__ row_pos,
                                    const int32_t *__restrict__ page_table, int pt_width, int R, int Hq, int Hkv, int hd,
@@ -130,15 +130,17 @@ __global__ void rope_append_kernel(const float *__restrict__ qkv, __nv_bfloat16 
   const int pos = row_pos[r];
   const int half = hd / 2;
   const int ld = (Hq + 2 * Hkv) * hd;
-  const float *src = qkv + static_cast<size_t>(r) * ld;
+  float *src = qkv + static_cast<size_t>(r) * ld;
   if (pos < 0 || pos >= max_pos) {
     if (threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
+    for (int i = threadIdx.x; i < ld; i += blockDim.x) src[i] = 0.f;      // keep the buffer's zero invariant
     return;
   }
   const int page = page_table[static_cast<size_t>(row_pt[r]) * pt_width + pos / page_size];
   const int off = pos % page_size;
   if (page < 0 || page >= n_pages) {
     if (threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
+    for (int i = threadIdx.x; i < ld; i += blockDim.x) src[i] = 0.f;
     return;
   }
   const float2 *cs = rope_table + static_cast<size_t>(pos) * half;
@@ -157,8 +159,8 @@ __global__ void rope_append_kernel(const float *__restrict__ qkv, __nv_bfloat16 
 #pragma unroll 2
   for (int idx = threadIdx.x; idx < Hkv * half; idx += blockDim.x) {
     const int head = idx / half, i = idx % half;
-    const float *ks = src + (Hq + head) * hd;
-    const float *vs = src + (Hq + Hkv + head) * hd;
+    float *ks = src + (Hq + head) * hd;
+    float *vs = src + (Hq + Hkv + head) * hd;
     const float2 t = cs[i];
     __nv_bfloat16 *kd = kv_layer + ((static_cast<size_t>(page) * Hkv + head) * 2 + 0) * page_elems + off * hd;
     __nv_bfloat16 *vd = kd + page_elems;
@@ -167,6 +169,15 @@ __global__ void rope_append_kernel(const float *__restrict__ qkv, __nv_bfloat16 
     kd[i + half] = __float2bfloat16(b * t.x + a * t.y);
     vd[i] = __float2bfloat16(vs[i]);
     vd[i + half] = __float2bfloat16(vs[i + half]);
+  }
+  // the row is consumed: leave zeros for the next projection, whose k-slices add into this buffer
+  // (a separate pass, so that the loads above are not ordered behind stores to the same array)
+  __syncthreads();
+  if ((ld & 3) == 0) {
+    float4 *z = reinterpret_cast<float4 *>(src);
+    for (int i = threadIdx.x; i < ld / 4; i += blockDim.x) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  } else {
+    for (int i = threadIdx.x; i < ld; i += blockDim.x) src[i] = 0.f;
   }
 }
 
@@ -366,7 +377,7 @@ cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double t
   rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(table, max_pos, half, theta, head_dim);
   return cudaGetLastError();
 }
-cudaError_t rope_append_launch(const float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer, const float2 *rope_table,
+cudaError_t rope_append_launch(float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer, const float2 *rope_table,
                                RowMeta meta, const int32_t *page_table, int pt_width, int R, int Hq, int Hkv, int hd,
                                int page_size, int n_pages, int max_pos, int *status, cudaStream_t s) {
   rope_append_kernel<<<R, 256, 0, s>>>(qkv, q, kv_layer, rope_table, meta.row_pt, meta.row_pos, page_table, pt_width,

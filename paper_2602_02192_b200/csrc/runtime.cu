@@ -257,7 +257,7 @@ int pick_bnb(int rows) {
 
 // Y = X * W^T through the tensor-core kernel (or the SIMT reference when selected).
 int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, const __nv_bfloat16 *X, void *Y, int ldY,
-             int M, int N, int K, int epilogue) {
+             int M, int N, int K, int epilogue, bool y_holds_zeros = false) {
   ProfScope prof(ctx, PROF_GEMM);
   if (ctx->use_simt) {
     if (epilogue == EPI_SWIGLU) {
@@ -278,7 +278,7 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
   GemmArgs a{tmW, &tmX, Y, ldY, M, N, K, bnb, epilogue, ctx->ptr<int>(ctx->lo.status),
              ctx->ptr<float>(ctx->lo.gemm_ws), ctx->ptr<int>(ctx->lo.gemm_counters), kMaxCtas, 0, ctx->use_pdl ? 1 : 0,
              ctx->deterministic ? 0 : 1};
-  if (a.independent_splits && epilogue == EPI_STORE && N < 8 * 4096) {
+  if (a.independent_splits && epilogue == EPI_STORE && N < 8 * 4096 && !y_holds_zeros) {
     // the k-slices add into Y: it must start at zero.  The memset is the GEMM's predecessor on the
     // stream, so this launch does not use the early start.
     CK(cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * ldY * sizeof(float), ctx->stream));
@@ -310,7 +310,8 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int d
   for (int l = 0; l < D.L; ++l) {
     __nv_bfloat16 *kv_layer = ctx->ptr<__nv_bfloat16>(lo.kv) + static_cast<size_t>(l) * lo.kv_layer_elems;
     LAUNCH(rmsnorm_launch(x, w.attn_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream));
-    TRY(run_gemm(ctx, &w.tm_qkv[l], w.wqkv[l], h, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE));
+    // the qkv buffer holds zeros here: rope_append clears every row it consumes
+    TRY(run_gemm(ctx, &w.tm_qkv[l], w.wqkv[l], h, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE, !ctx->use_simt));
     LAUNCH(rope_append_launch(qkv, q, kv_layer, rope, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
                               ctx->M.n_pages, ctx->M.max_pos, status, ctx->stream));
     if (decode_P > 0 && ctx->fast_decode) {
@@ -739,6 +740,9 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
   }
   if ((e = cudaMemsetAsync(ctx->arena + lo.status, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
   if ((e = cudaMemsetAsync(ctx->arena + lo.d_step, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
+  if ((e = cudaMemsetAsync(ctx->arena + lo.qkv, 0, static_cast<size_t>(ctx->M.R) * ctx->D.n_qkv() * 4, ctx->stream)) !=
+      cudaSuccess)
+    return bail(e, "cudaMemset");
   if ((e = cudaMemsetAsync(ctx->arena + lo.gemm_counters, 0, static_cast<size_t>(kGemmMaxUnits) * 4, ctx->stream)) !=
       cudaSuccess)
     return bail(e, "cudaMemset");
