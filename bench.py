@@ -236,7 +236,8 @@ def run_ours(args):
     clk = clocks.stop() if rank == 0 else None
     prof_steps, prof_ms = eng.echo_profile_read()
     eng.echo_profile_config(0)
-    install_ms = eng.echo_get_stats()["install_ms"]
+    st_last = eng.echo_get_stats()
+    install_ms = st_last["install_ms"]
     elapsed_ms = max_over_ranks(elapsed_ms, dev, world)
     value = job_tokens_per_second(P * G * T, world, args.steps, elapsed_ms)
 
@@ -295,6 +296,8 @@ def run_ours(args):
                    "policy_swap": "one echo_load_policy of a re-seeded weight set during timed step 0" if swap
                    else "none", "versions_served": versions_seen, "e2e_version": int(ver_e2e[0, 0]),
                    "install_ms": round(install_ms, 1),
+                   "last_rollout_prefill_ms": round(st_last["prefill_ms"], 1),
+                   "last_rollout_decode_ms_per_step": round(st_last["decode_ms"] / max(1, T - 1), 3),
                    "l2": "inputs larger than L2 (weights + KV >> 126 MB)", "parallelism": f"replicas x{world}"},
         "clocks": clk,
         "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": int(hp.numel() * 4),

@@ -87,6 +87,9 @@ typedef struct echo_stats {
   int64_t decode_steps;       /* T-1                                            */
   int64_t n_pages;            /* KV pages the plan used                         */
   float   install_ms;         /* duration of the last completed install (device) */
+  float   prefill_ms;         /* last rollout: prompt prefill + first token (device time; valid once
+                                 the rollout has finished, else 0)                                */
+  float   decode_ms;          /* last rollout: the T-1 decode steps (device time; same condition)  */
   float   reserved;
 } echo_stats;
 

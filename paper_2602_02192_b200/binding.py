@@ -53,7 +53,8 @@ class EchoWeights(C.Structure):
 class EchoStats(C.Structure):
     _fields_ = [
         ("version_served", C.c_int64), ("tokens_generated", C.c_int64), ("kernels_launched", C.c_int64),
-        ("decode_steps", C.c_int64), ("n_pages", C.c_int64), ("install_ms", C.c_float), ("reserved", C.c_float),
+        ("decode_steps", C.c_int64), ("n_pages", C.c_int64), ("install_ms", C.c_float), ("prefill_ms", C.c_float),
+        ("decode_ms", C.c_float), ("reserved", C.c_float),
     ]
 
 

@@ -527,7 +527,9 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     __syncwarp();
     if (!plain) {
-      cluster_sync_all();                                 // all partials of this accumulator are in place
+      // all partials of this accumulator are in place (a cluster of one only needs its own warps)
+      if (S_split > 1) cluster_sync_all();
+      else if (warp >= 2) epi_bar();
       if (warp >= 2 && a > 0) {
         if (lane == 0) bulk_wait_read();                  // TMA has read the previous result out of out_stage
         epi_bar();
@@ -593,7 +595,11 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
     }
     __syncwarp();
-    if (!plain) cluster_sync_all();                       // peers have finished reading this CTA's partial
+    // peers have finished reading this CTA's partial
+    if (!plain) {
+      if (S_split > 1) cluster_sync_all();
+      else if (warp >= 2) epi_bar();
+    }
     if (warp >= 2) {
       fence_proxy_async();
       epi_bar();

@@ -161,6 +161,7 @@ struct echo_ctx {
   int64_t newest_version = 0;
   bool any_version = false;
   cudaEvent_t plan_done = nullptr, all_done = nullptr;
+  cudaEvent_t ev_begin = nullptr, ev_first = nullptr, ev_end = nullptr;   // phases of the last rollout
   bool plan_in_flight = false;
   // pinned staging for the plan tables
   int32_t *h_tables = nullptr;
@@ -569,6 +570,7 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   float *x = ctx->ptr<float>(lo.x);
   int *status = ctx->ptr<int>(lo.status);
 
+  CK(cudaEventRecord(ctx->ev_begin, ctx->stream));
   // ---- prefill: once per prompt, in chunks of kChunkRows tokens -------------
   for (int c = 0; c < pl.n_chunks; ++c) {
     const int r0 = c * kChunkRows, R = std::min(kChunkRows, pl.n_tok - r0);
@@ -590,6 +592,7 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, D.V, G, nullptr, nullptr, 0, temperature, seed, forced, T,
                         out_tokens, out_logprobs, T, ctx->stream));
 
+  CK(cudaEventRecord(ctx->ev_first, ctx->stream));
   // ---- decode steps 1..T-1 ----------------------------------------------------
   const int32_t *tok_hist = forced ? forced : out_tokens;
   const int n_steps = T - 1;
@@ -634,8 +637,10 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   if (exec) cudaGraphExecDestroy(exec);      // executions already enqueued keep their resources
   if (graph) cudaGraphDestroy(graph);
   if (rc_steps != ECHO_OK) return rc_steps;
+  CK(cudaEventRecord(ctx->ev_end, ctx->stream));
   CK(cudaEventRecord(wp->last_use, ctx->stream));
   wp->used = true;
+  ctx->stats.prefill_ms = ctx->stats.decode_ms = 0.f;
 
   ctx->stats.version_served = w.version;
   ctx->stats.tokens_generated = static_cast<int64_t>(pl.B) * T;
@@ -712,6 +717,9 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
     return bail(e, "cudaEventCreate");
   if ((e = cudaEventCreateWithFlags(&ctx->all_done, cudaEventDisableTiming)) != cudaSuccess)
     return bail(e, "cudaEventCreate");
+  if ((e = cudaEventCreate(&ctx->ev_begin)) != cudaSuccess || (e = cudaEventCreate(&ctx->ev_first)) != cudaSuccess ||
+      (e = cudaEventCreate(&ctx->ev_end)) != cudaSuccess)
+    return bail(e, "cudaEventCreate");
   const Limits &M = ctx->M;
   ctx->h_tables_ints = static_cast<size_t>(M.B + M.P) * M.pt_width + 3ull * M.P * M.Lp +
                        static_cast<size_t>(lo.n_chunks_max) * M.P + 5ull * M.B;
@@ -768,6 +776,9 @@ int echo_destroy(echo_ctx *ctx) {
   }
   if (ctx->plan_done) cudaEventDestroy(ctx->plan_done);
   if (ctx->all_done) cudaEventDestroy(ctx->all_done);
+  if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
+  if (ctx->ev_first) cudaEventDestroy(ctx->ev_first);
+  if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
   if (ctx->h_tables) cudaFreeHost(ctx->h_tables);
   for (cudaEvent_t e : ctx->prof_pool) cudaEventDestroy(e);
   delete ctx;
@@ -910,6 +921,15 @@ int echo_sync(echo_ctx *ctx) {
 
 int echo_get_stats(echo_ctx *ctx, echo_stats *out) {
   if (!ctx || !out) return ECHO_ERR_INVALID;
+  if (ctx->ev_end && cudaEventQuery(ctx->ev_end) == cudaSuccess) {
+    float a = 0.f, b = 0.f;
+    if (cudaEventElapsedTime(&a, ctx->ev_begin, ctx->ev_first) == cudaSuccess &&
+        cudaEventElapsedTime(&b, ctx->ev_first, ctx->ev_end) == cudaSuccess) {
+      ctx->stats.prefill_ms = a;
+      ctx->stats.decode_ms = b;
+    }
+  }
+  cudaGetLastError();
   *out = ctx->stats;
   return ECHO_OK;
 }
