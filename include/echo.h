@@ -195,6 +195,15 @@ int echo_profile_read(echo_ctx *ctx, int32_t *steps, float *ms, int32_t capacity
  * query them.  n is the capacity of `out` in int32 elements. */
 int echo_debug_page_table(echo_ctx *ctx, int32_t *out, size_t n, int32_t *rows, int32_t *width);
 
+/* The KV page plan of a rollout, computed on the host without a context or a GPU (the same
+ * routine echo_rollout uses).  prompt_lens host int32 [P].  Writes out_table (host int32
+ * [(P*G + P)][*width], capacity in elements): rows 0..P*G-1 are the sequences' page tables
+ * (sequence s = p*G + g), rows P*G..P*G+P-1 the pages each prompt's prefill writes; unused
+ * entries are -1.  *width = logical pages per row, *n_pages = physical pages used.  Pass
+ * out_table = NULL to query width and n_pages. */
+int echo_plan_page_table(const int32_t *prompt_lens, int32_t P, int32_t G, int32_t T, int32_t page_size,
+                         int32_t *out_table, size_t capacity, int32_t *width, int32_t *n_pages);
+
 /* ---- stand-alone kernel entry points (used by the parity tests) ---------- */
 
 /* Philox words and uniforms exactly as the sampler draws them: for vocab ids

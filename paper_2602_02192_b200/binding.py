@@ -79,6 +79,8 @@ def _load() -> C.CDLL:
     lib.echo_profile_config.argtypes = [vp, i32]
     lib.echo_profile_read.argtypes = [vp, vp, vp, i32, C.POINTER(i32)]
     lib.echo_debug_page_table.argtypes = [vp, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32)]
+    lib.echo_plan_page_table.argtypes = [vp, i32, i32, i32, i32, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32)]
+    lib.echo_plan_page_table.restype = C.c_int
     lib.echo_debug_noise.argtypes = [u64, u32, u32, u32, u32, vp, vp, vp]
     lib.echo_sample.argtypes = [vp, i32, i32, i32, vp, u32, f32, u64, vp, vp, vp, vp]
     lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]
@@ -108,7 +110,7 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_rollout", "echo_rollout_forced", "echo_rollout_host", "echo_group_advantage", "echo_sync",
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
             "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_decode_attention",
-            "echo_decode_attention_scratch_bytes", "echo_strerror", "echo_last_error"]
+            "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -354,3 +356,15 @@ def echo_decode_attention(q: torch.Tensor, kv_pool: torch.Tensor, page_table: to
                                          page_table.shape[1], row_pos.data_ptr(), full_pages.data_ptr(), P, G, Hq,
                                          Hkv, hd, scratch.data_ptr(), n, out.data_ptr(), _stream_ptr(None)))
     return out
+
+
+def echo_plan_page_table(prompt_lens, G: int, T: int, page_size: int = 16):
+    """Host-only: (table int32 [P*G][width], prefill_table int32 [P][width], n_pages)."""
+    lens = np.ascontiguousarray(np.asarray(prompt_lens, dtype=np.int32))
+    P = len(lens)
+    width, n_pages = C.c_int32(), C.c_int32()
+    _check(lib.echo_plan_page_table(lens.ctypes.data, P, G, T, page_size, None, 0, C.byref(width), C.byref(n_pages)))
+    out = np.zeros((P * G + P, width.value), dtype=np.int32)
+    _check(lib.echo_plan_page_table(lens.ctypes.data, P, G, T, page_size, out.ctypes.data, out.size,
+                                    C.byref(width), C.byref(n_pages)))
+    return out[: P * G], out[P * G:], n_pages.value

@@ -415,6 +415,43 @@ struct Plan {
   int P, G, T, B, n_tok, n_chunks, n_copies, n_pages, width;
 };
 
+// The page plan itself (pure host arithmetic).  Writes pt[(P*G + P)][W]: rows 0..P*G-1 are the
+// sequences' tables, rows P*G.. are where each prompt's prefill writes; entries past a row's last
+// page are -1.  copy_src/copy_dst (capacity P*G each, may be null) list the partial prompt pages
+// to duplicate into each sample's first decode page.  Returns the number of physical pages.
+int plan_tables(const int32_t *lens, int P, int G, int T, int Z, int W, int32_t *pt, int32_t *copy_src,
+                int32_t *copy_dst, int *n_copies_out) {
+  const int B = P * G;
+  std::fill(pt, pt + static_cast<size_t>(B + P) * W, -1);
+  int next_page = 0;
+  std::vector<int> pre_base(P);
+  for (int p = 0; p < P; ++p) {
+    pre_base[p] = next_page;
+    next_page += ceil_div(lens[p], Z);
+  }
+  int n_copies = 0;
+  for (int p = 0; p < P; ++p) {
+    const int full = lens[p] / Z, n_pre = ceil_div(lens[p], Z);
+    const int n_dec = ceil_div(lens[p] + T - 1, Z) - full;
+    int32_t *pre_row = pt + static_cast<size_t>(B + p) * W;
+    for (int qi = 0; qi < n_pre; ++qi) pre_row[qi] = pre_base[p] + qi;
+    for (int g = 0; g < G; ++g) {
+      const int s = p * G + g;
+      int32_t *row = pt + static_cast<size_t>(s) * W;
+      for (int qi = 0; qi < full; ++qi) row[qi] = pre_base[p] + qi;
+      for (int qi = 0; qi < n_dec; ++qi) row[full + qi] = next_page + qi;
+      if (n_pre > full && n_dec > 0) {          // partial last prompt page: private copy per sample
+        if (copy_src) copy_src[n_copies] = pre_base[p] + full;
+        if (copy_dst) copy_dst[n_copies] = next_page;
+        ++n_copies;
+      }
+      next_page += n_dec;
+    }
+  }
+  if (n_copies_out) *n_copies_out = n_copies;
+  return next_page;
+}
+
 // Page tables and row lists, written into the pinned staging block in the order of the
 // device-side table regions.  Sequence id s = p*G + g.  Prefix pages of prompt p:
 // pre_base[p] + [0, ceil(Lp/Z)); decode pages of s: dec_base[s] + [0, n_dec_p).
@@ -434,36 +471,16 @@ int build_plan(echo_ctx *ctx, const int32_t *lens, int P, int G, int T, Plan *pl
   int32_t *h_csrc = h_full + M.B;
   int32_t *h_cdst = h_csrc + M.B;
 
-  std::fill(h_pt, h_pt + static_cast<size_t>(M.B + M.P) * W, -1);
-  int next_page = 0;
-  std::vector<int> pre_base(P);
-  for (int p = 0; p < P; ++p) {
-    pre_base[p] = next_page;
-    next_page += ceil_div(lens[p], Z);
-  }
   int n_copies = 0;
-  for (int p = 0; p < P; ++p) {
-    const int full = lens[p] / Z, n_pre = ceil_div(lens[p], Z);
-    const int n_dec = ceil_div(lens[p] + T - 1, Z) - full;
-    // prefill row of prompt p sits after the B sequence rows
-    int32_t *pre_row = h_pt + static_cast<size_t>(B + p) * W;
-    for (int qi = 0; qi < n_pre; ++qi) pre_row[qi] = pre_base[p] + qi;
+  const int next_page = plan_tables(lens, P, G, T, Z, W, h_pt, h_csrc, h_cdst, &n_copies);
+  std::fill(h_pt + static_cast<size_t>(B + P) * W, h_pt + static_cast<size_t>(M.B + M.P) * W, -1);
+  for (int p = 0; p < P; ++p)
     for (int g = 0; g < G; ++g) {
       const int s = p * G + g;
-      int32_t *row = h_pt + static_cast<size_t>(s) * W;
-      for (int qi = 0; qi < full; ++qi) row[qi] = pre_base[p] + qi;
-      for (int qi = 0; qi < n_dec; ++qi) row[full + qi] = next_page + qi;
-      if (n_pre > full && n_dec > 0) {          // partial last prompt page: private copy per sample
-        h_csrc[n_copies] = pre_base[p] + full;
-        h_cdst[n_copies] = next_page;
-        ++n_copies;
-      }
-      next_page += n_dec;
       h_dec_pt[s] = s;
       h_len0[s] = lens[p];
-      h_full[s] = full;
+      h_full[s] = lens[p] / Z;
     }
-  }
   if (next_page > M.n_pages) return ECHO_ERR_INVALID;
   int n_tok = 0;
   for (int p = 0; p < P; ++p) n_tok += lens[p];
@@ -942,6 +959,26 @@ int echo_debug_page_table(echo_ctx *ctx, int32_t *out, size_t n, int32_t *rows, 
     if (n < ctx->last_table.size()) return ECHO_ERR_INVALID;
     std::copy(ctx->last_table.begin(), ctx->last_table.end(), out);
   }
+  return ECHO_OK;
+}
+
+int echo_plan_page_table(const int32_t *prompt_lens, int32_t P, int32_t G, int32_t T, int32_t page_size,
+                         int32_t *out_table, size_t capacity, int32_t *width, int32_t *n_pages) {
+  if (!prompt_lens || !width || !n_pages || P < 1 || G < 1 || T < 1 || page_size < 1) return ECHO_ERR_INVALID;
+  int W = 0;
+  for (int p = 0; p < P; ++p) {
+    if (prompt_lens[p] < 1) return ECHO_ERR_INVALID;
+    W = std::max(W, std::max(ceil_div(prompt_lens[p] + T - 1, page_size), ceil_div(prompt_lens[p], page_size)));
+  }
+  *width = W;
+  const size_t need = static_cast<size_t>(P) * G * W + static_cast<size_t>(P) * W;
+  if (!out_table) {
+    std::vector<int32_t> tmp(need);
+    *n_pages = plan_tables(prompt_lens, P, G, T, page_size, W, tmp.data(), nullptr, nullptr, nullptr);
+    return ECHO_OK;
+  }
+  if (capacity < need) return ECHO_ERR_INVALID;
+  *n_pages = plan_tables(prompt_lens, P, G, T, page_size, W, out_table, nullptr, nullptr, nullptr);
   return ECHO_OK;
 }
 

@@ -45,3 +45,24 @@ def test_config_validation_needs_no_gpu():
     # 8B-shape workload: 2 x 16.4 GB weights + ~80 GB KV must fit a 180 GB part
     big = binding.make_config(synth.SHAPES["8B"], 32, 8, 512, 2048)
     assert 110e9 < binding.echo_arena_bytes(big) < 125e9
+
+
+def test_host_page_plan_matches_oracle_bit_for_bit():
+    """The library's page plan (host arithmetic, no GPU) against the oracle's on ragged cases."""
+    import numpy as np
+    from oracle import pages
+    from paper_2602_02192_b200 import binding
+    rng = np.random.default_rng(11)
+    cases = [([32] * 4, 4, 32, 16), ([512] * 32, 8, 2048, 16), ([20, 33, 16, 1], 3, 9, 16), ([5], 2, 1, 16),
+             ([17, 31], 2, 40, 8), ([1024] * 16, 8, 2048, 16)]
+    for _ in range(20):
+        P = int(rng.integers(1, 9))
+        cases.append(([int(x) for x in rng.integers(1, 200, size=P)], int(rng.integers(1, 6)),
+                      int(rng.integers(1, 70)), int(rng.choice([4, 16, 32]))))
+    for lens, G, T, Z in cases:
+        plan = pages.build(lens, G, T, Z)
+        table, prefill, n_pages = binding.echo_plan_page_table(lens, G, T, Z)
+        assert n_pages == plan.n_pages
+        assert table.shape[1] == plan.width
+        assert np.array_equal(table, plan.table)
+        assert np.array_equal(prefill, plan.prefill_table)
