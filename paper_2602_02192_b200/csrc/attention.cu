@@ -273,7 +273,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
   };
   auto row_head = [&](int r) -> int { return h * REP + (PREFIX ? (mt * 16 + r) % REP : r); };
 
-  if (!PREFIX) griddep_launch();             // the output projection may start prefetching its weights
+  early_start_sync();        // (the output projection may start prefetching its weights)
   if (threadIdx.x == 0) {
     for (int i = 0; i < kDecWarps * kDecStages; ++i) mbar_init(&bars[i], 1);
     *abort_flag = 0;
@@ -533,15 +533,13 @@ cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
   const int REP = a.Hq / a.Hkv;
   const int MT = (a.G * REP + 15) / 16;
   const float scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(HD));
-  attn_decode_kernel<HD, true><<<a.P * a.Hkv * MT, kDecWarps * 32, S::kTotal, s>>>(
-      *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages, a.layer_row0, a.Hq,
-      a.Hkv, a.G, a.n_pages, scale_log2, a.status);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_early(attn_decode_kernel<HD, true>, dim3(a.P * a.Hkv * MT), dim3(kDecWarps * 32), S::kTotal, s,
+                               *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos,
+                               a.full_pages, a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.status);
   if (e != cudaSuccess) return e;
-  attn_decode_kernel<HD, false><<<a.P * a.G * a.Hkv, kDecWarps * 32, S::kTotal, s>>>(
-      *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages, a.layer_row0, a.Hq,
-      a.Hkv, a.G, a.n_pages, scale_log2, a.status);
-  return cudaGetLastError();
+  return launch_early(attn_decode_kernel<HD, false>, dim3(a.P * a.G * a.Hkv), dim3(kDecWarps * 32), S::kTotal, s,
+                      *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages,
+                      a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.status);
 }
 
 }  // namespace

@@ -23,6 +23,35 @@ constexpr int kGemmTileK = 64;       // bf16 elements per pipeline stage (one 12
 constexpr int kMaxBatchTile = 256;   // rows of activations per MMA (UMMA N)
 constexpr int kGemmMaxUnits = 8192;  // output tiles per launch the tile counters cover
 
+// ---- launches that may start early (programmatic stream serialization) --------------------------
+// A kernel launched through launch_early may be scheduled while its predecessor on the stream is
+// still draining, which hides the launch latency between the many short kernels of a decode step.
+// Such a kernel MUST begin with early_start_sync(): it lets its own successor be scheduled and then
+// waits until the predecessor has completed and its writes are visible, before touching memory.
+extern bool g_early_start;          // cleared to launch everything the ordinary way
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_early(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = g_early_start ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void early_start_sync() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+
 // ---- dense projections (gemm.cu) ------------------------------------------
 // Y[m][n] (+)= sum_k X[m][k] * W[n][k], bf16 inputs, fp32 accumulation.
 // tmW: tensor map over W [N][K] with box {64, 128}; tmX over X [M][K] with box {64, bnb}.

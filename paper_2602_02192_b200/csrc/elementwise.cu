@@ -6,6 +6,8 @@
 
 namespace echo {
 
+bool g_early_start = true;
+
 namespace {
 
 // ---------------------------------------------------------------------------
@@ -32,6 +34,7 @@ __device__ __forceinline__ float gumbel_from_uniform(float w) { return -logf(-lo
 // ---------------------------------------------------------------------------
 __global__ void embed_kernel(const __nv_bfloat16 *embed, const int32_t *tok_src, const int32_t *tok_idx, float *x,
                              int R, int d, int vocab, int *status) {
+  early_start_sync();
   const int r = blockIdx.x;
   if (r >= R) return;
   int tok = tok_src[tok_idx ? tok_idx[r] : r];
@@ -64,8 +67,7 @@ __global__ void __launch_bounds__(kNormThreads)
 rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ gain, __nv_bfloat16 *__restrict__ h,
                int R, int d, float eps) {
   __shared__ float scratch[32];
-  // lets a projection launched with programmatic serialization begin its weight prefetch now
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  early_start_sync();       // (also lets the following projection begin its weight prefetch)
   const int r = blockIdx.x;
   const float *xr = x + static_cast<size_t>(r) * d;
   __nv_bfloat16 *hr = h + static_cast<size_t>(r) * d;
@@ -126,6 +128,7 @@ __global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__res
                                    const int32_t *__restrict__ row_pt, const int32_t *__restrict__ row_pos,
                                    const int32_t *__restrict__ page_table, int pt_width, int R, int Hq, int Hkv, int hd,
                                    int page_size, int n_pages, int max_pos, int *status) {
+  early_start_sync();
   const int r = blockIdx.x;
   const int pos = row_pos[r];
   const int half = hd / 2;
@@ -209,6 +212,7 @@ __global__ void copy_pages_kernel(__nv_bfloat16 *kv, const int32_t *src_page, co
 // position len0[b] + j - 1.  One block; the counter is bumped after every thread has read it.
 __global__ void decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
                                    int32_t *row_tok, int32_t *row_pos, int B) {
+  early_start_sync();
   const int j = *d_step + 1;
   __syncthreads();
   for (int b = threadIdx.x; b < B; b += blockDim.x) {
@@ -264,6 +268,7 @@ sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t
                int forced_stride, int32_t *out_tok, float *out_lp, int out_stride) {
   __shared__ float sm_m[32], sm_l[32], sm_score[32];
   __shared__ int sm_id[32];
+  early_start_sync();
   const int r = blockIdx.x;
   const uint32_t j = d_step ? static_cast<uint32_t>(*d_step) : j_host;
   const uint32_t s_id = seq_ids ? static_cast<uint32_t>(seq_ids[r]) : static_cast<uint32_t>(r);
@@ -364,13 +369,11 @@ __global__ void advantage_kernel(const float *r, int P, int G, float eps, float 
 
 cudaError_t embed_launch(const __nv_bfloat16 *embed, const int32_t *tok_src, const int32_t *tok_idx, float *x, int R,
                          int d, int vocab, int *status, cudaStream_t s) {
-  embed_kernel<<<R, 256, 0, s>>>(embed, tok_src, tok_idx, x, R, d, vocab, status);
-  return cudaGetLastError();
+  return launch_early(embed_kernel, dim3(R), dim3(256), 0, s, embed, tok_src, tok_idx, x, R, d, vocab, status);
 }
 cudaError_t rmsnorm_launch(const float *x, const __nv_bfloat16 *gain, __nv_bfloat16 *h, int R, int d, float eps,
                            cudaStream_t s) {
-  rmsnorm_kernel<<<R, kNormThreads, 0, s>>>(x, gain, h, R, d, eps);
-  return cudaGetLastError();
+  return launch_early(rmsnorm_kernel, dim3(R), dim3(kNormThreads), 0, s, x, gain, h, R, d, eps);
 }
 cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double theta, cudaStream_t s) {
   const int half = head_dim / 2, n = max_pos * half;
@@ -380,9 +383,8 @@ cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double t
 cudaError_t rope_append_launch(float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer, const float2 *rope_table,
                                RowMeta meta, const int32_t *page_table, int pt_width, int R, int Hq, int Hkv, int hd,
                                int page_size, int n_pages, int max_pos, int *status, cudaStream_t s) {
-  rope_append_kernel<<<R, 256, 0, s>>>(qkv, q, kv_layer, rope_table, meta.row_pt, meta.row_pos, page_table, pt_width,
-                                       R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
-  return cudaGetLastError();
+  return launch_early(rope_append_kernel, dim3(R), dim3(256), 0, s, qkv, q, kv_layer, rope_table, meta.row_pt,
+                      meta.row_pos, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
 }
 cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s) {
   const size_t n = static_cast<size_t>(R) * F;
@@ -402,18 +404,15 @@ cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page
 }
 cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
                                int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s) {
-  decode_prep_kernel<<<1, 512, 0, s>>>(d_step, tok_hist, T, seq_len0, row_tok, row_pos, B);
-  return cudaGetLastError();
+  return launch_early(decode_prep_kernel, dim3(1), dim3(512), 0, s, d_step, tok_hist, T, seq_len0, row_tok, row_pos, B);
 }
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row, const int32_t *seq_ids,
                            const int32_t *d_step, uint32_t j_host, float temperature, uint64_t seed,
                            const int32_t *forced, int forced_stride, int32_t *out_tok, float *out_lp, int out_stride,
                            cudaStream_t s) {
-  sampler_kernel<<<R, kSamplerThreads, 0, s>>>(logits, V, rows_per_logit_row, seq_ids, d_step, j_host,
-                                               1.0f / temperature, static_cast<uint32_t>(seed & 0xffffffffu),
-                                               static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok,
-                                               out_lp, out_stride);
-  return cudaGetLastError();
+  return launch_early(sampler_kernel, dim3(R), dim3(kSamplerThreads), 0, s, logits, V, rows_per_logit_row, seq_ids,
+                      d_step, j_host, 1.0f / temperature, static_cast<uint32_t>(seed & 0xffffffffu),
+                      static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok, out_lp, out_stride);
 }
 cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n, uint32_t *words,
                                float *uniform, cudaStream_t s) {

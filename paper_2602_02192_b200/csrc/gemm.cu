@@ -177,6 +177,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_launch();
   griddep_wait();          // inputs produced by the preceding kernel are complete from here on
 
   if (warp == 0) {
@@ -696,6 +697,9 @@ cudaError_t launch_variant(const GemmArgs &a, cudaStream_t stream) {
   }
   if (a.max_ctas > 0 && grid > a.max_ctas) grid = a.max_ctas;
   if (grid > total) grid = static_cast<int>(total);
+  if (a.allow_early_start)
+    return launch_early(gemm_streamk_kernel<BNB>, dim3(grid), dim3(kThreads), S::kTotal, stream, *a.tmW, *a.tmX, a.Y,
+                        a.ldY, a.M, a.N, a.K, a.epilogue, n_tiles, a.workspace, a.counters, a.status);
   gemm_streamk_kernel<BNB><<<grid, kThreads, S::kTotal, stream>>>(*a.tmW, *a.tmX, a.Y, a.ldY, a.M, a.N, a.K,
                                                                  a.epilogue, n_tiles, a.workspace, a.counters,
                                                                  a.status);

@@ -708,6 +708,7 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
   ctx->deterministic = det && det[0] == '1';
   const char *pdl = getenv("ECHO_NO_PDL");
   ctx->use_pdl = !(pdl && pdl[0] == '1');
+  g_early_start = ctx->use_pdl;
 
   auto bail = [&](cudaError_t e, const char *what) {
     fail_cuda(ctx, e, what);
