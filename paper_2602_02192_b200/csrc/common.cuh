@@ -89,6 +89,29 @@ cudaError_t gemm_simt_launch(const __nv_bfloat16 *X, const __nv_bfloat16 *W, flo
 int make_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
                     uint32_t box_rows);
 
+// Output tile map over a row-major [rows][cols] fp32 or bf16 matrix, no swizzle, box {box_cols, box_rows}.
+int make_out_map_box(CUtensorMap *out, void *base, uint64_t rows, uint64_t cols, uint64_t ld, bool bf16,
+                     uint32_t box_cols, uint32_t box_rows);
+
+// ---- projections on SM pairs (gemm_pair.cu) ---------------------------------
+// Same arithmetic as above with 2-CTA MMAs: used for more than 64 activation rows.
+struct PairGemmArgs {
+  const CUtensorMap *tmW;   // tensor map over W with box {64, 128}; for EPI_SWIGLU over [2N][K] (gate rows, then up rows)
+  const void *X;            // bf16 [M][K], contiguous
+  void *Y;                  // fp32 [M][ldY], or bf16 for EPI_SWIGLU; 16-byte aligned rows
+  int ldY;
+  int M, N, K;
+  int epilogue;
+  int *status;
+  int allow_early_start;
+  int force_split;          // 0 = choose; k > 0 = k slices along K (linear epilogues only)
+};
+cudaError_t gemm_pair_configure();
+bool gemm_pair_supported(const void *Y, int ldY, int M, int N, int K, int epilogue);
+// k-slices per tile the launch will use; with more than one slice and EPI_STORE, Y must hold zeros
+int gemm_pair_split(int M, int N, int K, int epilogue, int force_split);
+cudaError_t gemm_pair_launch(const PairGemmArgs &a, cudaStream_t stream);
+
 // ---- element-wise / row-wise kernels (elementwise.cu) ------------------------
 struct RowMeta {
   const int32_t *row_pt;     // page-table row of each activation row

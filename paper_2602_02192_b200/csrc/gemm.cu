@@ -771,6 +771,24 @@ int make_out_map(CUtensorMap *out, void *base, uint64_t rows, uint64_t cols, uin
 
 }  // namespace
 
+int make_out_map_box(CUtensorMap *out, void *base, uint64_t rows, uint64_t cols, uint64_t ld, bool bf16,
+                     uint32_t box_cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return -1;
+  const uint64_t es = bf16 ? 2 : 4;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || ((ld * es) & 15) || box_cols == 0 || box_cols > 256 ||
+      box_rows == 0 || box_rows > 256)
+    return -2;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld * es};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -3;
+}
+
 int make_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
                     uint32_t box_rows) {
   EncodeTiledFn fn = encode_fn();

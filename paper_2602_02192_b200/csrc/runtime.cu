@@ -139,6 +139,7 @@ struct WeightBuf {
   __nv_bfloat16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
   std::vector<__nv_bfloat16 *> wqkv, wo, wgu, wdown, attn_norm, mlp_norm;
   std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_down;
+  std::vector<CUtensorMap> tm_gu_pair;       // gate/up with a 128-row box, for the SM-pair kernel
   CUtensorMap tm_lm;
   int64_t version = -1;
   bool has_data = false;       // an install was enqueued into this buffer
@@ -171,7 +172,7 @@ struct echo_ctx {
   int last_rows = 0, last_width = 0;
   echo_stats stats{};
   int64_t launches = 0;
-  bool use_simt = false, use_graph = true, fast_decode = false, deterministic = false, use_pdl = true;
+  bool use_simt = false, use_graph = true, fast_decode = false, deterministic = false, use_pdl = true, use_pair = true;
   CUtensorMap tm_kv;
   std::string last_error;
   // sampled per-kernel timing (echo_profile_config / echo_profile_read)
@@ -258,8 +259,20 @@ int pick_bnb(int rows) {
 
 // Y = X * W^T through the tensor-core kernel (or the SIMT reference when selected).
 int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, const __nv_bfloat16 *X, void *Y, int ldY,
-             int M, int N, int K, int epilogue, bool y_holds_zeros = false) {
+             int M, int N, int K, int epilogue, bool y_holds_zeros = false, const CUtensorMap *tmW_pair = nullptr) {
   ProfScope prof(ctx, PROF_GEMM);
+  if (ctx->use_pair && !ctx->use_simt && !ctx->deterministic && (epilogue != EPI_SWIGLU || tmW_pair) &&
+      gemm_pair_supported(Y, ldY, M, N, K, epilogue)) {
+    // more than 64 rows: 2-CTA MMAs, k-slices added into Y in memory
+    PairGemmArgs a{tmW_pair ? tmW_pair : tmW, X, Y, ldY, M, N, K, epilogue, ctx->ptr<int>(ctx->lo.status),
+                   ctx->use_pdl ? 1 : 0, 0};
+    if (epilogue == EPI_STORE && !y_holds_zeros && gemm_pair_split(M, N, K, epilogue, 0) > 1) {
+      CK(cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * ldY * sizeof(float), ctx->stream));
+      a.allow_early_start = 0;
+    }
+    LAUNCH(gemm_pair_launch(a, ctx->stream));
+    return ECHO_OK;
+  }
   if (ctx->use_simt) {
     if (epilogue == EPI_SWIGLU) {
       float *gu = ctx->ptr<float>(ctx->lo.gu);
@@ -330,7 +343,7 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int d
     }
     TRY(run_gemm(ctx, &w.tm_o[l], w.wo[l], attn, x, D.d, R, D.d, D.Hq * D.hd, EPI_ACCUM));
     LAUNCH(rmsnorm_launch(x, w.mlp_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream));
-    TRY(run_gemm(ctx, &w.tm_gu[l], w.wgu[l], h, act, D.F, R, D.F, D.d, EPI_SWIGLU));
+    TRY(run_gemm(ctx, &w.tm_gu[l], w.wgu[l], h, act, D.F, R, D.F, D.d, EPI_SWIGLU, false, &w.tm_gu_pair[l]));
     TRY(run_gemm(ctx, &w.tm_down[l], w.wdown[l], act, x, D.d, R, D.d, D.F, EPI_ACCUM));
   }
   return ECHO_OK;
@@ -358,7 +371,7 @@ void carve_weights(echo_ctx *ctx, WeightBuf &w, uint8_t *base) {
   w.final_norm = take(D.d);
   w.wqkv.resize(D.L); w.wo.resize(D.L); w.wgu.resize(D.L); w.wdown.resize(D.L);
   w.attn_norm.resize(D.L); w.mlp_norm.resize(D.L);
-  w.tm_qkv.resize(D.L); w.tm_o.resize(D.L); w.tm_gu.resize(D.L); w.tm_down.resize(D.L);
+  w.tm_qkv.resize(D.L); w.tm_o.resize(D.L); w.tm_gu.resize(D.L); w.tm_down.resize(D.L); w.tm_gu_pair.resize(D.L);
   for (int l = 0; l < D.L; ++l) {
     w.wqkv[l] = take(static_cast<size_t>(D.n_qkv()) * D.d);
     w.wo[l] = take(static_cast<size_t>(D.d) * D.Hq * D.hd);
@@ -377,6 +390,7 @@ int make_weight_maps(echo_ctx *ctx, WeightBuf &w) {
     rc |= make_tensor_map(&w.tm_qkv[l], w.wqkv[l], D.n_qkv(), D.d, D.d, kGemmTileN);
     rc |= make_tensor_map(&w.tm_o[l], w.wo[l], D.d, D.Hq * D.hd, D.Hq * D.hd, kGemmTileN);
     rc |= make_tensor_map(&w.tm_gu[l], w.wgu[l], 2ull * D.F, D.d, D.d, 64);
+    rc |= make_tensor_map(&w.tm_gu_pair[l], w.wgu[l], 2ull * D.F, D.d, D.d, kGemmTileN);
     rc |= make_tensor_map(&w.tm_down[l], w.wdown[l], D.d, D.F, D.F, kGemmTileN);
   }
   if (rc) {
@@ -702,6 +716,7 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
   ctx->stream = static_cast<cudaStream_t>(cuda_stream);
   const char *impl = getenv("ECHO_GEMM_IMPL");
   ctx->use_simt = impl && !strcmp(impl, "simt");
+  ctx->use_pair = !(impl && !strcmp(impl, "single"));
   const char *ng = getenv("ECHO_NO_GRAPH");
   ctx->use_graph = !(ng && ng[0] == '1');
   const char *det = getenv("ECHO_DETERMINISTIC");
@@ -745,6 +760,7 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
       cudaSuccess)
     return bail(e, "cudaHostAlloc");
   if ((e = gemm_tc_configure()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute");
+  if ((e = gemm_pair_configure()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute");
   // padding keys of a partly filled page take part in the P*V products with weight zero: the pool
   // must never hold NaN/Inf bit patterns
   if ((e = cudaMemsetAsync(ctx->arena + lo.kv, 0, lo.kv_layer_elems * ctx->D.L * 2, ctx->stream)) != cudaSuccess)
@@ -1058,6 +1074,19 @@ int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, 
     return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
   }
   if (gemm_tc_configure() != cudaSuccess) return ECHO_ERR_CUDA;
+  if (impl >= 300) {
+    // SM-pair kernel, impl - 300 k-slices per tile (0 = choose)
+    if (gemm_pair_configure() != cudaSuccess) return ECHO_ERR_CUDA;
+    if (!gemm_pair_supported(Y, N, M, N, K, epilogue)) return ECHO_ERR_UNSUPPORTED;
+    const bool gu2 = epilogue == EPI_SWIGLU;
+    CUtensorMap tmW2;
+    if (make_tensor_map(&tmW2, W, gu2 ? 2ull * N : N, K, K, kGemmTileN) != 0) return ECHO_ERR_CUDA;
+    PairGemmArgs pa{&tmW2, X, Y, N, M, N, K, epilogue, nullptr, 0, impl - 300};
+    if (epilogue == EPI_STORE && gemm_pair_split(M, N, K, epilogue, impl - 300) > 1 &&
+        cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * N * sizeof(float), s) != cudaSuccess)
+      return ECHO_ERR_CUDA;
+    return gemm_pair_launch(pa, s) == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+  }
   const int bnb = pick_bnb(M);
   const size_t ws_bytes = align_up(gemm_workspace_bytes(bnb));
   if (!workspace || workspace_bytes < ws_bytes + static_cast<size_t>(kGemmMaxUnits) * 4 ||
