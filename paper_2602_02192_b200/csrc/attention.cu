@@ -208,7 +208,7 @@ namespace {
 using namespace ptx;
 
 constexpr int kDecWarps = 4;
-constexpr int kDecStages = 3;
+constexpr int kDecStages = 2;      // 64 KiB per CTA at head_dim 128: three CTAs share an SM
 constexpr int kPageTokens = 16;
 
 template <int HD>
@@ -244,6 +244,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
   const int REP = Hq / Hkv;
   const int quad = lane >> 2, qi = lane & 3;
 
+  // row positions are written earlier in the same step: read nothing before the predecessor is complete
+  early_start_sync();        // (the output projection may start prefetching its weights)
+
   // ---- which query rows and which keys this CTA handles ------------------------------------
   int h, seq0, first_page, n_keys, mt = 0;
   if (PREFIX) {
@@ -273,7 +276,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
   };
   auto row_head = [&](int r) -> int { return h * REP + (PREFIX ? (mt * 16 + r) % REP : r); };
 
-  early_start_sync();        // (the output projection may start prefetching its weights)
   if (threadIdx.x == 0) {
     for (int i = 0; i < kDecWarps * kDecStages; ++i) mbar_init(&bars[i], 1);
     *abort_flag = 0;

@@ -184,6 +184,73 @@ __global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__res
   }
 }
 
+// Vector form of rope_append_kernel for head_dim % 8 == 0: a work item is four consecutive
+// rotation pairs of one head (for a kv head: of its key, plus the matching eight values), moved
+// with 16-byte loads and 8-byte stores.  Every qkv element is read by exactly one thread, which
+// zeroes it right after reading, so no second pass over the row is needed.
+__device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 o;
+  o.x = *reinterpret_cast<uint32_t *>(&lo);
+  o.y = *reinterpret_cast<uint32_t *>(&hi);
+  return o;
+}
+__global__ void __launch_bounds__(256)
+rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ kv_layer,
+                       const float2 *__restrict__ rope_table, const int32_t *__restrict__ row_pt,
+                       const int32_t *__restrict__ row_pos, const int32_t *__restrict__ page_table, int pt_width,
+                       int R, int Hq, int Hkv, int hd, int page_size, int n_pages, int max_pos, int *status) {
+  early_start_sync();
+  const int r = blockIdx.x;
+  const int pos = row_pos[r];
+  const int half = hd / 2, q4 = half / 4;
+  const int ld = (Hq + 2 * Hkv) * hd;
+  float *src = qkv + static_cast<size_t>(r) * ld;
+  const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  int page = -1;
+  if (pos >= 0 && pos < max_pos) page = page_table[static_cast<size_t>(row_pt[r]) * pt_width + pos / page_size];
+  if (page < 0 || page >= n_pages) {
+    if (threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
+    for (int i = threadIdx.x; i < ld / 4; i += blockDim.x) reinterpret_cast<float4 *>(src)[i] = zero4;
+    return;
+  }
+  const int off = pos % page_size;
+  const float4 *cs4 = reinterpret_cast<const float4 *>(rope_table + static_cast<size_t>(pos) * half);
+  const size_t page_elems = static_cast<size_t>(page_size) * hd;
+  const int n_items = (Hq + Hkv) * q4;
+  for (int item = threadIdx.x; item < n_items; item += blockDim.x) {
+    const int unit = item / q4, i = (item % q4) * 4;
+    float4 *pa = reinterpret_cast<float4 *>(src + unit * hd + i);
+    float4 *pb = reinterpret_cast<float4 *>(src + unit * hd + i + half);
+    const float4 a = *pa, b = *pb;
+    const float4 t01 = cs4[i / 2], t23 = cs4[i / 2 + 1];         // (cos, sin) of pairs i..i+3
+    *pa = zero4;
+    *pb = zero4;
+    const uint2 lo = pack_bf16x4(a.x * t01.x - b.x * t01.y, a.y * t01.z - b.y * t01.w, a.z * t23.x - b.z * t23.y,
+                                 a.w * t23.z - b.w * t23.w);
+    const uint2 hi = pack_bf16x4(b.x * t01.x + a.x * t01.y, b.y * t01.z + a.y * t01.w, b.z * t23.x + a.z * t23.y,
+                                 b.w * t23.z + a.w * t23.w);
+    if (unit < Hq) {
+      __nv_bfloat16 *dst = q + static_cast<size_t>(r) * Hq * hd + unit * hd + i;
+      *reinterpret_cast<uint2 *>(dst) = lo;
+      *reinterpret_cast<uint2 *>(dst + half) = hi;
+    } else {
+      const int head = unit - Hq;
+      __nv_bfloat16 *kd = kv_layer + ((static_cast<size_t>(page) * Hkv + head) * 2 + 0) * page_elems + off * hd + i;
+      *reinterpret_cast<uint2 *>(kd) = lo;
+      *reinterpret_cast<uint2 *>(kd + half) = hi;
+      float4 *va = reinterpret_cast<float4 *>(src + (unit + Hkv) * hd + i);
+      float4 *vb = reinterpret_cast<float4 *>(src + (unit + Hkv) * hd + i + half);
+      const float4 v0 = *va, v1 = *vb;
+      *va = zero4;
+      *vb = zero4;
+      __nv_bfloat16 *vd = kd + page_elems;
+      *reinterpret_cast<uint2 *>(vd) = pack_bf16x4(v0.x, v0.y, v0.z, v0.w);
+      *reinterpret_cast<uint2 *>(vd + half) = pack_bf16x4(v1.x, v1.y, v1.z, v1.w);
+    }
+  }
+}
+
 __global__ void swiglu_kernel(const float *gu, __nv_bfloat16 *act, int R, int F) {
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= static_cast<size_t>(R) * F) return;
@@ -383,6 +450,9 @@ cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double t
 cudaError_t rope_append_launch(float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer, const float2 *rope_table,
                                RowMeta meta, const int32_t *page_table, int pt_width, int R, int Hq, int Hkv, int hd,
                                int page_size, int n_pages, int max_pos, int *status, cudaStream_t s) {
+  if (hd % 8 == 0 && (reinterpret_cast<uintptr_t>(qkv) & 15) == 0)
+    return launch_early(rope_append_vec_kernel, dim3(R), dim3(256), 0, s, qkv, q, kv_layer, rope_table, meta.row_pt,
+                        meta.row_pos, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
   return launch_early(rope_append_kernel, dim3(R), dim3(256), 0, s, qkv, q, kv_layer, rope_table, meta.row_pt,
                       meta.row_pos, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
 }
