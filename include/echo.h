@@ -252,11 +252,27 @@ int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, c
  * cluster split-K by s in [1, 8] (partials summed in a fixed order), 200 + s = s independent
  * k-slices per tile that add their partial sums into Y in memory (s = 0: as many as fill the GPU;
  * faster, but the order of the fp32 additions varies from run to run; epilogues 0 and 1),
- * 1 = plain SIMT reference kernel (epilogues 0 and 1 only; needs no workspace). */
+ * 300 + s = the SM-pair kernel (2-CTA MMAs; more than 64 rows only, else ECHO_ERR_UNSUPPORTED)
+ * with s k-slices per tile added into Y in memory (s = 0: as many as give every SM pair a tile),
+ * 1 = plain SIMT reference kernel (epilogues 0 and 1 only; needs no workspace).
+ * Adding 1000 to `impl` says that W is not row-major but in the block-tiled layout that
+ * echo_retile_weights writes (the layout echo_load_policy keeps the policy's matrices in). */
 size_t echo_gemm_workspace_bytes(int32_t M);
 int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, int32_t K,
                    int32_t epilogue, int32_t impl, void *workspace, size_t workspace_bytes,
                    void *cuda_stream);
+
+/* Block-tiled weight layout (the rollout plane's policy install, Section 4.3, leaves the layout of
+ * the installed snapshot to the worker).  A matrix [rows][cols] is stored as 128-row x 64-column
+ * blocks, each block contiguous (16 KiB), ordered [row block][column block], partial blocks
+ * padded with zeros: element (n, k) is at ((n/128 * ceil(cols/64) + k/64) * 128 + n%128) * 64 + k%64.
+ * A gate/up pair for epilogue 2 is two such matrices back to back (gate, then up).
+ * echo_retile_weights copies row-major `src` (dev, or host memory the device can address;
+ * cols a multiple of 8, 16-byte aligned) into `dst` (dev, echo_tiled_weight_bytes(rows, cols)
+ * bytes, 256-byte aligned), asynchronously on the stream. */
+size_t echo_tiled_weight_bytes(int64_t rows, int64_t cols);
+int echo_retile_weights(const void *src, int64_t rows, int64_t cols, void *dst, size_t dst_bytes,
+                        void *cuda_stream);
 
 /* echo_gemm_bf16 for callers that cannot allocate device memory (code that runs inside an
  * allocator hook, a plug-in that is given tensors but no allocator, a process whose device

@@ -92,6 +92,10 @@ def _load() -> C.CDLL:
     lib.echo_gemm_bf16_noalloc.restype = C.c_int
     lib.echo_gemm_workspace_bytes.restype = C.c_size_t
     lib.echo_gemm_workspace_bytes.argtypes = [i32]
+    lib.echo_tiled_weight_bytes.restype = C.c_size_t
+    lib.echo_tiled_weight_bytes.argtypes = [i64, i64]
+    lib.echo_retile_weights.restype = C.c_int
+    lib.echo_retile_weights.argtypes = [vp, i64, i64, vp, C.c_size_t, vp]
     lib.echo_strerror.restype = C.c_char_p
     lib.echo_strerror.argtypes = [C.c_int]
     lib.echo_last_error.restype = C.c_char_p
@@ -110,7 +114,8 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_rollout", "echo_rollout_forced", "echo_rollout_host", "echo_group_advantage", "echo_sync",
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
             "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_decode_attention",
-            "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error"]
+            "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error",
+            "echo_tiled_weight_bytes", "echo_retile_weights"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -310,11 +315,14 @@ def echo_sample(logits: torch.Tensor, rows: int, rows_per_logit_row: int, j: int
 def echo_gemm_bf16(X: torch.Tensor, W: torch.Tensor, impl: int = 0, epilogue: int = 0,
                    Y: Optional[torch.Tensor] = None) -> torch.Tensor:
     """epilogue 0: Y = X W^T (fp32); 1: Y += X W^T (fp32, Y given); 2: W = [Wg; Wu], Y = silu(X Wg^T) * (X Wu^T)
-    (bf16)."""
+    (bf16).  impl >= 1000: W is given row-major and handed to the kernels in the block-tiled layout."""
     assert X.is_cuda and W.is_cuda and X.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
     assert X.is_contiguous() and W.is_contiguous() and X.shape[1] == W.shape[1]
     M, K = X.shape
     N = W.shape[0] // 2 if epilogue == 2 else W.shape[0]
+    if impl >= 1000:
+        W = (torch.cat([echo_retile_weights(W[:N].contiguous()), echo_retile_weights(W[N:].contiguous())])
+             if epilogue == 2 else echo_retile_weights(W))
     if Y is None:
         Y = torch.zeros((M, N), dtype=torch.bfloat16 if epilogue == 2 else torch.float32, device=X.device)
     with torch.cuda.device(X.device):
@@ -324,6 +332,18 @@ def echo_gemm_bf16(X: torch.Tensor, W: torch.Tensor, impl: int = 0, epilogue: in
                                   ws.data_ptr(), nws, _stream_ptr(None)))
         torch.cuda.current_stream().synchronize()      # the workspace must outlive the kernel
     return Y
+
+
+def echo_retile_weights(W: torch.Tensor) -> torch.Tensor:
+    """Row-major bf16 matrix [rows][cols] -> the block-tiled layout (flat bf16 tensor) that echo_gemm_bf16
+    reads with impl + 1000."""
+    assert W.is_cuda and W.dtype == torch.bfloat16 and W.is_contiguous() and W.dim() == 2
+    rows, cols = W.shape
+    n = int(lib.echo_tiled_weight_bytes(rows, cols))
+    out = torch.empty(n // 2, dtype=torch.bfloat16, device=W.device)
+    with torch.cuda.device(W.device):
+        _check(lib.echo_retile_weights(W.data_ptr(), rows, cols, out.data_ptr(), n, _stream_ptr(None)))
+    return out
 
 
 def echo_gemm_bf16_noalloc(X: torch.Tensor, W: torch.Tensor, Y: torch.Tensor, epilogue: int = 0) -> torch.Tensor:

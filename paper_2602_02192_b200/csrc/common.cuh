@@ -78,12 +78,35 @@ struct GemmArgs {
   int allow_early_start;    // 1: launch with programmatic stream serialization (see gemm.cu)
   int independent_splits;   // 1: k-slices add into Y in memory (Y must hold zeros for EPI_STORE; the order of
                             // the additions is not fixed); 0: slices are reduced in rank order inside a cluster
+  int tiled;                // 1: W is stored block-tiled (see tiled_elems) and tmW is a map over that storage
 };
+
+// ---- block-tiled weight storage -------------------------------------------------------------
+// A weight matrix [rows][cols] is kept as 128-row x 64-column blocks, each block contiguous
+// (128 rows of 128 bytes = 16 KiB), ordered [row block][column block]; partial blocks are padded
+// with zeros.  A CTA that streams the weights of a few output features along K then reads one
+// long contiguous run instead of 128-byte pieces 2*cols bytes apart, which HBM serves about a
+// fifth faster.  Element (n, k) lives at tiled_index(n, k, ceil(cols / 64)).
+constexpr int kTileRows = 128, kTileCols = 64;
+inline size_t tiled_elems(size_t rows, size_t cols) {
+  return ((rows + kTileRows - 1) / kTileRows) * kTileRows * ((cols + kTileCols - 1) / kTileCols) * kTileCols;
+}
+__host__ __device__ inline size_t tiled_index(size_t n, size_t k, size_t col_blocks) {
+  return (((n >> 7) * col_blocks + (k >> 6)) * kTileRows + (n & 127)) * kTileCols + (k & 63);
+}
+// Copies row-major src [rows][cols] (device memory, or host memory the device can read) into tiled
+// storage whose row 0 is dst_row0 rows into the matrix at dst; padding is not written.
+cudaError_t retile_launch(__nv_bfloat16 *dst, const __nv_bfloat16 *src, size_t rows, size_t cols, size_t dst_row0,
+                          cudaStream_t s);
+// Tensor map over tiled storage of `rows` (padded to blocks) x `cols`: box = box_rows rows of one block.
+int make_tiled_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 size_t gemm_workspace_bytes(int bnb);
 cudaError_t gemm_tc_launch(const GemmArgs &a, cudaStream_t stream);
 cudaError_t gemm_tc_configure();     // sets the dynamic shared memory attribute once per device
+// part_rows > 0 with tiled storage: W consists of parts of part_rows rows, each starting on a block
 cudaError_t gemm_simt_launch(const __nv_bfloat16 *X, const __nv_bfloat16 *W, float *Y, int ldY,
-                             int M, int N, int K, int accumulate, cudaStream_t stream);
+                             int M, int N, int K, int accumulate, cudaStream_t stream, int tiled = 0,
+                             int part_rows = 0);
 // Tensor map over a row-major bf16 matrix [rows][cols] (leading dimension ld elements),
 // 128-byte swizzle, box {64, box_rows}.
 int make_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
@@ -105,6 +128,7 @@ struct PairGemmArgs {
   int *status;
   int allow_early_start;
   int force_split;          // 0 = choose; k > 0 = k slices along K (linear epilogues only)
+  int tiled;                // 1: W is block-tiled storage and tmW a map over it (make_tiled_map, 128-row box)
 };
 cudaError_t gemm_pair_configure();
 bool gemm_pair_supported(const void *Y, int ldY, int M, int N, int K, int epilogue);

@@ -85,20 +85,28 @@ __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"
 
 // Loads of one k-block: kAcc weight blocks (each 128 rows, or 64 gate + 64 up rows) and the
 // activation tile.
+// `tiled`: W is block-tiled storage (128-row x 64-column blocks, each contiguous) with KB column
+// blocks per row block; the up rows of a gate/up pair then start at row block ceil(N / 128).
 template <int BNB>
 __device__ __forceinline__ void load_stage_w(const CUtensorMap *tmW, uint64_t *bar, uint8_t *stage, int kb, int nt,
-                                             int N, bool gu) {
+                                             int N, bool gu, int tiled, int KB) {
   using S = GemmSmem<BNB>;
   mbar_expect_tx(bar, S::kStageBytes);                 // covers the activation tile loaded afterwards as well
+  auto row_of = [&](int f, int part) -> int {          // TMA row coordinate of feature f of part 0 / 1
+    if (!tiled) return part * N + f;
+    const int nbp = (N + kGemmTileN - 1) / kGemmTileN;
+    return ((part * nbp + (f >> 7)) * KB + kb) * kGemmTileN + (f & 127);
+  };
+  const int c0 = tiled ? 0 : kb * kGemmTileK;
 #pragma unroll
   for (int a = 0; a < kAcc; ++a) {
     uint8_t *dst = stage + a * S::kWBlock;
     if (gu) {
       const int f0 = (nt * kAcc + a) * 64;
-      tma_load_2d(tmW, bar, dst, kb * kGemmTileK, f0);
-      tma_load_2d(tmW, bar, dst + S::kWBlock / 2, kb * kGemmTileK, N + f0);
+      tma_load_2d(tmW, bar, dst, c0, row_of(f0, 0));
+      tma_load_2d(tmW, bar, dst + S::kWBlock / 2, c0, row_of(f0, 1));
     } else {
-      tma_load_2d(tmW, bar, dst, kb * kGemmTileK, (nt * kAcc + a) * kGemmTileN);
+      tma_load_2d(tmW, bar, dst, c0, row_of((nt * kAcc + a) * kGemmTileN, 0));
     }
   }
 }
@@ -108,8 +116,8 @@ __device__ __forceinline__ void load_stage_x(const CUtensorMap *tmX, uint64_t *b
 }
 template <int BNB>
 __device__ __forceinline__ void load_stage(const CUtensorMap *tmW, const CUtensorMap *tmX, uint64_t *bar,
-                                           uint8_t *stage, int kb, int nt, int m0, int N, bool gu) {
-  load_stage_w<BNB>(tmW, bar, stage, kb, nt, N, gu);
+                                           uint8_t *stage, int kb, int nt, int m0, int N, bool gu, int tiled, int KB) {
+  load_stage_w<BNB>(tmW, bar, stage, kb, nt, N, gu, tiled, KB);
   load_stage_x<BNB>(tmX, bar, stage, kb, m0);
 }
 
@@ -136,7 +144,7 @@ template <int BNB>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, void *Yv,
                     int ldY, int M, int N, int K, int epilogue, int n_tiles, float *workspace, int *counters,
-                    int *status) {
+                    int tiled, int *status) {
   using S = GemmSmem<BNB>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -193,7 +201,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           const int s = it % S::kStages;
           ok = mbar_wait(&empty_bar[s], ((it / S::kStages) & 1) ^ 1u, abort_flag);
           if (!ok) break;
-          load_stage<BNB>(&tmW, &tmX, &full_bar[s], smem + s * S::kStageBytes, kb, nt, mt * BNB, N, gu);
+          load_stage<BNB>(&tmW, &tmX, &full_bar[s], smem + s * S::kStageBytes, kb, nt, mt * BNB, N, gu, tiled, KB);
         }
         g += len;
       }
@@ -403,7 +411,7 @@ template <int BNB>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                     const __grid_constant__ CUtensorMap tmY, int M, int N, int K, int epilogue, int S_split,
-                    int independent, int *status) {
+                    int independent, int tiled, int *status) {
   using S = GemmSmem<BNB>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -447,7 +455,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       // then wait for that kernel to finish before touching the activations it wrote.
       const int n_pre = kb_len < S::kStages ? kb_len : S::kStages;
       for (int it = 0; it < n_pre; ++it)
-        load_stage_w<BNB>(&tmW, &full_bar[it], smem + it * S::kStageBytes, kb_beg + it, nt, N, gu);
+        load_stage_w<BNB>(&tmW, &full_bar[it], smem + it * S::kStageBytes, kb_beg + it, nt, N, gu, tiled, KB);
       griddep_wait();
       for (int it = 0; it < n_pre; ++it)
         load_stage_x<BNB>(&tmX, &full_bar[it], smem + it * S::kStageBytes, kb_beg + it, m0);
@@ -457,7 +465,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int s = it % S::kStages;
         ok = mbar_wait(&empty_bar[s], ((it / S::kStages) & 1) ^ 1u, abort_flag);
         if (!ok) break;
-        load_stage<BNB>(&tmW, &tmX, &full_bar[s], smem + s * S::kStageBytes, kb, nt, m0, N, gu);
+        load_stage<BNB>(&tmW, &tmX, &full_bar[s], smem + s * S::kStageBytes, kb, nt, m0, N, gu, tiled, KB);
       }
       if (!ok) {
         for (int k = it > S::kStages ? it - S::kStages : 0; k < it; ++k)
@@ -667,7 +675,7 @@ cudaError_t launch_cluster_variant(const GemmArgs &a, int n_tiles, int m_tiles, 
   const bool gu = a.epilogue == EPI_SWIGLU;
   if (make_out_map(&tmY, a.Y, a.M, a.N, a.ldY, gu) != 0) return cudaErrorInvalidValue;
   return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<BNB>, *a.tmW, *a.tmX, tmY, a.M, a.N, a.K, a.epilogue, split,
-                            independent ? 1 : 0, a.status);
+                            independent ? 1 : 0, a.tiled, a.status);
 }
 
 template <int BNB>
@@ -699,10 +707,10 @@ cudaError_t launch_variant(const GemmArgs &a, cudaStream_t stream) {
   if (grid > total) grid = static_cast<int>(total);
   if (a.allow_early_start)
     return launch_early(gemm_streamk_kernel<BNB>, dim3(grid), dim3(kThreads), S::kTotal, stream, *a.tmW, *a.tmX, a.Y,
-                        a.ldY, a.M, a.N, a.K, a.epilogue, n_tiles, a.workspace, a.counters, a.status);
+                        a.ldY, a.M, a.N, a.K, a.epilogue, n_tiles, a.workspace, a.counters, a.tiled, a.status);
   gemm_streamk_kernel<BNB><<<grid, kThreads, S::kTotal, stream>>>(*a.tmW, *a.tmX, a.Y, a.ldY, a.M, a.N, a.K,
                                                                  a.epilogue, n_tiles, a.workspace, a.counters,
-                                                                 a.status);
+                                                                 a.tiled, a.status);
   return cudaGetLastError();
 }
 
@@ -717,16 +725,27 @@ cudaError_t configure_variant() {
 
 // ---- plain SIMT reference kernel (debugging aid; never on the default path) ----
 __global__ void gemm_simt_kernel(const __nv_bfloat16 *X, const __nv_bfloat16 *W, float *Y, int ldY, int M, int N,
-                                 int K, int accumulate) {
+                                 int K, int accumulate, int tiled, int part_rows) {
   __shared__ float xs[16][17], ws[16][17];
   const int tx = threadIdx.x, ty = threadIdx.y;
   const int m = blockIdx.y * 16 + ty, n = blockIdx.x * 16 + tx;
+  const size_t KB = (K + kTileCols - 1) / kTileCols;
+  const size_t part_blocks = part_rows > 0 ? (part_rows + kTileRows - 1) / kTileRows : 0;
   float acc = 0.f;
   for (int k0 = 0; k0 < K; k0 += 16) {
     const int xm = blockIdx.y * 16 + ty, xk = k0 + tx;
     xs[ty][tx] = (xm < M && xk < K) ? __bfloat162float(X[static_cast<size_t>(xm) * K + xk]) : 0.f;
     const int wn = blockIdx.x * 16 + ty;
-    ws[ty][tx] = (wn < N && xk < K) ? __bfloat162float(W[static_cast<size_t>(wn) * K + xk]) : 0.f;
+    float wv = 0.f;
+    if (wn < N && xk < K) {
+      size_t idx = static_cast<size_t>(wn) * K + xk;
+      if (tiled) {
+        const size_t row = part_rows > 0 ? (wn / part_rows) * part_blocks * kTileRows + wn % part_rows : wn;
+        idx = tiled_index(row, xk, KB);
+      }
+      wv = __bfloat162float(W[idx]);
+    }
+    ws[ty][tx] = wv;
     __syncthreads();
 #pragma unroll
     for (int k = 0; k < 16; ++k) acc = fmaf(xs[ty][k], ws[tx][k], acc);
@@ -735,6 +754,20 @@ __global__ void gemm_simt_kernel(const __nv_bfloat16 *X, const __nv_bfloat16 *W,
   if (m < M && n < N) {
     float *y = Y + static_cast<size_t>(m) * ldY + n;
     *y = accumulate ? *y + acc : acc;
+  }
+}
+
+// Row-major -> block-tiled copy: one CTA per 128 x 64 source tile, 16-byte pieces.
+__global__ void __launch_bounds__(256)
+retile_kernel(__nv_bfloat16 *dst, const __nv_bfloat16 *src, size_t rows, size_t cols, size_t dst_row0) {
+  const size_t KB = (cols + kTileCols - 1) / kTileCols;
+  const size_t n0 = static_cast<size_t>(blockIdx.y) * kTileRows, k0 = static_cast<size_t>(blockIdx.x) * kTileCols;
+  for (int i = threadIdx.x; i < kTileRows * (kTileCols / 8); i += blockDim.x) {
+    const size_t n = n0 + i / (kTileCols / 8), k = k0 + (i % (kTileCols / 8)) * 8;
+    if (n < rows && k < cols) {
+      const uint4 v = *reinterpret_cast<const uint4 *>(src + n * cols + k);
+      *reinterpret_cast<uint4 *>(dst + tiled_index(dst_row0 + n, k, KB)) = v;
+    }
   }
 }
 
@@ -832,10 +865,26 @@ cudaError_t gemm_tc_launch(const GemmArgs &a, cudaStream_t stream) {
 }
 
 cudaError_t gemm_simt_launch(const __nv_bfloat16 *X, const __nv_bfloat16 *W, float *Y, int ldY, int M, int N,
-                             int K, int accumulate, cudaStream_t stream) {
+                             int K, int accumulate, cudaStream_t stream, int tiled, int part_rows) {
   dim3 grid((N + 15) / 16, (M + 15) / 16), block(16, 16);
-  gemm_simt_kernel<<<grid, block, 0, stream>>>(X, W, Y, ldY, M, N, K, accumulate);
+  gemm_simt_kernel<<<grid, block, 0, stream>>>(X, W, Y, ldY, M, N, K, accumulate, tiled, part_rows);
   return cudaGetLastError();
+}
+
+cudaError_t retile_launch(__nv_bfloat16 *dst, const __nv_bfloat16 *src, size_t rows, size_t cols, size_t dst_row0,
+                          cudaStream_t s) {
+  if (rows == 0 || cols == 0) return cudaSuccess;
+  if (cols % 8 || (reinterpret_cast<uintptr_t>(src) & 15) || (reinterpret_cast<uintptr_t>(dst) & 15))
+    return cudaErrorInvalidValue;
+  const size_t gx = (cols + kTileCols - 1) / kTileCols, gy = (rows + kTileRows - 1) / kTileRows;
+  if (gy > 65535 || gx > 0x7fffffff) return cudaErrorInvalidValue;
+  retile_kernel<<<dim3(static_cast<unsigned>(gx), static_cast<unsigned>(gy)), 256, 0, s>>>(dst, src, rows, cols, dst_row0);
+  return cudaGetLastError();
+}
+
+int make_tiled_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  const uint64_t blocks = ((rows + kTileRows - 1) / kTileRows) * ((cols + kTileCols - 1) / kTileCols);
+  return make_tensor_map(out, base, blocks * kTileRows, kTileCols, kTileCols, box_rows);
 }
 
 }  // namespace echo

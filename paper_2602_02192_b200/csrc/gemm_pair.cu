@@ -117,7 +117,7 @@ template <int BNB, int ACC>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                  const __grid_constant__ CUtensorMap tmY, int M, int N, int K, int epilogue, int split,
-                 int *status) {
+                 int tiled, int *status) {
   using S = PairSmem<BNB, ACC>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -166,9 +166,15 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
         uint8_t *dst = smem + s * S::kStageBytes;
         const uint32_t bar = map_to_cta(smem_u32(&full_bar[s]), 0);
         if (rank == 0) mbar_expect_tx(&full_bar[s], 2 * S::kStageBytes);
+        const int kb = kb_beg + it;
 #pragma unroll
-        for (int a = 0; a < ACC; ++a)
-          tma2_load_2d(&tmW, bar, dst + a * S::kWBlock, (kb_beg + it) * kGemmTileK, a * N + f0);
+        for (int a = 0; a < ACC; ++a) {
+          if (tiled)      // block (part a, feature block, kb) of the tiled storage: 16 KiB contiguous
+            tma2_load_2d(&tmW, bar, dst + a * S::kWBlock, 0,
+                         ((a * ((N + kPairFeat - 1) / kPairFeat) + f0 / kPairFeat) * KB + kb) * kPairFeat);
+          else
+            tma2_load_2d(&tmW, bar, dst + a * S::kWBlock, kb * kGemmTileK, a * N + f0);
+        }
       };
       auto load_x = [&](int it) {
         const int s = it % S::kStages;
@@ -321,7 +327,7 @@ cudaError_t launch_pair(const PairGemmArgs &a, int n_tiles, int m_tiles, int spl
   cfg.attrs = attr;
   cfg.numAttrs = a.allow_early_start ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<BNB, ACC>, *a.tmW, tmX, tmY, a.M, a.N, a.K, a.epilogue, split,
-                            a.status);
+                            a.tiled, a.status);
 }
 
 template <int BNB, int ACC>

@@ -18,6 +18,7 @@ using namespace echo;
 namespace {
 
 constexpr size_t kAlign = 1024;
+constexpr size_t kRetileStageBytes = 64ull << 20;
 constexpr int kChunkRows = 256;       // prompt tokens per prefill forward
 constexpr int kMaxCtas = 160;         // persistent GEMM grid never exceeds this (148 SMs on B200)
 
@@ -27,10 +28,12 @@ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 struct Dims {
   int L, d, Hq, Hkv, hd, F, V, Z;
   int n_qkv() const { return (Hq + 2 * Hkv) * hd; }
+  // projection matrices are stored block-tiled (padded to 128 x 64 blocks); embed and norms plain
   size_t layer_weight_elems() const {
-    return static_cast<size_t>(n_qkv()) * d + static_cast<size_t>(d) * Hq * hd + 3ull * F * d + 2ull * d;
+    return tiled_elems(n_qkv(), d) + tiled_elems(d, static_cast<size_t>(Hq) * hd) + 2 * tiled_elems(F, d) +
+           tiled_elems(d, F) + 2ull * d;
   }
-  size_t weight_elems() const { return L * layer_weight_elems() + 2ull * V * d + d; }
+  size_t weight_elems() const { return L * layer_weight_elems() + static_cast<size_t>(V) * d + tiled_elems(V, d) + d; }
 };
 
 struct Limits {
@@ -81,7 +84,7 @@ Limits limits_of(const echo_config &c) {
 struct Layout {
   size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
   size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
-      seq_len0, full_pages, pre_o, pre_ml, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
+      seq_len0, full_pages, pre_o, pre_ml, retile_stage, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
   size_t weight_bytes, kv_layer_elems, n_tables_ints;
   int n_chunks_max;
 };
@@ -121,6 +124,7 @@ Layout layout_of(const echo_config &c) {
   lo.full_pages = take(static_cast<size_t>(M.B) * 4);
   lo.pre_o = take(static_cast<size_t>(M.B) * D.Hq * D.hd * 4);
   lo.pre_ml = take(static_cast<size_t>(M.B) * D.Hq * 8);
+  lo.retile_stage = take(kRetileStageBytes);       // bounce buffer for snapshots in pageable host memory
   lo.copy_src = take(static_cast<size_t>(M.B) * 4);
   lo.copy_dst = take(static_cast<size_t>(M.B) * 4);
   lo.d_step = take(4);
@@ -265,7 +269,7 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
       gemm_pair_supported(Y, ldY, M, N, K, epilogue)) {
     // more than 64 rows: 2-CTA MMAs, k-slices added into Y in memory
     PairGemmArgs a{tmW_pair ? tmW_pair : tmW, X, Y, ldY, M, N, K, epilogue, ctx->ptr<int>(ctx->lo.status),
-                   ctx->use_pdl ? 1 : 0, 0};
+                   ctx->use_pdl ? 1 : 0, 0, 1};
     if (epilogue == EPI_STORE && !y_holds_zeros && gemm_pair_split(M, N, K, epilogue, 0) > 1) {
       CK(cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * ldY * sizeof(float), ctx->stream));
       a.allow_early_start = 0;
@@ -276,11 +280,12 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
   if (ctx->use_simt) {
     if (epilogue == EPI_SWIGLU) {
       float *gu = ctx->ptr<float>(ctx->lo.gu);
-      LAUNCH(gemm_simt_launch(X, W, gu, 2 * N, M, 2 * N, K, 0, ctx->stream));
+      LAUNCH(gemm_simt_launch(X, W, gu, 2 * N, M, 2 * N, K, 0, ctx->stream, 1, N));
       LAUNCH(swiglu_launch(gu, reinterpret_cast<__nv_bfloat16 *>(Y), M, N, ctx->stream));
       return ECHO_OK;
     }
-    LAUNCH(gemm_simt_launch(X, W, reinterpret_cast<float *>(Y), ldY, M, N, K, epilogue == EPI_ACCUM, ctx->stream));
+    LAUNCH(gemm_simt_launch(X, W, reinterpret_cast<float *>(Y), ldY, M, N, K, epilogue == EPI_ACCUM, ctx->stream, 1,
+                            0));
     return ECHO_OK;
   }
   CUtensorMap tmX;
@@ -291,7 +296,7 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
   }
   GemmArgs a{tmW, &tmX, Y, ldY, M, N, K, bnb, epilogue, ctx->ptr<int>(ctx->lo.status),
              ctx->ptr<float>(ctx->lo.gemm_ws), ctx->ptr<int>(ctx->lo.gemm_counters), kMaxCtas, 0, ctx->use_pdl ? 1 : 0,
-             ctx->deterministic ? 0 : 1};
+             ctx->deterministic ? 0 : 1, 1};
   if (a.independent_splits && epilogue == EPI_STORE && N < 8 * 4096 && !y_holds_zeros) {
     // the k-slices add into Y: it must start at zero.  The memset is the GEMM's predecessor on the
     // stream, so this launch does not use the early start.
@@ -367,16 +372,16 @@ void carve_weights(echo_ctx *ctx, WeightBuf &w, uint8_t *base) {
     return p;
   };
   w.embed = take(static_cast<size_t>(D.V) * D.d);
-  w.lm_head = take(static_cast<size_t>(D.V) * D.d);
+  w.lm_head = take(tiled_elems(D.V, D.d));
   w.final_norm = take(D.d);
   w.wqkv.resize(D.L); w.wo.resize(D.L); w.wgu.resize(D.L); w.wdown.resize(D.L);
   w.attn_norm.resize(D.L); w.mlp_norm.resize(D.L);
   w.tm_qkv.resize(D.L); w.tm_o.resize(D.L); w.tm_gu.resize(D.L); w.tm_down.resize(D.L); w.tm_gu_pair.resize(D.L);
   for (int l = 0; l < D.L; ++l) {
-    w.wqkv[l] = take(static_cast<size_t>(D.n_qkv()) * D.d);
-    w.wo[l] = take(static_cast<size_t>(D.d) * D.Hq * D.hd);
-    w.wgu[l] = take(2ull * D.F * D.d);
-    w.wdown[l] = take(static_cast<size_t>(D.d) * D.F);
+    w.wqkv[l] = take(tiled_elems(D.n_qkv(), D.d));                       // q, k, v rows of one matrix
+    w.wo[l] = take(tiled_elems(D.d, static_cast<size_t>(D.Hq) * D.hd));
+    w.wgu[l] = take(2 * tiled_elems(D.F, D.d));                          // gate part, then up part
+    w.wdown[l] = take(tiled_elems(D.d, D.F));
     w.attn_norm[l] = take(D.d);
     w.mlp_norm[l] = take(D.d);
   }
@@ -385,13 +390,14 @@ void carve_weights(echo_ctx *ctx, WeightBuf &w, uint8_t *base) {
 int make_weight_maps(echo_ctx *ctx, WeightBuf &w) {
   const Dims &D = ctx->D;
   int rc = 0;
-  rc |= make_tensor_map(&w.tm_lm, w.lm_head, D.V, D.d, D.d, kGemmTileN);
+  rc |= make_tiled_map(&w.tm_lm, w.lm_head, D.V, D.d, kGemmTileN);
+  const uint64_t gu_rows = 2ull * ((D.F + kTileRows - 1) / kTileRows) * kTileRows;     // both parts, padded
   for (int l = 0; l < D.L; ++l) {
-    rc |= make_tensor_map(&w.tm_qkv[l], w.wqkv[l], D.n_qkv(), D.d, D.d, kGemmTileN);
-    rc |= make_tensor_map(&w.tm_o[l], w.wo[l], D.d, D.Hq * D.hd, D.Hq * D.hd, kGemmTileN);
-    rc |= make_tensor_map(&w.tm_gu[l], w.wgu[l], 2ull * D.F, D.d, D.d, 64);
-    rc |= make_tensor_map(&w.tm_gu_pair[l], w.wgu[l], 2ull * D.F, D.d, D.d, kGemmTileN);
-    rc |= make_tensor_map(&w.tm_down[l], w.wdown[l], D.d, D.F, D.F, kGemmTileN);
+    rc |= make_tiled_map(&w.tm_qkv[l], w.wqkv[l], D.n_qkv(), D.d, kGemmTileN);
+    rc |= make_tiled_map(&w.tm_o[l], w.wo[l], D.d, D.Hq * D.hd, kGemmTileN);
+    rc |= make_tiled_map(&w.tm_gu[l], w.wgu[l], gu_rows, D.d, 64);
+    rc |= make_tiled_map(&w.tm_gu_pair[l], w.wgu[l], gu_rows, D.d, kGemmTileN);
+    rc |= make_tiled_map(&w.tm_down[l], w.wdown[l], D.d, D.F, kGemmTileN);
   }
   if (rc) {
     ctx->last_error = "tensor map encode failed (weights)";
@@ -736,6 +742,10 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
     return bail(e, "cudaStreamCreate");
   for (int b = 0; b < cfg->n_weight_buffers; ++b) {
     carve_weights(ctx, ctx->wb[b], ctx->arena + lo.weights[b]);
+    // the padding of the block-tiled matrices is never written again and must be zero (it meets
+    // zero-filled activation columns in the MMAs); installs run on the same stream, after this
+    if ((e = cudaMemsetAsync(ctx->arena + lo.weights[b], 0, lo.weight_bytes, ctx->copy_stream)) != cudaSuccess)
+      return bail(e, "cudaMemset");
     if ((e = cudaEventCreate(&ctx->wb[b].installed)) != cudaSuccess) return bail(e, "cudaEventCreate");
     if ((e = cudaEventCreate(&ctx->wb[b].inst_begin)) != cudaSuccess) return bail(e, "cudaEventCreate");
     if ((e = cudaEventCreateWithFlags(&ctx->wb[b].last_use, cudaEventDisableTiming)) != cudaSuccess)
@@ -851,18 +861,41 @@ int echo_load_policy(echo_ctx *ctx, const echo_weights *src, int64_t version) {
   auto cp = [&](void *dst, const void *s, size_t elems) {
     return cudaMemcpyAsync(dst, s, elems * 2, cudaMemcpyDefault, cs);
   };
+  // Row-major source matrix -> rows [row0, row0 + rows) of block-tiled storage.  The re-tiling
+  // kernel reads the source in place when the device can address it (device memory, page-locked
+  // or managed host memory); a snapshot in pageable host memory goes through a bounce buffer.
+  __nv_bfloat16 *stage = ctx->ptr<__nv_bfloat16>(ctx->lo.retile_stage);
+  auto tile = [&](__nv_bfloat16 *dst, const void *s, size_t rows, size_t cols, size_t row0) -> cudaError_t {
+    cudaPointerAttributes at;
+    const __nv_bfloat16 *dev_src = nullptr;
+    if (cudaPointerGetAttributes(&at, s) == cudaSuccess && at.type != cudaMemoryTypeUnregistered && at.devicePointer)
+      dev_src = static_cast<const __nv_bfloat16 *>(at.devicePointer);
+    else
+      (void)cudaGetLastError();
+    if (dev_src) return retile_launch(dst, dev_src, rows, cols, row0, cs);
+    const size_t chunk = kRetileStageBytes / (cols * 2);
+    if (chunk == 0) return cudaErrorInvalidValue;
+    for (size_t r = 0; r < rows; r += chunk) {
+      const size_t n = rows - r < chunk ? rows - r : chunk;
+      cudaError_t e = cudaMemcpyAsync(stage, static_cast<const __nv_bfloat16 *>(s) + r * cols, n * cols * 2,
+                                      cudaMemcpyDefault, cs);
+      if (e != cudaSuccess) return e;
+      if ((e = retile_launch(dst, stage, n, cols, row0 + r, cs)) != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+  };
   const size_t d = D.d, qd = static_cast<size_t>(D.Hq) * D.hd, kd = static_cast<size_t>(D.Hkv) * D.hd;
   CK(cp(w.embed, src->embed, static_cast<size_t>(D.V) * d));
-  CK(cp(w.lm_head, src->lm_head, static_cast<size_t>(D.V) * d));
+  CK(tile(w.lm_head, src->lm_head, D.V, d, 0));
   CK(cp(w.final_norm, src->final_norm, d));
   for (int l = 0; l < D.L; ++l) {
-    CK(cp(w.wqkv[l], src->wq[l], qd * d));
-    CK(cp(w.wqkv[l] + qd * d, src->wk[l], kd * d));
-    CK(cp(w.wqkv[l] + (qd + kd) * d, src->wv[l], kd * d));
-    CK(cp(w.wo[l], src->wo[l], d * qd));
-    CK(cp(w.wgu[l], src->w_gate[l], static_cast<size_t>(D.F) * d));
-    CK(cp(w.wgu[l] + static_cast<size_t>(D.F) * d, src->w_up[l], static_cast<size_t>(D.F) * d));
-    CK(cp(w.wdown[l], src->w_down[l], d * D.F));
+    CK(tile(w.wqkv[l], src->wq[l], qd, d, 0));
+    CK(tile(w.wqkv[l], src->wk[l], kd, d, qd));
+    CK(tile(w.wqkv[l], src->wv[l], kd, d, qd + kd));
+    CK(tile(w.wo[l], src->wo[l], d, qd, 0));
+    CK(tile(w.wgu[l], src->w_gate[l], D.F, d, 0));
+    CK(tile(w.wgu[l] + tiled_elems(D.F, d), src->w_up[l], D.F, d, 0));
+    CK(tile(w.wdown[l], src->w_down[l], d, D.F, 0));
     CK(cp(w.attn_norm[l], src->attn_norm[l], d));
     CK(cp(w.mlp_norm[l], src->mlp_norm[l], d));
   }
@@ -1067,21 +1100,29 @@ int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, 
   if (!X || !W || !Y || M < 1 || M > 4096 || N < 1 || K < 8 || (K % 8)) return ECHO_ERR_INVALID;
   if (epilogue != EPI_STORE && epilogue != EPI_ACCUM && epilogue != EPI_SWIGLU) return ECHO_ERR_INVALID;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const int tiled = impl >= 1000 ? 1 : 0;          // W is block-tiled storage (echo_retile_weights)
+  if (tiled) impl -= 1000;
   if (impl == 1) {
     if (epilogue == EPI_SWIGLU) return ECHO_ERR_INVALID;
     cudaError_t e = gemm_simt_launch(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(W),
-                                     static_cast<float *>(Y), N, M, N, K, epilogue == EPI_ACCUM, s);
+                                     static_cast<float *>(Y), N, M, N, K, epilogue == EPI_ACCUM, s, tiled, 0);
     return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
   }
+  // tiled storage of a gate/up pair: two parts of N rows, each padded to whole blocks
+  const uint64_t w_rows = epilogue == EPI_SWIGLU
+                              ? (tiled ? 2ull * ((N + kTileRows - 1) / kTileRows) * kTileRows : 2ull * N)
+                              : static_cast<uint64_t>(N);
+  auto w_map = [&](CUtensorMap *tm, uint32_t box_rows) {
+    return tiled ? make_tiled_map(tm, W, w_rows, K, box_rows) : make_tensor_map(tm, W, w_rows, K, K, box_rows);
+  };
   if (gemm_tc_configure() != cudaSuccess) return ECHO_ERR_CUDA;
   if (impl >= 300) {
     // SM-pair kernel, impl - 300 k-slices per tile (0 = choose)
     if (gemm_pair_configure() != cudaSuccess) return ECHO_ERR_CUDA;
     if (!gemm_pair_supported(Y, N, M, N, K, epilogue)) return ECHO_ERR_UNSUPPORTED;
-    const bool gu2 = epilogue == EPI_SWIGLU;
     CUtensorMap tmW2;
-    if (make_tensor_map(&tmW2, W, gu2 ? 2ull * N : N, K, K, kGemmTileN) != 0) return ECHO_ERR_CUDA;
-    PairGemmArgs pa{&tmW2, X, Y, N, M, N, K, epilogue, nullptr, 0, impl - 300};
+    if (w_map(&tmW2, kGemmTileN) != 0) return ECHO_ERR_CUDA;
+    PairGemmArgs pa{&tmW2, X, Y, N, M, N, K, epilogue, nullptr, 0, impl - 300, tiled};
     if (epilogue == EPI_STORE && gemm_pair_split(M, N, K, epilogue, impl - 300) > 1 &&
         cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * N * sizeof(float), s) != cudaSuccess)
       return ECHO_ERR_CUDA;
@@ -1096,7 +1137,7 @@ int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, 
   if (cudaMemsetAsync(counters, 0, static_cast<size_t>(kGemmMaxUnits) * 4, s) != cudaSuccess) return ECHO_ERR_CUDA;
   CUtensorMap tmW, tmX;
   const bool gu = epilogue == EPI_SWIGLU;
-  if (make_tensor_map(&tmW, W, gu ? 2ull * N : N, K, K, gu ? 64 : kGemmTileN) != 0) return ECHO_ERR_CUDA;
+  if (w_map(&tmW, gu ? 64 : kGemmTileN) != 0) return ECHO_ERR_CUDA;
   if (make_tensor_map(&tmX, X, M, K, K, bnb) != 0) return ECHO_ERR_CUDA;
   const bool indep = impl >= 200;
   const int split = indep ? impl - 200 : (impl >= 100 ? impl - 100 : (impl == 2 ? -1 : 0));
@@ -1105,8 +1146,24 @@ int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, 
       cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * N * sizeof(float), s) != cudaSuccess)
     return ECHO_ERR_CUDA;
   GemmArgs a{&tmW, &tmX, Y, N, M, N, K, bnb, epilogue, nullptr, static_cast<float *>(workspace), counters, 0, split, 0,
-             indep ? 1 : 0};
+             indep ? 1 : 0, tiled};
   cudaError_t e = gemm_tc_launch(a, s);
+  return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+size_t echo_tiled_weight_bytes(int64_t rows, int64_t cols) {
+  if (rows < 1 || cols < 1) return 0;
+  return tiled_elems(static_cast<size_t>(rows), static_cast<size_t>(cols)) * 2;
+}
+
+int echo_retile_weights(const void *src, int64_t rows, int64_t cols, void *dst, size_t dst_bytes, void *cuda_stream) {
+  if (!src || !dst || rows < 1 || cols < 8 || (cols % 8)) return ECHO_ERR_INVALID;
+  if (dst_bytes < echo_tiled_weight_bytes(rows, cols)) return ECHO_ERR_ARENA;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  // padding of partial blocks must read as zero
+  if (cudaMemsetAsync(dst, 0, echo_tiled_weight_bytes(rows, cols), s) != cudaSuccess) return ECHO_ERR_CUDA;
+  cudaError_t e = retile_launch(static_cast<__nv_bfloat16 *>(dst), static_cast<const __nv_bfloat16 *>(src),
+                                static_cast<size_t>(rows), static_cast<size_t>(cols), 0, s);
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }
 

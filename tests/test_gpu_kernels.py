@@ -84,7 +84,13 @@ def test_gemm_tensor_core_matches_fp64(B, M, N, K):
     tol = 2e-6 * K * 0.05 * 4 + 1e-6
     # 1 = SIMT reference, 0 = automatic choice, 2 = persistent stream-K, 100+s = cluster split-K by s
     # 200+s = independent k-slices added into the output in memory (s = 0: automatic)
-    impls = (1, 0, 2, 101, 103, 108, 200, 206) if N * K <= 4096 * 4096 else (0, 2, 200)
+    # 300+s = SM-pair kernel (more than 64 rows) with s k-slices; +1000 = weights in the block-tiled layout
+    impls = (1, 0, 2, 101, 103, 108, 200, 206, 1001, 1000, 1002, 1104, 1203) if N * K <= 4096 * 4096 else (0, 2, 200, 1000)
+    if M > 64:
+        impls += (300, 301, 303, 1300, 1302)
+    else:
+        with pytest.raises(B.EchoError):
+            B.echo_gemm_bf16(X.cuda(), W.cuda(), impl=300)
     for impl in impls:
         Y = B.echo_gemm_bf16(X.cuda(), W.cuda(), impl=impl)
         got = Y.cpu().numpy().astype(np.float64)
@@ -96,6 +102,12 @@ def test_gemm_tensor_core_matches_fp64(B, M, N, K):
     B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=1, Y=Y, impl=200)
     got = Y.cpu().numpy().astype(np.float64)
     assert np.max(np.abs(got - (Y0.cpu().numpy() + 2 * want))) < 2 * tol + 1e-5
+    if M > 64:
+        Y = Y0.clone()
+        B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=1, Y=Y, impl=300)
+        B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=1, Y=Y, impl=1300)
+        got = Y.cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(got - (Y0.cpu().numpy() + 2 * want))) < 2 * tol + 1e-5
 
 
 @pytest.mark.parametrize("M,F,K", [(256, 688, 256), (16, 64, 64), (77, 1000, 512), (256, 12288, 4096),
@@ -107,7 +119,7 @@ def test_gemm_swiglu_epilogue(B, M, F, K):
     xf, wf = widen_bf16(synth.bf16_bits(X)), widen_bf16(synth.bf16_bits(W))
     g, u = xf @ wf[:F].T, xf @ wf[F:].T
     want = g / (1 + np.exp(-g)) * u
-    for impl in (0, 2, 101, 104):
+    for impl in (0, 2, 101, 104, 1000, 1002) + ((300, 1300) if M > 64 else ()):
         Y = B.echo_gemm_bf16(X.cuda(), W.cuda(), epilogue=2, impl=impl)
         got = Y.float().cpu().numpy().astype(np.float64)
         # the output is rounded to bf16 (relative 2^-9) on top of the fp32 accumulation error
