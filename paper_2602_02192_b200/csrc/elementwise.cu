@@ -202,51 +202,81 @@ rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, _
                        int R, int Hq, int Hkv, int hd, int page_size, int n_pages, int max_pos, int *status) {
   early_start_sync();
   const int r = blockIdx.x;
-  const int pos = row_pos[r];
   const int half = hd / 2, q4 = half / 4;
   const int ld = (Hq + 2 * Hkv) * hd;
   float *src = qkv + static_cast<size_t>(r) * ld;
   const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  const int n_items = (Hq + Hkv) * q4;
+  // All loads of the row are issued before anything depends on the row's position, so the
+  // position -> page -> rotation-table chain runs under their latency.
+  constexpr int kItems = 3;                             // items per thread held in registers
+  float4 a[kItems], b[kItems], v0[kItems], v1[kItems];
+#pragma unroll
+  for (int j = 0; j < kItems; ++j) {
+    const int item = threadIdx.x + j * 256;
+    if (item < n_items) {
+      const int unit = item / q4, i = (item % q4) * 4;
+      a[j] = *reinterpret_cast<const float4 *>(src + unit * hd + i);
+      b[j] = *reinterpret_cast<const float4 *>(src + unit * hd + i + half);
+      if (unit >= Hq) {
+        v0[j] = *reinterpret_cast<const float4 *>(src + (unit + Hkv) * hd + i);
+        v1[j] = *reinterpret_cast<const float4 *>(src + (unit + Hkv) * hd + i + half);
+      }
+    }
+  }
+  const int pos = row_pos[r];
   int page = -1;
   if (pos >= 0 && pos < max_pos) page = page_table[static_cast<size_t>(row_pt[r]) * pt_width + pos / page_size];
-  if (page < 0 || page >= n_pages) {
-    if (threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
-    for (int i = threadIdx.x; i < ld / 4; i += blockDim.x) reinterpret_cast<float4 *>(src)[i] = zero4;
-    return;
-  }
-  const int off = pos % page_size;
-  const float4 *cs4 = reinterpret_cast<const float4 *>(rope_table + static_cast<size_t>(pos) * half);
+  const bool bad = page < 0 || page >= n_pages;
+  if (bad && threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
+  const int off = bad ? 0 : pos % page_size;
+  const float4 *cs4 = reinterpret_cast<const float4 *>(rope_table + static_cast<size_t>(bad ? 0 : pos) * half);
   const size_t page_elems = static_cast<size_t>(page_size) * hd;
-  const int n_items = (Hq + Hkv) * q4;
-  for (int item = threadIdx.x; item < n_items; item += blockDim.x) {
-    const int unit = item / q4, i = (item % q4) * 4;
-    float4 *pa = reinterpret_cast<float4 *>(src + unit * hd + i);
-    float4 *pb = reinterpret_cast<float4 *>(src + unit * hd + i + half);
-    const float4 a = *pa, b = *pb;
-    const float4 t01 = cs4[i / 2], t23 = cs4[i / 2 + 1];         // (cos, sin) of pairs i..i+3
-    *pa = zero4;
-    *pb = zero4;
-    const uint2 lo = pack_bf16x4(a.x * t01.x - b.x * t01.y, a.y * t01.z - b.y * t01.w, a.z * t23.x - b.z * t23.y,
-                                 a.w * t23.z - b.w * t23.w);
-    const uint2 hi = pack_bf16x4(b.x * t01.x + a.x * t01.y, b.y * t01.z + a.y * t01.w, b.z * t23.x + a.z * t23.y,
-                                 b.w * t23.z + a.w * t23.w);
-    if (unit < Hq) {
-      __nv_bfloat16 *dst = q + static_cast<size_t>(r) * Hq * hd + unit * hd + i;
-      *reinterpret_cast<uint2 *>(dst) = lo;
-      *reinterpret_cast<uint2 *>(dst + half) = hi;
-    } else {
-      const int head = unit - Hq;
-      __nv_bfloat16 *kd = kv_layer + ((static_cast<size_t>(page) * Hkv + head) * 2 + 0) * page_elems + off * hd + i;
-      *reinterpret_cast<uint2 *>(kd) = lo;
-      *reinterpret_cast<uint2 *>(kd + half) = hi;
+  for (int j0 = 0; j0 < (n_items + 255) / 256; j0 += kItems) {
+#pragma unroll
+    for (int j = 0; j < kItems; ++j) {
+      const int item = threadIdx.x + (j0 + j) * 256;
+      if (item >= n_items) continue;
+      const int unit = item / q4, i = (item % q4) * 4;
+      float4 *pa = reinterpret_cast<float4 *>(src + unit * hd + i);
+      float4 *pb = reinterpret_cast<float4 *>(src + unit * hd + i + half);
       float4 *va = reinterpret_cast<float4 *>(src + (unit + Hkv) * hd + i);
       float4 *vb = reinterpret_cast<float4 *>(src + (unit + Hkv) * hd + i + half);
-      const float4 v0 = *va, v1 = *vb;
-      *va = zero4;
-      *vb = zero4;
-      __nv_bfloat16 *vd = kd + page_elems;
-      *reinterpret_cast<uint2 *>(vd) = pack_bf16x4(v0.x, v0.y, v0.z, v0.w);
-      *reinterpret_cast<uint2 *>(vd + half) = pack_bf16x4(v1.x, v1.y, v1.z, v1.w);
+      if (j0 > 0) {                                     // rows longer than 3 x 256 items: load late
+        a[j] = *pa;
+        b[j] = *pb;
+        if (unit >= Hq) {
+          v0[j] = *va;
+          v1[j] = *vb;
+        }
+      }
+      // the row is consumed: leave zeros for the next projection, whose k-slices add into it
+      *pa = zero4;
+      *pb = zero4;
+      if (unit >= Hq) {
+        *va = zero4;
+        *vb = zero4;
+      }
+      if (bad) continue;
+      const float4 t01 = cs4[i / 2], t23 = cs4[i / 2 + 1];       // (cos, sin) of pairs i..i+3
+      const float4 x = a[j], y = b[j];
+      const uint2 lo = pack_bf16x4(x.x * t01.x - y.x * t01.y, x.y * t01.z - y.y * t01.w, x.z * t23.x - y.z * t23.y,
+                                   x.w * t23.z - y.w * t23.w);
+      const uint2 hi = pack_bf16x4(y.x * t01.x + x.x * t01.y, y.y * t01.z + x.y * t01.w, y.z * t23.x + x.z * t23.y,
+                                   y.w * t23.z + x.w * t23.w);
+      if (unit < Hq) {
+        __nv_bfloat16 *dst = q + static_cast<size_t>(r) * Hq * hd + unit * hd + i;
+        *reinterpret_cast<uint2 *>(dst) = lo;
+        *reinterpret_cast<uint2 *>(dst + half) = hi;
+      } else {
+        const int head = unit - Hq;
+        __nv_bfloat16 *kd = kv_layer + ((static_cast<size_t>(page) * Hkv + head) * 2 + 0) * page_elems + off * hd + i;
+        *reinterpret_cast<uint2 *>(kd) = lo;
+        *reinterpret_cast<uint2 *>(kd + half) = hi;
+        __nv_bfloat16 *vd = kd + page_elems;
+        *reinterpret_cast<uint2 *>(vd) = pack_bf16x4(v0[j].x, v0[j].y, v0[j].z, v0[j].w);
+        *reinterpret_cast<uint2 *>(vd + half) = pack_bf16x4(v1[j].x, v1[j].y, v1[j].z, v1[j].w);
+      }
     }
   }
 }
@@ -346,25 +376,41 @@ sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t
   Best best = {-INFINITY, 0x7fffffff};
   const int nblk = (V + 3) >> 2;
   const bool vec_ok = (V & 3) == 0;
-  for (int blk = threadIdx.x; blk < nblk; blk += blockDim.x) {
-    const uint4 w = philox4x32_10(make_uint4(static_cast<uint32_t>(blk), j, s_id, 0u), key);
-    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
-    float zz[4];
-    const int v0 = blk << 2;
-    if (vec_ok) {
-      const float4 t = *reinterpret_cast<const float4 *>(z + v0);
-      zz[0] = t.x; zz[1] = t.y; zz[2] = t.z; zz[3] = t.w;
-    } else {
+  // The two accurate logarithms of the Gumbel transform are what this kernel's time goes to, and
+  // almost no draw can win: -log1p(-w) >= w, so g <= -log(w), and a draw whose score plus that
+  // bound (taken with the fast logarithm and a margin far above its error) stays below the best
+  // perturbed score the warp has seen is skipped.  Skipping never changes the winner or a tie.
+  float warp_best = -INFINITY;
+  int it = 0;
+  for (int base = 0; base < nblk; base += blockDim.x, ++it) {       // same trip count in every thread
+    const int blk = base + threadIdx.x;
+    if (blk < nblk) {
+      const uint4 w = philox4x32_10(make_uint4(static_cast<uint32_t>(blk), j, s_id, 0u), key);
+      const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+      float zz[4];
+      const int v0 = blk << 2;
+      if (vec_ok) {
+        const float4 t = *reinterpret_cast<const float4 *>(z + v0);
+        zz[0] = t.x; zz[1] = t.y; zz[2] = t.z; zz[3] = t.w;
+      } else {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) zz[i] = (v0 + i < V) ? z[v0 + i] : -INFINITY;
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      if (v0 + i < V) {
-        const float s = zz[i] * inv_temperature;
-        lse_update(m, l, s);
-        best_update(best, s + gumbel_from_uniform(uniform_from_word(words[i])), v0 + i);
+        for (int i = 0; i < 4; ++i) zz[i] = (v0 + i < V) ? z[v0 + i] : -INFINITY;
       }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (v0 + i < V) {
+          const float s = zz[i] * inv_temperature;
+          lse_update(m, l, s);
+          const float u01 = uniform_from_word(words[i]);
+          if (s - __logf(u01) + 1e-3f >= warp_best) best_update(best, s + gumbel_from_uniform(u01), v0 + i);
+        }
+      }
+    }
+    if ((it & 3) == 3) {                     // every few blocks: share the best score across the warp
+      float b = best.score;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) b = fmaxf(b, __shfl_xor_sync(0xffffffffu, b, o));
+      warp_best = b;
     }
   }
   // warp reduction
