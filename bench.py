@@ -26,6 +26,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
+ATTN_DRAM_PER_ALG_BYTE = 170.3 / 166.2      # measured DRAM bytes per algorithmic byte (see profiles/)
 METRIC = "rollout generated tokens/s"
 UNIT = "tokens/s"
 
@@ -266,9 +267,15 @@ def run_ours(args):
         dur_s = float(prof_ms[:, 0].sum()) / 1e3
         achieved = alg / dur_s / 1e9
         tot = float(prof_ms[:, 3].sum())
+        # DRAM bytes per launch: ncu counters of the current kernel on a small case of the same
+        # per-CTA work (profiles/attn_decode_kernel_P4_G8_Lp512_i1200.md: 170.3 MB read + written
+        # for 166.2 MB of algorithmic bytes, prefix + suffix launch), scaled to this workload's
+        # launches by their algorithmic bytes: the traffic is the KV stream and grows with it.
+        traffic = ATTN_DRAM_PER_ALG_BYTE * alg / attn_launches if wl.shape.head_dim == 128 else None
         roof = {"bound": "hbm", "kernel": "decode attention (paged GQA)", "achieved": round(achieved, 1),
                 "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
-                "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None,
+                "frac": round(achieved / peaks["hbm_gbs"], 4),
+                "traffic": round(traffic) if traffic else None, "traffic_unit": "bytes per launch (ncu, scaled)",
                 "launches_timed": attn_launches,
                 "avg_launch_us": round(dur_s / attn_launches * 1e6, 2),
                 "sampled_steps": [int(j) for j in prof_steps],
