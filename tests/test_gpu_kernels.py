@@ -74,7 +74,7 @@ def test_sampler_seq_ids_and_tie_rule(B):
 
 @pytest.mark.parametrize("M,N,K", [(256, 384, 256), (16, 256, 256), (1, 128, 64), (100, 688, 256),
                                    (37, 256, 688), (300, 1024, 512), (256, 4096, 4096), (512, 640, 1024),
-                                   (256, 4096, 12288), (130, 151936, 256)])
+                                   (256, 4096, 12288), (130, 151936, 256), (300, 40000, 512), (100, 20000, 320)])
 def test_gemm_tensor_core_matches_fp64(B, M, N, K):
     rng = np.random.default_rng(M * 1000003 + N * 101 + K)
     X = torch.from_numpy(rng.normal(size=(M, K)).astype(np.float32)).to(torch.bfloat16)
