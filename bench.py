@@ -426,6 +426,63 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_projections(args):
+    """Diagnostic (--projections): every projection shape of one decode step of the workload, alone,
+    with rotating weight sets larger than L2, through echo_gemm_bf16 (SM-pair kernel, block-tiled
+    weights, fused epilogue) and, as context, through torch.matmul (cuBLAS, bf16 output, no epilogue).
+    One JSON line per shape."""
+    from paper_2602_02192_b200 import binding, synth
+    lib = binding.lib
+    wl = synth.WORKLOADS[args.workload]
+    sh = wl.shape
+    M = wl.n_prompts * wl.G
+    dev = torch.device("cuda:0")
+    nws = int(lib.echo_gemm_workspace_bytes(M))
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    qkv = (sh.n_q_heads + 2 * sh.n_kv_heads) * sh.head_dim
+    shapes = [("qkv", qkv, sh.d_model, 0), ("o", sh.d_model, sh.n_q_heads * sh.head_dim, 1),
+              ("gate_up_swiglu", sh.d_ff, sh.d_model, 2), ("down", sh.d_model, sh.d_ff, 1),
+              ("lm_head", sh.vocab, sh.d_model, 0)]
+
+    def timed(fn, iters):
+        for i in range(max(4, iters // 4)):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / iters
+
+    for name, N, K, epi in shapes:
+        rows_w = 2 * N if epi == 2 else N
+        nbuf = 2 if rows_w * K * 2 > 400e6 else int(400e6 // (rows_w * K * 2)) + 2
+        Ws = [torch.empty(rows_w, K, device=dev, dtype=torch.bfloat16).normal_(0, 0.02) for _ in range(nbuf)]
+        X = torch.empty(M, K, device=dev, dtype=torch.bfloat16).normal_()
+        Y = torch.zeros(M, N, device=dev, dtype=torch.bfloat16 if epi == 2 else torch.float32)
+        Yb = torch.empty(M, rows_w, device=dev, dtype=torch.bfloat16)
+        # timing only: the same buffers stand in for block-tiled storage (identical size for these shapes)
+        impl = 1300 if M > 64 else 1000
+
+        def ours(i):
+            rc = lib.echo_gemm_bf16(X.data_ptr(), Ws[i % nbuf].data_ptr(), Y.data_ptr(), M, N, K, epi, impl,
+                                    ws.data_ptr(), nws, st)
+            assert rc == 0, rc
+
+        def cublas(i):
+            torch.matmul(X, Ws[i % nbuf].t(), out=Yb)
+
+        t_ours, t_lib = timed(ours, 10 * nbuf), timed(cublas, 10 * nbuf)
+        flops = 2.0 * M * rows_w * K
+        print(json.dumps({"projection": name, "rows": M, "features": rows_w, "k": K, "epilogue": epi,
+                          "us": round(t_ours, 2), "weights_gbs": round(rows_w * K * 2 / t_ours / 1e3, 1),
+                          "tflops": round(flops / t_ours / 1e6, 1), "cublas_us": round(t_lib, 2),
+                          "cublas_tflops": round(flops / t_lib / 1e6, 1)}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -438,8 +495,12 @@ def main():
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (diagnostic runs only)")
     ap.add_argument("--no-swap", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--projections", action="store_true",
+                    help="diagnostic: time each projection shape alone (with cuBLAS beside it) and exit")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.projections:
+        run_projections(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
