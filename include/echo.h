@@ -62,7 +62,11 @@ typedef struct echo_config {
   int32_t max_new_tokens;     /* largest T                          */
   int32_t n_weight_buffers;   /* 2: a new snapshot installs while the old one serves
                                  (staleness bound 1); 1: installs block generation  */
-  int32_t eos_id;             /* must be -1: every sequence produces exactly T tokens */
+  int32_t eos_id;             /* -1: every sequence produces exactly T sampled tokens.  A token id in
+                                 [0, vocab): a sequence that emits it is finished; its later positions
+                                 hold eos_id with log-probability 0 (Section 5.1 generates up to a
+                                 maximum length; responses end earlier at the end token).  Finished
+                                 sequences keep their place in the batch until the call returns. */
 } echo_config;
 
 /* One snapshot: a pointer per tensor, bf16, row-major [out, in]; each pointer

@@ -237,10 +237,21 @@ class Rollout:
     version: int
 
 
+def _finish(toks, lps, mg, ru, p, g, j, eos_id):
+    """End-of-sequence rule: a sequence that has emitted eos_id is finished; every
+    later position holds eos_id with log-probability 0 (it is not sampled, so it
+    contributes nothing to a sum of log-probabilities) and an infinite margin."""
+    toks[p, g, j + 1:] = eos_id
+    lps[p, g, j + 1:] = 0.0
+    mg[p, g, j + 1:] = np.inf
+    ru[p, g, j + 1:] = eos_id
+
+
 def rollout_cached(dims, w, prompts, prompt_lens, G, T, temperature, seed,
-                   version: int = 0, share_prefix: bool = True) -> Rollout:
+                   version: int = 0, share_prefix: bool = True, eos_id: int = -1) -> Rollout:
     """Mode A.  share_prefix=False prefills every sample on its own (used to pin
-    prefix sharing)."""
+    prefix sharing).  eos_id >= 0 enables the end-of-sequence rule (Section 5.1
+    generates up to a maximum length: responses end earlier at the end token)."""
     P = len(prompts)
     toks = np.zeros((P, G, T), dtype=np.int32)
     lps = np.zeros((P, G, T))
@@ -260,13 +271,16 @@ def rollout_cached(dims, w, prompts, prompt_lens, G, T, temperature, seed,
                 d = sampler.draw(z, temperature, seed, s, j)
                 toks[p, g, j], lps[p, g, j], mg[p, g, j], ru[p, g, j] = \
                     d.token, d.logprob, d.margin, d.runner_up
+                if eos_id >= 0 and d.token == eos_id:
+                    _finish(toks, lps, mg, ru, p, g, j, eos_id)
+                    break
                 if j + 1 < T:
                     z = step(dims, w, d.token, cache)
     return Rollout(toks, lps, mg, ru, version)
 
 
 def rollout_recompute(dims, w, prompts, prompt_lens, G, T, temperature, seed,
-                      version: int = 0) -> Rollout:
+                      version: int = 0, eos_id: int = -1) -> Rollout:
     """Mode B: the whole sequence is recomputed for every new token."""
     P = len(prompts)
     toks = np.zeros((P, G, T), dtype=np.int32)
@@ -283,6 +297,9 @@ def rollout_recompute(dims, w, prompts, prompt_lens, G, T, temperature, seed,
                 d = sampler.draw(z, temperature, seed, s, j)
                 toks[p, g, j], lps[p, g, j], mg[p, g, j], ru[p, g, j] = \
                     d.token, d.logprob, d.margin, d.runner_up
+                if eos_id >= 0 and d.token == eos_id:
+                    _finish(toks, lps, mg, ru, p, g, j, eos_id)
+                    break
                 seq.append(d.token)
     return Rollout(toks, lps, mg, ru, version)
 
@@ -297,7 +314,7 @@ class Scored:
 
 
 def score_forced(dims, w, prompt, given_tokens, temperature, seed, s,
-                 layer_provider=None, steps: Optional[int] = None) -> Scored:
+                 layer_provider=None, steps: Optional[int] = None, eos_id: int = -1) -> Scored:
     """Mode C: teacher-forced along `given_tokens` (the T tokens some other
     implementation produced for sequence id s).  At step j the context is the
     prompt plus given_tokens[:j]; returns the log-prob of given_tokens[j] and the
@@ -309,9 +326,15 @@ def score_forced(dims, w, prompt, given_tokens, temperature, seed, s,
     z = forward_sequence(dims, w, seq, want_from=len(prompt) - 1, layer_provider=layer_provider)
     out = Scored(np.zeros(T), np.zeros(T, dtype=np.int32), np.zeros(T),
                  np.zeros(T, dtype=np.int32), np.zeros(T))
+    finished = False                 # the GIVEN tokens decide where the sequence ends
     for j in range(T):
+        if finished:
+            out.logprob_given[j], out.own_token[j], out.own_logprob[j] = 0.0, eos_id, 0.0
+            out.runner_up[j], out.margin[j] = eos_id, np.inf
+            continue
         d = sampler.draw(z[j], temperature, seed, s, j)
         out.logprob_given[j] = d.logprobs[given[j]]
         out.own_token[j], out.own_logprob[j] = d.token, d.logprob
         out.runner_up[j], out.margin[j] = d.runner_up, d.margin
+        finished = eos_id >= 0 and given[j] == eos_id
     return out

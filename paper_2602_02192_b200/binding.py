@@ -132,12 +132,12 @@ def _check(rc: int, ctx=None):
 
 
 def make_config(shape, max_prompts: int, max_G: int, max_prompt_len: int, max_new_tokens: int,
-                n_weight_buffers: int = 2, page_size: int = 16) -> EchoConfig:
+                n_weight_buffers: int = 2, page_size: int = 16, eos_id: int = -1) -> EchoConfig:
     """shape: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab,
     rms_eps, rope_theta attributes."""
     return EchoConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                       shape.d_ff, shape.vocab, shape.rms_eps, shape.rope_theta, page_size,
-                      max_prompts, max_G, max_prompt_len, max_new_tokens, n_weight_buffers, -1)
+                      max_prompts, max_G, max_prompt_len, max_new_tokens, n_weight_buffers, eos_id)
 
 
 def echo_arena_bytes(cfg: EchoConfig) -> int:

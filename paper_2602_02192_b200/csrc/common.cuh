@@ -165,7 +165,7 @@ cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, 
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row,
                            const int32_t *seq_ids, const int32_t *d_step, uint32_t j_host,
                            float temperature, uint64_t seed, const int32_t *forced, int forced_stride,
-                           int32_t *out_tok, float *out_lp, int out_stride, cudaStream_t s);
+                           int32_t *out_tok, float *out_lp, int out_stride, cudaStream_t s, int eos_id = -1);
 cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n,
                                uint32_t *words, float *uniform, cudaStream_t s);
 cudaError_t advantage_launch(const float *r, int P, int G, float eps, float *out, cudaStream_t s);

@@ -362,12 +362,25 @@ constexpr int kSamplerThreads = 1024;
 __global__ void __launch_bounds__(kSamplerThreads)
 sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t *seq_ids, const int32_t *d_step,
                uint32_t j_host, float inv_temperature, uint32_t key0, uint32_t key1, const int32_t *forced,
-               int forced_stride, int32_t *out_tok, float *out_lp, int out_stride) {
+               int forced_stride, int32_t *out_tok, float *out_lp, int out_stride, int eos_id) {
   __shared__ float sm_m[32], sm_l[32], sm_score[32];
   __shared__ int sm_id[32];
   early_start_sync();
   const int r = blockIdx.x;
   const uint32_t j = d_step ? static_cast<uint32_t>(*d_step) : j_host;
+  if (eos_id >= 0 && j > 0) {
+    // End-of-sequence rule: the sequence is finished once its previous token (the forced one when
+    // scoring a given trajectory) is eos_id; finished positions hold eos_id with log-probability 0.
+    const size_t prev = forced ? static_cast<size_t>(r) * forced_stride + (j - 1)
+                               : static_cast<size_t>(r) * out_stride + (j - 1);
+    if ((forced ? forced[prev] : out_tok[prev]) == eos_id) {
+      if (threadIdx.x == 0) {
+        out_tok[static_cast<size_t>(r) * out_stride + j] = eos_id;
+        out_lp[static_cast<size_t>(r) * out_stride + j] = 0.f;
+      }
+      return;
+    }
+  }
   const uint32_t s_id = seq_ids ? static_cast<uint32_t>(seq_ids[r]) : static_cast<uint32_t>(r);
   const float *z = logits + static_cast<size_t>(r / rows_per_logit_row) * V;
   const uint2 key = make_uint2(key0, key1);
@@ -525,10 +538,10 @@ cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, 
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row, const int32_t *seq_ids,
                            const int32_t *d_step, uint32_t j_host, float temperature, uint64_t seed,
                            const int32_t *forced, int forced_stride, int32_t *out_tok, float *out_lp, int out_stride,
-                           cudaStream_t s) {
+                           cudaStream_t s, int eos_id) {
   return launch_early(sampler_kernel, dim3(R), dim3(kSamplerThreads), 0, s, logits, V, rows_per_logit_row, seq_ids,
                       d_step, j_host, 1.0f / temperature, static_cast<uint32_t>(seed & 0xffffffffu),
-                      static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok, out_lp, out_stride);
+                      static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok, out_lp, out_stride, eos_id);
 }
 cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n, uint32_t *words,
                                float *uniform, cudaStream_t s) {

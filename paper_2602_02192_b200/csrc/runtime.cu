@@ -54,7 +54,7 @@ bool config_ok(const echo_config *c) {
   if (c->kv_page_size < 1 || c->kv_page_size > 256 || (c->kv_page_size * c->head_dim) % 8) return false;
   if (c->max_prompts < 1 || c->max_G < 1 || c->max_prompt_len < 1 || c->max_new_tokens < 1) return false;
   if (c->n_weight_buffers != 1 && c->n_weight_buffers != 2) return false;
-  if (c->eos_id != -1) return false;
+  if (c->eos_id < -1 || c->eos_id >= c->vocab) return false;
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return false;
   if (static_cast<long long>(c->max_prompts) * c->max_G > (1 << 20)) return false;
   return true;
@@ -571,7 +571,7 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
   {
     ProfScope prof(ctx, PROF_SAMPLER);
     LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, ctx->D.V, 1, nullptr, d_step, 0, temperature, seed,
-                          forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream));
+                          forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream, ctx->cfg.eos_id));
   }
   return ECHO_OK;
 }
@@ -627,7 +627,7 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   TRY(lm_head(ctx, w, ctx->ptr<float>(lo.xlast), P));
   LAUNCH(set_int_launch(ctx->ptr<int32_t>(lo.d_step), 0, ctx->stream));
   LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, D.V, G, nullptr, nullptr, 0, temperature, seed, forced, T,
-                        out_tokens, out_logprobs, T, ctx->stream));
+                        out_tokens, out_logprobs, T, ctx->stream, ctx->cfg.eos_id));
 
   CK(cudaEventRecord(ctx->ev_first, ctx->stream));
   // ---- decode steps 1..T-1 ----------------------------------------------------

@@ -32,7 +32,7 @@ def score_sequences(dims, w, prompts, lens, G, temperature, seed, tokens, logpro
 
 
 def check_sequences(dims, w, prompts, lens, G, temperature, seed, tokens, logprobs, seqs, steps=None,
-                    layer_provider=None):
+                    layer_provider=None, eos_id=-1):
     """Teacher-forced oracle scoring along the GPU's own tokens for the given sequence ids.
     Returns (n_checked, n_exempt, max |dlogprob|).  Asserts the acceptance rule."""
     n_checked = n_exempt = 0
@@ -40,7 +40,7 @@ def check_sequences(dims, w, prompts, lens, G, temperature, seed, tokens, logpro
     for s in seqs:
         p, g = divmod(s, G)
         sc = decoder.score_forced(dims, w, prompts[p][: int(lens[p])], tokens[p, g], temperature, seed, s,
-                                  layer_provider=layer_provider, steps=steps)
+                                  layer_provider=layer_provider, steps=steps, eos_id=eos_id)
         T = len(sc.own_token)
         for j in range(T):
             y = int(tokens[p, g, j])

@@ -39,7 +39,7 @@ def test_config_validation_needs_no_gpu():
     bad.head_dim = 48
     assert binding.echo_arena_bytes(bad) == 0
     bad = binding.make_config(shape, 4, 4, 32, 32)
-    bad.eos_id = 2
+    bad.eos_id = shape.vocab                 # the end token must be a token id (or -1)
     assert binding.echo_arena_bytes(bad) == 0
     assert binding.lib.echo_strerror(-5) == b"an install is still pending"
     # 8B-shape workload: 2 x 16.4 GB weights + ~80 GB KV must fit a 180 GB part

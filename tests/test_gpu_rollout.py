@@ -5,7 +5,7 @@ import torch
 
 from oracle import decoder, pages
 from paper_2602_02192_b200 import synth
-from helpers import assert_same_rollout, check_sequences, dims_of
+from helpers import LOGPROB_TOL, assert_same_rollout, check_sequences, dims_of
 
 pytestmark = pytest.mark.gpu
 
@@ -60,6 +60,42 @@ def test_tiny_config_full_parity(B, tiny):
     assert_same_rollout(tok2.cpu().numpy(), lp2.cpu().numpy(), tok, lp)
     st = eng.echo_get_stats()
     assert st["tokens_generated"] == tok.size and st["kernels_launched"] > 100
+    eng.close()
+
+
+def test_end_of_sequence_rule(B, tiny):
+    """eos_id set: a sequence that emits the end token holds eos / log-probability 0 from then on,
+    everything else is unchanged; checked against the oracle's rule, free-running and teacher-forced."""
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 3, 3, 20, 12
+    prompts = synth.make_prompts(P, Lp, wl.shape.vocab, 77)
+    lens = [Lp, Lp - 3, Lp]
+    dp = torch.from_numpy(prompts).cuda()
+    eng = _engine(B, wl.shape, P, G, Lp, T)
+    eng.echo_load_policy(w_d, 1)
+    tok0, lp0, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 123)
+    eng.echo_sync()
+    tok0 = tok0.cpu().numpy()
+    eng.close()
+    eos = int(tok0[1, 1, 4])
+    eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, eos_id=eos))
+    eng.echo_load_policy(w_d, 1)
+    tok, lp, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 123)
+    eng.echo_sync()
+    tok_h, lp_h = tok.cpu().numpy(), lp.cpu().numpy()
+    n, ex, worst = check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 1.0, 123, tok_h, lp_h, range(P * G),
+                                   eos_id=eos)
+    assert n == P * G * T and ex <= 2
+    e = int(np.flatnonzero(tok_h[1, 1] == eos)[0])
+    assert e <= 4 and np.all(tok_h[1, 1, e:] == eos) and np.all(lp_h[1, 1, e + 1:] == 0.0) and lp_h[1, 1, e] < 0
+    # teacher-forced along that trajectory: finished positions score 0 and "would sample" eos
+    tok_f, lp_f, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 123, forced=tok)
+    eng.echo_sync()
+    tok_f, lp_f = tok_f.cpu().numpy(), lp_f.cpu().numpy()
+    fin = np.zeros_like(tok_h, dtype=bool)
+    fin[..., 1:] = np.logical_or.accumulate(tok_h[..., :-1] == eos, axis=-1)
+    assert np.all(lp_f[fin] == 0.0) and np.all(tok_f[fin] == eos)
+    assert np.max(np.abs(lp_f - lp_h)[~fin]) < LOGPROB_TOL
     eng.close()
 
 

@@ -209,6 +209,41 @@ def test_cached_equals_recompute_equals_forced(tiny):
         assert np.allclose(z, zf, atol=1e-10)
 
 
+def test_end_of_sequence_rule(tiny):
+    """eos_id >= 0: a sequence ends at the first eos token it emits; later positions hold eos with
+    log-probability 0; everything before that, and every sequence that never emits it, is unchanged
+    (the noise streams do not depend on the trajectory).  Modes A, B and C agree."""
+    wl, dims, w = tiny
+    prompts = synth.make_prompts(2, 10, wl.shape.vocab, wl.prompt_seed)
+    lens = [10, 7]
+    G, T = 2, 6
+    base = decoder.rollout_cached(dims, w, prompts, lens, G, T, 1.0, wl.sample_seed)
+    p0, g0, j0 = 1, 0, 2
+    eos = int(base.tokens[p0, g0, j0])
+    a = decoder.rollout_cached(dims, w, prompts, lens, G, T, 1.0, wl.sample_seed, eos_id=eos)
+    b = decoder.rollout_recompute(dims, w, prompts, lens, G, T, 1.0, wl.sample_seed, eos_id=eos)
+    assert np.array_equal(a.tokens, b.tokens) and np.allclose(a.logprobs, b.logprobs, atol=1e-9)
+    for p in range(2):
+        for g in range(G):
+            hits = np.flatnonzero(base.tokens[p, g] == eos)
+            if len(hits) == 0:                      # never emitted: identical to the run without the rule
+                assert np.array_equal(a.tokens[p, g], base.tokens[p, g])
+                assert np.allclose(a.logprobs[p, g], base.logprobs[p, g], atol=1e-12)
+                continue
+            e = int(hits[0])
+            assert np.array_equal(a.tokens[p, g, : e + 1], base.tokens[p, g, : e + 1])
+            assert np.allclose(a.logprobs[p, g, : e + 1], base.logprobs[p, g, : e + 1], atol=1e-12)
+            assert np.all(a.tokens[p, g, e + 1:] == eos) and np.all(a.logprobs[p, g, e + 1:] == 0.0)
+            sc = decoder.score_forced(dims, w, prompts[p][:lens[p]], a.tokens[p, g], 1.0, wl.sample_seed,
+                                      p * G + g, eos_id=eos)
+            assert np.array_equal(sc.own_token, a.tokens[p, g])
+            assert np.allclose(sc.logprob_given, a.logprobs[p, g], atol=1e-9)
+    assert int(np.flatnonzero(base.tokens[p0, g0] == eos)[0]) <= j0 and np.all(a.tokens[p0, g0, j0 + 1:] == eos)
+    # the sum of log-probabilities of a finished sequence is that of its tokens up to and including eos
+    e = int(np.flatnonzero(a.tokens[p0, g0] == eos)[0])
+    assert math.isclose(a.logprobs[p0, g0].sum(), base.logprobs[p0, g0, : e + 1].sum(), rel_tol=1e-12)
+
+
 def test_prefix_shared_equals_per_sample_prefill(tiny):
     wl, dims, w = tiny
     prompts = synth.make_prompts(1, 10, wl.shape.vocab, 5)
