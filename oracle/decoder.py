@@ -248,7 +248,8 @@ def _finish(toks, lps, mg, ru, p, g, j, eos_id):
 
 
 def rollout_cached(dims, w, prompts, prompt_lens, G, T, temperature, seed,
-                   version: int = 0, share_prefix: bool = True, eos_id: int = -1) -> Rollout:
+                   version: int = 0, share_prefix: bool = True, eos_id: int = -1,
+                   top_p: float = 1.0) -> Rollout:
     """Mode A.  share_prefix=False prefills every sample on its own (used to pin
     prefix sharing).  eos_id >= 0 enables the end-of-sequence rule (Section 5.1
     generates up to a maximum length: responses end earlier at the end token)."""
@@ -268,7 +269,7 @@ def rollout_cached(dims, w, prompts, prompt_lens, G, T, temperature, seed,
             else:
                 cache, z = prefill(dims, w, prompt)
             for j in range(T):
-                d = sampler.draw(z, temperature, seed, s, j)
+                d = sampler.draw(z, temperature, seed, s, j, top_p)
                 toks[p, g, j], lps[p, g, j], mg[p, g, j], ru[p, g, j] = \
                     d.token, d.logprob, d.margin, d.runner_up
                 if eos_id >= 0 and d.token == eos_id:
@@ -280,7 +281,7 @@ def rollout_cached(dims, w, prompts, prompt_lens, G, T, temperature, seed,
 
 
 def rollout_recompute(dims, w, prompts, prompt_lens, G, T, temperature, seed,
-                      version: int = 0, eos_id: int = -1) -> Rollout:
+                      version: int = 0, eos_id: int = -1, top_p: float = 1.0) -> Rollout:
     """Mode B: the whole sequence is recomputed for every new token."""
     P = len(prompts)
     toks = np.zeros((P, G, T), dtype=np.int32)
@@ -294,7 +295,7 @@ def rollout_recompute(dims, w, prompts, prompt_lens, G, T, temperature, seed,
             seq = list(prompt)
             for j in range(T):
                 z = forward_sequence(dims, w, seq, want_from=len(seq) - 1)[0]
-                d = sampler.draw(z, temperature, seed, s, j)
+                d = sampler.draw(z, temperature, seed, s, j, top_p)
                 toks[p, g, j], lps[p, g, j], mg[p, g, j], ru[p, g, j] = \
                     d.token, d.logprob, d.margin, d.runner_up
                 if eos_id >= 0 and d.token == eos_id:
@@ -314,7 +315,8 @@ class Scored:
 
 
 def score_forced(dims, w, prompt, given_tokens, temperature, seed, s,
-                 layer_provider=None, steps: Optional[int] = None, eos_id: int = -1) -> Scored:
+                 layer_provider=None, steps: Optional[int] = None, eos_id: int = -1,
+                 top_p: float = 1.0) -> Scored:
     """Mode C: teacher-forced along `given_tokens` (the T tokens some other
     implementation produced for sequence id s).  At step j the context is the
     prompt plus given_tokens[:j]; returns the log-prob of given_tokens[j] and the
@@ -332,7 +334,7 @@ def score_forced(dims, w, prompt, given_tokens, temperature, seed, s,
             out.logprob_given[j], out.own_token[j], out.own_logprob[j] = 0.0, eos_id, 0.0
             out.runner_up[j], out.margin[j] = eos_id, np.inf
             continue
-        d = sampler.draw(z[j], temperature, seed, s, j)
+        d = sampler.draw(z[j], temperature, seed, s, j, top_p)
         out.logprob_given[j] = d.logprobs[given[j]]
         out.own_token[j], out.own_logprob[j] = d.token, d.logprob
         out.runner_up[j], out.margin[j] = d.runner_up, d.margin

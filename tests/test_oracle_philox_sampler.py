@@ -156,3 +156,66 @@ def test_gumbel_max_frequencies_match_softmax():
             counts[sampler.draw(z, T, seed=1234, s=s, j=j).token] += 1
     chi2 = float(((counts - n * p) ** 2 / (n * p)).sum())
     assert chi2 < 24.3          # chi-square, 7 dof, p = 1e-3
+
+
+# ---- nucleus (top-p) sampling ------------------------------------------------------------------
+
+def test_nucleus_worked_example_and_renormalised_logprob():
+    """p = (0.5, 0.3, 0.15, 0.05): top_p 0.9 keeps three tokens (0.8 < 0.9 <= 0.95), top_p 0.8 two,
+    top_p 0.5 one; the log-probabilities are those of p / mass."""
+    p = np.array([0.3, 0.05, 0.5, 0.15])
+    z = np.log(p)
+    for top_p, keep in [(0.9, [0, 2, 3]), (0.8, [0, 2]), (0.5, [2]), (0.95, [0, 2, 3]), (0.96, [0, 1, 2, 3])]:
+        m = sampler.nucleus_mask(sampler.log_softmax(z), top_p)
+        assert sorted(np.flatnonzero(m)) == keep, (top_p, np.flatnonzero(m))
+        d = sampler.draw(z, 1.0, 7, 0, 0, top_p)
+        mass = p[keep].sum()
+        assert d.nucleus_size == len(keep) and math.isclose(d.nucleus_mass, mass, rel_tol=1e-12)
+        assert d.token in keep and math.isclose(d.logprob, math.log(p[d.token] / mass), rel_tol=1e-12, abs_tol=1e-12)
+        assert math.isclose(np.exp(d.logprobs[m]).sum(), 1.0, rel_tol=1e-12) and np.all(np.isneginf(d.logprobs[~m]))
+
+
+def test_nucleus_limits_ties_and_nesting():
+    rng = np.random.default_rng(5)
+    z = rng.normal(size=50)
+    full = sampler.draw(z, 0.7, 3, 2, 1)
+    same = sampler.draw(z, 0.7, 3, 2, 1, top_p=1.0)
+    assert full.token == same.token and full.logprob == same.logprob and same.nucleus_size == 50
+    # a vanishing top_p keeps only the most probable token, whatever the noise
+    for j in range(20):
+        d = sampler.draw(z, 0.7, 3, 2, j, top_p=1e-9)
+        assert d.token == int(np.argmax(z)) and abs(d.logprob) < 1e-12 and d.nucleus_size == 1
+    # equal probabilities at the boundary: the lower id enters first
+    zt = np.log(np.array([0.4, 0.2, 0.2, 0.2]))
+    assert sorted(np.flatnonzero(sampler.nucleus_mask(sampler.log_softmax(zt), 0.55))) == [0, 1]
+    assert sorted(np.flatnonzero(sampler.nucleus_mask(sampler.log_softmax(zt), 0.65))) == [0, 1, 2]
+    # nuclei are nested in top_p, and each is the smallest top-k set that reaches the mass
+    lp = sampler.log_softmax(z)
+    p = np.exp(lp)
+    prev = np.zeros(50, dtype=bool)
+    for top_p in (0.1, 0.3, 0.5, 0.9, 0.99):
+        m = sampler.nucleus_mask(lp, top_p)
+        assert np.all(m[prev]) and p[m].sum() >= top_p
+        assert p[m].min() >= p[~m].max()                    # a top-k set
+        assert p[m].sum() - p[m].min() < top_p              # dropping its least likely member falls short
+        prev = m
+    with pytest.raises(ValueError):
+        sampler.nucleus_mask(lp, 0.0)
+
+
+def test_nucleus_frequencies_match_renormalised_distribution():
+    z = np.array([0.3, -1.2, 2.0, 0.0, 1.1, -0.4, 0.9, -2.5])
+    T, top_p = 0.8, 0.9
+    lp = sampler.log_softmax(z / T)
+    m = sampler.nucleus_mask(lp, top_p)
+    q = np.where(m, np.exp(lp), 0.0)
+    q /= q.sum()
+    n = 20000
+    counts = np.zeros(len(z))
+    for s in range(200):
+        for j in range(n // 200):
+            counts[sampler.draw(z, T, seed=99, s=s, j=j, top_p=top_p).token] += 1
+    assert np.all(counts[~m] == 0)
+    k = int(m.sum())
+    chi2 = float(((counts[m] - n * q[m]) ** 2 / (n * q[m])).sum())
+    assert k >= 3 and chi2 < {2: 13.8, 3: 16.3, 4: 18.5, 5: 20.5, 6: 22.5, 7: 24.3}[k - 1]    # p = 1e-3
