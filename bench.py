@@ -180,7 +180,7 @@ def run_ours(args):
         Lp = args.prompt_len
     swap = args.workload == "8B" and not args.no_swap
     nbuf = 1 if args.workload == "32B" else 2
-    eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, nbuf), device=local_rank)
+    eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, nbuf, top_p=args.top_p), device=local_rank)
     if args.workload == "32B":
         # 65 GB of weights: the snapshot stays in page-locked host memory so that the device holds it once
         weights = synth.make_weights_pinned(shape, wl.weight_seed, gen_device=dev)
@@ -300,6 +300,7 @@ def run_ours(args):
         "config": {"workload": f"{wl.name}-shape decoder: L{shape.n_layers} d{shape.d_model} "
                                f"{shape.n_q_heads}q/{shape.n_kv_heads}kv hd{shape.head_dim} F{shape.d_ff} "
                                f"V{shape.vocab}; {P} prompts x G={G}, prompt {Lp}, {T} new tokens, T=1.0",
+                   "top_p": args.top_p,
                    "policy_swap": "one echo_load_policy of a re-seeded weight set during timed step 0" if swap
                    else "none", "versions_served": versions_seen, "e2e_version": int(ver_e2e[0, 0]),
                    "install_ms": round(install_ms, 1),
@@ -503,6 +504,8 @@ def main():
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (diagnostic runs only)")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the prompt length (diagnostic runs only)")
     ap.add_argument("--no-swap", action="store_true")
+    ap.add_argument("--top-p", type=float, default=1.0,
+                    help="nucleus sampling (the paper samples with 0.95); 1.0 = the benchmark's untruncated sampling")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--projections", action="store_true",
                     help="diagnostic: time each projection shape alone (with cuBLAS beside it) and exit")

@@ -67,6 +67,10 @@ typedef struct echo_config {
                                  hold eos_id with log-probability 0 (Section 5.1 generates up to a
                                  maximum length; responses end earlier at the end token).  Finished
                                  sequences keep their place in the batch until the call returns. */
+  float   top_p;              /* nucleus sampling (Section 5.1 samples with top-p 0.95): tokens are ranked
+                                 by probability (ties: lower id first), the shortest prefix whose mass
+                                 reaches top_p is kept, and the recorded log-probability is renormalised
+                                 over it.  0 or 1: no truncation; otherwise in (0, 1). */
 } echo_config;
 
 /* One snapshot: a pointer per tensor, bf16, row-major [out, in]; each pointer
@@ -224,6 +228,16 @@ int echo_sample(const float *logits, int32_t R, int32_t V, int32_t rows_per_logi
                 const int32_t *seq_ids, uint32_t j, float temperature, uint64_t seed,
                 const int32_t *forced, int32_t *out_tokens, float *out_logprobs,
                 void *cuda_stream);
+
+/* echo_sample with nucleus truncation (0 < top_p < 1; top_p = 1 equals echo_sample).  A first
+ * kernel finds each logits row's cut (the last member of the nucleus) by histograms of probability
+ * mass over score bins, the sampler then draws among the ids at or before the cut and renormalises
+ * the log-probability over them; a forced token outside the nucleus scores -inf.  `cut_scratch`:
+ * dev, 8 bytes per logits row ((R + rows_per_logit_row - 1) / rows_per_logit_row rows). */
+int echo_sample_top_p(const float *logits, int32_t R, int32_t V, int32_t rows_per_logit_row,
+                      const int32_t *seq_ids, uint32_t j, float temperature, float top_p, uint64_t seed,
+                      const int32_t *forced, int32_t *out_tokens, float *out_logprobs, void *cut_scratch,
+                      void *cuda_stream);
 
 /* Decode-step attention alone (paged GQA with the group's prompt pages read once for all G
  * samples).  B = P*G sequences, sequence s = p*G + g.

@@ -37,6 +37,7 @@ class EchoConfig(C.Structure):
         ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("kv_page_size", C.c_int32),
         ("max_prompts", C.c_int32), ("max_G", C.c_int32), ("max_prompt_len", C.c_int32),
         ("max_new_tokens", C.c_int32), ("n_weight_buffers", C.c_int32), ("eos_id", C.c_int32),
+        ("top_p", C.c_float),
     ]
 
 
@@ -83,6 +84,8 @@ def _load() -> C.CDLL:
     lib.echo_plan_page_table.restype = C.c_int
     lib.echo_debug_noise.argtypes = [u64, u32, u32, u32, u32, vp, vp, vp]
     lib.echo_sample.argtypes = [vp, i32, i32, i32, vp, u32, f32, u64, vp, vp, vp, vp]
+    lib.echo_sample_top_p.argtypes = [vp, i32, i32, i32, vp, u32, f32, f32, u64, vp, vp, vp, vp, vp]
+    lib.echo_sample_top_p.restype = C.c_int
     lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]
     lib.echo_decode_attention.argtypes = [vp, vp, i32, vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, vp]
     lib.echo_decode_attention.restype = C.c_int
@@ -115,7 +118,7 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
             "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_decode_attention",
             "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error",
-            "echo_tiled_weight_bytes", "echo_retile_weights"]
+            "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -132,12 +135,13 @@ def _check(rc: int, ctx=None):
 
 
 def make_config(shape, max_prompts: int, max_G: int, max_prompt_len: int, max_new_tokens: int,
-                n_weight_buffers: int = 2, page_size: int = 16, eos_id: int = -1) -> EchoConfig:
+                n_weight_buffers: int = 2, page_size: int = 16, eos_id: int = -1,
+                top_p: float = 1.0) -> EchoConfig:
     """shape: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab,
     rms_eps, rope_theta attributes."""
     return EchoConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                       shape.d_ff, shape.vocab, shape.rms_eps, shape.rope_theta, page_size,
-                      max_prompts, max_G, max_prompt_len, max_new_tokens, n_weight_buffers, eos_id)
+                      max_prompts, max_G, max_prompt_len, max_new_tokens, n_weight_buffers, eos_id, top_p)
 
 
 def echo_arena_bytes(cfg: EchoConfig) -> int:
@@ -310,6 +314,25 @@ def echo_sample(logits: torch.Tensor, rows: int, rows_per_logit_row: int, j: int
                                int(seed), forced.data_ptr() if forced is not None else None,
                                tok.data_ptr(), lp.data_ptr(), _stream_ptr(None)))
     return tok, lp
+
+
+def echo_sample_top_p(logits: torch.Tensor, rows: int, rows_per_logit_row: int, j: int, temperature: float,
+                      top_p: float, seed: int, seq_ids: Optional[torch.Tensor] = None,
+                      forced: Optional[torch.Tensor] = None):
+    """echo_sample with nucleus truncation; returns (tokens, logprobs, cuts) where cuts[row] = (score key, id)
+    of the last nucleus member of each logits row."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    V = logits.shape[-1]
+    tok = torch.empty(rows, dtype=torch.int32, device=logits.device)
+    lp = torch.empty(rows, dtype=torch.float32, device=logits.device)
+    n_rows = (rows + rows_per_logit_row - 1) // rows_per_logit_row
+    cuts = torch.zeros((n_rows, 2), dtype=torch.int64, device=logits.device).to(torch.int32).contiguous()
+    with torch.cuda.device(logits.device):
+        _check(lib.echo_sample_top_p(logits.data_ptr(), rows, V, rows_per_logit_row,
+                                     seq_ids.data_ptr() if seq_ids is not None else None, j, float(temperature),
+                                     float(top_p), int(seed), forced.data_ptr() if forced is not None else None,
+                                     tok.data_ptr(), lp.data_ptr(), cuts.data_ptr(), _stream_ptr(None)))
+    return tok, lp, cuts
 
 
 def echo_gemm_bf16(X: torch.Tensor, W: torch.Tensor, impl: int = 0, epilogue: int = 0,

@@ -46,6 +46,11 @@ inline cudaError_t launch_early(void (*kernel)(KArgs...), dim3 grid, dim3 block,
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #ifdef __CUDACC__
+// order-preserving 32-bit key of a float: a < b  <=>  order_key(a) < order_key(b)
+__device__ __forceinline__ uint32_t order_key(float s) {
+  const uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
 __device__ __forceinline__ void early_start_sync() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -165,7 +170,12 @@ cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, 
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row,
                            const int32_t *seq_ids, const int32_t *d_step, uint32_t j_host,
                            float temperature, uint64_t seed, const int32_t *forced, int forced_stride,
-                           int32_t *out_tok, float *out_lp, int out_stride, cudaStream_t s, int eos_id = -1);
+                           int32_t *out_tok, float *out_lp, int out_stride, cudaStream_t s, int eos_id = -1,
+                           const uint2 *nucleus_cut = nullptr);   // per logits row, from nucleus_cut_launch
+// Nucleus (top-p) cut of each logits row: cut[row] = (order-preserving key of the score of the last
+// nucleus member, its id; id 0x7fffffff = every id of that score).  nucleus.cu
+cudaError_t nucleus_cut_launch(const float *logits, int rows, int V, float temperature, float top_p, uint2 *cut,
+                               cudaStream_t s);
 cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n,
                                uint32_t *words, float *uniform, cudaStream_t s);
 cudaError_t advantage_launch(const float *r, int P, int G, float eps, float *out, cudaStream_t s);

@@ -362,7 +362,8 @@ constexpr int kSamplerThreads = 1024;
 __global__ void __launch_bounds__(kSamplerThreads)
 sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t *seq_ids, const int32_t *d_step,
                uint32_t j_host, float inv_temperature, uint32_t key0, uint32_t key1, const int32_t *forced,
-               int forced_stride, int32_t *out_tok, float *out_lp, int out_stride, int eos_id) {
+               int forced_stride, int32_t *out_tok, float *out_lp, int out_stride, int eos_id,
+               const uint2 *nucleus_cut) {
   __shared__ float sm_m[32], sm_l[32], sm_score[32];
   __shared__ int sm_id[32];
   early_start_sync();
@@ -384,6 +385,15 @@ sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t
   const uint32_t s_id = seq_ids ? static_cast<uint32_t>(seq_ids[r]) : static_cast<uint32_t>(r);
   const float *z = logits + static_cast<size_t>(r / rows_per_logit_row) * V;
   const uint2 key = make_uint2(key0, key1);
+  // top-p: only ids that rank at or before the row's cut (score descending, id ascending) belong to
+  // the distribution; the sum below then runs over the nucleus, which renormalises the log-probability
+  const bool topp = nucleus_cut != nullptr;
+  const uint2 cutv = topp ? nucleus_cut[r / rows_per_logit_row] : make_uint2(0u, 0x7fffffffu);
+  auto in_nucleus = [&](float s, int id) -> bool {
+    if (!topp) return true;
+    const uint32_t k = order_key(s);
+    return k > cutv.x || (k == cutv.x && static_cast<uint32_t>(id) <= cutv.y);
+  };
 
   float m = -INFINITY, l = 0.f;
   Best best = {-INFINITY, 0x7fffffff};
@@ -413,6 +423,7 @@ sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t
       for (int i = 0; i < 4; ++i) {
         if (v0 + i < V) {
           const float s = zz[i] * inv_temperature;
+          if (!in_nucleus(s, v0 + i)) continue;
           lse_update(m, l, s);
           const float u01 = uniform_from_word(words[i]);
           if (s - __logf(u01) + 1e-3f >= warp_best) best_update(best, s + gumbel_from_uniform(u01), v0 + i);
@@ -453,7 +464,8 @@ sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t
     out_tok[o] = tok;
     const int scored = forced ? forced[static_cast<size_t>(r) * forced_stride + j] : tok;
     const int sc_id = (scored >= 0 && scored < V) ? scored : 0;
-    out_lp[o] = z[sc_id] * inv_temperature - (mm + logf(ll));
+    const float s_sc = z[sc_id] * inv_temperature;
+    out_lp[o] = in_nucleus(s_sc, sc_id) ? s_sc - (mm + logf(ll)) : -INFINITY;
   }
 }
 
@@ -538,10 +550,11 @@ cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, 
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row, const int32_t *seq_ids,
                            const int32_t *d_step, uint32_t j_host, float temperature, uint64_t seed,
                            const int32_t *forced, int forced_stride, int32_t *out_tok, float *out_lp, int out_stride,
-                           cudaStream_t s, int eos_id) {
+                           cudaStream_t s, int eos_id, const uint2 *nucleus_cut) {
   return launch_early(sampler_kernel, dim3(R), dim3(kSamplerThreads), 0, s, logits, V, rows_per_logit_row, seq_ids,
                       d_step, j_host, 1.0f / temperature, static_cast<uint32_t>(seed & 0xffffffffu),
-                      static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok, out_lp, out_stride, eos_id);
+                      static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok, out_lp, out_stride, eos_id,
+                      nucleus_cut);
 }
 cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n, uint32_t *words,
                                float *uniform, cudaStream_t s) {

@@ -55,6 +55,7 @@ bool config_ok(const echo_config *c) {
   if (c->max_prompts < 1 || c->max_G < 1 || c->max_prompt_len < 1 || c->max_new_tokens < 1) return false;
   if (c->n_weight_buffers != 1 && c->n_weight_buffers != 2) return false;
   if (c->eos_id < -1 || c->eos_id >= c->vocab) return false;
+  if (!(c->top_p >= 0.f) || c->top_p > 1.f) return false;
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return false;
   if (static_cast<long long>(c->max_prompts) * c->max_G > (1 << 20)) return false;
   return true;
@@ -84,7 +85,7 @@ Limits limits_of(const echo_config &c) {
 struct Layout {
   size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
   size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
-      seq_len0, full_pages, pre_o, pre_ml, retile_stage, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
+      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
   size_t weight_bytes, kv_layer_elems, n_tables_ints;
   int n_chunks_max;
 };
@@ -125,6 +126,7 @@ Layout layout_of(const echo_config &c) {
   lo.pre_o = take(static_cast<size_t>(M.B) * D.Hq * D.hd * 4);
   lo.pre_ml = take(static_cast<size_t>(M.B) * D.Hq * 8);
   lo.retile_stage = take(kRetileStageBytes);       // bounce buffer for snapshots in pageable host memory
+  lo.nucleus_cut = take(static_cast<size_t>(M.B) * 8);   // top-p: one (score key, id) cut per logits row
   lo.copy_src = take(static_cast<size_t>(M.B) * 4);
   lo.copy_dst = take(static_cast<size_t>(M.B) * 4);
   lo.d_step = take(4);
@@ -570,8 +572,14 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
   TRY(lm_head(ctx, w, ctx->ptr<float>(lo.x), pl.B));
   {
     ProfScope prof(ctx, PROF_SAMPLER);
+    const uint2 *cut = nullptr;
+    if (ctx->cfg.top_p > 0.f && ctx->cfg.top_p < 1.f) {
+      LAUNCH(nucleus_cut_launch(ctx->ptr<float>(lo.logits), pl.B, ctx->D.V, temperature, ctx->cfg.top_p,
+                                ctx->ptr<uint2>(lo.nucleus_cut), ctx->stream));
+      cut = ctx->ptr<uint2>(lo.nucleus_cut);
+    }
     LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, ctx->D.V, 1, nullptr, d_step, 0, temperature, seed,
-                          forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream, ctx->cfg.eos_id));
+                          forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream, ctx->cfg.eos_id, cut));
   }
   return ECHO_OK;
 }
@@ -626,8 +634,14 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   // ---- first token of every sample from the prompt's last logits row --------
   TRY(lm_head(ctx, w, ctx->ptr<float>(lo.xlast), P));
   LAUNCH(set_int_launch(ctx->ptr<int32_t>(lo.d_step), 0, ctx->stream));
+  const uint2 *cut0 = nullptr;
+  if (ctx->cfg.top_p > 0.f && ctx->cfg.top_p < 1.f) {
+    LAUNCH(nucleus_cut_launch(ctx->ptr<float>(lo.logits), P, D.V, temperature, ctx->cfg.top_p,
+                              ctx->ptr<uint2>(lo.nucleus_cut), ctx->stream));
+    cut0 = ctx->ptr<uint2>(lo.nucleus_cut);
+  }
   LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, D.V, G, nullptr, nullptr, 0, temperature, seed, forced, T,
-                        out_tokens, out_logprobs, T, ctx->stream, ctx->cfg.eos_id));
+                        out_tokens, out_logprobs, T, ctx->stream, ctx->cfg.eos_id, cut0));
 
   CK(cudaEventRecord(ctx->ev_first, ctx->stream));
   // ---- decode steps 1..T-1 ----------------------------------------------------
@@ -1050,6 +1064,26 @@ int echo_sample(const float *logits, int32_t R, int32_t V, int32_t rows_per_logi
   cudaError_t e = sampler_launch(logits, R, V, rows_per_logit_row, seq_ids, nullptr, j, temperature, seed,
                                  forced ? forced - j : nullptr, 1, out_tokens - j, out_logprobs - j, 1,
                                  static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+int echo_sample_top_p(const float *logits, int32_t R, int32_t V, int32_t rows_per_logit_row, const int32_t *seq_ids,
+                      uint32_t j, float temperature, float top_p, uint64_t seed, const int32_t *forced,
+                      int32_t *out_tokens, float *out_logprobs, void *cut_scratch, void *cuda_stream) {
+  if (!logits || !out_tokens || !out_logprobs || R < 0 || V < 1 || rows_per_logit_row < 1) return ECHO_ERR_INVALID;
+  if (!(temperature > 0.f) || !std::isfinite(temperature) || !(top_p > 0.f) || !(top_p <= 1.f)) return ECHO_ERR_INVALID;
+  if (R == 0) return ECHO_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const uint2 *cut = nullptr;
+  if (top_p < 1.f) {
+    if (!cut_scratch || (reinterpret_cast<uintptr_t>(cut_scratch) & 7)) return ECHO_ERR_INVALID;
+    const int rows = (R + rows_per_logit_row - 1) / rows_per_logit_row;
+    if (nucleus_cut_launch(logits, rows, V, temperature, top_p, static_cast<uint2 *>(cut_scratch), s) != cudaSuccess)
+      return ECHO_ERR_CUDA;
+    cut = static_cast<const uint2 *>(cut_scratch);
+  }
+  cudaError_t e = sampler_launch(logits, R, V, rows_per_logit_row, seq_ids, nullptr, j, temperature, seed,
+                                 forced ? forced - j : nullptr, 1, out_tokens - j, out_logprobs - j, 1, s, -1, cut);
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }
 

@@ -57,6 +57,78 @@ def test_sampler_matches_oracle(B, V, R, G, temp):
         assert abs(lp_f[r] - d.logprobs[int(forced[r])]) < 2e-5 * max(1.0, abs(d.logprobs[int(forced[r])]))
 
 
+def _row(kind, V, rng):
+    if kind == "normal":
+        return (rng.normal(size=V) * 1.3).astype(np.float32)
+    if kind == "peaked":
+        z = (rng.normal(size=V) * 0.5).astype(np.float32)
+        z[rng.integers(0, V, size=5)] += np.float32(9.0)
+        return z
+    if kind == "equal":
+        return np.full(V, 0.25, dtype=np.float32)
+    if kind == "levels":                               # many exactly equal scores on a few levels
+        return (np.round(rng.normal(size=V) * 2.0) / 2.0).astype(np.float32)
+    raise ValueError(kind)
+
+
+@pytest.mark.parametrize("V,kind,top_p,temp", [(8, "normal", 0.9, 1.0), (1000, "normal", 0.5, 0.7),
+                                               (4096, "peaked", 0.95, 1.0), (151936, "normal", 0.95, 1.0),
+                                               (151936, "equal", 0.95, 1.0), (151936, "levels", 0.9, 1.0),
+                                               (50000, "levels", 0.3, 1.3), (151936, "peaked", 0.05, 1.0),
+                                               (4096, "normal", 1.0, 1.0)])
+def test_top_p_sampler_matches_oracle(B, V, kind, top_p, temp):
+    """Nucleus cut, draw and renormalised log-probability against the oracle.  The cut is found from
+    fp32 mass sums, so it may sit a few ids away from the oracle's fp64 one: the kernel's nucleus must
+    be a prefix of the ranking whose mass reaches top_p and is minimal, both within 3e-5 of mass."""
+    rng = np.random.default_rng(V + int(top_p * 1000))
+    R = 6
+    z = np.stack([_row(kind, V, rng) for _ in range(R)])
+    seed, j = 0xABCDEF0123, 2
+    zc = torch.from_numpy(z).cuda()
+    tok, lp, cuts = B.echo_sample_top_p(zc, R, 1, j, temp, top_p, seed)
+    forced = torch.from_numpy(rng.integers(0, V, size=R).astype(np.int32)).cuda()
+    tok_f, lp_f, _ = B.echo_sample_top_p(zc, R, 1, j, temp, top_p, seed, forced=forced)
+    tok, lp, tok_f, lp_f = tok.cpu().numpy(), lp.cpu().numpy(), tok_f.cpu().numpy(), lp_f.cpu().numpy()
+    cuts = cuts.cpu().numpy().view(np.uint32)
+    inv_t = np.float32(1.0) / np.float32(temp)
+    ids = np.arange(V)
+    for r in range(R):
+        d = o_sampler.draw(z[r], temp, seed, r, j, top_p)
+        lp_full = o_sampler.log_softmax(z[r].astype(np.float64) / temp)
+        p = np.exp(lp_full)
+        if top_p >= 1.0:
+            mask = np.ones(V, dtype=bool)
+        else:
+            s32 = z[r] * inv_t                                   # the kernel's scores
+            u = s32.view(np.uint32)
+            key = np.where(u & 0x80000000, ~u, u | 0x80000000).astype(np.uint64)
+            ck, cid = int(cuts[r, 0]), int(cuts[r, 1])
+            mask = (key > ck) | ((key == ck) & (ids <= cid))
+            order = np.lexsort((ids, -s32.astype(np.float64)))
+            k = int(mask.sum())
+            assert k >= 1 and np.all(mask[order[:k]])            # a prefix of the ranking
+            mass = p[mask].sum()
+            assert mass >= top_p - 3e-5                          # reaches the target ...
+            assert mass - p[order[k - 1]] < top_p + 3e-5         # ... and no shorter prefix does
+            assert abs(k - d.nucleus_size) <= 8                  # a few ids around the oracle's cut
+        mass = p[mask].sum()
+        assert mask[tok[r]]
+        if tok[r] != d.token:
+            both = mask & np.isfinite(d.logprobs)
+            assert (d.margin < 1e-4 and tok[r] == d.runner_up) or not both[d.token] or not both[tok[r]]
+        want = lp_full[tok[r]] - np.log(mass)
+        assert abs(lp[r] - want) < 3e-5 * max(1.0, abs(want))
+        if np.isfinite(d.logprobs[tok[r]]):
+            assert abs(lp[r] - d.logprobs[tok[r]]) < 1e-4
+        assert tok_f[r] == tok[r]
+        f = int(forced[r])
+        if mask[f]:
+            wf = lp_full[f] - np.log(mass)
+            assert abs(lp_f[r] - wf) < 3e-5 * max(1.0, abs(wf))
+        else:
+            assert np.isneginf(lp_f[r])
+
+
 def test_sampler_seq_ids_and_tie_rule(B):
     V = 64
     z = np.zeros((1, V), dtype=np.float32)

@@ -99,6 +99,35 @@ def test_end_of_sequence_rule(B, tiny):
     eng.close()
 
 
+def test_top_p_rollout(B, tiny):
+    """Nucleus sampling inside the engine (config top_p): every token and renormalised log-probability
+    against the oracle, teacher-forced along the GPU's tokens; a smaller top_p gives log-probabilities
+    that are never lower than the untruncated ones for the same tokens."""
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 3, 4, 24, 10
+    prompts = synth.make_prompts(P, Lp, wl.shape.vocab, 31)
+    lens = [Lp, Lp - 5, Lp]
+    dp = torch.from_numpy(prompts).cuda()
+    top_p = 0.9
+    eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, top_p=top_p))
+    eng.echo_load_policy(w_d, 1)
+    tok, lp, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 2024)
+    eng.echo_sync()
+    tok_h, lp_h = tok.cpu().numpy(), lp.cpu().numpy()
+    n, ex, worst = check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 1.0, 2024, tok_h, lp_h, range(P * G),
+                                   top_p=top_p)
+    assert n == P * G * T and ex <= 0.05 * n and np.all(lp_h <= 0)
+    eng.close()
+    # the same tokens scored without truncation: log p - log(nucleus mass) >= log p
+    eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T))
+    eng.echo_load_policy(w_d, 1)
+    _, lp_full, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 2024, forced=tok)
+    eng.echo_sync()
+    d = lp_h - lp_full.cpu().numpy()
+    assert np.all(d > -1e-3) and np.all(d < -np.log(top_p) + 5e-2) and d.mean() > 0.02
+    eng.close()
+
+
 def test_forced_rollout_scores_oracle_trajectory(B, tiny):
     wl, w_o, w_d = tiny
     P, G, Lp, T = 2, 3, 20, 12                    # Lp not a multiple of the page size
