@@ -148,6 +148,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     mbar_init(acc_full, 1);
     *abort_flag = 0;
     mbar_fence_init();
+    // fetch the three tensor maps now, not at the first copy that uses each of them
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmW)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
   }
   if (warp == 1) tc2_alloc(tmem_slot, S::kTmemCols);
   tc_fence_before();
