@@ -180,6 +180,19 @@ int echo_rollout_host(echo_ctx *ctx, const int32_t *prompts_host, const int32_t 
 int echo_group_advantage(const float *rewards, int32_t P, int32_t G, float eps,
                          float *out_adv, void *cuda_stream);
 
+/* Learner-side objective of Appendix F ("GRPO-Style Policy Gradient Objective"), forward value per
+ * sequence: with rho_t = exp(logp_new - logp_old), the truncated importance ratio
+ * w_t = min(exp(logp_old - logp_sampler), C) and the response mask m_t,
+ *   out[i] = sum_t m_t w_t min(rho_t A_i, clip(rho_t, 1 - eps_clip, 1 + eps_clip) A_i) / sum_t m_t
+ * (0 for an empty mask; the KL term, which needs a reference policy, is not included).
+ * logp_* dev fp32 [n][T] are log-probabilities of the taken tokens (logp_sampler is what
+ * echo_rollout recorded, the other two come from echo_rollout_forced under the respective
+ * weights), adv dev fp32 [n] (echo_group_advantage), mask dev uint8 [n][T] or NULL (all ones),
+ * out dev fp32 [n].  eps_clip >= 0, C > 0.  Asynchronous on the stream. */
+int echo_grpo_surrogate(const float *logp_new, const float *logp_old, const float *logp_sampler,
+                        const float *adv, const uint8_t *mask, int32_t n, int32_t T, float eps_clip,
+                        float C, float *out, void *cuda_stream);
+
 /* Block until everything this context enqueued (rollouts and installs) is done;
  * reports ECHO_ERR_DEVICE_CHECK / ECHO_ERR_TIMEOUT if a kernel flagged one. */
 int echo_sync(echo_ctx *ctx);

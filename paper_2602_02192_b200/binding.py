@@ -86,6 +86,8 @@ def _load() -> C.CDLL:
     lib.echo_sample.argtypes = [vp, i32, i32, i32, vp, u32, f32, u64, vp, vp, vp, vp]
     lib.echo_sample_top_p.argtypes = [vp, i32, i32, i32, vp, u32, f32, f32, u64, vp, vp, vp, vp, vp]
     lib.echo_sample_top_p.restype = C.c_int
+    lib.echo_grpo_surrogate.argtypes = [vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp]
+    lib.echo_grpo_surrogate.restype = C.c_int
     lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]
     lib.echo_decode_attention.argtypes = [vp, vp, i32, vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, vp]
     lib.echo_decode_attention.restype = C.c_int
@@ -118,7 +120,7 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
             "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_decode_attention",
             "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error",
-            "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p"]
+            "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -291,6 +293,23 @@ def echo_group_advantage(rewards: torch.Tensor, eps: float = 1e-6, out: Optional
         out = torch.empty_like(rewards)
     with torch.cuda.device(rewards.device):
         _check(lib.echo_group_advantage(rewards.data_ptr(), P, G, float(eps), out.data_ptr(), _stream_ptr(stream)))
+    return out
+
+
+def echo_grpo_surrogate(logp_new: torch.Tensor, logp_old: torch.Tensor, logp_sampler: torch.Tensor,
+                        adv: torch.Tensor, mask: Optional[torch.Tensor], eps_clip: float, C_trunc: float) -> torch.Tensor:
+    """Clipped surrogate with truncated importance sampling, one value per sequence ([n][T] inputs)."""
+    n, T = logp_new.shape
+    for x in (logp_new, logp_old, logp_sampler, adv):
+        assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    assert logp_old.shape == (n, T) and logp_sampler.shape == (n, T) and adv.shape == (n,)
+    if mask is not None:
+        assert mask.is_cuda and mask.dtype == torch.uint8 and mask.is_contiguous() and mask.shape == (n, T)
+    out = torch.empty(n, dtype=torch.float32, device=logp_new.device)
+    with torch.cuda.device(logp_new.device):
+        _check(lib.echo_grpo_surrogate(logp_new.data_ptr(), logp_old.data_ptr(), logp_sampler.data_ptr(),
+                                       adv.data_ptr(), mask.data_ptr() if mask is not None else None, n, T,
+                                       float(eps_clip), float(C_trunc), out.data_ptr(), _stream_ptr(None)))
     return out
 
 

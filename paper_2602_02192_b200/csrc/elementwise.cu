@@ -321,6 +321,33 @@ __global__ void decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int
 
 __global__ void set_int_kernel(int32_t *p, int32_t v) { *p = v; }
 
+// Clipped surrogate with truncated importance sampling, one warp per sequence (all in fp32):
+// J_i = sum_t m_t min(exp(lo - ls), C) min(rho A, clip(rho, 1 - e, 1 + e) A) / sum_t m_t, rho = exp(ln - lo).
+__global__ void grpo_surrogate_kernel(const float *__restrict__ ln, const float *__restrict__ lo,
+                                      const float *__restrict__ ls, const float *__restrict__ adv,
+                                      const uint8_t *__restrict__ mask, int n, int T, float eps_clip, float C,
+                                      float *__restrict__ out) {
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (i >= n) return;
+  const size_t base = static_cast<size_t>(i) * T;
+  const float a = adv[i];
+  float num = 0.f, den = 0.f;
+  for (int t = lane; t < T; t += 32) {
+    if (mask && !mask[base + t]) continue;
+    const float rho = expf(ln[base + t] - lo[base + t]);
+    const float w = fminf(expf(lo[base + t] - ls[base + t]), C);
+    const float clipped = fminf(fmaxf(rho, 1.0f - eps_clip), 1.0f + eps_clip);
+    num += w * fminf(rho * a, clipped * a);
+    den += 1.0f;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    num += __shfl_xor_sync(0xffffffffu, num, o);
+    den += __shfl_xor_sync(0xffffffffu, den, o);
+  }
+  if (lane == 0) out[i] = den > 0.f ? num / den : 0.f;
+}
+
 // ---------------------------------------------------------------------------
 // Sampler: one block per sequence row.  Single pass over the logits row keeps, per
 // thread, the running (max, sum of exp) of s = z / T and the best perturbed score
@@ -567,6 +594,13 @@ cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_
 cudaError_t advantage_launch(const float *r, int P, int G, float eps, float *out, cudaStream_t s) {
   if (P == 0) return cudaSuccess;
   advantage_kernel<<<(P + 7) / 8, 256, 0, s>>>(r, P, G, eps, out);
+  return cudaGetLastError();
+}
+cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float *ls, const float *adv,
+                                  const uint8_t *mask, int n, int T, float eps_clip, float C, float *out,
+                                  cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  grpo_surrogate_kernel<<<(n + 7) / 8, 256, 0, s>>>(ln, lo, ls, adv, mask, n, T, eps_clip, C, out);
   return cudaGetLastError();
 }
 cudaError_t set_int_launch(int32_t *p, int32_t v, cudaStream_t s) {

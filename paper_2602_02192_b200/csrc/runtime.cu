@@ -978,6 +978,16 @@ int echo_group_advantage(const float *rewards, int32_t P, int32_t G, float eps, 
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }
 
+int echo_grpo_surrogate(const float *logp_new, const float *logp_old, const float *logp_sampler, const float *adv,
+                        const uint8_t *mask, int32_t n, int32_t T, float eps_clip, float C, float *out,
+                        void *cuda_stream) {
+  if (!logp_new || !logp_old || !logp_sampler || !adv || !out || n < 0 || T < 1) return ECHO_ERR_INVALID;
+  if (!(eps_clip >= 0.f) || !(C > 0.f)) return ECHO_ERR_INVALID;
+  cudaError_t e = grpo_surrogate_launch(logp_new, logp_old, logp_sampler, adv, mask, n, T, eps_clip, C, out,
+                                        static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
 int echo_sync(echo_ctx *ctx) {
   if (!ctx) return ECHO_ERR_INVALID;
   DeviceGuard guard(ctx->device);

@@ -241,3 +241,18 @@ def test_group_advantage_matches_oracle(B):
     assert np.all(B.echo_group_advantage(torch.from_numpy(r).cuda()).cpu().numpy() == 0)
     with pytest.raises(B.EchoError):
         B.echo_group_advantage(torch.zeros((4, 1), device="cuda"))
+
+
+def test_grpo_surrogate_matches_oracle(B):
+    from oracle import objective
+    rng = np.random.default_rng(17)
+    for n, T, with_mask in [(1, 1, False), (5, 33, True), (64, 2048, True), (256, 100, False)]:
+        ln, lo, ls = (-rng.exponential(1.0, size=(n, T)).astype(np.float32) for _ in range(3))
+        adv = rng.normal(size=n).astype(np.float32)
+        mask = (rng.random((n, T)) < 0.6).astype(np.uint8) if with_mask else None
+        if with_mask and n > 2:
+            mask[2] = 0
+        got = B.echo_grpo_surrogate(*(torch.from_numpy(x).cuda() for x in (ln, lo, ls, adv)),
+                                    torch.from_numpy(mask).cuda() if with_mask else None, 0.2, 1.7).cpu().numpy()
+        want = objective.grpo_surrogate(ln, lo, ls, adv, mask if with_mask else np.ones((n, T)), 0.2, 1.7)
+        assert np.allclose(got, want, rtol=2e-5, atol=2e-5)

@@ -141,3 +141,51 @@ def test_version_single_buffer_blocks():
     assert w.begin_rollout() == 0
     w.offer(1)
     assert w.begin_rollout() == 1           # single buffer: old weights are gone
+
+
+# ---- GRPO surrogate with truncated importance sampling (Appendix F) ----------------------------
+
+def test_grpo_surrogate_closed_forms():
+    from oracle import objective
+    T = 5
+    lp = np.log(np.array([[0.2, 0.5, 0.1, 0.7, 0.3]]))
+    ones = np.ones((1, T))
+    # same policy everywhere: rho = w = 1, J = A
+    for A in (1.5, -0.7, 0.0):
+        assert np.allclose(objective.grpo_surrogate(lp, lp, lp, [A], ones, 0.2, 2.0), [A], atol=1e-15)
+    # the four clipping cases, one token: rho = 1.5 / 0.5 against eps = 0.2
+    up, down = lp + np.log(1.5), lp + np.log(0.5)
+    one = np.zeros((1, T)); one[0, 2] = 1
+    J = lambda new, A: float(objective.grpo_surrogate(new, lp, lp, [A], one, 0.2, 2.0)[0])
+    assert np.isclose(J(up, 2.0), 1.2 * 2.0)        # A > 0, rho above the clip: capped
+    assert np.isclose(J(down, 2.0), 0.5 * 2.0)      # A > 0, rho below: the unclipped (smaller) branch
+    assert np.isclose(J(up, -2.0), 1.5 * -2.0)      # A < 0, rho above: the unclipped (more negative) branch
+    assert np.isclose(J(down, -2.0), 0.8 * -2.0)    # A < 0, rho below the clip: capped
+    # truncated importance ratio: learner / sampler = 3 capped at C = 2; 0.5 passes through
+    samp_lo, samp_hi = lp - np.log(3.0), lp + np.log(2.0)
+    assert np.allclose(objective.grpo_surrogate(lp, lp, samp_lo, [1.0], ones, 0.2, 2.0), [2.0])
+    assert np.allclose(objective.grpo_surrogate(lp, lp, samp_hi, [1.0], ones, 0.2, 2.0), [0.5])
+    # the mask selects and normalises: two of five tokens with weights 2 and 0.5 -> mean 1.25
+    mixed = lp.copy(); mixed[0, 0] -= np.log(3.0); mixed[0, 1] += np.log(2.0)
+    mk = np.array([[1, 1, 0, 0, 0]])
+    assert np.allclose(objective.grpo_surrogate(lp, lp, mixed, [1.0], mk, 0.2, 2.0), [1.25])
+    assert np.allclose(objective.grpo_surrogate(lp, lp, mixed, [1.0], np.zeros((1, T)), 0.2, 2.0), [0.0])
+    with pytest.raises(ValueError):
+        objective.grpo_surrogate(lp, lp, lp, [1.0, 2.0], ones, 0.2, 2.0)
+
+
+def test_grpo_surrogate_against_vector_formula():
+    from oracle import objective
+    rng = np.random.default_rng(3)
+    n, T = 7, 33
+    ln, lo, ls = (-rng.exponential(1.0, size=(n, T)) for _ in range(3))
+    adv = rng.normal(size=n)
+    mask = (rng.random((n, T)) < 0.6).astype(np.float64)
+    mask[3] = 0
+    got = objective.grpo_surrogate(ln, lo, ls, adv, mask, 0.2, 1.7)
+    rho = np.exp(ln - lo)
+    w = np.minimum(np.exp(lo - ls), 1.7)
+    term = np.minimum(rho * adv[:, None], np.clip(rho, 0.8, 1.2) * adv[:, None])
+    den = mask.sum(1)
+    want = np.where(den > 0, (mask * w * term).sum(1) / np.maximum(den, 1), 0.0)
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-15)
