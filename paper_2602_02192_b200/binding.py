@@ -14,7 +14,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libecho_b200.so")
+LIB_PATH = os.environ.get("ECHO_B200_LIB") or os.path.join(_HERE, "libecho_b200.so")   # override: another build of the library
 
 ECHO_OK = 0
 ERRORS = {

@@ -67,11 +67,21 @@ __global__ void __launch_bounds__(kNormThreads)
 rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ gain, __nv_bfloat16 *__restrict__ h,
                int R, int d, float eps) {
   __shared__ float scratch[32];
-  early_start_sync();       // (also lets the following projection begin its weight prefetch)
   const int r = blockIdx.x;
   const float *xr = x + static_cast<size_t>(r) * d;
   __nv_bfloat16 *hr = h + static_cast<size_t>(r) * d;
   const bool fast = (d % 4 == 0) && d <= 4 * kNormVecs * kNormThreads;
+  // the gains are part of the installed snapshot, not of the preceding kernel's output: they are
+  // fetched before the dependency wait
+  uint2 graw[kNormVecs];
+  if (fast) {
+#pragma unroll
+    for (int i = 0; i < kNormVecs; ++i) {
+      const int idx = threadIdx.x + i * kNormThreads;
+      graw[i] = idx < d / 4 ? reinterpret_cast<const uint2 *>(gain)[idx] : make_uint2(0u, 0u);
+    }
+  }
+  early_start_sync();       // (also lets the following projection begin its weight prefetch)
   if (fast) {
     const int nv = d / 4;
     float4 v[kNormVecs];
@@ -88,9 +98,8 @@ rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ ga
     for (int i = 0; i < kNormVecs; ++i) {
       const int idx = threadIdx.x + i * kNormThreads;
       if (idx < nv) {
-        const uint2 graw = reinterpret_cast<const uint2 *>(gain)[idx];
-        const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw.x));
-        const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw.y));
+        const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw[i].x));
+        const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw[i].y));
         __nv_bfloat162 o0 = __floats2bfloat162_rn(v[i].x * scale * g0.x, v[i].y * scale * g0.y);
         __nv_bfloat162 o1 = __floats2bfloat162_rn(v[i].z * scale * g1.x, v[i].w * scale * g1.y);
         uint2 o;
