@@ -225,6 +225,26 @@ int echo_debug_page_table(echo_ctx *ctx, int32_t *out, size_t n, int32_t *rows, 
 int echo_plan_page_table(const int32_t *prompt_lens, int32_t P, int32_t G, int32_t T, int32_t page_size,
                          int32_t *out_table, size_t capacity, int32_t *width, int32_t *n_pages);
 
+/* ---- host-side closed forms of the control plane (no GPU work) -------------
+ * Section 3.1, capacity requirement: the aggregate rollout throughput (rollouts/s) that keeps the
+ * learner busy when it consumes R trajectories per step of T_train seconds and publishes every
+ * kappa steps, with T_bcast seconds from publication to a usable snapshot:
+ *   mu_min = kappa R / (kappa T_train - T_bcast).   ECHO_ERR_UNSUPPORTED if kappa T_train <= T_bcast. */
+int echo_mu_min(double kappa, double R, double T_train, double T_bcast, double *out);
+/* Section 3.1 ("Linking (S, kappa)") / Appendix on staleness: conservative bound
+ *   Delta_max <= kappa + ceil((T_bcast + R / mu_pool) / T_train) - 1. */
+int echo_staleness_bound(int32_t kappa, double T_bcast, double R, double mu_pool, double T_train,
+                         int32_t *out);
+/* Section 3.2, greedy provisioning: rank workers by unit throughput cost rho_i = cost_i / mu_i
+ * (equal rho: lower index first) and activate the cheapest prefix whose cumulative throughput
+ * reaches mu_target.  active[n] (host) receives 0/1; n_active and total_cost may be NULL.
+ * ECHO_ERR_UNSUPPORTED (with every worker active) if the whole pool stays below the target. */
+int echo_greedy_provision(const double *mu, const double *cost, int32_t n, double mu_target,
+                          uint8_t *active, int32_t *n_active, double *total_cost);
+/* Section 4.2, replay buffer: a trajectory tagged v is admissible at learner version v_t under
+ * the staleness budget S iff v_t - S <= v <= v_t.  Returns 1 or 0. */
+int echo_admissible(int64_t v, int64_t v_t, int64_t S);
+
 /* ---- stand-alone kernel entry points (used by the parity tests) ---------- */
 
 /* Philox words and uniforms exactly as the sampler draws them: for vocab ids

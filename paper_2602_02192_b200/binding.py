@@ -88,6 +88,14 @@ def _load() -> C.CDLL:
     lib.echo_sample_top_p.restype = C.c_int
     lib.echo_grpo_surrogate.argtypes = [vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp]
     lib.echo_grpo_surrogate.restype = C.c_int
+    dbl = C.c_double
+    lib.echo_mu_min.argtypes = [dbl, dbl, dbl, dbl, C.POINTER(dbl)]
+    lib.echo_staleness_bound.argtypes = [i32, dbl, dbl, dbl, dbl, C.POINTER(i32)]
+    lib.echo_greedy_provision.argtypes = [C.POINTER(dbl), C.POINTER(dbl), i32, dbl, C.POINTER(C.c_uint8),
+                                          C.POINTER(i32), C.POINTER(dbl)]
+    lib.echo_admissible.argtypes = [i64, i64, i64]
+    for name in ("echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible"):
+        getattr(lib, name).restype = C.c_int
     lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]
     lib.echo_decode_attention.argtypes = [vp, vp, i32, vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, vp]
     lib.echo_decode_attention.restype = C.c_int
@@ -120,7 +128,8 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
             "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_decode_attention",
             "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error",
-            "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate"]
+            "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate",
+            "echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:

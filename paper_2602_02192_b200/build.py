@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libecho_b200.so")
-SOURCES = ["gemm.cu", "gemm_pair.cu", "elementwise.cu", "nucleus.cu", "attention.cu", "runtime.cu"]
+SOURCES = ["gemm.cu", "gemm_pair.cu", "elementwise.cu", "nucleus.cu", "attention.cu", "runtime.cu", "control.cu"]
 HEADERS = ["common.cuh", "ptx.cuh", os.path.join("..", "..", "include", "echo.h")]
 
 
