@@ -244,8 +244,19 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
   const int REP = Hq / Hkv;
   const int quad = lane >> 2, qi = lane & 3;
 
-  // row positions are written earlier in the same step: read nothing before the predecessor is complete
-  early_start_sync();        // (the output projection may start prefetching its weights)
+  // Ordering under programmatic dependent launch.  The prefix launch waits for its predecessor
+  // (the kernel that wrote q and the new K/V rows) and only THEN lets the suffix launch be
+  // scheduled: a suffix CTA therefore finds q, the KV pool and the row positions complete without
+  // waiting itself, and streams its pages while prefix CTAs are still running.  It waits for the
+  // prefix launch only just before it merges with the prefix partials, at the end.
+  // A suffix CTA that runs before its own wait must not trust this SM's L1: q, the row positions
+  // and the page table are read with L2-only loads (the pages themselves come through TMA).
+  if (PREFIX) {
+    griddep_wait();
+    griddep_launch();
+  } else {
+    griddep_launch();        // (the output projection may start prefetching its weights)
+  }
 
   // ---- which query rows and which keys this CTA handles ------------------------------------
   int h, seq0, first_page, n_keys, mt = 0;
@@ -256,12 +267,12 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
     h = ph % Hkv;
     seq0 = (ph / Hkv) * G;                   // first sequence of the group
     first_page = 0;
-    n_keys = full_pages[seq0] * kPageTokens;
+    n_keys = __ldcg(&full_pages[seq0]) * kPageTokens;
   } else {
     h = blockIdx.x % Hkv;
     seq0 = blockIdx.x / Hkv;
-    first_page = full_pages[seq0];
-    n_keys = row_pos[seq0] + 1 - first_page * kPageTokens;
+    first_page = __ldcg(&full_pages[seq0]);
+    n_keys = __ldcg(&row_pos[seq0]) + 1 - first_page * kPageTokens;
   }
   const int n_tiles = (n_keys + kPageTokens - 1) / kPageTokens;
   const int32_t *pt = page_table + static_cast<size_t>(seq0) * pt_width + first_page;
@@ -297,7 +308,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
     if (k < pg_base || k >= pg_base + 32 || pg_base < 0) {
       pg_base = k;
       const int kk = k + lane;
-      pg_cache = kk < n_my ? pt[warp + kDecWarps * kk] : 0;
+      pg_cache = kk < n_my ? __ldcg(&pt[warp + kDecWarps * kk]) : 0;
     }
     return __shfl_sync(0xffffffffu, pg_cache, k - pg_base);
   };
@@ -322,26 +333,6 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
   for (int k = 0; k < n_pro; ++k) issue(k);
 
   // (the first pages are on their way; everything below overlaps their latency)
-  // prefix partials this thread will merge at the end (suffix kernel): fetched now, used last
-  constexpr int kPre = 4;
-  float pre_val[kPre];
-  float2 pre_stat[kPre];
-  const bool pre_ok = !PREFIX && REP * HD <= kPre * kDecWarps * 32;
-  if (pre_ok) {
-#pragma unroll
-    for (int i = 0; i < kPre; ++i) {
-      const int idx = threadIdx.x + i * kDecWarps * 32;
-      pre_val[i] = 0.f;
-      pre_stat[i] = make_float2(-INFINITY, 0.f);
-      if (idx < REP * HD) {
-        const int r = idx / HD, d = idx % HD;
-        const size_t rh = static_cast<size_t>(seq0) * Hq + h * REP + r;
-        pre_stat[i] = pre_ml[rh];
-        pre_val[i] = pre_o[rh * HD + d];
-      }
-    }
-  }
-
   // ---- Q fragments (A operand), kept in registers for the whole loop ---------------------------
   uint32_t qf[KSTEPS][4];
   {
@@ -354,10 +345,10 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
                                      : nullptr;
 #pragma unroll
     for (int kk = 0; kk < KSTEPS; ++kk) {
-      qf[kk][0] = q_lo ? q_lo[kk * 8 + qi] : 0u;
-      qf[kk][1] = q_hi ? q_hi[kk * 8 + qi] : 0u;
-      qf[kk][2] = q_lo ? q_lo[kk * 8 + 4 + qi] : 0u;
-      qf[kk][3] = q_hi ? q_hi[kk * 8 + 4 + qi] : 0u;
+      qf[kk][0] = q_lo ? __ldcg(&q_lo[kk * 8 + qi]) : 0u;
+      qf[kk][1] = q_hi ? __ldcg(&q_hi[kk * 8 + qi]) : 0u;
+      qf[kk][2] = q_lo ? __ldcg(&q_lo[kk * 8 + 4 + qi]) : 0u;
+      qf[kk][3] = q_hi ? __ldcg(&q_hi[kk * 8 + 4 + qi]) : 0u;
     }
   }
 
@@ -459,6 +450,27 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
     l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
   }
 
+  // ---- prefix partials (suffix kernel): the prefix launch must be complete from here on --------
+  constexpr int kPre = 4;
+  float pre_val[kPre];
+  float2 pre_stat[kPre];
+  const bool pre_ok = !PREFIX && REP * HD <= kPre * kDecWarps * 32;
+  if (!PREFIX) griddep_wait();
+  if (pre_ok) {
+#pragma unroll
+    for (int i = 0; i < kPre; ++i) {
+      const int idx = threadIdx.x + i * kDecWarps * 32;
+      pre_val[i] = 0.f;
+      pre_stat[i] = make_float2(-INFINITY, 0.f);
+      if (idx < REP * HD) {
+        const int r = idx / HD, d = idx % HD;
+        const size_t rh = static_cast<size_t>(seq0) * Hq + h * REP + r;
+        pre_stat[i] = __ldcg(&pre_ml[rh]);
+        pre_val[i] = __ldcg(&pre_o[rh * HD + d]);
+      }
+    }
+  }
+
   // ---- combine the four warps through shared memory (the pipeline buffers are free now) -------
   __syncthreads();
   float *m_s = reinterpret_cast<float *>(smem);                      // [warp][16]
@@ -514,8 +526,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
             po = pre_val[i];
           }
       } else {
-        ml = pre_ml[static_cast<size_t>(s) * Hq + row_head(r)];
-        po = pre_o[oi];
+        ml = __ldcg(&pre_ml[static_cast<size_t>(s) * Hq + row_head(r)]);
+        po = __ldcg(&pre_o[oi]);
       }
       float Mt = fmaxf(M, ml.x);
       if (Mt == -INFINITY) Mt = 0.f;
