@@ -26,7 +26,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-ATTN_DRAM_PER_ALG_BYTE = 170.3 / 166.2      # measured DRAM bytes per algorithmic byte (see profiles/)
+ATTN_DRAM_PER_ALG_BYTE = 170.4 / 166.2      # measured DRAM bytes per algorithmic byte (see profiles/)
 METRIC = "rollout generated tokens/s"
 UNIT = "tokens/s"
 
@@ -268,7 +268,7 @@ def run_ours(args):
         achieved = alg / dur_s / 1e9
         tot = float(prof_ms[:, 3].sum())
         # DRAM bytes per launch: ncu counters of the current kernel on a small case of the same
-        # per-CTA work (profiles/attn_decode_kernel_P4_G8_Lp512_i1200.md: 170.3 MB read + written
+        # per-CTA work (profiles/attn_decode_kernel_P4_G8_Lp512_i1200.md: 170.4 MB read + written
         # for 166.2 MB of algorithmic bytes, prefix + suffix launch), scaled to this workload's
         # launches by their algorithmic bytes: the traffic is the KV stream and grows with it.
         traffic = ATTN_DRAM_PER_ALG_BYTE * alg / attn_launches if wl.shape.head_dim == 128 else None
