@@ -436,6 +436,51 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_variable_length(args):
+    """Diagnostic (--variable-length): responses of uniformly random length in [1, T] (the paper's
+    responses average about half the maximum length), produced by teacher-forcing given tokens that
+    hold the end token at each sequence's length.  Compares one rollout with the end-of-sequence rule
+    (ended sequences are no longer attended) with the same rollout without it.  One JSON line."""
+    from paper_2602_02192_b200 import binding, synth
+    wl = synth.WORKLOADS[args.workload]
+    shape, P, G, Lp = wl.shape, wl.n_prompts, wl.G, wl.prompt_len
+    T = args.new_tokens or wl.new_tokens
+    weights = synth.make_weights(shape, wl.weight_seed, device="cuda")
+    prompts = torch.from_numpy(synth.make_prompts(P, Lp, shape.vocab, wl.prompt_seed)).cuda()
+    rng = np.random.default_rng(7)
+    eos = shape.vocab - 1
+    given = rng.integers(0, eos, size=(P, G, T)).astype(np.int32)
+    lengths = rng.integers(1, T + 1, size=(P, G))
+    for p in range(P):
+        for g in range(G):
+            given[p, g, lengths[p, g] - 1:] = eos
+    forced = torch.from_numpy(given).cuda()
+    out = {}
+    for name, eos_id in (("with_rule", eos), ("without_rule", -1)):
+        eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, 1, eos_id=eos_id))
+        eng.echo_load_policy(weights, 1)
+        eng.echo_wait_policy()
+        times = []
+        for it in range(2):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(eng.stream)
+            eng.echo_rollout(prompts, [Lp] * P, G, T, wl.temperature, wl.sample_seed, forced=forced)
+            e1.record(eng.stream)
+            eng.echo_sync()
+            times.append(e0.elapsed_time(e1))
+        st = eng.echo_get_stats()
+        out[name] = {"ms": round(times[-1], 1), "decode_ms_per_step": round(st["decode_ms"] / max(1, T - 1), 3)}
+        eng.close()
+        del eng
+        torch.cuda.empty_cache()
+    useful = int(lengths.sum())
+    print(json.dumps({"diagnostic": "variable-length responses, teacher-forced", "workload": wl.name, "max_new_tokens": T,
+                      "mean_length": round(float(lengths.mean()), 1), "useful_tokens": useful,
+                      "with_rule": out["with_rule"], "without_rule": out["without_rule"],
+                      "useful_tokens_per_s_with_rule": round(useful / out["with_rule"]["ms"] * 1e3, 1),
+                      "useful_tokens_per_s_without_rule": round(useful / out["without_rule"]["ms"] * 1e3, 1)}))
+
+
 def run_projections(args):
     """Diagnostic (--projections): every projection shape of one decode step of the workload, alone,
     with rotating weight sets larger than L2, through echo_gemm_bf16 (SM-pair kernel, block-tiled
@@ -507,10 +552,14 @@ def main():
     ap.add_argument("--top-p", type=float, default=1.0,
                     help="nucleus sampling (the paper samples with 0.95); 1.0 = the benchmark's untruncated sampling")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--variable-length", action="store_true",
+                    help="diagnostic: random response lengths with and without the end-of-sequence rule, and exit")
     ap.add_argument("--projections", action="store_true",
                     help="diagnostic: time each projection shape alone (with cuBLAS beside it) and exit")
     args = ap.parse_args()
-    if args.projections:
+    if args.variable_length:
+        run_variable_length(args)
+    elif args.projections:
         run_projections(args)
     elif args.impl == "reference":
         run_reference(args)

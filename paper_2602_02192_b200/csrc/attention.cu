@@ -231,7 +231,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
                    __nv_bfloat16 *__restrict__ out, float *__restrict__ pre_o, float2 *__restrict__ pre_ml,
                    const int32_t *__restrict__ page_table, int pt_width, const int32_t *__restrict__ row_pos,
                    const int32_t *__restrict__ full_pages, int layer_row0, int Hq, int Hkv, int G, int n_pages,
-                   float scale_log2, int *status) {
+                   float scale_log2, const int32_t *__restrict__ row_done, int *status) {
   using S = DecSmem<HD>;
   constexpr int KSTEPS = HD / 16;           // MMA k-steps over the head dimension
   constexpr int HALVES = HD / 64;           // 64-element (128-byte) column blocks per row
@@ -256,6 +256,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
     griddep_launch();
   } else {
     griddep_launch();        // (the output projection may start prefetching its weights)
+    // a sequence that has ended (its end token was fed) is not attended: its row is not used
+    if (row_done && __ldcg(&row_done[blockIdx.x / Hkv])) return;
   }
 
   // ---- which query rows and which keys this CTA handles ------------------------------------
@@ -549,11 +551,11 @@ cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
   const float scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(HD));
   cudaError_t e = launch_early(attn_decode_kernel<HD, true>, dim3(a.P * a.Hkv * MT), dim3(kDecWarps * 32), S::kTotal, s,
                                *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos,
-                               a.full_pages, a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.status);
+                               a.full_pages, a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
   if (e != cudaSuccess) return e;
   return launch_early(attn_decode_kernel<HD, false>, dim3(a.P * a.G * a.Hkv), dim3(kDecWarps * 32), S::kTotal, s,
                       *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages,
-                      a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.status);
+                      a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
 }
 
 }  // namespace

@@ -145,6 +145,8 @@ cudaError_t gemm_pair_launch(const PairGemmArgs &a, cudaStream_t stream);
 struct RowMeta {
   const int32_t *row_pt;     // page-table row of each activation row
   const int32_t *row_pos;    // absolute position of each activation row
+  const int32_t *row_done;   // optional: non-zero = the row's sequence has ended (end token fed): nothing is
+                             // appended or attended for it, its outputs are not used
 };
 
 cudaError_t embed_launch(const __nv_bfloat16 *embed, const int32_t *tok_src, const int32_t *tok_idx,
@@ -166,7 +168,8 @@ cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page
                                       int page_elems, cudaStream_t s);
 // decode-step preparation: advances the step counter, sets the rows' token and position
 cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
-                               int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s);
+                               int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s, int eos_id = -1,
+                               int32_t *row_done = nullptr);
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row,
                            const int32_t *seq_ids, const int32_t *d_step, uint32_t j_host,
                            float temperature, uint64_t seed, const int32_t *forced, int forced_stride,
@@ -207,6 +210,7 @@ struct DecodeAttnArgs {
   int layer_row0;                 // first row of this layer in the pool's row space
   int P, G, Hq, Hkv, hd, n_pages;
   int *status;
+  const int32_t *row_done;        // optional, per sequence: non-zero = ended, its suffix CTAs return at once
 };
 cudaError_t attention_decode_configure();
 bool attention_decode_supported(int hd, int page_size, int Hq, int Hkv);

@@ -135,16 +135,17 @@ __global__ void rope_table_kernel(float2 *table, int max_pos, int half, double t
 __global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q,
                                    __nv_bfloat16 *__restrict__ kv_layer, const float2 *__restrict__ rope_table,
                                    const int32_t *__restrict__ row_pt, const int32_t *__restrict__ row_pos,
-                                   const int32_t *__restrict__ page_table, int pt_width, int R, int Hq, int Hkv, int hd,
-                                   int page_size, int n_pages, int max_pos, int *status) {
+                                   const int32_t *__restrict__ row_done, const int32_t *__restrict__ page_table,
+                                   int pt_width, int R, int Hq, int Hkv, int hd, int page_size, int n_pages,
+                                   int max_pos, int *status) {
   early_start_sync();
   const int r = blockIdx.x;
-  const int pos = row_pos[r];
+  const int pos = (row_done && row_done[r]) ? -1 : row_pos[r];      // an ended row is only cleared
   const int half = hd / 2;
   const int ld = (Hq + 2 * Hkv) * hd;
   float *src = qkv + static_cast<size_t>(r) * ld;
   if (pos < 0 || pos >= max_pos) {
-    if (threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
+    if (threadIdx.x == 0 && !(row_done && row_done[r])) atomicExch(status, STATUS_BAD_PAGE);
     for (int i = threadIdx.x; i < ld; i += blockDim.x) src[i] = 0.f;      // keep the buffer's zero invariant
     return;
   }
@@ -207,7 +208,8 @@ __device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d)
 __global__ void __launch_bounds__(256)
 rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ kv_layer,
                        const float2 *__restrict__ rope_table, const int32_t *__restrict__ row_pt,
-                       const int32_t *__restrict__ row_pos, const int32_t *__restrict__ page_table, int pt_width,
+                       const int32_t *__restrict__ row_pos, const int32_t *__restrict__ row_done,
+                       const int32_t *__restrict__ page_table, int pt_width,
                        int R, int Hq, int Hkv, int hd, int page_size, int n_pages, int max_pos, int *status) {
   early_start_sync();
   const int r = blockIdx.x;
@@ -233,11 +235,12 @@ rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, _
       }
     }
   }
-  const int pos = row_pos[r];
+  const bool ended = row_done && row_done[r];            // an ended row is only cleared
+  const int pos = ended ? -1 : row_pos[r];
   int page = -1;
   if (pos >= 0 && pos < max_pos) page = page_table[static_cast<size_t>(row_pt[r]) * pt_width + pos / page_size];
   const bool bad = page < 0 || page >= n_pages;
-  if (bad && threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
+  if (bad && !ended && threadIdx.x == 0) atomicExch(status, STATUS_BAD_PAGE);
   const int off = bad ? 0 : pos % page_size;
   const float4 *cs4 = reinterpret_cast<const float4 *>(rope_table + static_cast<size_t>(bad ? 0 : pos) * half);
   const size_t page_elems = static_cast<size_t>(page_size) * hd;
@@ -317,13 +320,17 @@ __global__ void copy_pages_kernel(__nv_bfloat16 *kv, const int32_t *src_page, co
 // Start of decode step j = *d_step + 1: row b feeds the token produced at step j-1 at
 // position len0[b] + j - 1.  One block; the counter is bumped after every thread has read it.
 __global__ void decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
-                                   int32_t *row_tok, int32_t *row_pos, int B) {
+                                   int32_t *row_tok, int32_t *row_pos, int B, int eos_id, int32_t *row_done) {
   early_start_sync();
   const int j = *d_step + 1;
   __syncthreads();
   for (int b = threadIdx.x; b < B; b += blockDim.x) {
-    row_tok[b] = tok_hist[static_cast<size_t>(b) * T + (j - 1)];
+    const int32_t tok = tok_hist[static_cast<size_t>(b) * T + (j - 1)];
+    row_tok[b] = tok;
     row_pos[b] = seq_len0[b] + j - 1;
+    // a sequence that is fed its end token has ended: every later token is the end token too, so
+    // the row stays marked; its attention and cache writes are skipped from here on
+    if (row_done) row_done[b] = (eos_id >= 0 && tok == eos_id) ? 1 : 0;
   }
   if (threadIdx.x == 0) *d_step = j;
 }
@@ -559,9 +566,9 @@ cudaError_t rope_append_launch(float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_l
                                int page_size, int n_pages, int max_pos, int *status, cudaStream_t s) {
   if (hd % 8 == 0 && (reinterpret_cast<uintptr_t>(qkv) & 15) == 0)
     return launch_early(rope_append_vec_kernel, dim3(R), dim3(256), 0, s, qkv, q, kv_layer, rope_table, meta.row_pt,
-                        meta.row_pos, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
+                        meta.row_pos, meta.row_done, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
   return launch_early(rope_append_kernel, dim3(R), dim3(256), 0, s, qkv, q, kv_layer, rope_table, meta.row_pt,
-                      meta.row_pos, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
+                      meta.row_pos, meta.row_done, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
 }
 cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s) {
   const size_t n = static_cast<size_t>(R) * F;
@@ -580,8 +587,10 @@ cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page
   return cudaGetLastError();
 }
 cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
-                               int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s) {
-  return launch_early(decode_prep_kernel, dim3(1), dim3(512), 0, s, d_step, tok_hist, T, seq_len0, row_tok, row_pos, B);
+                               int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s, int eos_id,
+                               int32_t *row_done) {
+  return launch_early(decode_prep_kernel, dim3(1), dim3(512), 0, s, d_step, tok_hist, T, seq_len0, row_tok, row_pos, B,
+                      eos_id, row_done);
 }
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row, const int32_t *seq_ids,
                            const int32_t *d_step, uint32_t j_host, float temperature, uint64_t seed,

@@ -85,7 +85,7 @@ Limits limits_of(const echo_config &c) {
 struct Layout {
   size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
   size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
-      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
+      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, row_done, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
   size_t weight_bytes, kv_layer_elems, n_tables_ints;
   int n_chunks_max;
 };
@@ -127,6 +127,7 @@ Layout layout_of(const echo_config &c) {
   lo.pre_ml = take(static_cast<size_t>(M.B) * D.Hq * 8);
   lo.retile_stage = take(kRetileStageBytes);       // bounce buffer for snapshots in pageable host memory
   lo.nucleus_cut = take(static_cast<size_t>(M.B) * 8);   // top-p: one (score key, id) cut per logits row
+  lo.row_done = take(static_cast<size_t>(M.B) * 4);      // end-of-sequence rule: rows whose sequence has ended
   lo.copy_src = take(static_cast<size_t>(M.B) * 4);
   lo.copy_dst = take(static_cast<size_t>(M.B) * 4);
   lo.d_step = take(4);
@@ -340,7 +341,7 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int d
       DecodeAttnArgs da{&ctx->tm_kv, q, attn, ctx->ptr<float>(lo.pre_o), ctx->ptr<float2>(lo.pre_ml), pt,
                         ctx->M.pt_width, meta.row_pos, ctx->ptr<int32_t>(lo.full_pages),
                         static_cast<int>(static_cast<size_t>(l) * (lo.kv_layer_elems / D.hd)), decode_P, decode_G,
-                        D.Hq, D.Hkv, D.hd, ctx->M.n_pages, status};
+                        D.Hq, D.Hkv, D.hd, ctx->M.n_pages, status, meta.row_done};
       LAUNCH(attention_decode_launch(da, ctx->stream));
       ctx->launches++;                      // two kernels per call
     } else {
@@ -563,11 +564,12 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
   int32_t *row_tok = ctx->ptr<int32_t>(lo.dec_row_tok);
   int32_t *row_pos = ctx->ptr<int32_t>(lo.dec_row_pos);
   ProfScope prof_step(ctx, PROF_STEP);
+  int32_t *row_done = ctx->cfg.eos_id >= 0 ? ctx->ptr<int32_t>(lo.row_done) : nullptr;
   LAUNCH(decode_prep_launch(d_step, tok_hist, pl.T, ctx->ptr<int32_t>(lo.seq_len0), row_tok, row_pos, pl.B,
-                            ctx->stream));
+                            ctx->stream, ctx->cfg.eos_id, row_done));
   LAUNCH(embed_launch(w.embed, row_tok, nullptr, ctx->ptr<float>(lo.x), pl.B, ctx->D.d, ctx->D.V,
                       ctx->ptr<int>(lo.status), ctx->stream));
-  RowMeta meta{ctx->ptr<int32_t>(lo.dec_row_pt), row_pos};
+  RowMeta meta{ctx->ptr<int32_t>(lo.dec_row_pt), row_pos, row_done};
   TRY(forward_layers(ctx, w, pl.B, meta, pl.P, pl.G));
   TRY(lm_head(ctx, w, ctx->ptr<float>(lo.x), pl.B));
   {
@@ -621,7 +623,7 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
     const int r0 = c * kChunkRows, R = std::min(kChunkRows, pl.n_tok - r0);
     LAUNCH(embed_launch(w.embed, prompts, ctx->ptr<int32_t>(lo.pre_tok_idx) + r0, x, R, D.d, D.V, status,
                         ctx->stream));
-    RowMeta meta{ctx->ptr<int32_t>(lo.pre_row_pt) + r0, ctx->ptr<int32_t>(lo.pre_row_pos) + r0};
+    RowMeta meta{ctx->ptr<int32_t>(lo.pre_row_pt) + r0, ctx->ptr<int32_t>(lo.pre_row_pos) + r0, nullptr};
     TRY(forward_layers(ctx, w, R, meta));
     LAUNCH(gather_rows_launch(x, ctx->ptr<int32_t>(lo.gather_map) + static_cast<size_t>(c) * P,
                               ctx->ptr<float>(lo.xlast), P, D.d, ctx->stream));
@@ -1124,7 +1126,7 @@ int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, c
   int *status = reinterpret_cast<int *>(reinterpret_cast<uint8_t *>(pre_ml) + align_up(static_cast<size_t>(B) * Hq * 8));
   if (cudaMemsetAsync(status, 0, 4, s) != cudaSuccess) return ECHO_ERR_CUDA;
   DecodeAttnArgs da{&tm, static_cast<const __nv_bfloat16 *>(q), static_cast<__nv_bfloat16 *>(out), pre_o, pre_ml,
-                    page_table, pt_width, row_pos, full_pages, 0, P, G, Hq, Hkv, hd, n_pages, status};
+                    page_table, pt_width, row_pos, full_pages, 0, P, G, Hq, Hkv, hd, n_pages, status, nullptr};
   if (attention_decode_launch(da, s) != cudaSuccess) return ECHO_ERR_CUDA;
   int st = 0;
   if (cudaMemcpyAsync(&st, status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ECHO_ERR_CUDA;
