@@ -453,7 +453,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
   }
 
   // ---- prefix partials (suffix kernel): the prefix launch must be complete from here on --------
-  constexpr int kPre = 4;
+  constexpr int kPre = 8;
   float pre_val[kPre];
   float2 pre_stat[kPre];
   const bool pre_ok = !PREFIX && REP * HD <= kPre * kDecWarps * 32;
