@@ -192,9 +192,12 @@ cudaError_t attention_rows_launch(const __nv_bfloat16 *q, const __nv_bfloat16 *k
 //   prefix kernel   one CTA per (prompt, kv head, 16-row tile of the group's query rows); keys =
 //                   the prompt's full pages; writes un-normalised partial outputs with their
 //                   running max and sum to scratch.
-//   suffix kernel   one CTA per (sequence, kv head); keys = the sequence's private pages (copy of
+//   suffix kernel   per (sequence, kv head) item: keys = the sequence's private pages (copy of
 //                   the prompt's partial last page + generated tokens); merges with the prefix
-//                   partial and writes the final bf16 output.
+//                   partial and writes the final bf16 output.  Two forms: one CTA per item
+//                   (attn_decode_kernel<HD, false>), and a grid of resident CTAs that draw items
+//                   from a counter and keep their page pipelines running across item boundaries
+//                   (attn_suffix_resident_kernel, used while sequences hold few generated tokens).
 //
 // Both run the same tile loop: the four warps of a CTA take pages round-robin; each warp streams
 // its pages (one 16-token page of one kv head = K burst + V burst) through its own TMA pipeline
@@ -223,6 +226,96 @@ struct DecSmem {
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// One 16-token page of one kv head against the warp's 16 query rows: S = Q K^T, online softmax
+// (exp2 domain), O += P V.  st = shared-memory address of the page (K burst then V burst, 128-byte
+// swizzle); key0 = index of the page's first key; keys at or beyond n_keys are masked.
+template <int HD>
+__device__ __forceinline__ void decode_tile(uint32_t st, int key0, int n_keys, float scale_log2, int lane,
+                                            const uint32_t (&qf)[HD / 16][4], float (&o_acc)[HD / 8][4],
+                                            float (&m_run)[2], float (&l_run)[2]) {
+  using S = DecSmem<HD>;
+  constexpr int KSTEPS = HD / 16;
+  constexpr int HALVES = HD / 64;
+  const int qi = lane & 3;
+
+  // ---- S = Q K^T : 16 rows x 16 keys -------------------------------------------------------
+  float sc[2][4];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f;
+  {
+    const int id = lane >> 3, rr = lane & 7;
+    const int key = (id >> 1) * 8 + rr;
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+      const int c = 2 * (kk & 3) + (id & 1);
+      const uint32_t addr = st + (kk >> 2) * (S::kStageBytes / HALVES) + key * 128 + ((c ^ (key & 7)) << 4);
+      uint32_t b0, b1, b2, b3;
+      ldmatrix_x4(addr, b0, b1, b2, b3);
+      mma_bf16_16816(sc[0], qf[kk], b0, b1);
+      mma_bf16_16816(sc[1], qf[kk], b2, b3);
+    }
+  }
+  // ---- online softmax (exp2 domain) ---------------------------------------------------------
+  float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+  for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int key = key0 + 8 * nt + 2 * qi + (e & 1);
+      const float v = key < n_keys ? sc[nt][e] * scale_log2 : -INFINITY;
+      sc[nt][e] = v;
+      mx[e >> 1] = fmaxf(mx[e >> 1], v);
+    }
+  }
+  uint32_t pa[4];
+  {
+    float corr[2], msafe[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+      mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+      const float m_new = fmaxf(m_run[r], mx[r]);
+      msafe[r] = m_new == -INFINITY ? 0.f : m_new;
+      corr[r] = exp2f(m_run[r] - msafe[r]);           // 0 when nothing was accumulated yet
+      m_run[r] = m_new;
+    }
+    float p[2][4], ps[2] = {0.f, 0.f};
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        p[nt][e] = exp2f(sc[nt][e] - msafe[e >> 1]);
+        ps[e >> 1] += p[nt][e];
+      }
+    l_run[0] = l_run[0] * corr[0] + ps[0];
+    l_run[1] = l_run[1] * corr[1] + ps[1];
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) {
+      o_acc[i][0] *= corr[0]; o_acc[i][1] *= corr[0];
+      o_acc[i][2] *= corr[1]; o_acc[i][3] *= corr[1];
+    }
+    pa[0] = pack_bf16(p[0][0], p[0][1]);
+    pa[1] = pack_bf16(p[0][2], p[0][3]);
+    pa[2] = pack_bf16(p[1][0], p[1][1]);
+    pa[3] = pack_bf16(p[1][2], p[1][3]);
+  }
+  // ---- O += P V ---------------------------------------------------------------------------
+  {
+    const int id = lane >> 3, rr = lane & 7;
+    const int key = (id & 1) * 8 + rr;
+#pragma unroll
+    for (int dt = 0; dt < KSTEPS; ++dt) {
+      const int c = 2 * (dt & 3) + (id >> 1);
+      const uint32_t addr = st + (dt >> 2) * (S::kStageBytes / HALVES) + kPageTokens * 128 + key * 128 +
+                            ((c ^ (key & 7)) << 4);
+      uint32_t v0, v1, v2, v3;
+      ldmatrix_x4_trans(addr, v0, v1, v2, v3);
+      mma_bf16_16816(o_acc[2 * dt], pa, v0, v1);
+      mma_bf16_16816(o_acc[2 * dt + 1], pa, v2, v3);
+    }
+  }
 }
 
 template <int HD, bool PREFIX>
@@ -361,83 +454,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
     if (!ok) break;
     const uint32_t st = smem_u32(my_stages + (k % kDecStages) * S::kStageBytes);
     const int key0 = (warp + kDecWarps * k) * kPageTokens;
-
-    // ---- S = Q K^T : 16 rows x 16 keys -------------------------------------------------------
-    float sc[2][4];
-#pragma unroll
-    for (int i = 0; i < 2; ++i) sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f;
-    {
-      const int id = lane >> 3, rr = lane & 7;
-      const int key = (id >> 1) * 8 + rr;
-#pragma unroll
-      for (int kk = 0; kk < KSTEPS; ++kk) {
-        const int c = 2 * (kk & 3) + (id & 1);
-        const uint32_t addr = st + (kk >> 2) * (S::kStageBytes / HALVES) + key * 128 + ((c ^ (key & 7)) << 4);
-        uint32_t b0, b1, b2, b3;
-        ldmatrix_x4(addr, b0, b1, b2, b3);
-        mma_bf16_16816(sc[0], qf[kk], b0, b1);
-        mma_bf16_16816(sc[1], qf[kk], b2, b3);
-      }
-    }
-    // ---- online softmax (exp2 domain) ---------------------------------------------------------
-    float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int key = key0 + 8 * nt + 2 * qi + (e & 1);
-        const float v = key < n_keys ? sc[nt][e] * scale_log2 : -INFINITY;
-        sc[nt][e] = v;
-        mx[e >> 1] = fmaxf(mx[e >> 1], v);
-      }
-    }
-    uint32_t pa[4];
-    {
-      float corr[2], msafe[2];
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-        const float m_new = fmaxf(m_run[r], mx[r]);
-        msafe[r] = m_new == -INFINITY ? 0.f : m_new;
-        corr[r] = exp2f(m_run[r] - msafe[r]);           // 0 when nothing was accumulated yet
-        m_run[r] = m_new;
-      }
-      float p[2][4], ps[2] = {0.f, 0.f};
-#pragma unroll
-      for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          p[nt][e] = exp2f(sc[nt][e] - msafe[e >> 1]);
-          ps[e >> 1] += p[nt][e];
-        }
-      l_run[0] = l_run[0] * corr[0] + ps[0];
-      l_run[1] = l_run[1] * corr[1] + ps[1];
-#pragma unroll
-      for (int i = 0; i < HD / 8; ++i) {
-        o_acc[i][0] *= corr[0]; o_acc[i][1] *= corr[0];
-        o_acc[i][2] *= corr[1]; o_acc[i][3] *= corr[1];
-      }
-      pa[0] = pack_bf16(p[0][0], p[0][1]);
-      pa[1] = pack_bf16(p[0][2], p[0][3]);
-      pa[2] = pack_bf16(p[1][0], p[1][1]);
-      pa[3] = pack_bf16(p[1][2], p[1][3]);
-    }
-    // ---- O += P V ---------------------------------------------------------------------------
-    {
-      const int id = lane >> 3, rr = lane & 7;
-      const int key = (id & 1) * 8 + rr;
-#pragma unroll
-      for (int dt = 0; dt < KSTEPS; ++dt) {
-        const int c = 2 * (dt & 3) + (id >> 1);
-        const uint32_t addr = st + (dt >> 2) * (S::kStageBytes / HALVES) + kPageTokens * 128 + key * 128 +
-                              ((c ^ (key & 7)) << 4);
-        uint32_t v0, v1, v2, v3;
-        ldmatrix_x4_trans(addr, v0, v1, v2, v3);
-        mma_bf16_16816(o_acc[2 * dt], pa, v0, v1);
-        mma_bf16_16816(o_acc[2 * dt + 1], pa, v2, v3);
-      }
-    }
+    decode_tile<HD>(st, key0, n_keys, scale_log2, lane, qf, o_acc, m_run, l_run);
     __syncwarp();
     if (k + kDecStages < n_my) issue(k + kDecStages);
   }
@@ -543,6 +560,319 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, STATUS_WAIT_TIMEOUT);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Suffix attention with resident CTAs.  With one CTA per (sequence, kv head) every CTA pays its
+// start-up chain (row position -> page ids -> first pages) and its merge with an idle copy
+// pipeline, and CTAs of equal length march through those phases together.  Here a grid that just
+// fills the GPU walks the (sequence, kv head) items round-robin, and each warp's page pipeline
+// runs on across item boundaries: the first pages of the next item are requested before the
+// current item is merged, and the next item's row position and page ids are fetched one item
+// ahead, so the copy engine stays busy while partial results are combined and written.
+// Shared memory: the four warps' page stages, then a merge area of REP rows per warp.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSufPre = 4;                  // merged outputs per thread: REP * HD <= kSufPre * threads
+
+template <int HD>
+struct SufSmem {
+  static constexpr int kStageBytes = DecSmem<HD>::kStageBytes;
+  static constexpr int kPipeBytes = DecSmem<HD>::kPipeBytes;
+  static constexpr int kRowStride = HD + 8;                                    // floats; spreads rows over banks
+  static constexpr int kStatFloats = 2 * kDecWarps * 16;                       // running max and sum per warp row
+  static constexpr int merge_bytes(int rep) { return (kStatFloats + kDecWarps * rep * kRowStride) * 4; }
+  static constexpr int total(int rep) { return 1024 + kPipeBytes + merge_bytes(rep) + 256; }
+};
+
+template <int HD>
+__global__ void __launch_bounds__(kDecWarps * 32)
+attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16 *__restrict__ q,
+                            __nv_bfloat16 *__restrict__ out, const float *__restrict__ pre_o,
+                            const float2 *__restrict__ pre_ml, const int32_t *__restrict__ page_table, int pt_width,
+                            const int32_t *__restrict__ row_pos, const int32_t *__restrict__ full_pages,
+                            int layer_row0, int Hq, int Hkv, int n_items, int n_pages, float scale_log2,
+                            const int32_t *__restrict__ row_done, int *status, int *work) {
+  using S = SufSmem<HD>;
+  constexpr int KSTEPS = HD / 16;
+  constexpr int HALVES = HD / 64;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int REP = Hq / Hkv;
+  float *m_s = reinterpret_cast<float *>(smem + S::kPipeBytes);               // [warp][16]
+  float *l_s = m_s + kDecWarps * 16;
+  float *o_s = l_s + kDecWarps * 16;                                          // [warp][REP][kRowStride]
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + S::kPipeBytes + S::merge_bytes(REP));   // [warp][stage]
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + kDecWarps * kDecStages);
+  volatile int *ticket_s = abort_flag + 1;   // [2]: item numbers drawn by thread 0, alternating slots
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int quad = lane >> 2, qi = lane & 3;
+
+  // Items are handed out through a counter: CTA b starts with item b and draws every later item
+  // (work[0] counts the draws), so CTAs that start late or run slow take fewer items.  A draw is made
+  // two items ahead by thread 0 and passed on at a barrier the merge needs anyway.  work[1] counts
+  // finished CTAs; the last one puts both words back to zero for the next launch.
+  // The prefix launch (the predecessor) let this grid start only after its own dependency wait:
+  // q, the KV pool, row positions and page ids are complete.  They are read with L2-only loads or
+  // TMA; the prefix partials are read after griddep_wait() below.
+  griddep_launch();
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kDecWarps * kDecStages; ++i) mbar_init(&bars[i], 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+    ticket_s[1] = gridDim.x + atomicAdd(&work[0], 1);
+  }
+  __syncthreads();
+  int m1 = ticket_s[1];                      // the item after this CTA's first one
+
+  uint8_t *my_stages = smem + warp * kDecStages * S::kStageBytes;
+  uint64_t *my_bars = bars + warp * kDecStages;
+  uint32_t g_iss = 0, g_cons = 0;            // pages requested / consumed by this warp since the start
+
+  auto issue_page = [&](int page, int h) {   // warp-uniform arguments
+    if (lane == 0) {
+      uint64_t *bar = &my_bars[g_iss % kDecStages];
+      uint8_t *dst = my_stages + (g_iss % kDecStages) * S::kStageBytes;
+      if (page < 0 || page >= n_pages) {
+        atomicExch(status, STATUS_BAD_PAGE);
+        mbar_arrive(bar);                    // nothing to load: complete the phase by hand
+      } else {
+        const int row = layer_row0 + (page * Hkv + h) * 2 * kPageTokens;
+        mbar_expect_tx(bar, S::kStageBytes);
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf) tma_load_2d(&tmKV, bar, dst + hf * (S::kStageBytes / HALVES), hf * 64, row);
+      }
+    }
+    ++g_iss;
+  };
+  // Item m -> (sequence, kv head).  Its description is fetched in two hops that are issued well
+  // before their results are used: raw words (ended flag, prompt pages, position) first, then the
+  // page ids of this warp's first 32 pages, whose address depends on the first hop.
+  auto raw_words = [&](int m, int &seq, int &h, int &dn, int &fp, int &rp) {
+    const bool valid = m < n_items;
+    seq = valid ? m / Hkv : 0;
+    h = valid ? m - seq * Hkv : 0;
+    dn = row_done ? __ldcg(&row_done[seq]) : 0;
+    fp = __ldcg(&full_pages[seq]);
+    rp = __ldcg(&row_pos[seq]);
+    if (!valid) dn = 1;
+  };
+  // keys of the item (-1: an ended sequence or past the last item: nothing to do, nothing written),
+  // this warp's number of pages, and lane j's page id of the warp's page j
+  auto shape = [&](int seq, int dn, int fp, int rp, int &n_keys, int &n_my, int &pg) {
+    n_keys = dn ? -1 : rp + 1 - fp * kPageTokens;
+    const int n_tiles = dn ? 0 : (n_keys + kPageTokens - 1) / kPageTokens;
+    n_my = n_tiles > warp ? (n_tiles - warp + kDecWarps - 1) / kDecWarps : 0;
+    pg = lane < n_my ? __ldcg(&page_table[static_cast<size_t>(seq) * pt_width + fp + warp + kDecWarps * lane]) : 0;
+  };
+  // Q fragments of an item (rows >= REP of the MMA tile are padding)
+  uint32_t qf[KSTEPS][4];
+  auto load_q = [&](int seq, int h) {
+    const uint32_t *q_lo = quad < REP ? reinterpret_cast<const uint32_t *>(
+                                            q + (static_cast<size_t>(seq) * Hq + h * REP + quad) * HD)
+                                      : nullptr;
+    const uint32_t *q_hi = quad + 8 < REP ? reinterpret_cast<const uint32_t *>(
+                                                q + (static_cast<size_t>(seq) * Hq + h * REP + quad + 8) * HD)
+                                          : nullptr;
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+      qf[kk][0] = q_lo ? __ldcg(&q_lo[kk * 8 + qi]) : 0u;
+      qf[kk][1] = q_hi ? __ldcg(&q_hi[kk * 8 + qi]) : 0u;
+      qf[kk][2] = q_lo ? __ldcg(&q_lo[kk * 8 + 4 + qi]) : 0u;
+      qf[kk][3] = q_hi ? __ldcg(&q_hi[kk * 8 + 4 + qi]) : 0u;
+    }
+  };
+
+  int m = blockIdx.x;
+  int c_seq, c_h, c_fp, c_keys, c_my, c_pg;
+  {
+    int dn, rp;
+    raw_words(m, c_seq, c_h, dn, c_fp, rp);
+    shape(c_seq, dn, c_fp, rp, c_keys, c_my, c_pg);
+  }
+  {
+    const int c_first = c_my < kDecStages ? c_my : kDecStages;
+    for (int k = 0; k < c_first; ++k) issue_page(__shfl_sync(0xffffffffu, c_pg, k), c_h);
+  }
+  load_q(c_seq, c_h);
+  bool waited = false;
+
+  for (int n = 0; m < n_items; ++n) {
+    // ---- the next item, one item ahead: first hop now, second hop after the first page ---------
+    // thread 0 draws the item after the next one, late in the current item (a CTA that commits to
+    // items early leaves others idle at the end of the launch) but a few pages before the barrier
+    // that passes it on, so that the counter's round trip is hidden
+    int drawn = 0;
+    const int draw_at = c_keys >= 0 && c_my > 3 ? c_my - 3 : -1;
+    if (threadIdx.x == 0 && draw_at < 0) drawn = gridDim.x + atomicAdd(&work[0], 1);
+    int n_seq, n_h, n_dn, n_fp, n_rp;
+    raw_words(m1, n_seq, n_h, n_dn, n_fp, n_rp);
+    int n_keys = -1, n_my = 0, n_pg = 0, n_first = 0, nxt_issued = 0, m2 = 0;
+    auto second_hop = [&]() {
+      shape(n_seq, n_dn, n_fp, n_rp, n_keys, n_my, n_pg);
+      n_first = n_my < kDecStages ? n_my : kDecStages;
+    };
+    auto issue_next = [&]() {                // one more of the next item's first pages
+      issue_page(__shfl_sync(0xffffffffu, n_pg, nxt_issued), n_h);
+      ++nxt_issued;
+    };
+
+    if (c_keys >= 0) {                       // CTA-uniform
+      float o_acc[HD / 8][4];
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
+      float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+      int pg_cache = c_pg, pg_base = 0;
+      const int32_t *pt = page_table + static_cast<size_t>(c_seq) * pt_width + c_fp;
+      bool ok = true;
+      if (c_my == 0) second_hop();
+
+      for (int k = 0; k < c_my; ++k) {
+        if (threadIdx.x == 0 && k == draw_at) drawn = gridDim.x + atomicAdd(&work[0], 1);
+        ok = mbar_wait(&my_bars[g_cons % kDecStages], (g_cons / kDecStages) & 1, abort_flag);
+        if (!ok) break;
+        const uint32_t st = smem_u32(my_stages + (g_cons % kDecStages) * S::kStageBytes);
+        decode_tile<HD>(st, (warp + kDecWarps * k) * kPageTokens, c_keys, scale_log2, lane, qf, o_acc, m_run, l_run);
+        __syncwarp();
+        ++g_cons;
+        if (k == 0) second_hop();
+        const int kn = k + kDecStages;
+        if (kn < c_my) {
+          if (kn >= pg_base + 32) {
+            pg_base = kn;
+            pg_cache = kn + lane < c_my ? __ldcg(&pt[warp + kDecWarps * (kn + lane)]) : 0;
+          }
+          issue_page(__shfl_sync(0xffffffffu, pg_cache, kn - pg_base), c_h);
+        } else if (nxt_issued < n_first) {
+          issue_next();
+        }
+      }
+      if (ok)
+        while (nxt_issued < n_first) issue_next();
+      // ---- prefix partials of this item: the prefix launch must be complete from here on -------
+      if (!waited) {
+        griddep_wait();
+        waited = true;
+      }
+      float pre_val[kSufPre];
+      float2 pre_stat[kSufPre];
+#pragma unroll
+      for (int i = 0; i < kSufPre; ++i) {
+        const int idx = threadIdx.x + i * kDecWarps * 32;
+        pre_val[i] = 0.f;
+        pre_stat[i] = make_float2(-INFINITY, 0.f);
+        if (idx < REP * HD) {
+          const size_t rh = static_cast<size_t>(c_seq) * Hq + c_h * REP + idx / HD;
+          pre_stat[i] = __ldcg(&pre_ml[rh]);
+          pre_val[i] = __ldcg(&pre_o[rh * HD + idx % HD]);
+        }
+      }
+      if (ok && n_keys >= 0) load_q(n_seq, n_h);     // the next item's queries land during the merge
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+      }
+      // ---- combine the four warps ----------------------------------------------------------------
+      if (qi == 0) {
+        m_s[warp * 16 + quad] = m_run[0];
+        m_s[warp * 16 + quad + 8] = m_run[1];
+        l_s[warp * 16 + quad] = l_run[0];
+        l_s[warp * 16 + quad + 8] = l_run[1];
+      }
+      if (quad < REP) {
+        float *o_lo = o_s + (warp * REP + quad) * S::kRowStride + 2 * qi;
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i) *reinterpret_cast<float2 *>(o_lo + 8 * i) = make_float2(o_acc[i][0], o_acc[i][1]);
+      }
+      if (quad + 8 < REP) {
+        float *o_hi = o_s + (warp * REP + quad + 8) * S::kRowStride + 2 * qi;
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i) *reinterpret_cast<float2 *>(o_hi + 8 * i) = make_float2(o_acc[i][2], o_acc[i][3]);
+      }
+      if (threadIdx.x == 0) ticket_s[n & 1] = drawn;
+      __syncthreads();
+      if (*abort_flag) break;                // some warp gave up: every thread of the CTA sees it here
+      m2 = ticket_s[n & 1];
+#pragma unroll
+      for (int i = 0; i < kSufPre; ++i) {
+        const int idx = threadIdx.x + i * kDecWarps * 32;
+        if (idx < REP * HD) {
+          const int r = idx / HD, d = idx % HD;
+          float M = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, m_s[w * 16 + r]);
+          float L = 0.f, O = 0.f;
+#pragma unroll
+          for (int w = 0; w < kDecWarps; ++w) {
+            const float mw = m_s[w * 16 + r];
+            if (mw != -INFINITY) {
+              const float c = exp2f(mw - M);
+              L += l_s[w * 16 + r] * c;
+              O += o_s[(w * REP + r) * S::kRowStride + d] * c;
+            }
+          }
+          const float2 ml = pre_stat[i];
+          float Mt = fmaxf(M, ml.x);
+          if (Mt == -INFINITY) Mt = 0.f;
+          const float c_suf = M == -INFINITY ? 0.f : exp2f(M - Mt);
+          const float c_pre = ml.x == -INFINITY ? 0.f : exp2f(ml.x - Mt);
+          const float Lt = L * c_suf + ml.y * c_pre;
+          const float Ot = O * c_suf + (c_pre != 0.f ? pre_val[i] * c_pre : 0.f);
+          out[(static_cast<size_t>(c_seq) * Hq + c_h * REP + r) * HD + d] = __float2bfloat16(Ot / Lt);
+        }
+      }
+      __syncthreads();                       // the merge area is free for the next item
+    } else {
+      second_hop();
+      while (nxt_issued < n_first) issue_next();
+      if (n_keys >= 0) load_q(n_seq, n_h);
+      if (threadIdx.x == 0) ticket_s[n & 1] = drawn;
+      __syncthreads();
+      m2 = ticket_s[n & 1];
+    }
+    m = m1;
+    m1 = m2;
+    c_seq = n_seq; c_h = n_h; c_fp = n_fp; c_keys = n_keys; c_my = n_my; c_pg = n_pg;
+  }
+  if (*abort_flag) {
+    // give copies already in flight a chance to land before shared memory is released
+    for (uint32_t g = g_cons; g < g_iss; ++g) mbar_drain(&my_bars[g % kDecStages], (g / kDecStages) & 1);
+    if (threadIdx.x == 0) atomicExch(status, STATUS_WAIT_TIMEOUT);
+  }
+  if (!waited) griddep_wait();               // this grid never completes ahead of its predecessor
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(&work[1], 1) == static_cast<int>(gridDim.x) - 1) {
+      atomicExch(&work[0], 0);
+      atomicExch(&work[1], 0);
+    }
+  }
+}
+
+// ECHO_ATTN_IMPL=waves keeps one CTA per (sequence, kv head) for the suffix (diagnostic A/B runs).
+bool suffix_resident() {
+  static const bool on = [] {
+    const char *e = getenv("ECHO_ATTN_IMPL");
+    return !(e && !strcmp(e, "waves"));
+  }();
+  return on;
+}
+
+// CTAs of `kernel` that fit the current device at once (per device and REP; no stream work).
+template <typename K>
+int resident_slots(K kernel, int smem_bytes, int rep) {
+  static int cache[64][17] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || rep < 1 || rep > 16) return 0;
+  if (cache[dev][rep] == 0) {
+    int sms = 0, per_sm = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kDecWarps * 32, smem_bytes) != cudaSuccess)
+      return 0;
+    cache[dev][rep] = sms * per_sm;
+  }
+  return cache[dev][rep];
+}
+
 template <int HD>
 cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
   using S = DecSmem<HD>;
@@ -553,6 +883,16 @@ cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
                                *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos,
                                a.full_pages, a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
   if (e != cudaSuccess) return e;
+  if (suffix_resident() && a.work && REP * HD <= 512) {   // merge area small enough for three CTAs per SM
+    using R = SufSmem<HD>;
+    const int n_items = a.P * a.G * a.Hkv;
+    const int slots = resident_slots(attn_suffix_resident_kernel<HD>, R::total(REP), REP);
+    if (slots <= 0) return cudaErrorInvalidConfiguration;
+    return launch_early(attn_suffix_resident_kernel<HD>, dim3(n_items < slots ? n_items : slots), dim3(kDecWarps * 32),
+                        R::total(REP), s, *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos,
+                        a.full_pages, a.layer_row0, a.Hq, a.Hkv, n_items, a.n_pages, scale_log2, a.row_done, a.status,
+                        a.work);
+  }
   return launch_early(attn_decode_kernel<HD, false>, dim3(a.P * a.G * a.Hkv), dim3(kDecWarps * 32), S::kTotal, s,
                       *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages,
                       a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
@@ -566,6 +906,10 @@ cudaError_t attention_decode_configure() {
                                 DecSmem<128>::kTotal)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(attn_decode_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 DecSmem<128>::kTotal)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(attn_suffix_resident_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                SufSmem<128>::total(kSufPre * kDecWarps * 32 / 128))) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(attn_suffix_resident_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                SufSmem<64>::total(kSufPre * kDecWarps * 32 / 64))) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(attn_decode_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 DecSmem<64>::kTotal)) != cudaSuccess) return e;
   return cudaFuncSetAttribute(attn_decode_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -211,6 +211,8 @@ struct DecodeAttnArgs {
   int P, G, Hq, Hkv, hd, n_pages;
   int *status;
   const int32_t *row_done;        // optional, per sequence: non-zero = ended, its suffix CTAs return at once
+  int *work = nullptr;            // two zeroed ints: item counter of the resident suffix kernel, which leaves
+                                  // them zero again (null: one suffix CTA per (sequence, kv head))
 };
 cudaError_t attention_decode_configure();
 bool attention_decode_supported(int hd, int page_size, int Hq, int Hkv);

@@ -85,7 +85,7 @@ Limits limits_of(const echo_config &c) {
 struct Layout {
   size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
   size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
-      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, row_done, copy_src, copy_dst, d_step, status, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
+      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, row_done, copy_src, copy_dst, d_step, status, attn_work, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
   size_t weight_bytes, kv_layer_elems, n_tables_ints;
   int n_chunks_max;
 };
@@ -132,6 +132,7 @@ Layout layout_of(const echo_config &c) {
   lo.copy_dst = take(static_cast<size_t>(M.B) * 4);
   lo.d_step = take(4);
   lo.status = take(4);
+  lo.attn_work = take(8);
   lo.gemm_ws = take(static_cast<size_t>(kMaxCtas) * 3 * 2 * kGemmTileN * kMaxBatchTile * sizeof(float));
   lo.gemm_counters = take(static_cast<size_t>(kGemmMaxUnits) * 4);
   lo.stage_prompts = take(static_cast<size_t>(M.P) * M.Lp * 4);
@@ -180,6 +181,7 @@ struct echo_ctx {
   echo_stats stats{};
   int64_t launches = 0;
   bool use_simt = false, use_graph = true, fast_decode = false, deterministic = false, use_pdl = true, use_pair = true;
+  bool long_suffix = false;   // decode steps whose sequences hold many generated tokens (see kLongSuffix)
   CUtensorMap tm_kv;
   std::string last_error;
   // sampled per-kernel timing (echo_profile_config / echo_profile_read)
@@ -256,6 +258,10 @@ struct DeviceGuard {
     if (prev >= 0) cudaSetDevice(prev);
   }
 };
+
+// Decode step from which the suffix attention runs one CTA per (sequence, kv head) again (measured
+// crossover of the two suffix kernels at the 8B shape: ~1100 generated tokens per sequence).
+constexpr int kLongSuffix = 1088;
 
 int pick_bnb(int rows) {
   if (rows <= 32) return 32;
@@ -341,7 +347,8 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int d
       DecodeAttnArgs da{&ctx->tm_kv, q, attn, ctx->ptr<float>(lo.pre_o), ctx->ptr<float2>(lo.pre_ml), pt,
                         ctx->M.pt_width, meta.row_pos, ctx->ptr<int32_t>(lo.full_pages),
                         static_cast<int>(static_cast<size_t>(l) * (lo.kv_layer_elems / D.hd)), decode_P, decode_G,
-                        D.Hq, D.Hkv, D.hd, ctx->M.n_pages, status, meta.row_done};
+                        D.Hq, D.Hkv, D.hd, ctx->M.n_pages, status, meta.row_done,
+                        ctx->long_suffix ? nullptr : ctx->ptr<int>(lo.attn_work)};
       LAUNCH(attention_decode_launch(da, ctx->stream));
       ctx->launches++;                      // two kernels per call
     } else {
@@ -649,26 +656,37 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   // ---- decode steps 1..T-1 ----------------------------------------------------
   const int32_t *tok_hist = forced ? forced : out_tokens;
   const int n_steps = T - 1;
-  cudaGraph_t graph = nullptr;
-  cudaGraphExec_t exec = nullptr;
+  // Two captures of the same step, which differ in the suffix attention kernel: resident CTAs while
+  // the sequences hold few generated tokens (their fixed cost per item is what counts), one CTA per
+  // (sequence, kv head) from kLongSuffix generated tokens on (the launch is bound by the KV stream).
+  cudaGraph_t graph[2] = {nullptr, nullptr};
+  cudaGraphExec_t exec[2] = {nullptr, nullptr};
   int64_t per_step = 0;
   if (n_steps > 1 && ctx->use_graph && ctx->stream != nullptr) {
-    const int64_t before = ctx->launches;
-    if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+    for (int v = 0; v < 2; ++v) {
+      if (v == 1 && n_steps < kLongSuffix) break;
+      const int64_t before = ctx->launches;
+      if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        cudaGetLastError();
+        break;
+      }
+      ctx->long_suffix = v == 1;
       int src = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs);
-      cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
+      ctx->long_suffix = false;
+      cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph[v]);
       per_step = ctx->launches - before;
       ctx->launches = before;
       if (src != ECHO_OK) {
-        if (graph) cudaGraphDestroy(graph);
+        for (int u = 0; u < 2; ++u) {
+          if (exec[u]) cudaGraphExecDestroy(exec[u]);
+          if (graph[u]) cudaGraphDestroy(graph[u]);
+        }
         return src;
       }
-      if (e != cudaSuccess || cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) {
+      if (e != cudaSuccess || cudaGraphInstantiate(&exec[v], graph[v], 0) != cudaSuccess) {
         cudaGetLastError();
-        exec = nullptr;
+        exec[v] = nullptr;
       }
-    } else {
-      cudaGetLastError();
     }
   }
   ctx->prof_recs.clear();
@@ -676,19 +694,24 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   int rc_steps = ECHO_OK;
   for (int j = 1; j <= n_steps && rc_steps == ECHO_OK; ++j) {
     const bool sampled = ctx->prof_every > 0 && (j % ctx->prof_every == 0);
-    if (exec && !sampled) {
-      cudaError_t le = cudaGraphLaunch(exec, ctx->stream);
+    const int v = j >= kLongSuffix ? 1 : 0;
+    if (exec[v] && !sampled) {
+      cudaError_t le = cudaGraphLaunch(exec[v], ctx->stream);
       if (le != cudaSuccess) rc_steps = fail_cuda(ctx, le, "cudaGraphLaunch");
       ctx->launches += per_step;
     } else {
       ctx->prof_now = sampled;
       ctx->prof_step = j;
+      ctx->long_suffix = v == 1;
       rc_steps = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs);
+      ctx->long_suffix = false;
       ctx->prof_now = false;
     }
   }
-  if (exec) cudaGraphExecDestroy(exec);      // executions already enqueued keep their resources
-  if (graph) cudaGraphDestroy(graph);
+  for (int v = 0; v < 2; ++v) {
+    if (exec[v]) cudaGraphExecDestroy(exec[v]);      // executions already enqueued keep their resources
+    if (graph[v]) cudaGraphDestroy(graph[v]);
+  }
   if (rc_steps != ECHO_OK) return rc_steps;
   CK(cudaEventRecord(ctx->ev_end, ctx->stream));
   CK(cudaEventRecord(wp->last_use, ctx->stream));
@@ -807,6 +830,7 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
     }
   }
   if ((e = cudaMemsetAsync(ctx->arena + lo.status, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
+  if ((e = cudaMemsetAsync(ctx->arena + lo.attn_work, 0, 8, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
   if ((e = cudaMemsetAsync(ctx->arena + lo.d_step, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
   if ((e = cudaMemsetAsync(ctx->arena + lo.qkv, 0, static_cast<size_t>(ctx->M.R) * ctx->D.n_qkv() * 4, ctx->stream)) !=
       cudaSuccess)
@@ -1124,9 +1148,10 @@ int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, c
   float *pre_o = reinterpret_cast<float *>(sc);
   float2 *pre_ml = reinterpret_cast<float2 *>(sc + align_up(static_cast<size_t>(B) * Hq * hd * 4));
   int *status = reinterpret_cast<int *>(reinterpret_cast<uint8_t *>(pre_ml) + align_up(static_cast<size_t>(B) * Hq * 8));
-  if (cudaMemsetAsync(status, 0, 4, s) != cudaSuccess) return ECHO_ERR_CUDA;
+  if (cudaMemsetAsync(status, 0, 16, s) != cudaSuccess) return ECHO_ERR_CUDA;     // status word + item counters
   DecodeAttnArgs da{&tm, static_cast<const __nv_bfloat16 *>(q), static_cast<__nv_bfloat16 *>(out), pre_o, pre_ml,
-                    page_table, pt_width, row_pos, full_pages, 0, P, G, Hq, Hkv, hd, n_pages, status, nullptr};
+                    page_table, pt_width, row_pos, full_pages, 0, P, G, Hq, Hkv, hd, n_pages, status, nullptr,
+                    status + 2};
   if (attention_decode_launch(da, s) != cudaSuccess) return ECHO_ERR_CUDA;
   int st = 0;
   if (cudaMemcpyAsync(&st, status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ECHO_ERR_CUDA;

@@ -201,7 +201,9 @@ def test_gemm_swiglu_epilogue(B, M, F, K):
 
 
 @pytest.mark.parametrize("P,G,Hq,Hkv,hd,Lp,steps", [(4, 8, 32, 8, 128, 512, 1200), (3, 4, 4, 2, 64, 40, 37),
-                                                     (2, 2, 16, 2, 128, 7, 1), (2, 8, 8, 8, 128, 64, 300)])
+                                                     (2, 2, 16, 2, 128, 7, 1), (2, 8, 8, 8, 128, 64, 300),
+                                                     (16, 8, 32, 8, 128, 64, 70), (20, 8, 16, 8, 128, 16, 2),
+                                                     (40, 8, 8, 4, 64, 33, 150)])
 def test_decode_attention_matches_oracle(B, P, G, Hq, Hkv, hd, Lp, steps):
     """Shared-prefix decode attention against the oracle's single-query attention (fp64) on the same
     bf16-rounded q, K, V, gathered through the oracle's page plan."""
@@ -220,7 +222,10 @@ def test_decode_attention_matches_oracle(B, P, G, Hq, Hkv, hd, Lp, steps):
     out = out.float().cpu().numpy().astype(np.float64)
     poolf = widen_bf16(synth.bf16_bits(pool))
     qf = widen_bf16(synth.bf16_bits(q))
-    for s in sorted(set([0, 1, Bq // 2, Bq - 1])):
+    # more (sequence, kv head) items than CTAs fit the GPU at once: a resident CTA then walks several
+    # items and prefetches across their boundaries, so every fifth sequence is checked
+    many = Bq * Hkv > 400
+    for s in sorted(set([0, 1, Bq // 2, Bq - 1] + (list(range(0, Bq, 5)) if many else []))):
         n = int(pos[s]) + 1
         pg = plan.table[s, np.arange(n) // 16]
         K = poolf[pg, :, 0, np.arange(n) % 16, :]         # [n, Hkv, hd]
