@@ -26,7 +26,10 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-ATTN_DRAM_PER_ALG_BYTE = 170.4 / 166.2      # measured DRAM bytes per algorithmic byte (see profiles/)
+# measured DRAM bytes per algorithmic byte of the prefix + suffix launch (ncu, see profiles/): with the
+# resident suffix kernel (decode steps below LONG_SUFFIX_STEP) and with one suffix CTA per item (above)
+ATTN_DRAM_PER_ALG_BYTE = {"resident": 251.85 / 244.5, "waves": 171.06 / 166.2}
+LONG_SUFFIX_STEP = 1088
 METRIC = "rollout generated tokens/s"
 UNIT = "tokens/s"
 
@@ -267,11 +270,15 @@ def run_ours(args):
         dur_s = float(prof_ms[:, 0].sum()) / 1e3
         achieved = alg / dur_s / 1e9
         tot = float(prof_ms[:, 3].sum())
-        # DRAM bytes per launch: ncu counters of the current kernel on a small case of the same
-        # per-CTA work (profiles/attn_decode_kernel_P4_G8_Lp512_i1200.md: 170.4 MB read + written
-        # for 166.2 MB of algorithmic bytes, prefix + suffix launch), scaled to this workload's
-        # launches by their algorithmic bytes: the traffic is the KV stream and grows with it.
-        traffic = ATTN_DRAM_PER_ALG_BYTE * alg / attn_launches if wl.shape.head_dim == 128 else None
+        # DRAM bytes per launch: ncu counters of the current kernels on small cases of the same
+        # per-CTA work (profiles/attn_decode_kernels_small_cases.md: prefix + suffix launch, DRAM bytes
+        # read + written against their algorithmic bytes), scaled to this workload's launches by
+        # their algorithmic bytes: the traffic is the KV stream and grows with it.
+        traffic = None
+        if wl.shape.head_dim == 128:
+            small_merge = shape.n_q_heads // shape.n_kv_heads * shape.head_dim <= 512   # resident kernel's limit
+            traffic = sum(ATTN_DRAM_PER_ALG_BYTE["resident" if small_merge and int(j) < LONG_SUFFIX_STEP else "waves"] *
+                          attention_bytes(shape, P, G, Lp, int(j)) for j in prof_steps) * shape.n_layers / attn_launches
         roof = {"bound": "hbm", "kernel": "decode attention (paged GQA)", "achieved": round(achieved, 1),
                 "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                 "frac": round(achieved / peaks["hbm_gbs"], 4),

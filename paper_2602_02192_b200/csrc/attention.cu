@@ -189,9 +189,10 @@ cudaError_t attention_rows_launch(const __nv_bfloat16 *q, const __nv_bfloat16 *k
 // the prefix is attended ONCE per (group, kv head) for all G * (Hq/Hkv) query rows that use it,
 // and only each sample's own generated tokens are read per sample.
 //
-//   prefix kernel   one CTA per (prompt, kv head, 16-row tile of the group's query rows); keys =
-//                   the prompt's full pages; writes un-normalised partial outputs with their
-//                   running max and sum to scratch.
+//   prefix kernel   keys = the prompt's full pages; writes un-normalised partial outputs with their
+//                   running max and sum to scratch.  One CTA per (prompt, kv head) when the
+//                   group's query rows fill two 16-row tiles (attn_prefix_group_kernel), else one
+//                   CTA per (prompt, kv head, 16-row tile) (attn_decode_kernel<HD, true>).
 //   suffix kernel   per (sequence, kv head) item: keys = the sequence's private pages (copy of
 //                   the prompt's partial last page + generated tokens); merges with the prefix
 //                   partial and writes the final bf16 output.  Two forms: one CTA per item
@@ -848,14 +849,276 @@ attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv
   }
 }
 
-// ECHO_ATTN_IMPL=waves keeps one CTA per (sequence, kv head) for the suffix (diagnostic A/B runs).
-bool suffix_resident() {
-  static const bool on = [] {
-    const char *e = getenv("ECHO_ATTN_IMPL");
-    return !(e && !strcmp(e, "waves"));
-  }();
-  return on;
+// ---------------------------------------------------------------------------------------------
+// Prefix attention with all query rows of a group in one CTA.  With 16-row tiles a group of
+// G * REP = 32 rows takes two CTAs per (prompt, kv head), which stream the same pages twice (the
+// second time from L2) and make the launch larger than the GPU holds at once.  Here one CTA keeps
+// MT 16-row tiles: every K and V fragment it reads from shared memory feeds MT MMAs.  The queries
+// stay in shared memory (16-byte chunks swizzled by row, read back with ldmatrix) so that the MT
+// accumulators fit the register file.
+// ---------------------------------------------------------------------------------------------
+template <int HD, int MT>
+struct PreSmem {
+  static constexpr int kStageBytes = DecSmem<HD>::kStageBytes;
+  static constexpr int kPipeBytes = DecSmem<HD>::kPipeBytes;
+  static constexpr int kQBytes = MT * 16 * HD * 2;
+  static constexpr int kRowStride = HD + 8;                                    // floats; spreads rows over banks
+  static constexpr int kMergeBytes = kDecWarps * MT * 16 * (kRowStride + 2) * 4;
+  static constexpr int kBody = kPipeBytes + kQBytes > kMergeBytes ? kPipeBytes + kQBytes : kMergeBytes;
+  static constexpr int kTotal = kBody + 256 + 1024;
+};
+
+template <int HD, int MT>
+__global__ void __launch_bounds__(kDecWarps * 32)
+attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16 *__restrict__ q,
+                         float *__restrict__ pre_o, float2 *__restrict__ pre_ml,
+                         const int32_t *__restrict__ page_table, int pt_width, const int32_t *__restrict__ full_pages,
+                         int layer_row0, int Hq, int Hkv, int G, int n_pages, float scale_log2, int *status) {
+  using S = PreSmem<HD, MT>;
+  constexpr int KSTEPS = HD / 16;
+  constexpr int HALVES = HD / 64;
+  constexpr int CHUNKS = HD / 8;             // 16-byte chunks per query row
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t *q_s = smem + S::kPipeBytes;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + S::kBody);              // [warp][stage]
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + kDecWarps * kDecStages);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int REP = Hq / Hkv;
+  const int quad = lane >> 2, qi = lane & 3;
+  const int n_rows = G * REP;                // <= MT * 16
+
+  // wait for the kernel that wrote q and the new K/V rows, then let the suffix launch be scheduled
+  griddep_wait();
+  griddep_launch();
+
+  const int h = blockIdx.x % Hkv;
+  const int seq0 = (blockIdx.x / Hkv) * G;   // first sequence of the group
+  const int n_keys = __ldcg(&full_pages[seq0]) * kPageTokens;
+  const int n_tiles = n_keys / kPageTokens;
+  const int32_t *pt = page_table + static_cast<size_t>(seq0) * pt_width;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kDecWarps * kDecStages; ++i) mbar_init(&bars[i], 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  uint8_t *my_stages = smem + warp * kDecStages * S::kStageBytes;
+  uint64_t *my_bars = bars + warp * kDecStages;
+  const int n_my = n_tiles > warp ? (n_tiles - warp + kDecWarps - 1) / kDecWarps : 0;
+
+  int pg_cache = 0, pg_base = -1;            // page ids of 32 of this warp's tiles, one per lane
+  auto page_of = [&](int k) -> int {         // warp-uniform k
+    if (pg_base < 0 || k >= pg_base + 32) {
+      pg_base = k;
+      const int kk = k + lane;
+      pg_cache = kk < n_my ? __ldcg(&pt[warp + kDecWarps * kk]) : 0;
+    }
+    return __shfl_sync(0xffffffffu, pg_cache, k - pg_base);
+  };
+  auto issue = [&](int k) {
+    const int page = page_of(k);
+    if (lane == 0) {
+      uint64_t *bar = &my_bars[k % kDecStages];
+      uint8_t *dst = my_stages + (k % kDecStages) * S::kStageBytes;
+      if (page < 0 || page >= n_pages) {
+        atomicExch(status, STATUS_BAD_PAGE);
+        mbar_arrive(bar);                    // nothing to load: complete the phase by hand
+      } else {
+        const int row = layer_row0 + (page * Hkv + h) * 2 * kPageTokens;
+        mbar_expect_tx(bar, S::kStageBytes);
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf) tma_load_2d(&tmKV, bar, dst + hf * (S::kStageBytes / HALVES), hf * 64, row);
+      }
+    }
+  };
+  const int n_pro = n_my < kDecStages ? n_my : kDecStages;
+  for (int k = 0; k < n_pro; ++k) issue(k);
+
+  // ---- queries -> shared memory: row r = (sequence seq0 + r / REP, head h * REP + r % REP) ------
+  for (int c = threadIdx.x; c < MT * 16 * CHUNKS; c += kDecWarps * 32) {
+    const int r = c / CHUNKS, ch = c % CHUNKS;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (r < n_rows)
+      v = __ldcg(reinterpret_cast<const uint4 *>(q + (static_cast<size_t>(seq0 + r / REP) * Hq + h * REP + r % REP) * HD) +
+                 ch);
+    *reinterpret_cast<uint4 *>(q_s + r * (HD * 2) + ((ch ^ (r & 7)) << 4)) = v;
+  }
+  __syncthreads();
+
+  float o_acc[MT][HD / 8][4];
+  float m_run[MT][2], l_run[MT][2];
+#pragma unroll
+  for (int t = 0; t < MT; ++t) {
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) o_acc[t][i][0] = o_acc[t][i][1] = o_acc[t][i][2] = o_acc[t][i][3] = 0.f;
+    m_run[t][0] = m_run[t][1] = -INFINITY;
+    l_run[t][0] = l_run[t][1] = 0.f;
+  }
+  const uint32_t q_addr = smem_u32(q_s);
+
+  bool ok = true;
+  for (int k = 0; k < n_my; ++k) {
+    ok = mbar_wait(&my_bars[k % kDecStages], (k / kDecStages) & 1, abort_flag);
+    if (!ok) break;
+    const uint32_t st = smem_u32(my_stages + (k % kDecStages) * S::kStageBytes);
+    // ---- S = Q K^T : MT x (16 rows x 16 keys); all keys of a full prompt page are valid ---------
+    float sc[MT][2][4];
+#pragma unroll
+    for (int t = 0; t < MT; ++t)
+#pragma unroll
+      for (int i = 0; i < 2; ++i) sc[t][i][0] = sc[t][i][1] = sc[t][i][2] = sc[t][i][3] = 0.f;
+    {
+      const int id = lane >> 3, rr = lane & 7;
+      const int key = (id >> 1) * 8 + rr;
+      const int q_row = rr + 8 * (id & 1);   // ldmatrix source row of this lane within a 16-row tile
+#pragma unroll
+      for (int kk = 0; kk < KSTEPS; ++kk) {
+        const int c = 2 * (kk & 3) + (id & 1);
+        const uint32_t addr = st + (kk >> 2) * (S::kStageBytes / HALVES) + key * 128 + ((c ^ (key & 7)) << 4);
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4(addr, b0, b1, b2, b3);
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+          uint32_t a[4];
+          const int qc = 2 * kk + (id >> 1);
+          ldmatrix_x4(q_addr + (t * 16 + q_row) * (HD * 2) + ((qc ^ (q_row & 7)) << 4), a[0], a[1], a[2], a[3]);
+          mma_bf16_16816(sc[t][0], a, b0, b1);
+          mma_bf16_16816(sc[t][1], a, b2, b3);
+        }
+      }
+    }
+    // ---- online softmax (exp2 domain) ---------------------------------------------------------
+    uint32_t pa[MT][4];
+#pragma unroll
+    for (int t = 0; t < MT; ++t) {
+      float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          sc[t][nt][e] *= scale_log2;
+          mx[e >> 1] = fmaxf(mx[e >> 1], sc[t][nt][e]);
+        }
+      float corr[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+        mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+        const float m_new = fmaxf(m_run[t][r], mx[r]);           // finite: every key is valid
+        corr[r] = exp2f(m_run[t][r] - m_new);                    // 0 when nothing was accumulated yet
+        m_run[t][r] = m_new;
+      }
+      float ps[2] = {0.f, 0.f};
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          sc[t][nt][e] = exp2f(sc[t][nt][e] - m_run[t][e >> 1]);
+          ps[e >> 1] += sc[t][nt][e];
+        }
+      l_run[t][0] = l_run[t][0] * corr[0] + ps[0];
+      l_run[t][1] = l_run[t][1] * corr[1] + ps[1];
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i) {
+        o_acc[t][i][0] *= corr[0]; o_acc[t][i][1] *= corr[0];
+        o_acc[t][i][2] *= corr[1]; o_acc[t][i][3] *= corr[1];
+      }
+      pa[t][0] = pack_bf16(sc[t][0][0], sc[t][0][1]);
+      pa[t][1] = pack_bf16(sc[t][0][2], sc[t][0][3]);
+      pa[t][2] = pack_bf16(sc[t][1][0], sc[t][1][1]);
+      pa[t][3] = pack_bf16(sc[t][1][2], sc[t][1][3]);
+    }
+    // ---- O += P V ---------------------------------------------------------------------------
+    {
+      const int id = lane >> 3, rr = lane & 7;
+      const int key = (id & 1) * 8 + rr;
+#pragma unroll
+      for (int dt = 0; dt < KSTEPS; ++dt) {
+        const int c = 2 * (dt & 3) + (id >> 1);
+        const uint32_t addr = st + (dt >> 2) * (S::kStageBytes / HALVES) + kPageTokens * 128 + key * 128 +
+                              ((c ^ (key & 7)) << 4);
+        uint32_t v0, v1, v2, v3;
+        ldmatrix_x4_trans(addr, v0, v1, v2, v3);
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+          mma_bf16_16816(o_acc[t][2 * dt], pa[t], v0, v1);
+          mma_bf16_16816(o_acc[t][2 * dt + 1], pa[t], v2, v3);
+        }
+      }
+    }
+    __syncwarp();
+    if (k + kDecStages < n_my) issue(k + kDecStages);
+  }
+  if (!ok) {
+    // give copies already in flight a chance to land before shared memory is reused or released
+    for (int k = 0; k < n_my; ++k) mbar_drain(&my_bars[k % kDecStages], (k / kDecStages) & 1);
+  }
+#pragma unroll
+  for (int t = 0; t < MT; ++t)
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      l_run[t][r] += __shfl_xor_sync(0xffffffffu, l_run[t][r], 1);
+      l_run[t][r] += __shfl_xor_sync(0xffffffffu, l_run[t][r], 2);
+    }
+
+  // ---- combine the four warps through shared memory (pipeline and query buffers are free now) --
+  __syncthreads();
+  constexpr int ROWS = MT * 16;
+  float *m_s = reinterpret_cast<float *>(smem);                      // [warp][ROWS]
+  float *l_s = m_s + kDecWarps * ROWS;
+  float *o_s = l_s + kDecWarps * ROWS;                               // [warp][ROWS][HD]
+#pragma unroll
+  for (int t = 0; t < MT; ++t) {
+    const int r_lo = t * 16 + quad, r_hi = r_lo + 8;
+    if (qi == 0) {
+      m_s[warp * ROWS + r_lo] = m_run[t][0];
+      m_s[warp * ROWS + r_hi] = m_run[t][1];
+      l_s[warp * ROWS + r_lo] = l_run[t][0];
+      l_s[warp * ROWS + r_hi] = l_run[t][1];
+    }
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) {
+      *reinterpret_cast<float2 *>(o_s + (warp * ROWS + r_lo) * S::kRowStride + 8 * i + 2 * qi) =
+          make_float2(o_acc[t][i][0], o_acc[t][i][1]);
+      *reinterpret_cast<float2 *>(o_s + (warp * ROWS + r_hi) * S::kRowStride + 8 * i + 2 * qi) =
+          make_float2(o_acc[t][i][2], o_acc[t][i][3]);
+    }
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < n_rows * HD; idx += blockDim.x) {
+    const int r = idx / HD, d = idx % HD;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, m_s[w * ROWS + r]);
+    float L = 0.f, O = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) {
+      const float mw = m_s[w * ROWS + r];
+      if (mw != -INFINITY) {
+        const float c = exp2f(mw - M);
+        L += l_s[w * ROWS + r] * c;
+        O += o_s[(w * ROWS + r) * S::kRowStride + d] * c;
+      }
+    }
+    const size_t rh = static_cast<size_t>(seq0 + r / REP) * Hq + h * REP + r % REP;
+    pre_o[rh * HD + d] = O;
+    if (d == 0) pre_ml[rh] = make_float2(M, L);
+  }
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(status, STATUS_WAIT_TIMEOUT);
 }
+
+// Diagnostic switches, read at each launch (A/B runs and tests):
+// ECHO_ATTN_IMPL=waves     one suffix CTA per (sequence, kv head) at every length
+// ECHO_ATTN_PREFIX=tiles   one prefix CTA per 16-row tile of a group's query rows
+bool attn_env_is(const char *name, const char *value) {
+  const char *e = getenv(name);
+  return e && !strcmp(e, value);
+}
+bool suffix_resident() { return !attn_env_is("ECHO_ATTN_IMPL", "waves"); }
 
 // CTAs of `kernel` that fit the current device at once (per device and REP; no stream work).
 template <typename K>
@@ -879,9 +1142,17 @@ cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
   const int REP = a.Hq / a.Hkv;
   const int MT = (a.G * REP + 15) / 16;
   const float scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(HD));
-  cudaError_t e = launch_early(attn_decode_kernel<HD, true>, dim3(a.P * a.Hkv * MT), dim3(kDecWarps * 32), S::kTotal, s,
-                               *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos,
-                               a.full_pages, a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
+  cudaError_t e;
+  if (MT == 2 && !attn_env_is("ECHO_ATTN_PREFIX", "tiles")) {
+    // the group's two 16-row tiles in one CTA: the launch fits the GPU at once
+    e = launch_early(attn_prefix_group_kernel<HD, 2>, dim3(a.P * a.Hkv), dim3(kDecWarps * 32), PreSmem<HD, 2>::kTotal, s,
+                     *a.tmKV, a.q, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.full_pages, a.layer_row0, a.Hq,
+                     a.Hkv, a.G, a.n_pages, scale_log2, a.status);
+  } else {
+    e = launch_early(attn_decode_kernel<HD, true>, dim3(a.P * a.Hkv * MT), dim3(kDecWarps * 32), S::kTotal, s,
+                     *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages,
+                     a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
+  }
   if (e != cudaSuccess) return e;
   if (suffix_resident() && a.work && REP * HD <= 512) {   // merge area small enough for three CTAs per SM
     using R = SufSmem<HD>;
@@ -906,6 +1177,10 @@ cudaError_t attention_decode_configure() {
                                 DecSmem<128>::kTotal)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(attn_decode_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 DecSmem<128>::kTotal)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(attn_prefix_group_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                PreSmem<128, 2>::kTotal)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(attn_prefix_group_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                PreSmem<64, 2>::kTotal)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(attn_suffix_resident_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 SufSmem<128>::total(kSufPre * kDecWarps * 32 / 128))) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(attn_suffix_resident_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -203,10 +203,20 @@ def test_gemm_swiglu_epilogue(B, M, F, K):
 @pytest.mark.parametrize("P,G,Hq,Hkv,hd,Lp,steps", [(4, 8, 32, 8, 128, 512, 1200), (3, 4, 4, 2, 64, 40, 37),
                                                      (2, 2, 16, 2, 128, 7, 1), (2, 8, 8, 8, 128, 64, 300),
                                                      (16, 8, 32, 8, 128, 64, 70), (20, 8, 16, 8, 128, 16, 2),
-                                                     (40, 8, 8, 4, 64, 33, 150)])
-def test_decode_attention_matches_oracle(B, P, G, Hq, Hkv, hd, Lp, steps):
+                                                     (40, 8, 8, 4, 64, 33, 150), (16, 8, 32, 8, 128, 512, 400),
+                                                     (3, 8, 8, 2, 64, 48, 20), (2, 6, 32, 8, 128, 100, 9)])
+@pytest.mark.parametrize("suffix", ["resident", "waves", "tiles"])
+def test_decode_attention_matches_oracle(B, monkeypatch, suffix, P, G, Hq, Hkv, hd, Lp, steps):
     """Shared-prefix decode attention against the oracle's single-query attention (fp64) on the same
-    bf16-rounded q, K, V, gathered through the oracle's page plan."""
+    bf16-rounded q, K, V, gathered through the oracle's page plan.  Both suffix kernels (resident CTAs
+    that walk several (sequence, kv head) items; "waves" = one CTA per item) and both prefix kernels
+    (a group's query rows in one CTA where they fill two 16-row tiles; "tiles" = one CTA per tile)."""
+    monkeypatch.delenv("ECHO_ATTN_IMPL", raising=False)
+    monkeypatch.delenv("ECHO_ATTN_PREFIX", raising=False)
+    if suffix == "waves":
+        monkeypatch.setenv("ECHO_ATTN_IMPL", "waves")
+    if suffix == "tiles":
+        monkeypatch.setenv("ECHO_ATTN_PREFIX", "tiles")
     from oracle import decoder as o_dec
     from oracle import pages as o_pages
     rng = np.random.default_rng(P * 131 + Lp)
