@@ -850,10 +850,10 @@ attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv
 }
 
 // ---------------------------------------------------------------------------------------------
-// Prefix attention with all query rows of a group in one CTA.  With 16-row tiles a group of
-// G * REP = 32 rows takes two CTAs per (prompt, kv head), which stream the same pages twice (the
-// second time from L2) and make the launch larger than the GPU holds at once.  Here one CTA keeps
-// MT 16-row tiles: every K and V fragment it reads from shared memory feeds MT MMAs.  The queries
+// Prefix attention with MT 16-row tiles of a group's query rows in one CTA.  With one tile per CTA
+// a group of G * REP = 32 rows takes two CTAs per (prompt, kv head), which stream the same pages
+// twice (the second time from L2) and make the launch larger than the GPU holds at once.  Here one
+// CTA keeps MT tiles (a group with more rows takes ceil(rows / (MT * 16)) CTAs): every K and V fragment it reads from shared memory feeds MT MMAs.  The queries
 // stay in shared memory (16-byte chunks swizzled by row, read back with ldmatrix) so that the MT
 // accumulators fit the register file.
 // ---------------------------------------------------------------------------------------------
@@ -887,14 +887,17 @@ attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bf
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int REP = Hq / Hkv;
   const int quad = lane >> 2, qi = lane & 3;
-  const int n_rows = G * REP;                // <= MT * 16
+  // a group with more than MT * 16 query rows takes several CTAs per (prompt, kv head)
+  const int n_blocks = (G * REP + MT * 16 - 1) / (MT * 16);
+  const int row0 = (blockIdx.x % n_blocks) * MT * 16;
+  const int n_rows = G * REP - row0 < MT * 16 ? G * REP - row0 : MT * 16;
 
   // wait for the kernel that wrote q and the new K/V rows, then let the suffix launch be scheduled
   griddep_wait();
   griddep_launch();
 
-  const int h = blockIdx.x % Hkv;
-  const int seq0 = (blockIdx.x / Hkv) * G;   // first sequence of the group
+  const int h = (blockIdx.x / n_blocks) % Hkv;
+  const int seq0 = (blockIdx.x / n_blocks / Hkv) * G;   // first sequence of the group
   const int n_keys = __ldcg(&full_pages[seq0]) * kPageTokens;
   const int n_tiles = n_keys / kPageTokens;
   const int32_t *pt = page_table + static_cast<size_t>(seq0) * pt_width;
@@ -938,12 +941,13 @@ attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bf
   const int n_pro = n_my < kDecStages ? n_my : kDecStages;
   for (int k = 0; k < n_pro; ++k) issue(k);
 
-  // ---- queries -> shared memory: row r = (sequence seq0 + r / REP, head h * REP + r % REP) ------
+  // ---- queries -> shared memory: row r = (sequence seq0 + (row0 + r) / REP, head h * REP + (row0 + r) % REP)
   for (int c = threadIdx.x; c < MT * 16 * CHUNKS; c += kDecWarps * 32) {
     const int r = c / CHUNKS, ch = c % CHUNKS;
+    const int gr = row0 + r;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (r < n_rows)
-      v = __ldcg(reinterpret_cast<const uint4 *>(q + (static_cast<size_t>(seq0 + r / REP) * Hq + h * REP + r % REP) * HD) +
+      v = __ldcg(reinterpret_cast<const uint4 *>(q + (static_cast<size_t>(seq0 + gr / REP) * Hq + h * REP + gr % REP) * HD) +
                  ch);
     *reinterpret_cast<uint4 *>(q_s + r * (HD * 2) + ((ch ^ (r & 7)) << 4)) = v;
   }
@@ -1104,7 +1108,7 @@ attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bf
         O += o_s[(w * ROWS + r) * S::kRowStride + d] * c;
       }
     }
-    const size_t rh = static_cast<size_t>(seq0 + r / REP) * Hq + h * REP + r % REP;
+    const size_t rh = static_cast<size_t>(seq0 + (row0 + r) / REP) * Hq + h * REP + (row0 + r) % REP;
     pre_o[rh * HD + d] = O;
     if (d == 0) pre_ml[rh] = make_float2(M, L);
   }
@@ -1143,9 +1147,11 @@ cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
   const int MT = (a.G * REP + 15) / 16;
   const float scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(HD));
   cudaError_t e;
-  if (MT == 2 && !attn_env_is("ECHO_ATTN_PREFIX", "tiles")) {
-    // the group's two 16-row tiles in one CTA: the launch fits the GPU at once
-    e = launch_early(attn_prefix_group_kernel<HD, 2>, dim3(a.P * a.Hkv), dim3(kDecWarps * 32), PreSmem<HD, 2>::kTotal, s,
+  if (MT >= 2 && !attn_env_is("ECHO_ATTN_PREFIX", "tiles")) {
+    // two 16-row tiles of a group's query rows per CTA: half the CTAs, and at 32 rows per group the
+    // launch fits the GPU at once
+    e = launch_early(attn_prefix_group_kernel<HD, 2>, dim3(a.P * a.Hkv * ((MT + 1) / 2)), dim3(kDecWarps * 32),
+                     PreSmem<HD, 2>::kTotal, s,
                      *a.tmKV, a.q, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.full_pages, a.layer_row0, a.Hq,
                      a.Hkv, a.G, a.n_pages, scale_log2, a.status);
   } else {

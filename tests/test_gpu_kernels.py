@@ -204,7 +204,8 @@ def test_gemm_swiglu_epilogue(B, M, F, K):
                                                      (2, 2, 16, 2, 128, 7, 1), (2, 8, 8, 8, 128, 64, 300),
                                                      (16, 8, 32, 8, 128, 64, 70), (20, 8, 16, 8, 128, 16, 2),
                                                      (40, 8, 8, 4, 64, 33, 150), (16, 8, 32, 8, 128, 512, 400),
-                                                     (3, 8, 8, 2, 64, 48, 20), (2, 6, 32, 8, 128, 100, 9)])
+                                                     (3, 8, 8, 2, 64, 48, 20), (2, 6, 32, 8, 128, 100, 9),
+                                                     (2, 8, 16, 2, 128, 64, 30), (2, 5, 16, 2, 128, 80, 3)])
 @pytest.mark.parametrize("suffix", ["resident", "waves", "tiles"])
 def test_decode_attention_matches_oracle(B, monkeypatch, suffix, P, G, Hq, Hkv, hd, Lp, steps):
     """Shared-prefix decode attention against the oracle's single-query attention (fp64) on the same
