@@ -281,7 +281,8 @@ int echo_sample_top_p(const float *logits, int32_t R, int32_t V, int32_t rows_pe
  *   full_pages  dev int32 [B]: leading pages shared by the whole group (same value for its G
  *               sequences; the shared pages are taken from the group's first sequence)
  *   scratch     dev, echo_decode_attention_scratch_bytes(B, Hq, hd) bytes, 256-byte aligned:
- *               the prefix partial results handed from the first kernel to the second
+ *               the prefix partial results handed from the first kernel to the second, a status
+ *               word and the item counter of the second kernel (cleared by the call itself)
  *   out         dev bf16 [B][Hq][hd]
  * hd must be 64 or 128, pages hold 16 tokens.  Synchronises the stream and returns
  * ECHO_ERR_DEVICE_CHECK if a page id was out of range. */
