@@ -71,6 +71,15 @@ typedef struct echo_config {
                                  by probability (ties: lower id first), the shortest prefix whose mass
                                  reaches top_p is kept, and the recorded log-probability is renormalised
                                  over it.  0 or 1: no truncation; otherwise in (0, 1). */
+  int32_t half_layers;        /* The paper states no precision for its rollout engine (Section 5.1 names the
+                                 model family only).  In the first half_layers layers every 16-bit operand
+                                 (projection inputs and the installed projection weights, queries, cached
+                                 keys and values, attention probabilities) is IEEE half (11-bit significand)
+                                 instead of bf16 (8-bit); accumulation, residual stream and softmax are fp32
+                                 everywhere.  Same bytes, same tensor-core rate.  bf16 weights convert to
+                                 half exactly unless |w| < 2^-17 (then the error is at most 2^-25) or
+                                 |w| > 65504 (refused by nothing: it would become inf).  Activations of these
+                                 layers must stay below 65504.  0: bf16 everywhere.  In [0, n_layers]. */
 } echo_config;
 
 /* One snapshot: a pointer per tensor, bf16, row-major [out, in]; each pointer
@@ -193,6 +202,13 @@ int echo_grpo_surrogate(const float *logp_new, const float *logp_old, const floa
                         const float *adv, const uint8_t *mask, int32_t n, int32_t T, float eps_clip,
                         float C, float *out, void *cuda_stream);
 
+/* Offset of this context's sequence ids in the noise streams: sequence (p, g) of later rollouts draws
+ * from the Philox stream of id base + p*G + g.  Rollout workers are independent and share nothing but
+ * the snapshot and the buffer (Section 4.1), so a set of prompts can be cut by prompt over several
+ * contexts or GPUs; with base = (index of the context's first prompt) * G every sequence gets the
+ * tokens it would get in one call over the whole set.  Default 0. */
+int echo_set_sequence_base(echo_ctx *ctx, uint32_t base);
+
 /* Block until everything this context enqueued (rollouts and installs) is done;
  * reports ECHO_ERR_DEVICE_CHECK / ECHO_ERR_TIMEOUT if a kernel flagged one. */
 int echo_sync(echo_ctx *ctx);
@@ -215,6 +231,24 @@ int echo_profile_read(echo_ctx *ctx, int32_t *steps, float *ms, int32_t capacity
  * the number of rows are returned through the pointers; `out` may be NULL to
  * query them.  n is the capacity of `out` in int32 elements. */
 int echo_debug_page_table(echo_ctx *ctx, int32_t *out, size_t n, int32_t *rows, int32_t *width);
+
+/* Parity hook: from now on, rollouts on this context copy the fp32 residual stream x as it enters
+ * layer `layer` and as it leaves it (the decoder layer of Section 5.1's model family: attention block
+ * and MLP block, each added to x) into caller buffers, so that a test can feed one layer's own input
+ * to a reference implementation of that layer and compare outputs without the error of the layers
+ * before it.  pre_in / pre_out: dev fp32 [n_prompt_tokens][d_model], rows in prefill order (prompt 0's
+ * tokens, then prompt 1's, ...).  dec_in / dec_out: dev fp32 [T-1][P*G][d_model], decode step j
+ * (the one that feeds token j-1) at index j-1.  Any pointer may be NULL.  layer = -1 turns it off.
+ * The buffers must stay valid while rollouts run; d_model must be a multiple of 4. */
+int echo_debug_capture(echo_ctx *ctx, int32_t layer, float *pre_in, float *pre_out, float *dec_in, float *dec_out);
+
+/* Wait-limit probe.  Every device-side wait of this library (TMA pipelines, accumulator hand-over) is
+ * bounded: when the limit runs out the kernel records it, drains and returns, and the host reports
+ * ECHO_ERR_TIMEOUT.  This call runs that wait routine alone, in a one-warp kernel, on a barrier that
+ * nothing ever signals, with the given limit (1 ns .. 0.1 s) in place of the library's one second:
+ * the expected result is ECHO_ERR_TIMEOUT, with the time the warp waited in *waited_ns (host, may be
+ * NULL).  scratch: dev, 16 bytes, 8-byte aligned.  Synchronises the stream. */
+int echo_debug_wait_limit(uint64_t limit_ns, void *scratch, uint64_t *waited_ns, void *cuda_stream);
 
 /* The KV page plan of a rollout, computed on the host without a context or a GPU (the same
  * routine echo_rollout uses).  prompt_lens host int32 [P].  Writes out_table (host int32
@@ -284,13 +318,16 @@ int echo_sample_top_p(const float *logits, int32_t R, int32_t V, int32_t rows_pe
  *               the prefix partial results handed from the first kernel to the second, a status
  *               word and the item counter of the second kernel (cleared by the call itself)
  *   out         dev bf16 [B][Hq][hd]
+ *   operand_format  0: q, kv_pool and out hold bf16 values; 1: IEEE half (echo_config.half_layers)
+ *   kernel_choice   0: the kernels a rollout uses; bit 0: one suffix CTA per (sequence, kv head) at every
+ *               length; bit 1: one prefix CTA per 16-row tile of a group's query rows
  * hd must be 64 or 128, pages hold 16 tokens.  Synchronises the stream and returns
  * ECHO_ERR_DEVICE_CHECK if a page id was out of range. */
 size_t echo_decode_attention_scratch_bytes(int32_t B, int32_t Hq, int32_t hd);
 int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, const int32_t *page_table,
                           int32_t pt_width, const int32_t *row_pos, const int32_t *full_pages, int32_t P,
                           int32_t G, int32_t Hq, int32_t Hkv, int32_t hd, void *scratch, size_t scratch_bytes,
-                          void *out, void *cuda_stream);
+                          void *out, int32_t operand_format, int32_t kernel_choice, void *cuda_stream);
 
 /* Dense projection alone, on the tcgen05 tensor cores with fp32 accumulation:
  *   epilogue 0:  Y[M][N] (dev fp32)  = X[M][K] (dev bf16) * W[N][K]^T (dev bf16)
@@ -308,7 +345,9 @@ int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, c
  * with s k-slices per tile added into Y in memory (s = 0: as many as give every SM pair a tile),
  * 1 = plain SIMT reference kernel (epilogues 0 and 1 only; needs no workspace).
  * Adding 1000 to `impl` says that W is not row-major but in the block-tiled layout that
- * echo_retile_weights writes (the layout echo_load_policy keeps the policy's matrices in). */
+ * echo_retile_weights writes (the layout echo_load_policy keeps the policy's matrices in).
+ * Adding 2000 says that X and W (and the output of epilogue 2) hold IEEE half values instead of
+ * bf16 (the operand format of echo_config.half_layers); the arithmetic is otherwise the same. */
 size_t echo_gemm_workspace_bytes(int32_t M);
 int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, int32_t K,
                    int32_t epilogue, int32_t impl, void *workspace, size_t workspace_bytes,

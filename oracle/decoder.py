@@ -189,6 +189,31 @@ def prefill(dims: ModelDims, w: Weights, prompt) -> (KVCache, np.ndarray):
 # modes B / C: whole-sequence causal forward
 # ----------------------------------------------------------------------------
 
+def layer_sequence(dims: ModelDims, lw: dict, x: np.ndarray) -> np.ndarray:
+    """One decoder layer over a whole sequence, causal: x [n, d] (row t = position t) -> x [n, d].
+    The attention block and the MLP block of the module docstring, each added to x."""
+    n = x.shape[0]
+    Hq, Hkv, hd = dims.n_q_heads, dims.n_kv_heads, dims.head_dim
+    rep = Hq // Hkv
+    pos = np.arange(n)
+    causal = np.tril(np.ones((n, n), dtype=bool))
+    h = rmsnorm(x, lw["attn_norm"], dims.rms_eps)
+    q = (h @ lw["wq"].T).reshape(n, Hq, hd)
+    k = (h @ lw["wk"].T).reshape(n, Hkv, hd)
+    v = (h @ lw["wv"].T).reshape(n, Hkv, hd)
+    q = rope(q, pos, dims.rope_theta)
+    k = rope(k, pos, dims.rope_theta)
+    o = np.empty((n, Hq, hd))
+    for a in range(Hq):
+        kv = a // rep
+        sc = q[:, a, :] @ k[:, kv, :].T / np.sqrt(hd)         # [n, n]
+        sc = np.where(causal, sc, -np.inf)
+        o[:, a, :] = softmax(sc, axis=-1) @ v[:, kv, :]
+    x = x + o.reshape(n, Hq * hd) @ lw["wo"].T
+    h2 = rmsnorm(x, lw["mlp_norm"], dims.rms_eps)
+    return x + (silu(h2 @ lw["w_gate"].T) * (h2 @ lw["w_up"].T)) @ lw["w_down"].T
+
+
 def forward_sequence(dims: ModelDims, w: Weights, tokens, want_from: int = 0,
                      layer_provider=None) -> np.ndarray:
     """Causal forward over a whole sequence; logits for positions >= want_from,
@@ -197,29 +222,10 @@ def forward_sequence(dims: ModelDims, w: Weights, tokens, want_from: int = 0,
     layer_provider, if given, is a callable l -> layer dict (fp64), used instead of
     w.layers so that a large model can be streamed one layer at a time."""
     tokens = np.asarray(tokens, dtype=np.int64)
-    n = len(tokens)
-    Hq, Hkv, hd = dims.n_q_heads, dims.n_kv_heads, dims.head_dim
-    rep = Hq // Hkv
-    pos = np.arange(n)
     x = w.embed[tokens].copy()                                    # [n, d]
-    causal = np.tril(np.ones((n, n), dtype=bool))
     for l in range(dims.n_layers):
         lw = layer_provider(l) if layer_provider is not None else w.layers[l]
-        h = rmsnorm(x, lw["attn_norm"], dims.rms_eps)
-        q = (h @ lw["wq"].T).reshape(n, Hq, hd)
-        k = (h @ lw["wk"].T).reshape(n, Hkv, hd)
-        v = (h @ lw["wv"].T).reshape(n, Hkv, hd)
-        q = rope(q, pos, dims.rope_theta)
-        k = rope(k, pos, dims.rope_theta)
-        o = np.empty((n, Hq, hd))
-        for a in range(Hq):
-            kv = a // rep
-            sc = q[:, a, :] @ k[:, kv, :].T / np.sqrt(hd)         # [n, n]
-            sc = np.where(causal, sc, -np.inf)
-            o[:, a, :] = softmax(sc, axis=-1) @ v[:, kv, :]
-        x = x + o.reshape(n, Hq * hd) @ lw["wo"].T
-        h2 = rmsnorm(x, lw["mlp_norm"], dims.rms_eps)
-        x = x + (silu(h2 @ lw["w_gate"].T) * (h2 @ lw["w_up"].T)) @ lw["w_down"].T
+        x = layer_sequence(dims, lw, x)
     xf = rmsnorm(x[want_from:], w.final_norm, dims.rms_eps)
     return xf @ w.lm_head.T
 

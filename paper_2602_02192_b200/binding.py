@@ -37,7 +37,7 @@ class EchoConfig(C.Structure):
         ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("kv_page_size", C.c_int32),
         ("max_prompts", C.c_int32), ("max_G", C.c_int32), ("max_prompt_len", C.c_int32),
         ("max_new_tokens", C.c_int32), ("n_weight_buffers", C.c_int32), ("eos_id", C.c_int32),
-        ("top_p", C.c_float),
+        ("top_p", C.c_float), ("half_layers", C.c_int32),
     ]
 
 
@@ -82,6 +82,11 @@ def _load() -> C.CDLL:
     lib.echo_debug_page_table.argtypes = [vp, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32)]
     lib.echo_plan_page_table.argtypes = [vp, i32, i32, i32, i32, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32)]
     lib.echo_plan_page_table.restype = C.c_int
+    lib.echo_set_sequence_base.argtypes = [vp, u32]
+    lib.echo_debug_capture.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.echo_debug_wait_limit.argtypes = [u64, vp, C.POINTER(u64), vp]
+    for name in ("echo_set_sequence_base", "echo_debug_capture", "echo_debug_wait_limit"):
+        getattr(lib, name).restype = C.c_int
     lib.echo_debug_noise.argtypes = [u64, u32, u32, u32, u32, vp, vp, vp]
     lib.echo_sample.argtypes = [vp, i32, i32, i32, vp, u32, f32, u64, vp, vp, vp, vp]
     lib.echo_sample_top_p.argtypes = [vp, i32, i32, i32, vp, u32, f32, f32, u64, vp, vp, vp, vp, vp]
@@ -97,7 +102,7 @@ def _load() -> C.CDLL:
     for name in ("echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible"):
         getattr(lib, name).restype = C.c_int
     lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]
-    lib.echo_decode_attention.argtypes = [vp, vp, i32, vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, vp]
+    lib.echo_decode_attention.argtypes = [vp, vp, i32, vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, i32, i32, vp]
     lib.echo_decode_attention.restype = C.c_int
     lib.echo_decode_attention_scratch_bytes.argtypes = [i32, i32, i32]
     lib.echo_decode_attention_scratch_bytes.restype = C.c_size_t
@@ -129,7 +134,8 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_decode_attention",
             "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error",
             "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate",
-            "echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible"]
+            "echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible",
+            "echo_set_sequence_base", "echo_debug_capture", "echo_debug_wait_limit"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -147,12 +153,13 @@ def _check(rc: int, ctx=None):
 
 def make_config(shape, max_prompts: int, max_G: int, max_prompt_len: int, max_new_tokens: int,
                 n_weight_buffers: int = 2, page_size: int = 16, eos_id: int = -1,
-                top_p: float = 1.0) -> EchoConfig:
+                top_p: float = 1.0, half_layers: int = 0) -> EchoConfig:
     """shape: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab,
     rms_eps, rope_theta attributes."""
     return EchoConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                       shape.d_ff, shape.vocab, shape.rms_eps, shape.rope_theta, page_size,
-                      max_prompts, max_G, max_prompt_len, max_new_tokens, n_weight_buffers, eos_id, top_p)
+                      max_prompts, max_G, max_prompt_len, max_new_tokens, n_weight_buffers, eos_id, top_p,
+                      min(int(half_layers), shape.n_layers))
 
 
 def echo_arena_bytes(cfg: EchoConfig) -> int:
@@ -284,6 +291,19 @@ class Engine:
                    self._ctx)
         return steps, ms
 
+    def echo_set_sequence_base(self, base: int):
+        _check(lib.echo_set_sequence_base(self._ctx, int(base)))
+
+    def echo_debug_capture(self, layer: int, pre_in=None, pre_out=None, dec_in=None, dec_out=None):
+        """fp32 cuda tensors (or None) that later rollouts fill with the residual stream around `layer`."""
+        ptrs = []
+        for t in (pre_in, pre_out, dec_in, dec_out):
+            if t is not None:
+                assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+            ptrs.append(t.data_ptr() if t is not None else None)
+        self._capture_keep = (pre_in, pre_out, dec_in, dec_out)
+        _check(lib.echo_debug_capture(self._ctx, int(layer), *ptrs))
+
     def echo_debug_page_table(self) -> np.ndarray:
         rows, width = C.c_int32(), C.c_int32()
         _check(lib.echo_debug_page_table(self._ctx, None, 0, C.byref(rows), C.byref(width)))
@@ -320,6 +340,14 @@ def echo_grpo_surrogate(logp_new: torch.Tensor, logp_old: torch.Tensor, logp_sam
                                        adv.data_ptr(), mask.data_ptr() if mask is not None else None, n, T,
                                        float(eps_clip), float(C_trunc), out.data_ptr(), _stream_ptr(None)))
     return out
+
+
+def echo_debug_wait_limit(limit_ns: int):
+    """Runs the library's bounded wait on a barrier nobody signals; returns (return code, ns waited)."""
+    waited = C.c_uint64(0)
+    scratch = torch.zeros(2, dtype=torch.int64, device="cuda")
+    rc = lib.echo_debug_wait_limit(int(limit_ns), scratch.data_ptr(), C.byref(waited), _stream_ptr(None))
+    return rc, int(waited.value)
 
 
 def echo_debug_noise(seed: int, s: int, j: int, v0: int, n: int, device="cuda"):
@@ -367,19 +395,21 @@ def echo_gemm_bf16(X: torch.Tensor, W: torch.Tensor, impl: int = 0, epilogue: in
                    Y: Optional[torch.Tensor] = None) -> torch.Tensor:
     """epilogue 0: Y = X W^T (fp32); 1: Y += X W^T (fp32, Y given); 2: W = [Wg; Wu], Y = silu(X Wg^T) * (X Wu^T)
     (bf16).  impl >= 1000: W is given row-major and handed to the kernels in the block-tiled layout."""
-    assert X.is_cuda and W.is_cuda and X.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
+    assert X.is_cuda and W.is_cuda and X.dtype == W.dtype and X.dtype in (torch.bfloat16, torch.float16)
     assert X.is_contiguous() and W.is_contiguous() and X.shape[1] == W.shape[1]
     M, K = X.shape
     N = W.shape[0] // 2 if epilogue == 2 else W.shape[0]
+    half = X.dtype == torch.float16          # IEEE half operands (impl + 2000)
     if impl >= 1000:
         W = (torch.cat([echo_retile_weights(W[:N].contiguous()), echo_retile_weights(W[N:].contiguous())])
              if epilogue == 2 else echo_retile_weights(W))
     if Y is None:
-        Y = torch.zeros((M, N), dtype=torch.bfloat16 if epilogue == 2 else torch.float32, device=X.device)
+        Y = torch.zeros((M, N), dtype=X.dtype if epilogue == 2 else torch.float32, device=X.device)
     with torch.cuda.device(X.device):
         nws = int(lib.echo_gemm_workspace_bytes(M)) if impl != 1 else 256
         ws = torch.empty(nws, dtype=torch.uint8, device=X.device)
-        _check(lib.echo_gemm_bf16(X.data_ptr(), W.data_ptr(), Y.data_ptr(), M, N, K, epilogue, impl,
+        _check(lib.echo_gemm_bf16(X.data_ptr(), W.data_ptr(), Y.data_ptr(), M, N, K, epilogue,
+                                  impl + (2000 if half else 0),
                                   ws.data_ptr(), nws, _stream_ptr(None)))
         torch.cuda.current_stream().synchronize()      # the workspace must outlive the kernel
     return Y
@@ -388,10 +418,10 @@ def echo_gemm_bf16(X: torch.Tensor, W: torch.Tensor, impl: int = 0, epilogue: in
 def echo_retile_weights(W: torch.Tensor) -> torch.Tensor:
     """Row-major bf16 matrix [rows][cols] -> the block-tiled layout (flat bf16 tensor) that echo_gemm_bf16
     reads with impl + 1000."""
-    assert W.is_cuda and W.dtype == torch.bfloat16 and W.is_contiguous() and W.dim() == 2
+    assert W.is_cuda and W.dtype in (torch.bfloat16, torch.float16) and W.is_contiguous() and W.dim() == 2
     rows, cols = W.shape
     n = int(lib.echo_tiled_weight_bytes(rows, cols))
-    out = torch.empty(n // 2, dtype=torch.bfloat16, device=W.device)
+    out = torch.empty(n // 2, dtype=W.dtype, device=W.device)
     with torch.cuda.device(W.device):
         _check(lib.echo_retile_weights(W.data_ptr(), rows, cols, out.data_ptr(), n, _stream_ptr(None)))
     return out
@@ -413,8 +443,10 @@ def echo_gemm_bf16_noalloc(X: torch.Tensor, W: torch.Tensor, Y: torch.Tensor, ep
 
 
 def echo_decode_attention(q: torch.Tensor, kv_pool: torch.Tensor, page_table: torch.Tensor, row_pos: torch.Tensor,
-                          full_pages: torch.Tensor, P: int, G: int) -> torch.Tensor:
-    """q bf16 [B][Hq][hd]; kv_pool bf16 [n_pages][Hkv][2][16][hd]; int32 device tensors for the tables."""
+                          full_pages: torch.Tensor, P: int, G: int, kernel_choice: int = 0) -> torch.Tensor:
+    """q [B][Hq][hd]; kv_pool [n_pages][Hkv][2][16][hd], both bf16 or both float16; int32 device tensors
+    for the tables."""
+    assert q.dtype == kv_pool.dtype and q.dtype in (torch.bfloat16, torch.float16)
     B, Hq, hd = q.shape
     n_pages, Hkv = kv_pool.shape[0], kv_pool.shape[1]
     assert B == P * G and q.is_contiguous() and kv_pool.is_contiguous() and page_table.is_contiguous()
@@ -425,7 +457,8 @@ def echo_decode_attention(q: torch.Tensor, kv_pool: torch.Tensor, page_table: to
         scratch = torch.empty(n, dtype=torch.uint8, device=q.device)
         _check(lib.echo_decode_attention(q.data_ptr(), kv_pool.data_ptr(), n_pages, page_table.data_ptr(),
                                          page_table.shape[1], row_pos.data_ptr(), full_pages.data_ptr(), P, G, Hq,
-                                         Hkv, hd, scratch.data_ptr(), n, out.data_ptr(), _stream_ptr(None)))
+                                         Hkv, hd, scratch.data_ptr(), n, out.data_ptr(),
+                                         1 if q.dtype == torch.float16 else 0, int(kernel_choice), _stream_ptr(None)))
     return out
 
 

@@ -22,8 +22,9 @@ template <int HD, int REP>
 __global__ void __launch_bounds__(kAttnWarps * 32)
 attention_rows_kernel(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer, __nv_bfloat16 *out,
                       const int32_t *row_pt, const int32_t *row_pos, const int32_t *page_table, int pt_width,
-                      int Hq, int Hkv, int page_size, int n_pages, float scale, int *status) {
+                      int Hq, int Hkv, int page_size, int n_pages, float scale, int *status, int half_io) {
   constexpr int EPL = HD / 32;                       // output dims per lane
+  const bool hf = half_io != 0;                      // q, K, V and the output are IEEE half, not bf16
   __shared__ float q_s[REP][HD];
   __shared__ float red_m[kAttnWarps][REP], red_l[kAttnWarps][REP];
   __shared__ float red_o[kAttnWarps][REP][HD];
@@ -36,7 +37,7 @@ attention_rows_kernel(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer, __n
 
   for (int i = threadIdx.x; i < REP * HD; i += blockDim.x) {
     const int a = i / HD, d = i % HD;
-    q_s[a][d] = __bfloat162float(q[(static_cast<size_t>(r) * Hq + kvh * REP + a) * HD + d]) * scale;
+    q_s[a][d] = widen16(reinterpret_cast<const uint16_t *>(q)[(static_cast<size_t>(r) * Hq + kvh * REP + a) * HD + d], hf) * scale;
   }
   __syncthreads();
 
@@ -70,10 +71,10 @@ attention_rows_kernel(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer, __n
 #pragma unroll
         for (int d0 = 0; d0 < HD; d0 += 8) {
           const uint4 raw = *reinterpret_cast<const uint4 *>(krow + d0);
-          const __nv_bfloat162 *k2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+          const uint32_t *k2 = reinterpret_cast<const uint32_t *>(&raw);
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const float2 kf = __bfloat1622float2(k2[i]);
+            const float2 kf = widen16x2(k2[i], hf);
 #pragma unroll
             for (int a = 0; a < REP; ++a) {
               sc[a] = fmaf(q_s[a][d0 + 2 * i], kf.x, sc[a]);
@@ -113,12 +114,10 @@ attention_rows_kernel(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer, __n
       float vf[EPL];
       if (EPL == 4) {
         const uint2 raw = *reinterpret_cast<const uint2 *>(vr);
-        const __nv_bfloat162 *v2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-        const float2 a0 = __bfloat1622float2(v2[0]), a1 = __bfloat1622float2(v2[1]);
+        const float2 a0 = widen16x2(raw.x, hf), a1 = widen16x2(raw.y, hf);
         vf[0] = a0.x; vf[1] = a0.y; vf[2 % EPL] = a1.x; vf[3 % EPL] = a1.y;
       } else {
-        const __nv_bfloat162 v2 = *reinterpret_cast<const __nv_bfloat162 *>(vr);
-        const float2 a0 = __bfloat1622float2(v2);
+        const float2 a0 = widen16x2(*reinterpret_cast<const uint32_t *>(vr), hf);
         vf[0] = a0.x; vf[1] = a0.y;
       }
 #pragma unroll
@@ -152,17 +151,18 @@ attention_rows_kernel(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer, __n
       ll += red_l[w][a] * c;
       acc += red_o[w][a][d] * c;
     }
-    out[(static_cast<size_t>(r) * Hq + kvh * REP + a) * HD + d] = __float2bfloat16(acc / ll);
+    reinterpret_cast<uint16_t *>(out)[(static_cast<size_t>(r) * Hq + kvh * REP + a) * HD + d] = cvt16(acc / ll, hf);
   }
 }
 
 template <int HD, int REP>
 cudaError_t launch_rows(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer, __nv_bfloat16 *out, RowMeta meta,
                         const int32_t *page_table, int pt_width, int R, int Hq, int Hkv, int page_size, int n_pages,
-                        int *status, cudaStream_t s) {
+                        int *status, cudaStream_t s, bool half_io) {
   const float scale = 1.0f / sqrtf(static_cast<float>(HD));
   attention_rows_kernel<HD, REP><<<dim3(R, Hkv), kAttnWarps * 32, 0, s>>>(
-      q, kv_layer, out, meta.row_pt, meta.row_pos, page_table, pt_width, Hq, Hkv, page_size, n_pages, scale, status);
+      q, kv_layer, out, meta.row_pt, meta.row_pos, page_table, pt_width, Hq, Hkv, page_size, n_pages, scale, status,
+      half_io ? 1 : 0);
   return cudaGetLastError();
 }
 
@@ -170,12 +170,12 @@ cudaError_t launch_rows(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer, _
 
 cudaError_t attention_rows_launch(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer, __nv_bfloat16 *out,
                                   RowMeta meta, const int32_t *page_table, int pt_width, int R, int Hq, int Hkv,
-                                  int hd, int page_size, int n_pages, int *status, cudaStream_t s) {
+                                  int hd, int page_size, int n_pages, int *status, cudaStream_t s, bool half_io) {
   const int rep = Hq / Hkv;
 #define ECHO_ATTN_CASE(HD_, REP_)                                                                              \
   if (hd == HD_ && rep == REP_)                                                                                \
     return launch_rows<HD_, REP_>(q, kv_layer, out, meta, page_table, pt_width, R, Hq, Hkv, page_size, n_pages, \
-                                  status, s);
+                                  status, s, half_io);
   ECHO_ATTN_CASE(64, 1) ECHO_ATTN_CASE(64, 2) ECHO_ATTN_CASE(64, 4)
   ECHO_ATTN_CASE(128, 1) ECHO_ATTN_CASE(128, 2) ECHO_ATTN_CASE(128, 4) ECHO_ATTN_CASE(128, 8)
 #undef ECHO_ATTN_CASE
@@ -224,15 +224,19 @@ struct DecSmem {
   static constexpr int kTotal = kBody + 256 + 1024;                            // barriers + alignment slack
 };
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t *>(&v);
+// 16-bit operands of the warp-level MMAs: bf16, or IEEE half in the layers configured that way
+template <bool HALF>
+__device__ __forceinline__ uint32_t pack_16(float lo, float hi) { return cvt16x2(lo, hi, HALF); }
+template <bool HALF>
+__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  if (HALF) mma_f16_16816(d, a, b0, b1);
+  else mma_bf16_16816(d, a, b0, b1);
 }
 
 // One 16-token page of one kv head against the warp's 16 query rows: S = Q K^T, online softmax
 // (exp2 domain), O += P V.  st = shared-memory address of the page (K burst then V burst, 128-byte
 // swizzle); key0 = index of the page's first key; keys at or beyond n_keys are masked.
-template <int HD>
+template <int HD, bool HALF>
 __device__ __forceinline__ void decode_tile(uint32_t st, int key0, int n_keys, float scale_log2, int lane,
                                             const uint32_t (&qf)[HD / 16][4], float (&o_acc)[HD / 8][4],
                                             float (&m_run)[2], float (&l_run)[2]) {
@@ -254,8 +258,8 @@ __device__ __forceinline__ void decode_tile(uint32_t st, int key0, int n_keys, f
       const uint32_t addr = st + (kk >> 2) * (S::kStageBytes / HALVES) + key * 128 + ((c ^ (key & 7)) << 4);
       uint32_t b0, b1, b2, b3;
       ldmatrix_x4(addr, b0, b1, b2, b3);
-      mma_bf16_16816(sc[0], qf[kk], b0, b1);
-      mma_bf16_16816(sc[1], qf[kk], b2, b3);
+      mma_16816<HALF>(sc[0], qf[kk], b0, b1);
+      mma_16816<HALF>(sc[1], qf[kk], b2, b3);
     }
   }
   // ---- online softmax (exp2 domain) ---------------------------------------------------------
@@ -297,10 +301,10 @@ __device__ __forceinline__ void decode_tile(uint32_t st, int key0, int n_keys, f
       o_acc[i][0] *= corr[0]; o_acc[i][1] *= corr[0];
       o_acc[i][2] *= corr[1]; o_acc[i][3] *= corr[1];
     }
-    pa[0] = pack_bf16(p[0][0], p[0][1]);
-    pa[1] = pack_bf16(p[0][2], p[0][3]);
-    pa[2] = pack_bf16(p[1][0], p[1][1]);
-    pa[3] = pack_bf16(p[1][2], p[1][3]);
+    pa[0] = pack_16<HALF>(p[0][0], p[0][1]);
+    pa[1] = pack_16<HALF>(p[0][2], p[0][3]);
+    pa[2] = pack_16<HALF>(p[1][0], p[1][1]);
+    pa[3] = pack_16<HALF>(p[1][2], p[1][3]);
   }
   // ---- O += P V ---------------------------------------------------------------------------
   {
@@ -313,13 +317,13 @@ __device__ __forceinline__ void decode_tile(uint32_t st, int key0, int n_keys, f
                             ((c ^ (key & 7)) << 4);
       uint32_t v0, v1, v2, v3;
       ldmatrix_x4_trans(addr, v0, v1, v2, v3);
-      mma_bf16_16816(o_acc[2 * dt], pa, v0, v1);
-      mma_bf16_16816(o_acc[2 * dt + 1], pa, v2, v3);
+      mma_16816<HALF>(o_acc[2 * dt], pa, v0, v1);
+      mma_16816<HALF>(o_acc[2 * dt + 1], pa, v2, v3);
     }
   }
 }
 
-template <int HD, bool PREFIX>
+template <int HD, bool PREFIX, bool HALF>
 __global__ void __launch_bounds__(kDecWarps * 32)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16 *__restrict__ q,
                    __nv_bfloat16 *__restrict__ out, float *__restrict__ pre_o, float2 *__restrict__ pre_ml,
@@ -350,8 +354,12 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
     griddep_launch();
   } else {
     griddep_launch();        // (the output projection may start prefetching its weights)
-    // a sequence that has ended (its end token was fed) is not attended: its row is not used
-    if (row_done && __ldcg(&row_done[blockIdx.x / Hkv])) return;
+    // a sequence that has ended (its end token was fed) is not attended: its row is not used.  The CTA
+    // still waits for the prefix launch, so that this grid never completes ahead of its predecessor.
+    if (row_done && __ldcg(&row_done[blockIdx.x / Hkv])) {
+      griddep_wait();
+      return;
+    }
   }
 
   // ---- which query rows and which keys this CTA handles ------------------------------------
@@ -455,7 +463,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
     if (!ok) break;
     const uint32_t st = smem_u32(my_stages + (k % kDecStages) * S::kStageBytes);
     const int key0 = (warp + kDecWarps * k) * kPageTokens;
-    decode_tile<HD>(st, key0, n_keys, scale_log2, lane, qf, o_acc, m_run, l_run);
+    decode_tile<HD, HALF>(st, key0, n_keys, scale_log2, lane, qf, o_acc, m_run, l_run);
     __syncwarp();
     if (k + kDecStages < n_my) issue(k + kDecStages);
   }
@@ -555,7 +563,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
       const float c_pre = ml.x == -INFINITY ? 0.f : exp2f(ml.x - Mt);
       const float Lt = L * c_suf + ml.y * c_pre;
       const float Ot = O * c_suf + (c_pre != 0.f ? po * c_pre : 0.f);
-      out[oi] = __float2bfloat16(Ot / Lt);
+      reinterpret_cast<uint16_t *>(out)[oi] = cvt16(Ot / Lt, HALF);
     }
   }
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, STATUS_WAIT_TIMEOUT);
@@ -583,7 +591,7 @@ struct SufSmem {
   static constexpr int total(int rep) { return 1024 + kPipeBytes + merge_bytes(rep) + 256; }
 };
 
-template <int HD>
+template <int HD, bool HALF>
 __global__ void __launch_bounds__(kDecWarps * 32)
 attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16 *__restrict__ q,
                             __nv_bfloat16 *__restrict__ out, const float *__restrict__ pre_o,
@@ -731,7 +739,8 @@ attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv
         ok = mbar_wait(&my_bars[g_cons % kDecStages], (g_cons / kDecStages) & 1, abort_flag);
         if (!ok) break;
         const uint32_t st = smem_u32(my_stages + (g_cons % kDecStages) * S::kStageBytes);
-        decode_tile<HD>(st, (warp + kDecWarps * k) * kPageTokens, c_keys, scale_log2, lane, qf, o_acc, m_run, l_run);
+        decode_tile<HD, HALF>(st, (warp + kDecWarps * k) * kPageTokens, c_keys, scale_log2, lane, qf, o_acc, m_run,
+                              l_run);
         __syncwarp();
         ++g_cons;
         if (k == 0) second_hop();
@@ -818,7 +827,8 @@ attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv
           const float c_pre = ml.x == -INFINITY ? 0.f : exp2f(ml.x - Mt);
           const float Lt = L * c_suf + ml.y * c_pre;
           const float Ot = O * c_suf + (c_pre != 0.f ? pre_val[i] * c_pre : 0.f);
-          out[(static_cast<size_t>(c_seq) * Hq + c_h * REP + r) * HD + d] = __float2bfloat16(Ot / Lt);
+          reinterpret_cast<uint16_t *>(out)[(static_cast<size_t>(c_seq) * Hq + c_h * REP + r) * HD + d] =
+              cvt16(Ot / Lt, HALF);
         }
       }
       __syncthreads();                       // the merge area is free for the next item
@@ -868,7 +878,7 @@ struct PreSmem {
   static constexpr int kTotal = kBody + 256 + 1024;
 };
 
-template <int HD, int MT>
+template <int HD, int MT, bool HALF>
 __global__ void __launch_bounds__(kDecWarps * 32)
 attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16 *__restrict__ q,
                          float *__restrict__ pre_o, float2 *__restrict__ pre_ml,
@@ -990,8 +1000,8 @@ attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bf
           uint32_t a[4];
           const int qc = 2 * kk + (id >> 1);
           ldmatrix_x4(q_addr + (t * 16 + q_row) * (HD * 2) + ((qc ^ (q_row & 7)) << 4), a[0], a[1], a[2], a[3]);
-          mma_bf16_16816(sc[t][0], a, b0, b1);
-          mma_bf16_16816(sc[t][1], a, b2, b3);
+          mma_16816<HALF>(sc[t][0], a, b0, b1);
+          mma_16816<HALF>(sc[t][1], a, b2, b3);
         }
       }
     }
@@ -1031,10 +1041,10 @@ attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bf
         o_acc[t][i][0] *= corr[0]; o_acc[t][i][1] *= corr[0];
         o_acc[t][i][2] *= corr[1]; o_acc[t][i][3] *= corr[1];
       }
-      pa[t][0] = pack_bf16(sc[t][0][0], sc[t][0][1]);
-      pa[t][1] = pack_bf16(sc[t][0][2], sc[t][0][3]);
-      pa[t][2] = pack_bf16(sc[t][1][0], sc[t][1][1]);
-      pa[t][3] = pack_bf16(sc[t][1][2], sc[t][1][3]);
+      pa[t][0] = pack_16<HALF>(sc[t][0][0], sc[t][0][1]);
+      pa[t][1] = pack_16<HALF>(sc[t][0][2], sc[t][0][3]);
+      pa[t][2] = pack_16<HALF>(sc[t][1][0], sc[t][1][1]);
+      pa[t][3] = pack_16<HALF>(sc[t][1][2], sc[t][1][3]);
     }
     // ---- O += P V ---------------------------------------------------------------------------
     {
@@ -1049,8 +1059,8 @@ attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bf
         ldmatrix_x4_trans(addr, v0, v1, v2, v3);
 #pragma unroll
         for (int t = 0; t < MT; ++t) {
-          mma_bf16_16816(o_acc[t][2 * dt], pa[t], v0, v1);
-          mma_bf16_16816(o_acc[t][2 * dt + 1], pa[t], v2, v3);
+          mma_16816<HALF>(o_acc[t][2 * dt], pa[t], v0, v1);
+          mma_16816<HALF>(o_acc[t][2 * dt + 1], pa[t], v2, v3);
         }
       }
     }
@@ -1115,86 +1125,80 @@ attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bf
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, STATUS_WAIT_TIMEOUT);
 }
 
-// Diagnostic switches, read at each launch (A/B runs and tests):
-// ECHO_ATTN_IMPL=waves     one suffix CTA per (sequence, kv head) at every length
-// ECHO_ATTN_PREFIX=tiles   one prefix CTA per 16-row tile of a group's query rows
-bool attn_env_is(const char *name, const char *value) {
-  const char *e = getenv(name);
-  return e && !strcmp(e, value);
-}
-bool suffix_resident() { return !attn_env_is("ECHO_ATTN_IMPL", "waves"); }
-
-// CTAs of `kernel` that fit the current device at once (per device and REP; no stream work).
-template <typename K>
-int resident_slots(K kernel, int smem_bytes, int rep) {
-  static int cache[64][17] = {};
+// CTAs of the resident suffix kernel that fit the current device at once (cached per device, head
+// dimension, operand format and group ratio; no stream work).
+template <int HD, bool HALF>
+int resident_slots(int smem_bytes, int rep) {
+  static int cache[64][17] = {};             // one table per (HD, HALF) instantiation
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || rep < 1 || rep > 16) return 0;
   if (cache[dev][rep] == 0) {
     int sms = 0, per_sm = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kDecWarps * 32, smem_bytes) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attn_suffix_resident_kernel<HD, HALF>, kDecWarps * 32,
+                                                      smem_bytes) != cudaSuccess)
       return 0;
     cache[dev][rep] = sms * per_sm;
   }
   return cache[dev][rep];
 }
 
-template <int HD>
+template <int HD, bool HALF>
 cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
   using S = DecSmem<HD>;
   const int REP = a.Hq / a.Hkv;
   const int MT = (a.G * REP + 15) / 16;
   const float scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(HD));
   cudaError_t e;
-  if (MT >= 2 && !attn_env_is("ECHO_ATTN_PREFIX", "tiles")) {
+  if (MT >= 2 && a.prefix_impl != 1) {
     // two 16-row tiles of a group's query rows per CTA: half the CTAs, and at 32 rows per group the
     // launch fits the GPU at once
-    e = launch_early(attn_prefix_group_kernel<HD, 2>, dim3(a.P * a.Hkv * ((MT + 1) / 2)), dim3(kDecWarps * 32),
+    e = launch_early(attn_prefix_group_kernel<HD, 2, HALF>, dim3(a.P * a.Hkv * ((MT + 1) / 2)), dim3(kDecWarps * 32),
                      PreSmem<HD, 2>::kTotal, s,
                      *a.tmKV, a.q, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.full_pages, a.layer_row0, a.Hq,
                      a.Hkv, a.G, a.n_pages, scale_log2, a.status);
   } else {
-    e = launch_early(attn_decode_kernel<HD, true>, dim3(a.P * a.Hkv * MT), dim3(kDecWarps * 32), S::kTotal, s,
+    e = launch_early(attn_decode_kernel<HD, true, HALF>, dim3(a.P * a.Hkv * MT), dim3(kDecWarps * 32), S::kTotal, s,
                      *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages,
                      a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
   }
   if (e != cudaSuccess) return e;
-  if (suffix_resident() && a.work && REP * HD <= 512) {   // merge area small enough for three CTAs per SM
+  if (a.suffix_impl != 1 && a.work && REP * HD <= 512) {   // merge area small enough for three CTAs per SM
     using R = SufSmem<HD>;
     const int n_items = a.P * a.G * a.Hkv;
-    const int slots = resident_slots(attn_suffix_resident_kernel<HD>, R::total(REP), REP);
+    const int slots = resident_slots<HD, HALF>(R::total(REP), REP);
     if (slots <= 0) return cudaErrorInvalidConfiguration;
-    return launch_early(attn_suffix_resident_kernel<HD>, dim3(n_items < slots ? n_items : slots), dim3(kDecWarps * 32),
-                        R::total(REP), s, *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos,
-                        a.full_pages, a.layer_row0, a.Hq, a.Hkv, n_items, a.n_pages, scale_log2, a.row_done, a.status,
-                        a.work);
+    return launch_early(attn_suffix_resident_kernel<HD, HALF>, dim3(n_items < slots ? n_items : slots),
+                        dim3(kDecWarps * 32), R::total(REP), s, *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table,
+                        a.pt_width, a.row_pos, a.full_pages, a.layer_row0, a.Hq, a.Hkv, n_items, a.n_pages, scale_log2,
+                        a.row_done, a.status, a.work);
   }
-  return launch_early(attn_decode_kernel<HD, false>, dim3(a.P * a.G * a.Hkv), dim3(kDecWarps * 32), S::kTotal, s,
+  return launch_early(attn_decode_kernel<HD, false, HALF>, dim3(a.P * a.G * a.Hkv), dim3(kDecWarps * 32), S::kTotal, s,
                       *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages,
                       a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
+}
+
+template <int HD, bool HALF>
+cudaError_t configure_decode() {
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(attn_decode_kernel<HD, true, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                DecSmem<HD>::kTotal)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(attn_decode_kernel<HD, false, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                DecSmem<HD>::kTotal)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(attn_prefix_group_kernel<HD, 2, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                PreSmem<HD, 2>::kTotal)) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_suffix_resident_kernel<HD, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              SufSmem<HD>::total(kSufPre * kDecWarps * 32 / HD));
 }
 
 }  // namespace
 
 cudaError_t attention_decode_configure() {
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(attn_decode_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                DecSmem<128>::kTotal)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(attn_decode_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                DecSmem<128>::kTotal)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(attn_prefix_group_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                PreSmem<128, 2>::kTotal)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(attn_prefix_group_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                PreSmem<64, 2>::kTotal)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(attn_suffix_resident_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                SufSmem<128>::total(kSufPre * kDecWarps * 32 / 128))) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(attn_suffix_resident_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                SufSmem<64>::total(kSufPre * kDecWarps * 32 / 64))) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(attn_decode_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                DecSmem<64>::kTotal)) != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_decode_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              DecSmem<64>::kTotal);
+  if ((e = configure_decode<128, false>()) != cudaSuccess) return e;
+  if ((e = configure_decode<128, true>()) != cudaSuccess) return e;
+  if ((e = configure_decode<64, false>()) != cudaSuccess) return e;
+  return configure_decode<64, true>();
 }
 
 bool attention_decode_supported(int hd, int page_size, int Hq, int Hkv) {
@@ -1203,8 +1207,8 @@ bool attention_decode_supported(int hd, int page_size, int Hq, int Hkv) {
 }
 
 cudaError_t attention_decode_launch(const DecodeAttnArgs &a, cudaStream_t s) {
-  if (a.hd == 128) return launch_decode<128>(a, s);
-  if (a.hd == 64) return launch_decode<64>(a, s);
+  if (a.hd == 128) return a.half_io ? launch_decode<128, true>(a, s) : launch_decode<128, false>(a, s);
+  if (a.hd == 64) return a.half_io ? launch_decode<64, true>(a, s) : launch_decode<64, false>(a, s);
   return cudaErrorInvalidValue;
 }
 

@@ -3,6 +3,7 @@
 
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -46,6 +47,26 @@ inline cudaError_t launch_early(void (*kernel)(KArgs...), dim3 grid, dim3 block,
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #ifdef __CUDACC__
+// fp32 -> the 16-bit operand format of a layer (bf16, or IEEE half), as raw bits, and back
+__device__ __forceinline__ uint16_t cvt16(float v, bool half) {
+  if (half) return __half_as_ushort(__float2half_rn(v));
+  return __bfloat16_as_ushort(__float2bfloat16(v));
+}
+__device__ __forceinline__ uint32_t cvt16x2(float lo, float hi, bool half) {
+  if (half) {
+    const __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+  }
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t *>(&v);
+}
+__device__ __forceinline__ float widen16(uint16_t bits, bool half) {
+  return half ? __half2float(__ushort_as_half(bits)) : __uint_as_float(static_cast<uint32_t>(bits) << 16);
+}
+__device__ __forceinline__ float2 widen16x2(uint32_t w, bool half) {
+  if (half) return __half22float2(*reinterpret_cast<const __half2 *>(&w));
+  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
 // order-preserving 32-bit key of a float: a < b  <=>  order_key(a) < order_key(b)
 __device__ __forceinline__ uint32_t order_key(float s) {
   const uint32_t u = __float_as_uint(s);
@@ -84,6 +105,7 @@ struct GemmArgs {
   int independent_splits;   // 1: k-slices add into Y in memory (Y must hold zeros for EPI_STORE; the order of
                             // the additions is not fixed); 0: slices are reduced in rank order inside a cluster
   int tiled;                // 1: W is stored block-tiled (see tiled_elems) and tmW is a map over that storage
+  int half_in = 0;          // 1: X and W hold IEEE half values instead of bf16 (and a SwiGLU output is half)
 };
 
 // ---- block-tiled weight storage -------------------------------------------------------------
@@ -101,8 +123,9 @@ __host__ __device__ inline size_t tiled_index(size_t n, size_t k, size_t col_blo
 }
 // Copies row-major src [rows][cols] (device memory, or host memory the device can read) into tiled
 // storage whose row 0 is dst_row0 rows into the matrix at dst; padding is not written.
+// to_half: the bf16 values are converted to IEEE half on the way (exact unless |w| < 2^-17 or > 65504).
 cudaError_t retile_launch(__nv_bfloat16 *dst, const __nv_bfloat16 *src, size_t rows, size_t cols, size_t dst_row0,
-                          cudaStream_t s);
+                          cudaStream_t s, bool to_half = false);
 // Tensor map over tiled storage of `rows` (padded to blocks) x `cols`: box = box_rows rows of one block.
 int make_tiled_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 size_t gemm_workspace_bytes(int bnb);
@@ -111,7 +134,7 @@ cudaError_t gemm_tc_configure();     // sets the dynamic shared memory attribute
 // part_rows > 0 with tiled storage: W consists of parts of part_rows rows, each starting on a block
 cudaError_t gemm_simt_launch(const __nv_bfloat16 *X, const __nv_bfloat16 *W, float *Y, int ldY,
                              int M, int N, int K, int accumulate, cudaStream_t stream, int tiled = 0,
-                             int part_rows = 0);
+                             int part_rows = 0, int half_in = 0);
 // Tensor map over a row-major bf16 matrix [rows][cols] (leading dimension ld elements),
 // 128-byte swizzle, box {64, box_rows}.
 int make_tensor_map(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
@@ -134,6 +157,7 @@ struct PairGemmArgs {
   int allow_early_start;
   int force_split;          // 0 = choose; k > 0 = k slices along K (linear epilogues only)
   int tiled;                // 1: W is block-tiled storage and tmW a map over it (make_tiled_map, 128-row box)
+  int half_in = 0;          // 1: X and W hold IEEE half values instead of bf16 (and a SwiGLU output is half)
 };
 cudaError_t gemm_pair_configure();
 bool gemm_pair_supported(const void *Y, int ldY, int M, int N, int K, int epilogue);
@@ -151,16 +175,17 @@ struct RowMeta {
 
 cudaError_t embed_launch(const __nv_bfloat16 *embed, const int32_t *tok_src, const int32_t *tok_idx,
                          float *x, int R, int d, int vocab, int *status, cudaStream_t s);
+// out_half: h is written as IEEE half instead of bf16 (the gain stays bf16)
 cudaError_t rmsnorm_launch(const float *x, const __nv_bfloat16 *gain, __nv_bfloat16 *h, int R, int d,
-                           float eps, cudaStream_t s);
+                           float eps, cudaStream_t s, bool out_half = false);
 cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double theta, cudaStream_t s);
 // qkv fp32 [R][(Hq+2Hkv)*hd] -> q bf16 [R][Hq*hd], K/V into the paged cache of one layer; the rows
 // of qkv it consumes are left holding zeros
 cudaError_t rope_append_launch(float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer,
                                const float2 *rope_table, RowMeta meta, const int32_t *page_table,
                                int pt_width, int R, int Hq, int Hkv, int hd, int page_size,
-                               int n_pages, int max_pos, int *status, cudaStream_t s);
-cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s);
+                               int n_pages, int max_pos, int *status, cudaStream_t s, bool out_half = false);
+cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s, bool out_half = false);
 cudaError_t gather_rows_launch(const float *x, const int32_t *src_rows, float *dst, int n, int d,
                                cudaStream_t s);
 cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page, const int32_t *dst_page,
@@ -174,7 +199,9 @@ cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit
                            const int32_t *seq_ids, const int32_t *d_step, uint32_t j_host,
                            float temperature, uint64_t seed, const int32_t *forced, int forced_stride,
                            int32_t *out_tok, float *out_lp, int out_stride, cudaStream_t s, int eos_id = -1,
-                           const uint2 *nucleus_cut = nullptr);   // per logits row, from nucleus_cut_launch
+                           const uint2 *nucleus_cut = nullptr,    // per logits row, from nucleus_cut_launch
+                           const int32_t *row_done = nullptr,     // per row: non-zero = the sequence has ended
+                           uint32_t seq_base = 0);                // added to every sequence id of the noise streams
 // Nucleus (top-p) cut of each logits row: cut[row] = (order-preserving key of the score of the last
 // nucleus member, its id; id 0x7fffffff = every id of that score).  nucleus.cu
 cudaError_t nucleus_cut_launch(const float *logits, int rows, int V, float temperature, float top_p, uint2 *cut,
@@ -186,13 +213,17 @@ cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float 
                                   const uint8_t *mask, int n, int T, float eps_clip, float C, float *out,
                                   cudaStream_t s);
 cudaError_t set_int_launch(int32_t *p, int32_t v, cudaStream_t s);
+// copies n floats (a multiple of 4) of x into slot (*d_step - 1) of dst
+cudaError_t capture_step_launch(const float *x, float *dst, const int32_t *d_step, size_t n, cudaStream_t s);
+// one warp waits limit_ns for a barrier nobody signals, then sets *status = STATUS_WAIT_TIMEOUT
+cudaError_t wait_probe_launch(uint64_t limit_ns, int *status, unsigned long long *waited_ns, cudaStream_t s);
 
 // ---- attention (attention.cu) ------------------------------------------------
 // One query row per activation row, keys 0..pos of its page-table row (causal by construction).
 cudaError_t attention_rows_launch(const __nv_bfloat16 *q, const __nv_bfloat16 *kv_layer,
                                   __nv_bfloat16 *out, RowMeta meta, const int32_t *page_table,
                                   int pt_width, int R, int Hq, int Hkv, int hd, int page_size,
-                                  int n_pages, int *status, cudaStream_t s);
+                                  int n_pages, int *status, cudaStream_t s, bool half_io = false);
 
 
 // Decode-step attention with the group's prompt prefix read once for all G samples.
@@ -213,6 +244,9 @@ struct DecodeAttnArgs {
   const int32_t *row_done;        // optional, per sequence: non-zero = ended, its suffix CTAs return at once
   int *work = nullptr;            // two zeroed ints: item counter of the resident suffix kernel, which leaves
                                   // them zero again (null: one suffix CTA per (sequence, kv head))
+  int half_io = 0;                // 1: q, the pool and out hold IEEE half values; probabilities are rounded to half
+  int suffix_impl = 0;            // 0: choose; 1: always one suffix CTA per (sequence, kv head)
+  int prefix_impl = 0;            // 0: choose; 1: always one prefix CTA per 16-row tile
 };
 cudaError_t attention_decode_configure();
 bool attention_decode_supported(int hd, int page_size, int Hq, int Hkv);

@@ -3,6 +3,7 @@
 // group advantage, and the small bookkeeping kernels a decode step needs.
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace echo {
 
@@ -65,7 +66,7 @@ constexpr int kNormThreads = 256;
 constexpr int kNormVecs = 8;          // float4 per thread held in registers (d <= 8192)
 __global__ void __launch_bounds__(kNormThreads)
 rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ gain, __nv_bfloat16 *__restrict__ h,
-               int R, int d, float eps) {
+               int R, int d, float eps, int out_half) {
   __shared__ float scratch[32];
   const int r = blockIdx.x;
   const float *xr = x + static_cast<size_t>(r) * d;
@@ -100,11 +101,9 @@ rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ ga
       if (idx < nv) {
         const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw[i].x));
         const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw[i].y));
-        __nv_bfloat162 o0 = __floats2bfloat162_rn(v[i].x * scale * g0.x, v[i].y * scale * g0.y);
-        __nv_bfloat162 o1 = __floats2bfloat162_rn(v[i].z * scale * g1.x, v[i].w * scale * g1.y);
         uint2 o;
-        o.x = *reinterpret_cast<uint32_t *>(&o0);
-        o.y = *reinterpret_cast<uint32_t *>(&o1);
+        o.x = cvt16x2(v[i].x * scale * g0.x, v[i].y * scale * g0.y, out_half != 0);
+        o.y = cvt16x2(v[i].z * scale * g1.x, v[i].w * scale * g1.y, out_half != 0);
         reinterpret_cast<uint2 *>(hr)[idx] = o;
       }
     }
@@ -118,7 +117,7 @@ rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ ga
   ss = block_sum(ss, scratch);
   const float scale = rsqrtf(ss / static_cast<float>(d) + eps);
   for (int i = threadIdx.x; i < d; i += blockDim.x)
-    hr[i] = __float2bfloat16(xr[i] * scale * __bfloat162float(gain[i]));
+    reinterpret_cast<uint16_t *>(hr)[i] = cvt16(xr[i] * scale * __bfloat162float(gain[i]), out_half != 0);
 }
 
 // table[pos][i] = (cos, sin)(pos * theta^(-2i/hd)), angles in fp64
@@ -137,8 +136,9 @@ __global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__res
                                    const int32_t *__restrict__ row_pt, const int32_t *__restrict__ row_pos,
                                    const int32_t *__restrict__ row_done, const int32_t *__restrict__ page_table,
                                    int pt_width, int R, int Hq, int Hkv, int hd, int page_size, int n_pages,
-                                   int max_pos, int *status) {
+                                   int max_pos, int *status, int out_half) {
   early_start_sync();
+  const bool oh = out_half != 0;
   const int r = blockIdx.x;
   const int pos = (row_done && row_done[r]) ? -1 : row_pos[r];      // an ended row is only cleared
   const int half = hd / 2;
@@ -163,9 +163,9 @@ __global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__res
     const int head = idx / half, i = idx % half;
     const float a = src[head * hd + i], b = src[head * hd + i + half];
     const float2 t = cs[i];
-    __nv_bfloat16 *dst = q + static_cast<size_t>(r) * Hq * hd + head * hd;
-    dst[i] = __float2bfloat16(a * t.x - b * t.y);
-    dst[i + half] = __float2bfloat16(b * t.x + a * t.y);
+    uint16_t *dst = reinterpret_cast<uint16_t *>(q) + static_cast<size_t>(r) * Hq * hd + head * hd;
+    dst[i] = cvt16(a * t.x - b * t.y, oh);
+    dst[i + half] = cvt16(b * t.x + a * t.y, oh);
   }
   // k heads (rotated) and v heads (plain) into the page slot
   const size_t page_elems = static_cast<size_t>(page_size) * hd;
@@ -175,13 +175,14 @@ __global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__res
     float *ks = src + (Hq + head) * hd;
     float *vs = src + (Hq + Hkv + head) * hd;
     const float2 t = cs[i];
-    __nv_bfloat16 *kd = kv_layer + ((static_cast<size_t>(page) * Hkv + head) * 2 + 0) * page_elems + off * hd;
-    __nv_bfloat16 *vd = kd + page_elems;
+    uint16_t *kd = reinterpret_cast<uint16_t *>(kv_layer) +
+                   ((static_cast<size_t>(page) * Hkv + head) * 2 + 0) * page_elems + off * hd;
+    uint16_t *vd = kd + page_elems;
     const float a = ks[i], b = ks[i + half];
-    kd[i] = __float2bfloat16(a * t.x - b * t.y);
-    kd[i + half] = __float2bfloat16(b * t.x + a * t.y);
-    vd[i] = __float2bfloat16(vs[i]);
-    vd[i + half] = __float2bfloat16(vs[i + half]);
+    kd[i] = cvt16(a * t.x - b * t.y, oh);
+    kd[i + half] = cvt16(b * t.x + a * t.y, oh);
+    vd[i] = cvt16(vs[i], oh);
+    vd[i + half] = cvt16(vs[i + half], oh);
   }
   // the row is consumed: leave zeros for the next projection, whose k-slices add into this buffer
   // (a separate pass, so that the loads above are not ordered behind stores to the same array)
@@ -198,20 +199,18 @@ __global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__res
 // rotation pairs of one head (for a kv head: of its key, plus the matching eight values), moved
 // with 16-byte loads and 8-byte stores.  Every qkv element is read by exactly one thread, which
 // zeroes it right after reading, so no second pass over the row is needed.
-__device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d) {
-  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-  uint2 o;
-  o.x = *reinterpret_cast<uint32_t *>(&lo);
-  o.y = *reinterpret_cast<uint32_t *>(&hi);
-  return o;
+__device__ __forceinline__ uint2 pack_16x4(float a, float b, float c, float d, bool half) {
+  return make_uint2(cvt16x2(a, b, half), cvt16x2(c, d, half));
 }
 __global__ void __launch_bounds__(256)
 rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ kv_layer,
                        const float2 *__restrict__ rope_table, const int32_t *__restrict__ row_pt,
                        const int32_t *__restrict__ row_pos, const int32_t *__restrict__ row_done,
                        const int32_t *__restrict__ page_table, int pt_width,
-                       int R, int Hq, int Hkv, int hd, int page_size, int n_pages, int max_pos, int *status) {
+                       int R, int Hq, int Hkv, int hd, int page_size, int n_pages, int max_pos, int *status,
+                       int out_half) {
   early_start_sync();
+  const bool oh = out_half != 0;
   const int r = blockIdx.x;
   const int half = hd / 2, q4 = half / 4;
   const int ld = (Hq + 2 * Hkv) * hd;
@@ -272,10 +271,10 @@ rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, _
       if (bad) continue;
       const float4 t01 = cs4[i / 2], t23 = cs4[i / 2 + 1];       // (cos, sin) of pairs i..i+3
       const float4 x = a[j], y = b[j];
-      const uint2 lo = pack_bf16x4(x.x * t01.x - y.x * t01.y, x.y * t01.z - y.y * t01.w, x.z * t23.x - y.z * t23.y,
-                                   x.w * t23.z - y.w * t23.w);
-      const uint2 hi = pack_bf16x4(y.x * t01.x + x.x * t01.y, y.y * t01.z + x.y * t01.w, y.z * t23.x + x.z * t23.y,
-                                   y.w * t23.z + x.w * t23.w);
+      const uint2 lo = pack_16x4(x.x * t01.x - y.x * t01.y, x.y * t01.z - y.y * t01.w, x.z * t23.x - y.z * t23.y,
+                                 x.w * t23.z - y.w * t23.w, oh);
+      const uint2 hi = pack_16x4(y.x * t01.x + x.x * t01.y, y.y * t01.z + x.y * t01.w, y.z * t23.x + x.z * t23.y,
+                                 y.w * t23.z + x.w * t23.w, oh);
       if (unit < Hq) {
         __nv_bfloat16 *dst = q + static_cast<size_t>(r) * Hq * hd + unit * hd + i;
         *reinterpret_cast<uint2 *>(dst) = lo;
@@ -286,19 +285,19 @@ rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, _
         *reinterpret_cast<uint2 *>(kd) = lo;
         *reinterpret_cast<uint2 *>(kd + half) = hi;
         __nv_bfloat16 *vd = kd + page_elems;
-        *reinterpret_cast<uint2 *>(vd) = pack_bf16x4(v0[j].x, v0[j].y, v0[j].z, v0[j].w);
-        *reinterpret_cast<uint2 *>(vd + half) = pack_bf16x4(v1[j].x, v1[j].y, v1[j].z, v1[j].w);
+        *reinterpret_cast<uint2 *>(vd) = pack_16x4(v0[j].x, v0[j].y, v0[j].z, v0[j].w, oh);
+        *reinterpret_cast<uint2 *>(vd + half) = pack_16x4(v1[j].x, v1[j].y, v1[j].z, v1[j].w, oh);
       }
     }
   }
 }
 
-__global__ void swiglu_kernel(const float *gu, __nv_bfloat16 *act, int R, int F) {
+__global__ void swiglu_kernel(const float *gu, __nv_bfloat16 *act, int R, int F, int out_half) {
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= static_cast<size_t>(R) * F) return;
   const size_t r = idx / F, f = idx % F;
   const float g = gu[r * 2 * F + f], u = gu[r * 2 * F + F + f];
-  act[idx] = __float2bfloat16(g / (1.0f + __expf(-g)) * u);
+  reinterpret_cast<uint16_t *>(act)[idx] = cvt16(g / (1.0f + __expf(-g)) * u, out_half != 0);
 }
 
 __global__ void gather_rows_kernel(const float *x, const int32_t *src_rows, float *dst, int n, int d) {
@@ -328,14 +327,42 @@ __global__ void decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int
     const int32_t tok = tok_hist[static_cast<size_t>(b) * T + (j - 1)];
     row_tok[b] = tok;
     row_pos[b] = seq_len0[b] + j - 1;
-    // a sequence that is fed its end token has ended: every later token is the end token too, so
-    // the row stays marked; its attention and cache writes are skipped from here on
-    if (row_done) row_done[b] = (eos_id >= 0 && tok == eos_id) ? 1 : 0;
+    // a sequence that is fed its end token has ended and stays ended whatever the token buffer holds
+    // at later positions (a given trajectory may be padded with other ids after its end token); its
+    // attention and cache writes are skipped from here on.  The flags are cleared when a rollout begins.
+    if (row_done && eos_id >= 0 && tok == eos_id) row_done[b] = 1;
   }
   if (threadIdx.x == 0) *d_step = j;
 }
 
 __global__ void set_int_kernel(int32_t *p, int32_t v) { *p = v; }
+
+// Parity hook: copies n floats of the residual stream into slot (*d_step - 1) of dst.
+__global__ void capture_step_kernel(const float *__restrict__ x, float *__restrict__ dst, const int32_t *d_step,
+                                    size_t n) {
+  const size_t slot = static_cast<size_t>(*d_step - 1);
+  const size_t i = (static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 4;
+  if (i < n) *reinterpret_cast<float4 *>(dst + slot * n + i) = *reinterpret_cast<const float4 *>(x + i);
+}
+
+// Wait-limit probe: one warp waits, with the given limit, for a barrier phase that nothing completes.
+// The wait gives up, the kernel records STATUS_WAIT_TIMEOUT and returns; nothing else depends on it.
+__global__ void wait_probe_kernel(uint64_t limit_ns, int *status, unsigned long long *waited_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar, 1);
+    abort_flag = 0;
+    ptx::mbar_fence_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint64_t t0 = ptx::global_timer_ns();
+    const bool ok = ptx::mbar_wait(&bar, 0, &abort_flag, limit_ns);
+    *waited_ns = ptx::global_timer_ns() - t0;
+    if (!ok) atomicExch(status, STATUS_WAIT_TIMEOUT);
+  }
+}
 
 // Clipped surrogate with truncated importance sampling, one warp per sequence (all in fp32):
 // J_i = sum_t m_t min(exp(lo - ls), C) min(rho A, clip(rho, 1 - e, 1 + e) A) / sum_t m_t, rho = exp(ln - lo).
@@ -406,18 +433,17 @@ __global__ void __launch_bounds__(kSamplerThreads)
 sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t *seq_ids, const int32_t *d_step,
                uint32_t j_host, float inv_temperature, uint32_t key0, uint32_t key1, const int32_t *forced,
                int forced_stride, int32_t *out_tok, float *out_lp, int out_stride, int eos_id,
-               const uint2 *nucleus_cut) {
+               const uint2 *nucleus_cut, const int32_t *row_done, uint32_t seq_base) {
   __shared__ float sm_m[32], sm_l[32], sm_score[32];
   __shared__ int sm_id[32];
   early_start_sync();
   const int r = blockIdx.x;
   const uint32_t j = d_step ? static_cast<uint32_t>(*d_step) : j_host;
-  if (eos_id >= 0 && j > 0) {
-    // End-of-sequence rule: the sequence is finished once its previous token (the forced one when
-    // scoring a given trajectory) is eos_id; finished positions hold eos_id with log-probability 0.
-    const size_t prev = forced ? static_cast<size_t>(r) * forced_stride + (j - 1)
-                               : static_cast<size_t>(r) * out_stride + (j - 1);
-    if ((forced ? forced[prev] : out_tok[prev]) == eos_id) {
+  if (eos_id >= 0 && j > 0 && row_done) {
+    // End-of-sequence rule: the sequence is finished once one of the tokens fed so far (the forced
+    // ones when scoring a given trajectory) was eos_id, which the step's preparation kernel records
+    // per row; finished positions hold eos_id with log-probability 0.
+    if (row_done[r]) {
       if (threadIdx.x == 0) {
         out_tok[static_cast<size_t>(r) * out_stride + j] = eos_id;
         out_lp[static_cast<size_t>(r) * out_stride + j] = 0.f;
@@ -425,7 +451,7 @@ sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t
       return;
     }
   }
-  const uint32_t s_id = seq_ids ? static_cast<uint32_t>(seq_ids[r]) : static_cast<uint32_t>(r);
+  const uint32_t s_id = seq_base + (seq_ids ? static_cast<uint32_t>(seq_ids[r]) : static_cast<uint32_t>(r));
   const float *z = logits + static_cast<size_t>(r / rows_per_logit_row) * V;
   const uint2 key = make_uint2(key0, key1);
   // top-p: only ids that rank at or before the row's cut (score descending, id ascending) belong to
@@ -553,8 +579,8 @@ cudaError_t embed_launch(const __nv_bfloat16 *embed, const int32_t *tok_src, con
   return launch_early(embed_kernel, dim3(R), dim3(256), 0, s, embed, tok_src, tok_idx, x, R, d, vocab, status);
 }
 cudaError_t rmsnorm_launch(const float *x, const __nv_bfloat16 *gain, __nv_bfloat16 *h, int R, int d, float eps,
-                           cudaStream_t s) {
-  return launch_early(rmsnorm_kernel, dim3(R), dim3(kNormThreads), 0, s, x, gain, h, R, d, eps);
+                           cudaStream_t s, bool out_half) {
+  return launch_early(rmsnorm_kernel, dim3(R), dim3(kNormThreads), 0, s, x, gain, h, R, d, eps, out_half ? 1 : 0);
 }
 cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double theta, cudaStream_t s) {
   const int half = head_dim / 2, n = max_pos * half;
@@ -563,16 +589,18 @@ cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double t
 }
 cudaError_t rope_append_launch(float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer, const float2 *rope_table,
                                RowMeta meta, const int32_t *page_table, int pt_width, int R, int Hq, int Hkv, int hd,
-                               int page_size, int n_pages, int max_pos, int *status, cudaStream_t s) {
+                               int page_size, int n_pages, int max_pos, int *status, cudaStream_t s, bool out_half) {
   if (hd % 8 == 0 && (reinterpret_cast<uintptr_t>(qkv) & 15) == 0)
     return launch_early(rope_append_vec_kernel, dim3(R), dim3(256), 0, s, qkv, q, kv_layer, rope_table, meta.row_pt,
-                        meta.row_pos, meta.row_done, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
+                        meta.row_pos, meta.row_done, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos,
+                        status, out_half ? 1 : 0);
   return launch_early(rope_append_kernel, dim3(R), dim3(256), 0, s, qkv, q, kv_layer, rope_table, meta.row_pt,
-                      meta.row_pos, meta.row_done, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos, status);
+                      meta.row_pos, meta.row_done, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos,
+                      status, out_half ? 1 : 0);
 }
-cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s) {
+cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s, bool out_half) {
   const size_t n = static_cast<size_t>(R) * F;
-  swiglu_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(gu, act, R, F);
+  swiglu_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(gu, act, R, F, out_half ? 1 : 0);
   return cudaGetLastError();
 }
 cudaError_t gather_rows_launch(const float *x, const int32_t *src_rows, float *dst, int n, int d, cudaStream_t s) {
@@ -595,11 +623,12 @@ cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, 
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row, const int32_t *seq_ids,
                            const int32_t *d_step, uint32_t j_host, float temperature, uint64_t seed,
                            const int32_t *forced, int forced_stride, int32_t *out_tok, float *out_lp, int out_stride,
-                           cudaStream_t s, int eos_id, const uint2 *nucleus_cut) {
+                           cudaStream_t s, int eos_id, const uint2 *nucleus_cut, const int32_t *row_done,
+                           uint32_t seq_base) {
   return launch_early(sampler_kernel, dim3(R), dim3(kSamplerThreads), 0, s, logits, V, rows_per_logit_row, seq_ids,
                       d_step, j_host, 1.0f / temperature, static_cast<uint32_t>(seed & 0xffffffffu),
                       static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok, out_lp, out_stride, eos_id,
-                      nucleus_cut);
+                      nucleus_cut, row_done, seq_base);
 }
 cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n, uint32_t *words,
                                float *uniform, cudaStream_t s) {
@@ -619,6 +648,16 @@ cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float 
                                   cudaStream_t s) {
   if (n == 0) return cudaSuccess;
   grpo_surrogate_kernel<<<(n + 7) / 8, 256, 0, s>>>(ln, lo, ls, adv, mask, n, T, eps_clip, C, out);
+  return cudaGetLastError();
+}
+cudaError_t capture_step_launch(const float *x, float *dst, const int32_t *d_step, size_t n, cudaStream_t s) {
+  if (n == 0) return cudaSuccess;
+  if (n % 4) return cudaErrorInvalidValue;
+  capture_step_kernel<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, s>>>(x, dst, d_step, n);
+  return cudaGetLastError();
+}
+cudaError_t wait_probe_launch(uint64_t limit_ns, int *status, unsigned long long *waited_ns, cudaStream_t s) {
+  wait_probe_kernel<<<1, 32, 0, s>>>(limit_ns, status, waited_ns);
   return cudaGetLastError();
 }
 cudaError_t set_int_launch(int32_t *p, int32_t v, cudaStream_t s) {

@@ -122,9 +122,9 @@ __device__ __forceinline__ void load_stage(const CUtensorMap *tmW, const CUtenso
 }
 
 template <int BNB>
-__device__ __forceinline__ void mma_stage(uint32_t tmem_base, uint32_t stage_addr, bool first) {
+__device__ __forceinline__ void mma_stage(uint32_t tmem_base, uint32_t stage_addr, bool first, bool half_in) {
   using S = GemmSmem<BNB>;
-  constexpr uint32_t idesc = instr_desc_bf16(BNB);
+  const uint32_t idesc = idesc_operands(instr_desc_bf16(BNB), half_in);
   const uint64_t xdesc = smem_desc_sw128(stage_addr + S::kWBytes);
 #pragma unroll
   for (int a = 0; a < kAcc; ++a) {
@@ -144,7 +144,7 @@ template <int BNB>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, void *Yv,
                     int ldY, int M, int N, int K, int epilogue, int n_tiles, float *workspace, int *counters,
-                    int tiled, int *status) {
+                    int tiled, int half_in, int *status) {
   using S = GemmSmem<BNB>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -227,7 +227,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           ok = mbar_wait(&full_bar[s], (it / S::kStages) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          mma_stage<BNB>(tmem_base, smem_u32(smem + s * S::kStageBytes), kb == 0);
+          mma_stage<BNB>(tmem_base, smem_u32(smem + s * S::kStageBytes), kb == 0, half_in != 0);
           tc_commit(&empty_bar[s]);      // frees the stage once these MMAs have read it
         }
         if (ok) tc_commit(acc_full);
@@ -312,7 +312,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         for (int a = 0; a < kAcc; ++a) {
           if (gu) {
             // thread -> feature f of the 64-wide block and every second column of a 32-column chunk
-            __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(Yv);
+            uint16_t *Y = reinterpret_cast<uint16_t *>(Yv);
             const int f = et & 63, half = et >> 6;
             const int n = (nt * kAcc + a) * 64 + f;
 #pragma unroll 1
@@ -334,7 +334,7 @@ gemm_streamk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                   const int c = c0 + half + 2 * i;
-                  if (c < cols) Y[static_cast<size_t>(m0 + c) * ldY + n] = __float2bfloat16(silu_f(gs[i]) * us[i]);
+                  if (c < cols) Y[static_cast<size_t>(m0 + c) * ldY + n] = cvt16(silu_f(gs[i]) * us[i], half_in != 0);
                 }
               }
             }
@@ -411,7 +411,7 @@ template <int BNB>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                     const __grid_constant__ CUtensorMap tmY, int M, int N, int K, int epilogue, int S_split,
-                    int independent, int tiled, int *status) {
+                    int independent, int tiled, int half_in, int *status) {
   using S = GemmSmem<BNB>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -480,7 +480,7 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         ok = mbar_wait(&full_bar[s], (it / S::kStages) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        mma_stage<BNB>(tmem_base, smem_u32(smem + s * S::kStageBytes), it == 0);
+        mma_stage<BNB>(tmem_base, smem_u32(smem + s * S::kStageBytes), it == 0, half_in != 0);
         tc_commit(&empty_bar[s]);
       }
       if (ok) tc_commit(acc_full);
@@ -568,12 +568,12 @@ gemm_cluster_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                 }
               }
             }
-            __nv_bfloat162 *o = reinterpret_cast<__nv_bfloat162 *>(out_stage);   // [column - c_lo][64]
+            uint32_t *o = reinterpret_cast<uint32_t *>(out_stage);               // [column - c_lo][64] 16-bit
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const int c = cb + j * kEpiWarps;
               if (c < c_hi)
-                o[(c - c_lo) * 32 + lane] = __floats2bfloat162_rn(silu_f(gs[j].x) * us[j].x, silu_f(gs[j].y) * us[j].y);
+                o[(c - c_lo) * 32 + lane] = cvt16x2(silu_f(gs[j].x) * us[j].x, silu_f(gs[j].y) * us[j].y, half_in != 0);
             }
           } else {
             float4 acc[4];
@@ -675,7 +675,7 @@ cudaError_t launch_cluster_variant(const GemmArgs &a, int n_tiles, int m_tiles, 
   const bool gu = a.epilogue == EPI_SWIGLU;
   if (make_out_map(&tmY, a.Y, a.M, a.N, a.ldY, gu) != 0) return cudaErrorInvalidValue;
   return cudaLaunchKernelEx(&cfg, gemm_cluster_kernel<BNB>, *a.tmW, *a.tmX, tmY, a.M, a.N, a.K, a.epilogue, split,
-                            independent ? 1 : 0, a.tiled, a.status);
+                            independent ? 1 : 0, a.tiled, a.half_in, a.status);
 }
 
 template <int BNB>
@@ -707,10 +707,11 @@ cudaError_t launch_variant(const GemmArgs &a, cudaStream_t stream) {
   if (grid > total) grid = static_cast<int>(total);
   if (a.allow_early_start)
     return launch_early(gemm_streamk_kernel<BNB>, dim3(grid), dim3(kThreads), S::kTotal, stream, *a.tmW, *a.tmX, a.Y,
-                        a.ldY, a.M, a.N, a.K, a.epilogue, n_tiles, a.workspace, a.counters, a.tiled, a.status);
+                        a.ldY, a.M, a.N, a.K, a.epilogue, n_tiles, a.workspace, a.counters, a.tiled, a.half_in,
+                        a.status);
   gemm_streamk_kernel<BNB><<<grid, kThreads, S::kTotal, stream>>>(*a.tmW, *a.tmX, a.Y, a.ldY, a.M, a.N, a.K,
                                                                  a.epilogue, n_tiles, a.workspace, a.counters,
-                                                                 a.tiled, a.status);
+                                                                 a.tiled, a.half_in, a.status);
   return cudaGetLastError();
 }
 
@@ -725,7 +726,8 @@ cudaError_t configure_variant() {
 
 // ---- plain SIMT reference kernel (debugging aid; never on the default path) ----
 __global__ void gemm_simt_kernel(const __nv_bfloat16 *X, const __nv_bfloat16 *W, float *Y, int ldY, int M, int N,
-                                 int K, int accumulate, int tiled, int part_rows) {
+                                 int K, int accumulate, int tiled, int part_rows, int half_in) {
+  const uint16_t *X16 = reinterpret_cast<const uint16_t *>(X), *W16 = reinterpret_cast<const uint16_t *>(W);
   __shared__ float xs[16][17], ws[16][17];
   const int tx = threadIdx.x, ty = threadIdx.y;
   const int m = blockIdx.y * 16 + ty, n = blockIdx.x * 16 + tx;
@@ -734,7 +736,7 @@ __global__ void gemm_simt_kernel(const __nv_bfloat16 *X, const __nv_bfloat16 *W,
   float acc = 0.f;
   for (int k0 = 0; k0 < K; k0 += 16) {
     const int xm = blockIdx.y * 16 + ty, xk = k0 + tx;
-    xs[ty][tx] = (xm < M && xk < K) ? __bfloat162float(X[static_cast<size_t>(xm) * K + xk]) : 0.f;
+    xs[ty][tx] = (xm < M && xk < K) ? widen16(X16[static_cast<size_t>(xm) * K + xk], half_in != 0) : 0.f;
     const int wn = blockIdx.x * 16 + ty;
     float wv = 0.f;
     if (wn < N && xk < K) {
@@ -743,7 +745,7 @@ __global__ void gemm_simt_kernel(const __nv_bfloat16 *X, const __nv_bfloat16 *W,
         const size_t row = part_rows > 0 ? (wn / part_rows) * part_blocks * kTileRows + wn % part_rows : wn;
         idx = tiled_index(row, xk, KB);
       }
-      wv = __bfloat162float(W[idx]);
+      wv = widen16(W16[idx], half_in != 0);
     }
     ws[ty][tx] = wv;
     __syncthreads();
@@ -759,13 +761,19 @@ __global__ void gemm_simt_kernel(const __nv_bfloat16 *X, const __nv_bfloat16 *W,
 
 // Row-major -> block-tiled copy: one CTA per 128 x 64 source tile, 16-byte pieces.
 __global__ void __launch_bounds__(256)
-retile_kernel(__nv_bfloat16 *dst, const __nv_bfloat16 *src, size_t rows, size_t cols, size_t dst_row0) {
+retile_kernel(__nv_bfloat16 *dst, const __nv_bfloat16 *src, size_t rows, size_t cols, size_t dst_row0, int to_half) {
   const size_t KB = (cols + kTileCols - 1) / kTileCols;
   const size_t n0 = static_cast<size_t>(blockIdx.y) * kTileRows, k0 = static_cast<size_t>(blockIdx.x) * kTileCols;
   for (int i = threadIdx.x; i < kTileRows * (kTileCols / 8); i += blockDim.x) {
     const size_t n = n0 + i / (kTileCols / 8), k = k0 + (i % (kTileCols / 8)) * 8;
     if (n < rows && k < cols) {
-      const uint4 v = *reinterpret_cast<const uint4 *>(src + n * cols + k);
+      uint4 v = *reinterpret_cast<const uint4 *>(src + n * cols + k);
+      if (to_half) {
+        uint32_t *w2 = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          w2[j] = cvt16x2(__uint_as_float(w2[j] << 16), __uint_as_float(w2[j] & 0xffff0000u), true);
+      }
       *reinterpret_cast<uint4 *>(dst + tiled_index(dst_row0 + n, k, KB)) = v;
     }
   }
@@ -865,20 +873,21 @@ cudaError_t gemm_tc_launch(const GemmArgs &a, cudaStream_t stream) {
 }
 
 cudaError_t gemm_simt_launch(const __nv_bfloat16 *X, const __nv_bfloat16 *W, float *Y, int ldY, int M, int N,
-                             int K, int accumulate, cudaStream_t stream, int tiled, int part_rows) {
+                             int K, int accumulate, cudaStream_t stream, int tiled, int part_rows, int half_in) {
   dim3 grid((N + 15) / 16, (M + 15) / 16), block(16, 16);
-  gemm_simt_kernel<<<grid, block, 0, stream>>>(X, W, Y, ldY, M, N, K, accumulate, tiled, part_rows);
+  gemm_simt_kernel<<<grid, block, 0, stream>>>(X, W, Y, ldY, M, N, K, accumulate, tiled, part_rows, half_in);
   return cudaGetLastError();
 }
 
 cudaError_t retile_launch(__nv_bfloat16 *dst, const __nv_bfloat16 *src, size_t rows, size_t cols, size_t dst_row0,
-                          cudaStream_t s) {
+                          cudaStream_t s, bool to_half) {
   if (rows == 0 || cols == 0) return cudaSuccess;
   if (cols % 8 || (reinterpret_cast<uintptr_t>(src) & 15) || (reinterpret_cast<uintptr_t>(dst) & 15))
     return cudaErrorInvalidValue;
   const size_t gx = (cols + kTileCols - 1) / kTileCols, gy = (rows + kTileRows - 1) / kTileRows;
   if (gy > 65535 || gx > 0x7fffffff) return cudaErrorInvalidValue;
-  retile_kernel<<<dim3(static_cast<unsigned>(gx), static_cast<unsigned>(gy)), 256, 0, s>>>(dst, src, rows, cols, dst_row0);
+  retile_kernel<<<dim3(static_cast<unsigned>(gx), static_cast<unsigned>(gy)), 256, 0, s>>>(dst, src, rows, cols, dst_row0,
+                                                                                           to_half ? 1 : 0);
   return cudaGetLastError();
 }
 

@@ -117,7 +117,7 @@ template <int BNB, int ACC>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                  const __grid_constant__ CUtensorMap tmY, int M, int N, int K, int epilogue, int split,
-                 int tiled, int *status) {
+                 int tiled, int half_in, int *status) {
   using S = PairSmem<BNB, ACC>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -205,7 +205,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     }
   } else if (warp == 1) {
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = instr_desc_pair(BNB);
+      const uint32_t idesc = idesc_operands(instr_desc_pair(BNB), half_in != 0);
       bool ok = true;
       for (int it = 0; it < kb_len; ++it) {
         const int s = it % S::kStages;
@@ -251,7 +251,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
           }
         }
       } else {
-        __nv_bfloat16 *stage = reinterpret_cast<__nv_bfloat16 *>(smem);   // [feature half][column][64]
+        uint16_t *stage = reinterpret_cast<uint16_t *>(smem);             // [feature half][column][64]
         const int h = row >> 6, fl = row & 63;
 #pragma unroll
         for (int j = 0; j < CH / 32; ++j) {
@@ -264,7 +264,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
 #pragma unroll
             for (int c = 0; c < 32; ++c)
               stage[(h * BNB + c0 + c) * 64 + fl] =
-                  __float2bfloat16(silu_pair(__uint_as_float(g[c])) * __uint_as_float(u[c]));
+                  cvt16(silu_pair(__uint_as_float(g[c])) * __uint_as_float(u[c]), half_in != 0);
           }
         }
       }
@@ -331,7 +331,7 @@ cudaError_t launch_pair(const PairGemmArgs &a, int n_tiles, int m_tiles, int spl
   cfg.attrs = attr;
   cfg.numAttrs = a.allow_early_start ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<BNB, ACC>, *a.tmW, tmX, tmY, a.M, a.N, a.K, a.epilogue, split,
-                            a.tiled, a.status);
+                            a.tiled, a.half_in, a.status);
 }
 
 template <int BNB, int ACC>

@@ -57,6 +57,7 @@ bool config_ok(const echo_config *c) {
   if (c->eos_id < -1 || c->eos_id >= c->vocab) return false;
   if (!(c->top_p >= 0.f) || c->top_p > 1.f) return false;
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return false;
+  if (c->half_layers < 0 || c->half_layers > c->n_layers) return false;
   if (static_cast<long long>(c->max_prompts) * c->max_G > (1 << 20)) return false;
   return true;
 }
@@ -182,6 +183,13 @@ struct echo_ctx {
   int64_t launches = 0;
   bool use_simt = false, use_graph = true, fast_decode = false, deterministic = false, use_pdl = true, use_pair = true;
   bool long_suffix = false;   // decode steps whose sequences hold many generated tokens (see kLongSuffix)
+  int attn_suffix_impl = 0, attn_prefix_impl = 0;   // diagnostic kernel choices (ECHO_ATTN_IMPL / ECHO_ATTN_PREFIX)
+  uint32_t seq_base = 0;      // added to p * G + g in the noise streams (echo_set_sequence_base)
+  // parity hook (echo_debug_capture): residual stream before / after one layer
+  int cap_layer = -1;
+  float *cap_pre_in = nullptr, *cap_pre_out = nullptr, *cap_dec_in = nullptr, *cap_dec_out = nullptr;
+  int cap_row0 = 0;           // first prefill row of the chunk being run
+  bool cap_decode = false;    // the forward being enqueued is a decode step
   CUtensorMap tm_kv;
   std::string last_error;
   // sampled per-kernel timing (echo_profile_config / echo_profile_read)
@@ -272,13 +280,14 @@ int pick_bnb(int rows) {
 
 // Y = X * W^T through the tensor-core kernel (or the SIMT reference when selected).
 int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, const __nv_bfloat16 *X, void *Y, int ldY,
-             int M, int N, int K, int epilogue, bool y_holds_zeros = false, const CUtensorMap *tmW_pair = nullptr) {
+             int M, int N, int K, int epilogue, bool y_holds_zeros = false, const CUtensorMap *tmW_pair = nullptr,
+             bool half_in = false) {
   ProfScope prof(ctx, PROF_GEMM);
   if (ctx->use_pair && !ctx->use_simt && !ctx->deterministic && (epilogue != EPI_SWIGLU || tmW_pair) &&
       gemm_pair_supported(Y, ldY, M, N, K, epilogue)) {
     // more than 64 rows: 2-CTA MMAs, k-slices added into Y in memory
     PairGemmArgs a{tmW_pair ? tmW_pair : tmW, X, Y, ldY, M, N, K, epilogue, ctx->ptr<int>(ctx->lo.status),
-                   ctx->use_pdl ? 1 : 0, 0, 1};
+                   ctx->use_pdl ? 1 : 0, 0, 1, half_in ? 1 : 0};
     if (epilogue == EPI_STORE && !y_holds_zeros && gemm_pair_split(M, N, K, epilogue, 0) > 1) {
       CK(cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * ldY * sizeof(float), ctx->stream));
       a.allow_early_start = 0;
@@ -289,12 +298,12 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
   if (ctx->use_simt) {
     if (epilogue == EPI_SWIGLU) {
       float *gu = ctx->ptr<float>(ctx->lo.gu);
-      LAUNCH(gemm_simt_launch(X, W, gu, 2 * N, M, 2 * N, K, 0, ctx->stream, 1, N));
-      LAUNCH(swiglu_launch(gu, reinterpret_cast<__nv_bfloat16 *>(Y), M, N, ctx->stream));
+      LAUNCH(gemm_simt_launch(X, W, gu, 2 * N, M, 2 * N, K, 0, ctx->stream, 1, N, half_in ? 1 : 0));
+      LAUNCH(swiglu_launch(gu, reinterpret_cast<__nv_bfloat16 *>(Y), M, N, ctx->stream, half_in));
       return ECHO_OK;
     }
     LAUNCH(gemm_simt_launch(X, W, reinterpret_cast<float *>(Y), ldY, M, N, K, epilogue == EPI_ACCUM, ctx->stream, 1,
-                            0));
+                            0, half_in ? 1 : 0));
     return ECHO_OK;
   }
   CUtensorMap tmX;
@@ -305,7 +314,7 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
   }
   GemmArgs a{tmW, &tmX, Y, ldY, M, N, K, bnb, epilogue, ctx->ptr<int>(ctx->lo.status),
              ctx->ptr<float>(ctx->lo.gemm_ws), ctx->ptr<int>(ctx->lo.gemm_counters), kMaxCtas, 0, ctx->use_pdl ? 1 : 0,
-             ctx->deterministic ? 0 : 1, 1};
+             ctx->deterministic ? 0 : 1, 1, half_in ? 1 : 0};
   if (a.independent_splits && epilogue == EPI_STORE && N < 8 * 4096 && !y_holds_zeros) {
     // the k-slices add into Y: it must start at zero.  The memset is the GEMM's predecessor on the
     // stream, so this launch does not use the early start.
@@ -337,29 +346,44 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int d
   const float2 *rope = ctx->ptr<float2>(lo.rope);
   for (int l = 0; l < D.L; ++l) {
     __nv_bfloat16 *kv_layer = ctx->ptr<__nv_bfloat16>(lo.kv) + static_cast<size_t>(l) * lo.kv_layer_elems;
-    LAUNCH(rmsnorm_launch(x, w.attn_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream));
+    // the 16-bit operands of this layer (projection inputs and weights, q, cached K/V, probabilities)
+    // are IEEE half instead of bf16
+    const bool hf = l < ctx->cfg.half_layers;
+    auto capture = [&](float *pre, float *dec) -> cudaError_t {
+      const size_t n = static_cast<size_t>(R) * D.d;
+      if (ctx->cap_decode)
+        return dec ? capture_step_launch(x, dec, ctx->ptr<int32_t>(lo.d_step), n, ctx->stream) : cudaSuccess;
+      return pre ? cudaMemcpyAsync(pre + static_cast<size_t>(ctx->cap_row0) * D.d, x, n * 4, cudaMemcpyDeviceToDevice,
+                                   ctx->stream)
+                 : cudaSuccess;
+    };
+    if (l == ctx->cap_layer) CK(capture(ctx->cap_pre_in, ctx->cap_dec_in));
+    LAUNCH(rmsnorm_launch(x, w.attn_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream, hf));
     // the qkv buffer holds zeros here: rope_append clears every row it consumes
-    TRY(run_gemm(ctx, &w.tm_qkv[l], w.wqkv[l], h, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE, !ctx->use_simt));
+    TRY(run_gemm(ctx, &w.tm_qkv[l], w.wqkv[l], h, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE, !ctx->use_simt, nullptr,
+                 hf));
     LAUNCH(rope_append_launch(qkv, q, kv_layer, rope, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
-                              ctx->M.n_pages, ctx->M.max_pos, status, ctx->stream));
+                              ctx->M.n_pages, ctx->M.max_pos, status, ctx->stream, hf));
     if (decode_P > 0 && ctx->fast_decode) {
       ProfScope prof(ctx, PROF_ATTN);
       DecodeAttnArgs da{&ctx->tm_kv, q, attn, ctx->ptr<float>(lo.pre_o), ctx->ptr<float2>(lo.pre_ml), pt,
                         ctx->M.pt_width, meta.row_pos, ctx->ptr<int32_t>(lo.full_pages),
                         static_cast<int>(static_cast<size_t>(l) * (lo.kv_layer_elems / D.hd)), decode_P, decode_G,
                         D.Hq, D.Hkv, D.hd, ctx->M.n_pages, status, meta.row_done,
-                        ctx->long_suffix ? nullptr : ctx->ptr<int>(lo.attn_work)};
+                        ctx->long_suffix ? nullptr : ctx->ptr<int>(lo.attn_work), hf ? 1 : 0, ctx->attn_suffix_impl,
+                        ctx->attn_prefix_impl};
       LAUNCH(attention_decode_launch(da, ctx->stream));
       ctx->launches++;                      // two kernels per call
     } else {
       ProfScope prof(ctx, PROF_ATTN);
       LAUNCH(attention_rows_launch(q, kv_layer, attn, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
-                                   ctx->M.n_pages, status, ctx->stream));
+                                   ctx->M.n_pages, status, ctx->stream, hf));
     }
-    TRY(run_gemm(ctx, &w.tm_o[l], w.wo[l], attn, x, D.d, R, D.d, D.Hq * D.hd, EPI_ACCUM));
-    LAUNCH(rmsnorm_launch(x, w.mlp_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream));
-    TRY(run_gemm(ctx, &w.tm_gu[l], w.wgu[l], h, act, D.F, R, D.F, D.d, EPI_SWIGLU, false, &w.tm_gu_pair[l]));
-    TRY(run_gemm(ctx, &w.tm_down[l], w.wdown[l], act, x, D.d, R, D.d, D.F, EPI_ACCUM));
+    TRY(run_gemm(ctx, &w.tm_o[l], w.wo[l], attn, x, D.d, R, D.d, D.Hq * D.hd, EPI_ACCUM, false, nullptr, hf));
+    LAUNCH(rmsnorm_launch(x, w.mlp_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream, hf));
+    TRY(run_gemm(ctx, &w.tm_gu[l], w.wgu[l], h, act, D.F, R, D.F, D.d, EPI_SWIGLU, false, &w.tm_gu_pair[l], hf));
+    TRY(run_gemm(ctx, &w.tm_down[l], w.wdown[l], act, x, D.d, R, D.d, D.F, EPI_ACCUM, false, nullptr, hf));
+    if (l == ctx->cap_layer) CK(capture(ctx->cap_pre_out, ctx->cap_dec_out));
   }
   return ECHO_OK;
 }
@@ -577,7 +601,10 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
   LAUNCH(embed_launch(w.embed, row_tok, nullptr, ctx->ptr<float>(lo.x), pl.B, ctx->D.d, ctx->D.V,
                       ctx->ptr<int>(lo.status), ctx->stream));
   RowMeta meta{ctx->ptr<int32_t>(lo.dec_row_pt), row_pos, row_done};
-  TRY(forward_layers(ctx, w, pl.B, meta, pl.P, pl.G));
+  ctx->cap_decode = true;
+  const int rc_layers = forward_layers(ctx, w, pl.B, meta, pl.P, pl.G);
+  ctx->cap_decode = false;
+  TRY(rc_layers);
   TRY(lm_head(ctx, w, ctx->ptr<float>(lo.x), pl.B));
   {
     ProfScope prof(ctx, PROF_SAMPLER);
@@ -588,7 +615,8 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
       cut = ctx->ptr<uint2>(lo.nucleus_cut);
     }
     LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, ctx->D.V, 1, nullptr, d_step, 0, temperature, seed,
-                          forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream, ctx->cfg.eos_id, cut));
+                          forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream, ctx->cfg.eos_id, cut, row_done,
+                          ctx->seq_base));
   }
   return ECHO_OK;
 }
@@ -625,12 +653,15 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   int *status = ctx->ptr<int>(lo.status);
 
   CK(cudaEventRecord(ctx->ev_begin, ctx->stream));
+  if (ctx->cfg.eos_id >= 0)       // no sequence has ended yet
+    CK(cudaMemsetAsync(ctx->arena + lo.row_done, 0, static_cast<size_t>(pl.B) * 4, ctx->stream));
   // ---- prefill: once per prompt, in chunks of kChunkRows tokens -------------
   for (int c = 0; c < pl.n_chunks; ++c) {
     const int r0 = c * kChunkRows, R = std::min(kChunkRows, pl.n_tok - r0);
     LAUNCH(embed_launch(w.embed, prompts, ctx->ptr<int32_t>(lo.pre_tok_idx) + r0, x, R, D.d, D.V, status,
                         ctx->stream));
     RowMeta meta{ctx->ptr<int32_t>(lo.pre_row_pt) + r0, ctx->ptr<int32_t>(lo.pre_row_pos) + r0, nullptr};
+    ctx->cap_row0 = r0;
     TRY(forward_layers(ctx, w, R, meta));
     LAUNCH(gather_rows_launch(x, ctx->ptr<int32_t>(lo.gather_map) + static_cast<size_t>(c) * P,
                               ctx->ptr<float>(lo.xlast), P, D.d, ctx->stream));
@@ -650,7 +681,7 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
     cut0 = ctx->ptr<uint2>(lo.nucleus_cut);
   }
   LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, D.V, G, nullptr, nullptr, 0, temperature, seed, forced, T,
-                        out_tokens, out_logprobs, T, ctx->stream, ctx->cfg.eos_id, cut0));
+                        out_tokens, out_logprobs, T, ctx->stream, ctx->cfg.eos_id, cut0, nullptr, ctx->seq_base));
 
   CK(cudaEventRecord(ctx->ev_first, ctx->stream));
   // ---- decode steps 1..T-1 ----------------------------------------------------
@@ -816,6 +847,9 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
     return bail(e, "cudaMemset(kv)");
   {
     const char *na = getenv("ECHO_ATTN_IMPL");
+    const char *np = getenv("ECHO_ATTN_PREFIX");
+    ctx->attn_suffix_impl = na && !strcmp(na, "waves") ? 1 : 0;
+    ctx->attn_prefix_impl = np && !strcmp(np, "tiles") ? 1 : 0;
     const size_t kv_rows = lo.kv_layer_elems / ctx->D.hd * ctx->D.L;
     if (!(na && !strcmp(na, "rows")) && kv_rows < (1ull << 31) &&
         attention_decode_supported(ctx->D.hd, ctx->D.Z, ctx->D.Hq, ctx->D.Hkv)) {
@@ -905,14 +939,15 @@ int echo_load_policy(echo_ctx *ctx, const echo_weights *src, int64_t version) {
   // kernel reads the source in place when the device can address it (device memory, page-locked
   // or managed host memory); a snapshot in pageable host memory goes through a bounce buffer.
   __nv_bfloat16 *stage = ctx->ptr<__nv_bfloat16>(ctx->lo.retile_stage);
-  auto tile = [&](__nv_bfloat16 *dst, const void *s, size_t rows, size_t cols, size_t row0) -> cudaError_t {
+  auto tile = [&](__nv_bfloat16 *dst, const void *s, size_t rows, size_t cols, size_t row0,
+                  bool to_half) -> cudaError_t {
     cudaPointerAttributes at;
     const __nv_bfloat16 *dev_src = nullptr;
     if (cudaPointerGetAttributes(&at, s) == cudaSuccess && at.type != cudaMemoryTypeUnregistered && at.devicePointer)
       dev_src = static_cast<const __nv_bfloat16 *>(at.devicePointer);
     else
       (void)cudaGetLastError();
-    if (dev_src) return retile_launch(dst, dev_src, rows, cols, row0, cs);
+    if (dev_src) return retile_launch(dst, dev_src, rows, cols, row0, cs, to_half);
     const size_t chunk = kRetileStageBytes / (cols * 2);
     if (chunk == 0) return cudaErrorInvalidValue;
     for (size_t r = 0; r < rows; r += chunk) {
@@ -920,22 +955,23 @@ int echo_load_policy(echo_ctx *ctx, const echo_weights *src, int64_t version) {
       cudaError_t e = cudaMemcpyAsync(stage, static_cast<const __nv_bfloat16 *>(s) + r * cols, n * cols * 2,
                                       cudaMemcpyDefault, cs);
       if (e != cudaSuccess) return e;
-      if ((e = retile_launch(dst, stage, n, cols, row0 + r, cs)) != cudaSuccess) return e;
+      if ((e = retile_launch(dst, stage, n, cols, row0 + r, cs, to_half)) != cudaSuccess) return e;
     }
     return cudaSuccess;
   };
   const size_t d = D.d, qd = static_cast<size_t>(D.Hq) * D.hd, kd = static_cast<size_t>(D.Hkv) * D.hd;
   CK(cp(w.embed, src->embed, static_cast<size_t>(D.V) * d));
-  CK(tile(w.lm_head, src->lm_head, D.V, d, 0));
+  CK(tile(w.lm_head, src->lm_head, D.V, d, 0, false));
   CK(cp(w.final_norm, src->final_norm, d));
   for (int l = 0; l < D.L; ++l) {
-    CK(tile(w.wqkv[l], src->wq[l], qd, d, 0));
-    CK(tile(w.wqkv[l], src->wk[l], kd, d, qd));
-    CK(tile(w.wqkv[l], src->wv[l], kd, d, qd + kd));
-    CK(tile(w.wo[l], src->wo[l], d, qd, 0));
-    CK(tile(w.wgu[l], src->w_gate[l], D.F, d, 0));
-    CK(tile(w.wgu[l] + tiled_elems(D.F, d), src->w_up[l], D.F, d, 0));
-    CK(tile(w.wdown[l], src->w_down[l], d, D.F, 0));
+    const bool hf = l < ctx->cfg.half_layers;      // this layer's matrices are kept as IEEE half
+    CK(tile(w.wqkv[l], src->wq[l], qd, d, 0, hf));
+    CK(tile(w.wqkv[l], src->wk[l], kd, d, qd, hf));
+    CK(tile(w.wqkv[l], src->wv[l], kd, d, qd + kd, hf));
+    CK(tile(w.wo[l], src->wo[l], d, qd, 0, hf));
+    CK(tile(w.wgu[l], src->w_gate[l], D.F, d, 0, hf));
+    CK(tile(w.wgu[l] + tiled_elems(D.F, d), src->w_up[l], D.F, d, 0, hf));
+    CK(tile(w.wdown[l], src->w_down[l], d, D.F, 0, hf));
     CK(cp(w.attn_norm[l], src->attn_norm[l], d));
     CK(cp(w.mlp_norm[l], src->mlp_norm[l], d));
   }
@@ -1131,7 +1167,8 @@ size_t echo_decode_attention_scratch_bytes(int32_t B, int32_t Hq, int32_t hd) {
 int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, const int32_t *page_table,
                           int32_t pt_width, const int32_t *row_pos, const int32_t *full_pages, int32_t P, int32_t G,
                           int32_t Hq, int32_t Hkv, int32_t hd, void *scratch, size_t scratch_bytes, void *out,
-                          void *cuda_stream) {
+                          int32_t operand_format, int32_t kernel_choice, void *cuda_stream) {
+  if (operand_format < 0 || operand_format > 1 || kernel_choice < 0 || kernel_choice > 3) return ECHO_ERR_INVALID;
   if (!q || !kv_pool || !page_table || !row_pos || !full_pages || !scratch || !out) return ECHO_ERR_INVALID;
   if (P < 1 || G < 1 || n_pages < 1 || pt_width < 1 || Hkv < 1 || Hq % Hkv) return ECHO_ERR_INVALID;
   if (!attention_decode_supported(hd, 16, Hq, Hkv)) return ECHO_ERR_UNSUPPORTED;
@@ -1151,7 +1188,7 @@ int echo_decode_attention(const void *q, const void *kv_pool, int32_t n_pages, c
   if (cudaMemsetAsync(status, 0, 16, s) != cudaSuccess) return ECHO_ERR_CUDA;     // status word + item counters
   DecodeAttnArgs da{&tm, static_cast<const __nv_bfloat16 *>(q), static_cast<__nv_bfloat16 *>(out), pre_o, pre_ml,
                     page_table, pt_width, row_pos, full_pages, 0, P, G, Hq, Hkv, hd, n_pages, status, nullptr,
-                    status + 2};
+                    status + 2, operand_format, kernel_choice & 1, (kernel_choice >> 1) & 1};
   if (attention_decode_launch(da, s) != cudaSuccess) return ECHO_ERR_CUDA;
   int st = 0;
   if (cudaMemcpyAsync(&st, status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ECHO_ERR_CUDA;
@@ -1171,12 +1208,14 @@ int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, 
   if (!X || !W || !Y || M < 1 || M > 4096 || N < 1 || K < 8 || (K % 8)) return ECHO_ERR_INVALID;
   if (epilogue != EPI_STORE && epilogue != EPI_ACCUM && epilogue != EPI_SWIGLU) return ECHO_ERR_INVALID;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const int half_in = impl >= 2000 ? 1 : 0;        // X and W hold IEEE half values
+  if (half_in) impl -= 2000;
   const int tiled = impl >= 1000 ? 1 : 0;          // W is block-tiled storage (echo_retile_weights)
   if (tiled) impl -= 1000;
   if (impl == 1) {
     if (epilogue == EPI_SWIGLU) return ECHO_ERR_INVALID;
     cudaError_t e = gemm_simt_launch(static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(W),
-                                     static_cast<float *>(Y), N, M, N, K, epilogue == EPI_ACCUM, s, tiled, 0);
+                                     static_cast<float *>(Y), N, M, N, K, epilogue == EPI_ACCUM, s, tiled, 0, half_in);
     return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
   }
   // tiled storage of a gate/up pair: two parts of N rows, each padded to whole blocks
@@ -1193,7 +1232,7 @@ int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, 
     if (!gemm_pair_supported(Y, N, M, N, K, epilogue)) return ECHO_ERR_UNSUPPORTED;
     CUtensorMap tmW2;
     if (w_map(&tmW2, kGemmTileN) != 0) return ECHO_ERR_CUDA;
-    PairGemmArgs pa{&tmW2, X, Y, N, M, N, K, epilogue, nullptr, 0, impl - 300, tiled};
+    PairGemmArgs pa{&tmW2, X, Y, N, M, N, K, epilogue, nullptr, 0, impl - 300, tiled, half_in};
     if (epilogue == EPI_STORE && gemm_pair_split(M, N, K, epilogue, impl - 300) > 1 &&
         cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * N * sizeof(float), s) != cudaSuccess)
       return ECHO_ERR_CUDA;
@@ -1217,7 +1256,7 @@ int echo_gemm_bf16(const void *X, const void *W, void *Y, int32_t M, int32_t N, 
       cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * N * sizeof(float), s) != cudaSuccess)
     return ECHO_ERR_CUDA;
   GemmArgs a{&tmW, &tmX, Y, N, M, N, K, bnb, epilogue, nullptr, static_cast<float *>(workspace), counters, 0, split, 0,
-             indep ? 1 : 0, tiled};
+             indep ? 1 : 0, tiled, half_in};
   cudaError_t e = gemm_tc_launch(a, s);
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }
@@ -1236,6 +1275,39 @@ int echo_retile_weights(const void *src, int64_t rows, int64_t cols, void *dst, 
   cudaError_t e = retile_launch(static_cast<__nv_bfloat16 *>(dst), static_cast<const __nv_bfloat16 *>(src),
                                 static_cast<size_t>(rows), static_cast<size_t>(cols), 0, s);
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+int echo_set_sequence_base(echo_ctx *ctx, uint32_t base) {
+  if (!ctx) return ECHO_ERR_INVALID;
+  ctx->seq_base = base;
+  return ECHO_OK;
+}
+
+int echo_debug_capture(echo_ctx *ctx, int32_t layer, float *pre_in, float *pre_out, float *dec_in, float *dec_out) {
+  if (!ctx || layer < -1 || layer >= ctx->D.L) return ECHO_ERR_INVALID;
+  if (ctx->D.d % 4) return ECHO_ERR_UNSUPPORTED;
+  ctx->cap_layer = layer;
+  ctx->cap_pre_in = pre_in;
+  ctx->cap_pre_out = pre_out;
+  ctx->cap_dec_in = dec_in;
+  ctx->cap_dec_out = dec_out;
+  return ECHO_OK;
+}
+
+int echo_debug_wait_limit(uint64_t limit_ns, void *scratch, uint64_t *waited_ns, void *cuda_stream) {
+  if (limit_ns == 0 || limit_ns > 100000000ull || !scratch || (reinterpret_cast<uintptr_t>(scratch) & 7))
+    return ECHO_ERR_INVALID;                                                    // at most 0.1 s
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  struct Probe { int status; int pad; unsigned long long waited; };
+  Probe *d = static_cast<Probe *>(scratch);
+  Probe h{};
+  if (cudaMemsetAsync(d, 0, sizeof(Probe), s) != cudaSuccess ||
+      wait_probe_launch(limit_ns, &d->status, &d->waited, s) != cudaSuccess ||
+      cudaMemcpyAsync(&h, d, sizeof(Probe), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return ECHO_ERR_CUDA;
+  if (waited_ns) *waited_ns = h.waited;
+  return h.status == STATUS_WAIT_TIMEOUT ? ECHO_ERR_TIMEOUT : ECHO_OK;
 }
 
 int echo_profile_config(echo_ctx *ctx, int32_t every_n_steps) {
