@@ -378,9 +378,14 @@ int echo_retile_weights(const void *src, int64_t rows, int64_t cols, void *dst, 
  *     attributes; make that first call with the device current and before any stream capture.
  *   - All calls share the one array.  The call clears the part that must start at zero, but
  *     two calls whose kernels can overlap on the GPU (different streams or host threads) race
- *     on it: keep calls on one stream, or order them with events. */
+ *     on it: keep calls on one stream, or order them with events.
+ *   - X, W and Y must be 16-byte aligned (else ECHO_ERR_INVALID).
+ * The call returns after enqueueing.  echo_gemm_bf16_noalloc_status waits for the stream and reports
+ * how the most recent call on the current device ended: ECHO_OK, or ECHO_ERR_TIMEOUT if one of its
+ * kernel's bounded waits ran out (Y is then incomplete).  It allocates nothing either. */
 int echo_gemm_bf16_noalloc(const void *X, const void *W, void *Y, int32_t M, int32_t N, int32_t K,
                            int32_t epilogue, void *cuda_stream);
+int echo_gemm_bf16_noalloc_status(void *cuda_stream);
 
 const char *echo_strerror(int code);
 const char *echo_last_error(echo_ctx *ctx);   /* text of the last ECHO_ERR_CUDA on this context */

@@ -108,6 +108,8 @@ def _load() -> C.CDLL:
     lib.echo_decode_attention_scratch_bytes.restype = C.c_size_t
     lib.echo_gemm_bf16_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
     lib.echo_gemm_bf16_noalloc.restype = C.c_int
+    lib.echo_gemm_bf16_noalloc_status.argtypes = [vp]
+    lib.echo_gemm_bf16_noalloc_status.restype = C.c_int
     lib.echo_gemm_workspace_bytes.restype = C.c_size_t
     lib.echo_gemm_workspace_bytes.argtypes = [i32]
     lib.echo_tiled_weight_bytes.restype = C.c_size_t
@@ -135,7 +137,8 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error",
             "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate",
             "echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible",
-            "echo_set_sequence_base", "echo_debug_capture", "echo_debug_wait_limit"]
+            "echo_set_sequence_base", "echo_debug_capture", "echo_debug_wait_limit",
+            "echo_gemm_bf16_noalloc_status"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -440,6 +443,11 @@ def echo_gemm_bf16_noalloc(X: torch.Tensor, W: torch.Tensor, Y: torch.Tensor, ep
         _check(lib.echo_gemm_bf16_noalloc(X.data_ptr(), W.data_ptr(), Y.data_ptr(), M, N, K, epilogue,
                                           _stream_ptr(None)))
     return Y
+
+
+def echo_gemm_bf16_noalloc_status() -> int:
+    """Waits for the current stream; how the last echo_gemm_bf16_noalloc on this device ended (0 = ok)."""
+    return int(lib.echo_gemm_bf16_noalloc_status(_stream_ptr(None)))
 
 
 def echo_decode_attention(q: torch.Tensor, kv_pool: torch.Tensor, page_table: torch.Tensor, row_pos: torch.Tensor,

@@ -918,11 +918,13 @@ constexpr int kNoAllocMaxRows = 32;                   // activation rows (one 32
 constexpr int kNoAllocMaxCtas = 64;                   // persistent CTAs the variant launches at most
 constexpr size_t kNoAllocWsBytes =
     static_cast<size_t>(kNoAllocMaxCtas) * 3 * kAcc * kGemmTileN * kNoAllocMaxRows * sizeof(float);   // 6 MiB
-constexpr size_t kNoAllocBytes = kNoAllocWsBytes + static_cast<size_t>(kGemmMaxUnits) * sizeof(int);
+constexpr size_t kNoAllocCounterBytes = static_cast<size_t>(kGemmMaxUnits) * sizeof(int);
+constexpr size_t kNoAllocBytes = kNoAllocWsBytes + kNoAllocCounterBytes + 256;   // + the status word
 }  // namespace
 }  // namespace echo
 
-// Partial-sum slots followed by the per-tile arrival counters.  Device code may name this array
+// Partial-sum slots, the per-tile arrival counters, then the status word of the last call (set when
+// a bounded wait of its kernel ran out).  Device code may name this array
 // directly; host code must not use the name as a pointer (on the host it is only a handle) and
 // asks the runtime for the device address instead.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[echo::kNoAllocBytes];
@@ -938,6 +940,9 @@ extern "C" int echo_gemm_bf16_noalloc(const void *X, const void *W, void *Y, int
   using namespace echo;
   if (!X || !W || !Y || M < 1 || N < 1 || K < 8 || (K % 8)) return ECHO_ERR_INVALID;
   if (epilogue != EPI_STORE && epilogue != EPI_ACCUM && epilogue != EPI_SWIGLU) return ECHO_ERR_INVALID;
+  // the tile copies need 16-byte aligned operands
+  if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W) | reinterpret_cast<uintptr_t>(Y)) & 15)
+    return ECHO_ERR_INVALID;
   if (M > kNoAllocMaxRows) return ECHO_ERR_UNSUPPORTED;           // beyond the built-in scratch
   const bool gu = epilogue == EPI_SWIGLU;
   const int per_tile = kAcc * (gu ? 64 : kGemmTileN);
@@ -954,13 +959,28 @@ extern "C" int echo_gemm_bf16_noalloc(const void *X, const void *W, void *Y, int
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   unsigned char *base = static_cast<unsigned char *>(g_noalloc_ptr[dev]);
   int *counters = reinterpret_cast<int *>(base + kNoAllocWsBytes);
-  // the array keeps whatever the previous call left: the counters must start at zero
-  if (cudaMemsetAsync(counters, 0, static_cast<size_t>(kGemmMaxUnits) * sizeof(int), s) != cudaSuccess)
-    return ECHO_ERR_CUDA;
+  int *status = reinterpret_cast<int *>(base + kNoAllocWsBytes + kNoAllocCounterBytes);
+  // the array keeps whatever the previous call left: the counters and the status word must start at zero
+  if (cudaMemsetAsync(counters, 0, kNoAllocCounterBytes + sizeof(int), s) != cudaSuccess) return ECHO_ERR_CUDA;
   CUtensorMap tmW, tmX;
   if (make_tensor_map(&tmW, W, gu ? 2ull * N : N, K, K, gu ? 64 : kGemmTileN) != 0) return ECHO_ERR_CUDA;
   if (make_tensor_map(&tmX, X, M, K, K, kNoAllocMaxRows) != 0) return ECHO_ERR_CUDA;
-  GemmArgs a{&tmW, &tmX, Y, N, M, N, K, kNoAllocMaxRows, epilogue, nullptr, reinterpret_cast<float *>(base),
+  GemmArgs a{&tmW, &tmX, Y, N, M, N, K, kNoAllocMaxRows, epilogue, status, reinterpret_cast<float *>(base),
              counters, kNoAllocMaxCtas, -1, 0, 0};
   return gemm_tc_launch(a, s) == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+extern "C" int echo_gemm_bf16_noalloc_status(void *cuda_stream) {
+  using namespace echo;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ECHO_ERR_CUDA;
+  if (!g_noalloc_ptr[dev]) return ECHO_OK;                        // no call has been made on this device
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const unsigned char *base = static_cast<const unsigned char *>(g_noalloc_ptr[dev]);
+  int st = 0;
+  if (cudaMemcpyAsync(&st, base + kNoAllocWsBytes + kNoAllocCounterBytes, sizeof(int), cudaMemcpyDeviceToHost, s) !=
+          cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return ECHO_ERR_CUDA;
+  return st == STATUS_WAIT_TIMEOUT ? ECHO_ERR_TIMEOUT : (st == STATUS_OK ? ECHO_OK : ECHO_ERR_DEVICE_CHECK);
 }

@@ -13,13 +13,16 @@ import torch
 
 from oracle import pages
 from paper_2602_02192_b200 import synth
-from helpers import LOGPROB_TOL, MARGIN_EXEMPT, StreamedWeights, check_sequences, dims_of, score_sequences
+from helpers import LOGPROB_TOL, MARGIN_EXEMPT, StreamedWeights, dims_of, score_sequences
 
 pytestmark = pytest.mark.gpu
 
-CASES = [("0.6B", [0, 257], 1024), ("8B", [3, 200], 12)]
+# (workload, sequences scored by the oracle, decode steps scored).  The 32B shape (65 GB of weights
+# generated into page-locked host memory, a 64-layer oracle pass over 1056 positions) takes about ten
+# minutes on its own and runs with ECHO_TEST_ALL_CONFIGS=1.
+CASES = [("0.6B", [0, 257], 1024), ("4B", [5, 100], 32), ("8B", [3, 200], 32)]
 if os.environ.get("ECHO_TEST_ALL_CONFIGS") == "1":
-    CASES += [("4B", [5], 6), ("32B", [1], 4)]
+    CASES += [("32B", [1], 8)]
 
 
 @pytest.mark.parametrize("name,seqs,steps", CASES)
@@ -29,7 +32,7 @@ def test_full_size_rollout(name, seqs, steps):
     shape, P, G, Lp, T = wl.shape, wl.n_prompts, wl.G, wl.prompt_len, wl.new_tokens
     torch.cuda.empty_cache()
     free, total = torch.cuda.mem_get_info()
-    cfg = B.make_config(shape, P, G, Lp, T, 1)
+    cfg = B.make_config(shape, P, G, Lp, T, 1, half_layers=wl.half_layers)     # as bench.py runs it
     on_host = 2 * shape.n_params() > 40e9              # snapshot kept in pinned host memory
     need = B.echo_arena_bytes(cfg) + (0 if on_host else 2 * shape.n_params()) + (2 << 30)
     if free < need:
@@ -54,43 +57,30 @@ def test_full_size_rollout(name, seqs, steps):
     # Teacher-forced replay of the GPU's own tokens reproduces its log-probabilities at every step.
     # With ECHO_DETERMINISTIC=1 (fixed-order reductions) bit for bit.  By default the split
     # projections add their k-slices in whatever order the CTAs finish; a last-bit difference that
-    # flips the bf16 rounding of an activation or a cached key decorrelates the later roundings, so
+    # flips the 16-bit rounding of an activation or a cached key decorrelates the later roundings, so
     # two runs differ from each other about as much as either differs from exact arithmetic.
     tok_f, lp_f, _ = eng.echo_rollout(dp, lens, G, T, wl.temperature, wl.sample_seed, forced=tok)
     eng.echo_sync()
     dlp = np.abs(lp_f.cpu().numpy() - lp_h)
+    print(f"{name}: free run vs teacher-forced replay: mean {dlp.mean():.2e} q99.9 {np.quantile(dlp, 0.999):.2e} "
+          f"max {dlp.max():.2e} same tokens {(tok_f.cpu().numpy() == tok_h).mean():.4f}")
     if os.environ.get("ECHO_DETERMINISTIC") == "1":
         assert dlp.max() == 0.0 and np.array_equal(tok_f.cpu().numpy(), tok_h)
     else:
-        assert dlp.mean() < 4e-2 and np.quantile(dlp, 0.999) < 0.25, (dlp.mean(), dlp.max())
-        assert (tok_f.cpu().numpy() == tok_h).mean() > 0.9
-    # sampled sequences against the oracle
+        # measured on B200: mean 1.8e-3 / 7.1e-3 / 1.1e-2 and 99.9 % below 7.5e-3 / 2.9e-2 / 4.5e-2 at the
+        # 0.6B / 4B / 8B shapes, 99.2 % or more of the tokens equal
+        assert dlp.mean() < 1.5e-2 and np.quantile(dlp, 0.999) < 6.5e-2, (dlp.mean(), dlp.max())
+        assert (tok_f.cpu().numpy() == tok_h).mean() > 0.985
+    # sampled sequences against the oracle: the acceptance rule, token by token
     sw = StreamedWeights(w)
-    if shape.n_layers * shape.d_model <= 28 * 1024:
-        n, ex, worst = check_sequences(dims_of(shape), sw, prompts, lens, G, wl.temperature, wl.sample_seed, tok_h,
-                                       lp_h, seqs, steps=steps, layer_provider=sw.layer)
-        assert n == len(seqs) * steps and ex <= max(2, 0.05 * n)
-    else:
-        # At 36+ layers x 4096+ channels the bf16 rounding of the activations (GEMM inputs, q, K, V,
-        # probabilities) is amplified layer by layer in a random-init network: two runs of the GPU
-        # path that differ only in fp32 summation order already differ by 2e-2 on average (above),
-        # and the error against fp64 arithmetic is of the same size (measured on 24 tokens: mean
-        # 3.1e-2, median 2.5e-2, max 9.8e-2, 79 % within 5e-2).  The 5e-2 bound therefore cannot hold
-        # token by token at this shape with bf16 GEMM inputs; it is asserted on the bulk, with a
-        # cap on the mean and on the worst token, and the statistics are printed.
-        delta, same, second, margin = score_sequences(dims_of(shape), sw, prompts, lens, G, wl.temperature,
-                                                      wl.sample_seed, tok_h, lp_h, seqs, steps=steps,
-                                                      layer_provider=sw.layer)
-        print(f"{name}: n={delta.size} mean|dlp|={delta.mean():.4f} median={np.median(delta):.4f} "
-              f"max={delta.max():.4f} within_tol={(delta <= LOGPROB_TOL).mean():.3f} "
-              f"token_match={same.mean():.3f}")
-        # The amplification grows with depth: at 64 layers (32B shape) the mean itself sits at the bound
-        # (measured on 4 tokens: 5.8e-2 with the SM-pair projections, 6.2e-2 with the one-CTA kernels,
-        # worst token 0.10 / 0.17), so the bulk criteria are scaled with sqrt(layers / 36) there.
-        depth = max(1.0, (shape.n_layers / 36.0) ** 0.5)
-        assert delta.mean() <= LOGPROB_TOL * 1.2 * depth if depth > 1 else delta.mean() <= LOGPROB_TOL
-        assert delta.max() <= 0.3
-        assert (delta <= LOGPROB_TOL * depth).mean() >= 0.6
-        bad = ~same
-        assert np.all(second[bad]) and np.all(margin[bad] < 15 * MARGIN_EXEMPT)
+    delta, same, second, margin = score_sequences(dims_of(shape), sw, prompts, lens, G, wl.temperature,
+                                                  wl.sample_seed, tok_h, lp_h, seqs, steps=steps,
+                                                  layer_provider=sw.layer)
+    print(f"{name}: half_layers={wl.half_layers} n={delta.size} mean|dlp|={delta.mean():.4f} "
+          f"median={np.median(delta):.4f} max={delta.max():.4f} within_tol={(delta <= LOGPROB_TOL).mean():.3f} "
+          f"token_match={same.mean():.3f} exempt={int((~same).sum())}")
+    assert delta.size == len(seqs) * steps
+    assert delta.max() <= LOGPROB_TOL
+    bad = ~same
+    assert np.all(second[bad]) and np.all(margin[bad] < MARGIN_EXEMPT) and bad.sum() <= max(2, 0.05 * delta.size)
     eng.close()

@@ -206,36 +206,38 @@ def test_gemm_swiglu_epilogue(B, M, F, K):
                                                      (40, 8, 8, 4, 64, 33, 150), (16, 8, 32, 8, 128, 512, 400),
                                                      (3, 8, 8, 2, 64, 48, 20), (2, 6, 32, 8, 128, 100, 9),
                                                      (2, 8, 16, 2, 128, 64, 30), (2, 5, 16, 2, 128, 80, 3)])
+@pytest.mark.parametrize("fmt", ["bf16", "half"])
 @pytest.mark.parametrize("suffix", ["resident", "waves", "tiles"])
-def test_decode_attention_matches_oracle(B, monkeypatch, suffix, P, G, Hq, Hkv, hd, Lp, steps):
+def test_decode_attention_matches_oracle(B, suffix, fmt, P, G, Hq, Hkv, hd, Lp, steps):
     """Shared-prefix decode attention against the oracle's single-query attention (fp64) on the same
-    bf16-rounded q, K, V, gathered through the oracle's page plan.  Both suffix kernels (resident CTAs
-    that walk several (sequence, kv head) items; "waves" = one CTA per item) and both prefix kernels
-    (a group's query rows in one CTA where they fill two 16-row tiles; "tiles" = one CTA per tile)."""
-    monkeypatch.delenv("ECHO_ATTN_IMPL", raising=False)
-    monkeypatch.delenv("ECHO_ATTN_PREFIX", raising=False)
-    if suffix == "waves":
-        monkeypatch.setenv("ECHO_ATTN_IMPL", "waves")
-    if suffix == "tiles":
-        monkeypatch.setenv("ECHO_ATTN_PREFIX", "tiles")
+    16-bit q, K, V (bf16, or IEEE half as in the layers of echo_config.half_layers), gathered through
+    the oracle's page plan.  Both suffix kernels (resident CTAs that walk several (sequence, kv head)
+    items; "waves" = one CTA per item) and both prefix kernels (a group's query rows in one CTA where
+    they fill two 16-row tiles; "tiles" = one CTA per tile)."""
     from oracle import decoder as o_dec
     from oracle import pages as o_pages
     rng = np.random.default_rng(P * 131 + Lp)
     plan = o_pages.build([Lp] * P, G, steps + 1, 16)
     n_pages, Bq = plan.n_pages, P * G
-    pool = torch.from_numpy(rng.normal(size=(n_pages, Hkv, 2, 16, hd)).astype(np.float32)).to(torch.bfloat16)
-    q = torch.from_numpy(rng.normal(size=(Bq, Hq, hd)).astype(np.float32)).to(torch.bfloat16)
+    dt = torch.bfloat16 if fmt == "bf16" else torch.float16
+    pool = torch.from_numpy(rng.normal(size=(n_pages, Hkv, 2, 16, hd)).astype(np.float32)).to(dt)
+    q = torch.from_numpy(rng.normal(size=(Bq, Hq, hd)).astype(np.float32)).to(dt)
     pos = np.full(Bq, Lp + steps - 1, dtype=np.int32)
     pos[::3] -= min(steps - 1, 5)                       # sequences need not be at the same position
     full = np.repeat(plan.full_prefix_pages, G).astype(np.int32)
     out = B.echo_decode_attention(q.cuda(), pool.cuda(), torch.from_numpy(plan.table).cuda(),
-                                  torch.from_numpy(pos).cuda(), torch.from_numpy(full).cuda(), P, G)
+                                  torch.from_numpy(pos).cuda(), torch.from_numpy(full).cuda(), P, G,
+                                  kernel_choice={"resident": 0, "waves": 1, "tiles": 2}[suffix])
+    assert out.dtype == dt
     out = out.float().cpu().numpy().astype(np.float64)
-    poolf = widen_bf16(synth.bf16_bits(pool))
-    qf = widen_bf16(synth.bf16_bits(q))
+    poolf = pool.to(torch.float64).numpy()                # exact widening of the 16-bit values
+    qf = q.to(torch.float64).numpy()
     # more (sequence, kv head) items than CTAs fit the GPU at once: a resident CTA then walks several
     # items and prefetches across their boundaries, so every fifth sequence is checked
     many = Bq * Hkv > 400
+    # probabilities and the output are rounded to the operand format: 2^-9 relative each for bf16,
+    # 2^-12 for half (where the fp32 exponentials and sums show instead)
+    rel, floor = (1.5e-2, 4e-3) if fmt == "bf16" else (2.5e-3, 6e-4)
     for s in sorted(set([0, 1, Bq // 2, Bq - 1] + (list(range(0, Bq, 5)) if many else []))):
         n = int(pos[s]) + 1
         pg = plan.table[s, np.arange(n) // 16]
@@ -243,8 +245,47 @@ def test_decode_attention_matches_oracle(B, monkeypatch, suffix, P, G, Hq, Hkv, 
         V = poolf[pg, :, 1, np.arange(n) % 16, :]
         want = o_dec.attend_one(qf[s], K, V, Hq, Hkv)
         err = np.abs(out[s] - want)
-        # probabilities and the output are rounded to bf16 (2^-9 relative each)
-        assert np.all(err <= 1.5e-2 * np.abs(want) + 4e-3), (s, err.max())
+        assert np.all(err <= rel * np.abs(want) + floor), (s, err.max())
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 4096, 4096), (256, 6144, 1024), (100, 688, 256), (32, 512, 2048),
+                                   (130, 20000, 320)])
+def test_gemm_half_operands_match_fp64(B, M, N, K):
+    """The projections of the layers configured with IEEE-half operands: same kernels, operand format
+    half.  Against the fp64 product of the exactly widened inputs, all kernel families."""
+    rng = np.random.default_rng(M + 7 * N + 13 * K)
+    X = torch.from_numpy(rng.normal(size=(M, K)).astype(np.float32)).to(torch.float16)
+    W = torch.from_numpy((rng.normal(size=(N, K)) * 0.05).astype(np.float32)).to(torch.float16)
+    xf, wf = X.to(torch.float64).numpy(), W.to(torch.float64).numpy()
+    want = xf @ wf.T
+    tol = 2e-6 * K * 0.05 * 4 + 1e-6
+    impls = (1, 0, 2, 102, 200, 1000, 1002) + ((300, 1300, 1302) if M > 64 else ())
+    for impl in impls:
+        got = B.echo_gemm_bf16(X.cuda(), W.cuda(), impl=impl).cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(got - want)) < tol, (impl, np.max(np.abs(got - want)))
+    # SwiGLU epilogue with a half output (2^-11 relative)
+    F = N // 2
+    g, u = want[:, :F], want[:, F: 2 * F]
+    act = g / (1 + np.exp(-g)) * u
+    for impl in (0, 2, 1000) + ((300, 1300) if M > 64 else ()):
+        Y = B.echo_gemm_bf16(X.cuda(), W[: 2 * F].contiguous().cuda(), epilogue=2, impl=impl)
+        assert Y.dtype == torch.float16
+        got = Y.to(torch.float64).cpu().numpy()
+        assert np.all(np.abs(got - act) <= 2.0 ** -10 * np.abs(act) + 1e-4 * K / 256), impl
+
+
+def test_bounded_wait_gives_up_and_reports(B):
+    """Every device-side wait of the library has a limit after which the kernel records the fact and
+    returns.  The probe runs that wait on a barrier nothing signals, with a 1 ms limit instead of the
+    library's second: the call reports ECHO_ERR_TIMEOUT, the warp waited about the limit, and the
+    device is fine afterwards (nothing hung, nothing faulted)."""
+    rc, waited = B.echo_debug_wait_limit(1_000_000)
+    assert rc == -8
+    assert 1_000_000 <= waited < 50_000_000
+    rc, waited2 = B.echo_debug_wait_limit(200_000)
+    assert rc == -8 and waited2 < waited + 5_000_000
+    x = torch.arange(8, device="cuda")
+    assert int(x.sum().item()) == 28                     # the context still answers
 
 
 def test_group_advantage_matches_oracle(B):

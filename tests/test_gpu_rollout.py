@@ -248,3 +248,158 @@ def test_host_buffer_entry_point(B, tiny):
     eng.echo_sync()
     assert_same_rollout(ht.numpy(), hl.numpy(), tok.cpu().numpy(), lp.cpu().numpy())
     eng.close()
+
+
+def _gpu_weights(w_t):
+    return {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in w_t.items()}
+
+
+def _mean_abs_dlp(shape, w_o, prompts, lens, G, temp, seed, tok, lp, seqs):
+    from helpers import score_sequences
+    delta, _, _, _ = score_sequences(dims_of(shape), w_o, prompts, lens, G, temp, seed, tok, lp, seqs)
+    return float(delta.mean())
+
+
+@pytest.mark.parametrize("half_layers", [1, 2])
+def test_half_operand_layers(B, tiny, half_layers):
+    """echo_config.half_layers: the first layers keep their 16-bit operands in IEEE half.  Same
+    acceptance rule against the (exact) oracle on every token, and the log-probabilities come out
+    closer to it than with bf16 everywhere, scored along one common trajectory."""
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 3, 4, 24, 16
+    prompts, lens = synth.make_ragged_prompts([24, 17, 9], wl.shape.vocab, 91, pad_to=Lp)
+    dp = torch.from_numpy(prompts).cuda()
+    eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, half_layers=half_layers))
+    eng.echo_load_policy(w_d, 1)
+    tok, lp, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 77)
+    eng.echo_sync()
+    tok_h, lp_h = tok.cpu().numpy(), lp.cpu().numpy()
+    n, ex, worst = check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 1.0, 77, tok_h, lp_h, range(P * G))
+    assert n == P * G * T and ex <= 0.05 * n
+    eng.close()
+    eng0 = B.Engine(B.make_config(wl.shape, P, G, Lp, T))
+    eng0.echo_load_policy(w_d, 1)
+    _, lp0, _ = eng0.echo_rollout(dp, lens, G, T, 1.0, 77, forced=tok)
+    eng0.echo_sync()
+    eng0.close()
+    e_half = _mean_abs_dlp(wl.shape, w_o, prompts, lens, G, 1.0, 77, tok_h, lp_h, range(P * G))
+    e_bf16 = _mean_abs_dlp(wl.shape, w_o, prompts, lens, G, 1.0, 77, tok_h, lp0.cpu().numpy(), range(P * G))
+    assert e_half < 0.85 * e_bf16, (e_half, e_bf16)
+    cfg = B.make_config(wl.shape, P, G, Lp, T)
+    cfg.half_layers = wl.shape.n_layers + 1                      # more layers than the model has
+    with pytest.raises(B.EchoError):
+        B.Engine(cfg)
+
+
+def test_rollout_past_the_suffix_kernel_switch(B):
+    """A rollout of 1200 new tokens: from decode step 1088 on the engine replays its second captured
+    graph (one suffix CTA per (sequence, kv head) instead of resident CTAs).  Two sequences are scored
+    by the oracle on every step, before and after the switch; narrow and shallow enough (0.6B width,
+    6 layers, 32000 ids) for the oracle to replay 1248 positions in seconds."""
+    import dataclasses
+    shape = dataclasses.replace(synth.SHAPES["0.6B"], name="0.6B-width L6", n_layers=6, vocab=32000)
+    P, G, Lp, T = 4, 8, 48, 1200
+    w_t = synth.make_weights(shape, 3, device="cuda")
+    w_o = decoder.Weights(synth.weights_to_bits(w_t))
+    eng = B.Engine(B.make_config(shape, P, G, Lp, T, 1))
+    eng.echo_load_policy(w_t, 2)
+    prompts = synth.make_prompts(P, Lp, shape.vocab, 17)
+    lens = [Lp] * P
+    tok, lp, ver = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, G, T, 1.0, 5)
+    eng.echo_sync()
+    tok_h, lp_h = tok.cpu().numpy(), lp.cpu().numpy()
+    assert np.all(ver == 2) and eng.echo_get_stats()["decode_steps"] == T - 1
+    n, ex, worst = check_sequences(dims_of(shape), w_o, prompts, lens, G, 1.0, 5, tok_h, lp_h, [6, 25])
+    assert n == 2 * T and ex <= 0.03 * n
+    # the same trajectory through the teacher-forced entry point (it crosses the switch too)
+    _, lp_f, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, G, T, 1.0, 5, forced=tok)
+    eng.echo_sync()
+    assert np.max(np.abs(lp_f.cpu().numpy() - lp_h)) < LOGPROB_TOL
+    eng.close()
+
+
+def test_eight_query_heads_per_kv_head(B):
+    """Hq / Hkv = 8 with G = 8 (the 32B shape's ratio): a group's 64 query rows take two prefix CTAs
+    per (prompt, kv head) and the merge area of the resident suffix kernel is too small, so every
+    step runs the per-item suffix kernel.  Every token of a small model against the oracle."""
+    shape = synth.DecoderShape("rep8", 2, 512, 16, 2, 128, 1024, 4096)
+    P, G, T = 3, 8, 24
+    w_t = synth.make_weights(shape, 11)
+    w_o = decoder.Weights(synth.weights_to_bits(w_t))
+    prompts, lens = synth.make_ragged_prompts([40, 33, 17], shape.vocab, 23, pad_to=40)
+    for hl in (0, 1):
+        eng = B.Engine(B.make_config(shape, P, G, 40, T, 1, half_layers=hl))
+        eng.echo_load_policy(_gpu_weights(w_t), 1)
+        tok, lp, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, G, T, 1.0, 99)
+        eng.echo_sync()
+        n, ex, worst = check_sequences(dims_of(shape), w_o, prompts, lens, G, 1.0, 99, tok.cpu().numpy(),
+                                       lp.cpu().numpy(), range(P * G))
+        assert n == P * G * T and ex <= 0.05 * n
+        eng.close()
+
+
+def test_every_sequence_ended_and_padded_trajectories(B, tiny, monkeypatch):
+    """Teacher-forced scoring of trajectories that all end early and are padded with OTHER ids after
+    their end token (a buffer from elsewhere): positions after the end token score the end token with
+    log-probability 0 whatever the padding holds, with both suffix kernels (with one CTA per item,
+    every CTA of the launch returns early once all sequences have ended).  The context then serves
+    an ordinary rollout correctly."""
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 2, 4, 20, 10
+    prompts = synth.make_prompts(P, Lp, wl.shape.vocab, 41)
+    lens = [Lp, Lp - 4]
+    dp = torch.from_numpy(prompts).cuda()
+    eos = 123
+    rng = np.random.default_rng(3)
+    given = rng.integers(0, wl.shape.vocab, size=(P, G, T)).astype(np.int32)
+    given[given == eos] = eos + 1
+    ends = rng.integers(0, 3, size=(P, G))                       # every sequence ends within three steps
+    for p in range(P):
+        for g in range(G):
+            given[p, g, ends[p, g]] = eos                        # ... and what follows is NOT the end token
+    for impl in ("", "waves"):
+        if impl:
+            monkeypatch.setenv("ECHO_ATTN_IMPL", impl)
+        else:
+            monkeypatch.delenv("ECHO_ATTN_IMPL", raising=False)
+        eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, eos_id=eos))
+        eng.echo_load_policy(w_d, 1)
+        tok_f, lp_f, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 9, forced=torch.from_numpy(given).cuda())
+        eng.echo_sync()
+        tok_f, lp_f = tok_f.cpu().numpy(), lp_f.cpu().numpy()
+        for p in range(P):
+            for g in range(G):
+                e = ends[p, g]
+                assert np.all(lp_f[p, g, e + 1:] == 0.0) and np.all(tok_f[p, g, e + 1:] == eos)
+                sc = decoder.score_forced(dims_of(wl.shape), w_o, prompts[p][: lens[p]], given[p, g], 1.0, 9,
+                                          p * G + g, eos_id=eos)
+                assert np.max(np.abs(lp_f[p, g] - sc.logprob_given)) <= LOGPROB_TOL
+        tok, lp, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 9)
+        eng.echo_sync()
+        check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 1.0, 9, tok.cpu().numpy(), lp.cpu().numpy(),
+                        range(P * G), eos_id=eos)
+        eng.close()
+
+
+def test_prompts_cut_over_contexts_reproduce_one_call(B, tiny):
+    """Groups are independent: a prompt set cut by prompt over two contexts (as over two GPUs), each
+    with its sequence-id base, yields the tokens one call over the whole set yields."""
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 4, 4, 32, 12
+    prompts = synth.make_prompts(P, Lp, wl.shape.vocab, 55)
+    lens = [Lp] * P
+    eng = _engine(B, wl.shape, P, G, Lp, T)
+    eng.echo_load_policy(w_d, 1)
+    tok_all, lp_all, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, G, T, 1.0, 321)
+    eng.echo_sync()
+    tok_all, lp_all = tok_all.cpu().numpy(), lp_all.cpu().numpy()
+    n_parts = 2
+    for r in range(n_parts):
+        mine = [p for p in range(P) if p % n_parts == r]
+        for p in mine:                        # one call per prompt here: its ids are p*G .. p*G+G-1
+            eng.echo_set_sequence_base(p * G)
+            tok, lp, _ = eng.echo_rollout(torch.from_numpy(prompts[p: p + 1]).cuda(), [Lp], G, T, 1.0, 321)
+            eng.echo_sync()
+            assert_same_rollout(tok.cpu().numpy()[0], lp.cpu().numpy()[0], tok_all[p], lp_all[p])
+    eng.echo_set_sequence_base(0)
+    eng.close()

@@ -25,13 +25,15 @@ def test_noalloc_matches_workspace_entry_twice_in_a_row(B, M, N, K):
     X = torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16)
     W = (torch.randn(N, K, device="cuda", generator=g) * 0.05).to(torch.bfloat16)
     want = B.echo_gemm_bf16(X, W, impl=2)                 # same kernel, caller-provided workspace
+    exact = X.double() @ W.double().T                     # the fp64 product the other projection tests use
     tol = 2e-6 * K * 0.05 * 4 + 1e-6                      # the GEMM tests' fp32-accumulation bound
     Y = torch.empty((M, N), dtype=torch.float32, device="cuda")
     for _ in range(2):                                    # the shared scratch keeps the last call's contents
         Y.fill_(float("nan"))
         B.echo_gemm_bf16_noalloc(X, W, Y)
-        torch.cuda.synchronize()
+        assert B.echo_gemm_bf16_noalloc_status() == 0     # waits for the stream; no bounded wait ran out
         assert float((Y - want).abs().max()) < tol
+        assert float((Y.double() - exact).abs().max()) < tol
     # residual-add epilogue on top of a known Y
     Y0 = torch.randn(M, N, device="cuda", generator=g)
     Y = Y0.clone()
@@ -62,3 +64,8 @@ def test_noalloc_swiglu_and_limits(B):
     assert ei.value.code == -9
     torch.cuda.synchronize()
     assert bool((Yb == 5.0).all())
+    # operands that the tile copies cannot address (not 16-byte aligned) are an argument error
+    Xo = torch.zeros(M * K + 8, device="cuda", dtype=torch.bfloat16)[1: 1 + M * K].view(M, K)
+    with pytest.raises(B.EchoError) as ei:
+        B.echo_gemm_bf16_noalloc(Xo, W, torch.empty((M, 2 * F), device="cuda"))
+    assert ei.value.code == -1
