@@ -140,9 +140,12 @@ def rollout_roofline_seconds(shape, P, G, Lp, T, bw_gbs, tflops):
 # ---------------------------------------------------------------------------------------------
 # multi-GPU: independent replicas (no data-path collective); helpers shared with the CPU tests
 # ---------------------------------------------------------------------------------------------
-def rank_prompt_seed(base_seed: int, rank: int) -> int:
-    """Every rank works on its own prompts (groups are never split across ranks)."""
-    return base_seed + 7919 * rank
+def rank_prompt_range(n_prompts: int, rank: int, world: int):
+    """Prompts [lo, hi) of the job's prompt set that rank `rank` of `world` works on: contiguous
+    blocks, groups never split.  Its sequence ids start at lo * G."""
+    per, extra = divmod(n_prompts, world)
+    lo = rank * per + min(rank, extra)
+    return lo, lo + per + (1 if rank < extra else 0)
 
 
 def max_over_ranks(value: float, device, world: int) -> float:
@@ -183,7 +186,9 @@ def run_ours(args):
         Lp = args.prompt_len
     swap = args.workload == "8B" and not args.no_swap
     nbuf = 1 if args.workload == "32B" else 2
-    eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, nbuf, top_p=args.top_p), device=local_rank)
+    half_layers = wl.half_layers if args.half_layers < 0 else min(args.half_layers, shape.n_layers)
+    eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, nbuf, top_p=args.top_p, half_layers=half_layers),
+                         device=local_rank)
     if args.workload == "32B":
         # 65 GB of weights: the snapshot stays in page-locked host memory so that the device holds it once
         weights = synth.make_weights_pinned(shape, wl.weight_seed, gen_device=dev)
@@ -198,8 +203,13 @@ def run_ours(args):
         w_next = synth.make_weights(shape, wl.weight_seed + 1, device=dev)
         torch.cuda.synchronize()
 
-    # every rank is an independent replica working on its own prompts (groups never split)
-    prompts = torch.from_numpy(synth.make_prompts(P, Lp, shape.vocab, rank_prompt_seed(wl.prompt_seed, rank))).to(dev)
+    # Every rank is an independent replica (groups never split): the job's prompt set is world * P
+    # prompts, rank r takes prompts [r * P, (r + 1) * P) of it and numbers its sequences from r * P * G,
+    # so the job's tokens do not depend on how many GPUs share it.
+    all_prompts = synth.make_prompts(world * P, Lp, shape.vocab, wl.prompt_seed)
+    lo_p, hi_p = rank_prompt_range(world * P, rank, world)
+    prompts = torch.from_numpy(all_prompts[lo_p:hi_p]).to(dev)
+    eng.echo_set_sequence_base(lo_p * G)
     lens = [Lp] * P
     out_tok = torch.empty((P, G, T), dtype=torch.int32, device=dev)
     out_lp = torch.empty((P, G, T), dtype=torch.float32, device=dev)
@@ -247,6 +257,7 @@ def run_ours(args):
 
     # ---- end to end: host buffers, copies inside the timed region -------------------------
     hp = prompts.cpu().pin_memory()
+    h2d_bytes = int(hp.numel() * 4)
     ht = torch.empty((P, G, T), dtype=torch.int32).pin_memory()
     hl = torch.empty((P, G, T), dtype=torch.float32).pin_memory()
     barrier()
@@ -261,6 +272,25 @@ def run_ours(args):
         if world > 1:
             dist.destroy_process_group()
         return
+
+    # ---- outside the timed region (rank 0): where the prefill's time goes, and a read-only peak ----
+    prefill = None
+    eng.echo_profile_config(-1)
+    eng.echo_rollout(prompts, lens, G, min(T, 2), wl.temperature, wl.sample_seed + 7, out_tokens=out_tok[:, :, : min(T, 2)].contiguous(),
+                     out_logprobs=out_lp[:, :, : min(T, 2)].contiguous())
+    pf_steps, pf_ms = eng.echo_profile_read()
+    eng.echo_profile_config(0)
+    if len(pf_steps) and int(pf_steps[0]) == 0:
+        a, g_, _, tot = (float(x) for x in pf_ms[0])
+        prefill = {"ms": round(tot, 1), "projections_ms": round(g_, 1), "attention_ms": round(a, 1),
+                   "other_ms": round(tot - a - g_, 1),
+                   "note": "kernel-by-kernel launches with events (no early start between kernels)"}
+    read_gbs = None
+    try:
+        del hp
+        read_gbs = binding.echo_probe_read_bandwidth(2 << 30, 10, device=dev)
+    except Exception as e:                      # not enough free memory for the probe buffer
+        read_gbs = None
 
     # ---- roofline of the dominant kernel (decode attention), from the sampled steps ---------
     attn_launches = len(prof_steps) * shape.n_layers
@@ -282,6 +312,10 @@ def run_ours(args):
         roof = {"bound": "hbm", "kernel": "decode attention (paged GQA)", "achieved": round(achieved, 1),
                 "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                 "frac": round(achieved / peaks["hbm_gbs"], 4),
+                "peak_read_only": round(read_gbs, 1) if read_gbs else None,
+                "peak_read_only_note": "this library's read-only streaming probe (2 GiB, 16-byte loads, nothing "
+                                       "written); the driver's peak is a copy, which also writes",
+                "frac_of_read_only_peak": round(achieved / read_gbs, 4) if read_gbs else None,
                 "traffic": round(traffic) if traffic else None, "traffic_unit": "bytes per launch (ncu, scaled)",
                 "launches_timed": attn_launches,
                 "avg_launch_us": round(dur_s / attn_launches * 1e6, 2),
@@ -298,24 +332,29 @@ def run_ours(args):
 
     cpu = None
     if not args.no_cpu_baseline:
-        cpu = cpu_baseline_sample(shape, w_next if swap else weights, prompts, ht, wl)
+        cpu = cpu_baseline_sample(eng, shape, w_next if swap else weights, prompts, wl, dev)
 
     line = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(elapsed_ms / args.steps, 2), "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if half_layers == 0 else f"bf16 (f16 operands in layers 0-{half_layers - 1})",
+        "data": "synthetic",
         "config": {"workload": f"{wl.name}-shape decoder: L{shape.n_layers} d{shape.d_model} "
                                f"{shape.n_q_heads}q/{shape.n_kv_heads}kv hd{shape.head_dim} F{shape.d_ff} "
                                f"V{shape.vocab}; {P} prompts x G={G}, prompt {Lp}, {T} new tokens, T=1.0",
-                   "top_p": args.top_p,
+                   "top_p": args.top_p, "half_layers": half_layers,
                    "policy_swap": "one echo_load_policy of a re-seeded weight set during timed step 0" if swap
                    else "none", "versions_served": versions_seen, "e2e_version": int(ver_e2e[0, 0]),
                    "install_ms": round(install_ms, 1),
-                   "last_rollout_prefill_ms": round(st_last["prefill_ms"], 1),
+                   "last_rollout_prefill_ms": round(st_last["prefill_ms"], 1), "prefill_breakdown": prefill,
                    "last_rollout_decode_ms_per_step": round(st_last["decode_ms"] / max(1, T - 1), 3),
                    "l2": "inputs larger than L2 (weights + KV >> 126 MB)", "parallelism": f"replicas x{world}"},
         "clocks": clk,
-        "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": int(hp.numel() * 4),
+        # time x median SM clock: compares runs on GPUs that settle at different clocks under the power cap
+        "sm_gigacycles_per_step": (round(elapsed_ms / args.steps * clk["sm_mhz"] / 1e6, 3)
+                                   if clk and clk.get("sm_mhz") else None),
+        "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d_bytes,
                 "d2h_bytes_per_step": int(ht.numel() * 4 + hl.numel() * 4)},
         "gpu_launches": int(launches),
         "roofline": roof,
@@ -375,24 +414,72 @@ def _oracle_sample_pass(shape, sw, prompt_ids, given, temperature, seed, s):
                                 layer_provider=sw.layer)
 
 
-SAMPLE_PROMPT = 24
-SAMPLE_NEW = 8
+SAMPLE_PROMPT = 64        # the 8B-shape slice the oracle finishes in tens of seconds
+SAMPLE_NEW = 4
 
 
-def cpu_baseline_sample(shape, weights, prompts, host_tokens, wl):
-    """Times the oracle, as it stands, on a bounded sample of the same workload."""
+def _time_gpu(eng, prompts, lens, G, T, temperature, seed):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    eng.echo_rollout(prompts, lens, G, T, temperature, seed)            # warm-up of this shape of call
+    eng.echo_sync()
+    e0.record(eng.stream)
+    tok, lp, _ = eng.echo_rollout(prompts, lens, G, T, temperature, seed)
+    e1.record(eng.stream)
+    eng.echo_sync()
+    st = eng.echo_get_stats()
+    return e0.elapsed_time(e1) / 1e3, st, tok
+
+
+def cpu_baseline_sample(eng, shape, weights, prompts, wl, dev):
+    """The oracle as it stands, timed on this machine's host cores beside the GPU on the SAME inputs:
+    (i) the tiny workload in full, KV-cached decoding (mode A); (ii) a slice of this workload."""
+    from oracle import decoder
+    from paper_2602_02192_b200 import binding, synth
     cores = os.cpu_count() or 1
-    prompt_ids = prompts[0, :SAMPLE_PROMPT].cpu().numpy()
-    given = host_tokens[0, 0, :SAMPLE_NEW].numpy()
+    # ---- (i) tiny, whole workload, mode A ---------------------------------------------------
+    tw = synth.WORKLOADS["tiny"]
+    ts = tw.shape
+    w_t = synth.make_weights(ts, tw.weight_seed)
+    t_prompts = synth.make_prompts(tw.n_prompts, tw.prompt_len, ts.vocab, tw.prompt_seed)
+    t_lens = [tw.prompt_len] * tw.n_prompts
+    w_o = decoder.Weights(synth.weights_to_bits(w_t))
+    t0 = time.perf_counter()
+    decoder.rollout_cached(_oracle_dims(ts), w_o, t_prompts, t_lens, tw.G, tw.new_tokens, tw.temperature,
+                           tw.sample_seed)
+    t_cpu = time.perf_counter() - t0
+    n_tiny = tw.n_prompts * tw.G * tw.new_tokens
+    teng = binding.Engine(binding.make_config(ts, tw.n_prompts, tw.G, tw.prompt_len, tw.new_tokens, 1),
+                          device=torch.device(dev).index or 0)
+    teng.echo_load_policy({k: ([t.to(dev) for t in v] if isinstance(v, list) else v.to(dev)) for k, v in w_t.items()}, 1)
+    t_gpu, _, _ = _time_gpu(teng, torch.from_numpy(t_prompts).to(dev), t_lens, tw.G, tw.new_tokens, tw.temperature,
+                            tw.sample_seed)
+    teng.close()
+    tiny = {"oracle_tokens_per_s": round(n_tiny / t_cpu, 2), "oracle_s": round(t_cpu, 2),
+            "gpu_tokens_per_s": round(n_tiny / t_gpu, 1), "gpu_s": round(t_gpu, 5),
+            "sample": f"tiny workload in full ({tw.n_prompts} prompts x G={tw.G}, prompt {tw.prompt_len}, "
+                      f"{tw.new_tokens} new tokens), oracle mode A (KV-cached, token by token)"}
+    # ---- (ii) a slice of this workload: 1 prompt x G = 1, first SAMPLE_PROMPT prompt tokens, SAMPLE_NEW new tokens
+    Lp_s = min(SAMPLE_PROMPT, prompts.shape[1])
+    sl_prompts = prompts[:1].clone()
+    t_gpu, st, tok = _time_gpu(eng, sl_prompts, [Lp_s], 1, SAMPLE_NEW, wl.temperature, wl.sample_seed)
+    given = tok[0, 0].cpu().numpy()
+    prompt_ids = sl_prompts[0, :Lp_s].cpu().numpy()
     t0 = time.perf_counter()
     sw = _StreamedWeights(weights)
+    t_w = time.perf_counter() - t0
     _oracle_sample_pass(shape, sw, prompt_ids, given, wl.temperature, wl.sample_seed, 0)
     dt = time.perf_counter() - t0
     return {"value": round(SAMPLE_NEW / dt, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
             "seconds": round(dt, 2),
-            "sample": f"1 sequence of the {wl.name}-shape workload: first {SAMPLE_PROMPT} prompt tokens + "
-                      f"{SAMPLE_NEW} generated tokens scored teacher-forced in one causal pass (fp64 numpy), "
-                      f"all {shape.n_layers} layers streamed from the bf16 weights (widening included)"}
+            "sample": f"slice of the {wl.name}-shape workload: 1 prompt x G=1, first {Lp_s} prompt tokens, "
+                      f"{SAMPLE_NEW} new tokens, scored teacher-forced along the GPU's tokens in one causal "
+                      f"pass (mode C, fp64 numpy), all {shape.n_layers} layers streamed from the bf16 weights "
+                      f"(widening included).  The slice SURVEY planned (1 prompt x G=8, prompt 512, 4 tokens, "
+                      f"mode A) is beyond numpy: token-by-token decoding re-reads 8 bytes per parameter per "
+                      f"token (60 GB at this shape).",
+            "gpu_same_input": {"tokens_per_s": round(SAMPLE_NEW / t_gpu, 1), "seconds": round(t_gpu, 5),
+                               "prefill_ms": round(st["prefill_ms"], 3), "decode_ms": round(st["decode_ms"], 3)},
+            "tiny": tiny}
 
 
 def run_reference(args):
@@ -559,11 +646,23 @@ def main():
     ap.add_argument("--top-p", type=float, default=1.0,
                     help="nucleus sampling (the paper samples with 0.95); 1.0 = the benchmark's untruncated sampling")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--half-layers", type=int, default=-1,
+                    help="leading layers with IEEE-half operands; default: the workload's setting")
     ap.add_argument("--variable-length", action="store_true",
                     help="diagnostic: random response lengths with and without the end-of-sequence rule, and exit")
     ap.add_argument("--projections", action="store_true",
                     help="diagnostic: time each projection shape alone (with cuBLAS beside it) and exit")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours" and not (
+            args.variable_length or args.projections):
+        # one process per GPU: start the ranks (the same command line under the torch launcher)
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        os.execv(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                  f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+                                  "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:])
     if args.variable_length:
         run_variable_length(args)
     elif args.projections:

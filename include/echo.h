@@ -217,7 +217,8 @@ int echo_get_stats(echo_ctx *ctx, echo_stats *out);
 
 /* Sampled per-kernel timing.  With every_n_steps = n > 0, every n-th decode step of later
  * rollouts is launched kernel by kernel (not as a graph replay) with CUDA events around the
- * attention launches, the dense projections, the sampler and the whole step; 0 turns it off.
+ * attention launches, the dense projections, the sampler and the whole step; 0 turns it off;
+ * -1 times the prompt prefill that way instead (reported as step 0; the decode steps run untimed).
  * echo_profile_read waits for the stream and returns, for each sampled step of the most
  * recent rollout, its index in steps[i] (host int32) and four summed durations in
  * milliseconds in ms[4*i + c] (host fp32): c = 0 attention, 1 projections, 2 sampler,
@@ -241,6 +242,14 @@ int echo_debug_page_table(echo_ctx *ctx, int32_t *out, size_t n, int32_t *rows, 
  * (the one that feeds token j-1) at index j-1.  Any pointer may be NULL.  layer = -1 turns it off.
  * The buffers must stay valid while rollouts run; d_model must be a multiple of 4. */
 int echo_debug_capture(echo_ctx *ctx, int32_t layer, float *pre_in, float *pre_out, float *dec_in, float *dec_out);
+
+/* Read-only streaming probe (measurement aid; the paper has no counterpart): a kernel that reads
+ * `bytes` (a multiple of 16) of device memory at `buf` once per pass, with 16-byte loads from every
+ * SM, and writes nothing.  Decode attention and weight streaming are read-only streams; a copy, the
+ * usual bandwidth yardstick, also writes.  One warm-up pass, then `repeats` (1..1000) passes between
+ * two events; *ms_per_pass (host) = their mean duration.  scratch: dev, 4 bytes.  Synchronises. */
+int echo_probe_read_bandwidth(const void *buf, size_t bytes, int32_t repeats, void *scratch, float *ms_per_pass,
+                              void *cuda_stream);
 
 /* Wait-limit probe.  Every device-side wait of this library (TMA pipelines, accumulator hand-over) is
  * bounded: when the limit runs out the kernel records it, drains and returns, and the host reports

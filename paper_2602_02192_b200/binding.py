@@ -82,6 +82,8 @@ def _load() -> C.CDLL:
     lib.echo_debug_page_table.argtypes = [vp, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32)]
     lib.echo_plan_page_table.argtypes = [vp, i32, i32, i32, i32, vp, C.c_size_t, C.POINTER(i32), C.POINTER(i32)]
     lib.echo_plan_page_table.restype = C.c_int
+    lib.echo_probe_read_bandwidth.argtypes = [vp, C.c_size_t, i32, vp, C.POINTER(f32), vp]
+    lib.echo_probe_read_bandwidth.restype = C.c_int
     lib.echo_set_sequence_base.argtypes = [vp, u32]
     lib.echo_debug_capture.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.echo_debug_wait_limit.argtypes = [u64, vp, C.POINTER(u64), vp]
@@ -138,7 +140,7 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate",
             "echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible",
             "echo_set_sequence_base", "echo_debug_capture", "echo_debug_wait_limit",
-            "echo_gemm_bf16_noalloc_status"]
+            "echo_gemm_bf16_noalloc_status", "echo_probe_read_bandwidth"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -343,6 +345,19 @@ def echo_grpo_surrogate(logp_new: torch.Tensor, logp_old: torch.Tensor, logp_sam
                                        adv.data_ptr(), mask.data_ptr() if mask is not None else None, n, T,
                                        float(eps_clip), float(C_trunc), out.data_ptr(), _stream_ptr(None)))
     return out
+
+
+def echo_probe_read_bandwidth(n_bytes: int = 4 << 30, repeats: int = 10, device="cuda") -> float:
+    """GB/s of a read-only pass over n_bytes of device memory (larger than L2 by default)."""
+    buf = torch.empty(n_bytes // 16 * 16, dtype=torch.uint8, device=device)
+    buf.zero_()
+    sink = torch.zeros(1, dtype=torch.int32, device=device)
+    ms = C.c_float(0.0)
+    with torch.cuda.device(buf.device):
+        torch.cuda.current_stream().synchronize()
+        _check(lib.echo_probe_read_bandwidth(buf.data_ptr(), buf.numel(), int(repeats), sink.data_ptr(),
+                                             C.byref(ms), _stream_ptr(None)))
+    return buf.numel() / (ms.value * 1e-3) / 1e9
 
 
 def echo_debug_wait_limit(limit_ns: int):

@@ -215,6 +215,8 @@ cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float 
 cudaError_t set_int_launch(int32_t *p, int32_t v, cudaStream_t s);
 // copies n floats (a multiple of 4) of x into slot (*d_step - 1) of dst
 cudaError_t capture_step_launch(const float *x, float *dst, const int32_t *d_step, size_t n, cudaStream_t s);
+// reads `bytes` (a multiple of 16) of buf once with n_blocks blocks of 512 threads; writes nothing
+cudaError_t read_probe_launch(const void *buf, size_t bytes, uint32_t *sink, int n_blocks, cudaStream_t s);
 // one warp waits limit_ns for a barrier nobody signals, then sets *status = STATUS_WAIT_TIMEOUT
 cudaError_t wait_probe_launch(uint64_t limit_ns, int *status, unsigned long long *waited_ns, cudaStream_t s);
 

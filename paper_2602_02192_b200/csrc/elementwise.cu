@@ -345,6 +345,24 @@ __global__ void capture_step_kernel(const float *__restrict__ x, float *__restri
   if (i < n) *reinterpret_cast<float4 *>(dst + slot * n + i) = *reinterpret_cast<const float4 *>(x + i);
 }
 
+// Read-only streaming probe: every thread walks the buffer with 16-byte loads and folds what it reads;
+// the fold is stored only if it has a value it cannot have, so nothing is written.
+__global__ void __launch_bounds__(512) read_probe_kernel(const uint4 *__restrict__ buf, size_t n_vec, uint32_t *sink) {
+  const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+  uint32_t acc = 0;
+  size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  for (; i + 3 * stride < n_vec; i += 4 * stride) {
+    const uint4 a = __ldcs(buf + i), b = __ldcs(buf + i + stride), c = __ldcs(buf + i + 2 * stride),
+                d = __ldcs(buf + i + 3 * stride);
+    acc ^= a.x ^ a.y ^ a.z ^ a.w ^ b.x ^ b.y ^ b.z ^ b.w ^ c.x ^ c.y ^ c.z ^ c.w ^ d.x ^ d.y ^ d.z ^ d.w;
+  }
+  for (; i < n_vec; i += stride) {
+    const uint4 a = __ldcs(buf + i);
+    acc ^= a.x ^ a.y ^ a.z ^ a.w;
+  }
+  if (acc == 0x9E3779B9u && sink) atomicAdd(sink, 1u);
+}
+
 // Wait-limit probe: one warp waits, with the given limit, for a barrier phase that nothing completes.
 // The wait gives up, the kernel records STATUS_WAIT_TIMEOUT and returns; nothing else depends on it.
 __global__ void wait_probe_kernel(uint64_t limit_ns, int *status, unsigned long long *waited_ns) {
@@ -654,6 +672,10 @@ cudaError_t capture_step_launch(const float *x, float *dst, const int32_t *d_ste
   if (n == 0) return cudaSuccess;
   if (n % 4) return cudaErrorInvalidValue;
   capture_step_kernel<<<static_cast<unsigned>((n / 4 + 255) / 256), 256, 0, s>>>(x, dst, d_step, n);
+  return cudaGetLastError();
+}
+cudaError_t read_probe_launch(const void *buf, size_t bytes, uint32_t *sink, int n_blocks, cudaStream_t s) {
+  read_probe_kernel<<<n_blocks, 512, 0, s>>>(static_cast<const uint4 *>(buf), bytes / 16, sink);
   return cudaGetLastError();
 }
 cudaError_t wait_probe_launch(uint64_t limit_ns, int *status, unsigned long long *waited_ns, cudaStream_t s) {

@@ -653,9 +653,17 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   int *status = ctx->ptr<int>(lo.status);
 
   CK(cudaEventRecord(ctx->ev_begin, ctx->stream));
+  ctx->prof_recs.clear();
+  ctx->prof_pool_used = 0;
+  if (ctx->prof_every < 0) {      // per-kernel-class timing of the prefill, reported as step 0
+    ctx->prof_now = true;
+    ctx->prof_step = 0;
+  }
   if (ctx->cfg.eos_id >= 0)       // no sequence has ended yet
     CK(cudaMemsetAsync(ctx->arena + lo.row_done, 0, static_cast<size_t>(pl.B) * 4, ctx->stream));
   // ---- prefill: once per prompt, in chunks of kChunkRows tokens -------------
+  cudaEvent_t pf_a = nullptr, pf_b = nullptr;
+  if (ctx->prof_now && (pf_a = prof_event(ctx)) && (pf_b = prof_event(ctx))) cudaEventRecord(pf_a, ctx->stream);
   for (int c = 0; c < pl.n_chunks; ++c) {
     const int r0 = c * kChunkRows, R = std::min(kChunkRows, pl.n_tok - r0);
     LAUNCH(embed_launch(w.embed, prompts, ctx->ptr<int32_t>(lo.pre_tok_idx) + r0, x, R, D.d, D.V, status,
@@ -683,6 +691,11 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, D.V, G, nullptr, nullptr, 0, temperature, seed, forced, T,
                         out_tokens, out_logprobs, T, ctx->stream, ctx->cfg.eos_id, cut0, nullptr, ctx->seq_base));
 
+  if (pf_a && pf_b) {
+    cudaEventRecord(pf_b, ctx->stream);
+    ctx->prof_recs.push_back({0, PROF_STEP, pf_a, pf_b});
+  }
+  ctx->prof_now = false;
   CK(cudaEventRecord(ctx->ev_first, ctx->stream));
   // ---- decode steps 1..T-1 ----------------------------------------------------
   const int32_t *tok_hist = forced ? forced : out_tokens;
@@ -720,8 +733,6 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
       }
     }
   }
-  ctx->prof_recs.clear();
-  ctx->prof_pool_used = 0;
   int rc_steps = ECHO_OK;
   for (int j = 1; j <= n_steps && rc_steps == ECHO_OK; ++j) {
     const bool sampled = ctx->prof_every > 0 && (j % ctx->prof_every == 0);
@@ -1277,6 +1288,37 @@ int echo_retile_weights(const void *src, int64_t rows, int64_t cols, void *dst, 
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }
 
+int echo_probe_read_bandwidth(const void *buf, size_t bytes, int32_t repeats, void *scratch, float *ms_per_pass,
+                              void *cuda_stream) {
+  if (!buf || !scratch || !ms_per_pass || bytes < 16 || (bytes % 16) || repeats < 1 || repeats > 1000 ||
+      (reinterpret_cast<uintptr_t>(buf) & 15) || (reinterpret_cast<uintptr_t>(scratch) & 3))
+    return ECHO_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return ECHO_ERR_CUDA;
+  cudaEvent_t a = nullptr, b = nullptr;
+  if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) {
+    if (a) cudaEventDestroy(a);
+    return ECHO_ERR_CUDA;
+  }
+  int rc = ECHO_OK;
+  uint32_t *sink = static_cast<uint32_t *>(scratch);
+  if (read_probe_launch(buf, bytes, sink, sms * 4, s) != cudaSuccess) rc = ECHO_ERR_CUDA;      // warm-up pass
+  if (rc == ECHO_OK && cudaEventRecord(a, s) != cudaSuccess) rc = ECHO_ERR_CUDA;
+  for (int i = 0; i < repeats && rc == ECHO_OK; ++i)
+    if (read_probe_launch(buf, bytes, sink, sms * 4, s) != cudaSuccess) rc = ECHO_ERR_CUDA;
+  if (rc == ECHO_OK && (cudaEventRecord(b, s) != cudaSuccess || cudaEventSynchronize(b) != cudaSuccess))
+    rc = ECHO_ERR_CUDA;
+  float ms = 0.f;
+  if (rc == ECHO_OK && cudaEventElapsedTime(&ms, a, b) != cudaSuccess) rc = ECHO_ERR_CUDA;
+  cudaEventDestroy(a);
+  cudaEventDestroy(b);
+  if (rc == ECHO_OK) *ms_per_pass = ms / static_cast<float>(repeats);
+  return rc;
+}
+
 int echo_set_sequence_base(echo_ctx *ctx, uint32_t base) {
   if (!ctx) return ECHO_ERR_INVALID;
   ctx->seq_base = base;
@@ -1311,7 +1353,7 @@ int echo_debug_wait_limit(uint64_t limit_ns, void *scratch, uint64_t *waited_ns,
 }
 
 int echo_profile_config(echo_ctx *ctx, int32_t every_n_steps) {
-  if (!ctx || every_n_steps < 0) return ECHO_ERR_INVALID;
+  if (!ctx || every_n_steps < -1) return ECHO_ERR_INVALID;
   ctx->prof_every = every_n_steps;
   return ECHO_OK;
 }

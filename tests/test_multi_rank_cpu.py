@@ -1,6 +1,8 @@
-"""The N > 1 path of the benchmark is N independent replicas: each rank takes its own prompts, no
-data-path collective, and the job's time is the slowest rank's.  Covered here with two gloo ranks
-on the CPU (no GPU needed)."""
+"""The N > 1 path of the benchmark is N independent replicas: the job's prompt set is cut by prompt
+(groups are never split), each rank numbers its sequences from its first prompt's global index, there
+is no data-path collective, and the job's time is the slowest rank's.  Covered here with two gloo
+ranks on the CPU (no GPU needed): the cut, drawn through the oracle's sampler with global sequence
+ids, reproduces what one process draws for the whole set."""
 import os
 import sys
 
@@ -15,15 +17,30 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def _worker(rank, world, port, out):
     sys.path.insert(0, ROOT)
     import bench
-    from oracle import advantage
+    from oracle import advantage, sampler
     from paper_2602_02192_b200 import synth
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
-    prompts = synth.make_prompts(4, 8, 4096, bench.rank_prompt_seed(1001, rank))
-    gathered = [torch.zeros(4, 8, dtype=torch.int32) for _ in range(world)]
-    dist.all_gather(gathered, torch.from_numpy(prompts))
-    distinct = all(not torch.equal(gathered[i], gathered[j]) for i in range(world) for j in range(i + 1, world))
+    # 7 prompts over 2 ranks: [0, 4) and [4, 7).  Every rank draws the first token of its own sequences
+    # from the logits row of their prompt, with the GLOBAL sequence id p * G + g in the noise stream
+    # (what echo_set_sequence_base(lo * G) makes the library do); gathered, the draws equal the ones a
+    # single process makes for the whole set.
+    n_prompts, G, V, seed = 7, 3, 257, 99
+    logits = np.random.default_rng(5).normal(size=(n_prompts, V))
+    lo, hi = bench.rank_prompt_range(n_prompts, rank, world)
+    mine = torch.full((n_prompts * G,), -1, dtype=torch.int64)
+    base = lo * G
+    for p_local in range(hi - lo):
+        for g in range(G):
+            s_local = p_local * G + g
+            mine[base + s_local] = sampler.draw(logits[lo + p_local], 1.0, seed, base + s_local, 0).token
+    gathered = [torch.zeros_like(mine) for _ in range(world)]
+    dist.all_gather(gathered, mine)
+    stacked = torch.stack(gathered)
+    covered_once = bool(((stacked >= 0).sum(dim=0) == 1).all())             # every sequence on exactly one rank
+    whole = torch.tensor([sampler.draw(logits[s // G], 1.0, seed, s, 0).token for s in range(n_prompts * G)])
+    distinct = covered_once and bool((stacked.max(dim=0).values == whole).all())
     # each rank is slower or faster; the job's time is the maximum
     elapsed = bench.max_over_ranks(100.0 * (rank + 1), "cpu", world)
     value = bench.job_tokens_per_second(4 * 4 * 32, world, 3, elapsed)
