@@ -288,6 +288,28 @@ int echo_greedy_provision(const double *mu, const double *cost, int32_t n, doubl
  * the staleness budget S iff v_t - S <= v <= v_t.  Returns 1 or 0. */
 int echo_admissible(int64_t v, int64_t v_t, int64_t S);
 
+/* Appendix C.3, "Worker scoring": Score = Decay (0.5 Speed + 0.35 Success + 0.15 Stability) with
+ *   Speed = 100 (log10(avg_speed) - 3) / 5 (avg_speed in bits per second: 100 at 100 Mbit/s; clamped to
+ *   [0, 100]: the appendix says it saturates at 100, the lower clamp is this library's reading),
+ *   Success = 100 success_rate, Stability = 0 after more than 3 consecutive failures, else
+ *   100 min(succ_count / 10, 1), Decay = 1 - min(elapsed_s / 600, 0.3). */
+int echo_peer_score(double avg_speed, double success_rate, int32_t succ_count, int32_t consecutive_failures,
+                    double elapsed_s, double *out);
+/* Section 4.3 / Appendix C.3, "Chain assembly": N_ch = floor(B0 / Bw) forwarding chains (at least 1, at
+ * most n); the N_ch best-scored workers are the first-hop seeds, the others are appended to the chain
+ * tails in rank order, round-robin over the chains (equal scores: lower index first).  chain_of[i] and
+ * hop_of[i] (host int32 [n]) receive worker i's chain and its hop (0 = seed, fed by the learner); its
+ * parent is the worker of the same chain at hop - 1, its only child the one at hop + 1 (fan-out 1). */
+int echo_chain_assemble(const double *score, int32_t n, double B0, double Bw, int32_t *chain_of, int32_t *hop_of,
+                        int32_t *n_chains);
+/* Section 4.3, chunked store-and-forward streaming along one chain, as a timeline: the time at which
+ * the worker at hop `hop` holds the whole snapshot of `bytes` when it is cut into chunks of
+ * chunk_bytes (the last may be shorter), every link carries Bw_bytes_per_s, a link forwards a chunk
+ * once it has arrived completely upstream, and each hop adds hop_latency_s per chunk.  With equal
+ * chunks and no latency: (number of chunks + hop) chunk times - a pipeline fill, then line rate. */
+int echo_chain_arrival_time(double bytes, double chunk_bytes, double Bw_bytes_per_s, int32_t hop,
+                            double hop_latency_s, double *out);
+
 /* ---- stand-alone kernel entry points (used by the parity tests) ---------- */
 
 /* Philox words and uniforms exactly as the sampler draws them: for vocab ids

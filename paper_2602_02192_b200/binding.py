@@ -101,7 +101,11 @@ def _load() -> C.CDLL:
     lib.echo_greedy_provision.argtypes = [C.POINTER(dbl), C.POINTER(dbl), i32, dbl, C.POINTER(C.c_uint8),
                                           C.POINTER(i32), C.POINTER(dbl)]
     lib.echo_admissible.argtypes = [i64, i64, i64]
-    for name in ("echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible"):
+    lib.echo_peer_score.argtypes = [dbl, dbl, i32, i32, dbl, C.POINTER(dbl)]
+    lib.echo_chain_assemble.argtypes = [C.POINTER(dbl), i32, dbl, dbl, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+    lib.echo_chain_arrival_time.argtypes = [dbl, dbl, dbl, i32, dbl, C.POINTER(dbl)]
+    for name in ("echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible",
+                 "echo_peer_score", "echo_chain_assemble", "echo_chain_arrival_time"):
         getattr(lib, name).restype = C.c_int
     lib.echo_gemm_bf16.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]
     lib.echo_decode_attention.argtypes = [vp, vp, i32, vp, i32, vp, vp, i32, i32, i32, i32, i32, vp, C.c_size_t, vp, i32, i32, vp]
@@ -140,7 +144,8 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate",
             "echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible",
             "echo_set_sequence_base", "echo_debug_capture", "echo_debug_wait_limit",
-            "echo_gemm_bf16_noalloc_status", "echo_probe_read_bandwidth"]
+            "echo_gemm_bf16_noalloc_status", "echo_probe_read_bandwidth", "echo_peer_score", "echo_chain_assemble",
+            "echo_chain_arrival_time"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:

@@ -1125,6 +1125,297 @@ attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bf
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, STATUS_WAIT_TIMEOUT);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Prompt prefill on the same tile loop: causal attention of a chunk of prompt tokens over the paged
+// cache, whose K/V rows (this chunk's included) were appended before the launch.  A CTA takes
+// 32 / REP consecutive rows of the chunk and one kv head, i.e. two 16-row MMA tiles of query rows
+// (token-major, REP heads per token), and walks the pages of keys 0..pos like the prefix kernel; a
+// query row attends keys up to its own position, so the tiles on the diagonal are masked per row.
+// A chunk concatenates prompts: where the CTA's rows straddle two prompts it makes one pass per
+// prompt, with the other prompt's rows masked off.
+// ---------------------------------------------------------------------------------------------
+template <int HD, bool HALF>
+__global__ void __launch_bounds__(kDecWarps * 32)
+attn_prefill_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16 *__restrict__ q,
+                    __nv_bfloat16 *__restrict__ out, const int32_t *__restrict__ row_pt,
+                    const int32_t *__restrict__ row_pos, const int32_t *__restrict__ page_table, int pt_width,
+                    int R, int layer_row0, int Hq, int Hkv, int n_pages, float scale_log2, int *status) {
+  constexpr int MT = 2;
+  using S = PreSmem<HD, MT>;
+  constexpr int KSTEPS = HD / 16;
+  constexpr int HALVES = HD / 64;
+  constexpr int CHUNKS = HD / 8;             // 16-byte chunks per query row
+  constexpr int ROWS = MT * 16;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t *q_s = smem + S::kPipeBytes;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + S::kBody);              // [warp][stage]
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + kDecWarps * kDecStages);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int REP = Hq / Hkv;
+  const int TPC = ROWS / REP;                // tokens per CTA
+  const int quad = lane >> 2, qi = lane & 3;
+  const int h = blockIdx.x % Hkv;
+  const int t0 = (blockIdx.x / Hkv) * TPC;   // first chunk row of this CTA
+  const int n_tok = R - t0 < TPC ? R - t0 : TPC;
+
+  early_start_sync();
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kDecWarps * kDecStages; ++i) mbar_init(&bars[i], 1);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  uint8_t *my_stages = smem + warp * kDecStages * S::kStageBytes;
+  uint64_t *my_bars = bars + warp * kDecStages;
+  uint32_t g_iss = 0, g_cons = 0;            // pages requested / consumed by this warp since the start
+  const uint32_t q_addr = smem_u32(q_s);
+  bool ok = true;
+
+  for (int seg_beg = 0; seg_beg < n_tok && ok;) {
+    // ---- the rows of one prompt: [seg_beg, seg_end) ------------------------------------------
+    const int pt_row = row_pt[t0 + seg_beg];
+    int seg_end = seg_beg + 1;
+    while (seg_end < n_tok && row_pt[t0 + seg_end] == pt_row) ++seg_end;
+    const int pos_max = row_pos[t0 + seg_end - 1];       // positions rise by one per row within a prompt
+    const int n_tiles = pos_max / kPageTokens + 1;
+    const int n_my = n_tiles > warp ? (n_tiles - warp + kDecWarps - 1) / kDecWarps : 0;
+    const int32_t *pt = page_table + static_cast<size_t>(pt_row) * pt_width;
+    // keys visible to MMA rows quad and quad + 8 of tile t (0: the row is not part of this pass)
+    int lim[MT][2];
+#pragma unroll
+    for (int t = 0; t < MT; ++t)
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int tok = (t * 16 + quad + 8 * hh) / REP;
+        lim[t][hh] = (tok >= seg_beg && tok < seg_end) ? row_pos[t0 + tok] + 1 : 0;
+      }
+
+    int pg_cache = 0, pg_base = -1;
+    auto page_of = [&](int k) -> int {       // warp-uniform k
+      if (pg_base < 0 || k >= pg_base + 32) {
+        pg_base = k;
+        const int kk = k + lane;
+        pg_cache = kk < n_my ? pt[warp + kDecWarps * kk] : 0;
+      }
+      return __shfl_sync(0xffffffffu, pg_cache, k - pg_base);
+    };
+    auto issue = [&](int k) {
+      const int page = page_of(k);
+      if (lane == 0) {
+        uint64_t *bar = &my_bars[g_iss % kDecStages];
+        uint8_t *dst = my_stages + (g_iss % kDecStages) * S::kStageBytes;
+        if (page < 0 || page >= n_pages) {
+          atomicExch(status, STATUS_BAD_PAGE);
+          mbar_arrive(bar);                  // nothing to load: complete the phase by hand
+        } else {
+          const int row = layer_row0 + (page * Hkv + h) * 2 * kPageTokens;
+          mbar_expect_tx(bar, S::kStageBytes);
+#pragma unroll
+          for (int hf = 0; hf < HALVES; ++hf)
+            tma_load_2d(&tmKV, bar, dst + hf * (S::kStageBytes / HALVES), hf * 64, row);
+        }
+      }
+      ++g_iss;
+    };
+    const int n_pro = n_my < kDecStages ? n_my : kDecStages;
+    for (int k = 0; k < n_pro; ++k) issue(k);
+
+    // ---- queries -> shared memory: row r = (chunk row t0 + r / REP, head h * REP + r % REP) -----
+    for (int c = threadIdx.x; c < ROWS * CHUNKS; c += kDecWarps * 32) {
+      const int r = c / CHUNKS, ch = c % CHUNKS;
+      const int tok = r / REP;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (tok < n_tok)
+        v = *(reinterpret_cast<const uint4 *>(q + (static_cast<size_t>(t0 + tok) * Hq + h * REP + r % REP) * HD) + ch);
+      *reinterpret_cast<uint4 *>(q_s + r * (HD * 2) + ((ch ^ (r & 7)) << 4)) = v;
+    }
+    __syncthreads();
+
+    float o_acc[MT][HD / 8][4];
+    float m_run[MT][2], l_run[MT][2];
+#pragma unroll
+    for (int t = 0; t < MT; ++t) {
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i) o_acc[t][i][0] = o_acc[t][i][1] = o_acc[t][i][2] = o_acc[t][i][3] = 0.f;
+      m_run[t][0] = m_run[t][1] = -INFINITY;
+      l_run[t][0] = l_run[t][1] = 0.f;
+    }
+
+    for (int k = 0; k < n_my; ++k) {
+      ok = mbar_wait(&my_bars[g_cons % kDecStages], (g_cons / kDecStages) & 1, abort_flag);
+      if (!ok) break;
+      const uint32_t st = smem_u32(my_stages + (g_cons % kDecStages) * S::kStageBytes);
+      ++g_cons;
+      const int key0 = (warp + kDecWarps * k) * kPageTokens;
+      // ---- S = Q K^T ------------------------------------------------------------------------------
+      float sc[MT][2][4];
+#pragma unroll
+      for (int t = 0; t < MT; ++t)
+#pragma unroll
+        for (int i = 0; i < 2; ++i) sc[t][i][0] = sc[t][i][1] = sc[t][i][2] = sc[t][i][3] = 0.f;
+      {
+        const int id = lane >> 3, rr = lane & 7;
+        const int key = (id >> 1) * 8 + rr;
+        const int q_row = rr + 8 * (id & 1);
+#pragma unroll
+        for (int kk = 0; kk < KSTEPS; ++kk) {
+          const int c = 2 * (kk & 3) + (id & 1);
+          const uint32_t addr = st + (kk >> 2) * (S::kStageBytes / HALVES) + key * 128 + ((c ^ (key & 7)) << 4);
+          uint32_t b0, b1, b2, b3;
+          ldmatrix_x4(addr, b0, b1, b2, b3);
+#pragma unroll
+          for (int t = 0; t < MT; ++t) {
+            uint32_t a[4];
+            const int qc = 2 * kk + (id >> 1);
+            ldmatrix_x4(q_addr + (t * 16 + q_row) * (HD * 2) + ((qc ^ (q_row & 7)) << 4), a[0], a[1], a[2], a[3]);
+            mma_16816<HALF>(sc[t][0], a, b0, b1);
+            mma_16816<HALF>(sc[t][1], a, b2, b3);
+          }
+        }
+      }
+      // ---- online softmax (exp2 domain), keys beyond a row's own position masked -------------------
+      uint32_t pa[MT][4];
+#pragma unroll
+      for (int t = 0; t < MT; ++t) {
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int key = key0 + 8 * nt + 2 * qi + (e & 1);
+            const float v = key < lim[t][e >> 1] ? sc[t][nt][e] * scale_log2 : -INFINITY;
+            sc[t][nt][e] = v;
+            mx[e >> 1] = fmaxf(mx[e >> 1], v);
+          }
+        float corr[2], msafe[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+          mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+          const float m_new = fmaxf(m_run[t][r], mx[r]);
+          msafe[r] = m_new == -INFINITY ? 0.f : m_new;
+          corr[r] = exp2f(m_run[t][r] - msafe[r]);         // 0 when nothing was accumulated yet
+          m_run[t][r] = m_new;
+        }
+        float ps[2] = {0.f, 0.f};
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            sc[t][nt][e] = exp2f(sc[t][nt][e] - msafe[e >> 1]);
+            ps[e >> 1] += sc[t][nt][e];
+          }
+        l_run[t][0] = l_run[t][0] * corr[0] + ps[0];
+        l_run[t][1] = l_run[t][1] * corr[1] + ps[1];
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i) {
+          o_acc[t][i][0] *= corr[0]; o_acc[t][i][1] *= corr[0];
+          o_acc[t][i][2] *= corr[1]; o_acc[t][i][3] *= corr[1];
+        }
+        pa[t][0] = pack_16<HALF>(sc[t][0][0], sc[t][0][1]);
+        pa[t][1] = pack_16<HALF>(sc[t][0][2], sc[t][0][3]);
+        pa[t][2] = pack_16<HALF>(sc[t][1][0], sc[t][1][1]);
+        pa[t][3] = pack_16<HALF>(sc[t][1][2], sc[t][1][3]);
+      }
+      // ---- O += P V -------------------------------------------------------------------------------
+      {
+        const int id = lane >> 3, rr = lane & 7;
+        const int key = (id & 1) * 8 + rr;
+#pragma unroll
+        for (int dt = 0; dt < KSTEPS; ++dt) {
+          const int c = 2 * (dt & 3) + (id >> 1);
+          const uint32_t addr = st + (dt >> 2) * (S::kStageBytes / HALVES) + kPageTokens * 128 + key * 128 +
+                                ((c ^ (key & 7)) << 4);
+          uint32_t v0, v1, v2, v3;
+          ldmatrix_x4_trans(addr, v0, v1, v2, v3);
+#pragma unroll
+          for (int t = 0; t < MT; ++t) {
+            mma_16816<HALF>(o_acc[t][2 * dt], pa[t], v0, v1);
+            mma_16816<HALF>(o_acc[t][2 * dt + 1], pa[t], v2, v3);
+          }
+        }
+      }
+      __syncwarp();
+      if (k + kDecStages < n_my) issue(k + kDecStages);
+    }
+    if (!ok) break;
+#pragma unroll
+    for (int t = 0; t < MT; ++t)
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        l_run[t][r] += __shfl_xor_sync(0xffffffffu, l_run[t][r], 1);
+        l_run[t][r] += __shfl_xor_sync(0xffffffffu, l_run[t][r], 2);
+      }
+    // ---- combine the four warps through shared memory (pipeline and query buffers are idle now) --
+    __syncthreads();
+    float *m_s = reinterpret_cast<float *>(smem);                      // [warp][ROWS]
+    float *l_s = m_s + kDecWarps * ROWS;
+    float *o_s = l_s + kDecWarps * ROWS;                               // [warp][ROWS][kRowStride]
+#pragma unroll
+    for (int t = 0; t < MT; ++t) {
+      const int r_lo = t * 16 + quad, r_hi = r_lo + 8;
+      if (qi == 0) {
+        m_s[warp * ROWS + r_lo] = m_run[t][0];
+        m_s[warp * ROWS + r_hi] = m_run[t][1];
+        l_s[warp * ROWS + r_lo] = l_run[t][0];
+        l_s[warp * ROWS + r_hi] = l_run[t][1];
+      }
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i) {
+        *reinterpret_cast<float2 *>(o_s + (warp * ROWS + r_lo) * S::kRowStride + 8 * i + 2 * qi) =
+            make_float2(o_acc[t][i][0], o_acc[t][i][1]);
+        *reinterpret_cast<float2 *>(o_s + (warp * ROWS + r_hi) * S::kRowStride + 8 * i + 2 * qi) =
+            make_float2(o_acc[t][i][2], o_acc[t][i][3]);
+      }
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < ROWS * HD; idx += blockDim.x) {
+      const int r = idx / HD, d = idx % HD;
+      const int tok = r / REP;
+      if (tok < seg_beg || tok >= seg_end) continue;
+      float M = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kDecWarps; ++w) M = fmaxf(M, m_s[w * ROWS + r]);
+      float L = 0.f, O = 0.f;
+#pragma unroll
+      for (int w = 0; w < kDecWarps; ++w) {
+        const float mw = m_s[w * ROWS + r];
+        if (mw != -INFINITY) {
+          const float c = exp2f(mw - M);
+          L += l_s[w * ROWS + r] * c;
+          O += o_s[(w * ROWS + r) * S::kRowStride + d] * c;
+        }
+      }
+      reinterpret_cast<uint16_t *>(out)[(static_cast<size_t>(t0 + tok) * Hq + h * REP + r % REP) * HD + d] =
+          cvt16(O / L, HALF);
+    }
+    seg_beg = seg_end;
+    if (seg_beg < n_tok) {
+      // another prompt's rows follow: the merge area is handed back to the copy engine
+      __syncthreads();
+      fence_proxy_async();
+    }
+  }
+  if (*abort_flag) {
+    for (uint32_t g = g_cons; g < g_iss; ++g) mbar_drain(&my_bars[g % kDecStages], (g / kDecStages) & 1);
+    if (threadIdx.x == 0) atomicExch(status, STATUS_WAIT_TIMEOUT);
+  }
+}
+
+template <int HD, bool HALF>
+cudaError_t launch_prefill(const PrefillAttnArgs &a, cudaStream_t s) {
+  const int REP = a.Hq / a.Hkv;
+  const int TPC = 32 / REP;
+  const float scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(HD));
+  return launch_early(attn_prefill_kernel<HD, HALF>, dim3(((a.R + TPC - 1) / TPC) * a.Hkv), dim3(kDecWarps * 32),
+                      PreSmem<HD, 2>::kTotal, s, *a.tmKV, a.q, a.out, a.row_pt, a.row_pos, a.page_table, a.pt_width,
+                      a.R, a.layer_row0, a.Hq, a.Hkv, a.n_pages, scale_log2, a.status);
+}
+
 // CTAs of the resident suffix kernel that fit the current device at once (cached per device, head
 // dimension, operand format and group ratio; no stream work).
 template <int HD, bool HALF>
@@ -1187,6 +1478,8 @@ cudaError_t configure_decode() {
                                 DecSmem<HD>::kTotal)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(attn_prefix_group_kernel<HD, 2, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 PreSmem<HD, 2>::kTotal)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(attn_prefill_kernel<HD, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                PreSmem<HD, 2>::kTotal)) != cudaSuccess) return e;
   return cudaFuncSetAttribute(attn_suffix_resident_kernel<HD, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               SufSmem<HD>::total(kSufPre * kDecWarps * 32 / HD));
 }
@@ -1204,6 +1497,14 @@ cudaError_t attention_decode_configure() {
 bool attention_decode_supported(int hd, int page_size, int Hq, int Hkv) {
   const int rep = Hq / Hkv;
   return (hd == 64 || hd == 128) && page_size == kPageTokens && rep >= 1 && rep <= 16;
+}
+
+cudaError_t attention_prefill_launch(const PrefillAttnArgs &a, cudaStream_t s) {
+  const int rep = a.Hkv > 0 ? a.Hq / a.Hkv : 0;
+  if (rep != 1 && rep != 2 && rep != 4 && rep != 8) return cudaErrorInvalidValue;
+  if (a.hd == 128) return a.half_io ? launch_prefill<128, true>(a, s) : launch_prefill<128, false>(a, s);
+  if (a.hd == 64) return a.half_io ? launch_prefill<64, true>(a, s) : launch_prefill<64, false>(a, s);
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t attention_decode_launch(const DecodeAttnArgs &a, cudaStream_t s) {

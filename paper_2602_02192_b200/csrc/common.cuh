@@ -250,6 +250,22 @@ struct DecodeAttnArgs {
   int suffix_impl = 0;            // 0: choose; 1: always one suffix CTA per (sequence, kv head)
   int prefix_impl = 0;            // 0: choose; 1: always one prefix CTA per 16-row tile
 };
+// Causal attention of a chunk of R prompt tokens (rows of q / out) over the paged cache; row r belongs
+// to page-table row row_pt[r] at position row_pos[r]; consecutive rows of one prompt have consecutive
+// positions.  Needs 16-token pages and Hq / Hkv in {1, 2, 4, 8} (attention_decode_supported).
+struct PrefillAttnArgs {
+  const CUtensorMap *tmKV;        // as in DecodeAttnArgs
+  const __nv_bfloat16 *q;         // [R][Hq][hd]
+  __nv_bfloat16 *out;             // [R][Hq][hd]
+  const int32_t *row_pt, *row_pos;
+  const int32_t *page_table;
+  int pt_width, R;
+  int layer_row0;
+  int Hq, Hkv, hd, n_pages;
+  int *status;
+  int half_io;
+};
+cudaError_t attention_prefill_launch(const PrefillAttnArgs &a, cudaStream_t s);
 cudaError_t attention_decode_configure();
 bool attention_decode_supported(int hd, int page_size, int Hq, int Hkv);
 cudaError_t attention_decode_launch(const DecodeAttnArgs &a, cudaStream_t s);

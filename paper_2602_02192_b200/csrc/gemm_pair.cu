@@ -130,10 +130,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();                // 0 = the CTA that issues the pair's MMAs
-  const int pair = blockIdx.x >> 1;
+  // pairs are numbered with the row tile fastest: the pairs that share a weight tile run side by side,
+  // so the tile comes from HBM once and from L2 for the other row tiles
+  const int m_tiles = (M + BNB - 1) / BNB;
+  const int pair = (blockIdx.x >> 1) / m_tiles;
   const int nt = pair / split;
   const int slice = pair % split;
-  const int m0 = blockIdx.y * BNB;
+  const int m0 = ((blockIdx.x >> 1) % m_tiles) * BNB;
   const int KB = (K + kGemmTileK - 1) / kGemmTileK;
   const int kq = KB / split, kr = KB % split;
   const int kb_beg = slice * kq + min(slice, kr);
@@ -317,7 +320,7 @@ cudaError_t launch_pair(const PairGemmArgs &a, int n_tiles, int m_tiles, int spl
   if (make_out_map_box(&tmY, a.Y, a.M, a.N, a.ldY, bf16_out, bf16_out ? 64 : kPairFeat, 32) != 0)
     return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * n_tiles * split, m_tiles, 1);
+  cfg.gridDim = dim3(2 * n_tiles * split * m_tiles, 1, 1);
   cfg.blockDim = dim3(kPairThreads, 1, 1);
   cfg.dynamicSmemBytes = S::kTotal;
   cfg.stream = stream;

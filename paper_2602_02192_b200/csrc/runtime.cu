@@ -19,7 +19,9 @@ namespace {
 
 constexpr size_t kAlign = 1024;
 constexpr size_t kRetileStageBytes = 64ull << 20;
-constexpr int kChunkRows = 256;       // prompt tokens per prefill forward
+constexpr int kChunkRows = 2048;      // prompt tokens per prefill forward: eight 256-row activation tiles share
+                                      // every weight tile (read from HBM once, seven times from L2)
+constexpr int kSmallChunkRows = 256;  // ... with the plain SIMT projection kernel (debugging aid)
 constexpr int kMaxCtas = 160;         // persistent GEMM grid never exceeds this (148 SMs on B200)
 
 size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
@@ -37,7 +39,7 @@ struct Dims {
 };
 
 struct Limits {
-  int P, G, Lp, T, B, R;            // R = rows of the activation buffers
+  int P, G, Lp, T, B, R;            // R = rows of the activation buffers (a prefill chunk or a decode step)
   int n_pre, n_dec, n_pages, pt_width, max_pos;
 };
 
@@ -108,12 +110,14 @@ Layout layout_of(const echo_config &c) {
   lo.q = take(static_cast<size_t>(M.R) * D.Hq * D.hd * 2);
   lo.attn = take(static_cast<size_t>(M.R) * D.Hq * D.hd * 2);
   lo.act = take(static_cast<size_t>(M.R) * D.F * 2);
-  lo.gu = take(static_cast<size_t>(M.R) * 2 * D.F * 4);
-  lo.xlast = take(static_cast<size_t>(M.R) * D.d * 4);
-  lo.hlast = take(static_cast<size_t>(M.R) * D.d * 2);
-  lo.logits = take(static_cast<size_t>(M.R) * D.V * 4);
+  // gate / up pre-activations of the SIMT path (chunks of kSmallChunkRows there); last-position rows,
+  // their normed copy and the logits: one row per sequence at most
+  lo.gu = take(static_cast<size_t>(std::max(M.B, kSmallChunkRows)) * 2 * D.F * 4);
+  lo.xlast = take(static_cast<size_t>(M.B) * D.d * 4);
+  lo.hlast = take(static_cast<size_t>(M.B) * D.d * 2);
+  lo.logits = take(static_cast<size_t>(M.B) * D.V * 4);
   const size_t n_pre_tok = static_cast<size_t>(M.P) * M.Lp;
-  lo.n_chunks_max = static_cast<int>((n_pre_tok + kChunkRows - 1) / kChunkRows);
+  lo.n_chunks_max = static_cast<int>((n_pre_tok + kSmallChunkRows - 1) / kSmallChunkRows);
   lo.page_table = take(static_cast<size_t>(M.B + M.P) * M.pt_width * 4);
   lo.pre_row_pt = take(n_pre_tok * 4);
   lo.pre_row_pos = take(n_pre_tok * 4);
@@ -184,6 +188,8 @@ struct echo_ctx {
   bool use_simt = false, use_graph = true, fast_decode = false, deterministic = false, use_pdl = true, use_pair = true;
   bool long_suffix = false;   // decode steps whose sequences hold many generated tokens (see kLongSuffix)
   int attn_suffix_impl = 0, attn_prefix_impl = 0;   // diagnostic kernel choices (ECHO_ATTN_IMPL / ECHO_ATTN_PREFIX)
+  int chunk_rows = kChunkRows;
+  bool prefill_rows = false;  // ECHO_ATTN_PREFILL=rows: the one-query-per-row kernel for the prompt prefill too
   uint32_t seq_base = 0;      // added to p * G + g in the noise streams (echo_set_sequence_base)
   // parity hook (echo_debug_capture): residual stream before / after one layer
   int cap_layer = -1;
@@ -374,6 +380,13 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int d
                         ctx->attn_prefix_impl};
       LAUNCH(attention_decode_launch(da, ctx->stream));
       ctx->launches++;                      // two kernels per call
+    } else if (decode_P == 0 && ctx->fast_decode && !ctx->prefill_rows) {
+      // prompt prefill: causal attention of the chunk on the warp-level tensor-core tile loop
+      ProfScope prof(ctx, PROF_ATTN);
+      PrefillAttnArgs pa{&ctx->tm_kv, q, attn, meta.row_pt, meta.row_pos, pt, ctx->M.pt_width, R,
+                         static_cast<int>(static_cast<size_t>(l) * (lo.kv_layer_elems / D.hd)), D.Hq, D.Hkv, D.hd,
+                         ctx->M.n_pages, status, hf ? 1 : 0};
+      LAUNCH(attention_prefill_launch(pa, ctx->stream));
     } else {
       ProfScope prof(ctx, PROF_ATTN);
       LAUNCH(attention_rows_launch(q, kv_layer, attn, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
@@ -538,7 +551,8 @@ int build_plan(echo_ctx *ctx, const int32_t *lens, int P, int G, int T, Plan *pl
   if (next_page > M.n_pages) return ECHO_ERR_INVALID;
   int n_tok = 0;
   for (int p = 0; p < P; ++p) n_tok += lens[p];
-  const int n_chunks = ceil_div(n_tok, kChunkRows);
+  const int chunk = ctx->chunk_rows;
+  const int n_chunks = ceil_div(n_tok, chunk);
   std::fill(h_gather, h_gather + static_cast<size_t>(n_chunks) * P, -1);
   int i = 0;
   for (int p = 0; p < P; ++p) {
@@ -548,7 +562,7 @@ int build_plan(echo_ctx *ctx, const int32_t *lens, int P, int G, int T, Plan *pl
       h_tok_idx[i] = p * M.Lp + t;
     }
     const int last = i - 1;
-    h_gather[static_cast<size_t>(last / kChunkRows) * P + p] = last % kChunkRows;
+    h_gather[static_cast<size_t>(last / chunk) * P + p] = last % chunk;
   }
   *plan = Plan{P, G, T, B, n_tok, n_chunks, n_copies, next_page, W};
   ctx->last_table.assign(h_pt, h_pt + static_cast<size_t>(B) * W);
@@ -661,11 +675,11 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   }
   if (ctx->cfg.eos_id >= 0)       // no sequence has ended yet
     CK(cudaMemsetAsync(ctx->arena + lo.row_done, 0, static_cast<size_t>(pl.B) * 4, ctx->stream));
-  // ---- prefill: once per prompt, in chunks of kChunkRows tokens -------------
+  // ---- prefill: once per prompt, in chunks of ctx->chunk_rows tokens --------
   cudaEvent_t pf_a = nullptr, pf_b = nullptr;
   if (ctx->prof_now && (pf_a = prof_event(ctx)) && (pf_b = prof_event(ctx))) cudaEventRecord(pf_a, ctx->stream);
   for (int c = 0; c < pl.n_chunks; ++c) {
-    const int r0 = c * kChunkRows, R = std::min(kChunkRows, pl.n_tok - r0);
+    const int r0 = c * ctx->chunk_rows, R = std::min(ctx->chunk_rows, pl.n_tok - r0);
     LAUNCH(embed_launch(w.embed, prompts, ctx->ptr<int32_t>(lo.pre_tok_idx) + r0, x, R, D.d, D.V, status,
                         ctx->stream));
     RowMeta meta{ctx->ptr<int32_t>(lo.pre_row_pt) + r0, ctx->ptr<int32_t>(lo.pre_row_pos) + r0, nullptr};
@@ -803,6 +817,7 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
   ctx->stream = static_cast<cudaStream_t>(cuda_stream);
   const char *impl = getenv("ECHO_GEMM_IMPL");
   ctx->use_simt = impl && !strcmp(impl, "simt");
+  ctx->chunk_rows = ctx->use_simt ? kSmallChunkRows : kChunkRows;
   ctx->use_pair = !(impl && !strcmp(impl, "single"));
   const char *ng = getenv("ECHO_NO_GRAPH");
   ctx->use_graph = !(ng && ng[0] == '1');
@@ -861,6 +876,8 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
     const char *np = getenv("ECHO_ATTN_PREFIX");
     ctx->attn_suffix_impl = na && !strcmp(na, "waves") ? 1 : 0;
     ctx->attn_prefix_impl = np && !strcmp(np, "tiles") ? 1 : 0;
+    const char *npf = getenv("ECHO_ATTN_PREFILL");
+    ctx->prefill_rows = npf && !strcmp(npf, "rows");
     const size_t kv_rows = lo.kv_layer_elems / ctx->D.hd * ctx->D.L;
     if (!(na && !strcmp(na, "rows")) && kv_rows < (1ull << 31) &&
         attention_decode_supported(ctx->D.hd, ctx->D.Z, ctx->D.Hq, ctx->D.Hkv)) {

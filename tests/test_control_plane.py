@@ -98,3 +98,90 @@ def test_library_matches_oracle(lib):
         assert math.isclose(c.value, want_c, rel_tol=1e-12, abs_tol=1e-12)
     for v, vt, S in [(7, 10, 3), (6, 10, 3), (10, 10, 0), (11, 10, 3), (5, 5, -1)]:
         assert lib.echo_admissible(v, vt, S) == int(S >= 0 and control.admissible(v, vt, S))
+
+
+# ---- Appendix C.3: peer score, chain assembly; Section 4.3: store-and-forward timeline ---------------
+
+def test_peer_score_facts_of_the_appendix():
+    # Speed saturates at 100 when the forwarding rate reaches 100 Mbit/s (log10 = 8)
+    best = control.peer_score(1e8, 1.0, 10, 0, 0.0)
+    assert math.isclose(best, 100.0, rel_tol=1e-12)
+    assert control.peer_score(1e9, 1.0, 10, 0, 0.0) == best                    # no credit beyond the cap
+    # weights 0.5 / 0.35 / 0.15, each term alone
+    assert math.isclose(control.peer_score(1e8, 0.0, 0, 0, 0.0), 50.0)
+    assert math.isclose(control.peer_score(1e3, 1.0, 0, 0, 0.0), 35.0)          # log10 = 3: Speed 0
+    assert math.isclose(control.peer_score(1e3, 0.0, 10, 0, 0.0), 15.0)
+    assert math.isclose(control.peer_score(1e3, 0.0, 5, 3, 0.0), 7.5)           # 5 of 10 successes, 3 failures still count
+    assert control.peer_score(1e3, 0.0, 10, 4, 0.0) == 0.0                      # more than 3 consecutive failures
+    # Speed is linear in log10 between 1 kbit/s and the cap: 10^5.5 is half way
+    assert math.isclose(control.peer_score(10 ** 5.5, 0.0, 0, 0, 0.0), 25.0, rel_tol=1e-12)
+    # Decay: 1 at once, 0.85 after 90 s, floor 0.7 from 180 s on
+    assert math.isclose(control.peer_score(1e8, 1.0, 10, 0, 90.0), 85.0)
+    assert math.isclose(control.peer_score(1e8, 1.0, 10, 0, 180.0), 70.0)
+    assert control.peer_score(1e8, 1.0, 10, 0, 1e6) == control.peer_score(1e8, 1.0, 10, 0, 180.0)
+
+
+def test_chain_assembly_rules():
+    scores = [10.0, 90.0, 50.0, 70.0, 30.0, 70.0, 20.0]
+    chains = control.chain_assemble(scores, 300.0, 100.0)                        # floor(300 / 100) = 3 chains
+    assert [c[0] for c in chains] == [1, 3, 5]                                  # the three best seed them (tie: lower index)
+    # ranking: 1 (90), 3 and 5 (70), 2 (50), 4 (30), 6 (20), 0 (10); ranks 3.. go to chains 0, 1, 2, 0, ...
+    assert chains == [[1, 2, 0], [3, 4], [5, 6]]
+    flat = sorted(w for c in chains for w in c)
+    assert flat == list(range(len(scores)))                                     # every worker in exactly one chain
+    assert len(control.chain_assemble(scores, 50.0, 100.0)) == 1                # an uplink below one worker's rate: one chain
+    assert len(control.chain_assemble(scores, 1e9, 100.0)) == len(scores)       # never more chains than workers (a star)
+    assert control.chain_assemble([], 300.0, 100.0) == []
+
+
+def test_store_and_forward_timeline_closed_forms():
+    Bw = 100.0
+    # one chunk: pure store and forward, the whole snapshot crosses hop + 1 links one after the other
+    assert math.isclose(control.chain_arrival_time(1000, 1000, Bw, 3), 4 * 10.0)
+    # equal chunks: (n_chunks + hop) chunk times - a pipeline fill, then line rate
+    for n_chunks, hop in [(10, 0), (10, 4), (64, 7), (1, 5)]:
+        t = control.chain_arrival_time(100 * n_chunks, 100, Bw, hop)
+        assert math.isclose(t, (n_chunks + hop) * 1.0)
+    # finer chunks approach the line rate bytes / Bw whatever the hop
+    assert control.chain_arrival_time(10000, 1, Bw, 7) < 100.0 * 1.001
+    # a shorter last chunk: brute force against the recurrence written out by hand for 2 chunks, 2 links
+    # sizes 100 and 50: link 0 ends them at 1.0 and 1.5; link 1 starts them at 1.0 and max(1.5, 2.0), ends at 2.5
+    assert math.isclose(control.chain_arrival_time(150, 100, Bw, 1), 2.5)
+    # per-hop latency is paid once per link by the last chunk when the links are otherwise idle for it
+    assert math.isclose(control.chain_arrival_time(100, 100, Bw, 2, hop_latency=0.25), 3 * (1.0 + 0.25))
+    # a deeper hop never holds the snapshot earlier
+    ts = [control.chain_arrival_time(12345, 1000, Bw, h, 0.01) for h in range(6)]
+    assert all(b > a for a, b in zip(ts, ts[1:]))
+
+
+def test_library_peer_score_chains_and_timeline_match_the_oracle(lib):
+    rng = np.random.default_rng(5)
+    out = C.c_double()
+    for _ in range(300):
+        a = (float(10 ** rng.uniform(1, 10)), float(rng.uniform(0, 1)), int(rng.integers(0, 25)),
+             int(rng.integers(0, 7)), float(rng.uniform(0, 1200)))
+        assert lib.echo_peer_score(*a, C.byref(out)) == 0
+        assert math.isclose(out.value, control.peer_score(*a), rel_tol=1e-12, abs_tol=1e-12)
+    assert lib.echo_peer_score(0.0, 0.5, 3, 0, 0.0, C.byref(out)) == 0 and math.isclose(out.value, 0.35 * 50 + 0.15 * 30)
+    assert lib.echo_peer_score(1e6, 1.5, 3, 0, 0.0, C.byref(out)) == -1
+    for _ in range(100):
+        n = int(rng.integers(0, 40))
+        scores = np.round(rng.uniform(0, 100, size=n), 0)                        # rounded: ties happen
+        B0, Bw = float(rng.uniform(50, 2000)), float(rng.choice([50.0, 100.0, 300.0]))
+        chain_of = (C.c_int32 * max(n, 1))()
+        hop_of = (C.c_int32 * max(n, 1))()
+        n_ch = C.c_int32()
+        rc = lib.echo_chain_assemble(scores.ctypes.data_as(C.POINTER(C.c_double)), n, B0, Bw, chain_of, hop_of,
+                                     C.byref(n_ch))
+        assert rc == 0
+        want = control.chain_assemble(list(scores), B0, Bw)
+        assert n_ch.value == len(want)
+        for c, chain in enumerate(want):
+            for h, w in enumerate(chain):
+                assert chain_of[w] == c and hop_of[w] == h
+    for _ in range(200):
+        n_bytes = float(rng.integers(1, 10 ** 7))
+        chunk = float(rng.integers(1, 10 ** 6))
+        Bw, hop, lat = float(rng.uniform(1e3, 1e6)), int(rng.integers(0, 12)), float(rng.uniform(0, 0.01))
+        assert lib.echo_chain_arrival_time(n_bytes, chunk, Bw, hop, lat, C.byref(out)) == 0
+        assert math.isclose(out.value, control.chain_arrival_time(n_bytes, chunk, Bw, hop, lat), rel_tol=1e-9)

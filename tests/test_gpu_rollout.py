@@ -403,3 +403,28 @@ def test_prompts_cut_over_contexts_reproduce_one_call(B, tiny):
             assert_same_rollout(tok.cpu().numpy()[0], lp.cpu().numpy()[0], tok_all[p], lp_all[p])
     eng.echo_set_sequence_base(0)
     eng.close()
+
+
+@pytest.mark.parametrize("prefill", ["tiles", "rows"])
+def test_prefill_attention_kernels(B, tiny, monkeypatch, prefill):
+    """Prompt prefill with the tensor-core tile kernel (default) and with the one-query-per-row kernel
+    (ECHO_ATTN_PREFILL=rows, also what serves page sizes other than 16): ragged prompts whose rows
+    straddle prompt boundaries inside one CTA, lengths that are not multiples of the page size, a
+    one-token prompt; every token against the oracle, with bf16 and with half operands."""
+    wl, w_o, w_d = tiny
+    if prefill == "rows":
+        monkeypatch.setenv("ECHO_ATTN_PREFILL", "rows")
+    else:
+        monkeypatch.delenv("ECHO_ATTN_PREFILL", raising=False)
+    lens_list = [37, 3, 1, 64, 18, 5, 33]
+    P, G, Lp, T = len(lens_list), 2, 64, 6
+    prompts, lens = synth.make_ragged_prompts(lens_list, wl.shape.vocab, 404, pad_to=Lp)
+    for hl in (0, 2):
+        eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, half_layers=hl))
+        eng.echo_load_policy(w_d, 1)
+        tok, lp, _ = eng.echo_rollout(torch.from_numpy(prompts).cuda(), lens, G, T, 1.0, 808)
+        eng.echo_sync()
+        n, ex, worst = check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 1.0, 808, tok.cpu().numpy(),
+                                       lp.cpu().numpy(), range(P * G))
+        assert n == P * G * T and ex <= 3
+        eng.close()
