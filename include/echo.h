@@ -173,6 +173,28 @@ int echo_rollout_forced(echo_ctx *ctx, const int32_t *prompts, const int32_t *pr
                         uint64_t seed, const int32_t *forced_tokens, int32_t *out_tokens,
                         float *out_logprobs, int64_t *out_versions);
 
+/* Learner-side scoring (Appendix F: the likelihood ratio and the truncated importance ratio need
+ * log pi_theta(y_t | x, y_<t) for whole trajectories from the buffer).  Same result as the
+ * out_logprobs of echo_rollout_forced for the same given tokens, but computed in prefill-shaped passes
+ * (the prompt once per group, then every sequence's given tokens as rows of large chunks with causal
+ * attention): the weights are streamed once per 2048 rows instead of once per decode step.
+ *   tokens       dev int32 [P][G][T]: the given trajectories
+ *   out_logprobs dev fp32  [P][G][T]: log-probability of tokens[p][g][j] under softmax(z / temperature)
+ *                of the installed snapshot (the full distribution: top_p is not applied); with an end
+ *                token configured, positions after a sequence's first end token score 0.
+ * Arguments otherwise as for echo_rollout; asynchronous on the context's stream. */
+int echo_score(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int32_t P, int32_t G,
+               int32_t max_new_tokens, float temperature, const int32_t *tokens, float *out_logprobs,
+               int64_t *out_versions);
+
+/* Turn-aware response mask (Appendix F, "Turn-Aware Masking"): with u_t = [x_t == turn_start_id] and
+ * c_t = u_0 + ... + u_t, m_t = [c_t > 1] * [c_t odd] selects the tokens of assistant turns after the
+ * system prompt.  tokens dev int32 [n][T] -> out_mask dev uint8 [n][T].  With shift_to_targets != 0 the
+ * mask is aligned with next-token targets y_t = x_{t+1}: out[t] = m_{t+1}, out[T-1] = 0.  The result is
+ * the `mask` argument of echo_grpo_surrogate.  Asynchronous on the stream; needs no context. */
+int echo_turn_mask(const int32_t *tokens, int32_t n, int32_t T, int32_t turn_start_id, int32_t shift_to_targets,
+                   uint8_t *out_mask, void *cuda_stream);
+
 /* echo_rollout with every buffer in HOST memory (prompts, outputs): copies the
  * prompts in, runs the rollout, copies tokens and log-probabilities out and
  * synchronises.  Page-locked buffers make the copies asynchronous. */

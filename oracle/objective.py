@@ -51,3 +51,27 @@ def grpo_surrogate(logp_new, logp_old, logp_sampler, adv, mask, eps_clip: float,
             den += 1.0
         out[i] = num / den if den > 0.0 else 0.0
     return out
+
+
+def turn_mask(tokens, turn_start_id: int, shift_to_targets: bool = False) -> np.ndarray:
+    """Appendix F, "Turn-Aware Masking": u_t = [x_t == turn_start], c_t = u_0 + ... + u_t (the chat-turn
+    index of token t), m_t = [c_t > 1] * [c_t mod 2 == 1]: tokens of assistant turns after the system
+    prompt.  tokens [n][T] -> uint8 [n][T].  shift_to_targets aligns the mask with next-token targets
+    y_t = x_{t+1}: out[t] = m_{t+1}, last column 0.
+
+    Pins: a hand-written five-turn dialogue; no turn-start token or a single one gives an empty mask;
+    the mask is a function of the turn index only."""
+    x = np.asarray(tokens)
+    n, T = x.shape
+    m = np.zeros((n, T), dtype=np.uint8)
+    for i in range(n):
+        c = 0
+        for t in range(T):
+            if x[i, t] == turn_start_id:
+                c += 1
+            m[i, t] = 1 if (c > 1 and c % 2 == 1) else 0
+    if shift_to_targets:
+        out = np.zeros_like(m)
+        out[:, : T - 1] = m[:, 1:]
+        return out
+    return m

@@ -74,6 +74,10 @@ def _load() -> C.CDLL:
     lib.echo_rollout.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp]
     lib.echo_rollout_forced.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp, vp]
     lib.echo_rollout_host.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp]
+    lib.echo_score.argtypes = [vp, vp, vp, i32, i32, i32, f32, vp, vp, vp]
+    lib.echo_score.restype = C.c_int
+    lib.echo_turn_mask.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+    lib.echo_turn_mask.restype = C.c_int
     lib.echo_group_advantage.argtypes = [vp, i32, i32, f32, vp, vp]
     lib.echo_sync.argtypes = [vp]
     lib.echo_get_stats.argtypes = [vp, C.POINTER(EchoStats)]
@@ -145,7 +149,7 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible",
             "echo_set_sequence_base", "echo_debug_capture", "echo_debug_wait_limit",
             "echo_gemm_bf16_noalloc_status", "echo_probe_read_bandwidth", "echo_peer_score", "echo_chain_assemble",
-            "echo_chain_arrival_time"]
+            "echo_chain_arrival_time", "echo_score", "echo_turn_mask"]
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -265,6 +269,23 @@ class Engine:
         _check(rc, self._ctx)
         return out_tokens, out_logprobs, versions
 
+    def echo_score(self, prompts: torch.Tensor, prompt_lens: Sequence[int], tokens: torch.Tensor, temperature: float,
+                   out_logprobs: Optional[torch.Tensor] = None):
+        """Log-probabilities of given trajectories (int32 cuda [P][G][T]) in prefill-shaped passes.
+        Returns (logprobs fp32 [P][G][T] on the device, versions)."""
+        P, G, T = tokens.shape
+        assert prompts.dtype == torch.int32 and prompts.is_cuda and prompts.is_contiguous()
+        assert prompts.shape == (P, self.cfg.max_prompt_len)
+        assert tokens.dtype == torch.int32 and tokens.is_cuda and tokens.is_contiguous()
+        lens = np.ascontiguousarray(np.asarray(prompt_lens, dtype=np.int32))
+        if out_logprobs is None:
+            out_logprobs = torch.empty((P, G, T), dtype=torch.float32, device=self.device)
+        versions = np.zeros((P, G), dtype=np.int64)
+        self.stream.wait_stream(torch.cuda.current_stream(self.device))
+        _check(lib.echo_score(self._ctx, prompts.data_ptr(), lens.ctypes.data, P, G, T, float(temperature),
+                              tokens.data_ptr(), out_logprobs.data_ptr(), versions.ctypes.data), self._ctx)
+        return out_logprobs, versions
+
     def echo_rollout_host(self, prompts: torch.Tensor, prompt_lens: Sequence[int], G: int, max_new_tokens: int,
                           temperature: float, seed: int, out_tokens: torch.Tensor, out_logprobs: torch.Tensor):
         """All buffers are host tensors (ideally pinned); returns versions.  Synchronous."""
@@ -332,6 +353,17 @@ def echo_group_advantage(rewards: torch.Tensor, eps: float = 1e-6, out: Optional
         out = torch.empty_like(rewards)
     with torch.cuda.device(rewards.device):
         _check(lib.echo_group_advantage(rewards.data_ptr(), P, G, float(eps), out.data_ptr(), _stream_ptr(stream)))
+    return out
+
+
+def echo_turn_mask(tokens: torch.Tensor, turn_start_id: int, shift_to_targets: bool = False) -> torch.Tensor:
+    """uint8 [n][T] response mask of int32 token rows [n][T] (Appendix F, turn-aware masking)."""
+    assert tokens.is_cuda and tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.dim() == 2
+    n, T = tokens.shape
+    out = torch.empty((n, T), dtype=torch.uint8, device=tokens.device)
+    with torch.cuda.device(tokens.device):
+        _check(lib.echo_turn_mask(tokens.data_ptr(), n, T, int(turn_start_id), 1 if shift_to_targets else 0,
+                                  out.data_ptr(), _stream_ptr(None)))
     return out
 
 

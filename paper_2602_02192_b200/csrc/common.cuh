@@ -213,6 +213,15 @@ cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float 
                                   const uint8_t *mask, int n, int T, float eps_clip, float C, float *out,
                                   cudaStream_t s);
 cudaError_t set_int_launch(int32_t *p, int32_t v, cudaStream_t s);
+// teacher-forced scoring of whole trajectories (see the kernels in elementwise.cu)
+cudaError_t score_rows_launch(int r0, int R, int T, const int32_t *seq_len0, int32_t *row_pt, int32_t *row_pos,
+                              int32_t *tok_idx, cudaStream_t s);
+cudaError_t first_end_launch(const int32_t *tokens, int B, int T, int eos_id, int32_t *first_end, cudaStream_t s);
+cudaError_t logprob_rows_launch(const float *logits, int rows, int V, int rows_per_logit_row, float temperature,
+                                const int32_t *tokens, const int32_t *tok_idx, int T, const int32_t *first_end,
+                                float *out, int *status, cudaStream_t s);
+cudaError_t turn_mask_launch(const int32_t *tokens, int n, int T, int turn_start, int shift, uint8_t *out,
+                             cudaStream_t s);
 // copies n floats (a multiple of 4) of x into slot (*d_step - 1) of dst
 cudaError_t capture_step_launch(const float *x, float *dst, const int32_t *d_step, size_t n, cudaStream_t s);
 // reads `bytes` (a multiple of 16) of buf once with n_blocks blocks of 512 threads; writes nothing

@@ -337,6 +337,92 @@ __global__ void decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int
 
 __global__ void set_int_kernel(int32_t *p, int32_t v) { *p = v; }
 
+__device__ __forceinline__ void lse_update(float &m, float &l, float s);
+__device__ __forceinline__ void lse_merge(float &m, float &l, float m2, float l2);
+
+// Rows of a teacher-forced scoring chunk, sequence-major: row r0 + i is token j = (r0 + i) % (T - 1) of
+// sequence s = (r0 + i) / (T - 1): it feeds given token j at position len0[s] + j.
+__global__ void score_rows_kernel(int r0, int R, int T, const int32_t *seq_len0, int32_t *row_pt, int32_t *row_pos,
+                                  int32_t *tok_idx) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= R) return;
+  const int r = r0 + i, s = r / (T - 1), j = r % (T - 1);
+  row_pt[i] = s;
+  row_pos[i] = seq_len0[s] + j;
+  tok_idx[i] = s * T + j;
+}
+
+// first_end[s] = index of the first end token among the T given tokens of sequence s (T if none)
+__global__ void first_end_kernel(const int32_t *tokens, int B, int T, int eos_id, int32_t *first_end) {
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= B) return;
+  int e = T;
+  if (eos_id >= 0)
+    for (int j = 0; j < T; ++j)
+      if (tokens[static_cast<size_t>(s) * T + j] == eos_id) {
+        e = j;
+        break;
+      }
+  first_end[s] = e;
+}
+
+// Log-probability of given tokens: row r of the launch reads logits row r / rows_per_logit_row and
+// scores token tokens[flat], flat = tok_idx ? tok_idx[r] + 1 : r * T (the first token of sequence r),
+// under softmax(z / temperature); positions after a sequence's end token score 0.
+__global__ void __launch_bounds__(512)
+logprob_rows_kernel(const float *logits, int V, int rows_per_logit_row, float inv_temperature, const int32_t *tokens,
+                    const int32_t *tok_idx, int T, const int32_t *first_end, float *out, int *status) {
+  __shared__ float sm_m[16], sm_l[16];
+  const int r = blockIdx.x;
+  const size_t flat = tok_idx ? static_cast<size_t>(tok_idx[r]) + 1 : static_cast<size_t>(r) * T;
+  const int s = static_cast<int>(flat / T), j = static_cast<int>(flat % T);
+  if (first_end && j > first_end[s]) {
+    if (threadIdx.x == 0) out[flat] = 0.f;
+    return;
+  }
+  const float *z = logits + static_cast<size_t>(r / rows_per_logit_row) * V;
+  float m = -INFINITY, l = 0.f;
+  for (int v = threadIdx.x; v < V; v += blockDim.x) lse_update(m, l, z[v] * inv_temperature);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, o), l2 = __shfl_xor_sync(0xffffffffu, l, o);
+    lse_merge(m, l, m2, l2);
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) {
+    sm_m[warp] = m;
+    sm_l[warp] = l;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float mm = -INFINITY, ll = 0.f;
+    for (int i = 0; i < (blockDim.x >> 5); ++i) lse_merge(mm, ll, sm_m[i], sm_l[i]);
+    int tok = tokens[flat];
+    if (tok < 0 || tok >= V) {
+      atomicExch(status, STATUS_BAD_TOKEN);
+      tok = 0;
+    }
+    out[flat] = z[tok] * inv_temperature - (mm + logf(ll));
+  }
+}
+
+// Appendix F, turn-aware masking: c_t = number of turn-start tokens among x_0..x_t,
+// m_t = [c_t > 1] [c_t odd]; with `shift`, m is aligned with the next-token targets (out[t] = m_{t+1}).
+__global__ void turn_mask_kernel(const int32_t *tokens, int n, int T, int turn_start, int shift, uint8_t *out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int32_t *x = tokens + static_cast<size_t>(i) * T;
+  uint8_t *o = out + static_cast<size_t>(i) * T;
+  int c = 0;
+  for (int t = 0; t < T; ++t) {
+    c += x[t] == turn_start ? 1 : 0;
+    const uint8_t m = (c > 1 && (c & 1)) ? 1 : 0;
+    if (!shift) o[t] = m;
+    else if (t > 0) o[t - 1] = m;
+  }
+  if (shift && T > 0) o[T - 1] = 0;
+}
+
 // Parity hook: copies n floats of the residual stream into slot (*d_step - 1) of dst.
 __global__ void capture_step_kernel(const float *__restrict__ x, float *__restrict__ dst, const int32_t *d_step,
                                     size_t n) {
@@ -666,6 +752,30 @@ cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float 
                                   cudaStream_t s) {
   if (n == 0) return cudaSuccess;
   grpo_surrogate_kernel<<<(n + 7) / 8, 256, 0, s>>>(ln, lo, ls, adv, mask, n, T, eps_clip, C, out);
+  return cudaGetLastError();
+}
+cudaError_t score_rows_launch(int r0, int R, int T, const int32_t *seq_len0, int32_t *row_pt, int32_t *row_pos,
+                              int32_t *tok_idx, cudaStream_t s) {
+  if (R <= 0) return cudaSuccess;
+  score_rows_kernel<<<(R + 255) / 256, 256, 0, s>>>(r0, R, T, seq_len0, row_pt, row_pos, tok_idx);
+  return cudaGetLastError();
+}
+cudaError_t first_end_launch(const int32_t *tokens, int B, int T, int eos_id, int32_t *first_end, cudaStream_t s) {
+  first_end_kernel<<<(B + 127) / 128, 128, 0, s>>>(tokens, B, T, eos_id, first_end);
+  return cudaGetLastError();
+}
+cudaError_t logprob_rows_launch(const float *logits, int rows, int V, int rows_per_logit_row, float temperature,
+                                const int32_t *tokens, const int32_t *tok_idx, int T, const int32_t *first_end,
+                                float *out, int *status, cudaStream_t s) {
+  if (rows <= 0) return cudaSuccess;
+  logprob_rows_kernel<<<rows, 512, 0, s>>>(logits, V, rows_per_logit_row, 1.0f / temperature, tokens, tok_idx, T,
+                                           first_end, out, status);
+  return cudaGetLastError();
+}
+cudaError_t turn_mask_launch(const int32_t *tokens, int n, int T, int turn_start, int shift, uint8_t *out,
+                             cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  turn_mask_kernel<<<(n + 127) / 128, 128, 0, s>>>(tokens, n, T, turn_start, shift, out);
   return cudaGetLastError();
 }
 cudaError_t capture_step_launch(const float *x, float *dst, const int32_t *d_step, size_t n, cudaStream_t s) {

@@ -117,11 +117,13 @@ Layout layout_of(const echo_config &c) {
   lo.hlast = take(static_cast<size_t>(M.B) * D.d * 2);
   lo.logits = take(static_cast<size_t>(M.B) * D.V * 4);
   const size_t n_pre_tok = static_cast<size_t>(M.P) * M.Lp;
+  // row lists: the prompt tokens of a rollout, or one chunk of a scoring pass
+  const size_t n_row_list = std::max<size_t>(n_pre_tok, kChunkRows);
   lo.n_chunks_max = static_cast<int>((n_pre_tok + kSmallChunkRows - 1) / kSmallChunkRows);
   lo.page_table = take(static_cast<size_t>(M.B + M.P) * M.pt_width * 4);
-  lo.pre_row_pt = take(n_pre_tok * 4);
-  lo.pre_row_pos = take(n_pre_tok * 4);
-  lo.pre_tok_idx = take(n_pre_tok * 4);
+  lo.pre_row_pt = take(n_row_list * 4);
+  lo.pre_row_pos = take(n_row_list * 4);
+  lo.pre_tok_idx = take(n_row_list * 4);
   lo.gather_map = take(static_cast<size_t>(lo.n_chunks_max) * M.P * 4);
   lo.dec_row_tok = take(static_cast<size_t>(M.B) * 4);
   lo.dec_row_pos = take(static_cast<size_t>(M.B) * 4);
@@ -635,6 +637,31 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
   return ECHO_OK;
 }
 
+// Prompt prefill of a planned rollout: every prompt once, in chunks of ctx->chunk_rows tokens; leaves
+// each prompt's last residual row in xlast and the private copies of partial prompt pages in place.
+int run_prefill(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t *prompts) {
+  const Layout &lo = ctx->lo;
+  const Dims &D = ctx->D;
+  float *x = ctx->ptr<float>(lo.x);
+  int *status = ctx->ptr<int>(lo.status);
+  for (int c = 0; c < pl.n_chunks; ++c) {
+    const int r0 = c * ctx->chunk_rows, R = std::min(ctx->chunk_rows, pl.n_tok - r0);
+    LAUNCH(embed_launch(w.embed, prompts, ctx->ptr<int32_t>(lo.pre_tok_idx) + r0, x, R, D.d, D.V, status,
+                        ctx->stream));
+    RowMeta meta{ctx->ptr<int32_t>(lo.pre_row_pt) + r0, ctx->ptr<int32_t>(lo.pre_row_pos) + r0, nullptr};
+    ctx->cap_row0 = r0;
+    TRY(forward_layers(ctx, w, R, meta));
+    LAUNCH(gather_rows_launch(x, ctx->ptr<int32_t>(lo.gather_map) + static_cast<size_t>(c) * pl.P,
+                              ctx->ptr<float>(lo.xlast), pl.P, D.d, ctx->stream));
+  }
+  if (pl.n_copies) {
+    LAUNCH(copy_partial_pages_launch(ctx->ptr<__nv_bfloat16>(lo.kv), ctx->ptr<int32_t>(lo.copy_src),
+                                     ctx->ptr<int32_t>(lo.copy_dst), pl.n_copies, D.L, lo.kv_layer_elems,
+                                     D.Hkv * 2 * D.Z * D.hd, ctx->stream));
+  }
+  return ECHO_OK;
+}
+
 int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int P, int G, int T,
                  float temperature, uint64_t seed, const int32_t *forced, int32_t *out_tokens, float *out_logprobs,
                  int64_t *out_versions) {
@@ -678,21 +705,7 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   // ---- prefill: once per prompt, in chunks of ctx->chunk_rows tokens --------
   cudaEvent_t pf_a = nullptr, pf_b = nullptr;
   if (ctx->prof_now && (pf_a = prof_event(ctx)) && (pf_b = prof_event(ctx))) cudaEventRecord(pf_a, ctx->stream);
-  for (int c = 0; c < pl.n_chunks; ++c) {
-    const int r0 = c * ctx->chunk_rows, R = std::min(ctx->chunk_rows, pl.n_tok - r0);
-    LAUNCH(embed_launch(w.embed, prompts, ctx->ptr<int32_t>(lo.pre_tok_idx) + r0, x, R, D.d, D.V, status,
-                        ctx->stream));
-    RowMeta meta{ctx->ptr<int32_t>(lo.pre_row_pt) + r0, ctx->ptr<int32_t>(lo.pre_row_pos) + r0, nullptr};
-    ctx->cap_row0 = r0;
-    TRY(forward_layers(ctx, w, R, meta));
-    LAUNCH(gather_rows_launch(x, ctx->ptr<int32_t>(lo.gather_map) + static_cast<size_t>(c) * P,
-                              ctx->ptr<float>(lo.xlast), P, D.d, ctx->stream));
-  }
-  if (pl.n_copies) {
-    LAUNCH(copy_partial_pages_launch(ctx->ptr<__nv_bfloat16>(lo.kv), ctx->ptr<int32_t>(lo.copy_src),
-                                     ctx->ptr<int32_t>(lo.copy_dst), pl.n_copies, D.L, lo.kv_layer_elems,
-                                     D.Hkv * 2 * D.Z * D.hd, ctx->stream));
-  }
+  TRY(run_prefill(ctx, w, pl, prompts));
   // ---- first token of every sample from the prompt's last logits row --------
   TRY(lm_head(ctx, w, ctx->ptr<float>(lo.xlast), P));
   LAUNCH(set_int_launch(ctx->ptr<int32_t>(lo.d_step), 0, ctx->stream));
@@ -778,6 +791,80 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   ctx->stats.tokens_generated = static_cast<int64_t>(pl.B) * T;
   ctx->stats.kernels_launched = ctx->launches - launches0;
   ctx->stats.decode_steps = n_steps;
+  ctx->stats.n_pages = pl.n_pages;
+  return ECHO_OK;
+}
+
+// Teacher-forced scoring of whole trajectories in prefill-shaped passes: the prompt once per group, then
+// every sequence's given tokens as rows of 2048-row chunks (sequence-major), each chunk through the
+// layers with causal attention over the paged cache, the lm_head and the log-probability kernel in
+// blocks of at most P*G rows (the logits buffer).
+int score_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int P, int G, int T,
+               float temperature, const int32_t *tokens, float *out_logprobs, int64_t *out_versions) {
+  if (!ctx || !prompts || !prompt_lens || !tokens || !out_logprobs || !out_versions) return ECHO_ERR_INVALID;
+  const Limits &M = ctx->M;
+  if (P < 1 || P > M.P || G < 1 || G > M.G || T < 1 || T > M.T) return ECHO_ERR_INVALID;
+  if (!(temperature > 0.f) || !std::isfinite(temperature)) return ECHO_ERR_INVALID;
+  for (int p = 0; p < P; ++p)
+    if (prompt_lens[p] < 1 || prompt_lens[p] > M.Lp) return ECHO_ERR_INVALID;
+  DeviceGuard guard(ctx->device);
+  int rc;
+  WeightBuf *wp = begin_rollout_version(ctx, &rc);
+  if (!wp) return rc;
+  const WeightBuf &w = *wp;
+  for (int i = 0; i < P * G; ++i) out_versions[i] = w.version;
+  if (ctx->plan_in_flight) {
+    CK(cudaEventSynchronize(ctx->plan_done));
+    ctx->plan_in_flight = false;
+  }
+  Plan pl;
+  TRY(build_plan(ctx, prompt_lens, P, G, T, &pl));
+  TRY(upload_plan(ctx, pl));
+  const Layout &lo = ctx->lo;
+  const Dims &D = ctx->D;
+  const int64_t launches0 = ctx->launches;
+  float *x = ctx->ptr<float>(lo.x);
+  int *status = ctx->ptr<int>(lo.status);
+  float *logits = ctx->ptr<float>(lo.logits);
+  int32_t *first_end = ctx->cfg.eos_id >= 0 ? ctx->ptr<int32_t>(lo.row_done) : nullptr;
+
+  CK(cudaEventRecord(ctx->ev_begin, ctx->stream));
+  ctx->prof_recs.clear();
+  ctx->prof_pool_used = 0;
+  if (first_end) LAUNCH(first_end_launch(tokens, pl.B, T, ctx->cfg.eos_id, first_end, ctx->stream));
+  TRY(run_prefill(ctx, w, pl, prompts));
+  // token 0 of every sample: scored on the prompt's last logits row
+  TRY(lm_head(ctx, w, ctx->ptr<float>(lo.xlast), P));
+  LAUNCH(logprob_rows_launch(logits, pl.B, D.V, G, temperature, tokens, nullptr, T, first_end, out_logprobs, status,
+                             ctx->stream));
+  CK(cudaEventRecord(ctx->ev_first, ctx->stream));
+  // tokens 1..T-1: row (s, j) feeds given token j at position len0[s] + j and scores token j + 1
+  const long n_rows = static_cast<long>(pl.B) * (T - 1);
+  int32_t *row_pt = ctx->ptr<int32_t>(lo.pre_row_pt), *row_pos = ctx->ptr<int32_t>(lo.pre_row_pos),
+          *tok_idx = ctx->ptr<int32_t>(lo.pre_tok_idx);
+  for (long r0 = 0; r0 < n_rows; r0 += ctx->chunk_rows) {
+    const int R = static_cast<int>(std::min<long>(ctx->chunk_rows, n_rows - r0));
+    LAUNCH(score_rows_launch(static_cast<int>(r0), R, T, ctx->ptr<int32_t>(lo.seq_len0), row_pt, row_pos, tok_idx,
+                             ctx->stream));
+    LAUNCH(embed_launch(w.embed, tokens, tok_idx, x, R, D.d, D.V, status, ctx->stream));
+    RowMeta meta{row_pt, row_pos, nullptr};
+    ctx->cap_row0 = 0;
+    TRY(forward_layers(ctx, w, R, meta));
+    for (int sub = 0; sub < R; sub += pl.B) {
+      const int rows = std::min(pl.B, R - sub);
+      TRY(lm_head(ctx, w, x + static_cast<size_t>(sub) * D.d, rows));
+      LAUNCH(logprob_rows_launch(logits, rows, D.V, 1, temperature, tokens, tok_idx + sub, T, first_end, out_logprobs,
+                                 status, ctx->stream));
+    }
+  }
+  CK(cudaEventRecord(ctx->ev_end, ctx->stream));
+  CK(cudaEventRecord(wp->last_use, ctx->stream));
+  wp->used = true;
+  ctx->stats.prefill_ms = ctx->stats.decode_ms = 0.f;
+  ctx->stats.version_served = w.version;
+  ctx->stats.tokens_generated = static_cast<int64_t>(pl.B) * T;
+  ctx->stats.kernels_launched = ctx->launches - launches0;
+  ctx->stats.decode_steps = 0;
   ctx->stats.n_pages = pl.n_pages;
   return ECHO_OK;
 }
@@ -1039,6 +1126,20 @@ int echo_rollout_forced(echo_ctx *ctx, const int32_t *prompts, const int32_t *pr
   if (!forced_tokens) return ECHO_ERR_INVALID;
   return rollout_impl(ctx, prompts, prompt_lens, P, G, max_new_tokens, temperature, seed, forced_tokens, out_tokens,
                       out_logprobs, out_versions);
+}
+
+int echo_score(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int32_t P, int32_t G,
+               int32_t max_new_tokens, float temperature, const int32_t *tokens, float *out_logprobs,
+               int64_t *out_versions) {
+  return score_impl(ctx, prompts, prompt_lens, P, G, max_new_tokens, temperature, tokens, out_logprobs, out_versions);
+}
+
+int echo_turn_mask(const int32_t *tokens, int32_t n, int32_t T, int32_t turn_start_id, int32_t shift_to_targets,
+                   uint8_t *out_mask, void *cuda_stream) {
+  if (!tokens || !out_mask || n < 0 || T < 1) return ECHO_ERR_INVALID;
+  cudaError_t e = turn_mask_launch(tokens, n, T, turn_start_id, shift_to_targets ? 1 : 0, out_mask,
+                                   static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }
 
 int echo_rollout_host(echo_ctx *ctx, const int32_t *prompts_host, const int32_t *prompt_lens, int32_t P, int32_t G,

@@ -428,3 +428,87 @@ def test_prefill_attention_kernels(B, tiny, monkeypatch, prefill):
                                        lp.cpu().numpy(), range(P * G))
         assert n == P * G * T and ex <= 3
         eng.close()
+
+
+def test_prefill_shaped_scoring(B, tiny):
+    """echo_score: log-probabilities of given trajectories in prefill-shaped passes.  Against the oracle
+    on every token (ragged prompts, lengths that are not multiples of the page size), against the
+    decode-shaped teacher-forced entry point, with the end-of-sequence rule, and for T = 1."""
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 3, 4, 40, 14
+    prompts, lens = synth.make_ragged_prompts([40, 21, 7], wl.shape.vocab, 515, pad_to=Lp)
+    dp = torch.from_numpy(prompts).cuda()
+    for hl in (0, 2):
+        eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, half_layers=hl))
+        eng.echo_load_policy(w_d, 4)
+        tok, lp, _ = eng.echo_rollout(dp, lens, G, T, 0.9, 11)
+        lp_s, ver = eng.echo_score(dp, lens, tok, 0.9)
+        _, lp_f, _ = eng.echo_rollout(dp, lens, G, T, 0.9, 11, forced=tok)
+        eng.echo_sync()
+        tok_h, lp_s, lp_f = tok.cpu().numpy(), lp_s.cpu().numpy(), lp_f.cpu().numpy()
+        assert np.all(ver == 4) and np.all(lp_s <= 0)
+        assert np.max(np.abs(lp_s - lp_f)) < LOGPROB_TOL / 5
+        n, ex, worst = check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 0.9, 11, tok_h, lp_s, range(P * G))
+        assert n == P * G * T
+        # a single token per sequence: only the prompt pass and the first-token rows
+        lp1, _ = eng.echo_score(dp, lens, tok[:, :, :1].contiguous(), 0.9)
+        eng.echo_sync()
+        assert np.max(np.abs(lp1.cpu().numpy()[..., 0] - lp_s[..., 0])) < LOGPROB_TOL / 5
+        eng.close()
+    # end-of-sequence rule: positions after a sequence's first end token score 0, the others are unchanged
+    eos = int(tok_h[1, 2, 5])
+    eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, eos_id=eos))
+    eng.echo_load_policy(w_d, 1)
+    lp_e, _ = eng.echo_score(dp, lens, tok, 0.9)
+    eng.echo_sync()
+    lp_e = lp_e.cpu().numpy()
+    ended = np.zeros_like(tok_h, dtype=bool)
+    ended[..., 1:] = np.logical_or.accumulate(tok_h[..., :-1] == eos, axis=-1)
+    assert ended.any() and np.all(lp_e[ended] == 0.0)
+    for s in range(P * G):
+        p, g = divmod(s, G)
+        sc = decoder.score_forced(dims_of(wl.shape), w_o, prompts[p][: lens[p]], tok_h[p, g], 0.9, 11, s, eos_id=eos)
+        assert np.max(np.abs(lp_e[p, g] - sc.logprob_given)) <= LOGPROB_TOL
+    eng.close()
+
+
+def test_prefill_shaped_scoring_is_faster_than_stepwise(B):
+    """A few hundred tokens per sequence at the 0.6B width: the scoring pass agrees with the decode-shaped
+    teacher-forced entry point on every token and takes a fraction of its time."""
+    import dataclasses
+    shape = dataclasses.replace(synth.SHAPES["0.6B"], name="0.6B-width L6", n_layers=6, vocab=32000)
+    P, G, Lp, T = 8, 8, 64, 384
+    w_t = synth.make_weights(shape, 3, device="cuda")
+    eng = B.Engine(B.make_config(shape, P, G, Lp, T, 1))
+    eng.echo_load_policy(w_t, 1)
+    prompts = torch.from_numpy(synth.make_prompts(P, Lp, shape.vocab, 29)).cuda()
+    lens = [Lp] * P
+    tok, lp, _ = eng.echo_rollout(prompts, lens, G, T, 1.0, 3)
+    eng.echo_sync()
+    times = {}
+    for name in ("score", "forced"):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(eng.stream)
+        if name == "score":
+            lp_s, _ = eng.echo_score(prompts, lens, tok, 1.0)
+        else:
+            _, lp_f, _ = eng.echo_rollout(prompts, lens, G, T, 1.0, 3, forced=tok)
+        e1.record(eng.stream)
+        eng.echo_sync()
+        times[name] = e0.elapsed_time(e1)
+    d = (lp_s - lp_f).abs()
+    print(f"score {times['score']:.1f} ms, stepwise {times['forced']:.1f} ms, max |dlogprob| {float(d.max()):.2e}")
+    assert float(d.max()) < LOGPROB_TOL / 2 and float((lp_s - lp).abs().max()) < LOGPROB_TOL / 2
+    assert times["score"] < 0.6 * times["forced"]
+    eng.close()
+
+
+def test_turn_mask_matches_oracle(B):
+    from oracle import objective
+    rng = np.random.default_rng(8)
+    for n, T, p_start in [(1, 1, 0.5), (7, 33, 0.2), (64, 2048, 0.01), (300, 100, 0.0)]:
+        x = rng.integers(0, 50, size=(n, T)).astype(np.int32)
+        x[rng.random((n, T)) < p_start] = 77
+        for shift in (False, True):
+            got = B.echo_turn_mask(torch.from_numpy(x).cuda(), 77, shift).cpu().numpy()
+            assert np.array_equal(got, objective.turn_mask(x, 77, shift))

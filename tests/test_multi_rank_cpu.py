@@ -91,3 +91,53 @@ def test_reference_arm_prints_the_contract_line():
         assert key in line, key
     assert line["impl"] == "reference" and line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+
+
+def _chain_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    from paper_2602_02192_b200 import chain, synth
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    shape = synth.SHAPES["tiny"]
+    # rank 0 holds the new snapshot; ranks 1..3 are rollout replicas ranked by a peer score
+    scores = [40.0, 90.0, 70.0]                                   # workers 0, 1, 2 = ranks 1, 2, 3
+    chains = [[w + 1 for w in c] for c in chain.plan_chains(scores, 200.0, 100.0)]     # floor(200 / 100) = 2 chains
+    flat = chain.pack(synth.make_weights(shape, 5), shape) if rank == 0 else None
+    got, version = chain.disseminate(flat, 17, shape, 0, chains, chunk_bytes=64 << 10)
+    want = chain.pack(synth.make_weights(shape, 5), shape)        # seeded: every rank can rebuild the bits
+    same = bool(torch.equal(got, want))
+    w = chain.unpack(got, shape)
+    ref = synth.make_weights(shape, 5)
+    views_ok = all(torch.equal(w[n][l], ref[n][l]) for n in chain.LAYER_TENSORS for l in range(shape.n_layers)) and \
+        all(torch.equal(w[n], ref[n]) for n in chain.GLOBAL_TENSORS)
+    aligned = all(w[n][l].data_ptr() % 16 == 0 for n in chain.LAYER_TENSORS for l in range(shape.n_layers))
+    dist.barrier()
+    out[rank] = (chains, version, same, views_ok, aligned)
+    dist.destroy_process_group()
+
+
+def test_snapshot_chain_dissemination_on_gloo():
+    """Section 4.3 on four CPU ranks: the source streams the snapshot in 64 KiB chunks to the two seeds,
+    the better seed's chain has a second hop that receives every chunk from the seed, not from the
+    source; every replica ends with the snapshot bit for bit and the new version tag."""
+    world = 4
+    port = 31500 + os.getpid() % 2000
+    mgr = mp.get_context("spawn").Manager()
+    out = mgr.dict()
+    mp.spawn(_chain_worker, args=(world, port, out), nprocs=world, join=True)
+    assert len(out) == world
+    for rank in range(world):
+        chains, version, same, views_ok, aligned = out[rank]
+        assert chains == [[2, 1], [3]]            # seeds: ranks 2 (score 90) and 3 (70); rank 1 behind the best seed
+        assert version == 17 and same and views_ok and aligned
+
+
+def test_chain_repair_closes_over_a_failed_relay():
+    sys.path.insert(0, ROOT)
+    from paper_2602_02192_b200 import chain
+    chains = [[4, 1, 7, 2], [5, 3], [6]]
+    assert chain.excise(chains, 1) == [[4, 7, 2], [5, 3], [6]]      # the tail reattaches to the nearest healthy parent
+    assert chain.excise(chains, 4) == [[1, 7, 2], [5, 3], [6]]      # a failed seed: its child becomes the seed
+    assert chain.excise(chains, 6) == [[4, 1, 7, 2], [5, 3]]        # a chain of one disappears
+    assert chain.excise(chains, 9) == chains

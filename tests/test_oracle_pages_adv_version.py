@@ -189,3 +189,29 @@ def test_grpo_surrogate_against_vector_formula():
     den = mask.sum(1)
     want = np.where(den > 0, (mask * w * term).sum(1) / np.maximum(den, 1), 0.0)
     assert np.allclose(got, want, rtol=1e-12, atol=1e-15)
+
+
+def test_turn_mask_hand_written_dialogue():
+    """Appendix F, turn-aware masking, on a dialogue written out by hand.  S = the turn-start id.
+    turns: system (c = 1), user (2), assistant (3), user (4), assistant (5): the mask selects turns 3 and 5,
+    the turn-start tokens of those turns included (c_t counts the token at t itself)."""
+    from oracle import objective
+    S = 9
+    x = np.array([[S, 1, 2, S, 3, S, 4, 5, 6, S, 7, S, 8, 8]])
+    want = np.array([[0, 0, 0, 0, 0, 1, 1, 1, 1, 0, 0, 1, 1, 1]], dtype=np.uint8)
+    assert np.array_equal(objective.turn_mask(x, S), want)
+    # aligned with next-token targets y_t = x_{t+1}: shifted left by one, last column empty
+    shifted = objective.turn_mask(x, S, shift_to_targets=True)
+    assert np.array_equal(shifted[:, :-1], want[:, 1:]) and shifted[0, -1] == 0
+    # no turn-start token, or only the system turn: nothing to learn from
+    assert objective.turn_mask(np.array([[1, 2, 3, 4]]), S).sum() == 0
+    assert objective.turn_mask(np.array([[S, 2, 3, 4]]), S).sum() == 0
+    # the mask depends on the turn index only: other ids are irrelevant
+    y = x.copy()
+    y[x != S] = 5
+    assert np.array_equal(objective.turn_mask(y, S), want)
+    # rows are independent
+    two = np.concatenate([x, np.array([[1, S, 2, S, 2, S, 2, 2, S, 1, 1, 1, 1, S]])])
+    got = objective.turn_mask(two, S)
+    assert np.array_equal(got[0], want[0])
+    assert np.array_equal(got[1], np.array([0, 0, 0, 0, 0, 1, 1, 1, 0, 0, 0, 0, 0, 1], dtype=np.uint8))
