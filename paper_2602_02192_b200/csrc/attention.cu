@@ -579,12 +579,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
 // ahead, so the copy engine stays busy while partial results are combined and written.
 // Shared memory: the four warps' page stages, then a merge area of REP rows per warp.
 // ---------------------------------------------------------------------------------------------
-// merged outputs per thread (template parameter PRE of the resident kernel): REP * HD <= PRE * threads.
-// 4 covers up to four query heads per kv head at head_dim 128 (three CTAs per SM); 8 covers eight
-// (the 32B shape: two CTAs per SM, still drawn from the item counter so that 1024 items do not
-// leave a third of the last wave empty).
-constexpr int kSufPre = 4;
-constexpr int kSufPreWide = 8;
+constexpr int kSufPre = 4;                  // merged outputs per thread: REP * HD <= kSufPre * threads
 
 template <int HD>
 struct SufSmem {
@@ -596,7 +591,7 @@ struct SufSmem {
   static constexpr int total(int rep) { return 1024 + kPipeBytes + merge_bytes(rep) + 256; }
 };
 
-template <int HD, bool HALF, int PRE>
+template <int HD, bool HALF>
 __global__ void __launch_bounds__(kDecWarps * 32)
 attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16 *__restrict__ q,
                             __nv_bfloat16 *__restrict__ out, const float *__restrict__ pre_o,
@@ -767,10 +762,10 @@ attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv
         griddep_wait();
         waited = true;
       }
-      float pre_val[PRE];
-      float2 pre_stat[PRE];
+      float pre_val[kSufPre];
+      float2 pre_stat[kSufPre];
 #pragma unroll
-      for (int i = 0; i < PRE; ++i) {
+      for (int i = 0; i < kSufPre; ++i) {
         const int idx = threadIdx.x + i * kDecWarps * 32;
         pre_val[i] = 0.f;
         pre_stat[i] = make_float2(-INFINITY, 0.f);
@@ -808,7 +803,7 @@ attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv
       if (*abort_flag) break;                // some warp gave up: every thread of the CTA sees it here
       m2 = ticket_s[n & 1];
 #pragma unroll
-      for (int i = 0; i < PRE; ++i) {
+      for (int i = 0; i < kSufPre; ++i) {
         const int idx = threadIdx.x + i * kDecWarps * 32;
         if (idx < REP * HD) {
           const int r = idx / HD, d = idx % HD;
@@ -1423,16 +1418,16 @@ cudaError_t launch_prefill(const PrefillAttnArgs &a, cudaStream_t s) {
 
 // CTAs of the resident suffix kernel that fit the current device at once (cached per device, head
 // dimension, operand format and group ratio; no stream work).
-template <int HD, bool HALF, int PRE>
+template <int HD, bool HALF>
 int resident_slots(int smem_bytes, int rep) {
-  static int cache[64][17] = {};             // one table per kernel instantiation
+  static int cache[64][17] = {};             // one table per (HD, HALF) instantiation
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || rep < 1 || rep > 16) return 0;
   if (cache[dev][rep] == 0) {
     int sms = 0, per_sm = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attn_suffix_resident_kernel<HD, HALF, PRE>,
-                                                      kDecWarps * 32, smem_bytes) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attn_suffix_resident_kernel<HD, HALF>, kDecWarps * 32,
+                                                      smem_bytes) != cudaSuccess)
       return 0;
     cache[dev][rep] = sms * per_sm;
   }
@@ -1459,15 +1454,12 @@ cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
                      a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
   }
   if (e != cudaSuccess) return e;
-  if (a.suffix_impl != 1 && a.work && REP * HD <= kSufPreWide * kDecWarps * 32) {
+  if (a.suffix_impl != 1 && a.work && REP * HD <= 512) {   // merge area small enough for three CTAs per SM
     using R = SufSmem<HD>;
     const int n_items = a.P * a.G * a.Hkv;
-    const bool wide = REP * HD > kSufPre * kDecWarps * 32;
-    const int slots = wide ? resident_slots<HD, HALF, kSufPreWide>(R::total(REP), REP)
-                           : resident_slots<HD, HALF, kSufPre>(R::total(REP), REP);
+    const int slots = resident_slots<HD, HALF>(R::total(REP), REP);
     if (slots <= 0) return cudaErrorInvalidConfiguration;
-    auto kernel = wide ? attn_suffix_resident_kernel<HD, HALF, kSufPreWide> : attn_suffix_resident_kernel<HD, HALF, kSufPre>;
-    return launch_early(kernel, dim3(n_items < slots ? n_items : slots),
+    return launch_early(attn_suffix_resident_kernel<HD, HALF>, dim3(n_items < slots ? n_items : slots),
                         dim3(kDecWarps * 32), R::total(REP), s, *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table,
                         a.pt_width, a.row_pos, a.full_pages, a.layer_row0, a.Hq, a.Hkv, n_items, a.n_pages, scale_log2,
                         a.row_done, a.status, a.work);
@@ -1488,10 +1480,7 @@ cudaError_t configure_decode() {
                                 PreSmem<HD, 2>::kTotal)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(attn_prefill_kernel<HD, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 PreSmem<HD, 2>::kTotal)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(attn_suffix_resident_kernel<HD, HALF, kSufPreWide>,
-                                cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                SufSmem<HD>::total(kSufPreWide * kDecWarps * 32 / HD))) != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_suffix_resident_kernel<HD, HALF, kSufPre>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  return cudaFuncSetAttribute(attn_suffix_resident_kernel<HD, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               SufSmem<HD>::total(kSufPre * kDecWarps * 32 / HD));
 }
 

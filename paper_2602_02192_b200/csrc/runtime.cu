@@ -730,16 +730,12 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   // Two captures of the same step, which differ in the suffix attention kernel: resident CTAs while
   // the sequences hold few generated tokens (their fixed cost per item is what counts), one CTA per
   // (sequence, kv head) from kLongSuffix generated tokens on (the launch is bound by the KV stream).
-  // With eight query heads per kv head at head_dim 128 the (sequence, kv head) items are few and long
-  // (two resident CTAs per SM): handing them out from the counter matters at every length, so that
-  // shape keeps the resident kernel throughout.
-  const bool wide_groups = (D.Hq / D.Hkv) * D.hd > 512;
   cudaGraph_t graph[2] = {nullptr, nullptr};
   cudaGraphExec_t exec[2] = {nullptr, nullptr};
   int64_t per_step = 0;
   if (n_steps > 1 && ctx->use_graph && ctx->stream != nullptr) {
     for (int v = 0; v < 2; ++v) {
-      if (v == 1 && (n_steps < kLongSuffix || wide_groups)) break;
+      if (v == 1 && n_steps < kLongSuffix) break;
       const int64_t before = ctx->launches;
       if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
         cudaGetLastError();
@@ -767,7 +763,7 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   int rc_steps = ECHO_OK;
   for (int j = 1; j <= n_steps && rc_steps == ECHO_OK; ++j) {
     const bool sampled = ctx->prof_every > 0 && (j % ctx->prof_every == 0);
-    const int v = (j >= kLongSuffix && !wide_groups) ? 1 : 0;
+    const int v = j >= kLongSuffix ? 1 : 0;
     if (exec[v] && !sampled) {
       cudaError_t le = cudaGraphLaunch(exec[v], ctx->stream);
       if (le != cudaSuccess) rc_steps = fail_cuda(ctx, le, "cudaGraphLaunch");

@@ -320,8 +320,8 @@ def test_rollout_past_the_suffix_kernel_switch(B):
 
 def test_eight_query_heads_per_kv_head(B):
     """Hq / Hkv = 8 with G = 8 (the 32B shape's ratio): a group's 64 query rows take two prefix CTAs
-    per (prompt, kv head), and the resident suffix kernel runs in its wide form (eight merged outputs
-    per thread, two CTAs per SM).  Every token of a small model against the oracle."""
+    per (prompt, kv head) and the merge area of the resident suffix kernel is too small, so every
+    step runs the per-item suffix kernel.  Every token of a small model against the oracle."""
     shape = synth.DecoderShape("rep8", 2, 512, 16, 2, 128, 1024, 4096)
     P, G, T = 3, 8, 24
     w_t = synth.make_weights(shape, 11)
