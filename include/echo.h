@@ -107,7 +107,9 @@ typedef struct echo_stats {
   float   prefill_ms;         /* last rollout: prompt prefill + first token (device time; valid once
                                  the rollout has finished, else 0)                                */
   float   decode_ms;          /* last rollout: the T-1 decode steps (device time; same condition)  */
-  float   reserved;
+  float   last_step_rows;     /* activation rows of the last decode step's projections: P*G, or fewer
+                                 once sequences have ended (with an end token the live sequences are
+                                 packed and the row count follows their number downwards) */
 } echo_stats;
 
 /* Bytes of device memory echo_create needs for this configuration (weight

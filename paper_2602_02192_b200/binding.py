@@ -55,7 +55,7 @@ class EchoStats(C.Structure):
     _fields_ = [
         ("version_served", C.c_int64), ("tokens_generated", C.c_int64), ("kernels_launched", C.c_int64),
         ("decode_steps", C.c_int64), ("n_pages", C.c_int64), ("install_ms", C.c_float), ("prefill_ms", C.c_float),
-        ("decode_ms", C.c_float), ("reserved", C.c_float),
+        ("decode_ms", C.c_float), ("last_step_rows", C.c_float),
     ]
 
 
@@ -306,7 +306,7 @@ class Engine:
     def echo_get_stats(self) -> dict:
         st = EchoStats()
         _check(lib.echo_get_stats(self._ctx, C.byref(st)))
-        return {k: getattr(st, k) for k, _ in EchoStats._fields_ if k != "reserved"}
+        return {k: getattr(st, k) for k, _ in EchoStats._fields_}
 
     def echo_profile_config(self, every_n_steps: int):
         _check(lib.echo_profile_config(self._ctx, int(every_n_steps)))

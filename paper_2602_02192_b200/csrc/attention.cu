@@ -329,7 +329,8 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
                    __nv_bfloat16 *__restrict__ out, float *__restrict__ pre_o, float2 *__restrict__ pre_ml,
                    const int32_t *__restrict__ page_table, int pt_width, const int32_t *__restrict__ row_pos,
                    const int32_t *__restrict__ full_pages, int layer_row0, int Hq, int Hkv, int G, int n_pages,
-                   float scale_log2, const int32_t *__restrict__ row_done, int *status) {
+                   float scale_log2, const int32_t *__restrict__ row_done, int *status,
+                   const int32_t *__restrict__ out_row) {
   using S = DecSmem<HD>;
   constexpr int KSTEPS = HD / 16;           // MMA k-steps over the head dimension
   constexpr int HALVES = HD / 64;           // 64-element (128-byte) column blocks per row
@@ -563,7 +564,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
       const float c_pre = ml.x == -INFINITY ? 0.f : exp2f(ml.x - Mt);
       const float Lt = L * c_suf + ml.y * c_pre;
       const float Ot = O * c_suf + (c_pre != 0.f ? po * c_pre : 0.f);
-      reinterpret_cast<uint16_t *>(out)[oi] = cvt16(Ot / Lt, HALF);
+      // compacted step: the sequence's output goes to the activation row it occupies
+      const size_t oo = out_row ? (static_cast<size_t>(__ldcg(&out_row[s])) * Hq + row_head(r)) * HD + d : oi;
+      reinterpret_cast<uint16_t *>(out)[oo] = cvt16(Ot / Lt, HALF);
     }
   }
   if (threadIdx.x == 0 && *abort_flag) atomicExch(status, STATUS_WAIT_TIMEOUT);
@@ -598,7 +601,8 @@ attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv
                             const float2 *__restrict__ pre_ml, const int32_t *__restrict__ page_table, int pt_width,
                             const int32_t *__restrict__ row_pos, const int32_t *__restrict__ full_pages,
                             int layer_row0, int Hq, int Hkv, int n_items, int n_pages, float scale_log2,
-                            const int32_t *__restrict__ row_done, int *status, int *work) {
+                            const int32_t *__restrict__ row_done, int *status, int *work,
+                            const int32_t *__restrict__ out_row) {
   using S = SufSmem<HD>;
   constexpr int KSTEPS = HD / 16;
   constexpr int HALVES = HD / 64;
@@ -827,8 +831,9 @@ attn_suffix_resident_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv
           const float c_pre = ml.x == -INFINITY ? 0.f : exp2f(ml.x - Mt);
           const float Lt = L * c_suf + ml.y * c_pre;
           const float Ot = O * c_suf + (c_pre != 0.f ? pre_val[i] * c_pre : 0.f);
-          reinterpret_cast<uint16_t *>(out)[(static_cast<size_t>(c_seq) * Hq + c_h * REP + r) * HD + d] =
-              cvt16(Ot / Lt, HALF);
+          // compacted step: the sequence's output goes to the activation row it occupies
+          const size_t o_seq = out_row ? static_cast<size_t>(__ldcg(&out_row[c_seq])) : static_cast<size_t>(c_seq);
+          reinterpret_cast<uint16_t *>(out)[(o_seq * Hq + c_h * REP + r) * HD + d] = cvt16(Ot / Lt, HALF);
         }
       }
       __syncthreads();                       // the merge area is free for the next item
@@ -1451,7 +1456,7 @@ cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
   } else {
     e = launch_early(attn_decode_kernel<HD, true, HALF>, dim3(a.P * a.Hkv * MT), dim3(kDecWarps * 32), S::kTotal, s,
                      *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages,
-                     a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
+                     a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status, a.out_row);
   }
   if (e != cudaSuccess) return e;
   if (a.suffix_impl != 1 && a.work && REP * HD <= 512) {   // merge area small enough for three CTAs per SM
@@ -1462,11 +1467,11 @@ cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
     return launch_early(attn_suffix_resident_kernel<HD, HALF>, dim3(n_items < slots ? n_items : slots),
                         dim3(kDecWarps * 32), R::total(REP), s, *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table,
                         a.pt_width, a.row_pos, a.full_pages, a.layer_row0, a.Hq, a.Hkv, n_items, a.n_pages, scale_log2,
-                        a.row_done, a.status, a.work);
+                        a.row_done, a.status, a.work, a.out_row);
   }
   return launch_early(attn_decode_kernel<HD, false, HALF>, dim3(a.P * a.G * a.Hkv), dim3(kDecWarps * 32), S::kTotal, s,
                       *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages,
-                      a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status);
+                      a.layer_row0, a.Hq, a.Hkv, a.G, a.n_pages, scale_log2, a.row_done, a.status, a.out_row);
 }
 
 template <int HD, bool HALF>

@@ -184,24 +184,34 @@ cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double t
 cudaError_t rope_append_launch(float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer,
                                const float2 *rope_table, RowMeta meta, const int32_t *page_table,
                                int pt_width, int R, int Hq, int Hkv, int hd, int page_size,
-                               int n_pages, int max_pos, int *status, cudaStream_t s, bool out_half = false);
+                               int n_pages, int max_pos, int *status, cudaStream_t s, bool out_half = false,
+                               const int32_t *q_row = nullptr);     // row of q each row writes (null: its own)
 cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s, bool out_half = false);
 cudaError_t gather_rows_launch(const float *x, const int32_t *src_rows, float *dst, int n, int d,
                                cudaStream_t s);
 cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page, const int32_t *dst_page,
                                       int n_copies, int n_layers, size_t layer_stride_elems,
                                       int page_elems, cudaStream_t s);
-// decode-step preparation: advances the step counter, sets the rows' token and position
+// Compaction of a decode step's rows (used with an end token): the sequences that have not ended are
+// packed to the front of the activation rows.  row_seq[r] = sequence of row r (-1: padding row),
+// seq_row[b] = row of sequence b (-1: ended), seq_pos[b] = position sequence b feeds, *n_live = rows in use.
+struct CompactRows {
+  int32_t *row_seq, *seq_row, *seq_pos, *n_live;
+};
+// decode-step preparation: advances the step counter, sets the rows' token and position; with `cr` it
+// also packs the live sequences and writes end token / 0 for the ended ones into the outputs
 cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
                                int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s, int eos_id = -1,
-                               int32_t *row_done = nullptr);
+                               int32_t *row_done = nullptr, const CompactRows *cr = nullptr,
+                               int32_t *out_tok = nullptr, float *out_lp = nullptr);
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row,
                            const int32_t *seq_ids, const int32_t *d_step, uint32_t j_host,
                            float temperature, uint64_t seed, const int32_t *forced, int forced_stride,
                            int32_t *out_tok, float *out_lp, int out_stride, cudaStream_t s, int eos_id = -1,
                            const uint2 *nucleus_cut = nullptr,    // per logits row, from nucleus_cut_launch
                            const int32_t *row_done = nullptr,     // per row: non-zero = the sequence has ended
-                           uint32_t seq_base = 0);                // added to every sequence id of the noise streams
+                           uint32_t seq_base = 0,                 // added to every sequence id of the noise streams
+                           const int32_t *row_seq = nullptr);     // compacted step: sequence of each logits row
 // Nucleus (top-p) cut of each logits row: cut[row] = (order-preserving key of the score of the last
 // nucleus member, its id; id 0x7fffffff = every id of that score).  nucleus.cu
 cudaError_t nucleus_cut_launch(const float *logits, int rows, int V, float temperature, float top_p, uint2 *cut,
@@ -258,6 +268,7 @@ struct DecodeAttnArgs {
   int half_io = 0;                // 1: q, the pool and out hold IEEE half values; probabilities are rounded to half
   int suffix_impl = 0;            // 0: choose; 1: always one suffix CTA per (sequence, kv head)
   int prefix_impl = 0;            // 0: choose; 1: always one prefix CTA per 16-row tile
+  const int32_t *out_row = nullptr;   // compacted step: row of `out` each sequence writes (null: its own)
 };
 // Causal attention of a chunk of R prompt tokens (rows of q / out) over the paged cache; row r belongs
 // to page-table row row_pt[r] at position row_pos[r]; consecutive rows of one prompt have consecutive

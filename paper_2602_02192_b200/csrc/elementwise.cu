@@ -136,16 +136,19 @@ __global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__res
                                    const int32_t *__restrict__ row_pt, const int32_t *__restrict__ row_pos,
                                    const int32_t *__restrict__ row_done, const int32_t *__restrict__ page_table,
                                    int pt_width, int R, int Hq, int Hkv, int hd, int page_size, int n_pages,
-                                   int max_pos, int *status, int out_half) {
+                                   int max_pos, int *status, int out_half, const int32_t *q_row) {
   early_start_sync();
   const bool oh = out_half != 0;
   const int r = blockIdx.x;
-  const int pos = (row_done && row_done[r]) ? -1 : row_pos[r];      // an ended row is only cleared
+  // an ended row (or a padding row of a compacted step: no page-table row) is only cleared
+  const bool skip = (row_done && row_done[r]) || row_pt[r] < 0;
+  const int pos = skip ? -1 : row_pos[r];
+  const int qr = (q_row && !skip) ? q_row[r] : r;                   // row of the query buffer this row writes
   const int half = hd / 2;
   const int ld = (Hq + 2 * Hkv) * hd;
   float *src = qkv + static_cast<size_t>(r) * ld;
   if (pos < 0 || pos >= max_pos) {
-    if (threadIdx.x == 0 && !(row_done && row_done[r])) atomicExch(status, STATUS_BAD_PAGE);
+    if (threadIdx.x == 0 && !skip) atomicExch(status, STATUS_BAD_PAGE);
     for (int i = threadIdx.x; i < ld; i += blockDim.x) src[i] = 0.f;      // keep the buffer's zero invariant
     return;
   }
@@ -163,7 +166,7 @@ __global__ void rope_append_kernel(float *__restrict__ qkv, __nv_bfloat16 *__res
     const int head = idx / half, i = idx % half;
     const float a = src[head * hd + i], b = src[head * hd + i + half];
     const float2 t = cs[i];
-    uint16_t *dst = reinterpret_cast<uint16_t *>(q) + static_cast<size_t>(r) * Hq * hd + head * hd;
+    uint16_t *dst = reinterpret_cast<uint16_t *>(q) + static_cast<size_t>(qr) * Hq * hd + head * hd;
     dst[i] = cvt16(a * t.x - b * t.y, oh);
     dst[i + half] = cvt16(b * t.x + a * t.y, oh);
   }
@@ -208,7 +211,7 @@ rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, _
                        const int32_t *__restrict__ row_pos, const int32_t *__restrict__ row_done,
                        const int32_t *__restrict__ page_table, int pt_width,
                        int R, int Hq, int Hkv, int hd, int page_size, int n_pages, int max_pos, int *status,
-                       int out_half) {
+                       int out_half, const int32_t *q_row) {
   early_start_sync();
   const bool oh = out_half != 0;
   const int r = blockIdx.x;
@@ -234,8 +237,10 @@ rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, _
       }
     }
   }
-  const bool ended = row_done && row_done[r];            // an ended row is only cleared
+  // an ended row (or a padding row of a compacted step: no page-table row) is only cleared
+  const bool ended = (row_done && row_done[r]) || row_pt[r] < 0;
   const int pos = ended ? -1 : row_pos[r];
+  const int qr = (q_row && !ended) ? q_row[r] : r;       // row of the query buffer this row writes
   int page = -1;
   if (pos >= 0 && pos < max_pos) page = page_table[static_cast<size_t>(row_pt[r]) * pt_width + pos / page_size];
   const bool bad = page < 0 || page >= n_pages;
@@ -276,7 +281,7 @@ rope_append_vec_kernel(float *__restrict__ qkv, __nv_bfloat16 *__restrict__ q, _
       const uint2 hi = pack_16x4(y.x * t01.x + x.x * t01.y, y.y * t01.z + x.y * t01.w, y.z * t23.x + x.z * t23.y,
                                  y.w * t23.z + x.w * t23.w, oh);
       if (unit < Hq) {
-        __nv_bfloat16 *dst = q + static_cast<size_t>(r) * Hq * hd + unit * hd + i;
+        __nv_bfloat16 *dst = q + static_cast<size_t>(qr) * Hq * hd + unit * hd + i;
         *reinterpret_cast<uint2 *>(dst) = lo;
         *reinterpret_cast<uint2 *>(dst + half) = hi;
       } else {
@@ -318,21 +323,87 @@ __global__ void copy_pages_kernel(__nv_bfloat16 *kv, const int32_t *src_page, co
 
 // Start of decode step j = *d_step + 1: row b feeds the token produced at step j-1 at
 // position len0[b] + j - 1.  One block; the counter is bumped after every thread has read it.
-__global__ void decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
-                                   int32_t *row_tok, int32_t *row_pos, int B, int eos_id, int32_t *row_done) {
+//
+// With `c` (compaction, used with an end token): the sequences that have not ended are packed to the
+// front of the activation rows, in sequence order, so that the step's projections run on the live
+// rows only.  row r of the step then belongs to sequence c.row_seq[r] (-1: padding row), sequence b
+// sits in row c.seq_row[b] (-1: ended), positions are kept both per row and per sequence, and an
+// ended sequence receives its end token / log-probability 0 for this step here.
+struct Compaction {
+  int32_t *row_seq, *seq_row, *seq_pos, *n_live;
+  int32_t *out_tok;
+  float *out_lp;
+};
+__global__ void __launch_bounds__(512)
+decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0, int32_t *row_tok,
+                   int32_t *row_pos, int B, int eos_id, int32_t *row_done, Compaction c) {
+  __shared__ int warp_sum[16];
+  __shared__ int base_s;
   early_start_sync();
   const int j = *d_step + 1;
+  if (threadIdx.x == 0) base_s = 0;
   __syncthreads();
-  for (int b = threadIdx.x; b < B; b += blockDim.x) {
-    const int32_t tok = tok_hist[static_cast<size_t>(b) * T + (j - 1)];
-    row_tok[b] = tok;
-    row_pos[b] = seq_len0[b] + j - 1;
-    // a sequence that is fed its end token has ended and stays ended whatever the token buffer holds
-    // at later positions (a given trajectory may be padded with other ids after its end token); its
-    // attention and cache writes are skipped from here on.  The flags are cleared when a rollout begins.
-    if (row_done && eos_id >= 0 && tok == eos_id) row_done[b] = 1;
+  if (!c.row_seq) {
+    for (int b = threadIdx.x; b < B; b += blockDim.x) {
+      const int32_t tok = tok_hist[static_cast<size_t>(b) * T + (j - 1)];
+      row_tok[b] = tok;
+      row_pos[b] = seq_len0[b] + j - 1;
+      // a sequence that is fed its end token has ended and stays ended whatever the token buffer holds
+      // at later positions (a given trajectory may be padded with other ids after its end token); its
+      // attention and cache writes are skipped from here on.  The flags are cleared when a rollout begins.
+      if (row_done && eos_id >= 0 && tok == eos_id) row_done[b] = 1;
+    }
+    if (threadIdx.x == 0) *d_step = j;
+    return;
   }
-  if (threadIdx.x == 0) *d_step = j;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  for (int b0 = 0; b0 < B; b0 += blockDim.x) {          // same trip count in every thread
+    const int b = b0 + threadIdx.x;
+    int32_t tok = 0;
+    int live = 0;
+    if (b < B) {
+      tok = tok_hist[static_cast<size_t>(b) * T + (j - 1)];
+      if (tok == eos_id) row_done[b] = 1;
+      live = row_done[b] ? 0 : 1;
+    }
+    // block-wide exclusive scan of the live flags
+    const unsigned ballot = __ballot_sync(0xffffffffu, live);
+    const int in_warp = __popc(ballot & ((1u << lane) - 1u));
+    if (lane == 0) warp_sum[warp] = __popc(ballot);
+    __syncthreads();
+    int before = base_s;
+    for (int w = 0; w < warp; ++w) before += warp_sum[w];
+    int total = 0;
+    for (int w = 0; w < nw; ++w) total += warp_sum[w];
+    if (b < B) {
+      const int pos = seq_len0[b] + j - 1;
+      c.seq_pos[b] = pos;
+      if (live) {
+        const int r = before + in_warp;
+        c.row_seq[r] = b;
+        c.seq_row[b] = r;
+        row_tok[r] = tok;
+        row_pos[r] = pos;
+      } else {
+        c.seq_row[b] = -1;
+        c.out_tok[static_cast<size_t>(b) * T + j] = eos_id;
+        c.out_lp[static_cast<size_t>(b) * T + j] = 0.f;
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) base_s += total;
+    __syncthreads();
+  }
+  const int n_live = base_s;
+  for (int r = n_live + threadIdx.x; r < B; r += blockDim.x) {      // padding rows: a valid token, no sequence
+    c.row_seq[r] = -1;
+    row_tok[r] = 0;
+    row_pos[r] = 0;
+  }
+  if (threadIdx.x == 0) {
+    *c.n_live = n_live;
+    *d_step = j;
+  }
 }
 
 __global__ void set_int_kernel(int32_t *p, int32_t v) { *p = v; }
@@ -537,25 +608,29 @@ __global__ void __launch_bounds__(kSamplerThreads)
 sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t *seq_ids, const int32_t *d_step,
                uint32_t j_host, float inv_temperature, uint32_t key0, uint32_t key1, const int32_t *forced,
                int forced_stride, int32_t *out_tok, float *out_lp, int out_stride, int eos_id,
-               const uint2 *nucleus_cut, const int32_t *row_done, uint32_t seq_base) {
+               const uint2 *nucleus_cut, const int32_t *row_done, uint32_t seq_base, const int32_t *row_seq) {
   __shared__ float sm_m[32], sm_l[32], sm_score[32];
   __shared__ int sm_id[32];
   early_start_sync();
   const int r = blockIdx.x;
+  // compacted step: logits row r belongs to sequence row_seq[r] (its noise stream, its output slot);
+  // a padding row has no sequence
+  const int seq = row_seq ? row_seq[r] : r;
+  if (seq < 0) return;
   const uint32_t j = d_step ? static_cast<uint32_t>(*d_step) : j_host;
   if (eos_id >= 0 && j > 0 && row_done) {
     // End-of-sequence rule: the sequence is finished once one of the tokens fed so far (the forced
     // ones when scoring a given trajectory) was eos_id, which the step's preparation kernel records
     // per row; finished positions hold eos_id with log-probability 0.
-    if (row_done[r]) {
+    if (row_done[seq]) {
       if (threadIdx.x == 0) {
-        out_tok[static_cast<size_t>(r) * out_stride + j] = eos_id;
-        out_lp[static_cast<size_t>(r) * out_stride + j] = 0.f;
+        out_tok[static_cast<size_t>(seq) * out_stride + j] = eos_id;
+        out_lp[static_cast<size_t>(seq) * out_stride + j] = 0.f;
       }
       return;
     }
   }
-  const uint32_t s_id = seq_base + (seq_ids ? static_cast<uint32_t>(seq_ids[r]) : static_cast<uint32_t>(r));
+  const uint32_t s_id = seq_base + (seq_ids ? static_cast<uint32_t>(seq_ids[r]) : static_cast<uint32_t>(seq));
   const float *z = logits + static_cast<size_t>(r / rows_per_logit_row) * V;
   const uint2 key = make_uint2(key0, key1);
   // top-p: only ids that rank at or before the row's cut (score descending, id ascending) belong to
@@ -633,9 +708,9 @@ sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t
       best_update(bb, sm_score[i], sm_id[i]);
     }
     const int tok = bb.id < V ? bb.id : 0;
-    const size_t o = static_cast<size_t>(r) * out_stride + j;
+    const size_t o = static_cast<size_t>(seq) * out_stride + j;
     out_tok[o] = tok;
-    const int scored = forced ? forced[static_cast<size_t>(r) * forced_stride + j] : tok;
+    const int scored = forced ? forced[static_cast<size_t>(seq) * forced_stride + j] : tok;
     const int sc_id = (scored >= 0 && scored < V) ? scored : 0;
     const float s_sc = z[sc_id] * inv_temperature;
     out_lp[o] = in_nucleus(s_sc, sc_id) ? s_sc - (mm + logf(ll)) : -INFINITY;
@@ -693,14 +768,15 @@ cudaError_t rope_table_launch(float2 *table, int max_pos, int head_dim, double t
 }
 cudaError_t rope_append_launch(float *qkv, __nv_bfloat16 *q, __nv_bfloat16 *kv_layer, const float2 *rope_table,
                                RowMeta meta, const int32_t *page_table, int pt_width, int R, int Hq, int Hkv, int hd,
-                               int page_size, int n_pages, int max_pos, int *status, cudaStream_t s, bool out_half) {
+                               int page_size, int n_pages, int max_pos, int *status, cudaStream_t s, bool out_half,
+                               const int32_t *q_row) {
   if (hd % 8 == 0 && (reinterpret_cast<uintptr_t>(qkv) & 15) == 0)
     return launch_early(rope_append_vec_kernel, dim3(R), dim3(256), 0, s, qkv, q, kv_layer, rope_table, meta.row_pt,
                         meta.row_pos, meta.row_done, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos,
-                        status, out_half ? 1 : 0);
+                        status, out_half ? 1 : 0, q_row);
   return launch_early(rope_append_kernel, dim3(R), dim3(256), 0, s, qkv, q, kv_layer, rope_table, meta.row_pt,
                       meta.row_pos, meta.row_done, page_table, pt_width, R, Hq, Hkv, hd, page_size, n_pages, max_pos,
-                      status, out_half ? 1 : 0);
+                      status, out_half ? 1 : 0, q_row);
 }
 cudaError_t swiglu_launch(const float *gu, __nv_bfloat16 *act, int R, int F, cudaStream_t s, bool out_half) {
   const size_t n = static_cast<size_t>(R) * F;
@@ -720,19 +796,21 @@ cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page
 }
 cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
                                int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s, int eos_id,
-                               int32_t *row_done) {
+                               int32_t *row_done, const CompactRows *cr, int32_t *out_tok, float *out_lp) {
+  Compaction c{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  if (cr) c = Compaction{cr->row_seq, cr->seq_row, cr->seq_pos, cr->n_live, out_tok, out_lp};
   return launch_early(decode_prep_kernel, dim3(1), dim3(512), 0, s, d_step, tok_hist, T, seq_len0, row_tok, row_pos, B,
-                      eos_id, row_done);
+                      eos_id, row_done, c);
 }
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row, const int32_t *seq_ids,
                            const int32_t *d_step, uint32_t j_host, float temperature, uint64_t seed,
                            const int32_t *forced, int forced_stride, int32_t *out_tok, float *out_lp, int out_stride,
                            cudaStream_t s, int eos_id, const uint2 *nucleus_cut, const int32_t *row_done,
-                           uint32_t seq_base) {
+                           uint32_t seq_base, const int32_t *row_seq) {
   return launch_early(sampler_kernel, dim3(R), dim3(kSamplerThreads), 0, s, logits, V, rows_per_logit_row, seq_ids,
                       d_step, j_host, 1.0f / temperature, static_cast<uint32_t>(seed & 0xffffffffu),
                       static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok, out_lp, out_stride, eos_id,
-                      nucleus_cut, row_done, seq_base);
+                      nucleus_cut, row_done, seq_base, row_seq);
 }
 cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n, uint32_t *words,
                                float *uniform, cudaStream_t s) {

@@ -88,7 +88,7 @@ Limits limits_of(const echo_config &c) {
 struct Layout {
   size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
   size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
-      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, row_done, copy_src, copy_dst, d_step, status, attn_work, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, total;
+      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, row_done, copy_src, copy_dst, d_step, status, attn_work, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, row_seq, seq_row, seq_pos, n_live, total;
   size_t weight_bytes, kv_layer_elems, n_tables_ints;
   int n_chunks_max;
 };
@@ -135,6 +135,10 @@ Layout layout_of(const echo_config &c) {
   lo.retile_stage = take(kRetileStageBytes);       // bounce buffer for snapshots in pageable host memory
   lo.nucleus_cut = take(static_cast<size_t>(M.B) * 8);   // top-p: one (score key, id) cut per logits row
   lo.row_done = take(static_cast<size_t>(M.B) * 4);      // end-of-sequence rule: rows whose sequence has ended
+  lo.row_seq = take(static_cast<size_t>(M.B) * 4);       // compaction of ended sequences out of a decode step's rows
+  lo.seq_row = take(static_cast<size_t>(M.B) * 4);
+  lo.seq_pos = take(static_cast<size_t>(M.B) * 4);
+  lo.n_live = take(4);
   lo.copy_src = take(static_cast<size_t>(M.B) * 4);
   lo.copy_dst = take(static_cast<size_t>(M.B) * 4);
   lo.d_step = take(4);
@@ -191,6 +195,11 @@ struct echo_ctx {
   bool long_suffix = false;   // decode steps whose sequences hold many generated tokens (see kLongSuffix)
   int attn_suffix_impl = 0, attn_prefix_impl = 0;   // diagnostic kernel choices (ECHO_ATTN_IMPL / ECHO_ATTN_PREFIX)
   int chunk_rows = kChunkRows;
+  // With an end token the decode steps run on the rows of the sequences that have not ended (see
+  // decode_step); the host follows the number of live rows two windows of steps behind the GPU.
+  bool compact = false;
+  int32_t *h_live = nullptr;          // page-locked: live rows reported at the end of each window
+  cudaEvent_t live_ev[3] = {nullptr, nullptr, nullptr};
   bool prefill_rows = false;  // ECHO_ATTN_PREFILL=rows: the one-query-per-row kernel for the prompt prefill too
   uint32_t seq_base = 0;      // added to p * G + g in the noise streams (echo_set_sequence_base)
   // parity hook (echo_debug_capture): residual stream before / after one layer
@@ -340,7 +349,8 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
   } while (0)
 
 // All layers for R activation rows already embedded in x.
-int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int decode_P = 0, int decode_G = 0) {
+int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int decode_P = 0, int decode_G = 0,
+                   const CompactRows *cr = nullptr) {
   const Dims &D = ctx->D;
   const Layout &lo = ctx->lo;
   float *x = ctx->ptr<float>(lo.x);
@@ -371,15 +381,18 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int d
     TRY(run_gemm(ctx, &w.tm_qkv[l], w.wqkv[l], h, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE, !ctx->use_simt, nullptr,
                  hf));
     LAUNCH(rope_append_launch(qkv, q, kv_layer, rope, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
-                              ctx->M.n_pages, ctx->M.max_pos, status, ctx->stream, hf));
+                              ctx->M.n_pages, ctx->M.max_pos, status, ctx->stream, hf, cr ? cr->row_seq : nullptr));
     if (decode_P > 0 && ctx->fast_decode) {
       ProfScope prof(ctx, PROF_ATTN);
+      // a compacted step: attention stays per sequence (q, positions, ended flags and page-table rows by
+      // sequence id) and writes each live sequence's output into the activation row it occupies
       DecodeAttnArgs da{&ctx->tm_kv, q, attn, ctx->ptr<float>(lo.pre_o), ctx->ptr<float2>(lo.pre_ml), pt,
-                        ctx->M.pt_width, meta.row_pos, ctx->ptr<int32_t>(lo.full_pages),
+                        ctx->M.pt_width, cr ? cr->seq_pos : meta.row_pos, ctx->ptr<int32_t>(lo.full_pages),
                         static_cast<int>(static_cast<size_t>(l) * (lo.kv_layer_elems / D.hd)), decode_P, decode_G,
-                        D.Hq, D.Hkv, D.hd, ctx->M.n_pages, status, meta.row_done,
+                        D.Hq, D.Hkv, D.hd, ctx->M.n_pages, status,
+                        cr ? ctx->ptr<int32_t>(lo.row_done) : meta.row_done,
                         ctx->long_suffix ? nullptr : ctx->ptr<int>(lo.attn_work), hf ? 1 : 0, ctx->attn_suffix_impl,
-                        ctx->attn_prefix_impl};
+                        ctx->attn_prefix_impl, cr ? cr->seq_row : nullptr};
       LAUNCH(attention_decode_launch(da, ctx->stream));
       ctx->launches++;                      // two kernels per call
     } else if (decode_P == 0 && ctx->fast_decode && !ctx->prefill_rows) {
@@ -605,34 +618,41 @@ int upload_plan(echo_ctx *ctx, const Plan &pl) {
 // One decode step: token j-1 in, token j out.  Every kernel reads the step index from
 // device memory, so the same launches (or the same captured graph) serve every step.
 int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t *tok_hist, float temperature,
-                uint64_t seed, const int32_t *forced, int32_t *out_tokens, float *out_logprobs) {
+                uint64_t seed, const int32_t *forced, int32_t *out_tokens, float *out_logprobs, int rows) {
+  // rows: activation rows of this step's projections.  Without an end token: all P*G sequences.  With
+  // one (ctx->compact): the preparation kernel packs the sequences that have not ended to the front,
+  // and `rows` is an upper bound of their number that the host knows (see rollout_impl).
   const Layout &lo = ctx->lo;
   int32_t *d_step = ctx->ptr<int32_t>(lo.d_step);
   int32_t *row_tok = ctx->ptr<int32_t>(lo.dec_row_tok);
   int32_t *row_pos = ctx->ptr<int32_t>(lo.dec_row_pos);
   ProfScope prof_step(ctx, PROF_STEP);
   int32_t *row_done = ctx->cfg.eos_id >= 0 ? ctx->ptr<int32_t>(lo.row_done) : nullptr;
+  CompactRows crs{ctx->ptr<int32_t>(lo.row_seq), ctx->ptr<int32_t>(lo.seq_row), ctx->ptr<int32_t>(lo.seq_pos),
+                  ctx->ptr<int32_t>(lo.n_live)};
+  const CompactRows *cr = ctx->compact ? &crs : nullptr;
   LAUNCH(decode_prep_launch(d_step, tok_hist, pl.T, ctx->ptr<int32_t>(lo.seq_len0), row_tok, row_pos, pl.B,
-                            ctx->stream, ctx->cfg.eos_id, row_done));
-  LAUNCH(embed_launch(w.embed, row_tok, nullptr, ctx->ptr<float>(lo.x), pl.B, ctx->D.d, ctx->D.V,
+                            ctx->stream, ctx->cfg.eos_id, row_done, cr, out_tokens, out_logprobs));
+  LAUNCH(embed_launch(w.embed, row_tok, nullptr, ctx->ptr<float>(lo.x), rows, ctx->D.d, ctx->D.V,
                       ctx->ptr<int>(lo.status), ctx->stream));
-  RowMeta meta{ctx->ptr<int32_t>(lo.dec_row_pt), row_pos, row_done};
+  // page-table row of an activation row: its sequence id (compacted: row_seq, -1 for padding rows)
+  RowMeta meta{cr ? cr->row_seq : ctx->ptr<int32_t>(lo.dec_row_pt), row_pos, cr ? nullptr : row_done};
   ctx->cap_decode = true;
-  const int rc_layers = forward_layers(ctx, w, pl.B, meta, pl.P, pl.G);
+  const int rc_layers = forward_layers(ctx, w, rows, meta, pl.P, pl.G, cr);
   ctx->cap_decode = false;
   TRY(rc_layers);
-  TRY(lm_head(ctx, w, ctx->ptr<float>(lo.x), pl.B));
+  TRY(lm_head(ctx, w, ctx->ptr<float>(lo.x), rows));
   {
     ProfScope prof(ctx, PROF_SAMPLER);
     const uint2 *cut = nullptr;
     if (ctx->cfg.top_p > 0.f && ctx->cfg.top_p < 1.f) {
-      LAUNCH(nucleus_cut_launch(ctx->ptr<float>(lo.logits), pl.B, ctx->D.V, temperature, ctx->cfg.top_p,
+      LAUNCH(nucleus_cut_launch(ctx->ptr<float>(lo.logits), rows, ctx->D.V, temperature, ctx->cfg.top_p,
                                 ctx->ptr<uint2>(lo.nucleus_cut), ctx->stream));
       cut = ctx->ptr<uint2>(lo.nucleus_cut);
     }
-    LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), pl.B, ctx->D.V, 1, nullptr, d_step, 0, temperature, seed,
-                          forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream, ctx->cfg.eos_id, cut, row_done,
-                          ctx->seq_base));
+    LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), rows, ctx->D.V, 1, nullptr, d_step, 0, temperature, seed,
+                          forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream, ctx->cfg.eos_id, cut,
+                          cr ? nullptr : row_done, ctx->seq_base, cr ? cr->row_seq : nullptr));
   }
   return ECHO_OK;
 }
@@ -702,6 +722,8 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   }
   if (ctx->cfg.eos_id >= 0)       // no sequence has ended yet
     CK(cudaMemsetAsync(ctx->arena + lo.row_done, 0, static_cast<size_t>(pl.B) * 4, ctx->stream));
+  if (ctx->compact)               // padding rows of a compacted step are read by the output projection: keep them finite
+    CK(cudaMemsetAsync(ctx->arena + lo.attn, 0, static_cast<size_t>(pl.B) * D.Hq * D.hd * 2, ctx->stream));
   // ---- prefill: once per prompt, in chunks of ctx->chunk_rows tokens --------
   cudaEvent_t pf_a = nullptr, pf_b = nullptr;
   if (ctx->prof_now && (pf_a = prof_event(ctx)) && (pf_b = prof_event(ctx))) cudaEventRecord(pf_a, ctx->stream);
@@ -727,60 +749,98 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   // ---- decode steps 1..T-1 ----------------------------------------------------
   const int32_t *tok_hist = forced ? forced : out_tokens;
   const int n_steps = T - 1;
-  // Two captures of the same step, which differ in the suffix attention kernel: resident CTAs while
-  // the sequences hold few generated tokens (their fixed cost per item is what counts), one CTA per
-  // (sequence, kv head) from kLongSuffix generated tokens on (the launch is bound by the KV stream).
-  cudaGraph_t graph[2] = {nullptr, nullptr};
-  cudaGraphExec_t exec[2] = {nullptr, nullptr};
-  int64_t per_step = 0;
-  if (n_steps > 1 && ctx->use_graph && ctx->stream != nullptr) {
-    for (int v = 0; v < 2; ++v) {
-      if (v == 1 && n_steps < kLongSuffix) break;
-      const int64_t before = ctx->launches;
-      if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
-        cudaGetLastError();
-        break;
-      }
-      ctx->long_suffix = v == 1;
-      int src = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs);
-      ctx->long_suffix = false;
-      cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph[v]);
-      per_step = ctx->launches - before;
-      ctx->launches = before;
-      if (src != ECHO_OK) {
-        for (int u = 0; u < 2; ++u) {
-          if (exec[u]) cudaGraphExecDestroy(exec[u]);
-          if (graph[u]) cudaGraphDestroy(graph[u]);
-        }
-        return src;
-      }
-      if (e != cudaSuccess || cudaGraphInstantiate(&exec[v], graph[v], 0) != cudaSuccess) {
-        cudaGetLastError();
-        exec[v] = nullptr;
-      }
+  // Captures of the same step.  They differ in the suffix attention kernel: resident CTAs while the
+  // sequences hold few generated tokens (their fixed cost per item is what counts), one CTA per
+  // (sequence, kv head) from kLongSuffix generated tokens on (the launch is bound by the KV stream);
+  // and, with an end token, in the number of activation rows: the projections' cost falls in steps
+  // (more than 128 rows, 65-128, 33-64, up to 32), so there is one capture per such row count below
+  // the batch size.  Captured when first needed.
+  std::vector<int> buckets{pl.B};
+  if (ctx->compact)
+    for (int m : {128, 64, 32})
+      if (m < pl.B) buckets.push_back(m);
+  const int n_b = static_cast<int>(buckets.size());
+  std::vector<cudaGraph_t> graph(2 * n_b, nullptr);
+  std::vector<cudaGraphExec_t> exec(2 * n_b, nullptr);
+  std::vector<char> tried(2 * n_b, 0);
+  std::vector<int64_t> per_step(2 * n_b, 0);
+  const bool graphs_ok = n_steps > 1 && ctx->use_graph && ctx->stream != nullptr;
+  auto release_graphs = [&]() {
+    for (size_t u = 0; u < exec.size(); ++u) {
+      if (exec[u]) cudaGraphExecDestroy(exec[u]);      // executions already enqueued keep their resources
+      if (graph[u]) cudaGraphDestroy(graph[u]);
     }
-  }
+  };
+  auto capture = [&](int v, int bi) -> int {
+    const int u = v * n_b + bi;
+    tried[u] = 1;
+    const int64_t before = ctx->launches;
+    if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      cudaGetLastError();
+      return ECHO_OK;
+    }
+    ctx->long_suffix = v == 1;
+    const int src = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs, buckets[bi]);
+    ctx->long_suffix = false;
+    cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph[u]);
+    per_step[u] = ctx->launches - before;
+    ctx->launches = before;
+    if (src != ECHO_OK) return src;
+    if (e != cudaSuccess || cudaGraphInstantiate(&exec[u], graph[u], 0) != cudaSuccess) {
+      cudaGetLastError();
+      exec[u] = nullptr;
+    }
+    return ECHO_OK;
+  };
+  // Live rows (compaction): the preparation kernel of every step leaves the number of sequences that
+  // have not ended in device memory; at the end of each window of kLiveWindow steps it is copied to
+  // page-locked host memory, and the host reads the value of window w - 2 before it enqueues window w.
+  // The count never rises during a rollout, so an older value is an upper bound of the current one.
+  constexpr int kLiveWindow = 32;
+  int live_bound = pl.B, bi = 0;
   int rc_steps = ECHO_OK;
   for (int j = 1; j <= n_steps && rc_steps == ECHO_OK; ++j) {
+    if (ctx->compact && (j - 1) % kLiveWindow == 0) {
+      const int wdw = (j - 1) / kLiveWindow;
+      if (wdw >= 2) {
+        cudaError_t se = cudaEventSynchronize(ctx->live_ev[(wdw - 2) % 3]);
+        if (se != cudaSuccess) {
+          rc_steps = fail_cuda(ctx, se, "cudaEventSynchronize(live rows)");
+          break;
+        }
+        live_bound = std::min(live_bound, static_cast<int>(ctx->h_live[(wdw - 2) % 3]));
+        bi = 0;
+        for (int k = 1; k < n_b; ++k)
+          if (buckets[k] >= live_bound) bi = k;          // buckets fall: the last one that still holds every live row
+      }
+    }
     const bool sampled = ctx->prof_every > 0 && (j % ctx->prof_every == 0);
     const int v = j >= kLongSuffix ? 1 : 0;
-    if (exec[v] && !sampled) {
-      cudaError_t le = cudaGraphLaunch(exec[v], ctx->stream);
+    const int u = v * n_b + bi;
+    if (graphs_ok && !sampled && !tried[u]) rc_steps = capture(v, bi);
+    if (rc_steps != ECHO_OK) break;
+    if (exec[u] && !sampled) {
+      cudaError_t le = cudaGraphLaunch(exec[u], ctx->stream);
       if (le != cudaSuccess) rc_steps = fail_cuda(ctx, le, "cudaGraphLaunch");
-      ctx->launches += per_step;
+      ctx->launches += per_step[u];
     } else {
       ctx->prof_now = sampled;
       ctx->prof_step = j;
       ctx->long_suffix = v == 1;
-      rc_steps = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs);
+      rc_steps = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs, buckets[bi]);
       ctx->long_suffix = false;
       ctx->prof_now = false;
     }
+    if (ctx->compact && rc_steps == ECHO_OK && (j % kLiveWindow == 0) && j < n_steps) {
+      const int wdw = j / kLiveWindow - 1;               // the window that just ended
+      cudaError_t ce = cudaMemcpyAsync(&ctx->h_live[wdw % 3], ctx->arena + lo.n_live, 4, cudaMemcpyDeviceToHost,
+                                       ctx->stream);
+      if (ce == cudaSuccess) ce = cudaEventRecord(ctx->live_ev[wdw % 3], ctx->stream);
+      if (ce != cudaSuccess) rc_steps = fail_cuda(ctx, ce, "live rows readback");
+    }
   }
-  for (int v = 0; v < 2; ++v) {
-    if (exec[v]) cudaGraphExecDestroy(exec[v]);      // executions already enqueued keep their resources
-    if (graph[v]) cudaGraphDestroy(graph[v]);
-  }
+  release_graphs();
+  ctx->stats.last_step_rows = static_cast<float>(buckets[bi]);
   if (rc_steps != ECHO_OK) return rc_steps;
   CK(cudaEventRecord(ctx->ev_end, ctx->stream));
   CK(cudaEventRecord(wp->last_use, ctx->stream));
@@ -952,6 +1012,12 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
   if ((e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_tables), ctx->h_tables_ints * 4, cudaHostAllocDefault)) !=
       cudaSuccess)
     return bail(e, "cudaHostAlloc");
+  if ((e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_live), 3 * sizeof(int32_t), cudaHostAllocDefault)) !=
+      cudaSuccess)
+    return bail(e, "cudaHostAlloc");
+  for (int i = 0; i < 3; ++i)
+    if ((e = cudaEventCreateWithFlags(&ctx->live_ev[i], cudaEventDisableTiming)) != cudaSuccess)
+      return bail(e, "cudaEventCreate");
   if ((e = gemm_tc_configure()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute");
   if ((e = gemm_pair_configure()) != cudaSuccess) return bail(e, "cudaFuncSetAttribute");
   // padding keys of a partly filled page take part in the P*V products with weight zero: the pool
@@ -977,6 +1043,10 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
       }
       ctx->fast_decode = true;
     }
+  }
+  {
+    const char *nc = getenv("ECHO_NO_COMPACT");
+    ctx->compact = ctx->cfg.eos_id >= 0 && ctx->fast_decode && !(nc && nc[0] == '1');
   }
   if ((e = cudaMemsetAsync(ctx->arena + lo.status, 0, 4, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
   if ((e = cudaMemsetAsync(ctx->arena + lo.attn_work, 0, 8, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
@@ -1013,6 +1083,9 @@ int echo_destroy(echo_ctx *ctx) {
   if (ctx->ev_first) cudaEventDestroy(ctx->ev_first);
   if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
   if (ctx->h_tables) cudaFreeHost(ctx->h_tables);
+  if (ctx->h_live) cudaFreeHost(ctx->h_live);
+  for (int i = 0; i < 3; ++i)
+    if (ctx->live_ev[i]) cudaEventDestroy(ctx->live_ev[i]);
   for (cudaEvent_t e : ctx->prof_pool) cudaEventDestroy(e);
   delete ctx;
   return ECHO_OK;

@@ -512,3 +512,86 @@ def test_turn_mask_matches_oracle(B):
         for shift in (False, True):
             got = B.echo_turn_mask(torch.from_numpy(x).cuda(), 77, shift).cpu().numpy()
             assert np.array_equal(got, objective.turn_mask(x, 77, shift))
+
+
+def test_rollout_of_8192_new_tokens(B):
+    """Section 5.1 generates up to 8192 new tokens per response.  A small two-layer model (head_dim 128,
+    two query heads on one kv head) decodes 8192 tokens per sequence: 513 KV pages per sequence, the
+    rotation table to position 8212, both captured graphs; one whole sequence is scored by the oracle
+    (a causal pass over 8211 positions), every step, and the scoring entry point replays it."""
+    shape = synth.DecoderShape("long", 2, 256, 2, 1, 128, 512, 2048)
+    P, G, Lp, T = 1, 2, 20, 8192
+    w_t = synth.make_weights(shape, 21)
+    w_o = decoder.Weights(synth.weights_to_bits(w_t))
+    eng = B.Engine(B.make_config(shape, P, G, Lp, T, 1))
+    eng.echo_load_policy(_gpu_weights(w_t), 1)
+    prompts = synth.make_prompts(P, Lp, shape.vocab, 61)
+    dp = torch.from_numpy(prompts).cuda()
+    tok, lp, _ = eng.echo_rollout(dp, [Lp], G, T, 1.0, 77)
+    st = eng.echo_get_stats()
+    assert st["decode_steps"] == T - 1 and st["n_pages"] == 2 + 2 * 513
+    lp_s, _ = eng.echo_score(dp, [Lp], tok, 1.0)
+    eng.echo_sync()
+    tok_h, lp_h = tok.cpu().numpy(), lp.cpu().numpy()
+    n, ex, worst = check_sequences(dims_of(shape), w_o, prompts, [Lp], G, 1.0, 77, tok_h, lp_h, [1])
+    assert n == T and ex <= 0.03 * T
+    assert float((lp_s - lp).abs().max()) < LOGPROB_TOL / 2
+    eng.close()
+
+
+def test_ended_sequences_leave_the_projection_rows(B, tiny, monkeypatch):
+    """With an end token the decode steps run on the rows of the sequences that have not ended: they are
+    packed to the front each step, and the host lowers the row count of the projections (64 -> 32 here)
+    as the count of live sequences, which it follows two windows of steps behind the GPU, falls.
+    Trajectories that end at scattered steps are scored teacher-forced: every position against the
+    oracle, ended positions = end token / 0, and the same outputs as with the packing switched off."""
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 8, 8, 16, 200
+    prompts = synth.make_prompts(P, Lp, wl.shape.vocab, 606)
+    lens = [Lp] * P
+    dp = torch.from_numpy(prompts).cuda()
+    eos = 7
+    rng = np.random.default_rng(12)
+    given = rng.integers(8, wl.shape.vocab, size=(P, G, T)).astype(np.int32)
+    ends = rng.integers(0, 150, size=(P, G))
+    ends[0, 0] = T + 5                                           # one sequence never ends
+    ends[3, 2] = 0                                               # one ends with its first token
+    for p in range(P):
+        for g in range(G):
+            if ends[p, g] < T:
+                given[p, g, ends[p, g]] = eos
+    forced = torch.from_numpy(given).cuda()
+    out = {}
+    for mode in ("packed", "unpacked"):
+        if mode == "unpacked":
+            monkeypatch.setenv("ECHO_NO_COMPACT", "1")
+        else:
+            monkeypatch.delenv("ECHO_NO_COMPACT", raising=False)
+        eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, eos_id=eos))
+        eng.echo_load_policy(w_d, 1)
+        tok_f, lp_f, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 4, forced=forced)
+        eng.echo_sync()
+        out[mode] = (tok_f.cpu().numpy(), lp_f.cpu().numpy())
+        # all but one sequence have ended by step 150: the last steps ran on 32 rows instead of 64
+        assert eng.echo_get_stats()["last_step_rows"] == (32 if mode == "packed" else 64)
+        # the context then serves a free-running rollout (all rows live again at its start)
+        tok, lp, _ = eng.echo_rollout(dp, lens, G, 12, 1.0, 4)
+        eng.echo_sync()
+        check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 1.0, 4, tok.cpu().numpy(), lp.cpu().numpy(),
+                        [0, 19, 63], eos_id=eos)
+        eng.close()
+    tok_f, lp_f = out["packed"]
+    for p in range(P):
+        for g in range(G):
+            e = ends[p, g]
+            if e < T:
+                assert np.all(lp_f[p, g, e + 1:] == 0.0) and np.all(tok_f[p, g, e + 1:] == eos)
+    for s in (0, 1, 26, 40, 63):
+        p, g = divmod(s, G)
+        sc = decoder.score_forced(dims_of(wl.shape), w_o, prompts[p], given[p, g], 1.0, 4, s, eos_id=eos)
+        assert np.max(np.abs(lp_f[p, g] - sc.logprob_given)) <= LOGPROB_TOL
+        live = np.arange(T) <= min(ends[p, g], T - 1)
+        diff = (tok_f[p, g] != sc.own_token) & live
+        assert np.all(sc.margin[diff] < 1e-2) and np.all(tok_f[p, g][diff] == sc.runner_up[diff])
+    assert np.max(np.abs(out["unpacked"][1] - lp_f)) < LOGPROB_TOL / 5
+    assert (out["unpacked"][0] == tok_f).mean() > 0.99
