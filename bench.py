@@ -590,7 +590,9 @@ def run_projections(args):
     ws = torch.empty(nws, dtype=torch.uint8, device=dev)
     st = torch.cuda.current_stream().cuda_stream
     qkv = (sh.n_q_heads + 2 * sh.n_kv_heads) * sh.head_dim
-    shapes = [("qkv", qkv, sh.d_model, 0), ("o", sh.d_model, sh.n_q_heads * sh.head_dim, 1),
+    # qkv: the engine's q/k/v projection adds into a buffer that the kernel consuming it leaves zeroed
+    # (epilogue 1 here); a stand-alone store (epilogue 0) would time a memset of the output as well
+    shapes = [("qkv", qkv, sh.d_model, 1), ("o", sh.d_model, sh.n_q_heads * sh.head_dim, 1),
               ("gate_up_swiglu", sh.d_ff, sh.d_model, 2), ("down", sh.d_model, sh.d_ff, 1),
               ("lm_head", sh.vocab, sh.d_model, 0)]
 
