@@ -474,9 +474,9 @@ def cpu_baseline_sample(eng, shape, weights, prompts, wl, dev):
             "sample": f"slice of the {wl.name}-shape workload: 1 prompt x G=1, first {Lp_s} prompt tokens, "
                       f"{SAMPLE_NEW} new tokens, scored teacher-forced along the GPU's tokens in one causal "
                       f"pass (mode C, fp64 numpy), all {shape.n_layers} layers streamed from the bf16 weights "
-                      f"(widening included).  The slice SURVEY planned (1 prompt x G=8, prompt 512, 4 tokens, "
-                      f"mode A) is beyond numpy: token-by-token decoding re-reads 8 bytes per parameter per "
-                      f"token (60 GB at this shape).",
+                      f"(widening included).  A larger slice in KV-cached mode (1 prompt x G=8, prompt 512, 4 tokens, "
+                      f"token by token) is beyond a numpy oracle: it re-reads 8 bytes per parameter per token "
+                      f"({8 * shape.n_params() / 1e9:.0f} GB at this shape).",
             "gpu_same_input": {"tokens_per_s": round(SAMPLE_NEW / t_gpu, 1), "seconds": round(t_gpu, 5),
                                "prefill_ms": round(st["prefill_ms"], 3), "decode_ms": round(st["decode_ms"], 3)},
             "tiny": tiny}

@@ -146,6 +146,17 @@ int make_out_map_box(CUtensorMap *out, void *base, uint64_t rows, uint64_t cols,
 
 // ---- projections on SM pairs (gemm_pair.cu) ---------------------------------
 // Same arithmetic as above with 2-CTA MMAs: used for more than 64 activation rows.
+// RMSNorm as the projection's prologue: before it loads activations, the launch itself computes
+// h[r] = 16-bit( x[r] * rsqrt(mean(x[r]^2) + eps) * gain ) for its M rows (each CTA a share of the rows),
+// meets at a grid-wide barrier and then reads h as its activation matrix X.  Needs every CTA of the
+// launch resident at once (gemm_pair_can_fuse_norm).  x == nullptr: off.
+struct NormPrologue {
+  const float *x = nullptr;          // fp32 [M][d]: the residual stream
+  const __nv_bfloat16 *gain = nullptr;
+  void *h = nullptr;                 // 16-bit [M][d]: written here, = PairGemmArgs::X
+  float eps = 0.f;
+  int *bar = nullptr;                // two ints, zero before the first launch: arrivals, generation
+};
 struct PairGemmArgs {
   const CUtensorMap *tmW;   // tensor map over W with box {64, 128}; for EPI_SWIGLU over [2N][K] (gate rows, then up rows)
   const void *X;            // bf16 [M][K], contiguous
@@ -158,7 +169,11 @@ struct PairGemmArgs {
   int force_split;          // 0 = choose; k > 0 = k slices along K (linear epilogues only)
   int tiled;                // 1: W is block-tiled storage and tmW a map over it (make_tiled_map, 128-row box)
   int half_in = 0;          // 1: X and W hold IEEE half values instead of bf16 (and a SwiGLU output is half)
+  NormPrologue norm;        // optional fused RMSNorm producing X (K = its row length)
 };
+// true if this launch's CTAs all fit the GPU at once (one row tile, at most as many SM pairs as can be
+// resident): the condition for the fused RMSNorm prologue
+bool gemm_pair_can_fuse_norm(int M, int N, int K, int epilogue);
 cudaError_t gemm_pair_configure();
 bool gemm_pair_supported(const void *Y, int ldY, int M, int N, int K, int epilogue);
 // k-slices per tile the launch will use; with more than one slice and EPI_STORE, Y must hold zeros

@@ -21,6 +21,8 @@
 // Both CTAs' loads report to the first CTA's "full" barriers; its MMA commits are multicast to
 // both CTAs' "empty" and "accumulator ready" barriers.  Every wait is bounded.
 
+#include <algorithm>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -113,11 +115,67 @@ __host__ __device__ constexpr uint32_t instr_desc_pair(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (16u << 24);
 }
 
+__device__ __forceinline__ int ld_acquire_gpu(const int *p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// RMSNorm prologue, run by the 512 epilogue threads of every CTA before the accumulators are due:
+// rows blockIdx.x, blockIdx.x + gridDim.x, ... of x are normalised into h (two passes over a row that
+// stays in L1/L2), then the CTA arrives at the grid-wide barrier.
+__device__ __forceinline__ void norm_rows_and_arrive(const NormPrologue &np, int M, int d, bool half_out,
+                                                     float *scratch /* 32 floats, shared */) {
+  const int tid = threadIdx.x - 64;                        // 0 .. kPairEpiThreads - 1
+  const int warp = tid >> 5, lane = tid & 31;
+  uint16_t *h = static_cast<uint16_t *>(np.h);
+  for (int r = blockIdx.x; r < M; r += gridDim.x) {
+    const float *xr = np.x + static_cast<size_t>(r) * d;
+    float ss = 0.f;
+    for (int i = tid * 4; i < d; i += kPairEpiThreads * 4) {
+      const float4 v = __ldcg(reinterpret_cast<const float4 *>(xr + i));
+      ss = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, fmaf(v.w, v.w, ss))));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (lane == 0) scratch[warp] = ss;
+    pair_epi_bar();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kPairEpiWarps; ++w) tot += scratch[w];      // same order in every thread
+    pair_epi_bar();
+    const float scale = rsqrtf(tot / static_cast<float>(d) + np.eps);
+    for (int i = tid * 4; i < d; i += kPairEpiThreads * 4) {
+      const float4 v = __ldcg(reinterpret_cast<const float4 *>(xr + i));
+      const uint2 graw = *reinterpret_cast<const uint2 *>(np.gain + i);
+      const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw.x));
+      const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&graw.y));
+      uint2 o;
+      o.x = cvt16x2(v.x * scale * g0.x, v.y * scale * g0.y, half_out);
+      o.y = cvt16x2(v.z * scale * g1.x, v.w * scale * g1.y, half_out);
+      *reinterpret_cast<uint2 *>(h + static_cast<size_t>(r) * d + i) = o;
+    }
+  }
+  __threadfence();
+  fence_proxy_async_all();                                 // the rows are read by other CTAs' tile copies
+  pair_epi_bar();
+  if (tid == 0) {
+    const int n_cta = static_cast<int>(gridDim.x);
+    if (atomicAdd(&np.bar[0], 1) == n_cta - 1) {           // last to arrive: reset the count, open the barrier
+      atomicExch(&np.bar[0], 0);
+      __threadfence();
+      atomicAdd(&np.bar[1], 1);
+    }
+  }
+}
+
 template <int BNB, int ACC>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                  const __grid_constant__ CUtensorMap tmY, int M, int N, int K, int epilogue, int split,
-                 int tiled, int half_in, int *status) {
+                 int tiled, int half_in, int *status, NormPrologue np) {
+  __shared__ float norm_scratch[32];
   using S = PairSmem<BNB, ACC>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -156,6 +214,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
   }
+  // generation of the grid-wide barrier as this launch finds it (read before any CTA can have arrived)
+  const int bar_gen0 = (np.x && threadIdx.x == 0) ? ld_acquire_gpu(&np.bar[1]) : 0;
   if (warp == 1) tc2_alloc(tmem_slot, S::kTmemCols);
   tc_fence_before();
   pair_cluster_sync();                                 // both CTAs' barriers exist before anything signals them
@@ -192,10 +252,27 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
       const int n_pre = kb_len < S::kStages ? kb_len : S::kStages;
       for (int it = 0; it < n_pre; ++it) load_w(it);
       griddep_wait();
-      for (int it = 0; it < n_pre; ++it) load_x(it);
+      bool x_ready = true;
+      if (np.x) {
+        // the activation matrix is being written by this very launch: wait (bounded) until every CTA
+        // has normalised its rows
+        x_ready = false;
+        const uint64_t t0 = global_timer_ns();
+        for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+          if (ld_acquire_gpu(&np.bar[1]) != bar_gen0) {
+            x_ready = true;
+            break;
+          }
+          if ((spin & 63u) == 63u && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) break;
+        }
+        if (!x_ready) *abort_flag = 1;
+        fence_proxy_async_all();
+      }
+      if (x_ready)
+        for (int it = 0; it < n_pre; ++it) load_x(it);
       int it = n_pre;
-      bool ok = true;
-      for (; it < kb_len; ++it) {
+      bool ok = x_ready;
+      for (; ok && it < kb_len; ++it) {
         ok = mbar_wait(&empty_bar[it % S::kStages], ((it / S::kStages) & 1) ^ 1u, abort_flag);
         if (!ok) break;
         load_w(it);
@@ -237,6 +314,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     const int cols = min(BNB, M - m0);
     constexpr int CH = BNB / 4;                         // columns per warp
     const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+    if (np.x) {
+      griddep_wait();                                  // x is the preceding kernel's output
+      norm_rows_and_arrive(np, M, K, half_in != 0, norm_scratch);
+    }
     const bool got = mbar_wait(acc_full, 0, abort_flag);
     tc_fence_after();
     if (got) {
@@ -310,6 +391,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
 }
 
 int g_pair_sms = 0;
+int g_pair_clusters = 0;        // SM pairs of the widest instantiation that can be resident at once
 
 template <int BNB, int ACC>
 cudaError_t launch_pair(const PairGemmArgs &a, int n_tiles, int m_tiles, int split, cudaStream_t stream) {
@@ -333,8 +415,10 @@ cudaError_t launch_pair(const PairGemmArgs &a, int n_tiles, int m_tiles, int spl
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = a.allow_early_start ? 2 : 1;
+  NormPrologue np = a.norm;
+  if (np.x && (m_tiles != 1 || 2 * n_tiles * split > 2 * g_pair_clusters || (a.K & 3))) return cudaErrorInvalidValue;
   return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<BNB, ACC>, *a.tmW, tmX, tmY, a.M, a.N, a.K, a.epilogue, split,
-                            a.tiled, a.half_in, a.status);
+                            a.tiled, a.half_in, a.status, np);
 }
 
 template <int BNB, int ACC>
@@ -345,6 +429,27 @@ cudaError_t configure_pair() {
 
 }  // namespace
 
+template <int BNB, int ACC>
+int max_resident_clusters(int sms) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(sms & ~1, 1, 1);
+  cfg.blockDim = dim3(kPairThreads, 1, 1);
+  cfg.dynamicSmemBytes = PairSmem<BNB, ACC>::kTotal;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<BNB, ACC>, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return n;
+}
+
 cudaError_t gemm_pair_configure() {
   cudaError_t e;
   int dev = 0;
@@ -354,7 +459,19 @@ cudaError_t gemm_pair_configure() {
   if ((e = configure_pair<256, 2>()) != cudaSuccess) return e;
   if ((e = configure_pair<128, 1>()) != cudaSuccess) return e;
   if ((e = configure_pair<128, 2>()) != cudaSuccess) return e;
+  // SM pairs that are resident at once (a GPC with an odd number of SMs leaves one without a partner):
+  // the smallest over the instantiations bounds every launch that uses the grid-wide barrier
+  g_pair_clusters = max_resident_clusters<256, 1>(g_pair_sms);
+  g_pair_clusters = std::min(g_pair_clusters, max_resident_clusters<256, 2>(g_pair_sms));
+  g_pair_clusters = std::min(g_pair_clusters, max_resident_clusters<128, 1>(g_pair_sms));
+  g_pair_clusters = std::min(g_pair_clusters, max_resident_clusters<128, 2>(g_pair_sms));
   return cudaSuccess;
+}
+
+bool gemm_pair_can_fuse_norm(int M, int N, int K, int epilogue) {
+  if (M <= 64 || M > 256 || (K & 3) || g_pair_clusters <= 0) return false;
+  const int n_tiles = (N + 2 * kPairFeat - 1) / (2 * kPairFeat);
+  return n_tiles * gemm_pair_split(M, N, K, epilogue, 0) <= g_pair_clusters;
 }
 
 bool gemm_pair_supported(const void *Y, int ldY, int M, int N, int K, int epilogue) {

@@ -88,7 +88,7 @@ Limits limits_of(const echo_config &c) {
 struct Layout {
   size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
   size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
-      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, row_done, copy_src, copy_dst, d_step, status, attn_work, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, row_seq, seq_row, seq_pos, n_live, total;
+      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, row_done, copy_src, copy_dst, d_step, status, attn_work, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, row_seq, seq_row, seq_pos, n_live, gemm_bar, total;
   size_t weight_bytes, kv_layer_elems, n_tables_ints;
   int n_chunks_max;
 };
@@ -139,6 +139,7 @@ Layout layout_of(const echo_config &c) {
   lo.seq_row = take(static_cast<size_t>(M.B) * 4);
   lo.seq_pos = take(static_cast<size_t>(M.B) * 4);
   lo.n_live = take(4);
+  lo.gemm_bar = take(8);                                 // grid-wide barrier of the fused RMSNorm prologue
   lo.copy_src = take(static_cast<size_t>(M.B) * 4);
   lo.copy_dst = take(static_cast<size_t>(M.B) * 4);
   lo.d_step = take(4);
@@ -197,6 +198,7 @@ struct echo_ctx {
   int chunk_rows = kChunkRows;
   // With an end token the decode steps run on the rows of the sequences that have not ended (see
   // decode_step); the host follows the number of live rows two windows of steps behind the GPU.
+  bool fuse_norm = false;     // RMSNorm as the prologue of the projection that consumes it (decode steps)
   bool compact = false;
   int32_t *h_live = nullptr;          // page-locked: live rows reported at the end of each window
   cudaEvent_t live_ev[3] = {nullptr, nullptr, nullptr};
@@ -298,13 +300,14 @@ int pick_bnb(int rows) {
 // Y = X * W^T through the tensor-core kernel (or the SIMT reference when selected).
 int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, const __nv_bfloat16 *X, void *Y, int ldY,
              int M, int N, int K, int epilogue, bool y_holds_zeros = false, const CUtensorMap *tmW_pair = nullptr,
-             bool half_in = false) {
+             bool half_in = false, const NormPrologue *norm = nullptr) {
   ProfScope prof(ctx, PROF_GEMM);
   if (ctx->use_pair && !ctx->use_simt && !ctx->deterministic && (epilogue != EPI_SWIGLU || tmW_pair) &&
       gemm_pair_supported(Y, ldY, M, N, K, epilogue)) {
     // more than 64 rows: 2-CTA MMAs, k-slices added into Y in memory
     PairGemmArgs a{tmW_pair ? tmW_pair : tmW, X, Y, ldY, M, N, K, epilogue, ctx->ptr<int>(ctx->lo.status),
                    ctx->use_pdl ? 1 : 0, 0, 1, half_in ? 1 : 0};
+    if (norm) a.norm = *norm;
     if (epilogue == EPI_STORE && !y_holds_zeros && gemm_pair_split(M, N, K, epilogue, 0) > 1) {
       CK(cudaMemsetAsync(Y, 0, static_cast<size_t>(M) * ldY * sizeof(float), ctx->stream));
       a.allow_early_start = 0;
@@ -342,6 +345,12 @@ int run_gemm(echo_ctx *ctx, const CUtensorMap *tmW, const __nv_bfloat16 *W, cons
   return ECHO_OK;
 }
 
+// true if run_gemm will take the SM-pair kernel for this projection
+bool takes_pair_kernel(echo_ctx *ctx, const void *Y, int ldY, int M, int N, int K, int epilogue, bool has_pair_map) {
+  return ctx->use_pair && !ctx->use_simt && !ctx->deterministic && (epilogue != EPI_SWIGLU || has_pair_map) &&
+         gemm_pair_supported(Y, ldY, M, N, K, epilogue);
+}
+
 #define TRY(expr)                 \
   do {                            \
     int rc__ = (expr);            \
@@ -376,10 +385,16 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int d
                  : cudaSuccess;
     };
     if (l == ctx->cap_layer) CK(capture(ctx->cap_pre_in, ctx->cap_dec_in));
-    LAUNCH(rmsnorm_launch(x, w.attn_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream, hf));
+    // RMSNorm: a kernel of its own, or (decode steps, when every CTA of the projection is resident at
+    // once) the prologue of the projection that consumes it
+    NormPrologue np_attn{x, w.attn_norm[l], h, ctx->cfg.rms_eps, ctx->ptr<int>(lo.gemm_bar)};
+    const bool fuse_attn = ctx->fuse_norm && decode_P > 0 &&
+                           takes_pair_kernel(ctx, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE, false) &&
+                           gemm_pair_can_fuse_norm(R, D.n_qkv(), D.d, EPI_STORE);
+    if (!fuse_attn) LAUNCH(rmsnorm_launch(x, w.attn_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream, hf));
     // the qkv buffer holds zeros here: rope_append clears every row it consumes
     TRY(run_gemm(ctx, &w.tm_qkv[l], w.wqkv[l], h, qkv, D.n_qkv(), R, D.n_qkv(), D.d, EPI_STORE, !ctx->use_simt, nullptr,
-                 hf));
+                 hf, fuse_attn ? &np_attn : nullptr));
     LAUNCH(rope_append_launch(qkv, q, kv_layer, rope, meta, pt, ctx->M.pt_width, R, D.Hq, D.Hkv, D.hd, D.Z,
                               ctx->M.n_pages, ctx->M.max_pos, status, ctx->stream, hf, cr ? cr->row_seq : nullptr));
     if (decode_P > 0 && ctx->fast_decode) {
@@ -408,8 +423,13 @@ int forward_layers(echo_ctx *ctx, const WeightBuf &w, int R, RowMeta meta, int d
                                    ctx->M.n_pages, status, ctx->stream, hf));
     }
     TRY(run_gemm(ctx, &w.tm_o[l], w.wo[l], attn, x, D.d, R, D.d, D.Hq * D.hd, EPI_ACCUM, false, nullptr, hf));
-    LAUNCH(rmsnorm_launch(x, w.mlp_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream, hf));
-    TRY(run_gemm(ctx, &w.tm_gu[l], w.wgu[l], h, act, D.F, R, D.F, D.d, EPI_SWIGLU, false, &w.tm_gu_pair[l], hf));
+    NormPrologue np_mlp{x, w.mlp_norm[l], h, ctx->cfg.rms_eps, ctx->ptr<int>(lo.gemm_bar)};
+    const bool fuse_mlp = ctx->fuse_norm && decode_P > 0 &&
+                          takes_pair_kernel(ctx, act, D.F, R, D.F, D.d, EPI_SWIGLU, true) &&
+                          gemm_pair_can_fuse_norm(R, D.F, D.d, EPI_SWIGLU);
+    if (!fuse_mlp) LAUNCH(rmsnorm_launch(x, w.mlp_norm[l], h, R, D.d, ctx->cfg.rms_eps, ctx->stream, hf));
+    TRY(run_gemm(ctx, &w.tm_gu[l], w.wgu[l], h, act, D.F, R, D.F, D.d, EPI_SWIGLU, false, &w.tm_gu_pair[l], hf,
+                 fuse_mlp ? &np_mlp : nullptr));
     TRY(run_gemm(ctx, &w.tm_down[l], w.wdown[l], act, x, D.d, R, D.d, D.F, EPI_ACCUM, false, nullptr, hf));
     if (l == ctx->cap_layer) CK(capture(ctx->cap_pre_out, ctx->cap_dec_out));
   }
@@ -1045,6 +1065,11 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
     }
   }
   {
+    const char *fn = getenv("ECHO_FUSE_NORM");
+    ctx->fuse_norm = fn && fn[0] == '1';
+  }
+  if ((e = cudaMemsetAsync(ctx->arena + lo.gemm_bar, 0, 8, ctx->stream)) != cudaSuccess) return bail(e, "cudaMemset");
+  {
     const char *nc = getenv("ECHO_NO_COMPACT");
     ctx->compact = ctx->cfg.eos_id >= 0 && ctx->fast_decode && !(nc && nc[0] == '1');
   }
@@ -1269,6 +1294,7 @@ int echo_sync(echo_ctx *ctx) {
   if (status != STATUS_OK) {
     cudaMemset(ctx->arena + ctx->lo.status, 0, 4);
     cudaMemset(ctx->arena + ctx->lo.gemm_counters, 0, static_cast<size_t>(kGemmMaxUnits) * 4);
+    cudaMemset(ctx->arena + ctx->lo.gemm_bar, 0, 8);
     return status == STATUS_WAIT_TIMEOUT ? ECHO_ERR_TIMEOUT : ECHO_ERR_DEVICE_CHECK;
   }
   return ECHO_OK;

@@ -69,8 +69,8 @@ WORKLOADS: Dict[str, Workload] = {
     "tiny": Workload("tiny", SHAPES["tiny"], 4, 4, 32, 32, prompt_seed=1001),
     "0.6B": Workload("0.6B", SHAPES["0.6B"], 64, 8, 256, 1024, prompt_seed=1002),
     "4B": Workload("4B", SHAPES["4B"], 32, 8, 512, 2048, prompt_seed=1003, half_layers=4),
-    "8B": Workload("8B", SHAPES["8B"], 32, 8, 512, 2048, prompt_seed=1004, half_layers=4),
-    "32B": Workload("32B", SHAPES["32B"], 16, 8, 1024, 2048, prompt_seed=1005, half_layers=8),
+    "8B": Workload("8B", SHAPES["8B"], 32, 8, 512, 2048, prompt_seed=1004, half_layers=8),
+    "32B": Workload("32B", SHAPES["32B"], 16, 8, 1024, 2048, prompt_seed=1005, half_layers=16),
 }
 
 # Tensor ids used in the per-tensor seed.  Layer index -1 is "not in a layer".

@@ -595,3 +595,42 @@ def test_ended_sequences_leave_the_projection_rows(B, tiny, monkeypatch):
         assert np.all(sc.margin[diff] < 1e-2) and np.all(tok_f[p, g][diff] == sc.runner_up[diff])
     assert np.max(np.abs(out["unpacked"][1] - lp_f)) < LOGPROB_TOL / 5
     assert (out["unpacked"][0] == tok_f).mean() > 0.99
+
+
+@pytest.mark.parametrize("env", [{"ECHO_DETERMINISTIC": "1"}, {"ECHO_GEMM_IMPL": "single"}, {"ECHO_GEMM_IMPL": "simt"},
+                                 {"ECHO_NO_GRAPH": "1"}, {"ECHO_NO_PDL": "1"}, {"ECHO_ATTN_IMPL": "rows"}])
+def test_diagnostic_switches_keep_parity(B, tiny, monkeypatch, env):
+    """The switches read at echo_create select other kernels or launch modes for the same arithmetic:
+    fixed-order reductions (then two runs are bit-identical), the one-CTA and the plain projection
+    kernels, no graph replay, no early kernel start, the general attention kernel.  Each against the
+    oracle on every token, with half operands in the first layer and the end-of-sequence rule on."""
+    wl, w_o, w_d = tiny
+    for k in ("ECHO_DETERMINISTIC", "ECHO_GEMM_IMPL", "ECHO_NO_GRAPH", "ECHO_NO_PDL", "ECHO_ATTN_IMPL"):
+        monkeypatch.delenv(k, raising=False)
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    P, G, Lp, T = 5, 8, 48, 40                      # 40 sequences: both projection kernel families see > 32 rows
+    prompts, lens = synth.make_ragged_prompts([48, 31, 16, 5, 40], wl.shape.vocab, 313, pad_to=Lp)
+    dp = torch.from_numpy(prompts).cuda()
+    eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, half_layers=1))
+    eng.echo_load_policy(w_d, 1)
+    tok, lp, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 99)
+    eng.echo_sync()
+    tok_h, lp_h = tok.cpu().numpy(), lp.cpu().numpy()
+    eng.close()
+    eos = int(tok_h[2, 3, 7])
+    eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, half_layers=1, eos_id=eos))
+    eng.echo_load_policy(w_d, 1)
+    tok, lp, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 99)
+    tok2, lp2, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 99)
+    eng.echo_sync()
+    tok_h, lp_h = tok.cpu().numpy(), lp.cpu().numpy()
+    n, ex, worst = check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 1.0, 99, tok_h, lp_h, range(P * G),
+                                   eos_id=eos)
+    assert n == P * G * T and ex <= 0.05 * n
+    assert np.any(tok_h[2, 3] == eos)
+    if env.get("ECHO_DETERMINISTIC") == "1":
+        assert np.array_equal(tok2.cpu().numpy(), tok_h) and np.array_equal(lp2.cpu().numpy(), lp_h)
+    else:
+        assert_same_rollout(tok2.cpu().numpy(), lp2.cpu().numpy(), tok_h, lp_h)
+    eng.close()
