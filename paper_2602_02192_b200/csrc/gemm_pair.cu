@@ -160,14 +160,7 @@ __device__ __forceinline__ void norm_rows_and_arrive(const NormPrologue &np, int
   __threadfence();
   fence_proxy_async_all();                                 // the rows are read by other CTAs' tile copies
   pair_epi_bar();
-  if (tid == 0) {
-    const int n_cta = static_cast<int>(gridDim.x);
-    if (atomicAdd(&np.bar[0], 1) == n_cta - 1) {           // last to arrive: reset the count, open the barrier
-      atomicExch(&np.bar[0], 0);
-      __threadfence();
-      atomicAdd(&np.bar[1], 1);
-    }
-  }
+  if (tid == 0) atomicAdd(&np.bar[0], 1);                  // bar[0] counts the CTAs whose rows are written
 }
 
 template <int BNB, int ACC>
@@ -214,8 +207,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmX)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
   }
-  // generation of the grid-wide barrier as this launch finds it (read before any CTA can have arrived)
-  const int bar_gen0 = (np.x && threadIdx.x == 0) ? ld_acquire_gpu(&np.bar[1]) : 0;
   if (warp == 1) tc2_alloc(tmem_slot, S::kTmemCols);
   tc_fence_before();
   pair_cluster_sync();                                 // both CTAs' barriers exist before anything signals them
@@ -254,18 +245,25 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant_
       griddep_wait();
       bool x_ready = true;
       if (np.x) {
-        // the activation matrix is being written by this very launch: wait (bounded) until every CTA
-        // has normalised its rows
+        // The activation matrix is being written by this very launch: wait (bounded) until every CTA
+        // has normalised its rows.  Both counters are zero when a launch starts: CTAs arrive only after
+        // the preceding kernels have completed, and the last CTA that has stopped looking at the
+        // arrival count (bar[1] counts those) clears both for the next launch.
         x_ready = false;
+        const int n_cta = static_cast<int>(gridDim.x);
         const uint64_t t0 = global_timer_ns();
         for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-          if (ld_acquire_gpu(&np.bar[1]) != bar_gen0) {
+          if (ld_acquire_gpu(&np.bar[0]) >= n_cta) {
             x_ready = true;
             break;
           }
           if ((spin & 63u) == 63u && (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs)) break;
         }
         if (!x_ready) *abort_flag = 1;
+        if (atomicAdd(&np.bar[1], 1) == n_cta - 1) {
+          atomicExch(&np.bar[0], 0);
+          atomicExch(&np.bar[1], 0);
+        }
         fence_proxy_async_all();
       }
       if (x_ready)

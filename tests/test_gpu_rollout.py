@@ -634,3 +634,26 @@ def test_diagnostic_switches_keep_parity(B, tiny, monkeypatch, env):
     else:
         assert_same_rollout(tok2.cpu().numpy(), lp2.cpu().numpy(), tok_h, lp_h)
     eng.close()
+
+
+def test_rmsnorm_as_projection_prologue(B, tiny, monkeypatch):
+    """ECHO_FUSE_NORM=1 moves the two RMSNorms of a decode layer into the projections that consume them
+    (a grid-wide barrier inside the kernel; needs more than 64 activation rows).  Same arithmetic: every
+    token against the oracle, and the step holds two kernels per layer fewer."""
+    wl, w_o, w_d = tiny
+    P, G, Lp, T = 9, 8, 24, 12
+    prompts, lens = synth.make_ragged_prompts([24, 9, 17, 24, 3, 20, 11, 24, 6], wl.shape.vocab, 77, pad_to=Lp)
+    dp = torch.from_numpy(prompts).cuda()
+    launched = {}
+    for mode in ("0", "1"):
+        monkeypatch.setenv("ECHO_FUSE_NORM", mode)
+        eng = B.Engine(B.make_config(wl.shape, P, G, Lp, T, half_layers=1))
+        eng.echo_load_policy(w_d, 1)
+        tok, lp, _ = eng.echo_rollout(dp, lens, G, T, 1.0, 5)
+        eng.echo_sync()
+        launched[mode] = eng.echo_get_stats()["kernels_launched"]
+        n, ex, worst = check_sequences(dims_of(wl.shape), w_o, prompts, lens, G, 1.0, 5, tok.cpu().numpy(),
+                                       lp.cpu().numpy(), range(0, P * G, 5))
+        assert ex <= 0.05 * n
+        eng.close()
+    assert launched["0"] - launched["1"] == 2 * wl.shape.n_layers * (T - 1)
