@@ -217,7 +217,7 @@ int echo_group_advantage(const float *rewards, int32_t P, int32_t G, float eps,
  * sequence: with rho_t = exp(logp_new - logp_old), the truncated importance ratio
  * w_t = min(exp(logp_old - logp_sampler), C) and the response mask m_t,
  *   out[i] = sum_t m_t w_t min(rho_t A_i, clip(rho_t, 1 - eps_clip, 1 + eps_clip) A_i) / sum_t m_t
- * (0 for an empty mask; the KL term, which needs a reference policy, is not included).
+ * (0 for an empty mask; without the KL term: echo_grpo_objective adds it).
  * logp_* dev fp32 [n][T] are log-probabilities of the taken tokens (logp_sampler is what
  * echo_rollout recorded, the other two come from echo_rollout_forced under the respective
  * weights), adv dev fp32 [n] (echo_group_advantage), mask dev uint8 [n][T] or NULL (all ones),
@@ -225,6 +225,19 @@ int echo_group_advantage(const float *rewards, int32_t P, int32_t G, float eps,
 int echo_grpo_surrogate(const float *logp_new, const float *logp_old, const float *logp_sampler,
                         const float *adv, const uint8_t *mask, int32_t n, int32_t T, float eps_clip,
                         float C, float *out, void *cuda_stream);
+
+/* The same objective with its KL regulariser (Appendix F, the equation for J-bar:
+ * ... - beta * D_KL(pi_theta || pi_ref)).  The appendix names no estimator; a rollout record holds
+ * log-probabilities of the taken tokens only, so the divergence enters as the per-token estimate
+ *   k_t = pi_ref(y_t)/pi_theta(y_t) - log(pi_ref(y_t)/pi_theta(y_t)) - 1 = exp(d) - d - 1,
+ *   d = logp_ref - logp_new  (non-negative; its mean over y_t ~ pi_theta is the exact divergence),
+ * inside the masked mean and under the truncated ratio that multiplies the whole of J-bar:
+ *   out[i] = sum_t m_t w_t (min(rho_t A_i, clip(rho_t) A_i) - beta k_t) / sum_t m_t.
+ * logp_ref dev fp32 [n][T] (echo_score / echo_rollout_forced under the reference weights); the other
+ * arguments as in echo_grpo_surrogate; beta >= 0.  Asynchronous on the stream. */
+int echo_grpo_objective(const float *logp_new, const float *logp_old, const float *logp_sampler,
+                        const float *logp_ref, const float *adv, const uint8_t *mask, int32_t n,
+                        int32_t T, float eps_clip, float C, float beta, float *out, void *cuda_stream);
 
 /* Offset of this context's sequence ids in the noise streams: sequence (p, g) of later rollouts draws
  * from the Philox stream of id base + p*G + g.  Rollout workers are independent and share nothing but

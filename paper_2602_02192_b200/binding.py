@@ -99,6 +99,8 @@ def _load() -> C.CDLL:
     lib.echo_sample_top_p.restype = C.c_int
     lib.echo_grpo_surrogate.argtypes = [vp, vp, vp, vp, vp, i32, i32, f32, f32, vp, vp]
     lib.echo_grpo_surrogate.restype = C.c_int
+    lib.echo_grpo_objective.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, f32, vp, vp]
+    lib.echo_grpo_objective.restype = C.c_int
     dbl = C.c_double
     lib.echo_mu_min.argtypes = [dbl, dbl, dbl, dbl, C.POINTER(dbl)]
     lib.echo_staleness_bound.argtypes = [i32, dbl, dbl, dbl, dbl, C.POINTER(i32)]
@@ -145,7 +147,7 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
             "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_decode_attention",
             "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error",
-            "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate",
+            "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate", "echo_grpo_objective",
             "echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible",
             "echo_set_sequence_base", "echo_debug_capture", "echo_debug_wait_limit",
             "echo_gemm_bf16_noalloc_status", "echo_probe_read_bandwidth", "echo_peer_score", "echo_chain_assemble",
@@ -364,6 +366,25 @@ def echo_turn_mask(tokens: torch.Tensor, turn_start_id: int, shift_to_targets: b
     with torch.cuda.device(tokens.device):
         _check(lib.echo_turn_mask(tokens.data_ptr(), n, T, int(turn_start_id), 1 if shift_to_targets else 0,
                                   out.data_ptr(), _stream_ptr(None)))
+    return out
+
+
+def echo_grpo_objective(logp_new: torch.Tensor, logp_old: torch.Tensor, logp_sampler: torch.Tensor,
+                        logp_ref: torch.Tensor, adv: torch.Tensor, mask: Optional[torch.Tensor], eps_clip: float,
+                        C_trunc: float, beta: float) -> torch.Tensor:
+    """The surrogate with the KL regulariser against a reference policy, one value per sequence."""
+    n, T = logp_new.shape
+    for x in (logp_new, logp_old, logp_sampler, logp_ref, adv):
+        assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    assert logp_old.shape == (n, T) and logp_sampler.shape == (n, T) and logp_ref.shape == (n, T) and adv.shape == (n,)
+    if mask is not None:
+        assert mask.is_cuda and mask.dtype == torch.uint8 and mask.is_contiguous() and mask.shape == (n, T)
+    out = torch.empty(n, dtype=torch.float32, device=logp_new.device)
+    with torch.cuda.device(logp_new.device):
+        _check(lib.echo_grpo_objective(logp_new.data_ptr(), logp_old.data_ptr(), logp_sampler.data_ptr(),
+                                       logp_ref.data_ptr(), adv.data_ptr(),
+                                       mask.data_ptr() if mask is not None else None, n, T, float(eps_clip),
+                                       float(C_trunc), float(beta), out.data_ptr(), _stream_ptr(None)))
     return out
 
 

@@ -234,9 +234,9 @@ cudaError_t nucleus_cut_launch(const float *logits, int rows, int V, float tempe
 cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n,
                                uint32_t *words, float *uniform, cudaStream_t s);
 cudaError_t advantage_launch(const float *r, int P, int G, float eps, float *out, cudaStream_t s);
-cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float *ls, const float *adv,
-                                  const uint8_t *mask, int n, int T, float eps_clip, float C, float *out,
-                                  cudaStream_t s);
+cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float *ls, const float *lr,
+                                  const float *adv, const uint8_t *mask, int n, int T, float eps_clip, float C,
+                                  float beta, float *out, cudaStream_t s);
 cudaError_t set_int_launch(int32_t *p, int32_t v, cudaStream_t s);
 // teacher-forced scoring of whole trajectories (see the kernels in elementwise.cu)
 cudaError_t score_rows_launch(int r0, int R, int T, const int32_t *seq_len0, int32_t *row_pt, int32_t *row_pos,

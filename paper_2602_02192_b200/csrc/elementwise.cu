@@ -540,11 +540,12 @@ __global__ void wait_probe_kernel(uint64_t limit_ns, int *status, unsigned long 
 }
 
 // Clipped surrogate with truncated importance sampling, one warp per sequence (all in fp32):
-// J_i = sum_t m_t min(exp(lo - ls), C) min(rho A, clip(rho, 1 - e, 1 + e) A) / sum_t m_t, rho = exp(ln - lo).
+// J_i = sum_t m_t min(exp(lo - ls), C) (min(rho A, clip(rho, 1 - e, 1 + e) A) - beta k_t) / sum_t m_t,
+// rho = exp(ln - lo), k_t = exp(d) - d - 1 with d = lr - ln (lr may be null: no KL term).
 __global__ void grpo_surrogate_kernel(const float *__restrict__ ln, const float *__restrict__ lo,
-                                      const float *__restrict__ ls, const float *__restrict__ adv,
-                                      const uint8_t *__restrict__ mask, int n, int T, float eps_clip, float C,
-                                      float *__restrict__ out) {
+                                      const float *__restrict__ ls, const float *__restrict__ lr,
+                                      const float *__restrict__ adv, const uint8_t *__restrict__ mask, int n, int T,
+                                      float eps_clip, float C, float beta, float *__restrict__ out) {
   const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (i >= n) return;
   const size_t base = static_cast<size_t>(i) * T;
@@ -555,7 +556,12 @@ __global__ void grpo_surrogate_kernel(const float *__restrict__ ln, const float 
     const float rho = expf(ln[base + t] - lo[base + t]);
     const float w = fminf(expf(lo[base + t] - ls[base + t]), C);
     const float clipped = fminf(fmaxf(rho, 1.0f - eps_clip), 1.0f + eps_clip);
-    num += w * fminf(rho * a, clipped * a);
+    float term = fminf(rho * a, clipped * a);
+    if (lr) {
+      const float d = lr[base + t] - ln[base + t];
+      term -= beta * (expm1f(d) - d);
+    }
+    num += w * term;
     den += 1.0f;
   }
 #pragma unroll
@@ -825,11 +831,11 @@ cudaError_t advantage_launch(const float *r, int P, int G, float eps, float *out
   advantage_kernel<<<(P + 7) / 8, 256, 0, s>>>(r, P, G, eps, out);
   return cudaGetLastError();
 }
-cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float *ls, const float *adv,
-                                  const uint8_t *mask, int n, int T, float eps_clip, float C, float *out,
-                                  cudaStream_t s) {
+cudaError_t grpo_surrogate_launch(const float *ln, const float *lo, const float *ls, const float *lr,
+                                  const float *adv, const uint8_t *mask, int n, int T, float eps_clip, float C,
+                                  float beta, float *out, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
-  grpo_surrogate_kernel<<<(n + 7) / 8, 256, 0, s>>>(ln, lo, ls, adv, mask, n, T, eps_clip, C, out);
+  grpo_surrogate_kernel<<<(n + 7) / 8, 256, 0, s>>>(ln, lo, ls, lr, adv, mask, n, T, eps_clip, C, beta, out);
   return cudaGetLastError();
 }
 cudaError_t score_rows_launch(int r0, int R, int T, const int32_t *seq_len0, int32_t *row_pt, int32_t *row_pos,

@@ -1272,8 +1272,18 @@ int echo_grpo_surrogate(const float *logp_new, const float *logp_old, const floa
                         void *cuda_stream) {
   if (!logp_new || !logp_old || !logp_sampler || !adv || !out || n < 0 || T < 1) return ECHO_ERR_INVALID;
   if (!(eps_clip >= 0.f) || !(C > 0.f)) return ECHO_ERR_INVALID;
-  cudaError_t e = grpo_surrogate_launch(logp_new, logp_old, logp_sampler, adv, mask, n, T, eps_clip, C, out,
-                                        static_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = grpo_surrogate_launch(logp_new, logp_old, logp_sampler, nullptr, adv, mask, n, T, eps_clip, C, 0.f,
+                                        out, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
+}
+
+int echo_grpo_objective(const float *logp_new, const float *logp_old, const float *logp_sampler, const float *logp_ref,
+                        const float *adv, const uint8_t *mask, int32_t n, int32_t T, float eps_clip, float C,
+                        float beta, float *out, void *cuda_stream) {
+  if (!logp_new || !logp_old || !logp_sampler || !logp_ref || !adv || !out || n < 0 || T < 1) return ECHO_ERR_INVALID;
+  if (!(eps_clip >= 0.f) || !(C > 0.f) || !(beta >= 0.f)) return ECHO_ERR_INVALID;
+  cudaError_t e = grpo_surrogate_launch(logp_new, logp_old, logp_sampler, logp_ref, adv, mask, n, T, eps_clip, C,
+                                        beta, out, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? ECHO_OK : ECHO_ERR_CUDA;
 }
 

@@ -191,6 +191,39 @@ def test_grpo_surrogate_against_vector_formula():
     assert np.allclose(got, want, rtol=1e-12, atol=1e-15)
 
 
+def test_kl_estimate_and_regularised_objective():
+    """Appendix F, the KL term of J-bar.  The per-token estimate is 0 for equal policies, positive
+    otherwise, and its mean over tokens drawn from pi_theta is the textbook divergence
+    sum_v pi_theta(v) log(pi_theta(v) / pi_ref(v)) (written out here over whole small distributions)."""
+    from oracle import objective
+    rng = np.random.default_rng(11)
+    for V in (2, 5, 17):
+        p = rng.dirichlet(np.ones(V))
+        q = rng.dirichlet(np.ones(V))
+        k = objective.kl_token_estimate(np.log(p), np.log(q))
+        assert np.all(k > 0) and np.allclose(objective.kl_token_estimate(np.log(p), np.log(p)), 0.0, atol=1e-15)
+        exact = sum(p[v] * (np.log(p[v]) - np.log(q[v])) for v in range(V))
+        assert np.isclose(float(np.dot(p, k)), exact, rtol=1e-12)
+        # the other direction is a different number: an estimator with the operands swapped fails this
+        assert not np.isclose(float(np.dot(p, objective.kl_token_estimate(np.log(q), np.log(p)))), exact, rtol=1e-3)
+    # one hand-worked value: pi_ref / pi_theta = 2 -> 2 - ln 2 - 1
+    assert np.isclose(objective.kl_token_estimate([np.log(0.25)], [np.log(0.5)])[0], 1.0 - np.log(2.0))
+    # in the objective: A = 0 leaves -beta * masked mean of k (w = 1); beta = 0 gives the surrogate back
+    T = 6
+    ln, lo, ls, lr = (-rng.exponential(1.0, size=(3, T)) for _ in range(4))
+    mask = np.array([[1, 1, 0, 1, 0, 0], [0] * 6, [1] * 6], dtype=np.float64)
+    adv = np.array([0.7, -1.0, 2.0])
+    k = objective.kl_token_estimate(ln, lr)
+    got = objective.grpo_objective(ln, lo, lo, lr, np.zeros(3), mask, 0.2, 2.0, 0.3)
+    assert np.allclose(got, [-0.3 * k[0, [0, 1, 3]].mean(), 0.0, -0.3 * k[2].mean()])
+    assert np.allclose(objective.grpo_objective(ln, lo, ls, lr, adv, mask, 0.2, 1.7, 0.0),
+                       objective.grpo_surrogate(ln, lo, ls, adv, mask, 0.2, 1.7))
+    # the truncated ratio multiplies the regulariser too (it multiplies the whole of J-bar): w = 2 doubles it
+    assert np.allclose(objective.grpo_objective(ln, lo, lo - np.log(3.0), lr, np.zeros(3), mask, 0.2, 2.0, 0.3), 2 * got)
+    with pytest.raises(ValueError):
+        objective.grpo_objective(ln, lo, ls, lr, adv, mask, 0.2, 1.7, -0.1)
+
+
 def test_turn_mask_hand_written_dialogue():
     """Appendix F, turn-aware masking, on a dialogue written out by hand.  S = the turn-start id.
     turns: system (c = 1), user (2), assistant (3), user (4), assistant (5): the mask selects turns 3 and 5,
