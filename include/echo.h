@@ -166,6 +166,29 @@ int echo_rollout(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
                  uint64_t seed, int32_t *out_tokens, float *out_logprobs,
                  int64_t *out_versions);
 
+/* The same rollout over a QUEUE of prompts longer than the context holds at once (Section 5.1: responses
+ * of up to 8192 tokens that end at very different lengths; Section 3.1 counts rollouts per unit time):
+ * continuous refill.  The context's max_prompts groups are slots; when every sample of a slot has ended
+ * (end token, or all T tokens generated) the next prompt of the queue is prefilled into the slot between
+ * two decode steps, while the other slots keep decoding.  Sequence (p, g) keeps the noise stream and the
+ * output row of its id p*G + g (plus the sequence base) and counts its token index from the step it was
+ * admitted at, so every sequence gets exactly the tokens echo_rollout gives it in a call that holds all
+ * n_prompts at once; only the order in which the work runs differs.
+ *   prompts      dev  int32 [n_prompts][cfg.max_prompt_len], prompt_lens host int32 [n_prompts];
+ *                n_prompts >= 1, not bounded by max_prompts
+ *   out_tokens / out_logprobs  dev [n_prompts][G][T]; positions after a sequence's end token hold the
+ *                end token / 0, as in echo_rollout
+ *   out_versions host int64 [n_prompts][G] (one version for the whole call)
+ *   forced_tokens NULL, or dev int32 [n_prompts][G][T]: teacher-forced as in echo_rollout_forced (the
+ *                sequences then end where the given tokens hold the end token)
+ * The host follows the ended flags once every 16 decode steps (it waits for the GPU at those points), so
+ * the call returns when the last steps are enqueued, not before.  Needs the tensor-core decode attention
+ * (else ECHO_ERR_UNSUPPORTED).  echo_get_stats().decode_steps reports the steps the queue took. */
+int echo_rollout_queue(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens,
+                       int32_t n_prompts, int32_t G, int32_t max_new_tokens, float temperature,
+                       uint64_t seed, const int32_t *forced_tokens, int32_t *out_tokens,
+                       float *out_logprobs, int64_t *out_versions);
+
 /* Teacher-forced variant: step j feeds forced_tokens[p][g][j] (dev int32
  * [P][G][T]) instead of the sampled token.  out_tokens[p][g][j] is the token
  * that would have been sampled at step j, out_logprobs[p][g][j] the

@@ -73,6 +73,8 @@ def _load() -> C.CDLL:
     lib.echo_wait_policy.argtypes = [vp]
     lib.echo_rollout.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp]
     lib.echo_rollout_forced.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp, vp]
+    lib.echo_rollout_queue.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp, vp]
+    lib.echo_rollout_queue.restype = C.c_int
     lib.echo_rollout_host.argtypes = [vp, vp, vp, i32, i32, i32, f32, u64, vp, vp, vp]
     lib.echo_score.argtypes = [vp, vp, vp, i32, i32, i32, f32, vp, vp, vp]
     lib.echo_score.restype = C.c_int
@@ -147,7 +149,7 @@ EXPORTED = ["echo_arena_bytes", "echo_create", "echo_destroy", "echo_load_policy
             "echo_get_stats", "echo_profile_config", "echo_profile_read", "echo_debug_page_table", "echo_debug_noise", "echo_sample", "echo_gemm_bf16",
             "echo_gemm_workspace_bytes", "echo_gemm_bf16_noalloc", "echo_decode_attention",
             "echo_decode_attention_scratch_bytes", "echo_plan_page_table", "echo_strerror", "echo_last_error",
-            "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate", "echo_grpo_objective",
+            "echo_tiled_weight_bytes", "echo_retile_weights", "echo_sample_top_p", "echo_grpo_surrogate", "echo_grpo_objective", "echo_rollout_queue",
             "echo_mu_min", "echo_staleness_bound", "echo_greedy_provision", "echo_admissible",
             "echo_set_sequence_base", "echo_debug_capture", "echo_debug_wait_limit",
             "echo_gemm_bf16_noalloc_status", "echo_probe_read_bandwidth", "echo_peer_score", "echo_chain_assemble",
@@ -269,6 +271,28 @@ class Engine:
                                          float(temperature), int(seed), forced.data_ptr(),
                                          out_tokens.data_ptr(), out_logprobs.data_ptr(), versions.ctypes.data)
         _check(rc, self._ctx)
+        return out_tokens, out_logprobs, versions
+
+    def echo_rollout_queue(self, prompts: torch.Tensor, prompt_lens: Sequence[int], G: int, max_new_tokens: int,
+                           temperature: float, seed: int, forced: Optional[torch.Tensor] = None):
+        """Rollout over a queue of prompts [n][cfg.max_prompt_len] (n may exceed cfg.max_prompts): freed
+        slots are refilled from the queue.  Returns (tokens [n][G][T], logprobs [n][G][T], versions [n][G])."""
+        n = prompts.shape[0]
+        assert prompts.dtype == torch.int32 and prompts.is_cuda and prompts.is_contiguous()
+        assert prompts.shape[1] == self.cfg.max_prompt_len
+        lens = np.ascontiguousarray(np.asarray(prompt_lens, dtype=np.int32))
+        assert lens.shape == (n,)
+        T = max_new_tokens
+        out_tokens = torch.empty((n, G, T), dtype=torch.int32, device=self.device)
+        out_logprobs = torch.empty((n, G, T), dtype=torch.float32, device=self.device)
+        versions = np.zeros((n, G), dtype=np.int64)
+        if forced is not None:
+            assert forced.dtype == torch.int32 and forced.is_cuda and forced.is_contiguous()
+            assert tuple(forced.shape) == (n, G, T)
+        self.stream.wait_stream(torch.cuda.current_stream(self.device))
+        _check(lib.echo_rollout_queue(self._ctx, prompts.data_ptr(), lens.ctypes.data, n, G, T, float(temperature),
+                                      int(seed), forced.data_ptr() if forced is not None else None,
+                                      out_tokens.data_ptr(), out_logprobs.data_ptr(), versions.ctypes.data), self._ctx)
         return out_tokens, out_logprobs, versions
 
     def echo_score(self, prompts: torch.Tensor, prompt_lens: Sequence[int], tokens: torch.Tensor, temperature: float,

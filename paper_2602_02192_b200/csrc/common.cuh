@@ -210,8 +210,12 @@ cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page
 // Compaction of a decode step's rows (used with an end token): the sequences that have not ended are
 // packed to the front of the activation rows.  row_seq[r] = sequence of row r (-1: padding row),
 // seq_row[b] = row of sequence b (-1: ended), seq_pos[b] = position sequence b feeds, *n_live = rows in use.
+// With a prompt queue (groups admitted into freed slots during the rollout) a slot's sequence b also
+// has seq_gid[b] = the sequence id it currently generates (prompt index * G + g; -1: empty slot) and
+// seq_t0[b] = the step counter's value when its token 0 was sampled; both null otherwise (gid = b, t0 = 0).
 struct CompactRows {
   int32_t *row_seq, *seq_row, *seq_pos, *n_live;
+  int32_t *seq_gid = nullptr, *seq_t0 = nullptr;
 };
 // decode-step preparation: advances the step counter, sets the rows' token and position; with `cr` it
 // also packs the live sequences and writes end token / 0 for the ended ones into the outputs
@@ -219,6 +223,12 @@ cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, 
                                int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s, int eos_id = -1,
                                int32_t *row_done = nullptr, const CompactRows *cr = nullptr,
                                int32_t *out_tok = nullptr, float *out_lp = nullptr);
+// Slots that change hands: for i < n, sequence slot admit_seq[i] finishes the outputs of the sequence
+// it held (end token / 0 from its current position on, if eos_id >= 0), takes sequence id admit_gid[i]
+// (-1: stays empty) with its token 0 due at the step counter's current value, and is live again.
+cudaError_t admit_launch(int n, const int32_t *admit_seq, const int32_t *admit_gid, const int32_t *d_step,
+                         int32_t *seq_gid, int32_t *seq_t0, int32_t *row_done, int32_t *out_tok, float *out_lp, int T,
+                         int eos_id, cudaStream_t s);
 cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit_row,
                            const int32_t *seq_ids, const int32_t *d_step, uint32_t j_host,
                            float temperature, uint64_t seed, const int32_t *forced, int forced_stride,
@@ -226,7 +236,9 @@ cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit
                            const uint2 *nucleus_cut = nullptr,    // per logits row, from nucleus_cut_launch
                            const int32_t *row_done = nullptr,     // per row: non-zero = the sequence has ended
                            uint32_t seq_base = 0,                 // added to every sequence id of the noise streams
-                           const int32_t *row_seq = nullptr);     // compacted step: sequence of each logits row
+                           const int32_t *row_seq = nullptr,      // compacted step: sequence of each logits row
+                           const int32_t *seq_gid = nullptr,      // prompt queue: sequence id a slot generates and
+                           const int32_t *seq_t0 = nullptr);      // the step its token 0 was sampled at
 // Nucleus (top-p) cut of each logits row: cut[row] = (order-preserving key of the score of the last
 // nucleus member, its id; id 0x7fffffff = every id of that score).  nucleus.cu
 cudaError_t nucleus_cut_launch(const float *logits, int rows, int V, float temperature, float top_p, uint2 *cut,

@@ -333,6 +333,7 @@ struct Compaction {
   int32_t *row_seq, *seq_row, *seq_pos, *n_live;
   int32_t *out_tok;
   float *out_lp;
+  const int32_t *seq_gid, *seq_t0;      // prompt queue: sequence id and first step of what slot b holds
 };
 __global__ void __launch_bounds__(512)
 decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0, int32_t *row_tok,
@@ -361,9 +362,20 @@ decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_
     const int b = b0 + threadIdx.x;
     int32_t tok = 0;
     int live = 0;
+    // the sequence slot b generates (itself without a prompt queue) and the index t of the token this
+    // step produces for it (token t - 1 is fed); a sequence also ends once all T tokens exist
+    int gid = b, t = j;
     if (b < B) {
-      tok = tok_hist[static_cast<size_t>(b) * T + (j - 1)];
-      if (tok == eos_id) row_done[b] = 1;
+      if (c.seq_gid) {
+        gid = c.seq_gid[b];
+        t = j - c.seq_t0[b];
+      }
+      if (gid < 0 || t >= T) {
+        row_done[b] = 1;
+      } else {
+        tok = tok_hist[static_cast<size_t>(gid) * T + (t - 1)];
+        if (tok == eos_id) row_done[b] = 1;
+      }
       live = row_done[b] ? 0 : 1;
     }
     // block-wide exclusive scan of the live flags
@@ -376,7 +388,7 @@ decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_
     int total = 0;
     for (int w = 0; w < nw; ++w) total += warp_sum[w];
     if (b < B) {
-      const int pos = seq_len0[b] + j - 1;
+      const int pos = seq_len0[b] + t - 1;
       c.seq_pos[b] = pos;
       if (live) {
         const int r = before + in_warp;
@@ -386,8 +398,10 @@ decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_
         row_pos[r] = pos;
       } else {
         c.seq_row[b] = -1;
-        c.out_tok[static_cast<size_t>(b) * T + j] = eos_id;
-        c.out_lp[static_cast<size_t>(b) * T + j] = 0.f;
+        if (gid >= 0 && t < T) {
+          c.out_tok[static_cast<size_t>(gid) * T + t] = eos_id;
+          c.out_lp[static_cast<size_t>(gid) * T + t] = 0.f;
+        }
       }
     }
     __syncthreads();
@@ -407,6 +421,31 @@ decode_prep_kernel(int32_t *d_step, const int32_t *tok_hist, int T, const int32_
 }
 
 __global__ void set_int_kernel(int32_t *p, int32_t v) { *p = v; }
+
+// Slots changing hands between two decode steps (prompt queue); one block per slot sequence.
+__global__ void admit_kernel(const int32_t *admit_seq, const int32_t *admit_gid, const int32_t *d_step,
+                             int32_t *seq_gid, int32_t *seq_t0, int32_t *row_done, int32_t *out_tok, float *out_lp,
+                             int T, int eos_id) {
+  const int b = admit_seq[blockIdx.x];
+  const int j = *d_step;
+  const int old = seq_gid[b];
+  if (old >= 0 && eos_id >= 0) {
+    // the steps so far wrote the sequence's positions up to j - t0 (its own tokens, then the end token
+    // from the step that found it ended); the rest of its row follows here
+    const int t_from = max(j - seq_t0[b] + 1, 1);
+    for (int t = t_from + threadIdx.x; t < T; t += blockDim.x) {
+      out_tok[static_cast<size_t>(old) * T + t] = eos_id;
+      out_lp[static_cast<size_t>(old) * T + t] = 0.f;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int gid = admit_gid[blockIdx.x];
+    seq_gid[b] = gid;
+    seq_t0[b] = j;
+    row_done[b] = gid < 0 ? 1 : 0;
+  }
+}
 
 __device__ __forceinline__ void lse_update(float &m, float &l, float s);
 __device__ __forceinline__ void lse_merge(float &m, float &l, float m2, float l2);
@@ -614,16 +653,24 @@ __global__ void __launch_bounds__(kSamplerThreads)
 sampler_kernel(const float *logits, int V, int rows_per_logit_row, const int32_t *seq_ids, const int32_t *d_step,
                uint32_t j_host, float inv_temperature, uint32_t key0, uint32_t key1, const int32_t *forced,
                int forced_stride, int32_t *out_tok, float *out_lp, int out_stride, int eos_id,
-               const uint2 *nucleus_cut, const int32_t *row_done, uint32_t seq_base, const int32_t *row_seq) {
+               const uint2 *nucleus_cut, const int32_t *row_done, uint32_t seq_base, const int32_t *row_seq,
+               const int32_t *seq_gid, const int32_t *seq_t0) {
   __shared__ float sm_m[32], sm_l[32], sm_score[32];
   __shared__ int sm_id[32];
   early_start_sync();
   const int r = blockIdx.x;
   // compacted step: logits row r belongs to sequence row_seq[r] (its noise stream, its output slot);
   // a padding row has no sequence
-  const int seq = row_seq ? row_seq[r] : r;
+  int seq = row_seq ? row_seq[r] : r;
   if (seq < 0) return;
-  const uint32_t j = d_step ? static_cast<uint32_t>(*d_step) : j_host;
+  uint32_t j = d_step ? static_cast<uint32_t>(*d_step) : j_host;
+  if (seq_gid) {
+    // prompt queue: slot `seq` generates sequence seq_gid[seq], whose token index is counted from the
+    // step its token 0 was sampled at; noise stream and output row are the sequence's, not the slot's
+    j -= static_cast<uint32_t>(seq_t0[seq]);
+    seq = seq_gid[seq];
+    if (seq < 0) return;
+  }
   if (eos_id >= 0 && j > 0 && row_done) {
     // End-of-sequence rule: the sequence is finished once one of the tokens fed so far (the forced
     // ones when scoring a given trajectory) was eos_id, which the step's preparation kernel records
@@ -803,8 +850,8 @@ cudaError_t copy_partial_pages_launch(__nv_bfloat16 *kv, const int32_t *src_page
 cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, const int32_t *seq_len0,
                                int32_t *row_tok, int32_t *row_pos, int B, cudaStream_t s, int eos_id,
                                int32_t *row_done, const CompactRows *cr, int32_t *out_tok, float *out_lp) {
-  Compaction c{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
-  if (cr) c = Compaction{cr->row_seq, cr->seq_row, cr->seq_pos, cr->n_live, out_tok, out_lp};
+  Compaction c{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  if (cr) c = Compaction{cr->row_seq, cr->seq_row, cr->seq_pos, cr->n_live, out_tok, out_lp, cr->seq_gid, cr->seq_t0};
   return launch_early(decode_prep_kernel, dim3(1), dim3(512), 0, s, d_step, tok_hist, T, seq_len0, row_tok, row_pos, B,
                       eos_id, row_done, c);
 }
@@ -812,11 +859,19 @@ cudaError_t sampler_launch(const float *logits, int R, int V, int rows_per_logit
                            const int32_t *d_step, uint32_t j_host, float temperature, uint64_t seed,
                            const int32_t *forced, int forced_stride, int32_t *out_tok, float *out_lp, int out_stride,
                            cudaStream_t s, int eos_id, const uint2 *nucleus_cut, const int32_t *row_done,
-                           uint32_t seq_base, const int32_t *row_seq) {
+                           uint32_t seq_base, const int32_t *row_seq, const int32_t *seq_gid,
+                           const int32_t *seq_t0) {
   return launch_early(sampler_kernel, dim3(R), dim3(kSamplerThreads), 0, s, logits, V, rows_per_logit_row, seq_ids,
                       d_step, j_host, 1.0f / temperature, static_cast<uint32_t>(seed & 0xffffffffu),
                       static_cast<uint32_t>(seed >> 32), forced, forced_stride, out_tok, out_lp, out_stride, eos_id,
-                      nucleus_cut, row_done, seq_base, row_seq);
+                      nucleus_cut, row_done, seq_base, row_seq, seq_gid, seq_t0);
+}
+cudaError_t admit_launch(int n, const int32_t *admit_seq, const int32_t *admit_gid, const int32_t *d_step,
+                         int32_t *seq_gid, int32_t *seq_t0, int32_t *row_done, int32_t *out_tok, float *out_lp, int T,
+                         int eos_id, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  admit_kernel<<<n, 128, 0, s>>>(admit_seq, admit_gid, d_step, seq_gid, seq_t0, row_done, out_tok, out_lp, T, eos_id);
+  return cudaGetLastError();
 }
 cudaError_t noise_debug_launch(uint64_t seed, uint32_t s_id, uint32_t j, uint32_t v0, uint32_t n, uint32_t *words,
                                float *uniform, cudaStream_t s) {

@@ -88,7 +88,7 @@ Limits limits_of(const echo_config &c) {
 struct Layout {
   size_t weights[2], kv, rope, x, h, qkv, q, attn, act, gu, xlast, hlast, logits;
   size_t page_table, pre_row_pt, pre_row_pos, pre_tok_idx, gather_map, dec_row_tok, dec_row_pos, dec_row_pt,
-      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, row_done, copy_src, copy_dst, d_step, status, attn_work, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, row_seq, seq_row, seq_pos, n_live, gemm_bar, total;
+      seq_len0, full_pages, pre_o, pre_ml, retile_stage, nucleus_cut, row_done, copy_src, copy_dst, d_step, status, attn_work, gemm_ws, gemm_counters, stage_prompts, stage_tok, stage_lp, row_seq, seq_row, seq_pos, n_live, gemm_bar, seq_gid, seq_t0, admit_seq, admit_gid, total;
   size_t weight_bytes, kv_layer_elems, n_tables_ints;
   int n_chunks_max;
 };
@@ -150,6 +150,11 @@ Layout layout_of(const echo_config &c) {
   lo.stage_prompts = take(static_cast<size_t>(M.P) * M.Lp * 4);
   lo.stage_tok = take(static_cast<size_t>(M.B) * M.T * 4);
   lo.stage_lp = take(static_cast<size_t>(M.B) * M.T * 4);
+  // prompt queue: what each sequence slot generates, since which step; the slots changing hands
+  lo.seq_gid = take(static_cast<size_t>(M.B) * 4);
+  lo.seq_t0 = take(static_cast<size_t>(M.B) * 4);
+  lo.admit_seq = take(static_cast<size_t>(M.B) * 4);
+  lo.admit_gid = take(static_cast<size_t>(M.B) * 4);
   lo.total = off;
   return lo;
 }
@@ -201,6 +206,8 @@ struct echo_ctx {
   bool fuse_norm = false;     // RMSNorm as the prologue of the projection that consumes it (decode steps)
   bool compact = false;
   int32_t *h_live = nullptr;          // page-locked: live rows reported at the end of each window
+  int32_t *h_queue = nullptr;         // page-locked: admit lists (2 x B) and three snapshots of the ended flags (3 x B)
+  bool queue_mode = false;            // the rollout being enqueued runs over a prompt queue
   cudaEvent_t live_ev[3] = {nullptr, nullptr, nullptr};
   bool prefill_rows = false;  // ECHO_ATTN_PREFILL=rows: the one-query-per-row kernel for the prompt prefill too
   uint32_t seq_base = 0;      // added to p * G + g in the noise streams (echo_set_sequence_base)
@@ -647,9 +654,13 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
   int32_t *row_tok = ctx->ptr<int32_t>(lo.dec_row_tok);
   int32_t *row_pos = ctx->ptr<int32_t>(lo.dec_row_pos);
   ProfScope prof_step(ctx, PROF_STEP);
-  int32_t *row_done = ctx->cfg.eos_id >= 0 ? ctx->ptr<int32_t>(lo.row_done) : nullptr;
+  int32_t *row_done = (ctx->cfg.eos_id >= 0 || ctx->compact) ? ctx->ptr<int32_t>(lo.row_done) : nullptr;
   CompactRows crs{ctx->ptr<int32_t>(lo.row_seq), ctx->ptr<int32_t>(lo.seq_row), ctx->ptr<int32_t>(lo.seq_pos),
                   ctx->ptr<int32_t>(lo.n_live)};
+  if (ctx->queue_mode) {
+    crs.seq_gid = ctx->ptr<int32_t>(lo.seq_gid);
+    crs.seq_t0 = ctx->ptr<int32_t>(lo.seq_t0);
+  }
   const CompactRows *cr = ctx->compact ? &crs : nullptr;
   LAUNCH(decode_prep_launch(d_step, tok_hist, pl.T, ctx->ptr<int32_t>(lo.seq_len0), row_tok, row_pos, pl.B,
                             ctx->stream, ctx->cfg.eos_id, row_done, cr, out_tokens, out_logprobs));
@@ -672,7 +683,7 @@ int decode_step(echo_ctx *ctx, const WeightBuf &w, const Plan &pl, const int32_t
     }
     LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), rows, ctx->D.V, 1, nullptr, d_step, 0, temperature, seed,
                           forced, pl.T, out_tokens, out_logprobs, pl.T, ctx->stream, ctx->cfg.eos_id, cut,
-                          cr ? nullptr : row_done, ctx->seq_base, cr ? cr->row_seq : nullptr));
+                          cr ? nullptr : row_done, ctx->seq_base, cr ? cr->row_seq : nullptr, crs.seq_gid, crs.seq_t0));
   }
   return ECHO_OK;
 }
@@ -875,6 +886,338 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
   return ECHO_OK;
 }
 
+
+// ---- rollout over a prompt queue ---------------------------------------------------------------
+// The context's max_prompts groups are SLOTS: a slot holds one prompt and its G samples, with a fixed
+// range of KV pages large enough for any admissible prompt.  When every sample of a slot has ended
+// (end token, or all T tokens generated) the next prompt of the queue is prefilled into it between two
+// decode steps.  A sequence keeps the noise stream and the output row of its id (prompt index * G + g)
+// and counts its tokens from the step it was admitted at, so its tokens do not depend on the slot or
+// the moment it ran.  The host learns which sequences have ended from snapshots of the ended flags
+// taken every kQueueWindow steps and read two windows later (it never waits for the GPU's current step).
+constexpr int kQueueWindow = 16;
+
+struct AdmitPlan {
+  int n_new, n_tok, n_chunks, n_copies;
+};
+
+// Host plan for admitting prompts `which[i]` into slots `slots[i]` (i < n_new): the slots' page-table
+// rows in the host mirror, the prefill row lists, the copies of partial prompt pages and the admit lists.
+AdmitPlan plan_admit(echo_ctx *ctx, const int32_t *lens, int S, int G, int T, const std::vector<int> &slots,
+                     const std::vector<int> &which) {
+  const Limits &M = ctx->M;
+  const int Z = ctx->D.Z, W = M.pt_width;
+  int32_t *h_pt = ctx->h_tables;
+  int32_t *h_row_pt = h_pt + static_cast<size_t>(M.B + M.P) * W;
+  int32_t *h_row_pos = h_row_pt + static_cast<size_t>(M.P) * M.Lp;
+  int32_t *h_tok_idx = h_row_pos + static_cast<size_t>(M.P) * M.Lp;
+  int32_t *h_gather = h_tok_idx + static_cast<size_t>(M.P) * M.Lp;
+  int32_t *h_dec_pt = h_gather + static_cast<size_t>(ctx->lo.n_chunks_max) * M.P;
+  int32_t *h_len0 = h_dec_pt + M.B;
+  int32_t *h_full = h_len0 + M.B;
+  int32_t *h_csrc = h_full + M.B;
+  int32_t *h_cdst = h_csrc + M.B;
+  int32_t *h_admit_seq = ctx->h_queue, *h_admit_gid = ctx->h_queue + M.B;
+  const int n_new = static_cast<int>(slots.size());
+  const int pages_per_slot = M.n_pre + M.G * M.n_dec;
+  AdmitPlan ap{n_new, 0, 0, 0};
+  for (int i = 0; i < n_new; ++i) ap.n_tok += lens[which[i]];
+  const int chunk = ctx->chunk_rows;
+  ap.n_chunks = ceil_div(ap.n_tok, chunk);
+  std::fill(h_gather, h_gather + static_cast<size_t>(ap.n_chunks) * n_new, -1);
+  int row = 0;
+  for (int i = 0; i < n_new; ++i) {
+    const int slot = slots[i], p = which[i], len = lens[p];
+    const int full = len / Z, n_pre = ceil_div(len, Z), n_dec = ceil_div(len + T - 1, Z) - full;
+    const int pre_base = slot * pages_per_slot;
+    int32_t *pre_row = h_pt + static_cast<size_t>(S * G + slot) * W;
+    std::fill(pre_row, pre_row + W, -1);
+    for (int qi = 0; qi < n_pre; ++qi) pre_row[qi] = pre_base + qi;
+    for (int g = 0; g < G; ++g) {
+      const int b = slot * G + g;
+      const int dec_base = pre_base + M.n_pre + g * M.n_dec;
+      int32_t *r = h_pt + static_cast<size_t>(b) * W;
+      std::fill(r, r + W, -1);
+      for (int qi = 0; qi < full; ++qi) r[qi] = pre_base + qi;
+      for (int qi = 0; qi < n_dec; ++qi) r[full + qi] = dec_base + qi;
+      if (n_pre > full && n_dec > 0) {          // partial last prompt page: private copy per sample
+        h_csrc[ap.n_copies] = pre_base + full;
+        h_cdst[ap.n_copies] = dec_base;
+        ++ap.n_copies;
+      }
+      h_len0[b] = len;
+      h_full[b] = full;
+      h_admit_seq[i * G + g] = b;
+      h_admit_gid[i * G + g] = p * G + g;
+    }
+    for (int t = 0; t < len; ++t, ++row) {
+      h_row_pt[row] = S * G + slot;
+      h_row_pos[row] = t;
+      h_tok_idx[row] = p * M.Lp + t;
+    }
+    const int last = row - 1;
+    h_gather[static_cast<size_t>(last / chunk) * n_new + i] = last % chunk;
+  }
+  return ap;
+}
+
+int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int Pq, int G, int T,
+                       float temperature, uint64_t seed, const int32_t *forced, int32_t *out_tokens,
+                       float *out_logprobs, int64_t *out_versions) {
+  if (!ctx || !prompts || !prompt_lens || !out_tokens || !out_logprobs || !out_versions) return ECHO_ERR_INVALID;
+  const Limits &M = ctx->M;
+  if (Pq < 1 || G < 1 || G > M.G || T < 1 || T > M.T) return ECHO_ERR_INVALID;
+  if (static_cast<long long>(Pq) * G > (1ll << 30) / T) return ECHO_ERR_INVALID;
+  if (!(temperature > 0.f) || !std::isfinite(temperature)) return ECHO_ERR_INVALID;
+  for (int p = 0; p < Pq; ++p)
+    if (prompt_lens[p] < 1 || prompt_lens[p] > M.Lp) return ECHO_ERR_INVALID;
+  if (!ctx->fast_decode) return ECHO_ERR_UNSUPPORTED;
+  DeviceGuard guard(ctx->device);
+
+  int rc;
+  WeightBuf *wp = begin_rollout_version(ctx, &rc);
+  if (!wp) return rc;
+  const WeightBuf &w = *wp;
+  for (long long i = 0; i < static_cast<long long>(Pq) * G; ++i) out_versions[i] = w.version;
+
+  const Layout &lo = ctx->lo;
+  const Dims &D = ctx->D;
+  const int S = std::min(M.P, Pq), B = S * G, W = M.pt_width;
+  const int eos = ctx->cfg.eos_id;
+  const int64_t launches0 = ctx->launches;
+  const Plan pl{S, G, T, B, 0, 0, 0, S * (M.n_pre + M.G * M.n_dec), W};
+  struct ModeGuard {                  // the step enqueued below packs its rows whatever the context's setting
+    echo_ctx *c;
+    bool compact0;
+    ModeGuard(echo_ctx *cc) : c(cc), compact0(cc->compact) { c->compact = true; c->queue_mode = true; }
+    ~ModeGuard() { c->compact = compact0; c->queue_mode = false; }
+  } mode_guard(ctx);
+
+  int32_t *d_step = ctx->ptr<int32_t>(lo.d_step);
+  int32_t *row_done = ctx->ptr<int32_t>(lo.row_done);
+  int32_t *seq_gid = ctx->ptr<int32_t>(lo.seq_gid), *seq_t0 = ctx->ptr<int32_t>(lo.seq_t0);
+  CK(cudaEventRecord(ctx->ev_begin, ctx->stream));
+  ctx->prof_recs.clear();
+  ctx->prof_pool_used = 0;
+  CK(cudaMemsetAsync(row_done, 0xff, static_cast<size_t>(B) * 4, ctx->stream));        // every slot empty
+  CK(cudaMemsetAsync(seq_gid, 0xff, static_cast<size_t>(B) * 4, ctx->stream));
+  CK(cudaMemsetAsync(seq_t0, 0, static_cast<size_t>(B) * 4, ctx->stream));
+  CK(cudaMemsetAsync(ctx->arena + lo.attn, 0, static_cast<size_t>(B) * D.Hq * D.hd * 2, ctx->stream));
+  LAUNCH(set_int_launch(d_step, 0, ctx->stream));
+  if (ctx->plan_in_flight) {
+    CK(cudaEventSynchronize(ctx->plan_done));
+    ctx->plan_in_flight = false;
+  }
+  std::fill(ctx->h_tables, ctx->h_tables + static_cast<size_t>(M.B + M.P) * W, -1);
+  ctx->last_rows = 0;
+
+  const int32_t *tok_hist = forced ? forced : out_tokens;
+  std::vector<int> slot_admit(S, -1);      // step after which the slot's current prompt was admitted; -1: empty
+  std::vector<int> slot_live(S, 0);        // upper bound of the slot's sequences that have not ended
+  int next_prompt = 0, j = 0, n_admits = 0;
+
+  auto admit = [&](const std::vector<int> &slots) -> int {
+    std::vector<int> which;
+    for (size_t i = 0; i < slots.size(); ++i) which.push_back(next_prompt + static_cast<int>(i));
+    if (ctx->plan_in_flight) {             // the staging block may still be read by the previous upload
+      CK(cudaEventSynchronize(ctx->plan_done));
+      ctx->plan_in_flight = false;
+    }
+    const AdmitPlan ap = plan_admit(ctx, prompt_lens, S, G, T, slots, which);
+    const size_t npt = static_cast<size_t>(M.P) * M.Lp;
+    const int32_t *h = ctx->h_tables;
+    size_t o = 0;
+    auto up = [&](size_t dev_off, size_t cap_ints, size_t n_ints) -> cudaError_t {
+      cudaError_t e = cudaSuccess;
+      if (n_ints) e = cudaMemcpyAsync(ctx->arena + dev_off, h + o, n_ints * 4, cudaMemcpyHostToDevice, ctx->stream);
+      o += cap_ints;
+      return e;
+    };
+    CK(up(lo.page_table, static_cast<size_t>(M.B + M.P) * W, static_cast<size_t>(B + S) * W));
+    CK(up(lo.pre_row_pt, npt, ap.n_tok));
+    CK(up(lo.pre_row_pos, npt, ap.n_tok));
+    CK(up(lo.pre_tok_idx, npt, ap.n_tok));
+    CK(up(lo.gather_map, static_cast<size_t>(lo.n_chunks_max) * M.P, static_cast<size_t>(ap.n_chunks) * ap.n_new));
+    CK(up(lo.dec_row_pt, M.B, 0));
+    CK(up(lo.seq_len0, M.B, B));
+    CK(up(lo.full_pages, M.B, B));
+    CK(up(lo.copy_src, M.B, ap.n_copies));
+    CK(up(lo.copy_dst, M.B, ap.n_copies));
+    const int n_seq = ap.n_new * G;
+    CK(cudaMemcpyAsync(ctx->arena + lo.admit_seq, ctx->h_queue, static_cast<size_t>(n_seq) * 4, cudaMemcpyHostToDevice,
+                       ctx->stream));
+    CK(cudaMemcpyAsync(ctx->arena + lo.admit_gid, ctx->h_queue + M.B, static_cast<size_t>(n_seq) * 4,
+                       cudaMemcpyHostToDevice, ctx->stream));
+    CK(cudaEventRecord(ctx->plan_done, ctx->stream));
+    ctx->plan_in_flight = true;
+    LAUNCH(admit_launch(n_seq, ctx->ptr<int32_t>(lo.admit_seq), ctx->ptr<int32_t>(lo.admit_gid), d_step, seq_gid, seq_t0,
+                        row_done, out_tokens, out_logprobs, T, eos, ctx->stream));
+    // prefill of the admitted prompts, then token 0 of each of their samples
+    const Plan apl{ap.n_new, G, T, n_seq, ap.n_tok, ap.n_chunks, ap.n_copies, pl.n_pages, W};
+    TRY(run_prefill(ctx, w, apl, prompts));
+    TRY(lm_head(ctx, w, ctx->ptr<float>(lo.xlast), ap.n_new));
+    const uint2 *cut0 = nullptr;
+    if (ctx->cfg.top_p > 0.f && ctx->cfg.top_p < 1.f) {
+      LAUNCH(nucleus_cut_launch(ctx->ptr<float>(lo.logits), ap.n_new, D.V, temperature, ctx->cfg.top_p,
+                                ctx->ptr<uint2>(lo.nucleus_cut), ctx->stream));
+      cut0 = ctx->ptr<uint2>(lo.nucleus_cut);
+    }
+    LAUNCH(sampler_launch(ctx->ptr<float>(lo.logits), n_seq, D.V, G, nullptr, d_step, 0, temperature, seed, forced, T,
+                          out_tokens, out_logprobs, T, ctx->stream, eos, cut0, nullptr, ctx->seq_base,
+                          ctx->ptr<int32_t>(lo.admit_seq), seq_gid, seq_t0));
+    for (size_t i = 0; i < slots.size(); ++i) {
+      slot_admit[slots[i]] = j;
+      slot_live[slots[i]] = G;
+    }
+    next_prompt += static_cast<int>(slots.size());
+    ++n_admits;
+    return ECHO_OK;
+  };
+
+  {
+    std::vector<int> all(S);
+    for (int i = 0; i < S; ++i) all[i] = i;
+    TRY(admit(all));
+  }
+  CK(cudaEventRecord(ctx->ev_first, ctx->stream));
+
+  // graphs of the decode step per (suffix kernel, row count), captured when first needed
+  std::vector<int> buckets{B};
+  for (int m : {128, 64, 32})
+    if (m < B) buckets.push_back(m);
+  const int n_b = static_cast<int>(buckets.size());
+  std::vector<cudaGraph_t> graph(2 * n_b, nullptr);
+  std::vector<cudaGraphExec_t> exec(2 * n_b, nullptr);
+  std::vector<char> tried(2 * n_b, 0);
+  std::vector<int64_t> per_step(2 * n_b, 0);
+  const bool graphs_ok = ctx->use_graph && ctx->stream != nullptr;
+  auto release_graphs = [&]() {
+    for (size_t u = 0; u < exec.size(); ++u) {
+      if (exec[u]) cudaGraphExecDestroy(exec[u]);
+      if (graph[u]) cudaGraphDestroy(graph[u]);
+    }
+  };
+  auto capture = [&](int v, int bi) -> int {
+    const int u = v * n_b + bi;
+    tried[u] = 1;
+    const int64_t before = ctx->launches;
+    if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+      cudaGetLastError();
+      return ECHO_OK;
+    }
+    ctx->long_suffix = v == 1;
+    const int src = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs, buckets[bi]);
+    ctx->long_suffix = false;
+    cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph[u]);
+    per_step[u] = ctx->launches - before;
+    ctx->launches = before;
+    if (src != ECHO_OK) return src;
+    if (e != cudaSuccess || cudaGraphInstantiate(&exec[u], graph[u], 0) != cudaSuccess) {
+      cudaGetLastError();
+      exec[u] = nullptr;
+    }
+    return ECHO_OK;
+  };
+
+  int32_t *h_snap = ctx->h_queue + 2 * static_cast<size_t>(M.B);
+  int bi = 0;
+  int rc_steps = ECHO_OK;
+  // a slot's sequences have all ended, as far as the host can know: by length, or by the flags of a
+  // snapshot taken after the slot's admission
+  auto by_length = [&](int slot) { return slot_admit[slot] < 0 || j >= slot_admit[slot] + T - 1; };
+  auto over = [&](int slot) { return by_length(slot) || slot_live[slot] == 0; };
+  auto refill = [&]() -> int {                // freed slots take the next prompts of the queue
+    if (next_prompt >= Pq) return ECHO_OK;
+    std::vector<int> freed;
+    for (int sl = 0; sl < S && next_prompt + static_cast<int>(freed.size()) < Pq; ++sl)
+      if (over(sl)) freed.push_back(sl);
+    return freed.empty() ? ECHO_OK : admit(freed);
+  };
+  auto choose_rows = [&]() {                  // the smallest captured row count that holds every live sequence
+    int bound = 0;
+    for (int sl = 0; sl < S; ++sl) bound += over(sl) ? 0 : slot_live[sl];
+    bi = 0;
+    for (int k = 1; k < n_b; ++k)
+      if (buckets[k] >= bound) bi = k;
+  };
+  for (;;) {
+    if ((rc_steps = refill()) != ECHO_OK) break;
+    bool all_over = true;
+    for (int sl = 0; sl < S && all_over; ++sl) all_over = over(sl);
+    if (all_over) break;
+    choose_rows();
+    ++j;
+    int age = 0;                             // most tokens any live slot's sequences may hold
+    for (int sl = 0; sl < S; ++sl)
+      if (!over(sl)) age = std::max(age, j - slot_admit[sl]);
+    const int v = age >= kLongSuffix ? 1 : 0;
+    const int u = v * n_b + bi;
+    if (graphs_ok && !tried[u]) rc_steps = capture(v, bi);
+    if (rc_steps != ECHO_OK) break;
+    if (exec[u]) {
+      cudaError_t le = cudaGraphLaunch(exec[u], ctx->stream);
+      if (le != cudaSuccess) rc_steps = fail_cuda(ctx, le, "cudaGraphLaunch");
+      ctx->launches += per_step[u];
+    } else {
+      ctx->long_suffix = v == 1;
+      rc_steps = decode_step(ctx, w, pl, tok_hist, temperature, seed, forced, out_tokens, out_logprobs, buckets[bi]);
+      ctx->long_suffix = false;
+    }
+    if (rc_steps != ECHO_OK) break;
+    if (j % kQueueWindow || eos < 0) continue;          // without an end token sequences end by length only
+    // ---- window boundary: read the ended flags as of this step.  The host waits for the GPU here (the
+    // steps it has enqueued so far), which costs one launch latency per window; what it learns decides
+    // the refill and the row count of the next window.
+    cudaError_t ce = cudaMemcpyAsync(h_snap, row_done, static_cast<size_t>(B) * 4, cudaMemcpyDeviceToHost, ctx->stream);
+    if (ce == cudaSuccess) ce = cudaEventRecord(ctx->live_ev[0], ctx->stream);
+    if (ce == cudaSuccess) ce = cudaEventSynchronize(ctx->live_ev[0]);
+    if (ce != cudaSuccess) {
+      rc_steps = fail_cuda(ctx, ce, "ended-flags snapshot");
+      break;
+    }
+    for (int sl = 0; sl < S; ++sl) {
+      if (slot_admit[sl] < 0 || slot_admit[sl] >= j) continue;      // nothing of the slot's prompt has run yet
+      int live = 0;
+      for (int g = 0; g < G; ++g) live += h_snap[sl * G + g] ? 0 : 1;
+      slot_live[sl] = std::min(slot_live[sl], live);
+    }
+  }
+  release_graphs();
+  if (rc_steps != ECHO_OK) return rc_steps;
+  {
+    // the outputs of sequences that ended before their T-th token are completed when their slot changes
+    // hands; the last occupants' here
+    if (ctx->plan_in_flight) {
+      CK(cudaEventSynchronize(ctx->plan_done));
+      ctx->plan_in_flight = false;
+    }
+    int32_t *h_admit_seq = ctx->h_queue, *h_admit_gid = ctx->h_queue + M.B;
+    for (int b = 0; b < B; ++b) {
+      h_admit_seq[b] = b;
+      h_admit_gid[b] = -1;
+    }
+    CK(cudaMemcpyAsync(ctx->arena + lo.admit_seq, h_admit_seq, static_cast<size_t>(B) * 4, cudaMemcpyHostToDevice,
+                       ctx->stream));
+    CK(cudaMemcpyAsync(ctx->arena + lo.admit_gid, h_admit_gid, static_cast<size_t>(B) * 4, cudaMemcpyHostToDevice,
+                       ctx->stream));
+    CK(cudaEventRecord(ctx->plan_done, ctx->stream));
+    ctx->plan_in_flight = true;
+    LAUNCH(admit_launch(B, ctx->ptr<int32_t>(lo.admit_seq), ctx->ptr<int32_t>(lo.admit_gid), d_step, seq_gid, seq_t0,
+                        row_done, out_tokens, out_logprobs, T, eos, ctx->stream));
+  }
+  ctx->stats.last_step_rows = static_cast<float>(buckets[bi]);
+  CK(cudaEventRecord(ctx->ev_end, ctx->stream));
+  CK(cudaEventRecord(wp->last_use, ctx->stream));
+  wp->used = true;
+  ctx->stats.prefill_ms = ctx->stats.decode_ms = 0.f;
+  ctx->stats.version_served = w.version;
+  ctx->stats.tokens_generated = static_cast<int64_t>(Pq) * G * T;
+  ctx->stats.kernels_launched = ctx->launches - launches0;
+  ctx->stats.decode_steps = j;
+  ctx->stats.n_pages = pl.n_pages;
+  return ECHO_OK;
+}
+
 // Teacher-forced scoring of whole trajectories in prefill-shaped passes: the prompt once per group, then
 // every sequence's given tokens as rows of 2048-row chunks (sequence-major), each chunk through the
 // layers with causal attention over the paged cache, the lm_head and the log-probability kernel in
@@ -1035,6 +1378,9 @@ int echo_create(const echo_config *cfg, int device, void *arena, size_t arena_by
   if ((e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_live), 3 * sizeof(int32_t), cudaHostAllocDefault)) !=
       cudaSuccess)
     return bail(e, "cudaHostAlloc");
+  if ((e = cudaHostAlloc(reinterpret_cast<void **>(&ctx->h_queue), 5ull * M.B * sizeof(int32_t),
+                         cudaHostAllocDefault)) != cudaSuccess)
+    return bail(e, "cudaHostAlloc");
   for (int i = 0; i < 3; ++i)
     if ((e = cudaEventCreateWithFlags(&ctx->live_ev[i], cudaEventDisableTiming)) != cudaSuccess)
       return bail(e, "cudaEventCreate");
@@ -1109,6 +1455,7 @@ int echo_destroy(echo_ctx *ctx) {
   if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
   if (ctx->h_tables) cudaFreeHost(ctx->h_tables);
   if (ctx->h_live) cudaFreeHost(ctx->h_live);
+  if (ctx->h_queue) cudaFreeHost(ctx->h_queue);
   for (int i = 0; i < 3; ++i)
     if (ctx->live_ev[i]) cudaEventDestroy(ctx->live_ev[i]);
   for (cudaEvent_t e : ctx->prof_pool) cudaEventDestroy(e);
@@ -1216,6 +1563,13 @@ int echo_rollout(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
                  int64_t *out_versions) {
   return rollout_impl(ctx, prompts, prompt_lens, P, G, max_new_tokens, temperature, seed, nullptr, out_tokens,
                       out_logprobs, out_versions);
+}
+
+int echo_rollout_queue(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int32_t n_prompts, int32_t G,
+                       int32_t max_new_tokens, float temperature, uint64_t seed, const int32_t *forced_tokens,
+                       int32_t *out_tokens, float *out_logprobs, int64_t *out_versions) {
+  return rollout_queue_impl(ctx, prompts, prompt_lens, n_prompts, G, max_new_tokens, temperature, seed, forced_tokens,
+                            out_tokens, out_logprobs, out_versions);
 }
 
 int echo_rollout_forced(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_lens, int32_t P, int32_t G,

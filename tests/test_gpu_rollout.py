@@ -657,3 +657,80 @@ def test_rmsnorm_as_projection_prologue(B, tiny, monkeypatch):
         assert ex <= 0.05 * n
         eng.close()
     assert launched["0"] - launched["1"] == 2 * wl.shape.n_layers * (T - 1)
+
+
+def test_prompt_queue_refills_freed_slots(B, tiny):
+    """echo_rollout_queue: 11 prompts through a context of 6 group slots.  A slot is refilled from the queue
+    when all of its samples have ended, between two decode steps of the others.  Every sequence keeps the
+    noise stream of its id and counts its tokens from its own admission, so every token of every sequence
+    is checked against the oracle's rollout of that sequence alone, and against one echo_rollout call of a
+    context that holds all 11 prompts at once.  Free-running without an end token (slots turn over by
+    length: two waves), then teacher-forced along given tokens that end at very different lengths."""
+    wl, w_o, w_d = tiny
+    Pq, S, G, Lp, T = 11, 6, 8, 40, 56
+    prompts, lens = synth.make_ragged_prompts([40, 7, 33, 16, 40, 1, 25, 17, 32, 9, 21], wl.shape.vocab, 909, pad_to=Lp)
+    dp = torch.from_numpy(prompts).cuda()
+    dims = dims_of(wl.shape)
+    # ---- no end token ---------------------------------------------------------------------------
+    big = B.Engine(B.make_config(wl.shape, Pq, G, Lp, T))
+    big.echo_load_policy(w_d, 3)
+    tok_all, lp_all, _ = big.echo_rollout(dp, lens, G, T, 1.0, 4242)
+    big.echo_sync()
+    tok_all, lp_all = tok_all.cpu().numpy(), lp_all.cpu().numpy()
+    big.close()
+    eng = B.Engine(B.make_config(wl.shape, S, G, Lp, T))
+    eng.echo_load_policy(w_d, 3)
+    tok, lp, ver = eng.echo_rollout_queue(dp, lens, G, T, 1.0, 4242)
+    eng.echo_sync()
+    st = eng.echo_get_stats()
+    tok_h, lp_h = tok.cpu().numpy(), lp.cpu().numpy()
+    assert tok_h.shape == (Pq, G, T) and np.all(ver == 3) and st["tokens_generated"] == Pq * G * T
+    assert st["decode_steps"] == 2 * (T - 1)
+    n, ex, worst = check_sequences(dims, w_o, prompts, lens, G, 1.0, 4242, tok_h, lp_h, range(Pq * G))
+    assert n == Pq * G * T and ex <= 0.05 * n
+    assert_same_rollout(tok_h, lp_h, tok_all, lp_all)
+    # a second call on the same context (slots, flags and tables start over); fewer prompts than slots;
+    # a single new token per sequence (no decode step at all)
+    tok2, lp2, _ = eng.echo_rollout_queue(dp, lens, G, T, 1.0, 4242)
+    tok3, lp3, _ = eng.echo_rollout_queue(dp[:2].contiguous(), lens[:2], G, T, 1.0, 4242)
+    tok4, lp4, _ = eng.echo_rollout_queue(dp, lens, G, 1, 1.0, 4242)
+    eng.echo_sync()
+    assert_same_rollout(tok2.cpu().numpy(), lp2.cpu().numpy(), tok_h, lp_h)
+    assert_same_rollout(tok3.cpu().numpy(), lp3.cpu().numpy(), tok_h[:2], lp_h[:2])
+    assert_same_rollout(tok4.cpu().numpy(), lp4.cpu().numpy(), tok_h[:, :, :1], lp_h[:, :, :1])
+    eng.close()
+    # ---- given tokens with an end token at a random place --------------------------------------------
+    eos = 7
+    rng = np.random.default_rng(5)
+    given = rng.integers(8, wl.shape.vocab, size=(Pq, G, T)).astype(np.int32)
+    ends = rng.integers(0, 30, size=(Pq, G))
+    ends[4] = rng.integers(0, 6, size=G)                         # one group ends at once: its slot turns over early
+    ends[0, 0] = T + 5                                           # one sequence never ends
+    for p in range(Pq):
+        for g in range(G):
+            if ends[p, g] < T:
+                given[p, g, ends[p, g]] = eos
+    forced = torch.from_numpy(given).cuda()
+    eng = B.Engine(B.make_config(wl.shape, S, G, Lp, T, eos_id=eos))
+    eng.echo_load_policy(w_d, 3)
+    tok_f, lp_f, _ = eng.echo_rollout_queue(dp, lens, G, T, 1.0, 4242, forced=forced)
+    eng.echo_sync()
+    st = eng.echo_get_stats()
+    tok_f, lp_f = tok_f.cpu().numpy(), lp_f.cpu().numpy()
+    assert T - 1 <= st["decode_steps"] < 2 * (T - 1) - 16        # fewer steps than two waves of six groups
+    assert st["last_step_rows"] == 32                            # and the last ones on the smallest row count
+    for s in range(Pq * G):
+        p, g = divmod(s, G)
+        e = ends[p, g]
+        if e < T:
+            assert np.all(lp_f[p, g, e + 1:] == 0.0) and np.all(tok_f[p, g, e + 1:] == eos)
+        sc = decoder.score_forced(dims, w_o, prompts[p][: int(lens[p])], given[p, g], 1.0, 4242, s, eos_id=eos)
+        assert np.max(np.abs(lp_f[p, g] - sc.logprob_given)) <= LOGPROB_TOL
+        live = np.arange(T) <= min(e, T - 1)
+        diff = (tok_f[p, g] != sc.own_token) & live
+        assert np.all(sc.margin[diff] < 1e-2) and np.all(tok_f[p, g][diff] == sc.runner_up[diff])
+    # the context then serves an ordinary rollout
+    tok5, lp5, _ = eng.echo_rollout(dp[:S].contiguous(), lens[:S], G, 12, 1.0, 4242)
+    eng.echo_sync()
+    check_sequences(dims, w_o, prompts, lens, G, 1.0, 4242, tok5.cpu().numpy(), lp5.cpu().numpy(), range(S * G), eos_id=eos)
+    eng.close()
