@@ -568,7 +568,43 @@ def run_variable_length(args):
         del eng
         torch.cuda.empty_cache()
     useful = int(lengths.sum())
+    # A queue of 3 P prompts through the same P group slots: three echo_rollout calls one after the other
+    # (each waits for its longest sequence) against one echo_rollout_queue call (a slot is refilled as soon
+    # as the host has seen all of its samples ended).
+    Q = 3 * P
+    q_prompts = torch.from_numpy(synth.make_prompts(Q, Lp, shape.vocab, wl.prompt_seed + 1)).cuda()
+    q_given = rng.integers(0, eos, size=(Q, G, T)).astype(np.int32)
+    q_len = rng.integers(1, T + 1, size=(Q, G))
+    for p in range(Q):
+        for g in range(G):
+            q_given[p, g, q_len[p, g] - 1:] = eos
+    q_forced = torch.from_numpy(q_given).cuda()
+    eng = binding.Engine(binding.make_config(shape, P, G, Lp, T, 1, eos_id=eos))
+    eng.echo_load_policy(weights, 1)
+    eng.echo_wait_policy()
+    eng.echo_rollout(prompts, [Lp] * P, G, min(T, 64), wl.temperature, wl.sample_seed)          # warm-up
+    eng.echo_sync()
+    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    e0.record(eng.stream)
+    for k in range(3):
+        eng.echo_rollout(q_prompts[k * P:(k + 1) * P], [Lp] * P, G, T, wl.temperature, wl.sample_seed,
+                         forced=q_forced[k * P:(k + 1) * P])
+    e1.record(eng.stream)
+    eng.echo_sync()
+    tok_q, lp_q, _ = eng.echo_rollout_queue(q_prompts, [Lp] * Q, G, T, wl.temperature, wl.sample_seed, forced=q_forced)
+    e2.record(eng.stream)
+    eng.echo_sync()
+    q_steps = eng.echo_get_stats()["decode_steps"]
+    q_useful = int(q_len.sum())
+    waves_ms, queue_ms = e0.elapsed_time(e1), e1.elapsed_time(e2)
+    eng.close()
+    queue = {"prompts": Q, "slots": P, "useful_tokens": q_useful,
+             "three_calls": {"ms": round(waves_ms, 1), "decode_steps": 3 * (T - 1),
+                             "useful_tokens_per_s": round(q_useful / waves_ms * 1e3, 1)},
+             "one_queue_call": {"ms": round(queue_ms, 1), "decode_steps": int(q_steps),
+                                "useful_tokens_per_s": round(q_useful / queue_ms * 1e3, 1)}}
     print(json.dumps({"diagnostic": "variable-length responses, teacher-forced", "workload": wl.name, "max_new_tokens": T,
+                      "queue": queue,
                       "mean_length": round(float(lengths.mean()), 1), "useful_tokens": useful,
                       "with_rule": out["with_rule"], "without_rule": out["without_rule"],
                       "useful_tokens_per_s_with_rule": round(useful / out["with_rule"]["ms"] * 1e3, 1),

@@ -80,6 +80,17 @@ typedef struct echo_config {
                                  half exactly unless |w| < 2^-17 (then the error is at most 2^-25) or
                                  |w| > 65504 (refused by nothing: it would become inf).  Activations of these
                                  layers must stay below 65504.  0: bf16 everywhere.  In [0, n_layers]. */
+  int32_t kv_pages;           /* Pages of the KV pool.  0: enough for max_prompts groups of max_G samples at
+                                 the longest prompt and max_new_tokens (no call can run out).  Smaller
+                                 values are for echo_rollout_queue, which hands pages to a sequence when it
+                                 is admitted and takes them back when it has ended, so that max_prompts can
+                                 count more group slots than the pool could hold at full length; at least
+                                 one group at full length.  echo_rollout refuses a call whose plan does
+                                 not fit the pool (ECHO_ERR_INVALID). */
+  int32_t queue_max_live;     /* echo_rollout_queue admits a further group only while the sequences that
+                                 have not ended, plus its max_G samples, stay within this number (the
+                                 activation rows a decode step's projections run on).  0: no limit
+                                 other than slots and pages. */
 } echo_config;
 
 /* One snapshot: a pointer per tensor, bf16, row-major [out, in]; each pointer

@@ -37,7 +37,7 @@ class EchoConfig(C.Structure):
         ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("kv_page_size", C.c_int32),
         ("max_prompts", C.c_int32), ("max_G", C.c_int32), ("max_prompt_len", C.c_int32),
         ("max_new_tokens", C.c_int32), ("n_weight_buffers", C.c_int32), ("eos_id", C.c_int32),
-        ("top_p", C.c_float), ("half_layers", C.c_int32),
+        ("top_p", C.c_float), ("half_layers", C.c_int32), ("kv_pages", C.c_int32), ("queue_max_live", C.c_int32),
     ]
 
 
@@ -171,13 +171,13 @@ def _check(rc: int, ctx=None):
 
 def make_config(shape, max_prompts: int, max_G: int, max_prompt_len: int, max_new_tokens: int,
                 n_weight_buffers: int = 2, page_size: int = 16, eos_id: int = -1,
-                top_p: float = 1.0, half_layers: int = 0) -> EchoConfig:
+                top_p: float = 1.0, half_layers: int = 0, kv_pages: int = 0, queue_max_live: int = 0) -> EchoConfig:
     """shape: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab,
     rms_eps, rope_theta attributes."""
     return EchoConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                       shape.d_ff, shape.vocab, shape.rms_eps, shape.rope_theta, page_size,
                       max_prompts, max_G, max_prompt_len, max_new_tokens, n_weight_buffers, eos_id, top_p,
-                      min(int(half_layers), shape.n_layers))
+                      min(int(half_layers), shape.n_layers), int(kv_pages), int(queue_max_live))
 
 
 def echo_arena_bytes(cfg: EchoConfig) -> int:

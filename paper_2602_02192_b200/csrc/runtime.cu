@@ -61,6 +61,7 @@ bool config_ok(const echo_config *c) {
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return false;
   if (c->half_layers < 0 || c->half_layers > c->n_layers) return false;
   if (static_cast<long long>(c->max_prompts) * c->max_G > (1 << 20)) return false;
+  if (c->kv_pages < 0 || c->queue_max_live < 0) return false;
   return true;
 }
 
@@ -79,6 +80,7 @@ Limits limits_of(const echo_config &c) {
   for (int b = 0; b < Z && b <= m.Lp; ++b) nd = std::max(nd, ceil_div(b + m.T - 1, Z));
   m.n_dec = nd;
   m.n_pages = m.P * m.n_pre + m.B * m.n_dec;
+  if (c.kv_pages > 0) m.n_pages = std::max(c.kv_pages, m.n_pre + m.G * m.n_dec);
   m.pt_width = std::max(ceil_div(m.Lp + m.T - 1, Z), m.n_pre);
   m.max_pos = m.Lp + m.T;
   return m;
@@ -888,13 +890,14 @@ int rollout_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *prompt_le
 
 
 // ---- rollout over a prompt queue ---------------------------------------------------------------
-// The context's max_prompts groups are SLOTS: a slot holds one prompt and its G samples, with a fixed
-// range of KV pages large enough for any admissible prompt.  When every sample of a slot has ended
-// (end token, or all T tokens generated) the next prompt of the queue is prefilled into it between two
-// decode steps.  A sequence keeps the noise stream and the output row of its id (prompt index * G + g)
-// and counts its tokens from the step it was admitted at, so its tokens do not depend on the slot or
-// the moment it ran.  The host learns which sequences have ended from snapshots of the ended flags
-// taken every kQueueWindow steps and read two windows later (it never waits for the GPU's current step).
+// The context's max_prompts groups are SLOTS: a slot holds one prompt and its G samples.  KV pages come
+// from a pool the host keeps: a group takes the pages of its prompt and of every sample's longest
+// possible continuation when it is admitted, a sample's pages go back when the host has seen it ended,
+// the prompt's when all samples have.  A group is admitted between two decode steps when a slot is free,
+// the pool holds its pages and the live sequences stay within the configured number.  A sequence keeps
+// the noise stream and the output row of its id (prompt index * G + g) and counts its tokens from the
+// step it was admitted at, so its tokens do not depend on the slot or the moment it ran.  The host
+// learns which sequences have ended from the ended flags, read every kQueueWindow steps.
 constexpr int kQueueWindow = 16;
 
 struct AdmitPlan {
@@ -903,8 +906,13 @@ struct AdmitPlan {
 
 // Host plan for admitting prompts `which[i]` into slots `slots[i]` (i < n_new): the slots' page-table
 // rows in the host mirror, the prefill row lists, the copies of partial prompt pages and the admit lists.
+struct SlotPages {
+  std::vector<int> prefix;                   // pages of the prompt (the last one may be partly filled)
+  std::vector<std::vector<int>> sample;      // per sample: its own pages, in order
+};
+
 AdmitPlan plan_admit(echo_ctx *ctx, const int32_t *lens, int S, int G, int T, const std::vector<int> &slots,
-                     const std::vector<int> &which) {
+                     const std::vector<int> &which, const std::vector<SlotPages> &pages) {
   const Limits &M = ctx->M;
   const int Z = ctx->D.Z, W = M.pt_width;
   int32_t *h_pt = ctx->h_tables;
@@ -919,7 +927,6 @@ AdmitPlan plan_admit(echo_ctx *ctx, const int32_t *lens, int S, int G, int T, co
   int32_t *h_cdst = h_csrc + M.B;
   int32_t *h_admit_seq = ctx->h_queue, *h_admit_gid = ctx->h_queue + M.B;
   const int n_new = static_cast<int>(slots.size());
-  const int pages_per_slot = M.n_pre + M.G * M.n_dec;
   AdmitPlan ap{n_new, 0, 0, 0};
   for (int i = 0; i < n_new; ++i) ap.n_tok += lens[which[i]];
   const int chunk = ctx->chunk_rows;
@@ -929,20 +936,19 @@ AdmitPlan plan_admit(echo_ctx *ctx, const int32_t *lens, int S, int G, int T, co
   for (int i = 0; i < n_new; ++i) {
     const int slot = slots[i], p = which[i], len = lens[p];
     const int full = len / Z, n_pre = ceil_div(len, Z), n_dec = ceil_div(len + T - 1, Z) - full;
-    const int pre_base = slot * pages_per_slot;
+    const SlotPages &sp = pages[slot];
     int32_t *pre_row = h_pt + static_cast<size_t>(S * G + slot) * W;
     std::fill(pre_row, pre_row + W, -1);
-    for (int qi = 0; qi < n_pre; ++qi) pre_row[qi] = pre_base + qi;
+    for (int qi = 0; qi < n_pre; ++qi) pre_row[qi] = sp.prefix[qi];
     for (int g = 0; g < G; ++g) {
       const int b = slot * G + g;
-      const int dec_base = pre_base + M.n_pre + g * M.n_dec;
       int32_t *r = h_pt + static_cast<size_t>(b) * W;
       std::fill(r, r + W, -1);
-      for (int qi = 0; qi < full; ++qi) r[qi] = pre_base + qi;
-      for (int qi = 0; qi < n_dec; ++qi) r[full + qi] = dec_base + qi;
+      for (int qi = 0; qi < full; ++qi) r[qi] = sp.prefix[qi];
+      for (int qi = 0; qi < n_dec; ++qi) r[full + qi] = sp.sample[g][qi];
       if (n_pre > full && n_dec > 0) {          // partial last prompt page: private copy per sample
-        h_csrc[ap.n_copies] = pre_base + full;
-        h_cdst[ap.n_copies] = dec_base;
+        h_csrc[ap.n_copies] = sp.prefix[full];
+        h_cdst[ap.n_copies] = sp.sample[g][0];
         ++ap.n_copies;
       }
       h_len0[b] = len;
@@ -985,7 +991,7 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
   const int S = std::min(M.P, Pq), B = S * G, W = M.pt_width;
   const int eos = ctx->cfg.eos_id;
   const int64_t launches0 = ctx->launches;
-  const Plan pl{S, G, T, B, 0, 0, 0, S * (M.n_pre + M.G * M.n_dec), W};
+  Plan pl{S, G, T, B, 0, 0, 0, 0, W};
   struct ModeGuard {                  // the step enqueued below packs its rows whatever the context's setting
     echo_ctx *c;
     bool compact0;
@@ -1015,15 +1021,50 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
   std::vector<int> slot_admit(S, -1);      // step after which the slot's current prompt was admitted; -1: empty
   std::vector<int> slot_live(S, 0);        // upper bound of the slot's sequences that have not ended
   int next_prompt = 0, j = 0, n_admits = 0;
+  // the page pool (host side): free pages as a stack, the pages each slot holds, the peak in use
+  const int Z = D.Z;
+  std::vector<int> free_pages(M.n_pages);
+  for (int i = 0; i < M.n_pages; ++i) free_pages[i] = M.n_pages - 1 - i;
+  std::vector<SlotPages> slot_pages(S);
+  int pages_peak = 0;
+  auto pages_of = [&](int len) { return ceil_div(len, Z) + G * (ceil_div(len + T - 1, Z) - len / Z); };
+  auto take_pages = [&](int n, std::vector<int> &dst) {
+    dst.assign(free_pages.end() - n, free_pages.end());
+    std::reverse(dst.begin(), dst.end());
+    free_pages.resize(free_pages.size() - n);
+  };
+  auto give_pages = [&](std::vector<int> &src) {
+    free_pages.insert(free_pages.end(), src.rbegin(), src.rend());
+    src.clear();
+  };
+  // a sample of a slot has ended (the host has seen its flag, or its length is reached): its pages
+  // return to the pool; with the last sample the prompt's pages and the slot itself
+  auto release_sample = [&](int slot, int g) {
+    if (!slot_pages[slot].sample[g].empty()) give_pages(slot_pages[slot].sample[g]);
+  };
+  auto release_slot = [&](int slot) {
+    for (int g = 0; g < G; ++g) release_sample(slot, g);
+    give_pages(slot_pages[slot].prefix);
+    slot_admit[slot] = -1;
+    slot_live[slot] = 0;
+  };
 
   auto admit = [&](const std::vector<int> &slots) -> int {
     std::vector<int> which;
-    for (size_t i = 0; i < slots.size(); ++i) which.push_back(next_prompt + static_cast<int>(i));
+    for (size_t i = 0; i < slots.size(); ++i) {
+      const int p = next_prompt + static_cast<int>(i), len = prompt_lens[p];
+      which.push_back(p);
+      SlotPages &sp = slot_pages[slots[i]];
+      take_pages(ceil_div(len, Z), sp.prefix);
+      sp.sample.assign(G, std::vector<int>());
+      for (int g = 0; g < G; ++g) take_pages(ceil_div(len + T - 1, Z) - len / Z, sp.sample[g]);
+    }
+    pages_peak = std::max(pages_peak, M.n_pages - static_cast<int>(free_pages.size()));
     if (ctx->plan_in_flight) {             // the staging block may still be read by the previous upload
       CK(cudaEventSynchronize(ctx->plan_done));
       ctx->plan_in_flight = false;
     }
-    const AdmitPlan ap = plan_admit(ctx, prompt_lens, S, G, T, slots, which);
+    const AdmitPlan ap = plan_admit(ctx, prompt_lens, S, G, T, slots, which, slot_pages);
     const size_t npt = static_cast<size_t>(M.P) * M.Lp;
     const int32_t *h = ctx->h_tables;
     size_t o = 0;
@@ -1053,7 +1094,7 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
     LAUNCH(admit_launch(n_seq, ctx->ptr<int32_t>(lo.admit_seq), ctx->ptr<int32_t>(lo.admit_gid), d_step, seq_gid, seq_t0,
                         row_done, out_tokens, out_logprobs, T, eos, ctx->stream));
     // prefill of the admitted prompts, then token 0 of each of their samples
-    const Plan apl{ap.n_new, G, T, n_seq, ap.n_tok, ap.n_chunks, ap.n_copies, pl.n_pages, W};
+    const Plan apl{ap.n_new, G, T, n_seq, ap.n_tok, ap.n_chunks, ap.n_copies, M.n_pages, W};
     TRY(run_prefill(ctx, w, apl, prompts));
     TRY(lm_head(ctx, w, ctx->ptr<float>(lo.xlast), ap.n_new));
     const uint2 *cut0 = nullptr;
@@ -1074,16 +1115,11 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
     return ECHO_OK;
   };
 
-  {
-    std::vector<int> all(S);
-    for (int i = 0; i < S; ++i) all[i] = i;
-    TRY(admit(all));
-  }
-  CK(cudaEventRecord(ctx->ev_first, ctx->stream));
-
-  // graphs of the decode step per (suffix kernel, row count), captured when first needed
+  // graphs of the decode step per (suffix kernel, row count), captured when first needed; row counts:
+  // all slots, the multiples of 128 below, 64 and 32
   std::vector<int> buckets{B};
-  for (int m : {128, 64, 32})
+  for (int m = (B - 1) / 128 * 128; m >= 128; m -= 128) buckets.push_back(m);
+  for (int m : {64, 32})
     if (m < B) buckets.push_back(m);
   const int n_b = static_cast<int>(buckets.size());
   std::vector<cudaGraph_t> graph(2 * n_b, nullptr);
@@ -1124,32 +1160,52 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
   int rc_steps = ECHO_OK;
   // a slot's sequences have all ended, as far as the host can know: by length, or by the flags of a
   // snapshot taken after the slot's admission
-  auto by_length = [&](int slot) { return slot_admit[slot] < 0 || j >= slot_admit[slot] + T - 1; };
-  auto over = [&](int slot) { return by_length(slot) || slot_live[slot] == 0; };
-  auto refill = [&]() -> int {                // freed slots take the next prompts of the queue
-    if (next_prompt >= Pq) return ECHO_OK;
-    std::vector<int> freed;
-    for (int sl = 0; sl < S && next_prompt + static_cast<int>(freed.size()) < Pq; ++sl)
-      if (over(sl)) freed.push_back(sl);
-    return freed.empty() ? ECHO_OK : admit(freed);
+  auto by_length = [&](int slot) { return slot_admit[slot] >= 0 && j >= slot_admit[slot] + T - 1; };
+  auto live_bound = [&]() {
+    int n = 0;
+    for (int sl = 0; sl < S; ++sl) n += slot_admit[sl] < 0 ? 0 : slot_live[sl];
+    return n;
+  };
+  const int max_live = ctx->cfg.queue_max_live > 0 ? std::max(ctx->cfg.queue_max_live, G) : B;
+  // Groups of the queue, in order, into free slots while pages and live rows allow.  A group that fits
+  // an empty pool always exists (the pool holds at least one group at full length), so the queue drains.
+  auto refill = [&]() -> int {
+    for (int sl = 0; sl < S; ++sl)
+      if (by_length(sl)) release_slot(sl);    // every sample has all its T tokens
+    std::vector<int> slots;
+    int need = 0, rows = live_bound();
+    for (int sl = 0; sl < S && next_prompt + static_cast<int>(slots.size()) < Pq; ++sl) {
+      if (slot_admit[sl] >= 0) continue;
+      const int p = next_prompt + static_cast<int>(slots.size());
+      const int pg = pages_of(prompt_lens[p]);
+      if (need + pg > static_cast<int>(free_pages.size()) || rows + G > max_live) break;
+      need += pg;
+      rows += G;
+      slots.push_back(sl);
+    }
+    return slots.empty() ? ECHO_OK : admit(slots);
   };
   auto choose_rows = [&]() {                  // the smallest captured row count that holds every live sequence
-    int bound = 0;
-    for (int sl = 0; sl < S; ++sl) bound += over(sl) ? 0 : slot_live[sl];
+    const int bound = live_bound();
     bi = 0;
     for (int k = 1; k < n_b; ++k)
       if (buckets[k] >= bound) bi = k;
   };
+  bool first = true;
   for (;;) {
     if ((rc_steps = refill()) != ECHO_OK) break;
-    bool all_over = true;
-    for (int sl = 0; sl < S && all_over; ++sl) all_over = over(sl);
+    if (first) {
+      first = false;
+      cudaEventRecord(ctx->ev_first, ctx->stream);
+    }
+    bool all_over = next_prompt >= Pq;
+    for (int sl = 0; sl < S && all_over; ++sl) all_over = slot_admit[sl] < 0;
     if (all_over) break;
     choose_rows();
     ++j;
     int age = 0;                             // most tokens any live slot's sequences may hold
     for (int sl = 0; sl < S; ++sl)
-      if (!over(sl)) age = std::max(age, j - slot_admit[sl]);
+      if (slot_admit[sl] >= 0) age = std::max(age, j - slot_admit[sl]);
     const int v = age >= kLongSuffix ? 1 : 0;
     const int u = v * n_b + bi;
     if (graphs_ok && !tried[u]) rc_steps = capture(v, bi);
@@ -1178,8 +1234,12 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
     for (int sl = 0; sl < S; ++sl) {
       if (slot_admit[sl] < 0 || slot_admit[sl] >= j) continue;      // nothing of the slot's prompt has run yet
       int live = 0;
-      for (int g = 0; g < G; ++g) live += h_snap[sl * G + g] ? 0 : 1;
+      for (int g = 0; g < G; ++g) {
+        if (h_snap[sl * G + g]) release_sample(sl, g);
+        else ++live;
+      }
       slot_live[sl] = std::min(slot_live[sl], live);
+      if (slot_live[sl] == 0) release_slot(sl);
     }
   }
   release_graphs();
@@ -1214,7 +1274,7 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
   ctx->stats.tokens_generated = static_cast<int64_t>(Pq) * G * T;
   ctx->stats.kernels_launched = ctx->launches - launches0;
   ctx->stats.decode_steps = j;
-  ctx->stats.n_pages = pl.n_pages;
+  ctx->stats.n_pages = pages_peak;
   return ECHO_OK;
 }
 

@@ -734,3 +734,57 @@ def test_prompt_queue_refills_freed_slots(B, tiny):
     eng.echo_sync()
     check_sequences(dims, w_o, prompts, lens, G, 1.0, 4242, tok5.cpu().numpy(), lp5.cpu().numpy(), range(S * G), eos_id=eos)
     eng.close()
+
+
+def test_prompt_queue_with_a_small_page_pool(B, tiny):
+    """More group slots than the KV pool could hold at full length: the queue hands a sequence its pages at
+    admission and takes them back when the host has seen it ended, and admits by free pages and by the
+    number of live sequences.  Same per-sequence check as above; the pool's peak stays within its size."""
+    wl, w_o, w_d = tiny
+    Pq, G, Lp, T = 14, 8, 40, 56
+    lens_l = [40, 7, 33, 16, 40, 1, 25, 17, 32, 9, 21, 40, 3, 28]
+    prompts, lens = synth.make_ragged_prompts(lens_l, wl.shape.vocab, 910, pad_to=Lp)
+    dp = torch.from_numpy(prompts).cuda()
+    dims = dims_of(wl.shape)
+    eos = 7
+    rng = np.random.default_rng(6)
+    given = rng.integers(8, wl.shape.vocab, size=(Pq, G, T)).astype(np.int32)
+    ends = rng.integers(0, 40, size=(Pq, G))
+    ends[1, 0] = T + 5
+    for p in range(Pq):
+        for g in range(G):
+            if ends[p, g] < T:
+                given[p, g, ends[p, g]] = eos
+    forced = torch.from_numpy(given).cuda()
+    Z = 16
+    per_group = -(-Lp // Z) + G * (-(-(Lp % Z + T - 1) // Z))   # pages of one group at the longest prompt
+    pool = 3 * per_group + 5                                      # three groups at full length and a little more
+    eng = B.Engine(B.make_config(wl.shape, Pq, G, Lp, T, eos_id=eos, kv_pages=pool, queue_max_live=40))
+    eng.echo_load_policy(w_d, 3)
+    tok_f, lp_f, _ = eng.echo_rollout_queue(dp, lens, G, T, 1.0, 77, forced=forced)
+    eng.echo_sync()
+    st = eng.echo_get_stats()
+    tok_f, lp_f = tok_f.cpu().numpy(), lp_f.cpu().numpy()
+    assert 0 < st["n_pages"] <= pool
+    for s in range(Pq * G):
+        p, g = divmod(s, G)
+        e = ends[p, g]
+        if e < T:
+            assert np.all(lp_f[p, g, e + 1:] == 0.0) and np.all(tok_f[p, g, e + 1:] == eos)
+        sc = decoder.score_forced(dims, w_o, prompts[p][: int(lens[p])], given[p, g], 1.0, 77, s, eos_id=eos)
+        assert np.max(np.abs(lp_f[p, g] - sc.logprob_given)) <= LOGPROB_TOL
+        live = np.arange(T) <= min(e, T - 1)
+        diff = (tok_f[p, g] != sc.own_token) & live
+        assert np.all(sc.margin[diff] < 1e-2) and np.all(tok_f[p, g][diff] == sc.runner_up[diff])
+    # free-running on the same context: sequences end only by length, groups pass through the pool three at a time
+    tok, lp, _ = eng.echo_rollout_queue(dp, lens, G, 20, 1.0, 78)
+    eng.echo_sync()
+    check_sequences(dims, w_o, prompts, lens, G, 1.0, 78, tok.cpu().numpy(), lp.cpu().numpy(), range(0, Pq * G, 3),
+                    eos_id=eos)
+    # a plain rollout of all 14 groups does not fit this pool and is refused; four groups do
+    with pytest.raises(B.EchoError):
+        eng.echo_rollout(dp, lens, G, T, 1.0, 78)
+    tok5, lp5, _ = eng.echo_rollout(dp[:3].contiguous(), lens[:3], G, 12, 1.0, 78)
+    eng.echo_sync()
+    check_sequences(dims, w_o, prompts, lens, G, 1.0, 78, tok5.cpu().numpy(), lp5.cpu().numpy(), range(3 * G), eos_id=eos)
+    eng.close()
