@@ -571,7 +571,7 @@ def run_variable_length(args):
     # A queue of 3 P prompts through the same P group slots: three echo_rollout calls one after the other
     # (each waits for its longest sequence) against one echo_rollout_queue call (a slot is refilled as soon
     # as the host has seen all of its samples ended).
-    Q = 3 * P
+    Q = max(2, args.queue_factor) * P
     q_prompts = torch.from_numpy(synth.make_prompts(Q, Lp, shape.vocab, wl.prompt_seed + 1)).cuda()
     q_given = rng.integers(0, eos, size=(Q, G, T)).astype(np.int32)
     q_len = rng.integers(1, T + 1, size=(Q, G))
@@ -586,7 +586,7 @@ def run_variable_length(args):
     eng.echo_sync()
     e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
     e0.record(eng.stream)
-    for k in range(3):
+    for k in range(Q // P):
         eng.echo_rollout(q_prompts[k * P:(k + 1) * P], [Lp] * P, G, T, wl.temperature, wl.sample_seed,
                          forced=q_forced[k * P:(k + 1) * P])
     e1.record(eng.stream)
@@ -597,12 +597,44 @@ def run_variable_length(args):
     q_steps = eng.echo_get_stats()["decode_steps"]
     q_useful = int(q_len.sum())
     waves_ms, queue_ms = e0.elapsed_time(e1), e1.elapsed_time(e2)
+    base_pages = eng.echo_get_stats()["n_pages"]
+    eng.close()
+    del eng
+    torch.cuda.empty_cache()
+    # The same queue with 3 P group slots over the SAME page pool (what P groups need at full length) and
+    # at most P*G live sequences: a sample's pages return to the pool when it has ended, so the rows that
+    # ended sequences leave are taken by further groups instead of waiting for the slowest sample.
+    Z = 16
+    pool = P * (-(-Lp // Z)) + P * G * max(-(-(b + T - 1) // Z) for b in range(min(Z, Lp + 1)))
+    eng = binding.Engine(binding.make_config(shape, min(Q, 3 * P), G, Lp, T, 1, eos_id=eos, kv_pages=pool,
+                                             queue_max_live=P * G))
+    eng.echo_load_policy(weights, 1)
+    eng.echo_wait_policy()
+    eng.echo_rollout_queue(q_prompts[:P], [Lp] * P, G, min(T, 64), wl.temperature, wl.sample_seed)    # warm-up
+    eng.echo_sync()
+    e3, e4 = (torch.cuda.Event(enable_timing=True) for _ in range(2))
+    e3.record(eng.stream)
+    tok_o, lp_o, _ = eng.echo_rollout_queue(q_prompts, [Lp] * Q, G, T, wl.temperature, wl.sample_seed, forced=q_forced)
+    e4.record(eng.stream)
+    eng.echo_sync()
+    o_stats = eng.echo_get_stats()
+    over_ms = e3.elapsed_time(e4)
+    same = float((tok_o == tok_q).float().mean())
+    gap = (lp_o - lp_q).abs().flatten()
+    lp_gap = float(gap.mean())
+    lp_gap_q = float(torch.quantile(gap[:: max(1, gap.numel() // 1000000)].float(), 0.999))
     eng.close()
     queue = {"prompts": Q, "slots": P, "useful_tokens": q_useful,
-             "three_calls": {"ms": round(waves_ms, 1), "decode_steps": 3 * (T - 1),
+             "calls_of_P_prompts": {"ms": round(waves_ms, 1), "decode_steps": (Q // P) * (T - 1),
                              "useful_tokens_per_s": round(q_useful / waves_ms * 1e3, 1)},
-             "one_queue_call": {"ms": round(queue_ms, 1), "decode_steps": int(q_steps),
-                                "useful_tokens_per_s": round(q_useful / queue_ms * 1e3, 1)}}
+             "one_queue_call": {"ms": round(queue_ms, 1), "decode_steps": int(q_steps), "kv_pages": int(base_pages),
+                                "useful_tokens_per_s": round(q_useful / queue_ms * 1e3, 1)},
+             "one_queue_call_3x_slots_same_pool": {
+                 "ms": round(over_ms, 1), "decode_steps": int(o_stats["decode_steps"]), "slots": min(Q, 3 * P), "kv_pages": int(pool),
+                 "kv_pages_peak": int(o_stats["n_pages"]), "max_live_sequences": P * G,
+                 "useful_tokens_per_s": round(q_useful / over_ms * 1e3, 1),
+                 "tokens_equal_to_the_P_slot_queue": round(same, 4), "mean_logprob_gap": round(lp_gap, 5),
+                 "q999_logprob_gap": round(lp_gap_q, 4)}}
     print(json.dumps({"diagnostic": "variable-length responses, teacher-forced", "workload": wl.name, "max_new_tokens": T,
                       "queue": queue,
                       "mean_length": round(float(lengths.mean()), 1), "useful_tokens": useful,
@@ -686,6 +718,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--half-layers", type=int, default=-1,
                     help="leading layers with IEEE-half operands; default: the workload's setting")
+    ap.add_argument("--queue-factor", type=int, default=3,
+                    help="--variable-length: prompts in the queue, as a multiple of the workload's prompt count")
     ap.add_argument("--variable-length", action="store_true",
                     help="diagnostic: random response lengths with and without the end-of-sequence rule, and exit")
     ap.add_argument("--projections", action="store_true",
