@@ -781,10 +781,22 @@ def test_prompt_queue_with_a_small_page_pool(B, tiny):
     eng.echo_sync()
     check_sequences(dims, w_o, prompts, lens, G, 1.0, 78, tok.cpu().numpy(), lp.cpu().numpy(), range(0, Pq * G, 3),
                     eos_id=eos)
-    # a plain rollout of all 14 groups does not fit this pool and is refused; four groups do
+    eng.close()
+    # the same with nucleus sampling and half operands in the first layer (the admission path samples token 0
+    # of every admitted group through the same cut kernel as a decode step)
+    eng = B.Engine(B.make_config(wl.shape, Pq, G, Lp, T, eos_id=eos, kv_pages=pool, queue_max_live=40, top_p=0.9,
+                                 half_layers=1))
+    eng.echo_load_policy(w_d, 3)
+    tok, lp, _ = eng.echo_rollout_queue(dp, lens, G, 20, 1.0, 79)
+    eng.echo_sync()
+    n, ex, _ = check_sequences(dims, w_o, prompts, lens, G, 1.0, 79, tok.cpu().numpy(), lp.cpu().numpy(),
+                               range(0, Pq * G, 3), eos_id=eos, top_p=0.9)
+    assert ex <= 0.05 * n
+    # a plain rollout of all 14 groups does not fit this pool and is refused; three groups do
     with pytest.raises(B.EchoError):
         eng.echo_rollout(dp, lens, G, T, 1.0, 78)
     tok5, lp5, _ = eng.echo_rollout(dp[:3].contiguous(), lens[:3], G, 12, 1.0, 78)
     eng.echo_sync()
-    check_sequences(dims, w_o, prompts, lens, G, 1.0, 78, tok5.cpu().numpy(), lp5.cpu().numpy(), range(3 * G), eos_id=eos)
+    check_sequences(dims, w_o, prompts, lens, G, 1.0, 78, tok5.cpu().numpy(), lp5.cpu().numpy(), range(3 * G), eos_id=eos,
+                    top_p=0.9)
     eng.close()
