@@ -294,12 +294,6 @@ def test_group_advantage_matches_oracle(B):
         got = B.echo_group_advantage(torch.from_numpy(r).cuda()).cpu().numpy()
         want = o_adv.group_advantage(r)
         assert np.allclose(got, want, rtol=2e-5, atol=2e-5)
-        # with the KL regulariser against a reference policy
-        lr = (ln + rng.normal(0, 0.3, size=(n, T))).astype(np.float32)
-        got = B.echo_grpo_objective(*(torch.from_numpy(x).cuda() for x in (ln, lo, ls, lr, adv)),
-                                    torch.from_numpy(mask).cuda() if with_mask else None, 0.2, 1.7, 0.04).cpu().numpy()
-        want = objective.grpo_objective(ln, lo, ls, lr, adv, mask if with_mask else np.ones((n, T)), 0.2, 1.7, 0.04)
-        assert np.allclose(got, want, rtol=2e-5, atol=2e-5)
     r = np.full((3, 5), 0.25, dtype=np.float32)
     assert np.all(B.echo_group_advantage(torch.from_numpy(r).cuda()).cpu().numpy() == 0)
     with pytest.raises(B.EchoError):
@@ -318,4 +312,10 @@ def test_grpo_surrogate_matches_oracle(B):
         got = B.echo_grpo_surrogate(*(torch.from_numpy(x).cuda() for x in (ln, lo, ls, adv)),
                                     torch.from_numpy(mask).cuda() if with_mask else None, 0.2, 1.7).cpu().numpy()
         want = objective.grpo_surrogate(ln, lo, ls, adv, mask if with_mask else np.ones((n, T)), 0.2, 1.7)
+        assert np.allclose(got, want, rtol=2e-5, atol=2e-5)
+        # with the KL regulariser against a reference policy
+        lr = (ln + rng.normal(0, 0.3, size=(n, T))).astype(np.float32)
+        got = B.echo_grpo_objective(*(torch.from_numpy(x).cuda() for x in (ln, lo, ls, lr, adv)),
+                                    torch.from_numpy(mask).cuda() if with_mask else None, 0.2, 1.7, 0.04).cpu().numpy()
+        want = objective.grpo_objective(ln, lo, ls, lr, adv, mask if with_mask else np.ones((n, T)), 0.2, 1.7, 0.04)
         assert np.allclose(got, want, rtol=2e-5, atol=2e-5)
