@@ -141,9 +141,11 @@ def test_error_against_depth(B, w8b):
               f"half_layers={hl} mean {curve[L][2]:.3e} max {curve[L][3]:.3e}")
     depths = sorted(curve)
     for a, b in zip(depths, depths[1:]):
-        # doubling the depth never multiplies the mean error by more than ~2.5 and never lets it fall
-        # by much: a curve, not a step
+        # from one depth to the next (x 2, once x 2.25) the mean error grows at most a little faster than
+        # the depth and never falls by much: a curve, not a step.  Measured ratios: 1.1-2.7 with bf16
+        # everywhere (the largest from 4 to 9 layers, 2.55-2.64 in different runs: the order of the split
+        # projections' sums varies), 1.1-1.8 with half layers.
         for col in (0, 2):
             r = curve[b][col] / curve[a][col]
-            assert 0.6 < r < 2.6, (a, b, col, r)
+            assert 0.6 < r < 1.4 * b / a, (a, b, col, r)
     assert curve[36][2] < 0.5 * curve[36][0]                  # what the half layers buy at full depth
