@@ -371,6 +371,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16
     const int ph = blockIdx.x / MT;
     h = ph % Hkv;
     seq0 = (ph / Hkv) * G;                   // first sequence of the group
+    if (row_done) {                          // a group whose sequences have all ended is not attended
+      bool any_live = false;
+      for (int g = 0; g < G; ++g) any_live |= __ldcg(&row_done[seq0 + g]) == 0;
+      if (!any_live) return;
+    }
     first_page = 0;
     n_keys = __ldcg(&full_pages[seq0]) * kPageTokens;
   } else {
@@ -888,7 +893,8 @@ __global__ void __launch_bounds__(kDecWarps * 32)
 attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bfloat16 *__restrict__ q,
                          float *__restrict__ pre_o, float2 *__restrict__ pre_ml,
                          const int32_t *__restrict__ page_table, int pt_width, const int32_t *__restrict__ full_pages,
-                         int layer_row0, int Hq, int Hkv, int G, int n_pages, float scale_log2, int *status) {
+                         int layer_row0, int Hq, int Hkv, int G, int n_pages, float scale_log2, int *status,
+                         const int32_t *__restrict__ row_done) {
   using S = PreSmem<HD, MT>;
   constexpr int KSTEPS = HD / 16;
   constexpr int HALVES = HD / 64;
@@ -913,6 +919,13 @@ attn_prefix_group_kernel(const __grid_constant__ CUtensorMap tmKV, const __nv_bf
 
   const int h = (blockIdx.x / n_blocks) % Hkv;
   const int seq0 = (blockIdx.x / n_blocks / Hkv) * G;   // first sequence of the group
+  if (row_done) {
+    // a group whose sequences have all ended (or a slot that holds no group) is not attended: nobody
+    // reads its partial results, and its page-table rows may be stale
+    bool any_live = false;
+    for (int g = 0; g < G; ++g) any_live |= __ldcg(&row_done[seq0 + g]) == 0;
+    if (!any_live) return;
+  }
   const int n_keys = __ldcg(&full_pages[seq0]) * kPageTokens;
   const int n_tiles = n_keys / kPageTokens;
   const int32_t *pt = page_table + static_cast<size_t>(seq0) * pt_width;
@@ -1452,7 +1465,7 @@ cudaError_t launch_decode(const DecodeAttnArgs &a, cudaStream_t s) {
     e = launch_early(attn_prefix_group_kernel<HD, 2, HALF>, dim3(a.P * a.Hkv * ((MT + 1) / 2)), dim3(kDecWarps * 32),
                      PreSmem<HD, 2>::kTotal, s,
                      *a.tmKV, a.q, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.full_pages, a.layer_row0, a.Hq,
-                     a.Hkv, a.G, a.n_pages, scale_log2, a.status);
+                     a.Hkv, a.G, a.n_pages, scale_log2, a.status, a.row_done);
   } else {
     e = launch_early(attn_decode_kernel<HD, true, HALF>, dim3(a.P * a.Hkv * MT), dim3(kDecWarps * 32), S::kTotal, s,
                      *a.tmKV, a.q, a.out, a.pre_o, a.pre_ml, a.page_table, a.pt_width, a.row_pos, a.full_pages,

@@ -1015,6 +1015,12 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
     ctx->plan_in_flight = false;
   }
   std::fill(ctx->h_tables, ctx->h_tables + static_cast<size_t>(M.B + M.P) * W, -1);
+  {
+    // slots that hold nothing yet: no prompt pages, length 0 (the prefix launch walks every slot's group)
+    int32_t *h_len0 = ctx->h_tables + static_cast<size_t>(M.B + M.P) * W + 3 * static_cast<size_t>(M.P) * M.Lp +
+                      static_cast<size_t>(lo.n_chunks_max) * M.P + M.B;
+    std::fill(h_len0, h_len0 + 2 * static_cast<size_t>(M.B), 0);          // prompt lengths, then full prompt pages
+  }
   ctx->last_rows = 0;
 
   const int32_t *tok_hist = forced ? forced : out_tokens;
