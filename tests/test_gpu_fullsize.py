@@ -31,6 +31,8 @@ def test_full_size_rollout(name, seqs, steps):
     from paper_2602_02192_b200 import binding as B
     wl = synth.WORKLOADS[name]
     shape, P, G, Lp, T = wl.shape, wl.n_prompts, wl.G, wl.prompt_len, wl.new_tokens
+    import gc
+    gc.collect()
     torch.cuda.empty_cache()
     free, total = torch.cuda.mem_get_info()
     cfg = B.make_config(shape, P, G, Lp, T, 1, half_layers=wl.half_layers)     # as bench.py runs it

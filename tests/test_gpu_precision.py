@@ -36,6 +36,9 @@ def B():
 @pytest.fixture(scope="module")
 def w8b():
     wl = synth.WORKLOADS["8B"]
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()                 # blocks cached from the tests before count as used otherwise
     free, _ = torch.cuda.mem_get_info()
     if free < 60e9:
         pytest.skip("needs 60 GB of device memory")
