@@ -800,3 +800,42 @@ def test_prompt_queue_with_a_small_page_pool(B, tiny):
     check_sequences(dims, w_o, prompts, lens, G, 1.0, 78, tok5.cpu().numpy(), lp5.cpu().numpy(), range(3 * G), eos_id=eos,
                     top_p=0.9)
     eng.close()
+
+
+def test_snapshot_from_a_chain_buffer_installs_and_serves(B, tiny):
+    """What a forwarding chain delivers is one flat byte buffer in this GPU's memory (chain.pack on the
+    sender, chunked transfers, chain.unpack on the receiver: views, no copy).  Installed from those views,
+    in chunks that arrive while the previous version is serving, it must serve exactly the rollout that a
+    direct install of the same snapshot serves, and the oracle's."""
+    from paper_2602_02192_b200 import chain
+    wl, w_o, w_d = tiny
+    w1_t = synth.make_weights(wl.shape, 21)
+    w1_o = decoder.Weights(synth.weights_to_bits(w1_t))
+    flat_src = chain.pack(w1_t, wl.shape)                               # on the sending side (host memory here)
+    entries, total = chain.snapshot_layout(wl.shape)
+    assert flat_src.numel() == total and all(off % 256 == 0 for _, _, off, _ in entries)
+    P, G, Lp, T = 3, 4, 16, 10
+    prompts = synth.make_prompts(P, Lp, wl.shape.vocab, 8)
+    dp = torch.from_numpy(prompts).cuda()
+    eng = _engine(B, wl.shape, P, G, Lp, T)
+    eng.echo_load_policy(w_d, 1)
+    t0, _, v0 = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 5)            # version 1 serves ...
+    flat = torch.empty(total, dtype=torch.uint8, device="cuda")          # ... while the chunks land
+    chunk = 1 << 16
+    for a in range(0, total, chunk):
+        flat[a:a + chunk].copy_(flat_src[a:a + chunk], non_blocking=True)
+    torch.cuda.current_stream().synchronize()
+    eng.echo_load_policy(chain.unpack(flat, wl.shape), 2)
+    eng.echo_wait_policy()
+    t1, l1, v1 = eng.echo_rollout(dp, [Lp] * P, G, T, 1.0, 5)
+    eng.echo_sync()
+    assert np.all(v0 == 1) and np.all(v1 == 2)
+    check_sequences(dims_of(wl.shape), w1_o, prompts, [Lp] * P, G, 1.0, 5, t1.cpu().numpy(), l1.cpu().numpy(),
+                    range(P * G))
+    eng.close()
+    ref = _engine(B, wl.shape, P, G, Lp, T)
+    ref.echo_load_policy({k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in w1_t.items()}, 2)
+    t2, l2, _ = ref.echo_rollout(dp, [Lp] * P, G, T, 1.0, 5)
+    ref.echo_sync()
+    assert_same_rollout(t2.cpu().numpy(), l2.cpu().numpy(), t1.cpu().numpy(), l1.cpu().numpy())
+    ref.close()
