@@ -28,7 +28,7 @@ import torch
 
 # measured DRAM bytes per algorithmic byte of the prefix + suffix launch (ncu, see profiles/): with the
 # resident suffix kernel (decode steps below LONG_SUFFIX_STEP) and with one suffix CTA per item (above)
-ATTN_DRAM_PER_ALG_BYTE = {"resident": 251.98 / 244.5, "waves": 170.56 / 166.2}
+ATTN_DRAM_PER_ALG_BYTE = {"resident": 251.56 / 244.5, "waves": 170.61 / 166.2}
 LONG_SUFFIX_STEP = 1088
 METRIC = "rollout generated tokens/s"
 UNIT = "tokens/s"
