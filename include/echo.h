@@ -66,7 +66,9 @@ typedef struct echo_config {
                                  [0, vocab): a sequence that emits it is finished; its later positions
                                  hold eos_id with log-probability 0 (Section 5.1 generates up to a
                                  maximum length; responses end earlier at the end token).  Finished
-                                 sequences keep their place in the batch until the call returns. */
+                                 sequences leave the activation rows of the later steps; within one
+                                 echo_rollout call nothing takes their place (echo_rollout_queue
+                                 admits further prompts instead). */
   float   top_p;              /* nucleus sampling (Section 5.1 samples with top-p 0.95): tokens are ranked
                                  by probability (ties: lower id first), the shortest prefix whose mass
                                  reaches top_p is kept, and the recorded log-probability is renormalised
