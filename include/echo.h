@@ -93,6 +93,16 @@ typedef struct echo_config {
                                  have not ended, plus its max_G samples, stay within this number (the
                                  activation rows a decode step's projections run on).  0: no limit
                                  other than slots and pages. */
+  int32_t queue_optimistic;   /* 0: echo_rollout_queue gives a sequence the pages of its longest possible
+                                 continuation when it is admitted, so the pool can never run dry.
+                                 n in 1..8: pages are handed out as positions are reached (every 16 decode
+                                 steps, for the 16 to come), a group is admitted while the pool has room
+                                 for it plus n - 1 further windows of everything live (a page per sequence
+                                 and window; 3 is a sensible value), and when the pool cannot cover the next steps
+                                 the most recently admitted groups are evicted: their pages return, their
+                                 prompts go back to the head of the queue and they are generated again
+                                 from their first token later (the same tokens: noise streams are keyed
+                                 by sequence id and token index). */
 } echo_config;
 
 /* One snapshot: a pointer per tensor, bf16, row-major [out, in]; each pointer
@@ -123,6 +133,7 @@ typedef struct echo_stats {
   float   last_step_rows;     /* activation rows of the last decode step's projections: P*G, or fewer
                                  once sequences have ended (with an end token the live sequences are
                                  packed and the row count follows their number downwards) */
+  int64_t queue_evictions;    /* echo_rollout_queue with queue_optimistic: groups evicted and generated again */
 } echo_stats;
 
 /* Bytes of device memory echo_create needs for this configuration (weight

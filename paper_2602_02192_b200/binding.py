@@ -38,6 +38,7 @@ class EchoConfig(C.Structure):
         ("max_prompts", C.c_int32), ("max_G", C.c_int32), ("max_prompt_len", C.c_int32),
         ("max_new_tokens", C.c_int32), ("n_weight_buffers", C.c_int32), ("eos_id", C.c_int32),
         ("top_p", C.c_float), ("half_layers", C.c_int32), ("kv_pages", C.c_int32), ("queue_max_live", C.c_int32),
+        ("queue_optimistic", C.c_int32),
     ]
 
 
@@ -55,7 +56,7 @@ class EchoStats(C.Structure):
     _fields_ = [
         ("version_served", C.c_int64), ("tokens_generated", C.c_int64), ("kernels_launched", C.c_int64),
         ("decode_steps", C.c_int64), ("n_pages", C.c_int64), ("install_ms", C.c_float), ("prefill_ms", C.c_float),
-        ("decode_ms", C.c_float), ("last_step_rows", C.c_float),
+        ("decode_ms", C.c_float), ("last_step_rows", C.c_float), ("queue_evictions", C.c_int64),
     ]
 
 
@@ -171,13 +172,15 @@ def _check(rc: int, ctx=None):
 
 def make_config(shape, max_prompts: int, max_G: int, max_prompt_len: int, max_new_tokens: int,
                 n_weight_buffers: int = 2, page_size: int = 16, eos_id: int = -1,
-                top_p: float = 1.0, half_layers: int = 0, kv_pages: int = 0, queue_max_live: int = 0) -> EchoConfig:
+                top_p: float = 1.0, half_layers: int = 0, kv_pages: int = 0, queue_max_live: int = 0,
+                queue_optimistic: int = 0) -> EchoConfig:
     """shape: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab,
     rms_eps, rope_theta attributes."""
     return EchoConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                       shape.d_ff, shape.vocab, shape.rms_eps, shape.rope_theta, page_size,
                       max_prompts, max_G, max_prompt_len, max_new_tokens, n_weight_buffers, eos_id, top_p,
-                      min(int(half_layers), shape.n_layers), int(kv_pages), int(queue_max_live))
+                      min(int(half_layers), shape.n_layers), int(kv_pages), int(queue_max_live),
+                      int(queue_optimistic))
 
 
 def echo_arena_bytes(cfg: EchoConfig) -> int:

@@ -225,7 +225,8 @@ cudaError_t decode_prep_launch(int32_t *d_step, const int32_t *tok_hist, int T, 
                                int32_t *out_tok = nullptr, float *out_lp = nullptr);
 // Slots that change hands: for i < n, sequence slot admit_seq[i] finishes the outputs of the sequence
 // it held (end token / 0 from its current position on, if eos_id >= 0), takes sequence id admit_gid[i]
-// (-1: stays empty) with its token 0 due at the step counter's current value, and is live again.
+// (-1: stays empty; -2: stays empty and the old sequence's outputs are NOT completed, it will be generated
+// again) with its token 0 due at the step counter's current value, and is live again.
 cudaError_t admit_launch(int n, const int32_t *admit_seq, const int32_t *admit_gid, const int32_t *d_step,
                          int32_t *seq_gid, int32_t *seq_t0, int32_t *row_done, int32_t *out_tok, float *out_lp, int T,
                          int eos_id, cudaStream_t s);

@@ -429,7 +429,9 @@ __global__ void admit_kernel(const int32_t *admit_seq, const int32_t *admit_gid,
   const int b = admit_seq[blockIdx.x];
   const int j = *d_step;
   const int old = seq_gid[b];
-  if (old >= 0 && eos_id >= 0) {
+  const int gid_new = admit_gid[blockIdx.x];
+  // gid -2: the slot's group is evicted and will be generated again later; its outputs are left alone
+  if (old >= 0 && eos_id >= 0 && gid_new != -2) {
     // the steps so far wrote the sequence's positions up to j - t0 (its own tokens, then the end token
     // from the step that found it ended); the rest of its row follows here
     const int t_from = max(j - seq_t0[b] + 1, 1);
@@ -440,7 +442,7 @@ __global__ void admit_kernel(const int32_t *admit_seq, const int32_t *admit_gid,
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int gid = admit_gid[blockIdx.x];
+    const int gid = gid_new < 0 ? -1 : gid_new;
     seq_gid[b] = gid;
     seq_t0[b] = j;
     row_done[b] = gid < 0 ? 1 : 0;

@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <deque>
 #include <new>
 #include <string>
 #include <vector>
@@ -61,7 +62,7 @@ bool config_ok(const echo_config *c) {
   if (!(c->rms_eps >= 0.f) || !(c->rope_theta > 0.f)) return false;
   if (c->half_layers < 0 || c->half_layers > c->n_layers) return false;
   if (static_cast<long long>(c->max_prompts) * c->max_G > (1 << 20)) return false;
-  if (c->kv_pages < 0 || c->queue_max_live < 0) return false;
+  if (c->kv_pages < 0 || c->queue_max_live < 0 || c->queue_optimistic < 0 || c->queue_optimistic > 8) return false;
   return true;
 }
 
@@ -945,8 +946,9 @@ AdmitPlan plan_admit(echo_ctx *ctx, const int32_t *lens, int S, int G, int T, co
       int32_t *r = h_pt + static_cast<size_t>(b) * W;
       std::fill(r, r + W, -1);
       for (int qi = 0; qi < full; ++qi) r[qi] = sp.prefix[qi];
-      for (int qi = 0; qi < n_dec; ++qi) r[full + qi] = sp.sample[g][qi];
-      if (n_pre > full && n_dec > 0) {          // partial last prompt page: private copy per sample
+      const int n_own = std::min(n_dec, static_cast<int>(sp.sample[g].size()));   // pages handed out so far
+      for (int qi = 0; qi < n_own; ++qi) r[full + qi] = sp.sample[g][qi];
+      if (n_pre > full && n_own > 0) {          // partial last prompt page: private copy per sample
         h_csrc[ap.n_copies] = sp.prefix[full];
         h_cdst[ap.n_copies] = sp.sample[g][0];
         ++ap.n_copies;
@@ -1026,14 +1028,29 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
   const int32_t *tok_hist = forced ? forced : out_tokens;
   std::vector<int> slot_admit(S, -1);      // step after which the slot's current prompt was admitted; -1: empty
   std::vector<int> slot_live(S, 0);        // upper bound of the slot's sequences that have not ended
-  int next_prompt = 0, j = 0, n_admits = 0;
+  std::vector<int> slot_prompt(S, -1);     // the prompt a slot holds
+  std::deque<int> pending;                 // prompts not admitted yet (an evicted group's prompt returns to the head)
+  for (int p = 0; p < Pq; ++p) pending.push_back(p);
+  int j = 0, n_admits = 0;
+  int64_t n_evictions = 0;
+  const bool optimistic = ctx->cfg.queue_optimistic != 0;
   // the page pool (host side): free pages as a stack, the pages each slot holds, the peak in use
   const int Z = D.Z;
   std::vector<int> free_pages(M.n_pages);
   for (int i = 0; i < M.n_pages; ++i) free_pages[i] = M.n_pages - 1 - i;
   std::vector<SlotPages> slot_pages(S);
   int pages_peak = 0;
-  auto pages_of = [&](int len) { return ceil_div(len, Z) + G * (ceil_div(len + T - 1, Z) - len / Z); };
+  // own pages of a sample whose prompt has `len` tokens once it may write positions below len + n
+  // (n <= T - 1 tokens fed back); a partly filled last prompt page counts, it is copied per sample
+  auto own_pages = [&](int len, int n) { return ceil_div(len + std::min(n, T - 1), Z) - len / Z; };
+  // tokens a group admitted after step `adm` may have fed back by the window boundary that follows step `now`
+  auto fed_by_next_boundary = [&](int adm, int now) { return (now / kQueueWindow + 1) * kQueueWindow - adm; };
+  // pages a group takes when it is admitted after step `now`: everything it can ever need, or (optimistic)
+  // what it needs up to the next boundary
+  auto pages_of = [&](int len, int now) {
+    return ceil_div(len, Z) + G * own_pages(len, optimistic ? fed_by_next_boundary(now, now) : T - 1);
+  };
+  std::vector<std::vector<char>> released(S, std::vector<char>(G, 1));
   auto take_pages = [&](int n, std::vector<int> &dst) {
     dst.assign(free_pages.end() - n, free_pages.end());
     std::reverse(dst.begin(), dst.end());
@@ -1047,23 +1064,29 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
   // return to the pool; with the last sample the prompt's pages and the slot itself
   auto release_sample = [&](int slot, int g) {
     if (!slot_pages[slot].sample[g].empty()) give_pages(slot_pages[slot].sample[g]);
+    released[slot][g] = 1;
   };
   auto release_slot = [&](int slot) {
     for (int g = 0; g < G; ++g) release_sample(slot, g);
     give_pages(slot_pages[slot].prefix);
     slot_admit[slot] = -1;
     slot_live[slot] = 0;
+    slot_prompt[slot] = -1;
   };
 
   auto admit = [&](const std::vector<int> &slots) -> int {
     std::vector<int> which;
     for (size_t i = 0; i < slots.size(); ++i) {
-      const int p = next_prompt + static_cast<int>(i), len = prompt_lens[p];
+      const int p = pending.front(), len = prompt_lens[p];
+      pending.pop_front();
       which.push_back(p);
       SlotPages &sp = slot_pages[slots[i]];
       take_pages(ceil_div(len, Z), sp.prefix);
       sp.sample.assign(G, std::vector<int>());
-      for (int g = 0; g < G; ++g) take_pages(ceil_div(len + T - 1, Z) - len / Z, sp.sample[g]);
+      const int n_own = own_pages(len, optimistic ? fed_by_next_boundary(j, j) : T - 1);
+      for (int g = 0; g < G; ++g) take_pages(n_own, sp.sample[g]);
+      slot_prompt[slots[i]] = p;
+      std::fill(released[slots[i]].begin(), released[slots[i]].end(), 0);
     }
     pages_peak = std::max(pages_peak, M.n_pages - static_cast<int>(free_pages.size()));
     if (ctx->plan_in_flight) {             // the staging block may still be read by the previous upload
@@ -1116,7 +1139,6 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
       slot_admit[slots[i]] = j;
       slot_live[slots[i]] = G;
     }
-    next_prompt += static_cast<int>(slots.size());
     ++n_admits;
     return ECHO_OK;
   };
@@ -1180,16 +1202,92 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
       if (by_length(sl)) release_slot(sl);    // every sample has all its T tokens
     std::vector<int> slots;
     int need = 0, rows = live_bound();
-    for (int sl = 0; sl < S && next_prompt + static_cast<int>(slots.size()) < Pq; ++sl) {
+    for (int sl = 0; sl < S && slots.size() < pending.size(); ++sl) {
       if (slot_admit[sl] >= 0) continue;
-      const int p = next_prompt + static_cast<int>(slots.size());
-      const int pg = pages_of(prompt_lens[p]);
-      if (need + pg > static_cast<int>(free_pages.size()) || rows + G > max_live) break;
+      const int p = pending[slots.size()];
+      const int pg = pages_of(prompt_lens[p], j);
+      // optimistic: keep queue_optimistic - 1 windows' worth of growth of everything live in hand (a page
+      // per sequence and window), unless nothing is resident at all
+      const int margin = optimistic && rows > 0 ? (ctx->cfg.queue_optimistic - 1) * (rows + G) : 0;
+      if (need + pg + margin > static_cast<int>(free_pages.size()) || rows + G > max_live) break;
       need += pg;
       rows += G;
       slots.push_back(sl);
     }
     return slots.empty() ? ECHO_OK : admit(slots);
+  };
+  // Optimistic mode, at a window boundary: every live sample gets the pages for the positions it reaches
+  // by the next boundary.  If the pool cannot cover that, the most recently admitted groups are evicted
+  // (their prompts return to the head of the queue; the pool holds one group at full length, so the
+  // oldest group always gets through).
+  auto extend = [&]() -> int {
+    auto wanted = [&](int sl) {
+      return own_pages(prompt_lens[slot_prompt[sl]], fed_by_next_boundary(slot_admit[sl], j));
+    };
+    auto missing = [&](int sl) {
+      const int want = wanted(sl);
+      int m = 0;
+      for (int g = 0; g < G; ++g)
+        if (!released[sl][g]) m += std::max(0, want - static_cast<int>(slot_pages[sl].sample[g].size()));
+      return m;
+    };
+    int need = 0;
+    for (int sl = 0; sl < S; ++sl)
+      if (slot_admit[sl] >= 0) need += missing(sl);
+    std::vector<int> evicted;
+    while (need > static_cast<int>(free_pages.size())) {
+      int victim = -1;
+      for (int sl = 0; sl < S; ++sl)
+        if (slot_admit[sl] >= 0 && (victim < 0 || slot_admit[sl] >= slot_admit[victim])) victim = sl;
+      if (victim < 0) return ECHO_ERR_INVALID;          // cannot happen: see above
+      need -= missing(victim);
+      pending.push_front(slot_prompt[victim]);
+      release_slot(victim);
+      evicted.push_back(victim);
+      ++n_evictions;
+    }
+    if (need == 0 && evicted.empty()) return ECHO_OK;
+    if (ctx->plan_in_flight) {
+      CK(cudaEventSynchronize(ctx->plan_done));
+      ctx->plan_in_flight = false;
+    }
+    int32_t *h_pt = ctx->h_tables;
+    for (int sl = 0; sl < S; ++sl) {
+      if (slot_admit[sl] < 0) continue;
+      const int want = wanted(sl), full = prompt_lens[slot_prompt[sl]] / Z;
+      for (int g = 0; g < G; ++g) {
+        if (released[sl][g]) continue;
+        std::vector<int> &own = slot_pages[sl].sample[g];
+        int32_t *r = h_pt + static_cast<size_t>(sl * G + g) * W;
+        while (static_cast<int>(own.size()) < want) {
+          own.push_back(free_pages.back());
+          free_pages.pop_back();
+          r[full + static_cast<int>(own.size()) - 1] = own.back();
+        }
+      }
+    }
+    pages_peak = std::max(pages_peak, M.n_pages - static_cast<int>(free_pages.size()));
+    CK(cudaMemcpyAsync(ctx->arena + lo.page_table, h_pt, static_cast<size_t>(B + S) * W * 4, cudaMemcpyHostToDevice,
+                       ctx->stream));
+    const int n_ev = static_cast<int>(evicted.size()) * G;
+    if (n_ev) {
+      int32_t *h_admit_seq = ctx->h_queue, *h_admit_gid = ctx->h_queue + M.B;
+      for (size_t i = 0; i < evicted.size(); ++i)
+        for (int g = 0; g < G; ++g) {
+          h_admit_seq[i * G + g] = evicted[i] * G + g;
+          h_admit_gid[i * G + g] = -2;
+        }
+      CK(cudaMemcpyAsync(ctx->arena + lo.admit_seq, h_admit_seq, static_cast<size_t>(n_ev) * 4, cudaMemcpyHostToDevice,
+                         ctx->stream));
+      CK(cudaMemcpyAsync(ctx->arena + lo.admit_gid, h_admit_gid, static_cast<size_t>(n_ev) * 4, cudaMemcpyHostToDevice,
+                         ctx->stream));
+    }
+    CK(cudaEventRecord(ctx->plan_done, ctx->stream));
+    ctx->plan_in_flight = true;
+    if (n_ev)
+      LAUNCH(admit_launch(n_ev, ctx->ptr<int32_t>(lo.admit_seq), ctx->ptr<int32_t>(lo.admit_gid), d_step, seq_gid, seq_t0,
+                          row_done, out_tokens, out_logprobs, T, eos, ctx->stream));
+    return ECHO_OK;
   };
   auto choose_rows = [&]() {                  // the smallest captured row count that holds every live sequence
     const int bound = live_bound();
@@ -1204,7 +1302,7 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
       first = false;
       cudaEventRecord(ctx->ev_first, ctx->stream);
     }
-    bool all_over = next_prompt >= Pq;
+    bool all_over = pending.empty();
     for (int sl = 0; sl < S && all_over; ++sl) all_over = slot_admit[sl] < 0;
     if (all_over) break;
     choose_rows();
@@ -1226,7 +1324,11 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
       ctx->long_suffix = false;
     }
     if (rc_steps != ECHO_OK) break;
-    if (j % kQueueWindow || eos < 0) continue;          // without an end token sequences end by length only
+    if (j % kQueueWindow) continue;
+    if (eos < 0) {                                       // without an end token sequences end by length only
+      if (optimistic && (rc_steps = extend()) != ECHO_OK) break;
+      continue;
+    }
     // ---- window boundary: read the ended flags as of this step.  The host waits for the GPU here (the
     // steps it has enqueued so far), which costs one launch latency per window; what it learns decides
     // the refill and the row count of the next window.
@@ -1247,6 +1349,9 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
       slot_live[sl] = std::min(slot_live[sl], live);
       if (slot_live[sl] == 0) release_slot(sl);
     }
+    for (int sl = 0; sl < S; ++sl)
+      if (by_length(sl)) release_slot(sl);
+    if (optimistic && (rc_steps = extend()) != ECHO_OK) break;
   }
   release_graphs();
   if (rc_steps != ECHO_OK) return rc_steps;
@@ -1281,6 +1386,7 @@ int rollout_queue_impl(echo_ctx *ctx, const int32_t *prompts, const int32_t *pro
   ctx->stats.kernels_launched = ctx->launches - launches0;
   ctx->stats.decode_steps = j;
   ctx->stats.n_pages = pages_peak;
+  ctx->stats.queue_evictions = n_evictions;
   return ECHO_OK;
 }
 

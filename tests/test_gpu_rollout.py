@@ -839,3 +839,55 @@ def test_snapshot_from_a_chain_buffer_installs_and_serves(B, tiny):
     ref.echo_sync()
     assert_same_rollout(t2.cpu().numpy(), l2.cpu().numpy(), t1.cpu().numpy(), l1.cpu().numpy())
     ref.close()
+
+
+def test_prompt_queue_optimistic_pages_and_eviction(B, tiny):
+    """queue_optimistic: pages are handed out window by window, groups are admitted without room for their
+    longest continuation, and when the pool cannot cover the next window the newest groups are evicted and
+    generated again later.  An evicted group's second run gives the same tokens (noise keyed by sequence id
+    and token index), so every sequence still matches the oracle's rollout of that sequence alone; the run
+    needs fewer decode steps than the one that reserves every continuation, in the same pool."""
+    wl, w_o, w_d = tiny
+    Pq, G, Lp, T = 14, 8, 40, 56
+    lens_l = [40, 7, 33, 16, 40, 1, 25, 17, 32, 9, 21, 40, 3, 28]
+    prompts, lens = synth.make_ragged_prompts(lens_l, wl.shape.vocab, 910, pad_to=Lp)
+    dp = torch.from_numpy(prompts).cuda()
+    dims = dims_of(wl.shape)
+    eos = 7
+    rng = np.random.default_rng(6)
+    given = rng.integers(8, wl.shape.vocab, size=(Pq, G, T)).astype(np.int32)
+    ends = rng.integers(0, T + 10, size=(Pq, G))
+    for p in range(Pq):
+        for g in range(G):
+            if ends[p, g] < T:
+                given[p, g, ends[p, g]] = eos
+    forced = torch.from_numpy(given).cuda()
+    stats = {}
+    for mode in (0, 1):
+        eng = B.Engine(B.make_config(wl.shape, Pq, G, Lp, T, eos_id=eos, kv_pages=60, queue_optimistic=mode))
+        eng.echo_load_policy(w_d, 3)
+        tok_f, lp_f, _ = eng.echo_rollout_queue(dp, lens, G, T, 1.0, 77, forced=forced)
+        eng.echo_sync()
+        stats[mode] = eng.echo_get_stats()
+        tok_f, lp_f = tok_f.cpu().numpy(), lp_f.cpu().numpy()
+        assert 0 < stats[mode]["n_pages"] <= 60
+        for s in range(Pq * G):
+            p, g = divmod(s, G)
+            e = ends[p, g]
+            if e < T:
+                assert np.all(lp_f[p, g, e + 1:] == 0.0) and np.all(tok_f[p, g, e + 1:] == eos)
+            sc = decoder.score_forced(dims, w_o, prompts[p][: int(lens[p])], given[p, g], 1.0, 77, s, eos_id=eos)
+            assert np.max(np.abs(lp_f[p, g] - sc.logprob_given)) <= LOGPROB_TOL
+            live = np.arange(T) <= min(e, T - 1)
+            diff = (tok_f[p, g] != sc.own_token) & live
+            assert np.all(sc.margin[diff] < 1e-2) and np.all(tok_f[p, g][diff] == sc.runner_up[diff])
+        if mode == 1:
+            # free-running too (no sequence ends early: the pool is under the most pressure)
+            tok, lp, _ = eng.echo_rollout_queue(dp, lens, G, 24, 1.0, 78)
+            eng.echo_sync()
+            assert eng.echo_get_stats()["queue_evictions"] > 0
+            check_sequences(dims, w_o, prompts, lens, G, 1.0, 78, tok.cpu().numpy(), lp.cpu().numpy(),
+                            range(0, Pq * G, 3), eos_id=eos)
+        eng.close()
+    assert stats[0]["queue_evictions"] == 0 and stats[1]["queue_evictions"] > 0
+    assert stats[1]["decode_steps"] < stats[0]["decode_steps"]
