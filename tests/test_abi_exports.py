@@ -29,6 +29,36 @@ def test_binding_lists_the_same_names():
     assert sorted(binding.EXPORTED) == _declared()
 
 
+def test_struct_layouts_match_the_header(tmp_path):
+    """The ctypes mirrors of echo_config and echo_stats against the C compiler's view of the header:
+    size and the offset of every field (a field added on one side only would shift everything after it)."""
+    import subprocess
+    from paper_2602_02192_b200 import binding
+    fields = {"echo_config": binding.EchoConfig, "echo_stats": binding.EchoStats}
+    lines = []
+    for name, cls in fields.items():
+        lines.append(f'printf("{name} %zu\\n", sizeof({name}));')
+        for f, _ in cls._fields_:
+            lines.append(f'printf("{name}.{f} %zu\\n", offsetof({name}, {f}));')
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stddef.h>\n#include <stdio.h>\n#include "echo.h"\nint main(void) {\n' + "\n".join(lines) +
+                   "\nreturn 0; }\n")
+    exe = tmp_path / "layout"
+    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
+    out = dict(l.split() for l in subprocess.check_output([str(exe)], text=True).splitlines())
+    for name, cls in fields.items():
+        assert int(out[name]) == ctypes.sizeof(cls), name
+        for f, _ in cls._fields_:
+            assert int(out[f"{name}.{f}"]) == getattr(cls, f).offset, (name, f)
+    # and the header declares no field the mirror lacks
+    text = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "echo.h")).read(), flags=re.S)
+    for name, cls in fields.items():
+        body = re.search(r"typedef struct %s \{(.*?)\} %s;" % (name, name), text, flags=re.S).group(1)
+        declared = [x.strip() for decl in body.split(";") if decl.strip()
+                    for x in re.sub(r"^\s*\w+\s+", "", decl.strip()).split(",")]
+        assert declared == [f for f, _ in cls._fields_], name
+
+
 def test_config_validation_needs_no_gpu():
     from paper_2602_02192_b200 import binding, synth
     shape = synth.SHAPES["tiny"]
